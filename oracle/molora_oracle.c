@@ -1,0 +1,178 @@
+/*
+ * CPU oracle for per-token routed LoRA.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, obviously-correct restatement of what the routed-LoRA path computes, written from
+ * the paper's definitions.  Every floating-point sum is carried in fp64, in index order, one token
+ * at a time in the ORIGINAL token order; the grouping (histogram / offsets / permutation) is never
+ * used to compute the LoRA result, so comparing the CUDA path's output with oracle_apply() checks
+ * routing, grouping and the grouped shrink/expand end to end.
+ *
+ * Nothing here is shared with the CUDA path (no headers, helpers, tables or constants), and only the
+ * tests, the smoke check and the benchmark's cpu-baseline leg may call it.
+ *
+ * Inputs are float32 arrays; for bf16 workloads they hold bf16-representable values, so the
+ * conversion to double below is exact for both storage types.
+ *
+ * The only parallelism is an OpenMP "for" over tokens (tokens are independent in Eq. 2); each
+ * token's arithmetic is serial and in index order, so results do not depend on the thread count.
+ *
+ * Pinned by tests/test_oracle_pins.py (constant routing == dense LoRA by a library matmul, selector
+ * closed forms, the grouping example of Figure 2, upper_bound for vocabulary routing, exhaustive
+ * routings on integer data, permutation equivariance, the N vs K*N work count of Theorem 3.6).
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Definition 3.1 / Eq. 3 (vocabulary routing), read 0-based: with breaks b_0 <= b_1 <= ... <= b_M,
+ * R(v) = m  <=>  b_m <= v < b_{m+1},  m in [0, M).  An id that lies in no range is unrouted (-1).
+ * Linear search over the M ranges, exactly as the definition reads. */
+int oracle_route_vocab(const int32_t *ids, int64_t N, const int32_t *breaks, int32_t M, int32_t *r)
+{
+    if (N < 0 || M <= 0) return 1;
+    for (int64_t i = 0; i < N; ++i) {
+        int32_t found = -1;
+        for (int32_t m = 0; m < M; ++m) {
+            if (breaks[m] <= ids[i] && ids[i] < breaks[m + 1]) { found = m; break; }
+        }
+        r[i] = found;
+    }
+    return 0;
+}
+
+/* Linear gate with top-1 selection (Eq. 8 with k = 1; the gate of Theorem 3.4 / Table 10 is
+ * softmax(W x + b)).  Softmax is monotone, so the winner is the argmax of the raw logits
+ * z[i][c] = sum_k x[i][k] * G[k][c] (+ bias[c]); with a single kept logit the softmax weight is 1.
+ * Ties go to the lowest index.  margin[i] = (largest logit) - (second largest logit); for C == 1 it
+ * is +infinity-like (1e300). */
+int oracle_route_gate(const float *x, int64_t N, int32_t d, int64_t ldx, const float *G, const float *bias,
+                      int32_t C, int32_t *r, double *z_out, double *margin_out)
+{
+    if (N < 0 || d <= 0 || C <= 0 || ldx < d) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < N; ++i) {
+        double best = 0.0, second = 0.0;
+        int32_t arg = -1;
+        for (int32_t c = 0; c < C; ++c) {
+            double z = 0.0;
+            for (int32_t k = 0; k < d; ++k) z += (double)x[i * ldx + k] * (double)G[(int64_t)k * C + c];
+            if (bias) z += (double)bias[c];
+            if (z_out) z_out[i * C + c] = z;
+            if (arg < 0) { best = z; arg = c; second = -1e300; }
+            else if (z > best) { second = best; best = z; arg = c; }
+            else if (z > second) { second = z; }
+        }
+        r[i] = arg;
+        if (margin_out) margin_out[i] = (C > 1) ? best - second : 1e300;
+    }
+    return 0;
+}
+
+/* Section 3.3 (unified dispatch), steps 1-3, with a deterministic order inside each group:
+ *   counts[c]  = |{ i : r[i] = c }|                        (the histogram h)
+ *   offsets[0] = 0, offsets[c+1] = offsets[c] + counts[c]   (position allocation)
+ *   perm[offsets[c] + k] = the k-th token, in ascending token index, routed to c
+ * Tokens with r[i] outside [0, C) belong to no group.  O(N*C) double loop: trivially stable. */
+int oracle_group(const int32_t *r, int64_t N, int32_t C, int32_t *counts, int32_t *offsets, int32_t *perm)
+{
+    if (N < 0 || C <= 0) return 1;
+    int64_t p = 0;
+    offsets[0] = 0;
+    for (int32_t c = 0; c < C; ++c) {
+        int32_t n = 0;
+        for (int64_t i = 0; i < N; ++i) {
+            if (r[i] == c) { perm[p++] = (int32_t)i; ++n; }
+        }
+        counts[c] = n;
+        offsets[c + 1] = offsets[c] + n;
+    }
+    return 0;
+}
+
+/* One token through one adapter: h = y + scale * (x A_c) B_c, A_c [d_in, rank], B_c [rank, d_out]. */
+static void lora_row(const float *x, const float *y, const float *Ac, const float *Bc, int32_t d_in, int32_t d_out,
+                     int32_t rank, double scale, double *t, double *h)
+{
+    for (int32_t k = 0; k < rank; ++k) {
+        double s = 0.0;
+        for (int32_t j = 0; j < d_in; ++j) s += (double)x[j] * (double)Ac[(int64_t)j * rank + k];
+        t[k] = s;
+    }
+    for (int32_t o = 0; o < d_out; ++o) {
+        double s = 0.0;
+        for (int32_t k = 0; k < rank; ++k) s += t[k] * (double)Bc[(int64_t)k * d_out + o];
+        h[o] = (double)y[o] + scale * s;
+    }
+}
+
+/* Eq. 2 (per-token routing): h_i = y_i + scale * x_i A_{r(i)} B_{r(i)} with y_i = x_i W supplied by the
+ * caller; tokens with r(i) outside [0, C) keep h_i = y_i.  Weight layout follows Table 10:
+ * A is (C, d_in, rank), B is (C, rank, d_out), both row-major.  *products counts token-adapter
+ * products (Theorem 3.6: N for per-token routing, counting routed tokens). */
+int oracle_apply(const float *x, int64_t ldx, const float *y, int64_t ldy, const float *A, const float *B,
+                 const int32_t *r, int64_t N, int32_t d_in, int32_t d_out, int32_t rank, int32_t C, double scale,
+                 double *h, int64_t *products)
+{
+    if (N < 0 || d_in <= 0 || d_out <= 0 || rank <= 0 || C <= 0 || ldx < d_in || ldy < d_out) return 1;
+    int64_t count = 0;
+#pragma omp parallel for schedule(static) reduction(+ : count)
+    for (int64_t i = 0; i < N; ++i) {
+        int32_t c = r[i];
+        double *hi = h + i * (int64_t)d_out;
+        if (c < 0 || c >= C) {
+            for (int32_t o = 0; o < d_out; ++o) hi[o] = (double)y[i * ldy + o];
+            continue;
+        }
+        double *t = (double *)malloc(sizeof(double) * (size_t)rank);
+        lora_row(x + i * ldx, y + i * ldy, A + (int64_t)c * d_in * rank, B + (int64_t)c * rank * d_out, d_in, d_out,
+                 rank, scale, t, hi);
+        free(t);
+        ++count;
+    }
+    if (products) *products = count;
+    return 0;
+}
+
+/* Per-sequence routing served as K passes (Eq. 1 applied once per adapter, Theorem 3.6): pass k runs
+ * the dense single-adapter LoRA of adapter k over ALL N tokens, then only rows with r[i] == k are kept.
+ * Work is K*N token-adapter products.  The result must equal oracle_apply() bit for bit. */
+int oracle_apply_perseq_kpass(const float *x, int64_t ldx, const float *y, int64_t ldy, const float *A,
+                              const float *B, const int32_t *r, int64_t N, int32_t d_in, int32_t d_out,
+                              int32_t rank, int32_t K, double scale, double *h, int64_t *products)
+{
+    if (N < 0 || d_in <= 0 || d_out <= 0 || rank <= 0 || K <= 0 || ldx < d_in || ldy < d_out) return 1;
+    int64_t count = 0;
+    double *pass = (double *)malloc(sizeof(double) * (size_t)(N > 0 ? N : 1) * (size_t)d_out);
+    if (!pass) return 2;
+    for (int64_t i = 0; i < N; ++i)
+        for (int32_t o = 0; o < d_out; ++o) h[i * (int64_t)d_out + o] = (double)y[i * ldy + o];
+    for (int32_t k = 0; k < K; ++k) {
+        int64_t pass_count = 0;
+#pragma omp parallel for schedule(static) reduction(+ : pass_count)
+        for (int64_t i = 0; i < N; ++i) {
+            double *t = (double *)malloc(sizeof(double) * (size_t)rank);
+            lora_row(x + i * ldx, y + i * ldy, A + (int64_t)k * d_in * rank, B + (int64_t)k * rank * d_out, d_in,
+                     d_out, rank, scale, t, pass + i * (int64_t)d_out);
+            free(t);
+            ++pass_count;
+        }
+        count += pass_count;
+        for (int64_t i = 0; i < N; ++i)
+            if (r[i] == k) memcpy(h + i * (int64_t)d_out, pass + i * (int64_t)d_out, sizeof(double) * (size_t)d_out);
+    }
+    free(pass);
+    if (products) *products = count;
+    return 0;
+}
