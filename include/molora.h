@@ -1,0 +1,149 @@
+/*
+ * molora.h -- C ABI of the B200 (sm_100a) routed-LoRA library.
+ *
+ * The library computes per-token routed LoRA (Eq. 2 of the MoLoRA paper)
+ *
+ *        h_i = x_i W + x_i A_{r(i)} B_{r(i)},      r : [N] -> [C]
+ *
+ * on a caller-provided base projection y = x W, in three steps that mirror the paper's dispatch
+ * pipeline (Section 3.3, Figure 2 right, Algorithms 1 and 2):
+ *
+ *   molora_route_*   the router r (vocabulary ranges, Definition 3.1; or a linear gate with top-1
+ *                    argmax, Eq. 8 with k = 1 and the gate of Theorem 3.4 / Table 10)
+ *   molora_group     histogram of r, exclusive scan into segment offsets, stable permutation
+ *   molora_apply     grouped shrink t_i = x_i A_c and expand h_i = y_i + scale * t_i B_c, in place in y
+ *
+ * Conventions (all entry points unless stated otherwise)
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, valid on the current device, and
+ *     must stay valid until the work enqueued on `stream` has completed.  The library allocates no
+ *     memory, keeps no global state, never synchronises the host and never reads device memory
+ *     from the host: each call only validates its scalar arguments and enqueues kernels on `stream`,
+ *     so calls may be captured into a CUDA graph.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Matrices are row-major; `ld*` is the row pitch in ELEMENTS.
+ *   - Return value: MOLORA_OK, or an error code detected on the host BEFORE anything is enqueued
+ *     (the call is then a no-op).  Conditions that can only be seen on the device (ids outside every
+ *     vocabulary range, routing values outside [-1, C)) never fault: the offending token is treated as
+ *     unrouted and the event is recorded in the optional device status word (see MOLORA_DEV_*).
+ *   - Routing value -1 means "unrouted": the token belongs to no segment and keeps h_i = y_i.
+ *
+ * Supported set: N in [0, 2^31 - 1), 1 <= C <= 256 (Example 3.3's 64 x 4 composite targets),
+ * rank in {8, 16, 32, 64}, element type fp32 or bf16 (x, y, A, B share it; accumulation is fp32),
+ * d_in / d_out / ld multiples of 8 elements and all tensor base pointers 16-byte aligned.
+ */
+#ifndef MOLORA_H_
+#define MOLORA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MOLORA_OK = 0,
+    MOLORA_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned pointer, pitch too small      */
+    MOLORA_ERR_UNSUPPORTED = 2, /* rank / dtype / C / dimension outside the supported set                */
+    MOLORA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than molora_*_workspace_bytes reports     */
+    MOLORA_ERR_CUDA = 4         /* the CUDA runtime refused a launch or a copy (cudaGetLastError for why)  */
+} molora_status_t;
+
+typedef enum { MOLORA_F32 = 0, MOLORA_BF16 = 1 } molora_dtype_t;
+
+/* Bits OR-ed by kernels into the optional device status word (uint32, zeroed by the caller). */
+#define MOLORA_DEV_ID_OUT_OF_RANGE 0x1u /* some token id lies in no vocabulary range: routed to -1          */
+#define MOLORA_DEV_BAD_ROUTE 0x2u       /* some routing value lies outside [-1, C): treated as unrouted       */
+#define MOLORA_DEV_TIMEOUT 0x4u         /* a bounded device-side wait gave up (results of that call invalid)   */
+
+#define MOLORA_MAX_ADAPTERS 256
+#define MOLORA_MAX_PROJECTIONS 8
+
+/* Library version string, e.g. "molora-b200 0.1 (sm_100a)".  Static storage. */
+const char *molora_version(void);
+
+/* Human-readable name of a status code.  Static storage. */
+const char *molora_status_string(molora_status_t status);
+
+/* ---------------------------------------------------------------------------------------------
+ * Router 1: vocabulary routing (Definition 3.1 / Eq. 3; Algorithm 1 "FindModality"), 0-based:
+ *     r_out[i] = m   with   breaks[m] <= ids[i] < breaks[m+1],  m in [0, M);   -1 if no range holds ids[i].
+ * ids      device int32[N]   token vocabulary indices
+ * breaks   device int32[M+1] non-decreasing range boundaries b_0..b_M (an empty range is legal), 1 <= M <= 256
+ * r_out    device int32[N]   routing decision per token
+ * dev_status  device uint32 or NULL; MOLORA_DEV_ID_OUT_OF_RANGE is OR-ed in if any id is unrouted
+ * Integer work, exact.  N == 0 is a no-op. */
+molora_status_t molora_route_vocab(const int32_t *ids, int64_t N, const int32_t *breaks, int32_t M, int32_t *r_out,
+                                   uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Router 2: learned linear gate with top-1 selection (Eq. 8 with k = 1; gate form softmax(W x + b) of
+ * Theorem 3.4 / Table 10).  Softmax is monotone and the weight of a single kept logit is 1, so
+ *     z[i][c] = sum_k x[i][k] * G[k][c] (+ bias[c]),    r_out[i] = argmax_c z[i][c]  (lowest c on ties).
+ * x        device [N, d] of type xdt, row pitch ldx >= d elements; d a multiple of 8; never written
+ * G        device fp32 [d, C] row-major (gate weights);  bias  device fp32 [C] or NULL;  1 <= C <= 64
+ * r_out    device int32[N]
+ * logits_out  device fp32 [N, C] or NULL (the logits as the kernel accumulated them, fp32)
+ * Products are exact in fp32 for bf16 x; accumulation is fp32 in a fixed, token-independent order. */
+molora_status_t molora_route_gate(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float *G,
+                                  const float *bias, int32_t C, int32_t *r_out, float *logits_out, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Grouping (Section 3.3 steps 1-3; Algorithm 2; Table 10 "histogram"):
+ *     counts[c]    = |{ i : r[i] = c }|
+ *     offsets[0]   = 0,  offsets[c+1] = offsets[c] + counts[c]
+ *     perm[offsets[c] + k] = index of the k-th token (ascending i) with r[i] = c
+ * The paper allocates positions with atomicAdd (order inside a group unspecified) and emits pointer
+ * pairs xs/ys; this library emits the unique STABLE order as 32-bit token indices, from which
+ * xs[c][k] = x + perm[offsets[c]+k]*ldx.  Results are exact and deterministic.
+ * r        device int32[N]; values outside [0, C) are unrouted (values < -1 or >= C also set
+ *          MOLORA_DEV_BAD_ROUTE in dev_status)
+ * counts   device int32[C];  offsets  device int32[C+1];  perm  device int32[N] (first offsets[C] entries valid)
+ * ws, ws_bytes  device scratch of at least molora_group_workspace_bytes(N, C) bytes, 16-byte aligned
+ *               (may be NULL when that function returns 0).  Contents are undefined afterwards.
+ * dev_status    device uint32 or NULL.
+ * offsets/perm of one call may feed any number of molora_apply calls (one routing per layer). */
+size_t molora_group_workspace_bytes(int64_t N, int32_t C);
+molora_status_t molora_group(const int32_t *r, int64_t N, int32_t C, int32_t *counts, int32_t *offsets, int32_t *perm,
+                             void *ws, size_t ws_bytes, uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Grouped LoRA application (Eq. 2; Figure 2 "Grouped GEMM" + "Scatter to original positions";
+ * weight shapes of Table 10): for every segment c and every token i = perm[j], offsets[c] <= j < offsets[c+1],
+ *     t_i = x_i A_c            (shrink, d_in -> rank, fp32, kept on chip)
+ *     y_i <- y_i + scale * t_i B_c   (expand, rank -> d_out; one rounding to the storage type)
+ * Rows of y that belong to no segment are not touched.
+ * x   device [N, d_in]  of type dt, pitch ldx;  never written
+ * y   device [N, d_out] of type dt, pitch ldy;  in: base projection x W, out: h
+ * A   device [C, d_in, rank] of type dt, dense;  B  device [C, rank, d_out] of type dt, dense
+ * offsets, perm   device outputs of molora_group for the same N, C (read on the device only)
+ * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes (NULL if that is 0)
+ * The kernel variant (CUDA-core path for small segments, tensor-core tiles for large ones) is chosen on
+ * the device from the segment sizes; the paper picks its tile shape from the histogram too (Eq. 12-13). */
+size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t d_out, int32_t rank);
+molora_status_t molora_apply(const void *x, int64_t ldx, void *y, int64_t ldy, molora_dtype_t dt, int64_t N,
+                             int32_t d_in, int32_t d_out, int32_t rank, const void *A, const void *B, int32_t C,
+                             const int32_t *offsets, const int32_t *perm, float scale, void *ws, size_t ws_bytes,
+                             void *stream);
+
+/* Same operation for P projections that share N, C, offsets and perm (the projections of one layer),
+ * enqueued as one launch.  `projs` is a HOST array of P descriptors (1 <= P <= MOLORA_MAX_PROJECTIONS),
+ * copied at enqueue time; the pointers inside are device pointers with the meaning given above. */
+typedef struct {
+    const void *x;
+    int64_t ldx;
+    void *y;
+    int64_t ldy;
+    const void *A;
+    const void *B;
+    int32_t d_in, d_out, rank;
+    float scale;
+} molora_proj_desc_t;
+molora_status_t molora_apply_batched(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N,
+                                     int32_t C, const int32_t *offsets, const int32_t *perm, void *ws, size_t ws_bytes,
+                                     void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOLORA_H_ */

@@ -1,0 +1,14 @@
+"""B200 (sm_100a) routed-LoRA library: Python binding over the C ABI declared in include/molora.h.
+
+The binding only marshals arguments (device pointers, sizes, the current CUDA stream); every step of
+the path -- routing, grouping, shrink/expand -- runs in the library's own kernels.  There is no CPU or
+PyTorch fallback: if the shared library is missing or a call is refused, an exception is raised.
+"""
+from .binding import (  # noqa: F401
+    MoloraError, lib_path, load_library, exported_symbols,
+    molora_version, molora_status_string,
+    molora_route_vocab, molora_route_gate,
+    molora_group_workspace_bytes, molora_group,
+    molora_apply_workspace_bytes, molora_apply, molora_apply_batched,
+    ProjDesc, F32, BF16,
+)

@@ -1,0 +1,257 @@
+"""ctypes binding of the C ABI in include/molora.h.  Argument marshalling only.
+
+Each ``molora_*`` function mirrors the C entry point of the same name: torch tensors stand for the
+device pointers (``data_ptr()``), sizes and pitches are read from their shapes and strides, and the
+stream is ``torch.cuda.current_stream()`` unless one is given.  Output tensors are allocated with
+torch when the caller does not pass them (device memory is PyTorch's job; the library allocates
+nothing).  A non-zero status raises :class:`MoloraError`; a missing shared library raises too --
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import re
+from dataclasses import dataclass
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+from .build import LIB_PATH, ROOT
+
+F32, BF16 = 0, 1
+MAX_ADAPTERS = 256
+MAX_PROJECTIONS = 8
+
+_lib = None
+
+
+class MoloraError(RuntimeError):
+    def __init__(self, fn: str, status: int, text: str):
+        super().__init__(f"{fn} failed: status {status} ({text})")
+        self.status = status
+
+
+class _ProjDescC(ctypes.Structure):
+    _fields_ = [("x", ctypes.c_void_p), ("ldx", ctypes.c_int64), ("y", ctypes.c_void_p), ("ldy", ctypes.c_int64),
+                ("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32),
+                ("rank", ctypes.c_int32), ("scale", ctypes.c_float)]
+
+
+def lib_path() -> str:
+    return LIB_PATH
+
+
+def exported_symbols() -> List[str]:
+    """Names of the functions include/molora.h declares (parsed from the header)."""
+    with open(os.path.join(ROOT, "include", "molora.h")) as f:
+        text = f.read()
+    return sorted(set(re.findall(r"\b(molora_[a-z_]+)\s*\(", text)))
+
+
+def load_library():
+    """dlopen the in-tree libmolora.so (built by ``paper_2603_15965_b200.build``) and declare signatures."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2603_15965_b200.build` "
+                          "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
+    lib.molora_version.restype = ctypes.c_char_p
+    lib.molora_version.argtypes = []
+    lib.molora_status_string.restype = ctypes.c_char_p
+    lib.molora_status_string.argtypes = [ctypes.c_int]
+    lib.molora_route_vocab.argtypes = [vp, i64, vp, i32, vp, vp, vp]
+    lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp]
+    lib.molora_group_workspace_bytes.restype = sz
+    lib.molora_group_workspace_bytes.argtypes = [i64, i32]
+    lib.molora_group.argtypes = [vp, i64, i32, vp, vp, vp, vp, sz, vp, vp]
+    lib.molora_apply_workspace_bytes.restype = sz
+    lib.molora_apply_workspace_bytes.argtypes = [i64, i32, i32, i32, i32]
+    lib.molora_apply.argtypes = [vp, i64, vp, i64, ctypes.c_int, i64, i32, i32, i32, vp, vp, i32, vp, vp, f32, vp, sz,
+                                 vp]
+    lib.molora_apply_batched.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64, i32, vp, vp, vp, sz, vp]
+    for name in ("molora_route_vocab", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched"):
+        getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+# ----------------------------------------------------------------------------- helpers
+def _check(fn: str, status: int) -> None:
+    if status != 0:
+        raise MoloraError(fn, status, load_library().molora_status_string(status).decode())
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported element type {t.dtype}: fp32 or bf16 only")
+
+
+def _matrix(t: torch.Tensor, name: str) -> Tuple[int, int, int]:
+    """(rows, cols, pitch in elements) of a 2-D row-major device tensor."""
+    if not t.is_cuda or t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError(f"{name}: expected a 2-D row-major CUDA tensor")
+    return t.shape[0], t.shape[1], (t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1]))
+
+
+def _i32_dev(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != torch.int32 or not t.is_contiguous():
+        raise ValueError(f"{name}: expected a contiguous int32 CUDA tensor")
+    return t
+
+
+# ----------------------------------------------------------------------------- entry points
+def molora_version() -> str:
+    return load_library().molora_version().decode()
+
+
+def molora_status_string(status: int) -> str:
+    return load_library().molora_status_string(int(status)).decode()
+
+
+def molora_route_vocab(ids: torch.Tensor, breaks: torch.Tensor, r_out: Optional[torch.Tensor] = None,
+                       dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """r_out[i] = m with breaks[m] <= ids[i] < breaks[m+1] (Definition 3.1, 0-based); -1 if unrouted."""
+    lib = load_library()
+    _i32_dev(ids, "ids"), _i32_dev(breaks, "breaks")
+    N, M = ids.numel(), breaks.numel() - 1
+    if r_out is None:
+        r_out = torch.empty(N, dtype=torch.int32, device=ids.device)
+    _check("molora_route_vocab", lib.molora_route_vocab(_ptr(ids), N, _ptr(breaks), M, _ptr(_i32_dev(r_out, "r_out")),
+                                                        _ptr(dev_status), _stream(stream)))
+    return r_out
+
+
+def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                      r_out: Optional[torch.Tensor] = None, logits_out: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    """r_out[i] = argmax_c sum_k x[i,k] G[k,c] (+ bias[c]) (Eq. 8, k = 1); lowest index on ties."""
+    lib = load_library()
+    N, d, ldx = _matrix(x, "x")
+    if G.dtype != torch.float32 or not G.is_cuda or not G.is_contiguous() or G.dim() != 2 or G.shape[0] != d:
+        raise ValueError("G: expected a contiguous fp32 CUDA tensor of shape [d, C]")
+    C = G.shape[1]
+    if bias is not None and (bias.dtype != torch.float32 or bias.numel() != C or not bias.is_contiguous()):
+        raise ValueError("bias: expected contiguous fp32 [C]")
+    if r_out is None:
+        r_out = torch.empty(N, dtype=torch.int32, device=x.device)
+    if logits_out is not None and (logits_out.dtype != torch.float32 or logits_out.shape != (N, C)
+                                   or not logits_out.is_contiguous()):
+        raise ValueError("logits_out: expected contiguous fp32 [N, C]")
+    _check("molora_route_gate", lib.molora_route_gate(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(G), _ptr(bias), C,
+                                                      _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
+                                                      _stream(stream)))
+    return r_out
+
+
+def molora_group_workspace_bytes(N: int, C: int) -> int:
+    return int(load_library().molora_group_workspace_bytes(N, C))
+
+
+def molora_group(r: torch.Tensor, C: int, counts: Optional[torch.Tensor] = None,
+                 offsets: Optional[torch.Tensor] = None, perm: Optional[torch.Tensor] = None,
+                 ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                 stream=None) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """(counts [C], offsets [C+1], perm [N]) of Section 3.3; perm is stable, its first offsets[C] entries valid."""
+    lib = load_library()
+    _i32_dev(r, "r")
+    N = r.numel()
+    dev = r.device
+    counts = torch.empty(C, dtype=torch.int32, device=dev) if counts is None else _i32_dev(counts, "counts")
+    offsets = torch.empty(C + 1, dtype=torch.int32, device=dev) if offsets is None else _i32_dev(offsets, "offsets")
+    perm = torch.empty(max(N, 1), dtype=torch.int32, device=dev) if perm is None else _i32_dev(perm, "perm")
+    need = molora_group_workspace_bytes(N, C)
+    if ws is None and need > 0:
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check("molora_group", lib.molora_group(_ptr(r), N, C, _ptr(counts), _ptr(offsets), _ptr(perm), _ptr(ws), ws_bytes,
+                                            _ptr(dev_status), _stream(stream)))
+    return counts, offsets, perm
+
+
+def molora_apply_workspace_bytes(N: int, C: int, d_in: int, d_out: int, rank: int) -> int:
+    return int(load_library().molora_apply_workspace_bytes(N, C, d_in, d_out, rank))
+
+
+def molora_apply(x: torch.Tensor, y: torch.Tensor, A: torch.Tensor, B: torch.Tensor, offsets: torch.Tensor,
+                 perm: torch.Tensor, scale: float = 1.0, ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """In place: y[i] += scale * (x[i] A[c]) B[c] for every token i of every segment c (Eq. 2).  Returns y."""
+    lib = load_library()
+    N, d_in, ldx = _matrix(x, "x")
+    Ny, d_out, ldy = _matrix(y, "y")
+    dt = _dtype_code(x)
+    if Ny != N or y.dtype != x.dtype or A.dtype != x.dtype or B.dtype != x.dtype:
+        raise ValueError("x, y, A, B must share the token count and the element type")
+    if A.dim() != 3 or B.dim() != 3 or not A.is_contiguous() or not B.is_contiguous():
+        raise ValueError("A [C, d_in, rank] and B [C, rank, d_out] must be dense 3-D tensors")
+    C, rank = A.shape[0], A.shape[2]
+    if A.shape[1] != d_in or tuple(B.shape) != (C, rank, d_out):
+        raise ValueError("A / B shapes do not match x / y")
+    if offsets.numel() != C + 1:
+        raise ValueError("offsets must have C + 1 entries")
+    need = molora_apply_workspace_bytes(N, C, d_in, d_out, rank)
+    if ws is None and need > 0:
+        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check("molora_apply", lib.molora_apply(_ptr(x), ldx, _ptr(y), ldy, dt, N, d_in, d_out, rank, _ptr(A), _ptr(B), C,
+                                            _ptr(_i32_dev(offsets, "offsets")), _ptr(_i32_dev(perm, "perm")),
+                                            float(scale), _ptr(ws), ws_bytes, _stream(stream)))
+    return y
+
+
+@dataclass
+class ProjDesc:
+    """One projection of a batched apply: tensors as in :func:`molora_apply`."""
+    x: torch.Tensor
+    y: torch.Tensor
+    A: torch.Tensor
+    B: torch.Tensor
+    scale: float = 1.0
+
+
+def pack_proj_descs(projs: Sequence[ProjDesc]):
+    """Marshal ProjDesc objects into the C descriptor array (reusable across calls while the tensors live)."""
+    arr = (_ProjDescC * len(projs))()
+    N = C = dt = None
+    for i, p in enumerate(projs):
+        n, d_in, ldx = _matrix(p.x, "x")
+        ny, d_out, ldy = _matrix(p.y, "y")
+        if ny != n or p.y.dtype != p.x.dtype or p.A.dtype != p.x.dtype or p.B.dtype != p.x.dtype:
+            raise ValueError("x, y, A, B must share the token count and the element type")
+        c, rank = p.A.shape[0], p.A.shape[2]
+        if (not p.A.is_contiguous() or not p.B.is_contiguous() or p.A.shape[1] != d_in
+                or tuple(p.B.shape) != (c, rank, d_out)):
+            raise ValueError("A / B shapes do not match x / y")
+        if N is None:
+            N, C, dt = n, c, _dtype_code(p.x)
+        elif (N, C, dt) != (n, c, _dtype_code(p.x)):
+            raise ValueError("all projections of a batched apply share N, C and the element type")
+        arr[i] = _ProjDescC(p.x.data_ptr(), ldx, p.y.data_ptr(), ldy, p.A.data_ptr(), p.B.data_ptr(), d_in, d_out,
+                            rank, float(p.scale))
+    return arr, N, C, dt
+
+
+def molora_apply_batched(projs, offsets: torch.Tensor, perm: torch.Tensor, ws: Optional[torch.Tensor] = None,
+                         stream=None, packed=None) -> None:
+    """One launch for the projections of a layer (shared N, C, offsets, perm).  ``projs``: ProjDesc list."""
+    lib = load_library()
+    arr, N, C, dt = packed if packed is not None else pack_proj_descs(projs)
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check("molora_apply_batched", lib.molora_apply_batched(arr, len(arr), dt, N, C, _ptr(offsets), _ptr(perm),
+                                                            _ptr(ws), ws_bytes, _stream(stream)))

@@ -1,0 +1,118 @@
+// C ABI: argument validation on the host, then enqueue.  Nothing here touches device memory from the host,
+// allocates, or synchronises.
+#include "common.cuh"
+
+using namespace molora;
+
+namespace {
+
+bool rank_supported(int r) { return r == 8 || r == 16 || r == 32 || r == 64; }
+
+molora_status_t check_proj(const molora_proj_desc_t& p, molora_dtype_t dt)
+{
+    if (p.x == nullptr || p.y == nullptr || p.A == nullptr || p.B == nullptr) return MOLORA_ERR_INVALID_ARG;
+    if (p.d_in <= 0 || p.d_out <= 0) return MOLORA_ERR_INVALID_ARG;
+    if (!rank_supported(p.rank)) return MOLORA_ERR_UNSUPPORTED;
+    if ((p.d_in % 8) != 0 || (p.d_out % 8) != 0 || (p.ldx % 8) != 0 || (p.ldy % 8) != 0) return MOLORA_ERR_UNSUPPORTED;
+    if (p.ldx < p.d_in || p.ldy < p.d_out) return MOLORA_ERR_INVALID_ARG;
+    if (!aligned16(p.x) || !aligned16(p.y) || !aligned16(p.A) || !aligned16(p.B)) return MOLORA_ERR_INVALID_ARG;
+    (void)dt;
+    return MOLORA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* molora_version(void) { return "molora-b200 0.1 (sm_100a)"; }
+
+const char* molora_status_string(molora_status_t status)
+{
+    switch (status) {
+        case MOLORA_OK: return "ok";
+        case MOLORA_ERR_INVALID_ARG: return "invalid argument";
+        case MOLORA_ERR_UNSUPPORTED: return "unsupported shape, rank or dtype";
+        case MOLORA_ERR_WORKSPACE: return "workspace missing or too small";
+        case MOLORA_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+molora_status_t molora_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M, int32_t* r_out,
+                                   uint32_t* dev_status, void* stream)
+{
+    if (N < 0 || N >= INT32_MAX) return MOLORA_ERR_INVALID_ARG;
+    if (M < 1) return MOLORA_ERR_INVALID_ARG;
+    if (M > MOLORA_MAX_ADAPTERS) return MOLORA_ERR_UNSUPPORTED;
+    if (breaks == nullptr || (N > 0 && (ids == nullptr || r_out == nullptr))) return MOLORA_ERR_INVALID_ARG;
+    return launch_route_vocab(ids, N, breaks, M, r_out, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+molora_status_t molora_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
+                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* stream)
+{
+    if (N < 0 || N >= INT32_MAX || d <= 0 || C < 1) return MOLORA_ERR_INVALID_ARG;
+    if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
+    if (C > 32 || (d % 8) != 0 || (ldx % 8) != 0) return MOLORA_ERR_UNSUPPORTED;
+    if (ldx < d || G == nullptr) return MOLORA_ERR_INVALID_ARG;
+    if (N > 0 && (x == nullptr || r_out == nullptr || !aligned16(x))) return MOLORA_ERR_INVALID_ARG;
+    return launch_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, static_cast<cudaStream_t>(stream));
+}
+
+size_t molora_group_workspace_bytes(int64_t N, int32_t C) { return group_workspace_bytes(N, C); }
+
+molora_status_t molora_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
+                             void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream)
+{
+    if (N < 0 || N >= INT32_MAX || C < 1) return MOLORA_ERR_INVALID_ARG;
+    if (C > MOLORA_MAX_ADAPTERS) return MOLORA_ERR_UNSUPPORTED;
+    if (counts == nullptr || offsets == nullptr) return MOLORA_ERR_INVALID_ARG;
+    if (N > 0 && (r == nullptr || perm == nullptr)) return MOLORA_ERR_INVALID_ARG;
+    const size_t need = group_workspace_bytes(N, C);
+    if (need > 0 && (ws == nullptr || ws_bytes < need || !aligned16(ws))) return MOLORA_ERR_WORKSPACE;
+    return launch_group(r, N, C, counts, offsets, perm, ws, ws_bytes, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+size_t molora_apply_workspace_bytes(int64_t /*N*/, int32_t /*C*/, int32_t /*d_in*/, int32_t /*d_out*/, int32_t /*rank*/)
+{
+    return 0;
+}
+
+molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
+                                     int32_t C, const int32_t* offsets, const int32_t* perm, void* ws, size_t ws_bytes,
+                                     void* stream)
+{
+    (void)ws;
+    (void)ws_bytes;
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS) return MOLORA_ERR_INVALID_ARG;
+    if (N < 0 || N >= INT32_MAX || C < 1) return MOLORA_ERR_INVALID_ARG;
+    if (C > MOLORA_MAX_ADAPTERS) return MOLORA_ERR_UNSUPPORTED;
+    if (dt != MOLORA_F32 && dt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
+    if (offsets == nullptr || (N > 0 && perm == nullptr)) return MOLORA_ERR_INVALID_ARG;
+    for (int i = 0; i < P; ++i) {
+        const molora_status_t st = check_proj(projs[i], dt);
+        if (st != MOLORA_OK) return st;
+    }
+    return launch_apply_rowtile(projs, P, dt, N, C, offsets, perm, static_cast<cudaStream_t>(stream));
+}
+
+molora_status_t molora_apply(const void* x, int64_t ldx, void* y, int64_t ldy, molora_dtype_t dt, int64_t N,
+                             int32_t d_in, int32_t d_out, int32_t rank, const void* A, const void* B, int32_t C,
+                             const int32_t* offsets, const int32_t* perm, float scale, void* ws, size_t ws_bytes,
+                             void* stream)
+{
+    molora_proj_desc_t p;
+    p.x = x;
+    p.ldx = ldx;
+    p.y = y;
+    p.ldy = ldy;
+    p.A = A;
+    p.B = B;
+    p.d_in = d_in;
+    p.d_out = d_out;
+    p.rank = rank;
+    p.scale = scale;
+    return molora_apply_batched(&p, 1, dt, N, C, offsets, perm, ws, ws_bytes, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,141 @@
+// Shared device/host helpers of the sm_100a routed-LoRA kernels.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "molora.h"
+
+namespace molora {
+
+constexpr int kWarp = 32;
+
+__host__ __device__ constexpr int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+__host__ __device__ constexpr int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- 16-byte vectors of the two storage types -------------------------------------------------
+// A Vec<T> is one 128-bit global/shared access: 4 fp32 or 8 bf16 elements.
+template <typename T>
+struct VecTraits;
+template <>
+struct VecTraits<float> {
+    static constexpr int kElems = 4;
+};
+template <>
+struct VecTraits<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+};
+
+__device__ __forceinline__ uint4 ldg128(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+// Streaming 128-bit load for data read exactly once (activations): do not keep it in L1.
+__device__ __forceinline__ uint4 ldg128_stream(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+// Streaming 128-bit load of memory this kernel also writes (y): coherent path, no L1 allocation.
+__device__ __forceinline__ uint4 ld128_rw_stream(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p)
+                 : "memory");
+    return v;
+}
+__device__ __forceinline__ void stg128(void* p, uint4 v) { *reinterpret_cast<uint4*>(p) = v; }
+
+// bf16 pair packed in a 32-bit word -> two fp32 (exact: bf16 is the top half of an fp32).
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+// two fp32 -> packed bf16 pair, round to nearest even (lo in the low half).
+__device__ __forceinline__ uint32_t f32x2_to_bf16x2(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Unpack one 16-byte vector into fp32 registers (kElems of them).
+template <typename T>
+__device__ __forceinline__ void unpack(const uint4& v, float* out);
+template <>
+__device__ __forceinline__ void unpack<float>(const uint4& v, float* out)
+{
+    out[0] = __uint_as_float(v.x);
+    out[1] = __uint_as_float(v.y);
+    out[2] = __uint_as_float(v.z);
+    out[3] = __uint_as_float(v.w);
+}
+template <>
+__device__ __forceinline__ void unpack<__nv_bfloat16>(const uint4& v, float* out)
+{
+    out[0] = bf16lo_to_f32(v.x);
+    out[1] = bf16hi_to_f32(v.x);
+    out[2] = bf16lo_to_f32(v.y);
+    out[3] = bf16hi_to_f32(v.y);
+    out[4] = bf16lo_to_f32(v.z);
+    out[5] = bf16hi_to_f32(v.z);
+    out[6] = bf16lo_to_f32(v.w);
+    out[7] = bf16hi_to_f32(v.w);
+}
+// Pack kElems fp32 registers into one 16-byte vector of T (one RNE rounding for bf16).
+template <typename T>
+__device__ __forceinline__ uint4 pack(const float* in);
+template <>
+__device__ __forceinline__ uint4 pack<float>(const float* in)
+{
+    return make_uint4(__float_as_uint(in[0]), __float_as_uint(in[1]), __float_as_uint(in[2]), __float_as_uint(in[3]));
+}
+template <>
+__device__ __forceinline__ uint4 pack<__nv_bfloat16>(const float* in)
+{
+    return make_uint4(f32x2_to_bf16x2(in[0], in[1]), f32x2_to_bf16x2(in[2], in[3]), f32x2_to_bf16x2(in[4], in[5]),
+                      f32x2_to_bf16x2(in[6], in[7]));
+}
+
+__device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
+
+// Segment lookup shared by the apply kernels: tile index -> (segment c, first row position, row count).
+// Segment c owns positions [offsets[c], offsets[c+1]) of perm and is cut into tiles of `tile_rows` rows.
+// Returns false when `tile` is past the last tile.  C <= 256, so a serial scan by every thread is a few
+// hundred cached loads at worst; all threads of a CTA get the same answer.
+__device__ __forceinline__ bool find_tile(const int32_t* __restrict__ offsets, int C, int tile_rows, int tile,
+                                          int& seg, int& row0, int& rows)
+{
+    int base = 0;
+    int prev = __ldg(offsets);
+    for (int c = 0; c < C; ++c) {
+        const int next = __ldg(offsets + c + 1);
+        const int n = next - prev;
+        const int tiles = (n + tile_rows - 1) / tile_rows;
+        if (tile < base + tiles) {
+            seg = c;
+            row0 = prev + (tile - base) * tile_rows;
+            rows = min(tile_rows, next - row0);
+            return true;
+        }
+        base += tiles;
+        prev = next;
+    }
+    return false;
+}
+
+// Host launchers implemented in the .cu files (stream already unwrapped).
+molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M, int32_t* r_out,
+                                   uint32_t* dev_status, cudaStream_t s);
+molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
+                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, cudaStream_t s);
+size_t group_workspace_bytes(int64_t N, int32_t C);
+molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
+                             void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
+molora_status_t launch_apply_rowtile(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
+                                     int32_t C, const int32_t* offsets, const int32_t* perm, cudaStream_t s);
+
+inline molora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? MOLORA_OK : MOLORA_ERR_CUDA; }
+
+}  // namespace molora

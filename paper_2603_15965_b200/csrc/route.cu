@@ -1,0 +1,183 @@
+// Routers: vocabulary-range routing (Definition 3.1) and the linear gate with top-1 argmax (Eq. 8, k = 1).
+#include "common.cuh"
+#include "warp_reduce.cuh"
+
+namespace molora {
+
+// ------------------------------------------------------------------------------------------------
+// Vocabulary routing: r = (number of interior/upper boundaries b_1..b_M that are <= v) when
+// b_0 <= v < b_M, else -1.  For non-decreasing breaks this is the unique m with b_m <= v < b_{m+1}
+// (an empty range b_m == b_{m+1} can hold no id and is skipped by the count).  M-1 integer compares
+// per token, as the paper notes for Theorem 3.4; boundaries live in shared memory.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) route_vocab_kernel(const int32_t* __restrict__ ids, int64_t N,
+                                                          const int32_t* __restrict__ breaks, int M,
+                                                          int32_t* __restrict__ r_out, uint32_t* dev_status)
+{
+    __shared__ int32_t b[MOLORA_MAX_ADAPTERS + 1];
+    for (int i = threadIdx.x; i <= M; i += blockDim.x) b[i] = __ldg(breaks + i);
+    __syncthreads();
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    bool any_bad = false;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += stride) {
+        const int32_t v = __ldg(ids + i);
+        int32_t m;
+        if (M <= 8) {
+            m = 0;
+#pragma unroll 8
+            for (int j = 1; j < 8; ++j) m += (j < M && b[j] <= v) ? 1 : 0;
+        } else {  // upper_bound(b_1..b_{M-1}, v) by bisection
+            int lo = 1, hi = M;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (b[mid] <= v) lo = mid + 1; else hi = mid;
+            }
+            m = lo - 1;
+        }
+        const bool inside = (v >= b[0]) && (v < b[M]);
+        r_out[i] = inside ? m : -1;
+        any_bad |= !inside;
+    }
+    if (dev_status != nullptr && __any_sync(0xFFFFFFFFu, any_bad) && lane_id() == 0)
+        atomicOr(dev_status, MOLORA_DEV_ID_OUT_OF_RANGE);
+}
+
+molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M, int32_t* r_out,
+                                   uint32_t* dev_status, cudaStream_t s)
+{
+    if (N == 0) return MOLORA_OK;
+    const int threads = 256;
+    const int64_t want = ceil_div64(N, threads);
+    const int blocks = (int)(want < 148 * 8 ? want : 148 * 8);
+    route_vocab_kernel<<<blocks, threads, 0, s>>>(ids, N, breaks, M, r_out, dev_status);
+    return cuda_ok(cudaGetLastError());
+}
+
+// ------------------------------------------------------------------------------------------------
+// Linear gate.  One warp owns TOK consecutive tokens; its 32 lanes split the hidden dimension in
+// 16-byte vectors (lane L reads elements [L*VEC, L*VEC+VEC) of every KC = 32*VEC wide chunk), so x is
+// streamed exactly once with fully coalesced 128-bit loads.  The matching KC x C slice of G is staged
+// in shared memory once per CTA (8 warps share it) and read as float4 with a 4-float skew per lane,
+// which makes the quarter-warp phases of LDS.128 bank-conflict free.  Each lane keeps TOK x CP fp32
+// partial logits; one butterfly reduce-scatter per warp finishes them.
+// ------------------------------------------------------------------------------------------------
+template <typename T, int CP, int TOK>
+__global__ void __launch_bounds__(256) route_gate_kernel(const T* __restrict__ x, int64_t N, int d, int64_t ldx,
+                                                         const float* __restrict__ G, const float* __restrict__ bias,
+                                                         int C, int32_t* __restrict__ r_out,
+                                                         float* __restrict__ logits_out)
+{
+    constexpr int VEC = VecTraits<T>::kElems;
+    constexpr int KC = 32 * VEC;                 // hidden elements per chunk
+    constexpr int LANE_STRIDE = VEC * CP + 4;    // floats between the G rows of consecutive lanes (skewed)
+    constexpr int WARPS = 8;
+    __shared__ __align__(16) float Gs[32 * LANE_STRIDE];
+    __shared__ float zs[WARPS][TOK][CP];
+
+    const int warp = threadIdx.x >> 5, lane = lane_id();
+    const int64_t tok0 = ((int64_t)blockIdx.x * WARPS + warp) * TOK;
+
+    float acc[TOK][CP];
+#pragma unroll
+    for (int t = 0; t < TOK; ++t)
+#pragma unroll
+        for (int c = 0; c < CP; ++c) acc[t][c] = 0.f;
+
+    const T* xrow[TOK];
+#pragma unroll
+    for (int t = 0; t < TOK; ++t) {
+        const int64_t i = tok0 + t < N ? tok0 + t : N - 1;   // clamp: tail tokens recompute the last row, never stored
+        xrow[t] = x + i * ldx;
+    }
+
+    for (int k0 = 0; k0 < d; k0 += KC) {
+        // stage G[k0 .. k0+KC) x [0, C) into the skewed layout, zero-filling c >= C and k >= d
+        for (int e = threadIdx.x; e < KC * CP; e += blockDim.x) {
+            const int kk = e / CP, c = e - kk * CP;
+            const int k = k0 + kk;
+            const float g = (k < d && c < C) ? __ldg(G + (int64_t)k * C + c) : 0.f;
+            Gs[(kk / VEC) * LANE_STRIDE + (kk % VEC) * CP + c] = g;
+        }
+        __syncthreads();
+        const int k = k0 + lane * VEC;
+        if (k < d) {   // d is a multiple of VEC, so a vector is either fully inside or fully outside
+            float xv[TOK][VEC];
+#pragma unroll
+            for (int t = 0; t < TOK; ++t) {
+                const uint4 v = ldg128_stream(xrow[t] + k);
+                unpack<T>(v, xv[t]);
+            }
+            const float* g = Gs + lane * LANE_STRIDE;
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) {
+#pragma unroll
+                for (int c4 = 0; c4 < CP; c4 += 4) {
+                    const float4 gv = *reinterpret_cast<const float4*>(g + j * CP + c4);
+#pragma unroll
+                    for (int t = 0; t < TOK; ++t) {
+                        acc[t][c4 + 0] = fmaf(xv[t][j], gv.x, acc[t][c4 + 0]);
+                        acc[t][c4 + 1] = fmaf(xv[t][j], gv.y, acc[t][c4 + 1]);
+                        acc[t][c4 + 2] = fmaf(xv[t][j], gv.z, acc[t][c4 + 2]);
+                        acc[t][c4 + 3] = fmaf(xv[t][j], gv.w, acc[t][c4 + 3]);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+
+    // finish the logits: reduce-scatter over the warp, then park them in shared memory
+    constexpr int NV = TOK * CP;
+    float* flat = &acc[0][0];
+    warp_reduce_scatter<NV>(flat, lane);
+    constexpr int PER_LANE = NV >= 32 ? NV / 32 : 1;
+    constexpr int REPLICAS = NV >= 32 ? 1 : 32 / NV;   // lanes that end up holding the same sum
+    const int base = reduce_scatter_base<NV>(lane);
+    if (lane % REPLICAS == 0) {
+#pragma unroll
+        for (int j = 0; j < PER_LANE; ++j) (&zs[warp][0][0])[base + j] = flat[j];
+    }
+    __syncwarp();
+    if (lane < TOK && tok0 + lane < N) {
+        const int64_t i = tok0 + lane;
+        float best = 0.f;
+        int arg = 0;
+        for (int c = 0; c < C; ++c) {
+            float z = zs[warp][lane][c];
+            if (bias != nullptr) z += __ldg(bias + c);
+            if (logits_out != nullptr) logits_out[i * C + c] = z;
+            if (c == 0 || z > best) { best = z; arg = c; }   // strict '>' keeps the lowest index on ties
+        }
+        r_out[i] = arg;
+    }
+}
+
+template <typename T, int CP, int TOK>
+static molora_status_t gate_launch(const void* x, int64_t N, int d, int64_t ldx, const float* G, const float* bias,
+                                   int C, int32_t* r_out, float* logits_out, cudaStream_t s)
+{
+    const int64_t blocks = ceil_div64(N, 8 * TOK);
+    route_gate_kernel<T, CP, TOK><<<(unsigned)blocks, 256, 0, s>>>(static_cast<const T*>(x), N, d, ldx, G, bias, C,
+                                                                   r_out, logits_out);
+    return cuda_ok(cudaGetLastError());
+}
+
+template <typename T>
+static molora_status_t gate_dispatch(const void* x, int64_t N, int d, int64_t ldx, const float* G, const float* bias,
+                                     int C, int32_t* r_out, float* logits_out, cudaStream_t s)
+{
+    if (C <= 4) return gate_launch<T, 4, 4>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
+    if (C <= 8) return gate_launch<T, 8, 4>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
+    if (C <= 16) return gate_launch<T, 16, 4>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
+    return gate_launch<T, 32, 2>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);   // C <= 32 checked by the caller
+}
+
+molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
+                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, cudaStream_t s)
+{
+    if (N == 0) return MOLORA_OK;
+    if (xdt == MOLORA_BF16) return gate_dispatch<__nv_bfloat16>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
+    return gate_dispatch<float>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
+}
+
+}  // namespace molora

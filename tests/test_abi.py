@@ -1,0 +1,54 @@
+"""The C-ABI library builds for sm_100a, loads, and exports every symbol the header declares; host-side
+argument validation returns error codes before anything is enqueued.  No GPU needed (no compute calls)."""
+import ctypes
+
+import paper_2603_15965_b200 as M
+from paper_2603_15965_b200.build import build_library
+
+
+def test_library_builds_loads_and_exports_header_symbols():
+    build_library()
+    lib = M.load_library()
+    names = M.exported_symbols()
+    assert {"molora_route_vocab", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched",
+            "molora_group_workspace_bytes", "molora_apply_workspace_bytes", "molora_version",
+            "molora_status_string"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), f"header declares {name} but the library does not export it"
+    assert "sm_100a" in M.molora_version()
+    assert M.molora_status_string(0) == "ok" and "workspace" in M.molora_status_string(3)
+
+
+def test_invalid_arguments_are_refused_before_any_launch():
+    lib = M.load_library()
+    fake = ctypes.c_void_p(0x1000)      # never dereferenced: validation fails first
+    # negative N
+    assert lib.molora_route_vocab(fake, -1, fake, 2, fake, None, None) == 1
+    # null breaks
+    assert lib.molora_route_vocab(fake, 4, None, 2, fake, None, None) == 1
+    # too many ranges
+    assert lib.molora_route_vocab(fake, 4, fake, 257, fake, None, None) == 2
+    # gate: d not a multiple of 8, C too large, pitch too small
+    assert lib.molora_route_gate(fake, M.BF16, 4, 12, 16, fake, None, 4, fake, None, None) == 2
+    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 33, fake, None, None) == 2
+    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 8, fake, None, 4, fake, None, None) == 1
+    # group: C out of range, null outputs
+    assert lib.molora_group(fake, 4, 0, fake, fake, fake, None, 0, None, None) == 1
+    assert lib.molora_group(fake, 4, 300, fake, fake, fake, None, 0, None, None) == 2
+    assert lib.molora_group(fake, 4, 2, None, fake, fake, None, 0, None, None) == 1
+    # apply: unsupported rank, misaligned pointer, bad dtype, null weights
+    ok = dict(ldx=64, ldy=64, dt=M.BF16, N=4, d_in=64, d_out=64, rank=16, C=2)
+
+    def apply(**kw):
+        a = dict(ok, **kw)
+        return lib.molora_apply(a.get("x", fake), a["ldx"], a.get("y", fake), a["ldy"], a["dt"], a["N"], a["d_in"],
+                                a["d_out"], a["rank"], a.get("A", fake), a.get("B", fake), a["C"], fake, fake, 1.0,
+                                None, 0, None)
+
+    assert apply(rank=12) == 2
+    assert apply(d_in=60) == 2
+    assert apply(dt=7) == 2
+    assert apply(x=ctypes.c_void_p(0x1004)) == 1
+    assert apply(A=None) == 1
+    assert apply(ldy=32) == 1
+    assert apply(N=-3) == 1

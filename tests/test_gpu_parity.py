@@ -1,0 +1,268 @@
+"""GPU parity: the CUDA path (through the C-ABI binding) against the CPU oracle, element by element,
+on the seeded workloads and on edge shapes.  Integer outputs bit-exact; floating point within
+|gpu - ref| <= 1e-3 + 2e-2 |ref| (and 1e-5 + 1e-4 |ref| for fp32 storage)."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2603_15965_b200 as M
+from paper_2603_15965_b200 import workloads as W
+
+from _harness import (assert_close, dev_tensor, gpu_route, oracle_route, run_and_check, sample_rows, to_f64)
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ the five configurations
+def test_c1_tiny_vocab_full():
+    stats = run_and_check(W.get("c1"))
+    assert stats["gate_flipped"] == 0
+
+
+def test_c2_prefill_gate_full():
+    stats = run_and_check(W.get("c2"))
+    print("c2", stats)
+
+
+def test_c3_decode_layer_full_and_batched():
+    run_and_check(W.get("c3"))
+    run_and_check(W.get("c3", layer=1), batched=True)
+
+
+def test_c4_prefill_reduced():
+    # 7 projections, rank 64, gate 4096x16: a token count the oracle finishes in seconds, several tiles + ragged tail
+    run_and_check(W.get("c4", n_tokens=1000 + 77), batched=True)
+
+
+def test_c5_multimodal_reduced_and_iid():
+    run_and_check(W.c5_multimodal(n_seqs=2, seq_len=700))
+    run_and_check(W.c5_multimodal(n_seqs=2, seq_len=300, iid=True))
+
+
+@pytest.mark.parametrize("name", ["c4", "c5", "c5-iid"])
+def test_full_size_sampled_rows(name):
+    w = W.get(name)
+    r_ref, _ = oracle_route(w)
+    rows = sample_rows(w, r_ref, n_random=384)
+    stats = run_and_check(w, rows=rows, batched=(name == "c4"))
+    print(name, stats, "rows checked:", rows.size)
+
+
+# ------------------------------------------------------------------ routers
+def test_route_vocab_boundaries_empty_ranges_and_status():
+    breaks = np.array([5, 17, 17, 200, 1000, 4096], dtype=np.int32)
+    ids = np.random.default_rng(0).integers(0, 5000, size=3001).astype(np.int32)
+    ids[:12] = [0, 4, 5, 16, 17, 18, 199, 200, 999, 1000, 4095, 4096]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    r = M.molora_route_vocab(dev_tensor(ids, "i"), dev_tensor(breaks, "i"), dev_status=status)
+    assert np.array_equal(r.cpu().numpy(), oracle.route_vocab(ids, breaks))
+    assert int(status.item()) & 1
+    status.zero_()
+    inside = np.clip(ids, 5, 4095)
+    r = M.molora_route_vocab(dev_tensor(inside, "i"), dev_tensor(breaks, "i"), dev_status=status)
+    assert np.array_equal(r.cpu().numpy(), oracle.route_vocab(inside, breaks)) and int(status.item()) == 0
+
+
+def test_route_vocab_many_ranges():
+    rng = np.random.default_rng(1)
+    breaks = np.concatenate([[0], np.sort(rng.integers(1, 100000, size=255)), [100000]]).astype(np.int32)
+    ids = rng.integers(0, 100000, size=10007).astype(np.int32)
+    r = M.molora_route_vocab(dev_tensor(ids, "i"), dev_tensor(breaks, "i"))
+    assert np.array_equal(r.cpu().numpy(), oracle.route_vocab(ids, breaks))
+
+
+@pytest.mark.parametrize("dtype,N,d,C", [("bf16", 257, 2048, 4), ("bf16", 100, 4096, 16), ("f32", 77, 520, 7),
+                                         ("bf16", 33, 264, 32), ("bf16", 5, 8, 1), ("f32", 64, 2048, 3)])
+def test_route_gate_logits_and_argmax(dtype, N, d, C):
+    rng = np.random.default_rng(N + d + C)
+    x = rng.standard_normal((N, d), dtype=np.float32)
+    if dtype == "bf16":
+        x = W.round_to_bf16(x)
+    G = (rng.standard_normal((d, C)) * d ** -0.5).astype(np.float32)
+    bias = rng.standard_normal(C).astype(np.float32) * 0.1
+    r_ref, z_ref, margin = oracle.route_gate(x, G, bias)
+    logits = torch.empty(N, C, dtype=torch.float32, device="cuda")
+    r = M.molora_route_gate(dev_tensor(x, dtype), dev_tensor(G, "f32"), dev_tensor(bias, "f32"), logits_out=logits)
+    assert_close(to_f64(logits), z_ref, 1e-4, 1e-4, what="gate logits")
+    keep = margin >= 1e-3
+    assert np.array_equal(r.cpu().numpy()[keep], r_ref[keep])
+
+
+def test_route_gate_ties_pick_lowest_index_and_unit_vectors():
+    d, C = 64, 6
+    G = np.zeros((d, C), np.float32)
+    G[:, 2] = 1.0
+    G[:, 4] = 1.0
+    x = np.ones((40, d), np.float32)
+    r = M.molora_route_gate(dev_tensor(x, "bf16"), dev_tensor(G, "f32"))
+    assert np.all(r.cpu().numpy() == 2)
+    G = np.random.default_rng(3).standard_normal((d, C)).astype(np.float32)
+    logits = torch.empty(d, C, dtype=torch.float32, device="cuda")
+    r = M.molora_route_gate(dev_tensor(np.eye(d, dtype=np.float32), "bf16"), dev_tensor(G, "f32"), logits_out=logits)
+    assert np.array_equal(logits.cpu().numpy(), G)            # x = e_k reads row k of G exactly
+    assert np.array_equal(r.cpu().numpy(), np.argmax(G, axis=1))
+
+
+# ------------------------------------------------------------------ grouping
+@pytest.mark.parametrize("N,C", [(0, 4), (1, 1), (6, 3), (31, 2), (32, 5), (33, 256), (1000, 16), (16384, 4),
+                                 (40000, 64), (100003, 7)])
+def test_group_bit_exact(N, C):
+    rng = np.random.default_rng(N * 1000 + C)
+    r = rng.integers(-1, C, size=N).astype(np.int32)
+    if N == 6:
+        r = np.array([0, 1, 0, 2, 0, 1], np.int32)                # Figure 2's example
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    r_dev = dev_tensor(r, "i") if N else torch.empty(0, dtype=torch.int32, device="cuda")
+    counts, offsets, perm = M.molora_group(r_dev, C, dev_status=status)
+    c_ref, o_ref, p_ref = oracle.group(r, C)
+    assert np.array_equal(counts.cpu().numpy(), c_ref)
+    assert np.array_equal(offsets.cpu().numpy(), o_ref)
+    assert np.array_equal(perm.cpu().numpy()[: int(o_ref[-1])], p_ref)
+    assert int(status.item()) == 0
+
+
+def test_group_flags_bad_routes_and_skewed_inputs():
+    r = np.array([0, 7, -2, 1, 1, 300, -1, 0], np.int32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), 2, dev_status=status)
+    c_ref, o_ref, p_ref = oracle.group(r, 2)
+    assert np.array_equal(counts.cpu().numpy(), c_ref) and np.array_equal(perm.cpu().numpy()[:4], p_ref)
+    assert int(status.item()) & 2
+    for r in (np.zeros(5000, np.int32), np.full(5000, 3, np.int32), np.full(100, -1, np.int32)):
+        counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), 4)
+        c_ref, o_ref, p_ref = oracle.group(r, 4)
+        assert np.array_equal(offsets.cpu().numpy(), o_ref)
+        assert np.array_equal(perm.cpu().numpy()[: int(o_ref[-1])], p_ref)
+
+
+# ------------------------------------------------------------------ apply: edge shapes
+SEG_SIZES = [0, 1, 15, 16, 17, 63, 64, 65, 127, 128, 129]
+
+
+@pytest.mark.parametrize("dtype,rank", [("bf16", 8), ("bf16", 16), ("bf16", 32), ("bf16", 64), ("f32", 8), ("f32", 16),
+                                        ("f32", 32), ("f32", 64)])
+def test_apply_segment_size_sweep(dtype, rank):
+    r = W.segment_sizes_routing(SEG_SIZES)
+    w = W.random_problem(100 + rank, r.size, len(SEG_SIZES), 256, 328, rank, dtype, r=r)
+    run_and_check(w)
+
+
+@pytest.mark.parametrize("N,C,d_in,d_out,rank", [(1, 1, 8, 8, 8), (1, 3, 2048, 1024, 16), (300, 1, 512, 512, 32),
+                                                 (257, 256, 64, 72, 8), (513, 5, 6144, 2048, 16), (90, 3, 40, 4104, 64)])
+def test_apply_odd_shapes(N, C, d_in, d_out, rank):
+    w = W.random_problem(N + C + rank, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.1 if N > 10 else 0.0)
+    run_and_check(w)
+
+
+def test_apply_all_tokens_one_adapter_and_all_unrouted():
+    w = W.random_problem(7, 200, 4, 256, 256, 16, "bf16", r=np.full(200, 2, np.int32))
+    run_and_check(w)
+    w = W.random_problem(8, 64, 4, 256, 256, 16, "bf16", r=np.full(64, -1, np.int32))
+    y0 = w.projections[0].y.copy()
+    run_and_check(w)
+    # unrouted rows must be untouched bit for bit
+    p = w.projections[0]
+    y = dev_tensor(p.y, "bf16")
+    counts, offsets, perm = M.molora_group(dev_tensor(w.r, "i"), w.C)
+    M.molora_apply(dev_tensor(w.inputs["x"], "bf16"), y, dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), offsets, perm)
+    assert np.array_equal(y.float().cpu().numpy(), y0)
+
+
+def test_apply_scale_and_pitched_views():
+    w = W.random_problem(9, 150, 3, 128, 192, 16, "bf16")
+    run_and_check(w, scale=0.5)
+    # x and y as column slices of wider buffers (ld > d)
+    p = w.projections[0]
+    xbig = torch.zeros(w.N, 256, dtype=torch.bfloat16, device="cuda")
+    ybig = torch.zeros(w.N, 320, dtype=torch.bfloat16, device="cuda")
+    xbig[:, 64:192] = dev_tensor(w.inputs["x"], "bf16")
+    ybig[:, 128:320] = dev_tensor(p.y, "bf16")
+    guard = ybig[:, :128].clone()
+    counts, offsets, perm = M.molora_group(dev_tensor(w.r, "i"), w.C)
+    M.molora_apply(xbig[:, 64:192], ybig[:, 128:320], dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), offsets, perm)
+    ref, _ = oracle.apply(w.inputs["x"], p.y, p.A, p.B, w.r)
+    assert_close(to_f64(ybig[:, 128:320]), ref, what="pitched")
+    assert torch.equal(ybig[:, :128], guard)
+
+
+def test_apply_selector_and_zero_B_exact():
+    # A_c = e_j e_k^T, B_c = e_k e_o^T  =>  h[i][o] = y[i][o] + x[i][j] exactly (bf16-representable integers)
+    N, C, d_in, d_out, rank = 70, 3, 64, 80, 8
+    rng = np.random.default_rng(5)
+    x = rng.integers(-8, 9, size=(N, d_in)).astype(np.float32)
+    y = rng.integers(-8, 9, size=(N, d_out)).astype(np.float32)
+    A = np.zeros((C, d_in, rank), np.float32)
+    B = np.zeros((C, rank, d_out), np.float32)
+    sel = [(1, 3, 70), (60, 0, 2), (33, 7, 41)]
+    for c, (j, k, o) in enumerate(sel):
+        A[c, j, k] = 1.0
+        B[c, k, o] = 1.0
+    r = rng.integers(0, C, size=N).astype(np.int32)
+    expect = y.copy()
+    for i in range(N):
+        j, k, o = sel[r[i]]
+        expect[i, o] += x[i, j]
+    for dtype in ("bf16", "f32"):
+        yd = dev_tensor(y, dtype)
+        counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), C)
+        M.molora_apply(dev_tensor(x, dtype), yd, dev_tensor(A, dtype), dev_tensor(B, dtype), offsets, perm)
+        assert np.array_equal(yd.float().cpu().numpy(), expect)
+        yd = dev_tensor(y, dtype)
+        M.molora_apply(dev_tensor(x, dtype), yd, dev_tensor(A, dtype), dev_tensor(np.zeros_like(B), dtype), offsets, perm)
+        assert np.array_equal(yd.float().cpu().numpy(), y)
+
+
+def test_exhaustive_routings_integer_data_exact():
+    # every C^N routing of a tiny problem with integer data: all arithmetic is exact, GPU must equal the oracle
+    N, C, d_in, d_out, rank = 5, 3, 8, 8, 8
+    rng = np.random.default_rng(11)
+    x = rng.integers(-3, 4, size=(N, d_in)).astype(np.float32)
+    y = rng.integers(-3, 4, size=(N, d_out)).astype(np.float32)
+    A = rng.integers(-2, 3, size=(C, d_in, rank)).astype(np.float32)
+    B = rng.integers(-2, 3, size=(C, rank, d_out)).astype(np.float32)
+    xd, Ad, Bd = dev_tensor(x, "f32"), dev_tensor(A, "f32"), dev_tensor(B, "f32")
+    for r in itertools.product(range(C), repeat=N):
+        r = np.array(r, np.int32)
+        yd = dev_tensor(y, "f32")
+        counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), C)
+        M.molora_apply(xd, yd, Ad, Bd, offsets, perm)
+        ref, _ = oracle.apply(x, y, A, B, r)
+        assert np.array_equal(yd.cpu().numpy().astype(np.float64), ref)
+
+
+def test_permutation_equivariance_on_gpu():
+    w = W.random_problem(21, 333, 5, 512, 384, 16, "bf16")
+    p = w.projections[0]
+    pi = np.random.default_rng(2).permutation(w.N)
+
+    def run(x, y, r):
+        yd = dev_tensor(y, "bf16")
+        counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), w.C)
+        M.molora_apply(dev_tensor(x, "bf16"), yd, dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), offsets, perm)
+        return yd.float().cpu().numpy()
+
+    h = run(w.inputs["x"], p.y, w.r)
+    hp = run(w.inputs["x"][pi], p.y[pi], w.r[pi])
+    assert_close(hp.astype(np.float64), h[pi].astype(np.float64), what="permuted tokens")
+
+
+def test_kpass_per_sequence_baseline_matches_single_pass():
+    # Theorem 3.6 on the GPU kernels: K passes of constant routing + a row mask equal the one-pass result
+    w = W.c5_multimodal(n_seqs=1, seq_len=600)
+    p = w.projections[0]
+    r = oracle.route_vocab(w.ids, w.breaks)
+    x, A, B = dev_tensor(w.inputs["x"], "bf16"), dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16")
+    y1 = dev_tensor(p.y, "bf16")
+    counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), w.C)
+    M.molora_apply(x, y1, A, B, offsets, perm)
+    out = dev_tensor(p.y, "bf16")
+    r_dev = dev_tensor(r, "i")
+    for k in range(w.C):
+        yk = dev_tensor(p.y, "bf16")
+        ck, ok, pk = M.molora_group(torch.full((w.N,), k, dtype=torch.int32, device="cuda"), w.C)
+        M.molora_apply(x, yk, A, B, ok, pk)
+        out[r_dev == k] = yk[r_dev == k]
+    assert_close(to_f64(out), to_f64(y1), what="k-pass vs one pass")
