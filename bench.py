@@ -133,7 +133,8 @@ def build_sets(W, torch, name, n_sets, rank):
             "ids": dev(w.ids, "i") if w.ids is not None else None,
             "r_given": dev(w.r, "i") if w.r is not None else None,
         })
-    shared = {"G": dev(w0.G, "f32") if w0.G is not None else None,
+    shared = {"status": torch.zeros(1, dtype=torch.int32, device="cuda"),
+              "G": dev(w0.G, "f32") if w0.G is not None else None,
               "breaks": dev(w0.breaks, "i") if w0.breaks is not None else None}
     return w0, sets, shared
 
@@ -161,7 +162,7 @@ def marshal_step(lib, w, s, shared, stream_handle):
                     vp(s["offsets"].data_ptr()), vp(s["perm"].data_ptr()), None, ctypes.c_size_t(0), None, st)
     arr, n, c, dt = s["packed"]
     apply = partial(lib.molora_apply_batched, arr, i32(len(arr)), dt, i64(n), i32(c), vp(s["offsets"].data_ptr()),
-                    vp(s["perm"].data_ptr()), None, ctypes.c_size_t(0), st)
+                    vp(s["perm"].data_ptr()), None, ctypes.c_size_t(0), vp(shared["status"].data_ptr()), st)
     return route, group, apply
 
 

@@ -118,13 +118,15 @@ molora_status_t molora_group(const int32_t *r, int64_t N, int32_t C, int32_t *co
  * A   device [C, d_in, rank] of type dt, dense;  B  device [C, rank, d_out] of type dt, dense
  * offsets, perm   device outputs of molora_group for the same N, C (read on the device only)
  * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes (NULL if that is 0)
+ * dev_status      device uint32 or NULL; MOLORA_DEV_TIMEOUT is OR-ed in if a bounded wait inside the
+ *                 tensor-core kernel gave up (the kernel then returns without hanging; y is incomplete)
  * The kernel variant (CUDA-core path for small segments, tensor-core tiles for large ones) is chosen on
  * the device from the segment sizes; the paper picks its tile shape from the histogram too (Eq. 12-13). */
 size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t d_out, int32_t rank);
 molora_status_t molora_apply(const void *x, int64_t ldx, void *y, int64_t ldy, molora_dtype_t dt, int64_t N,
                              int32_t d_in, int32_t d_out, int32_t rank, const void *A, const void *B, int32_t C,
                              const int32_t *offsets, const int32_t *perm, float scale, void *ws, size_t ws_bytes,
-                             void *stream);
+                             uint32_t *dev_status, void *stream);
 
 /* Same operation for P projections that share N, C, offsets and perm (the projections of one layer),
  * enqueued as one launch.  `projs` is a HOST array of P descriptors (1 <= P <= MOLORA_MAX_PROJECTIONS),
@@ -141,7 +143,7 @@ typedef struct {
 } molora_proj_desc_t;
 molora_status_t molora_apply_batched(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N,
                                      int32_t C, const int32_t *offsets, const int32_t *perm, void *ws, size_t ws_bytes,
-                                     void *stream);
+                                     uint32_t *dev_status, void *stream);
 
 #ifdef __cplusplus
 }

@@ -71,8 +71,9 @@ def load_library():
     lib.molora_apply_workspace_bytes.restype = sz
     lib.molora_apply_workspace_bytes.argtypes = [i64, i32, i32, i32, i32]
     lib.molora_apply.argtypes = [vp, i64, vp, i64, ctypes.c_int, i64, i32, i32, i32, vp, vp, i32, vp, vp, f32, vp, sz,
-                                 vp]
-    lib.molora_apply_batched.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64, i32, vp, vp, vp, sz, vp]
+                                 vp, vp]
+    lib.molora_apply_batched.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64, i32, vp, vp, vp, sz, vp,
+                                         vp]
     for name in ("molora_route_vocab", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
@@ -190,7 +191,8 @@ def molora_apply_workspace_bytes(N: int, C: int, d_in: int, d_out: int, rank: in
 
 
 def molora_apply(x: torch.Tensor, y: torch.Tensor, A: torch.Tensor, B: torch.Tensor, offsets: torch.Tensor,
-                 perm: torch.Tensor, scale: float = 1.0, ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+                 perm: torch.Tensor, scale: float = 1.0, ws: Optional[torch.Tensor] = None,
+                 dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """In place: y[i] += scale * (x[i] A[c]) B[c] for every token i of every segment c (Eq. 2).  Returns y."""
     lib = load_library()
     N, d_in, ldx = _matrix(x, "x")
@@ -211,7 +213,7 @@ def molora_apply(x: torch.Tensor, y: torch.Tensor, A: torch.Tensor, B: torch.Ten
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_apply", lib.molora_apply(_ptr(x), ldx, _ptr(y), ldy, dt, N, d_in, d_out, rank, _ptr(A), _ptr(B), C,
                                             _ptr(_i32_dev(offsets, "offsets")), _ptr(_i32_dev(perm, "perm")),
-                                            float(scale), _ptr(ws), ws_bytes, _stream(stream)))
+                                            float(scale), _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
     return y
 
 
@@ -248,10 +250,10 @@ def pack_proj_descs(projs: Sequence[ProjDesc]):
 
 
 def molora_apply_batched(projs, offsets: torch.Tensor, perm: torch.Tensor, ws: Optional[torch.Tensor] = None,
-                         stream=None, packed=None) -> None:
+                         dev_status: Optional[torch.Tensor] = None, stream=None, packed=None) -> None:
     """One launch for the projections of a layer (shared N, C, offsets, perm).  ``projs``: ProjDesc list."""
     lib = load_library()
     arr, N, C, dt = packed if packed is not None else pack_proj_descs(projs)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_apply_batched", lib.molora_apply_batched(arr, len(arr), dt, N, C, _ptr(offsets), _ptr(perm),
-                                                            _ptr(ws), ws_bytes, _stream(stream)))
+                                                            _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))

@@ -80,7 +80,7 @@ size_t molora_apply_workspace_bytes(int64_t /*N*/, int32_t /*C*/, int32_t /*d_in
 
 molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
                                      int32_t C, const int32_t* offsets, const int32_t* perm, void* ws, size_t ws_bytes,
-                                     void* stream)
+                                     uint32_t* dev_status, void* stream)
 {
     (void)ws;
     (void)ws_bytes;
@@ -93,13 +93,28 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
         const molora_status_t st = check_proj(projs[i], dt);
         if (st != MOLORA_OK) return st;
     }
-    return launch_apply_rowtile(projs, P, dt, N, C, offsets, perm, static_cast<cudaStream_t>(stream));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // Split the projections by eligibility for the tensor-core kernel.  For eligible ones both kernels are
+    // enqueued and each segment is taken by exactly one of them, chosen on the device from its row count.
+    molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
+    int n_tc = 0, n_cc = 0;
+    for (int i = 0; i < P; ++i) {
+        if (N >= kUmmaMinTokens && umma_eligible(projs[i], dt)) tc[n_tc++] = projs[i];
+        else cc[n_cc++] = projs[i];
+    }
+    molora_status_t st = MOLORA_OK;
+    if (n_tc > 0) {
+        st = launch_apply_umma(tc, n_tc, N, C, offsets, perm, dev_status, kUmmaMinRows, s);
+        if (st == MOLORA_OK) st = launch_apply_rowtile(tc, n_tc, dt, N, C, offsets, perm, kUmmaMinRows, s);
+    }
+    if (st == MOLORA_OK && n_cc > 0) st = launch_apply_rowtile(cc, n_cc, dt, N, C, offsets, perm, INT32_MAX, s);
+    return st;
 }
 
 molora_status_t molora_apply(const void* x, int64_t ldx, void* y, int64_t ldy, molora_dtype_t dt, int64_t N,
                              int32_t d_in, int32_t d_out, int32_t rank, const void* A, const void* B, int32_t C,
                              const int32_t* offsets, const int32_t* perm, float scale, void* ws, size_t ws_bytes,
-                             void* stream)
+                             uint32_t* dev_status, void* stream)
 {
     molora_proj_desc_t p;
     p.x = x;
@@ -112,7 +127,7 @@ molora_status_t molora_apply(const void* x, int64_t ldx, void* y, int64_t ldy, m
     p.d_out = d_out;
     p.rank = rank;
     p.scale = scale;
-    return molora_apply_batched(&p, 1, dt, N, C, offsets, perm, ws, ws_bytes, stream);
+    return molora_apply_batched(&p, 1, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, stream);
 }
 
 }  // extern "C"

@@ -26,6 +26,7 @@ struct ApplyBatchParams {
     const int32_t* perm;
     int32_t P;
     int32_t C;
+    int32_t max_rows;     // segments with at least this many rows belong to the tensor-core kernel
 };
 
 constexpr int kRowTileThreads = 256;
@@ -42,7 +43,7 @@ __global__ void __launch_bounds__(kRowTileThreads, 1) apply_rowtile_kernel(const
     if (pd.rank != R) return;                // a launch of this instantiation serves the projections of rank R
 
     int seg, row0, rows;
-    if (!find_tile(prm.offsets, prm.C, TM, blockIdx.x, seg, row0, rows)) return;
+    if (!find_tile(prm.offsets, prm.C, TM, blockIdx.x, 1, prm.max_rows, seg, row0, rows)) return;
 
     __shared__ __align__(16) float partial[WARPS][128];
     __shared__ __align__(16) float t_s[128];   // [TM][R]
@@ -140,7 +141,9 @@ template <typename T, int R>
 static cudaError_t rowtile_launch(const ApplyBatchParams& prm, int64_t N, cudaStream_t s)
 {
     constexpr int TM = 128 / R;
-    const int64_t tiles = ceil_div64(N, TM) + prm.C;   // every segment adds at most one partial tile
+    // every segment adds at most one partial tile; with a row cap only min(N, C * cap) rows can come here
+    const int64_t cap_rows = prm.max_rows == INT32_MAX ? N : (N < (int64_t)prm.C * prm.max_rows ? N : (int64_t)prm.C * prm.max_rows);
+    const int64_t tiles = ceil_div64(cap_rows, TM) + prm.C;
     dim3 grid((unsigned)tiles, (unsigned)prm.P);
     apply_rowtile_kernel<T, R><<<grid, kRowTileThreads, 0, s>>>(prm);
     return cudaGetLastError();
@@ -163,9 +166,10 @@ static cudaError_t rowtile_dispatch(const ApplyBatchParams& prm, int64_t N, cuda
 }
 
 molora_status_t launch_apply_rowtile(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
-                                     int32_t C, const int32_t* offsets, const int32_t* perm, cudaStream_t s)
+                                     int32_t C, const int32_t* offsets, const int32_t* perm, int32_t max_rows,
+                                     cudaStream_t s)
 {
-    if (N == 0) return MOLORA_OK;
+    if (N == 0 || P == 0) return MOLORA_OK;
     ApplyBatchParams prm;
     for (int i = 0; i < P; ++i) prm.p[i] = projs[i];
     for (int i = P; i < MOLORA_MAX_PROJECTIONS; ++i) prm.p[i] = molora_proj_desc_t{};
@@ -173,6 +177,7 @@ molora_status_t launch_apply_rowtile(const molora_proj_desc_t* projs, int32_t P,
     prm.perm = perm;
     prm.P = P;
     prm.C = C;
+    prm.max_rows = max_rows;
     return cuda_ok(dt == MOLORA_BF16 ? rowtile_dispatch<__nv_bfloat16>(prm, N, s) : rowtile_dispatch<float>(prm, N, s));
 }
 

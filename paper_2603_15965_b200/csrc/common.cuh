@@ -101,18 +101,20 @@ __device__ __forceinline__ uint4 pack<__nv_bfloat16>(const float* in)
 __device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
 
 // Segment lookup shared by the apply kernels: tile index -> (segment c, first row position, row count).
-// Segment c owns positions [offsets[c], offsets[c+1]) of perm and is cut into tiles of `tile_rows` rows.
-// Returns false when `tile` is past the last tile.  C <= 256, so a serial scan by every thread is a few
-// hundred cached loads at worst; all threads of a CTA get the same answer.
+// Segment c owns positions [offsets[c], offsets[c+1]) of perm; only segments whose size n satisfies
+// min_rows <= n < max_rows are cut into tiles of `tile_rows` rows and numbered (this is how a kernel path is
+// chosen per segment, on the device, from the histogram).  Returns false when `tile` is past the last tile.
+// C <= 256, so a serial scan by every thread is a few hundred cached loads at worst; all threads of a CTA
+// get the same answer.
 __device__ __forceinline__ bool find_tile(const int32_t* __restrict__ offsets, int C, int tile_rows, int tile,
-                                          int& seg, int& row0, int& rows)
+                                          int min_rows, int max_rows, int& seg, int& row0, int& rows)
 {
     int base = 0;
     int prev = __ldg(offsets);
     for (int c = 0; c < C; ++c) {
         const int next = __ldg(offsets + c + 1);
         const int n = next - prev;
-        const int tiles = (n + tile_rows - 1) / tile_rows;
+        const int tiles = (n >= min_rows && n < max_rows) ? (n + tile_rows - 1) / tile_rows : 0;
         if (tile < base + tiles) {
             seg = c;
             row0 = prev + (tile - base) * tile_rows;
@@ -133,8 +135,20 @@ molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, 
 size_t group_workspace_bytes(int64_t N, int32_t C);
 molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
                              void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
+// CUDA-core path for the segments with fewer than max_rows rows (INT32_MAX: every segment).
 molora_status_t launch_apply_rowtile(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
-                                     int32_t C, const int32_t* offsets, const int32_t* perm, cudaStream_t s);
+                                     int32_t C, const int32_t* offsets, const int32_t* perm, int32_t max_rows,
+                                     cudaStream_t s);
+// tcgen05 path for the segments with at least min_rows rows (bf16, rank 16/32/64, d_in and d_out multiples of 64).
+bool umma_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
+molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
+                                  const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
+                                  cudaStream_t s);
+
+// Path selection: a segment goes to the tensor-core kernel when it has at least kUmmaMinRows rows and the call
+// has at least kUmmaMinTokens tokens (known on the host); everything else runs on the CUDA-core kernel.
+constexpr int32_t kUmmaMinRows = 32;
+constexpr int64_t kUmmaMinTokens = 1024;
 
 inline molora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? MOLORA_OK : MOLORA_ERR_CUDA; }
 

@@ -43,7 +43,7 @@ def test_invalid_arguments_are_refused_before_any_launch():
         a = dict(ok, **kw)
         return lib.molora_apply(a.get("x", fake), a["ldx"], a.get("y", fake), a["ldy"], a["dt"], a["N"], a["d_in"],
                                 a["d_out"], a["rank"], a.get("A", fake), a.get("B", fake), a["C"], fake, fake, 1.0,
-                                None, 0, None)
+                                None, 0, None, None)
 
     assert apply(rank=12) == 2
     assert apply(d_in=60) == 2

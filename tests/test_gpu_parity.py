@@ -266,3 +266,46 @@ def test_kpass_per_sequence_baseline_matches_single_pass():
         M.molora_apply(x, yk, A, B, ok, pk)
         out[r_dev == k] = yk[r_dev == k]
     assert_close(to_f64(out), to_f64(y1), what="k-pass vs one pass")
+
+
+# ------------------------------------------------------------------ tensor-core path (N >= 1024, segments >= 32 rows)
+@pytest.mark.parametrize("rank", [16, 32, 64])
+def test_tensor_path_segment_size_sweep(rank):
+    # segment sizes straddle the 32-row path threshold, the 4-row gather groups and the 128-row tile
+    sizes = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 130, 131, 255, 256, 257, 300]
+    r = W.segment_sizes_routing(sizes)
+    assert r.size >= 1024
+    w = W.random_problem(200 + rank, r.size, len(sizes), 256, 320, rank, "bf16", r=r)
+    run_and_check(w)
+
+
+@pytest.mark.parametrize("N,C,d_in,d_out,rank", [(1024, 1, 64, 64, 16), (1500, 3, 2048, 1024, 16),
+                                                 (1100, 2, 6144, 2048, 32), (2048, 4, 128, 6144, 64)])
+def test_tensor_path_shapes(N, C, d_in, d_out, rank):
+    w = W.random_problem(N + rank, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.05)
+    run_and_check(w, scale=0.75)
+
+
+def test_tensor_path_selector_exact_and_status_clean():
+    N, C, d_in, d_out, rank = 1200, 2, 128, 192, 16
+    rng = np.random.default_rng(6)
+    x = rng.integers(-8, 9, size=(N, d_in)).astype(np.float32)
+    y = rng.integers(-8, 9, size=(N, d_out)).astype(np.float32)
+    A = np.zeros((C, d_in, rank), np.float32)
+    B = np.zeros((C, rank, d_out), np.float32)
+    sel = [(77, 3, 130), (5, 15, 64)]
+    for c, (j, k, o) in enumerate(sel):
+        A[c, j, k] = 1.0
+        B[c, k, o] = 1.0
+    r = rng.integers(0, C, size=N).astype(np.int32)
+    expect = y.copy()
+    for i in range(N):
+        j, k, o = sel[r[i]]
+        expect[i, o] += x[i, j]
+    yd = dev_tensor(y, "bf16")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), C)
+    M.molora_apply(dev_tensor(x, "bf16"), yd, dev_tensor(A, "bf16"), dev_tensor(B, "bf16"), offsets, perm,
+                   dev_status=status)
+    assert np.array_equal(yd.float().cpu().numpy(), expect)
+    assert int(status.item()) == 0
