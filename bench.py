@@ -265,7 +265,7 @@ def run_ours(args):
     value = world * N / (ms_per_step * 1e-3)
 
     # ------------------------------------------------------------------ end to end with host buffers
-    e2e = run_e2e(args, torch, M, w, sets, shared, world, dist) if rank == 0 or dist is not None else None
+    e2e = None if args.profile else run_e2e(args, torch, M, w, sets, shared, world, dist)
 
     out = None
     if rank == 0:
@@ -288,7 +288,7 @@ def run_ours(args):
                          "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES.get(name),
                          "algorithmic_bytes": step_bytes, "kernel_ms": apply_ms,
                          "algorithmic_tflops": step_flops / (apply_ms * 1e-3) / 1e12},
-            "cpu_baseline": cpu_baseline(name),
+            "cpu_baseline": None if args.profile else cpu_baseline(name),
         }
     if dist is not None:
         dist.destroy_process_group()
@@ -446,6 +446,8 @@ def main():
     ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c5-iid"])
     ap.add_argument("--max-sets", type=int, default=32)
     ap.add_argument("--e2e-steps", type=int, default=50)
+    ap.add_argument("--profile", action="store_true",
+                    help="timed steps only: skip the host-buffer e2e leg and the oracle leg (for ncu captures)")
     args = ap.parse_args()
     out = run_reference(args) if args.impl == "reference" else run_ours(args)
     if out is not None:

@@ -9,18 +9,22 @@
 //   expand   D[128, 64]  = T_hi * B_c[:, n0:n0+64] + T_lo * B_c[:, n0:n0+64]   per 64-column chunk of d_out
 //   epilogue y[rows, n0:n0+64] += D    (fp32 add, one rounding to bf16, written back at the original rows)
 //
-// Data movement is all TMA: the token rows of a tile are NOT contiguous (they come from perm), so X and Y
-// chunks are fetched four rows per instruction with the row-gather form of the tensor copy, land in the
-// 128-byte-swizzled K-major layout tcgen05.mma reads, and Y goes back with the row-scatter form.  A_c / B_c
-// chunks are plain 2-D tiled loads; both are used as MN-major B operands exactly as they lie in memory
-// ([d_in, R] and [R, d_out] row-major), so no transposition pass exists.
+// Data movement.  The token rows of a tile are NOT contiguous (they come from perm).  The row-gather form of
+// the tensor copy moves only four 128-byte rows per instruction and measured ~75 cycles per instruction on
+// B200 (about 13 GB/s per SM), so rows are gathered with 16-byte cp.async copies instead: eight lanes fetch one
+// 128-byte row segment (a full line) and write it straight into the 128-byte-swizzled K-major layout that
+// tcgen05.mma reads.  A_c / B_c chunks are plain 2-D tiled TMA loads and are used as MN-major B operands
+// exactly as they lie in memory ([d_in, R] and [R, d_out] row-major), so no transposition pass exists.
+// Results leave through shared memory too: the epilogue adds D to the Y chunk in place (thread = row, the
+// swizzle makes that conflict-free), then the same threads copy the chunk out with the row-segment mapping
+// so that every global store instruction writes full 128-byte lines.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warps 2-5 = epilogue
-// (one thread per tile row / TMEM lane).  X chunks and Y chunks travel through ONE ring of shared-memory
-// stages, so Y prefetch overlaps the shrink and the shrink -> expand hand-over.  Every mbarrier wait is
-// bounded: after ~1 s a waiter raises an abort flag (and MOLORA_DEV_TIMEOUT in the status word); from then
-// on all waits fall through and no further copies are issued, so control flow stays convergent, TMEM is
-// freed and the kernel returns.
+// Warp roles (416 threads): warps 0-3 gather X and Y chunks, warp 4 issues the MMAs and owns TMEM, warps
+// 5-8 and 9-12 are two epilogue groups that take alternate 64-column chunks.  X chunks and Y chunks travel
+// through ONE ring of shared-memory stages, so Y prefetch overlaps the shrink and the shrink -> expand
+// hand-over.  Every mbarrier wait is bounded: after ~1 s a waiter raises an abort flag (and
+// MOLORA_DEV_TIMEOUT in the status word); from then on all waits fall through and no further copies are
+// issued, so control flow stays convergent, TMEM is freed and the kernel returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -30,16 +34,25 @@ namespace molora {
 
 using namespace ptx;
 
-constexpr int kUmmaThreads = 192;
+constexpr int kProducerWarps = 4;
+constexpr int kProducerThreads = kProducerWarps * 32;
+constexpr int kMmaWarp = kProducerWarps;
+constexpr int kEpiGroups = 2;
+constexpr int kEpiWarp0 = kMmaWarp + 1;
+constexpr int kUmmaThreads = (kEpiWarp0 + 4 * kEpiGroups) * 32;   // 416
 constexpr int kTileM = 128;                 // rows per tile = TMEM lanes
 constexpr int kChunkCols = 64;              // bf16 columns per stage: one 128-byte swizzle row
 constexpr int kTileBytes = kTileM * 128;    // 16 KB: X or Y chunk
 constexpr int kDBufs = 4;                   // expand accumulators in flight (64 TMEM columns each)
 constexpr int kTmemCols = 512;
+constexpr int kLag = 3;                     // cp.async groups a producer thread keeps in flight
 constexpr long long kTimeoutCycles = 2000000000LL;
 
 struct UmmaProj {
-    CUtensorMap tm_x, tm_y, tm_a, tm_b;
+    CUtensorMap tm_a, tm_b;
+    const __nv_bfloat16* x;
+    __nv_bfloat16* y;
+    int64_t ldx, ldy;
     int32_t d_in, d_out, rank;
     float scale;
 };
@@ -109,17 +122,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int KX = pj.d_in / kChunkCols, NY = pj.d_out / kChunkCols;
-    const int ngroups = (rows + 3) >> 2;                      // 4-row gather/scatter groups that hold valid rows
-    const uint32_t tile_tx = (uint32_t)ngroups * 512u;
+    const int total = KX + NY;
 
     // ---------------------------------------------------------------- set-up
     if (tid == 0) {
-        prefetch_tensormap(&pj.tm_x);
-        prefetch_tensormap(&pj.tm_y);
         prefetch_tensormap(&pj.tm_a);
         prefetch_tensormap(&pj.tm_b);
         for (int s = 0; s < Cfg::kStages; ++s) {
-            mbar_init(bar(&ctrl->full[s]), 1);
+            mbar_init(bar(&ctrl->full[s]), kProducerThreads + 1);   // every gathering thread + the weight-chunk arrival
             mbar_init(bar(&ctrl->empty[s]), 1);
         }
         mbar_init(bar(&ctrl->t_full), 1);
@@ -131,15 +141,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         ctrl->abort_flag = 0;
         fence_mbar_init();
     }
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
         tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
         tmem_relinquish();
     }
-    if (tid < kTileM) {
-        // rows past the end of the tile repeat the last valid row: a partly filled 4-row group then reads and
-        // writes that row more than once with identical bytes, which is harmless
-        ctrl->rows[tid] = __ldg(prm.perm + row0 + (tid < rows ? tid : rows - 1));
-    }
+    if (tid < kTileM) ctrl->rows[tid] = tid < rows ? __ldg(prm.perm + row0 + tid) : -1;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -147,36 +153,53 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     const uint32_t tmem_T = tmem;                               // columns [0, R)
     auto tmem_D = [&](int b) { return tmem + 64u + 64u * (uint32_t)b; };
 
-    if (warp == 0) {
-        // ============================================================ TMA producer
-        if (lane == 0) {
-            const int total = KX + NY;
-            for (int it = 0; it < total; ++it) {
+    if (warp < kProducerWarps) {
+        // ============================================================ gather producer
+        // Thread t moves the 16-byte piece (t & 7) of rows (t >> 3) + 16 i, i = 0..7, of every chunk: eight lanes
+        // cover one 128-byte row segment.  Completion: each thread waits for its own copies (kLag chunks
+        // later), makes them visible to the tensor-core (async) proxy and arrives on the stage's barrier.
+        const int piece = tid & 7;
+        int64_t xoff[8], yoff[8];
+        uint32_t soff[8];
+        bool valid[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = (tid >> 3) + 16 * i;
+            const int tok = ctrl->rows[r];
+            valid[i] = tok >= 0;
+            xoff[i] = (int64_t)(valid[i] ? tok : 0) * pj.ldx + piece * 8;
+            yoff[i] = (int64_t)(valid[i] ? tok : 0) * pj.ldy + piece * 8;
+            soff[i] = swizzle_offset((uint32_t)r * 128u + piece * 16, 3);
+        }
+        for (int it = 0; it < total + kLag; ++it) {
+            if (it < total) {
                 const int s = it % Cfg::kStages;
                 const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
                 wait_bar(bar(&ctrl->empty[s]), ph ^ 1u, abort_flag, prm.dev_status);
-                if (*abort_flag) break;
-                const uint32_t fb = bar(&ctrl->full[s]);
-                mbar_arrive_expect_tx(fb, tile_tx + (uint32_t)Cfg::kWBytes);
                 const bool is_x = it < KX;
                 const int chunk = is_x ? it : it - KX;
-                const void* tm = is_x ? (const void*)&pj.tm_x : (const void*)&pj.tm_y;
                 const uint32_t dst = stage(s);
-                for (int g = 0; g < ngroups; ++g) {
-                    const int4 rr = *reinterpret_cast<const int4*>(&ctrl->rows[4 * g]);
-                    tma_gather4(dst + (uint32_t)g * 512u, tm, chunk * kChunkCols, rr.x, rr.y, rr.z, rr.w, fb);
+                if (!*abort_flag) {
+                    if (tid == 0) {
+                        const uint32_t fb = bar(&ctrl->full[s]);
+                        mbar_arrive_expect_tx(fb, (uint32_t)Cfg::kWBytes);
+                        if (is_x) tma_load_2d(dst + kTileBytes, &pj.tm_a, 0, seg * pj.d_in + chunk * kChunkCols, fb);
+                        else tma_load_2d(dst + kTileBytes, &pj.tm_b, chunk * kChunkCols, seg * R, fb);
+                    }
+                    const __nv_bfloat16* src = (is_x ? pj.x : pj.y) + chunk * kChunkCols;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (valid[i]) cp_async_16(dst + soff[i], src + (is_x ? xoff[i] : yoff[i]));
                 }
-                if (is_x) tma_load_2d(dst + kTileBytes, &pj.tm_a, 0, seg * pj.d_in + chunk * kChunkCols, fb);
-                else tma_load_2d(dst + kTileBytes, &pj.tm_b, chunk * kChunkCols, seg * R, fb);
             }
-            if (*abort_flag) {
-                // give copies that are still in flight a bounded time to land before the CTA retires
-                const long long t0 = clock64();
-                while (clock64() - t0 < 400000) {}
+            cp_async_commit();
+            if (it >= kLag) {
+                cp_async_wait<kLag>();
+                fence_proxy_async_smem();
+                mbar_arrive(bar(&ctrl->full[(it - kLag) % Cfg::kStages]));
             }
         }
-        __syncwarp();
-    } else if (warp == 1) {
+    } else if (warp == kMmaWarp) {
         // ============================================================ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc_shrink = idesc_bf16_f32(kTileM, R, 0, 1);
@@ -227,15 +250,17 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         }
         __syncwarp();
     } else {
-        // ============================================================ epilogue: one thread per tile row
+        // ============================================================ epilogue groups
+        const int group = (warp - kEpiWarp0) >> 2;    // takes chunks group, group + 2, ...
+        const int et = tid - (kEpiWarp0 + 4 * group) * 32;   // 0..127 inside the group
         const int q = warp & 3;                       // TMEM lane quarter this warp may access
-        const int row = q * 32 + lane;
+        const int row = q * 32 + lane;                // tile row = TMEM lane this thread reads
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        const bool leader = row == 0;
 
-        wait_bar(bar(&ctrl->t_full), 0, abort_flag, prm.dev_status);
-        tc_fence_after();
-        {
+        if (group == 0) {
+            // T -> scaled bf16 hi/lo pair in shared memory, K-major, swizzled like a TMA tile of R*2-byte rows
+            wait_bar(bar(&ctrl->t_full), 0, abort_flag, prm.dev_status);
+            tc_fence_after();
             uint32_t tv[R];
 #pragma unroll
             for (int c = 0; c < R / 16; ++c) tmem_ld_x16(tmem_T + lane_addr + c * 16, tv + c * 16);
@@ -254,13 +279,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(thi + off), "r"(h.x), "r"(h.y), "r"(h.z), "r"(h.w) : "memory");
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(tlo + off), "r"(l.x), "r"(l.y), "r"(l.z), "r"(l.w) : "memory");
             }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(bar(&ctrl->t_ready));
         }
-        fence_proxy_async_smem();
-        tc_fence_before();
-        mbar_arrive(bar(&ctrl->t_ready));
 
-        int prev_stage = -1;
-        for (int nc = 0; nc < NY; ++nc) {
+        // copy-out mapping: piece (et & 7) of rows (et >> 3) + 16 i
+        const int piece = et & 7;
+        for (int nc = group; nc < NY; nc += kEpiGroups) {
             const int it = KX + nc;
             const int s = it % Cfg::kStages;
             const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
@@ -287,30 +313,30 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 v = pack<__nv_bfloat16>(yv);
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
             }
-            fence_proxy_async_smem();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (leader) {
-                if (!*abort_flag) {
-                    for (int g = 0; g < ngroups; ++g) {
-                        const int4 rr = *reinterpret_cast<const int4*>(&ctrl->rows[4 * g]);
-                        tma_scatter4(&pj.tm_y, ytile + (uint32_t)g * 512u, nc * kChunkCols, rr.x, rr.y, rr.z, rr.w);
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
+            if (!*abort_flag) {
+                __nv_bfloat16* dstc = pj.y + nc * kChunkCols + piece * 8;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = (et >> 3) + 16 * i;
+                    const int tok = ctrl->rows[r];
+                    if (tok >= 0) {
+                        const uint32_t addr = ytile + swizzle_offset((uint32_t)r * 128u + piece * 16, 3);
+                        uint4 v;
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+                        stg128(dstc + (int64_t)tok * pj.ldy, v);
                     }
                 }
-                bulk_commit_group();
-                if (prev_stage >= 0) {          // the previous chunk's stores have finished reading their stage
-                    bulk_wait_group_read<1>();
-                    mbar_arrive(bar(&ctrl->empty[prev_stage]));
-                }
             }
-            prev_stage = s;
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
+            if (et == 0) mbar_arrive(bar(&ctrl->empty[s]));   // the stage may be refilled
         }
-        if (leader) bulk_wait_group<0>();       // all rows of y are written before the CTA retires
     }
 
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -381,12 +407,14 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
         UmmaProj& u = prm.p[i];
         const CUtensorMapSwizzle wswz = d.rank == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
                                         : d.rank == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-        bool ok = make_map(&u.tm_x, d.x, d.d_in, N, d.ldx, kChunkCols, 1, CU_TENSOR_MAP_SWIZZLE_128B);
-        ok = ok && make_map(&u.tm_y, d.y, d.d_out, N, d.ldy, kChunkCols, 1, CU_TENSOR_MAP_SWIZZLE_128B);
-        ok = ok && make_map(&u.tm_a, d.A, d.rank, (uint64_t)C * d.d_in, d.rank, d.rank, kChunkCols, wswz);
+        bool ok = make_map(&u.tm_a, d.A, d.rank, (uint64_t)C * d.d_in, d.rank, d.rank, kChunkCols, wswz);
         ok = ok && make_map(&u.tm_b, d.B, d.d_out, (uint64_t)C * d.rank, d.d_out, kChunkCols, d.rank,
                             CU_TENSOR_MAP_SWIZZLE_128B);
         if (!ok) return MOLORA_ERR_CUDA;
+        u.x = static_cast<const __nv_bfloat16*>(d.x);
+        u.y = static_cast<__nv_bfloat16*>(d.y);
+        u.ldx = d.ldx;
+        u.ldy = d.ldy;
         u.d_in = d.d_in;
         u.d_out = d.d_out;
         u.rank = d.rank;
