@@ -19,13 +19,23 @@
 // swizzle makes that conflict-free), then the same threads copy the chunk out with the row-segment mapping
 // so that every global store instruction writes full 128-byte lines.
 //
-// Warp roles (416 threads): warps 0-3 gather X and Y chunks, warp 4 issues the MMAs and owns TMEM, warps
-// 5-8 and 9-12 are two epilogue groups that take alternate 64-column chunks.  X chunks and Y chunks travel
+// Occupancy.  A call with few tiles (N / 128 of them) cannot fill 148 SMs, so a tile may be shared by a
+// thread-block cluster of S = 2 or 4 CTAs: CTA q shrinks over the q-th slice of d_in, the S partial T
+// tiles (fp32) are exchanged through distributed shared memory and summed in rank order by every CTA (so
+// all of them hold the same bits), and CTA q then expands into the q-th slice of d_out.  x, y, A_c and B_c
+// are still read exactly once per tile.  The exchange uses mbarriers with remote arrives (bounded waits);
+// the only hardware cluster barriers are one after set-up and one before exit, which every thread reaches.
+//
+// Warp roles (448 threads): warps 0-3 gather X and Y chunks, warp 4 fetches the A_c / B_c chunks, warp 5 issues
+// the MMAs and owns TMEM, warps 6-9 and 10-13 are two epilogue groups that take alternate 64-column chunks.  X chunks and Y chunks travel
 // through ONE ring of shared-memory stages, so Y prefetch overlaps the shrink and the shrink -> expand
 // hand-over.  Every mbarrier wait is bounded: after ~1 s a waiter raises an abort flag (and
 // MOLORA_DEV_TIMEOUT in the status word); from then on all waits fall through and no further copies are
 // issued, so control flow stays convergent, TMEM is freed and the kernel returns.
 #include <cuda.h>
+#include <stdlib.h>
+
+#include <algorithm>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -36,16 +46,17 @@ using namespace ptx;
 
 constexpr int kProducerWarps = 4;
 constexpr int kProducerThreads = kProducerWarps * 32;
-constexpr int kMmaWarp = kProducerWarps;
+constexpr int kWeightWarp = kProducerWarps;
+constexpr int kMmaWarp = kWeightWarp + 1;
 constexpr int kEpiGroups = 2;
 constexpr int kEpiWarp0 = kMmaWarp + 1;
-constexpr int kUmmaThreads = (kEpiWarp0 + 4 * kEpiGroups) * 32;   // 416
+constexpr int kUmmaThreads = (kEpiWarp0 + 4 * kEpiGroups) * 32;   // 448
 constexpr int kTileM = 128;                 // rows per tile = TMEM lanes
 constexpr int kChunkCols = 64;              // bf16 columns per stage: one 128-byte swizzle row
 constexpr int kTileBytes = kTileM * 128;    // 16 KB: X or Y chunk
 constexpr int kDBufs = 4;                   // expand accumulators in flight (64 TMEM columns each)
 constexpr int kTmemCols = 512;
-constexpr int kLag = 3;                     // cp.async groups a producer thread keeps in flight
+constexpr int kMaxSplit = 4;                // largest cluster a tile is split over
 constexpr long long kTimeoutCycles = 2000000000LL;
 
 struct UmmaProj {
@@ -62,7 +73,32 @@ struct UmmaParams {
     const int32_t* perm;
     uint32_t* dev_status;
     int32_t P, C, min_rows;
+#ifdef MOLORA_TRACE
+    long long* trace;     // development builds only: clock64 stamps of CTA 0, [role][iteration][slot]
+#endif
 };
+
+#ifdef MOLORA_TRACE
+#define MOLORA_TR(role, it, slot)                                                        \
+    do {                                                                                 \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && prm.trace != nullptr && (it) < 256)    \
+            prm.trace[((role) * 256 + (it)) * 8 + (slot)] = clock64();                   \
+    } while (0)
+__device__ __forceinline__ long long molora_gtime()
+{
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define MOLORA_TR_CTA(slot)                                                                              \
+    do {                                                                                                 \
+        if (prm.trace != nullptr && threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.x < 2048)            \
+            prm.trace[4 * 256 * 8 + blockIdx.x * 2 + (slot)] = molora_gtime();                           \
+    } while (0)
+#else
+#define MOLORA_TR(role, it, slot) do { } while (0)
+#define MOLORA_TR_CTA(slot) do { } while (0)
+#endif
 
 template <int R>
 struct UmmaCfg {
@@ -78,7 +114,7 @@ struct UmmaCfg {
 };
 
 struct Ctrl {                         // lives in shared memory after the tiles
-    uint64_t full[8], empty[8], t_full, t_ready, d_full[kDBufs], d_empty[kDBufs];
+    uint64_t full[8], empty[8], t_full, t_ready, d_full[kDBufs], d_empty[kDBufs], part_full, part_free;
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) int32_t rows[kTileM];
@@ -101,15 +137,34 @@ __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 
+// Same, for a barrier that CTAs of the cluster arrive on remotely (acquire at cluster scope).
+__device__ __forceinline__ void wait_bar_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                 uint32_t* dev_status)
+{
+    if (*abort_flag) return;
+    if (mbar_try_wait_cluster(bar, parity)) return;
+    const long long t0 = clock64();
+    while (!mbar_try_wait_cluster(bar, parity)) {
+        if (*abort_flag) return;
+        if (clock64() - t0 > kTimeoutCycles) {
+            *abort_flag = 1;
+            if (dev_status != nullptr) atomicOr(dev_status, MOLORA_DEV_TIMEOUT);
+            return;
+        }
+    }
+}
+
 template <int R>
 __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __grid_constant__ UmmaParams prm)
 {
     using Cfg = UmmaCfg<R>;
     extern __shared__ uint8_t smem_raw[];
+    MOLORA_TR_CTA(0);
     const UmmaProj& pj = prm.p[blockIdx.y];
     if (pj.rank != R) return;
     int seg, row0, rows;
-    if (!find_tile(prm.offsets, prm.C, kTileM, blockIdx.x, prm.min_rows, INT32_MAX, seg, row0, rows)) return;
+    const uint32_t S = cluster_nctarank(), crank = cluster_ctarank();   // CTAs sharing this tile, and my slice
+    if (!find_tile(prm.offsets, prm.C, kTileM, blockIdx.x / S, prm.min_rows, INT32_MAX, seg, row0, rows)) return;
 
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -121,10 +176,13 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     auto bar = [&](const uint64_t* b) { return smem_u32(b); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int KX = pj.d_in / kChunkCols, NY = pj.d_out / kChunkCols;
+    const int KXall = pj.d_in / kChunkCols, NYall = pj.d_out / kChunkCols;
+    const int kx0 = (int)(crank * KXall / S), KX = (int)((crank + 1) * KXall / S) - kx0;   // my slice of d_in
+    const int ny0 = (int)(crank * NYall / S), NY = (int)((crank + 1) * NYall / S) - ny0;   // my slice of d_out
     const int total = KX + NY;
 
     // ---------------------------------------------------------------- set-up
+    if (tid == 0) MOLORA_TR(3, 0, 0);
     if (tid == 0) {
         prefetch_tensormap(&pj.tm_a);
         prefetch_tensormap(&pj.tm_b);
@@ -138,6 +196,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             mbar_init(bar(&ctrl->d_full[b]), 1);
             mbar_init(bar(&ctrl->d_empty[b]), kTileM);
         }
+        mbar_init(bar(&ctrl->part_full), 4 * S);     // one arrival per epilogue warp of group 0 of every CTA
+        mbar_init(bar(&ctrl->part_free), 4 * S);
         ctrl->abort_flag = 0;
         fence_mbar_init();
     }
@@ -149,6 +209,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (tid == 0) MOLORA_TR(3, 0, 1);
+    if (S > 1) cluster_sync_all();     // every CTA of the cluster is running and has initialised its barriers
+    if (tid == 0) MOLORA_TR(3, 0, 2);
     const uint32_t tmem = ctrl->tmem_base;
     const uint32_t tmem_T = tmem;                               // columns [0, R)
     auto tmem_D = [&](int b) { return tmem + 64u + 64u * (uint32_t)b; };
@@ -156,49 +219,66 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     if (warp < kProducerWarps) {
         // ============================================================ gather producer
         // Thread t moves the 16-byte piece (t & 7) of rows (t >> 3) + 16 i, i = 0..7, of every chunk: eight lanes
-        // cover one 128-byte row segment.  Completion: each thread waits for its own copies (kLag chunks
-        // later), makes them visible to the tensor-core (async) proxy and arrives on the stage's barrier.
+        // cover one 128-byte row segment.  Each thread's arrival on the stage barrier is triggered by the
+        // hardware when its copies have landed, so up to kStages chunks are in flight per SM.
+        constexpr int kRowsPerThread = kTileM * 8 / kProducerThreads;
+        constexpr int kRowStep = kProducerThreads / 8;
         const int piece = tid & 7;
-        int64_t xoff[8], yoff[8];
-        uint32_t soff[8];
-        bool valid[8];
+        const __nv_bfloat16* xsrc[kRowsPerThread];
+        const __nv_bfloat16* ysrc[kRowsPerThread];
+        uint32_t soff[kRowsPerThread];
+        bool valid[kRowsPerThread];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = (tid >> 3) + 16 * i;
+        for (int i = 0; i < kRowsPerThread; ++i) {
+            const int r = (tid >> 3) + kRowStep * i;
             const int tok = ctrl->rows[r];
             valid[i] = tok >= 0;
-            xoff[i] = (int64_t)(valid[i] ? tok : 0) * pj.ldx + piece * 8;
-            yoff[i] = (int64_t)(valid[i] ? tok : 0) * pj.ldy + piece * 8;
+            xsrc[i] = pj.x + (int64_t)(valid[i] ? tok : 0) * pj.ldx + piece * 8 + kx0 * kChunkCols;
+            ysrc[i] = pj.y + (int64_t)(valid[i] ? tok : 0) * pj.ldy + piece * 8 + ny0 * kChunkCols;
             soff[i] = swizzle_offset((uint32_t)r * 128u + piece * 16, 3);
         }
-        for (int it = 0; it < total + kLag; ++it) {
-            if (it < total) {
-                const int s = it % Cfg::kStages;
-                const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
-                wait_bar(bar(&ctrl->empty[s]), ph ^ 1u, abort_flag, prm.dev_status);
-                const bool is_x = it < KX;
-                const int chunk = is_x ? it : it - KX;
-                const uint32_t dst = stage(s);
-                if (!*abort_flag) {
-                    if (tid == 0) {
-                        const uint32_t fb = bar(&ctrl->full[s]);
-                        mbar_arrive_expect_tx(fb, (uint32_t)Cfg::kWBytes);
-                        if (is_x) tma_load_2d(dst + kTileBytes, &pj.tm_a, 0, seg * pj.d_in + chunk * kChunkCols, fb);
-                        else tma_load_2d(dst + kTileBytes, &pj.tm_b, chunk * kChunkCols, seg * R, fb);
-                    }
-                    const __nv_bfloat16* src = (is_x ? pj.x : pj.y) + chunk * kChunkCols;
+        int s = 0;
+        uint32_t ph = 1;                                        // parity of the "empty" phase to wait for
+        for (int it = 0; it < total; ++it) {
+            if (tid == 0) MOLORA_TR(0, it, 0);
+            wait_bar(bar(&ctrl->empty[s]), ph, abort_flag, prm.dev_status);
+            if (tid == 0) MOLORA_TR(0, it, 1);
+            const uint32_t dst = stage(s);
+            if (!*abort_flag) {
+                if (it < KX) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        if (valid[i]) cp_async_16(dst + soff[i], src + (is_x ? xoff[i] : yoff[i]));
+                    for (int i = 0; i < kRowsPerThread; ++i) {
+                        if (valid[i]) cp_async_16(dst + soff[i], xsrc[i]);
+                        xsrc[i] += kChunkCols;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < kRowsPerThread; ++i) {
+                        if (valid[i]) cp_async_16(dst + soff[i], ysrc[i]);
+                        ysrc[i] += kChunkCols;
+                    }
                 }
             }
-            cp_async_commit();
-            if (it >= kLag) {
-                cp_async_wait<kLag>();
-                fence_proxy_async_smem();
-                mbar_arrive(bar(&ctrl->full[(it - kLag) % Cfg::kStages]));
+            cp_async_arrive_noinc(bar(&ctrl->full[s]));
+            if (tid == 0) MOLORA_TR(0, it, 2);
+            if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
+        }
+    } else if (warp == kWeightWarp) {
+        // ============================================================ weight-chunk producer (TMA)
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 1;
+            for (int it = 0; it < total; ++it) {
+                wait_bar(bar(&ctrl->empty[s]), ph, abort_flag, prm.dev_status);
+                if (*abort_flag) break;
+                const uint32_t fb = bar(&ctrl->full[s]);
+                mbar_arrive_expect_tx(fb, (uint32_t)Cfg::kWBytes);
+                if (it < KX) tma_load_2d(stage(s) + kTileBytes, &pj.tm_a, 0, seg * pj.d_in + (kx0 + it) * kChunkCols, fb);
+                else tma_load_2d(stage(s) + kTileBytes, &pj.tm_b, (ny0 + it - KX) * kChunkCols, seg * R, fb);
+                if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
             }
         }
+        __syncwarp();
     } else if (warp == kMmaWarp) {
         // ============================================================ MMA issuer
         if (lane == 0) {
@@ -208,7 +288,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             for (int it = 0; it < KX; ++it) {
                 const int s = it % Cfg::kStages;
                 const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
+                MOLORA_TR(1, it, 0);
                 wait_bar(bar(&ctrl->full[s]), ph, abort_flag, prm.dev_status);
+                MOLORA_TR(1, it, 1);
+                fence_proxy_async_smem();     // the gathered rows were written through the generic proxy
                 tc_fence_after();
                 if (!*abort_flag) {
                     const uint32_t a0 = stage(s), w0 = a0 + kTileBytes;
@@ -222,15 +305,20 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 }
             }
             if (!*abort_flag) umma_commit(bar(&ctrl->t_full));
+            MOLORA_TR(3, 1, 0);
             wait_bar(bar(&ctrl->t_ready), 0, abort_flag, prm.dev_status);
+            MOLORA_TR(3, 1, 1);
             tc_fence_after();
             for (int nc = 0; nc < NY; ++nc) {
                 const int it = KX + nc;
                 const int s = it % Cfg::kStages;
                 const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
                 const int b = nc % kDBufs;
+                MOLORA_TR(1, it, 0);
                 wait_bar(bar(&ctrl->full[s]), ph, abort_flag, prm.dev_status);
+                MOLORA_TR(1, it, 1);
                 wait_bar(bar(&ctrl->d_empty[b]), ((uint32_t)(nc / kDBufs) & 1u) ^ 1u, abort_flag, prm.dev_status);
+                MOLORA_TR(1, it, 2);
                 tc_fence_after();
                 if (!*abort_flag) {
                     const uint32_t w0 = stage(s) + kTileBytes;
@@ -259,12 +347,65 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 
         if (group == 0) {
             // T -> scaled bf16 hi/lo pair in shared memory, K-major, swizzled like a TMA tile of R*2-byte rows
+            if (et == 0) MOLORA_TR(3, 2, 0);
             wait_bar(bar(&ctrl->t_full), 0, abort_flag, prm.dev_status);
+            if (et == 0) MOLORA_TR(3, 2, 1);
             tc_fence_after();
             uint32_t tv[R];
 #pragma unroll
             for (int c = 0; c < R / 16; ++c) tmem_ld_x16(tmem_T + lane_addr + c * 16, tv + c * 16);
             tmem_wait_ld();
+            if (S > 1) {
+                // Exchange the partial T tiles.  Mine goes to the (still unused) T_hi/T_lo region as
+                // [R/4][128] float4, so a warp touches 512 contiguous bytes per access, locally and remotely.
+#pragma unroll
+                for (int c4 = 0; c4 < R / 4; ++c4)
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(thi + (uint32_t)(c4 * kTileM + row) * 16u),
+                                 "r"(tv[4 * c4]), "r"(tv[4 * c4 + 1]), "r"(tv[4 * c4 + 2]), "r"(tv[4 * c4 + 3]) : "memory");
+                __syncwarp();                                   // the warp's rows are written; lane q2 tells CTA q2
+                if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
+                if (et == 0) MOLORA_TR(3, 2, 2);
+                wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
+                if (et == 0) MOLORA_TR(3, 2, 3);
+#pragma unroll
+                for (int e = 0; e < R; ++e) tv[e] = 0u;
+                if (!*abort_flag) {
+                    // Sum in rank order (every CTA of the cluster gets the same bits).  Loads of one 16-column
+                    // slab from all peers are issued together so that their latencies overlap.
+                    uint32_t rbase[kMaxSplit];
+#pragma unroll
+                    for (int q2 = 0; q2 < kMaxSplit; ++q2) rbase[q2] = map_to_cta(thi, (uint32_t)q2 < S ? q2 : 0);
+#pragma unroll
+                    for (int slab = 0; slab < R / 16; ++slab) {
+                        float4 v[kMaxSplit][4];
+#pragma unroll
+                        for (int q2 = 0; q2 < kMaxSplit; ++q2)
+                            if ((uint32_t)q2 < S) {
+#pragma unroll
+                                for (int c = 0; c < 4; ++c)
+                                    v[q2][c] = ld_cluster_f32x4(rbase[q2] + (uint32_t)((slab * 4 + c) * kTileM + row) * 16u);
+                            }
+#pragma unroll
+                        for (int q2 = 0; q2 < kMaxSplit; ++q2)
+                            if ((uint32_t)q2 < S) {
+#pragma unroll
+                                for (int c = 0; c < 4; ++c) {
+                                    const int e = (slab * 4 + c) * 4;
+                                    tv[e + 0] = __float_as_uint(__uint_as_float(tv[e + 0]) + v[q2][c].x);
+                                    tv[e + 1] = __float_as_uint(__uint_as_float(tv[e + 1]) + v[q2][c].y);
+                                    tv[e + 2] = __float_as_uint(__uint_as_float(tv[e + 2]) + v[q2][c].z);
+                                    tv[e + 3] = __float_as_uint(__uint_as_float(tv[e + 3]) + v[q2][c].w);
+                                }
+                            }
+                    }
+                }
+                // nobody may overwrite its partial (with T_hi/T_lo) before every CTA has read it
+                __syncwarp();
+                if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_free), (uint32_t)lane));
+                if (et == 0) MOLORA_TR(3, 2, 4);
+                wait_bar_cluster(bar(&ctrl->part_free), 0, abort_flag, prm.dev_status);
+                if (et == 0) MOLORA_TR(3, 2, 5);
+            }
 #pragma unroll
             for (int c8 = 0; c8 < R / 8; ++c8) {
                 float hi[8], lo[8];
@@ -282,6 +423,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(bar(&ctrl->t_ready));
+            if (et == 0) MOLORA_TR(3, 2, 6);
         }
 
         // copy-out mapping: piece (et & 7) of rows (et >> 3) + 16 i
@@ -291,7 +433,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             const int s = it % Cfg::kStages;
             const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
             const int b = nc % kDBufs;
+            if (et == 0) MOLORA_TR(2, it, 0);
             wait_bar(bar(&ctrl->d_full[b]), (uint32_t)(nc / kDBufs) & 1u, abort_flag, prm.dev_status);
+            if (et == 0) MOLORA_TR(2, it, 1);
             tc_fence_after();
             uint32_t dv[64];
 #pragma unroll
@@ -299,7 +443,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive(bar(&ctrl->d_empty[b]));
+            if (et == 0) MOLORA_TR(2, it, 2);
             wait_bar(bar(&ctrl->full[s]), ph, abort_flag, prm.dev_status);   // the Y chunk of this stage has landed
+            if (et == 0) MOLORA_TR(2, it, 3);
             const uint32_t ytile = stage(s);
 #pragma unroll
             for (int c8 = 0; c8 < 8; ++c8) {
@@ -313,9 +459,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 v = pack<__nv_bfloat16>(yv);
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
             }
+            if (et == 0) MOLORA_TR(2, it, 4);
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
+            if (et == 0) MOLORA_TR(2, it, 5);
             if (!*abort_flag) {
-                __nv_bfloat16* dstc = pj.y + nc * kChunkCols + piece * 8;
+                __nv_bfloat16* dstc = pj.y + (ny0 + nc) * kChunkCols + piece * 8;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int r = (et >> 3) + 16 * i;
@@ -330,13 +478,19 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             }
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
             if (et == 0) mbar_arrive(bar(&ctrl->empty[s]));   // the stage may be refilled
+            if (et == 0) MOLORA_TR(2, it, 6);
         }
     }
 
     // ---------------------------------------------------------------- teardown
+    if (tid == 0) MOLORA_TR(3, 0, 3);
     tc_fence_before();
     __syncthreads();
+    if (tid == 0) MOLORA_TR(3, 0, 4);
     if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
+    if (S > 1) cluster_sync_all();     // no CTA retires while a peer could still touch its shared memory
+    if (tid == 0) MOLORA_TR(3, 0, 5);
+    MOLORA_TR_CTA(1);
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -379,7 +533,7 @@ bool umma_eligible(const molora_proj_desc_t& p, molora_dtype_t dt)
 }
 
 template <int R>
-static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, cudaStream_t s)
+static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, int split, cudaStream_t s)
 {
     using Cfg = UmmaCfg<R>;
     static bool configured = false;
@@ -390,9 +544,38 @@ static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, cudaStream_t s)
         configured = true;
     }
     const int64_t tiles = ceil_div64(N, kTileM) + prm.C;
-    dim3 grid((unsigned)tiles, (unsigned)prm.P);
-    apply_umma_kernel<R><<<grid, kUmmaThreads, Cfg::kSmemBytes, s>>>(prm);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles * split), (unsigned)prm.P, 1);
+    cfg.blockDim = dim3(kUmmaThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R>, prm);
+}
+
+// CTAs per tile.  Tiles are 128 rows, so small calls have too few of them for 148 SMs: split each tile over a
+// cluster of 2 or 4 CTAs while that still fits in one wave, keeping at least four 64-column chunks of d_in
+// per CTA.  (Clusters of 8 leave SMs of a GPC idle and their exchange costs more than it returns.)
+static int choose_split(const UmmaParams& prm, int64_t N)
+{
+    int min_kx = INT32_MAX;
+    int64_t tiles = 0;
+    for (int i = 0; i < prm.P; ++i) {
+        min_kx = std::min(min_kx, prm.p[i].d_in / kChunkCols);
+        tiles += ceil_div64(N, kTileM);
+    }
+    int split = 1;
+    const char* env = getenv("MOLORA_UMMA_SPLIT");          // tuning override
+    if (env != nullptr) split = std::min(atoi(env), kMaxSplit);
+    else while (split < 4 && tiles * split * 2 <= 148) split *= 2;
+    while (split > 1 && min_kx / split < 4) split /= 2;
+    return split < 1 ? 1 : split;
 }
 
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
@@ -428,10 +611,14 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
     prm.P = P;
     prm.C = C;
     prm.min_rows = min_rows;
+#ifdef MOLORA_TRACE
+    prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
+#endif
+    const int split = choose_split(prm, N);
     cudaError_t e = cudaSuccess;
-    if (has[0] && e == cudaSuccess) e = umma_launch<16>(prm, N, s);
-    if (has[1] && e == cudaSuccess) e = umma_launch<32>(prm, N, s);
-    if (has[2] && e == cudaSuccess) e = umma_launch<64>(prm, N, s);
+    if (has[0] && e == cudaSuccess) e = umma_launch<16>(prm, N, split, s);
+    if (has[1] && e == cudaSuccess) e = umma_launch<32>(prm, N, split, s);
+    if (has[2] && e == cudaSuccess) e = umma_launch<64>(prm, N, split, s);
     return cuda_ok(e);
 }
 
