@@ -124,8 +124,8 @@ static_assert(sizeof(Ctrl) <= 1024, "control block must fit its slot");
 // Bounded wait on an mbarrier phase.  Falls through once the CTA has aborted.
 __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* dev_status)
 {
-    if (*abort_flag) return;
     if (mbar_try_wait(bar, parity)) return;
+    if (*abort_flag) return;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (*abort_flag) return;
@@ -141,8 +141,8 @@ __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile
 __device__ __forceinline__ void wait_bar_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                  uint32_t* dev_status)
 {
-    if (*abort_flag) return;
     if (mbar_try_wait_cluster(bar, parity)) return;
+    if (*abort_flag) return;
     const long long t0 = clock64();
     while (!mbar_try_wait_cluster(bar, parity)) {
         if (*abort_flag) return;
@@ -428,6 +428,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 
         // copy-out mapping: piece (et & 7) of rows (et >> 3) + 16 i
         const int piece = et & 7;
+        int otok[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) otok[i] = ctrl->rows[(et >> 3) + 16 * i];
         for (int nc = group; nc < NY; nc += kEpiGroups) {
             const int it = KX + nc;
             const int s = it % Cfg::kStages;
@@ -446,35 +449,35 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             if (et == 0) MOLORA_TR(2, it, 2);
             wait_bar(bar(&ctrl->full[s]), ph, abort_flag, prm.dev_status);   // the Y chunk of this stage has landed
             if (et == 0) MOLORA_TR(2, it, 3);
-            const uint32_t ytile = stage(s);
+            uint8_t* ytile = smem_raw + (stage(s) - raw);
+            {
+                uint4 yp[8];
 #pragma unroll
-            for (int c8 = 0; c8 < 8; ++c8) {
-                const uint32_t addr = ytile + swizzle_offset((uint32_t)row * 128u + c8 * 16, 3);
-                uint4 v;
-                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-                float yv[8];
-                unpack<__nv_bfloat16>(v, yv);
+                for (int c8 = 0; c8 < 8; ++c8)
+                    yp[c8] = *reinterpret_cast<const uint4*>(ytile + swizzle_offset((uint32_t)row * 128u + c8 * 16, 3));
 #pragma unroll
-                for (int e = 0; e < 8; ++e) yv[e] += __uint_as_float(dv[c8 * 8 + e]);
-                v = pack<__nv_bfloat16>(yv);
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    float yv[8];
+                    unpack<__nv_bfloat16>(yp[c8], yv);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) yv[e] += __uint_as_float(dv[c8 * 8 + e]);
+                    *reinterpret_cast<uint4*>(ytile + swizzle_offset((uint32_t)row * 128u + c8 * 16, 3)) =
+                        pack<__nv_bfloat16>(yv);
+                }
             }
             if (et == 0) MOLORA_TR(2, it, 4);
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
             if (et == 0) MOLORA_TR(2, it, 5);
             if (!*abort_flag) {
                 __nv_bfloat16* dstc = pj.y + (ny0 + nc) * kChunkCols + piece * 8;
+                uint4 op[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int r = (et >> 3) + 16 * i;
-                    const int tok = ctrl->rows[r];
-                    if (tok >= 0) {
-                        const uint32_t addr = ytile + swizzle_offset((uint32_t)r * 128u + piece * 16, 3);
-                        uint4 v;
-                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-                        stg128(dstc + (int64_t)tok * pj.ldy, v);
-                    }
-                }
+                for (int i = 0; i < 8; ++i)
+                    op[i] = *reinterpret_cast<const uint4*>(
+                        ytile + swizzle_offset((uint32_t)((et >> 3) + 16 * i) * 128u + piece * 16, 3));
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (otok[i] >= 0) stg128(dstc + (int64_t)otok[i] * pj.ldy, op[i]);
             }
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
             if (et == 0) mbar_arrive(bar(&ctrl->empty[s]));   // the stage may be refilled
@@ -533,6 +536,22 @@ bool umma_eligible(const molora_proj_desc_t& p, molora_dtype_t dt)
 }
 
 template <int R>
+static void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int64_t tiles, int P, int split,
+                               cudaStream_t s)
+{
+    cfg.gridDim = dim3((unsigned)(tiles * split), (unsigned)P, 1);
+    cfg.blockDim = dim3(kUmmaThreads, 1, 1);
+    cfg.dynamicSmemBytes = UmmaCfg<R>::kSmemBytes;
+    cfg.stream = s;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+}
+
+template <int R>
 static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, int split, cudaStream_t s)
 {
     using Cfg = UmmaCfg<R>;
@@ -545,37 +564,56 @@ static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, int split, cuda
     }
     const int64_t tiles = ceil_div64(N, kTileM) + prm.C;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(tiles * split), (unsigned)prm.P, 1);
-    cfg.blockDim = dim3(kUmmaThreads, 1, 1);
-    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
-    cfg.stream = s;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)split;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    fill_launch_config<R>(cfg, attr, tiles, prm.P, split, s);
     return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R>, prm);
 }
 
-// CTAs per tile.  Tiles are 128 rows, so small calls have too few of them for 148 SMs: split each tile over a
-// cluster of 2 or 4 CTAs while that still fits in one wave, keeping at least four 64-column chunks of d_in
-// per CTA.  (Clusters of 8 leave SMs of a GPC idle and their exchange costs more than it returns.)
-static int choose_split(const UmmaParams& prm, int64_t N)
+// Clusters of `split` CTAs of this kernel that can be resident at once (cached per rank and split).
+template <int R>
+static int max_active_clusters(int split)
+{
+    static int cache[kMaxSplit + 1] = {0, 0, 0, 0, 0};
+    if (cache[split] == 0) {
+        cudaFuncSetAttribute(apply_umma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<R>::kSmemBytes);
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        fill_launch_config<R>(cfg, attr, 148, 1, split, nullptr);
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, apply_umma_kernel<R>, &cfg) != cudaSuccess || n <= 0) n = 148 / split;
+        cache[split] = n;
+    }
+    return cache[split];
+}
+
+// CTAs per tile.  Tiles are 128 rows, so small calls have too few of them for 148 SMs; a tile can be split over
+// a cluster of 2 or 4 CTAs.  Pick the split with the smallest estimated time: waves of resident clusters times
+// (work per CTA, which shrinks with the split, plus a fixed per-CTA cost and the cost of the exchange).
+template <int R>
+static int choose_split_for_rank(const UmmaParams& prm, int64_t N)
 {
     int min_kx = INT32_MAX;
     int64_t tiles = 0;
     for (int i = 0; i < prm.P; ++i) {
+        if (prm.p[i].rank != R) continue;
         min_kx = std::min(min_kx, prm.p[i].d_in / kChunkCols);
-        tiles += ceil_div64(N, kTileM);
+        tiles += ceil_div64(N, kTileM) + prm.C / 2;           // expected: every segment ends in a partial tile
     }
-    int split = 1;
     const char* env = getenv("MOLORA_UMMA_SPLIT");          // tuning override
-    if (env != nullptr) split = std::min(atoi(env), kMaxSplit);
-    else while (split < 4 && tiles * split * 2 <= 148) split *= 2;
-    while (split > 1 && min_kx / split < 4) split /= 2;
-    return split < 1 ? 1 : split;
+    int best = 1;
+    if (env != nullptr) {
+        best = std::max(1, std::min(atoi(env), kMaxSplit));
+    } else {
+        double best_cost = 1e30;
+        for (int split = 1; split <= kMaxSplit; split *= 2) {
+            const int resident = max_active_clusters<R>(split);
+            const double waves = (double)((tiles + resident - 1) / resident);
+            const double cost = waves * (1.0 / split + 0.15 + (split > 1 ? 0.10 : 0.0));
+            if (cost < best_cost - 1e-9) { best_cost = cost; best = split; }
+        }
+    }
+    while (best > 1 && min_kx / best < 4) best /= 2;         // keep at least four chunks of d_in per CTA
+    return best;
 }
 
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
@@ -614,11 +652,10 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
 #ifdef MOLORA_TRACE
     prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
 #endif
-    const int split = choose_split(prm, N);
     cudaError_t e = cudaSuccess;
-    if (has[0] && e == cudaSuccess) e = umma_launch<16>(prm, N, split, s);
-    if (has[1] && e == cudaSuccess) e = umma_launch<32>(prm, N, split, s);
-    if (has[2] && e == cudaSuccess) e = umma_launch<64>(prm, N, split, s);
+    if (has[0] && e == cudaSuccess) e = umma_launch<16>(prm, N, choose_split_for_rank<16>(prm, N), s);
+    if (has[1] && e == cudaSuccess) e = umma_launch<32>(prm, N, choose_split_for_rank<32>(prm, N), s);
+    if (has[2] && e == cudaSuccess) e = umma_launch<64>(prm, N, choose_split_for_rank<64>(prm, N), s);
     return cuda_ok(e);
 }
 
