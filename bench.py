@@ -133,7 +133,12 @@ def build_sets(W, torch, name, n_sets, rank):
             "ids": dev(w.ids, "i") if w.ids is not None else None,
             "r_given": dev(w.r, "i") if w.r is not None else None,
         })
-    shared = {"status": torch.zeros(1, dtype=torch.int32, device="cuda"),
+    gate_ws = None
+    if w0.G is not None:
+        import paper_2603_15965_b200 as M
+        need = M.molora_route_gate_workspace_bytes(1 if w0.dtype == "bf16" else 0, w0.G.shape[0], w0.G.shape[1])
+        gate_ws = torch.empty(need, dtype=torch.uint8, device="cuda") if need else None
+    shared = {"status": torch.zeros(1, dtype=torch.int32, device="cuda"), "gate_ws": gate_ws,
               "G": dev(w0.G, "f32") if w0.G is not None else None,
               "breaks": dev(w0.breaks, "i") if w0.breaks is not None else None}
     return w0, sets, shared
@@ -149,8 +154,11 @@ def marshal_step(lib, w, s, shared, stream_handle):
     route = None
     if w.router == "gate":
         x = s["x"][w.gate_x_key]
+        gws = shared["gate_ws"]
         route = partial(lib.molora_route_gate, vp(x.data_ptr()), 1 if w.dtype == "bf16" else 0, i64(N), i32(x.shape[1]),
-                        i64(x.stride(0)), vp(shared["G"].data_ptr()), None, i32(C), vp(s["r"].data_ptr()), None, st)
+                        i64(x.stride(0)), vp(shared["G"].data_ptr()), None, i32(C), vp(s["r"].data_ptr()), None,
+                        vp(gws.data_ptr()) if gws is not None else None,
+                        ctypes.c_size_t(gws.numel() if gws is not None else 0), st)
         r = s["r"]
     elif w.router == "vocab":
         route = partial(lib.molora_route_vocab, vp(s["ids"].data_ptr()), i64(N), vp(shared["breaks"].data_ptr()),
@@ -209,7 +217,8 @@ def run_ours(args):
         s["perm"] = torch.empty(N, dtype=torch.int32, device="cuda")
         s["packed"] = pack_proj_descs([M.ProjDesc(s["x"][p.x_key], y, A, B, 1.0) for p, y, A, B in
                                                  zip(w.projections, s["y"], s["A"], s["B"])])
-    launches_per_step = (0 if w.router == "given" else 1) + 1 + len({p.rank for p in w.projections})
+    gate_launches = 0 if w.router == "given" else (2 if (w.router == "gate" and shared["gate_ws"] is not None) else 1)
+    launches_per_step = gate_launches + 1 + len({p.rank for p in w.projections})
     for s in sets:
         s["calls"] = marshal_step(lib, w, s, shared, stream.cuda_stream)
 
@@ -325,7 +334,7 @@ def run_e2e(args, torch, M, w, sets, shared, world, dist):
         if hr is not None:
             s["r_given"].copy_(hr, non_blocking=True)
         if w.router == "gate":
-            M.molora_route_gate(s["x"][w.gate_x_key], shared["G"], r_out=s["r"])
+            M.molora_route_gate(s["x"][w.gate_x_key], shared["G"], r_out=s["r"], ws=shared["gate_ws"])
             r = s["r"]
         elif w.router == "vocab":
             M.molora_route_vocab(s["ids"], shared["breaks"], r_out=s["r"])

@@ -81,12 +81,17 @@ molora_status_t molora_route_vocab(const int32_t *ids, int64_t N, const int32_t 
  * Theorem 3.4 / Table 10).  Softmax is monotone and the weight of a single kept logit is 1, so
  *     z[i][c] = sum_k x[i][k] * G[k][c] (+ bias[c]),    r_out[i] = argmax_c z[i][c]  (lowest c on ties).
  * x        device [N, d] of type xdt, row pitch ldx >= d elements; d a multiple of 8; never written
- * G        device fp32 [d, C] row-major (gate weights);  bias  device fp32 [C] or NULL;  1 <= C <= 64
+ * G        device fp32 [d, C] row-major (gate weights);  bias  device fp32 [C] or NULL;  1 <= C <= 32
  * r_out    device int32[N]
  * logits_out  device fp32 [N, C] or NULL (the logits as the kernel accumulated them, fp32)
+ * ws, ws_bytes  device scratch of at least molora_route_gate_workspace_bytes(xdt, d, C) bytes, 16-byte aligned
+ *               (NULL when that is 0).  For bf16 x and C > 8 the kernel runs on the tensor cores and keeps there a
+ *               three-term bf16 split of G (hi + mid + lo = 24 mantissa bits), rebuilt on every call.
  * Products are exact in fp32 for bf16 x; accumulation is fp32 in a fixed, token-independent order. */
+size_t molora_route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
 molora_status_t molora_route_gate(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float *G,
-                                  const float *bias, int32_t C, int32_t *r_out, float *logits_out, void *stream);
+                                  const float *bias, int32_t C, int32_t *r_out, float *logits_out, void *ws,
+                                  size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Grouping (Section 3.3 steps 1-3; Algorithm 2; Table 10 "histogram"):

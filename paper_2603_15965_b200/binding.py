@@ -64,7 +64,9 @@ def load_library():
     lib.molora_status_string.restype = ctypes.c_char_p
     lib.molora_status_string.argtypes = [ctypes.c_int]
     lib.molora_route_vocab.argtypes = [vp, i64, vp, i32, vp, vp, vp]
-    lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp]
+    lib.molora_route_gate_workspace_bytes.restype = sz
+    lib.molora_route_gate_workspace_bytes.argtypes = [ctypes.c_int, i32, i32]
+    lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp]
     lib.molora_group_workspace_bytes.restype = sz
     lib.molora_group_workspace_bytes.argtypes = [i64, i32]
     lib.molora_group.argtypes = [vp, i64, i32, vp, vp, vp, vp, sz, vp, vp]
@@ -139,9 +141,13 @@ def molora_route_vocab(ids: torch.Tensor, breaks: torch.Tensor, r_out: Optional[
     return r_out
 
 
+def molora_route_gate_workspace_bytes(xdt: int, d: int, C: int) -> int:
+    return int(load_library().molora_route_gate_workspace_bytes(xdt, d, C))
+
+
 def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Tensor] = None,
                       r_out: Optional[torch.Tensor] = None, logits_out: Optional[torch.Tensor] = None,
-                      stream=None) -> torch.Tensor:
+                      ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """r_out[i] = argmax_c sum_k x[i,k] G[k,c] (+ bias[c]) (Eq. 8, k = 1); lowest index on ties."""
     lib = load_library()
     N, d, ldx = _matrix(x, "x")
@@ -155,9 +161,13 @@ def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Ten
     if logits_out is not None and (logits_out.dtype != torch.float32 or logits_out.shape != (N, C)
                                    or not logits_out.is_contiguous()):
         raise ValueError("logits_out: expected contiguous fp32 [N, C]")
+    need = molora_route_gate_workspace_bytes(_dtype_code(x), d, C)
+    if ws is None and need > 0:
+        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_route_gate", lib.molora_route_gate(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(G), _ptr(bias), C,
-                                                      _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
-                                                      _stream(stream)))
+                                                      _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out), _ptr(ws),
+                                                      ws_bytes, _stream(stream)))
     return r_out
 
 

@@ -48,15 +48,24 @@ molora_status_t molora_route_vocab(const int32_t* ids, int64_t N, const int32_t*
     return launch_route_vocab(ids, N, breaks, M, r_out, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+size_t molora_route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
+{
+    if (d <= 0 || C < 1 || C > 32) return 0;
+    return route_gate_workspace_bytes(xdt, d, C);
+}
+
 molora_status_t molora_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
-                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* stream)
+                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
+                                  size_t ws_bytes, void* stream)
 {
     if (N < 0 || N >= INT32_MAX || d <= 0 || C < 1) return MOLORA_ERR_INVALID_ARG;
     if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
     if (C > 32 || (d % 8) != 0 || (ldx % 8) != 0) return MOLORA_ERR_UNSUPPORTED;
     if (ldx < d || G == nullptr) return MOLORA_ERR_INVALID_ARG;
     if (N > 0 && (x == nullptr || r_out == nullptr || !aligned16(x))) return MOLORA_ERR_INVALID_ARG;
-    return launch_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, static_cast<cudaStream_t>(stream));
+    const size_t need = route_gate_workspace_bytes(xdt, d, C);
+    if (need > 0 && (ws == nullptr || ws_bytes < need || !aligned16(ws))) return MOLORA_ERR_WORKSPACE;
+    return launch_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, ws, static_cast<cudaStream_t>(stream));
 }
 
 size_t molora_group_workspace_bytes(int64_t N, int32_t C) { return group_workspace_bytes(N, C); }
@@ -104,8 +113,12 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
     }
     molora_status_t st = MOLORA_OK;
     if (n_tc > 0) {
-        st = launch_apply_umma(tc, n_tc, N, C, offsets, perm, dev_status, kUmmaMinRows, s);
-        if (st == MOLORA_OK) st = launch_apply_rowtile(tc, n_tc, dt, N, C, offsets, perm, kUmmaMinRows, s);
+        // With few adapters an under-filled 128-row tile is cheap, so the tensor-core kernel takes every segment
+        // and the second launch is saved; with many adapters (up to 256 composite targets) tiny segments are
+        // the norm and go to the CUDA-core kernel instead.
+        const int32_t min_rows = C <= kUmmaAllSegmentsMaxC ? 1 : kUmmaMinRows;
+        st = launch_apply_umma(tc, n_tc, N, C, offsets, perm, dev_status, min_rows, s);
+        if (st == MOLORA_OK && min_rows > 1) st = launch_apply_rowtile(tc, n_tc, dt, N, C, offsets, perm, min_rows, s);
     }
     if (st == MOLORA_OK && n_cc > 0) st = launch_apply_rowtile(cc, n_cc, dt, N, C, offsets, perm, INT32_MAX, s);
     return st;

@@ -130,8 +130,16 @@ __device__ __forceinline__ bool find_tile(const int32_t* __restrict__ offsets, i
 // Host launchers implemented in the .cu files (stream already unwrapped).
 molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M, int32_t* r_out,
                                    uint32_t* dev_status, cudaStream_t s);
+size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
 molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
-                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, cudaStream_t s);
+                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
+                                  cudaStream_t s);
+// Tensor-core (mma.sync) gate for bf16 activations; the CUDA-core kernel above serves fp32 activations.
+// Needs route_gate_mma_workspace_bytes(d, C) bytes of scratch for the split gate weights.
+size_t route_gate_mma_workspace_bytes(int32_t d, int32_t C);
+molora_status_t launch_route_gate_mma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
+                                      const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
+                                      cudaStream_t s);
 size_t group_workspace_bytes(int64_t N, int32_t C);
 molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
                              void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
@@ -149,6 +157,7 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
 // has at least kUmmaMinTokens tokens (known on the host); everything else runs on the CUDA-core kernel.
 constexpr int32_t kUmmaMinRows = 32;
 constexpr int64_t kUmmaMinTokens = 1024;
+constexpr int32_t kUmmaAllSegmentsMaxC = 64;   // up to this many adapters the tensor-core kernel takes all segments
 
 inline molora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? MOLORA_OK : MOLORA_ERR_CUDA; }
 

@@ -152,6 +152,138 @@ __global__ void __launch_bounds__(256) route_gate_kernel(const T* __restrict__ x
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Linear gate, few adapters (C <= 8) and d * CP * 4 bytes of G small enough to stay resident in shared
+// memory: no per-chunk staging and no block-wide synchronisation inside the token loop.  A CTA of four
+// warps copies G once (skewed per lane as above); then each warp streams its tokens two at a time with all
+// of their 16-byte loads issued before the first FMA, which keeps ~8 KB per warp in flight.
+// ------------------------------------------------------------------------------------------------
+template <typename T, int CP>
+__global__ void __launch_bounds__(128) route_gate_resident_kernel(const T* __restrict__ x, int64_t N, int d, int64_t ldx,
+                                                                  const float* __restrict__ G,
+                                                                  const float* __restrict__ bias, int C,
+                                                                  int32_t* __restrict__ r_out,
+                                                                  float* __restrict__ logits_out, int tokens_per_warp)
+{
+    constexpr int VEC = VecTraits<T>::kElems;
+    constexpr int KC = 32 * VEC;
+    constexpr int LANE_STRIDE = VEC * CP + 4;
+    constexpr int BATCH = 8;                       // 16-byte vectors per token kept in flight per lane
+    extern __shared__ __align__(16) float Gres[];  // [chunks][32 lanes][LANE_STRIDE]
+    const int chunks = (d + KC - 1) / KC;
+    for (int e = threadIdx.x; e < chunks * KC * CP; e += blockDim.x) {
+        const int k = e / CP, c = e - k * CP;
+        const float g = (k < d && c < C) ? __ldg(G + (int64_t)k * C + c) : 0.f;
+        const int ch = k / KC, kk = k - ch * KC;
+        Gres[(ch * 32 + kk / VEC) * LANE_STRIDE + (kk % VEC) * CP + c] = g;
+    }
+    __syncthreads();
+
+    const int warp = threadIdx.x >> 5, lane = lane_id();
+    const int64_t wtok0 = ((int64_t)blockIdx.x * 4 + warp) * tokens_per_warp;
+    for (int t0 = 0; t0 < tokens_per_warp; t0 += 2) {
+        const int64_t i0 = wtok0 + t0;
+        if (i0 >= N) break;
+        const int64_t i1 = i0 + 1 < N && t0 + 1 < tokens_per_warp ? i0 + 1 : i0;
+        const T* x0 = x + i0 * ldx + lane * VEC;
+        const T* x1 = x + i1 * ldx + lane * VEC;
+        float acc[2][CP];
+#pragma unroll
+        for (int c = 0; c < CP; ++c) acc[0][c] = acc[1][c] = 0.f;
+        for (int cb = 0; cb < chunks; cb += BATCH) {
+            uint4 v0[BATCH], v1[BATCH];
+#pragma unroll
+            for (int b = 0; b < BATCH; ++b) {
+                const int k = (cb + b) * KC + lane * VEC;
+                if (k < d) {
+                    v0[b] = ldg128_stream(x0 + (cb + b) * KC);
+                    v1[b] = ldg128_stream(x1 + (cb + b) * KC);
+                } else {
+                    v0[b] = make_uint4(0, 0, 0, 0);
+                    v1[b] = make_uint4(0, 0, 0, 0);
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < BATCH; ++b) {
+                if (cb + b < chunks) {
+                    float f0[VEC], f1[VEC];
+                    unpack<T>(v0[b], f0);
+                    unpack<T>(v1[b], f1);
+                    const float* g = Gres + ((cb + b) * 32 + lane) * LANE_STRIDE;
+#pragma unroll
+                    for (int j = 0; j < VEC; ++j) {
+#pragma unroll
+                        for (int c4 = 0; c4 < CP; c4 += 4) {
+                            const float4 gv = *reinterpret_cast<const float4*>(g + j * CP + c4);
+                            acc[0][c4 + 0] = fmaf(f0[j], gv.x, acc[0][c4 + 0]);
+                            acc[0][c4 + 1] = fmaf(f0[j], gv.y, acc[0][c4 + 1]);
+                            acc[0][c4 + 2] = fmaf(f0[j], gv.z, acc[0][c4 + 2]);
+                            acc[0][c4 + 3] = fmaf(f0[j], gv.w, acc[0][c4 + 3]);
+                            acc[1][c4 + 0] = fmaf(f1[j], gv.x, acc[1][c4 + 0]);
+                            acc[1][c4 + 1] = fmaf(f1[j], gv.y, acc[1][c4 + 1]);
+                            acc[1][c4 + 2] = fmaf(f1[j], gv.z, acc[1][c4 + 2]);
+                            acc[1][c4 + 3] = fmaf(f1[j], gv.w, acc[1][c4 + 3]);
+                        }
+                    }
+                }
+            }
+        }
+        // finish both tokens' logits: plain butterfly sums (2 * CP values, small next to the d / 32 FMAs per lane)
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int c = 0; c < CP; ++c) {
+                float v = acc[t][c];
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, off);
+                acc[t][c] = v;
+            }
+        if (lane < 2) {
+            const int64_t i = lane == 0 ? i0 : i1;
+            if (lane == 0 || i1 != i0) {
+                float best = 0.f;
+                int arg = 0;
+#pragma unroll
+                for (int c = 0; c < CP; ++c) {
+                    if (c < C) {
+                        float z = lane == 0 ? acc[0][c] : acc[1][c];
+                        if (bias != nullptr) z += __ldg(bias + c);
+                        if (logits_out != nullptr) logits_out[i * C + c] = z;
+                        if (c == 0 || z > best) { best = z; arg = c; }
+                    }
+                }
+                r_out[i] = arg;
+            }
+        }
+    }
+}
+
+template <typename T, int CP>
+static molora_status_t gate_resident_launch(const void* x, int64_t N, int d, int64_t ldx, const float* G,
+                                            const float* bias, int C, int32_t* r_out, float* logits_out,
+                                            cudaStream_t s, bool& handled)
+{
+    constexpr int VEC = VecTraits<T>::kElems;
+    const int chunks = (d + 32 * VEC - 1) / (32 * VEC);
+    const size_t smem = (size_t)chunks * 32 * (VEC * CP + 4) * sizeof(float);
+    handled = smem <= 96 * 1024;
+    if (!handled) return MOLORA_OK;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(route_gate_resident_kernel<T, CP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 96 * 1024) != cudaSuccess)
+            return MOLORA_ERR_CUDA;
+        configured = true;
+    }
+    // tokens per warp: 8 when that still gives at least ~one CTA per SM, otherwise fewer (small calls)
+    int tpw = 8;
+    while (tpw > 2 && ceil_div64(N, 4 * tpw) < 148) tpw /= 2;
+    const int64_t blocks = ceil_div64(N, 4 * tpw);
+    route_gate_resident_kernel<T, CP><<<(unsigned)blocks, 128, smem, s>>>(static_cast<const T*>(x), N, d, ldx, G, bias,
+                                                                         C, r_out, logits_out, tpw);
+    return cuda_ok(cudaGetLastError());
+}
+
 template <typename T, int CP, int TOK>
 static molora_status_t gate_launch(const void* x, int64_t N, int d, int64_t ldx, const float* G, const float* bias,
                                    int C, int32_t* r_out, float* logits_out, cudaStream_t s)
@@ -166,16 +298,30 @@ template <typename T>
 static molora_status_t gate_dispatch(const void* x, int64_t N, int d, int64_t ldx, const float* G, const float* bias,
                                      int C, int32_t* r_out, float* logits_out, cudaStream_t s)
 {
+    if (C <= 8) {   // few adapters: G stays resident in shared memory when it fits
+        bool handled = false;
+        const molora_status_t st =
+            C <= 4 ? gate_resident_launch<T, 4>(x, N, d, ldx, G, bias, C, r_out, logits_out, s, handled)
+                   : gate_resident_launch<T, 8>(x, N, d, ldx, G, bias, C, r_out, logits_out, s, handled);
+        if (handled || st != MOLORA_OK) return st;
+    }
     if (C <= 4) return gate_launch<T, 4, 4>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
     if (C <= 8) return gate_launch<T, 8, 4>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
     if (C <= 16) return gate_launch<T, 16, 4>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
     return gate_launch<T, 32, 2>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);   // C <= 32 checked by the caller
 }
 
+size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
+{
+    return xdt == MOLORA_BF16 ? route_gate_mma_workspace_bytes(d, C) : 0;
+}
+
 molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
-                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, cudaStream_t s)
+                                  const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
+                                  cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
+    if (xdt == MOLORA_BF16 && C > 8) return launch_route_gate_mma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
     if (xdt == MOLORA_BF16) return gate_dispatch<__nv_bfloat16>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
     return gate_dispatch<float>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
 }

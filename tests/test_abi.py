@@ -11,7 +11,8 @@ def test_library_builds_loads_and_exports_header_symbols():
     lib = M.load_library()
     names = M.exported_symbols()
     assert {"molora_route_vocab", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched",
-            "molora_group_workspace_bytes", "molora_apply_workspace_bytes", "molora_version",
+            "molora_group_workspace_bytes", "molora_apply_workspace_bytes", "molora_route_gate_workspace_bytes",
+            "molora_version",
             "molora_status_string"} <= set(names)
     for name in names:
         assert hasattr(lib, name), f"header declares {name} but the library does not export it"
@@ -29,9 +30,12 @@ def test_invalid_arguments_are_refused_before_any_launch():
     # too many ranges
     assert lib.molora_route_vocab(fake, 4, fake, 257, fake, None, None) == 2
     # gate: d not a multiple of 8, C too large, pitch too small
-    assert lib.molora_route_gate(fake, M.BF16, 4, 12, 16, fake, None, 4, fake, None, None) == 2
-    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 33, fake, None, None) == 2
-    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 8, fake, None, 4, fake, None, None) == 1
+    assert lib.molora_route_gate(fake, M.BF16, 4, 12, 16, fake, None, 4, fake, None, None, 0, None) == 2
+    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 33, fake, None, None, 0, None) == 2
+    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 8, fake, None, 4, fake, None, None, 0, None) == 1
+    # tensor-core gate (bf16, C > 8) without its workspace
+    assert M.molora_route_gate_workspace_bytes(M.BF16, 4096, 16) > 0 and M.molora_route_gate_workspace_bytes(M.BF16, 2048, 4) == 0
+    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 16, fake, None, None, 0, None) == 3
     # group: C out of range, null outputs
     assert lib.molora_group(fake, 4, 0, fake, fake, fake, None, 0, None, None) == 1
     assert lib.molora_group(fake, 4, 300, fake, fake, fake, None, 0, None, None) == 2
