@@ -2,34 +2,60 @@
 // segment offsets, STABLE permutation.  The paper allocates positions with atomicAdd, which leaves the
 // order inside a group to the hardware; here every position is computed from warp ballots/matches and
 // prefix sums only, so counts, offsets and perm are unique and bit-reproducible.
+//
+// One launch: a thread-block cluster of S <= 8 CTAs (1024 threads each) splits the tokens into S * 32
+// contiguous warp ranges, so "CTA rank, then warp, then iteration, then lane" is ascending token order.
+//   1. hist[w][c]  = tokens of adapter c in warp w's range (equal adapters of a 32-token step are grouped
+//                    by ballot / match; the lowest lane of a group adds its size -- distinct addresses,
+//                    no atomics)
+//   2. hist[w][c] <- exclusive prefix over the CTA's warps; tot[c] = the CTA's histogram
+//   3. hardware cluster barrier; every CTA reads all S histograms through distributed shared memory:
+//      counts[c] = their sum, lower[c] = sum over lower-ranked CTAs, seg[c] = exclusive prefix of counts
+//   4. second walk: position = seg[c] + lower[c] + hist[w][c] + (rank of the lane inside its group);
+//      the group leader then advances hist[w][c].
+// A final cluster barrier keeps every CTA's shared memory alive until all peers have read it.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace molora {
 
+using namespace ptx;
+
 constexpr int kGroupThreads = 1024;
 constexpr int kGroupWarps = kGroupThreads / 32;
+constexpr int kGroupMaxCluster = 8;
 
-// One CTA, three phases in shared memory.  Warp w owns the contiguous token range
-// [w*chunk, (w+1)*chunk) and walks it 32 tokens at a time, so "warp index, then iteration, then lane"
-// is ascending token order:
-//   1. hist[w][c]  = tokens of adapter c in warp w's range (match_any groups equal adapters in a step;
-//                    the lowest lane of each group adds the group's size -- distinct addresses, no atomics)
-//   2. hist[w][c] <- exclusive prefix over w;  seg[c] = exclusive prefix of the totals over c
-//   3. second walk: position = seg[c] + hist[w][c] + (rank of the lane inside its match group);
-//      the group leader then advances hist[w][c] by the group's size.
-__global__ void __launch_bounds__(kGroupThreads) group_single_cta_kernel(const int32_t* __restrict__ r, int64_t N,
-                                                                         int C, int32_t* __restrict__ counts,
-                                                                         int32_t* __restrict__ offsets,
-                                                                         int32_t* __restrict__ perm,
-                                                                         uint32_t* dev_status)
+// Lanes that hold the same routed adapter as this lane (0 for unrouted lanes are never used).
+__device__ __forceinline__ unsigned peers_of(int v, bool routed, int C)
+{
+    if (C <= 8) {   // a few ballots are cheaper than a match
+        unsigned mine = 0;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, routed && v == c);
+            if (v == c) mine = m;
+        }
+        return mine;
+    }
+    return __match_any_sync(0xFFFFFFFFu, routed ? v : -1);
+}
+
+__global__ void __launch_bounds__(kGroupThreads) group_cluster_kernel(const int32_t* __restrict__ r, int64_t N, int C,
+                                                                     int32_t* __restrict__ counts,
+                                                                     int32_t* __restrict__ offsets,
+                                                                     int32_t* __restrict__ perm, uint32_t* dev_status)
 {
     __shared__ int hist[kGroupWarps][MOLORA_MAX_ADAPTERS];
-    __shared__ int seg[MOLORA_MAX_ADAPTERS + 1];
+    __shared__ int tot[MOLORA_MAX_ADAPTERS];          // this CTA's histogram (read by the peers)
+    __shared__ int seg[MOLORA_MAX_ADAPTERS + 1];      // global exclusive prefix of counts
+    __shared__ int lower[MOLORA_MAX_ADAPTERS];        // tokens of adapter c in lower-ranked CTAs
     const int warp = threadIdx.x >> 5, lane = lane_id();
     const unsigned lt_mask = (1u << lane) - 1u;
+    const uint32_t S = cluster_nctarank(), crank = cluster_ctarank();
 
-    const int64_t chunk = ceil_div64(ceil_div64(N, kGroupWarps), 32) * 32;
-    const int64_t begin = (int64_t)warp * chunk;
+    const int64_t chunk = ceil_div64(ceil_div64(N, (int64_t)S * kGroupWarps), 32) * 32;
+    const int64_t begin0 = ((int64_t)crank * kGroupWarps + warp) * chunk;
+    const int64_t begin = begin0 < N ? begin0 : N;
     const int64_t end = begin + chunk < N ? begin + chunk : N;
 
     for (int c = lane; c < C; c += 32) hist[warp][c] = 0;
@@ -41,13 +67,13 @@ __global__ void __launch_bounds__(kGroupThreads) group_single_cta_kernel(const i
         const int v = i < end ? __ldg(r + i) : -1;
         const bool routed = v >= 0 && v < C;
         bad |= (v < -1) || (v >= C);
-        const unsigned peers = __match_any_sync(0xFFFFFFFFu, routed ? v : -1);
+        const unsigned peers = peers_of(v, routed, C);
         if (routed && lane == __ffs(peers) - 1) hist[warp][v] += __popc(peers);
         __syncwarp();
     }
     __syncthreads();
 
-    // exclusive prefix over warps, per adapter; totals are the histogram
+    // exclusive prefix over this CTA's warps, per adapter; the totals are the CTA's histogram
     for (int c = threadIdx.x; c < C; c += kGroupThreads) {
         int run = 0;
 #pragma unroll 8
@@ -56,8 +82,26 @@ __global__ void __launch_bounds__(kGroupThreads) group_single_cta_kernel(const i
             hist[w][c] = run;
             run += t;
         }
-        counts[c] = run;
-        seg[c + 1] = run;   // shifted by one: turned into the inclusive prefix below
+        tot[c] = run;
+    }
+    if (S > 1) cluster_sync_all(); else __syncthreads();
+
+    // global histogram and the part that precedes this CTA
+    for (int c = threadIdx.x; c < C; c += kGroupThreads) {
+        int all = 0, low = 0;
+        if (S > 1) {
+            for (uint32_t q = 0; q < S; ++q) {
+                int t;
+                asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(t) : "r"(map_to_cta(smem_u32(&tot[c]), q)) : "memory");
+                all += t;
+                if (q < crank) low += t;
+            }
+        } else {
+            all = tot[c];
+        }
+        lower[c] = low;
+        seg[c + 1] = all;      // shifted by one: turned into the prefix below
+        if (crank == 0) counts[c] = all;
     }
     __syncthreads();
 
@@ -87,16 +131,17 @@ __global__ void __launch_bounds__(kGroupThreads) group_single_cta_kernel(const i
         }
     }
     __syncthreads();
-    for (int c = threadIdx.x; c <= C; c += kGroupThreads) offsets[c] = seg[c];
+    if (crank == 0)
+        for (int c = threadIdx.x; c <= C; c += kGroupThreads) offsets[c] = seg[c];
 
     // stable scatter
     for (int64_t i0 = begin; i0 < end; i0 += 32) {
         const int64_t i = i0 + lane;
         const int v = i < end ? __ldg(r + i) : -1;
         const bool routed = v >= 0 && v < C;
-        const unsigned peers = __match_any_sync(0xFFFFFFFFu, routed ? v : -1);
+        const unsigned peers = peers_of(v, routed, C);
         if (routed) {
-            const int pos = seg[v] + hist[warp][v] + __popc(peers & lt_mask);
+            const int pos = seg[v] + lower[v] + hist[warp][v] + __popc(peers & lt_mask);
             perm[pos] = (int32_t)i;
         }
         __syncwarp();
@@ -104,6 +149,7 @@ __global__ void __launch_bounds__(kGroupThreads) group_single_cta_kernel(const i
         __syncwarp();
     }
     if (dev_status != nullptr && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(dev_status, MOLORA_DEV_BAD_ROUTE);
+    if (S > 1) cluster_sync_all();    // peers may still be reading tot[]
 }
 
 size_t group_workspace_bytes(int64_t /*N*/, int32_t /*C*/) { return 0; }
@@ -111,8 +157,22 @@ size_t group_workspace_bytes(int64_t /*N*/, int32_t /*C*/) { return 0; }
 molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
                              void* /*ws*/, size_t /*ws_bytes*/, uint32_t* dev_status, cudaStream_t s)
 {
-    group_single_cta_kernel<<<1, kGroupThreads, 0, s>>>(r, N, C, counts, offsets, perm, dev_status);
-    return cuda_ok(cudaGetLastError());
+    // one CTA per ~1024 tokens (one 32-token step per warp), at most 8 CTAs
+    int split = 1;
+    while (split < kGroupMaxCluster && (int64_t)split * 1024 < N) split *= 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)split, 1, 1);
+    cfg.blockDim = dim3(kGroupThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cuda_ok(cudaLaunchKernelEx(&cfg, group_cluster_kernel, r, N, C, counts, offsets, perm, dev_status));
 }
 
 }  // namespace molora

@@ -171,11 +171,26 @@ __global__ void __launch_bounds__(128) route_gate_resident_kernel(const T* __res
     constexpr int BATCH = 8;                       // 16-byte vectors per token kept in flight per lane
     extern __shared__ __align__(16) float Gres[];  // [chunks][32 lanes][LANE_STRIDE]
     const int chunks = (d + KC - 1) / KC;
-    for (int e = threadIdx.x; e < chunks * KC * CP; e += blockDim.x) {
-        const int k = e / CP, c = e - k * CP;
-        const float g = (k < d && c < C) ? __ldg(G + (int64_t)k * C + c) : 0.f;
-        const int ch = k / KC, kk = k - ch * KC;
-        Gres[(ch * 32 + kk / VEC) * LANE_STRIDE + (kk % VEC) * CP + c] = g;
+    if (C == CP && (d % KC) == 0) {
+        // G rows are CP floats = whole 16-byte vectors: copy them as they are (coalesced float4 loads)
+        constexpr int V = CP / 4;
+        // (asynchronous 16-byte copies: all of a thread's requests are in flight at once)
+        for (int e = threadIdx.x; e < d * V; e += blockDim.x) {
+            const int k = e / V, v = e - k * V;
+            const int ch = k / KC, kk = k - ch * KC;
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(
+                &Gres[(ch * 32 + kk / VEC) * LANE_STRIDE + (kk % VEC) * CP + v * 4]);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(reinterpret_cast<const float4*>(G) + e)
+                         : "memory");
+        }
+        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+    } else {
+        for (int e = threadIdx.x; e < chunks * KC * CP; e += blockDim.x) {
+            const int k = e / CP, c = e - k * CP;
+            const float g = (k < d && c < C) ? __ldg(G + (int64_t)k * C + c) : 0.f;
+            const int ch = k / KC, kk = k - ch * KC;
+            Gres[(ch * 32 + kk / VEC) * LANE_STRIDE + (kk % VEC) * CP + c] = g;
+        }
     }
     __syncthreads();
 
@@ -321,7 +336,7 @@ molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, 
                                   cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
-    if (xdt == MOLORA_BF16 && C > 8) return launch_route_gate_mma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
+    if (xdt == MOLORA_BF16 && C > 4) return launch_route_gate_mma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
     if (xdt == MOLORA_BF16) return gate_dispatch<__nv_bfloat16>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
     return gate_dispatch<float>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
 }

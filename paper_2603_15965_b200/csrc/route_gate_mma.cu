@@ -81,7 +81,8 @@ __global__ void __launch_bounds__(WARPS * 32) route_gate_mma_kernel(const __nv_b
     constexpr int CP = Img::CP, ROW = Img::ROW;
     constexpr int THREADS = WARPS * 32;
     constexpr int NB = KC / 32;                                      // 32-wide k blocks per chunk
-    __shared__ __align__(16) __nv_bfloat16 Gs[2][3][CP][ROW];         // [buffer][term][c][k']
+    constexpr int IB = 3;                                            // weight-image buffers (two requests ahead)
+    __shared__ __align__(16) __nv_bfloat16 Gs[IB][3][CP][ROW];        // [buffer][term][c][k']
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, q = lane & 3;
@@ -97,20 +98,18 @@ __global__ void __launch_bounds__(WARPS * 32) route_gate_mma_kernel(const __nv_b
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[n][i] = 0.f;
 
+    const int chunks = (d + KC - 1) / KC;
     auto copy_image = [&](int buf, int ch) {
         const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&Gs[buf][0][0][0]);
         const char* src = reinterpret_cast<const char*>(img + (int64_t)ch * Img::kElems);
-        for (int o = tid * 16; o < Img::kBytes; o += THREADS * 16)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + o), "l"(src + o) : "memory");
-        asm volatile("cp.async.commit_group;" ::: "memory");
+        if (ch < chunks)
+            for (int o = tid * 16; o < Img::kBytes; o += THREADS * 16)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + o), "l"(src + o) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");         // an empty group keeps the group count uniform
     };
 
-    const int chunks = (d + KC - 1) / KC;
-    copy_image(0, 0);
-    for (int ch = 0; ch < chunks; ++ch) {
-        const int k0 = ch * KC;
-        // this chunk's activations: NB blocks of 32 k, two rows, 16 bytes each
-        uint4 va[NB], vb[NB];
+    // activations of one chunk: NB blocks of 32 k, two rows, 16 bytes each
+    auto load_x = [&](uint4 (&va)[NB], uint4 (&vb)[NB], int k0) {
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
             const int k = k0 + b * 32 + q * 8;
@@ -122,35 +121,53 @@ __global__ void __launch_bounds__(WARPS * 32) route_gate_mma_kernel(const __nv_b
                 vb[b] = make_uint4(0, 0, 0, 0);
             }
         }
-        if (ch + 1 < chunks) {
-            copy_image((ch + 1) & 1, ch + 1);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-        } else {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-        }
-        __syncthreads();                                             // image `ch` is complete for every thread
-        const int buf = ch & 1;
+    };
+
+    // Software pipeline: the activations of kDepth - 1 chunks ahead and the next weight image are requested
+    // before a chunk's math, so ~kDepth chunks (4 KB each per warp) are in flight.  The register ring is indexed
+    // statically by unrolling the chunk loop kDepth times.
+    constexpr int kDepth = 4;
+    copy_image(0, 0);
+    copy_image(1, 1);
+    uint4 va[kDepth][NB], vb[kDepth][NB];
 #pragma unroll
-        for (int b = 0; b < NB; ++b) {
+    for (int u = 0; u < kDepth - 1; ++u)
+        if (u < chunks) load_x(va[u], vb[u], u * KC);
+    for (int ch0 = 0; ch0 < chunks; ch0 += kDepth) {
 #pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                // A fragment of k-step (b, s): a0 = row g k-slots 2q,2q+1; a1 = row g+8; a2 = row g slots 2q+8,+9; a3
-                uint32_t a[4];
-                a[0] = s ? va[b].z : va[b].x;
-                a[2] = s ? va[b].w : va[b].y;
-                a[1] = s ? vb[b].z : vb[b].x;
-                a[3] = s ? vb[b].w : vb[b].y;
+        for (int u = 0; u < kDepth; ++u) {
+            const int ch = ch0 + u;
+            if (ch < chunks) {                                       // uniform over the CTA
+                if (ch + kDepth - 1 < chunks)
+                    load_x(va[(u + kDepth - 1) % kDepth], vb[(u + kDepth - 1) % kDepth], (ch + kDepth - 1) * KC);
+                copy_image((ch + 2) % IB, ch + 2);                   // its buffer was released at the end of chunk ch - 1
+                asm volatile("cp.async.wait_group 2;" ::: "memory");
+                __syncthreads();                                     // image `ch` is complete for every thread
+                const int buf = ch % IB;
 #pragma unroll
-                for (int n = 0; n < NT; ++n) {
+                for (int b = 0; b < NB; ++b) {
 #pragma unroll
-                    for (int t = 0; t < 3; ++t) {
-                        const uint2 bb = *reinterpret_cast<const uint2*>(&Gs[buf][t][n * 8 + g][b * 32 + s * 16 + q * 4]);
-                        mma_bf16_16816(acc[n], a, bb.x, bb.y);
+                    for (int s = 0; s < 2; ++s) {
+                        // A fragment of k-step (b, s): a0 = row g k-slots 2q,2q+1; a1 = row g+8; a2 = row g slots 2q+8,+9
+                        uint32_t a[4];
+                        a[0] = s ? va[u][b].z : va[u][b].x;
+                        a[2] = s ? va[u][b].w : va[u][b].y;
+                        a[1] = s ? vb[u][b].z : vb[u][b].x;
+                        a[3] = s ? vb[u][b].w : vb[u][b].y;
+#pragma unroll
+                        for (int n = 0; n < NT; ++n) {
+#pragma unroll
+                            for (int t = 0; t < 3; ++t) {
+                                const uint2 bb =
+                                    *reinterpret_cast<const uint2*>(&Gs[buf][t][n * 8 + g][b * 32 + s * 16 + q * 4]);
+                                mma_bf16_16816(acc[n], a, bb.x, bb.y);
+                            }
+                        }
                     }
                 }
+                __syncthreads();                                     // this buffer is refilled by the next iteration's request
             }
         }
-        __syncthreads();                                             // buffer may be refilled two chunks later
     }
 
     // fragment -> logits: acc[n][0..1] = (row g, c = 8n + 2q, +1), acc[n][2..3] = (row g + 8, same columns)
@@ -199,7 +216,8 @@ static molora_status_t gate_mma_launch(const void* x, int64_t N, int d, int64_t 
 
 size_t route_gate_mma_workspace_bytes(int32_t d, int32_t C)
 {
-    if (C <= 8) return 0;
+    if (C <= 4) return 0;
+    if (C <= 8) return (size_t)((d + 127) / 128) * GateImage<1, 128>::kBytes;
     if (C <= 16) return (size_t)((d + 127) / 128) * GateImage<2, 128>::kBytes;
     return (size_t)((d + 63) / 64) * GateImage<4, 64>::kBytes;
 }
@@ -209,6 +227,7 @@ molora_status_t launch_route_gate_mma(const void* x, int64_t N, int32_t d, int64
                                       cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
+    if (C <= 8) return gate_mma_launch<1, 4, 128>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
     if (C <= 16) return gate_mma_launch<2, 4, 128>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
     return gate_mma_launch<4, 4, 64>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
 }

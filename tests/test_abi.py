@@ -33,7 +33,7 @@ def test_invalid_arguments_are_refused_before_any_launch():
     assert lib.molora_route_gate(fake, M.BF16, 4, 12, 16, fake, None, 4, fake, None, None, 0, None) == 2
     assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 33, fake, None, None, 0, None) == 2
     assert lib.molora_route_gate(fake, M.BF16, 4, 16, 8, fake, None, 4, fake, None, None, 0, None) == 1
-    # tensor-core gate (bf16, C > 8) without its workspace
+    # tensor-core gate (bf16, C > 4) without its workspace
     assert M.molora_route_gate_workspace_bytes(M.BF16, 4096, 16) > 0 and M.molora_route_gate_workspace_bytes(M.BF16, 2048, 4) == 0
     assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 16, fake, None, None, 0, None) == 3
     # group: C out of range, null outputs
