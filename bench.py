@@ -177,6 +177,7 @@ def marshal_step(lib, w, s, shared, stream_handle):
 def run_ours(args):
     import torch
     import paper_2603_15965_b200 as M
+    import paper_2603_15965_b200.binding  # noqa: F401
     from paper_2603_15965_b200 import workloads as W
     from paper_2603_15965_b200.binding import pack_proj_descs
     from paper_2603_15965_b200.build import build_library
@@ -305,58 +306,58 @@ def run_ours(args):
 
 
 def run_e2e(args, torch, M, w, sets, shared, world, dist):
-    """Same metric with HOST buffers: every step copies its activations (x, y; ids if vocab-routed) from pinned
-    host memory to the device, runs the path, and copies the result h back to pinned host memory."""
+    """Same metric through the host-buffer entry point: every step, molora_forward_host copies the step's
+    activations (x, y; ids / r if routed from integers) from pinned host memory into a device arena, runs
+    route -> group -> apply and copies h back to pinned host memory.  Two streams with one arena each alternate,
+    so the copies of consecutive steps overlap (the PCIe link is full duplex)."""
     N, C = w.N, w.C
-    stream = torch.cuda.current_stream()
-    s = sets[0]
-    hx = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in s["x"].items()}
-    hy = [torch.empty_like(v, device="cpu").pin_memory() for v in s["y"]]
-    hout = [torch.empty_like(v, device="cpu").pin_memory() for v in s["y"]]
-    hids = s["ids"].cpu().pin_memory() if s["ids"] is not None else None
-    hr = s["r_given"].cpu().pin_memory() if s["r_given"] is not None else None
-    for k, v in s["x"].items():
-        hx[k].copy_(v)
+    s0 = sets[0]
+    router = {"vocab": M.ROUTE_VOCAB, "gate": M.ROUTE_GATE, "given": M.ROUTE_GIVEN}[w.router]
+    gate_proj = 0
+    if w.router == "gate":
+        gate_proj = [p.x_key for p in w.projections].index(w.gate_x_key)
     pristine = build_pristine_y(w, torch)
-    for h, p in zip(hy, pristine):
-        h.copy_(p)
-    h2d = sum(t.numel() * t.element_size() for t in list(hx.values()) + hy) + \
-        (hids.numel() * 4 if hids is not None else 0) + (hr.numel() * 4 if hr is not None else 0)
-    d2h = sum(t.numel() * t.element_size() for t in hout)
+    lanes = []
+    for _ in range(2):
+        hx = {k: v.cpu().pin_memory() for k, v in s0["x"].items()}
+        hy = [p.clone().pin_memory() for p in pristine]
+        projs = [M.HostProj(hx[p.x_key], y, A, B, 1.0) for p, y, A, B in zip(w.projections, hy, s0["A"], s0["B"])]
+        packed = M.binding.pack_host_projs(projs)
+        arena = torch.empty(M.molora_forward_host_arena_bytes(None, router, gate_proj, packed=packed), dtype=torch.uint8,
+                            device="cuda")
+        src = None
+        if w.router == "vocab":
+            src = s0["ids"].cpu().pin_memory()
+        elif w.router == "given":
+            src = s0["r_given"].cpu().pin_memory()
+        lanes.append({"hx": hx, "hy": hy, "packed": packed, "arena": arena, "src": src, "stream": torch.cuda.Stream()})
+    h2d = sum(t.numel() * t.element_size() for t in list(lanes[0]["hx"].values()) + lanes[0]["hy"]) + \
+        (lanes[0]["src"].numel() * 4 if lanes[0]["src"] is not None else 0)
+    d2h = sum(t.numel() * t.element_size() for t in lanes[0]["hy"])
 
-    def step():
-        for k, v in s["x"].items():
-            v.copy_(hx[k], non_blocking=True)
-        for v, h in zip(s["y"], hy):
-            v.copy_(h, non_blocking=True)
-        if hids is not None:
-            s["ids"].copy_(hids, non_blocking=True)
-        if hr is not None:
-            s["r_given"].copy_(hr, non_blocking=True)
-        if w.router == "gate":
-            M.molora_route_gate(s["x"][w.gate_x_key], shared["G"], r_out=s["r"], ws=shared["gate_ws"])
-            r = s["r"]
-        elif w.router == "vocab":
-            M.molora_route_vocab(s["ids"], shared["breaks"], r_out=s["r"])
-            r = s["r"]
-        else:
-            r = s["r_given"]
-        M.molora_group(r, C, s["counts"], s["offsets"], s["perm"])
-        M.molora_apply_batched(None, s["offsets"], s["perm"], packed=s["packed"])
-        for h, v in zip(hout, s["y"]):
-            h.copy_(v, non_blocking=True)
+    def step(k):
+        ln = lanes[k % 2]
+        M.molora_forward_host(router, None, ln["arena"], route_src=ln["src"], breaks=shared["breaks"], G=shared["G"],
+                              gate_proj=gate_proj, dev_status=shared["status"], stream=ln["stream"], packed=ln["packed"])
 
-    K = max(3, min(args.steps, args.e2e_steps))
-    for _ in range(3):
-        step()
+    K = max(4, min(args.steps, args.e2e_steps))
+    for k in range(4):
+        step(k)
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
+    main = torch.cuda.current_stream()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record(stream)
-    for _ in range(K):
-        step()
-    t1.record(stream)
+    t0.record(main)
+    for ln in lanes:
+        ln["stream"].wait_event(t0)
+    for k in range(K):
+        step(k)
+    for ln in lanes:
+        done = torch.cuda.Event()
+        done.record(ln["stream"])
+        main.wait_event(done)
+    t1.record(main)
     torch.cuda.synchronize()
     ms = t0.elapsed_time(t1)
     if dist is not None:
@@ -365,7 +366,8 @@ def run_e2e(args, torch, M, w, sets, shared, world, dist):
         ms = float(t.item())
     return {"value": world * N / (ms / K * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
             "d2h_bytes_per_step": int(d2h), "steps": K, "ms_per_step": ms / K,
-            "note": "pinned host x, y (and ids) copied in, h copied out every step; weights resident"}
+            "note": "molora_forward_host: pinned host x, y (and ids / r) copied in, h copied out every step; "
+                    "adapter and gate weights resident; two streams alternate"}
 
 
 def build_pristine_y(w, torch):

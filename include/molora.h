@@ -150,6 +150,40 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t *projs, int32_t P,
                                      int32_t C, const int32_t *offsets, const int32_t *perm, void *ws, size_t ws_bytes,
                                      uint32_t *dev_status, void *stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * The whole path on HOST activations (one layer: route -> group -> apply for P projections), for callers
+ * whose activations live in host memory.  Everything is enqueued on `stream` in this order: host-to-device
+ * copies of the routing source and of every distinct x and every y into `arena`, the router, the grouping,
+ * one batched apply (Eq. 2), device-to-host copies of every y back into y_host.  The call returns without
+ * waiting; x_host / y_host must stay valid (and should be pinned for the copies to be asynchronous) until the
+ * stream has finished.  Adapter stacks, gate weights and vocabulary breaks are DEVICE pointers: weights stay
+ * resident at fixed addresses (the hot-set idea of Definition 5.1), only activations travel.
+ *
+ * router       MOLORA_ROUTE_VOCAB: route_src_host = ids int32[N], breaks_dev int32[M+1]
+ *              MOLORA_ROUTE_GATE:  the gate reads the staged x of projection `gate_proj`; G_dev fp32 [d_in, C],
+ *                                  bias_dev fp32 [C] or NULL
+ *              MOLORA_ROUTE_GIVEN: route_src_host = r int32[N]
+ * projs        HOST array of P descriptors (1 <= P <= MOLORA_MAX_PROJECTIONS); projections whose x_host
+ *              pointers are equal share one staged copy
+ * arena        device scratch of at least molora_forward_host_arena_bytes(...) bytes, 256-byte aligned
+ * dev_status   device uint32 or NULL (as for the individual calls)
+ * Errors are detected before anything is enqueued, as for the individual calls. */
+typedef enum { MOLORA_ROUTE_VOCAB = 0, MOLORA_ROUTE_GATE = 1, MOLORA_ROUTE_GIVEN = 2 } molora_router_t;
+typedef struct {
+    const void *x_host; /* [N, d_in]  dense (pitch d_in)                         */
+    void *y_host;       /* [N, d_out] dense; in: base projection x W, out: h     */
+    const void *A;      /* device [C, d_in, rank]                                */
+    const void *B;      /* device [C, rank, d_out]                               */
+    int32_t d_in, d_out, rank;
+    float scale;
+} molora_host_proj_t;
+size_t molora_forward_host_arena_bytes(const molora_host_proj_t *projs, int32_t P, molora_dtype_t dt, int64_t N,
+                                       int32_t C, molora_router_t router, int32_t gate_proj);
+molora_status_t molora_forward_host(molora_router_t router, const int32_t *route_src_host, const int32_t *breaks_dev,
+                                    int32_t M, const float *G_dev, const float *bias_dev, int32_t gate_proj,
+                                    const molora_host_proj_t *projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C,
+                                    void *arena, size_t arena_bytes, uint32_t *dev_status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -11,4 +11,5 @@ from .binding import (  # noqa: F401
     molora_group_workspace_bytes, molora_group,
     molora_apply_workspace_bytes, molora_apply, molora_apply_batched,
     ProjDesc, F32, BF16,
+    HostProj, molora_forward_host, molora_forward_host_arena_bytes, ROUTE_VOCAB, ROUTE_GATE, ROUTE_GIVEN,
 )

@@ -32,6 +32,11 @@ class MoloraError(RuntimeError):
         self.status = status
 
 
+class _HostProjC(ctypes.Structure):
+    _fields_ = [("x_host", ctypes.c_void_p), ("y_host", ctypes.c_void_p), ("A", ctypes.c_void_p), ("B", ctypes.c_void_p),
+                ("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32), ("rank", ctypes.c_int32), ("scale", ctypes.c_float)]
+
+
 class _ProjDescC(ctypes.Structure):
     _fields_ = [("x", ctypes.c_void_p), ("ldx", ctypes.c_int64), ("y", ctypes.c_void_p), ("ldy", ctypes.c_int64),
                 ("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32),
@@ -76,7 +81,13 @@ def load_library():
                                  vp, vp]
     lib.molora_apply_batched.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64, i32, vp, vp, vp, sz, vp,
                                          vp]
-    for name in ("molora_route_vocab", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched"):
+    lib.molora_forward_host_arena_bytes.restype = sz
+    lib.molora_forward_host_arena_bytes.argtypes = [ctypes.POINTER(_HostProjC), i32, ctypes.c_int, i64, i32, ctypes.c_int,
+                                                    i32]
+    lib.molora_forward_host.argtypes = [ctypes.c_int, vp, vp, i32, vp, vp, i32, ctypes.POINTER(_HostProjC), i32,
+                                        ctypes.c_int, i64, i32, vp, sz, vp, vp]
+    for name in ("molora_route_vocab", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched",
+                 "molora_forward_host"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -267,3 +278,57 @@ def molora_apply_batched(projs, offsets: torch.Tensor, perm: torch.Tensor, ws: O
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_apply_batched", lib.molora_apply_batched(arr, len(arr), dt, N, C, _ptr(offsets), _ptr(perm),
                                                             _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
+
+
+ROUTE_VOCAB, ROUTE_GATE, ROUTE_GIVEN = 0, 1, 2
+
+
+@dataclass
+class HostProj:
+    """One projection of :func:`molora_forward_host`: x, y dense HOST tensors (pinned for asynchronous copies),
+    A, B dense DEVICE tensors."""
+    x: torch.Tensor
+    y: torch.Tensor
+    A: torch.Tensor
+    B: torch.Tensor
+    scale: float = 1.0
+
+
+def pack_host_projs(projs: Sequence[HostProj]):
+    arr = (_HostProjC * len(projs))()
+    N = C = dt = None
+    for i, p in enumerate(projs):
+        if p.x.is_cuda or p.y.is_cuda or not p.x.is_contiguous() or not p.y.is_contiguous():
+            raise ValueError("x, y: expected dense host tensors")
+        if not p.A.is_cuda or not p.B.is_cuda or not p.A.is_contiguous() or not p.B.is_contiguous():
+            raise ValueError("A, B: expected dense device tensors")
+        n, d_in = p.x.shape
+        d_out = p.y.shape[1]
+        c, rank = p.A.shape[0], p.A.shape[2]
+        if p.y.shape[0] != n or p.A.shape[1] != d_in or tuple(p.B.shape) != (c, rank, d_out):
+            raise ValueError("shapes of x, y, A, B do not match")
+        if N is None:
+            N, C, dt = n, c, _dtype_code(p.x)
+        elif (N, C, dt) != (n, c, _dtype_code(p.x)):
+            raise ValueError("all projections share N, C and the element type")
+        arr[i] = _HostProjC(p.x.data_ptr(), p.y.data_ptr(), p.A.data_ptr(), p.B.data_ptr(), d_in, d_out, rank,
+                            float(p.scale))
+    return arr, N, C, dt
+
+
+def molora_forward_host_arena_bytes(projs, router: int, gate_proj: int = 0, packed=None) -> int:
+    arr, N, C, dt = packed if packed is not None else pack_host_projs(projs)
+    return int(load_library().molora_forward_host_arena_bytes(arr, len(arr), dt, N, C, router, gate_proj))
+
+
+def molora_forward_host(router: int, projs, arena: torch.Tensor, route_src: Optional[torch.Tensor] = None,
+                        breaks: Optional[torch.Tensor] = None, G: Optional[torch.Tensor] = None,
+                        bias: Optional[torch.Tensor] = None, gate_proj: int = 0,
+                        dev_status: Optional[torch.Tensor] = None, stream=None, packed=None) -> None:
+    """route -> group -> apply on HOST activations (copied in and out on the stream).  Asynchronous."""
+    lib = load_library()
+    arr, N, C, dt = packed if packed is not None else pack_host_projs(projs)
+    M = 0 if breaks is None else breaks.numel() - 1
+    _check("molora_forward_host", lib.molora_forward_host(
+        router, _ptr(route_src), _ptr(breaks), M, _ptr(G), _ptr(bias), gate_proj, arr, len(arr), dt, N, C,
+        _ptr(arena), arena.numel() * arena.element_size(), _ptr(dev_status), _stream(stream)))

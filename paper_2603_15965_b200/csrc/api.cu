@@ -143,4 +143,128 @@ molora_status_t molora_apply(const void* x, int64_t ldx, void* y, int64_t ldy, m
     return molora_apply_batched(&p, 1, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, stream);
 }
 
+// ---------------------------------------------------------------------------------------------- host-buffer path
+namespace {
+
+struct HostPlan {          // byte offsets into the arena
+    size_t ids, r, counts, offsets, perm, gate_ws, x[MOLORA_MAX_PROJECTIONS], y[MOLORA_MAX_PROJECTIONS], total;
+    int x_owner[MOLORA_MAX_PROJECTIONS];   // first projection with the same x_host (its staged copy is shared)
+};
+
+size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+bool plan_host(const molora_host_proj_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C,
+               molora_router_t router, int32_t gate_proj, HostPlan& pl)
+{
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 0 || C < 1 || C > MOLORA_MAX_ADAPTERS) return false;
+    if (dt != MOLORA_F32 && dt != MOLORA_BF16) return false;
+    const size_t e = dt == MOLORA_BF16 ? 2 : 4;
+    size_t off = 0;
+    pl.ids = off;      off = align256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
+    pl.r = off;        off = align256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
+    pl.counts = off;   off = align256(off + sizeof(int32_t) * (size_t)C);
+    pl.offsets = off;  off = align256(off + sizeof(int32_t) * (size_t)(C + 1));
+    pl.perm = off;     off = align256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
+    pl.gate_ws = off;
+    if (router == MOLORA_ROUTE_GATE) {
+        if (gate_proj < 0 || gate_proj >= P) return false;
+        off = align256(off + route_gate_workspace_bytes(dt, projs[gate_proj].d_in, C));
+    }
+    for (int i = 0; i < P; ++i) {
+        pl.x_owner[i] = i;
+        for (int j = 0; j < i; ++j)
+            if (projs[j].x_host == projs[i].x_host && projs[j].d_in == projs[i].d_in) { pl.x_owner[i] = j; break; }
+        if (pl.x_owner[i] == i) {
+            pl.x[i] = off;
+            off = align256(off + e * (size_t)N * (size_t)projs[i].d_in);
+        } else {
+            pl.x[i] = pl.x[pl.x_owner[i]];
+        }
+        pl.y[i] = off;
+        off = align256(off + e * (size_t)N * (size_t)projs[i].d_out);
+    }
+    pl.total = off;
+    return true;
+}
+
+}  // namespace
+
+size_t molora_forward_host_arena_bytes(const molora_host_proj_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
+                                       int32_t C, molora_router_t router, int32_t gate_proj)
+{
+    HostPlan pl;
+    return plan_host(projs, P, dt, N, C, router, gate_proj, pl) ? pl.total : 0;
+}
+
+molora_status_t molora_forward_host(molora_router_t router, const int32_t* route_src_host, const int32_t* breaks_dev,
+                                    int32_t M, const float* G_dev, const float* bias_dev, int32_t gate_proj,
+                                    const molora_host_proj_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C,
+                                    void* arena, size_t arena_bytes, uint32_t* dev_status, void* stream)
+{
+    HostPlan pl;
+    if (N >= INT32_MAX || !plan_host(projs, P, dt, N, C, router, gate_proj, pl)) return MOLORA_ERR_INVALID_ARG;
+    if (router != MOLORA_ROUTE_VOCAB && router != MOLORA_ROUTE_GATE && router != MOLORA_ROUTE_GIVEN)
+        return MOLORA_ERR_INVALID_ARG;
+    if (router != MOLORA_ROUTE_GATE && N > 0 && route_src_host == nullptr) return MOLORA_ERR_INVALID_ARG;
+    if (router == MOLORA_ROUTE_VOCAB && (breaks_dev == nullptr || M < 1 || M > MOLORA_MAX_ADAPTERS)) return MOLORA_ERR_INVALID_ARG;
+    if (router == MOLORA_ROUTE_GATE && (G_dev == nullptr || C > 32)) return G_dev == nullptr ? MOLORA_ERR_INVALID_ARG : MOLORA_ERR_UNSUPPORTED;
+    if (arena == nullptr || arena_bytes < pl.total || (reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return MOLORA_ERR_WORKSPACE;
+    char* base = static_cast<char*>(arena);
+    molora_proj_desc_t dev[MOLORA_MAX_PROJECTIONS];
+    for (int i = 0; i < P; ++i) {
+        if (projs[i].x_host == nullptr || projs[i].y_host == nullptr) return MOLORA_ERR_INVALID_ARG;
+        dev[i].x = base + pl.x[i];
+        dev[i].ldx = projs[i].d_in;
+        dev[i].y = base + pl.y[i];
+        dev[i].ldy = projs[i].d_out;
+        dev[i].A = projs[i].A;
+        dev[i].B = projs[i].B;
+        dev[i].d_in = projs[i].d_in;
+        dev[i].d_out = projs[i].d_out;
+        dev[i].rank = projs[i].rank;
+        dev[i].scale = projs[i].scale;
+        const molora_status_t st = check_proj(dev[i], dt);
+        if (st != MOLORA_OK) return st;
+    }
+    if (N == 0) return MOLORA_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t e = dt == MOLORA_BF16 ? 2 : 4;
+    int32_t* r = reinterpret_cast<int32_t*>(base + pl.r);
+    int32_t* ids = reinterpret_cast<int32_t*>(base + pl.ids);
+    // 1. activations and routing source: host -> device
+    if (router != MOLORA_ROUTE_GATE &&
+        cudaMemcpyAsync(router == MOLORA_ROUTE_VOCAB ? ids : r, route_src_host, sizeof(int32_t) * (size_t)N,
+                        cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return MOLORA_ERR_CUDA;
+    for (int i = 0; i < P; ++i) {
+        if (pl.x_owner[i] == i &&
+            cudaMemcpyAsync(base + pl.x[i], projs[i].x_host, e * (size_t)N * projs[i].d_in, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return MOLORA_ERR_CUDA;
+        if (cudaMemcpyAsync(base + pl.y[i], projs[i].y_host, e * (size_t)N * projs[i].d_out, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return MOLORA_ERR_CUDA;
+    }
+    // 2. route
+    molora_status_t st = MOLORA_OK;
+    if (router == MOLORA_ROUTE_VOCAB) {
+        st = launch_route_vocab(ids, N, breaks_dev, M, r, dev_status, s);
+    } else if (router == MOLORA_ROUTE_GATE) {
+        const molora_proj_desc_t& gp = dev[gate_proj];
+        if ((gp.d_in % 8) != 0) return MOLORA_ERR_UNSUPPORTED;
+        st = launch_route_gate(gp.x, dt, N, gp.d_in, gp.ldx, G_dev, bias_dev, C, r, nullptr, base + pl.gate_ws, s);
+    }
+    if (st != MOLORA_OK) return st;
+    // 3. group, 4. apply
+    int32_t* offsets = reinterpret_cast<int32_t*>(base + pl.offsets);
+    int32_t* perm = reinterpret_cast<int32_t*>(base + pl.perm);
+    st = launch_group(r, N, C, reinterpret_cast<int32_t*>(base + pl.counts), offsets, perm, nullptr, 0, dev_status, s);
+    if (st != MOLORA_OK) return st;
+    st = molora_apply_batched(dev, P, dt, N, C, offsets, perm, nullptr, 0, dev_status, stream);
+    if (st != MOLORA_OK) return st;
+    // 5. results: device -> host
+    for (int i = 0; i < P; ++i)
+        if (cudaMemcpyAsync(projs[i].y_host, base + pl.y[i], e * (size_t)N * projs[i].d_out, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return MOLORA_ERR_CUDA;
+    return MOLORA_OK;
+}
+
 }  // extern "C"

@@ -309,3 +309,38 @@ def test_tensor_path_selector_exact_and_status_clean():
                    dev_status=status)
     assert np.array_equal(yd.float().cpu().numpy(), expect)
     assert int(status.item()) == 0
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+@pytest.mark.parametrize("name", ["c1", "c2", "c3"])
+def test_forward_host_matches_oracle(name):
+    w = W.get(name) if name != "c2" else W.get("c2", n_tokens=1300)
+    bf16 = w.dtype == "bf16"
+    router = {"vocab": M.ROUTE_VOCAB, "gate": M.ROUTE_GATE, "given": M.ROUTE_GIVEN}[w.router]
+
+    def host(a):
+        t = torch.from_numpy(W.bf16_bits(a)).view(torch.bfloat16) if bf16 else torch.from_numpy(a.copy())
+        return t.pin_memory()
+
+    hx = {k: host(v) for k, v in w.inputs.items()}
+    hy = [host(p.y) for p in w.projections]
+    projs = [M.HostProj(hx[p.x_key], y, dev_tensor(p.A, w.dtype), dev_tensor(p.B, w.dtype)) for p, y in
+             zip(w.projections, hy)]
+    gate_proj = [p.x_key for p in w.projections].index(w.gate_x_key) if w.router == "gate" else 0
+    arena = torch.empty(M.molora_forward_host_arena_bytes(projs, router, gate_proj), dtype=torch.uint8, device="cuda")
+    src = None
+    if w.router == "vocab":
+        src = torch.from_numpy(w.ids).pin_memory()
+    elif w.router == "given":
+        src = torch.from_numpy(w.r).pin_memory()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    M.molora_forward_host(router, projs, arena, route_src=src,
+                          breaks=dev_tensor(w.breaks, "i") if w.breaks is not None else None,
+                          G=dev_tensor(w.G, "f32") if w.G is not None else None, gate_proj=gate_proj, dev_status=status)
+    torch.cuda.synchronize()
+    r_ref, margin = oracle_route(w)
+    keep = np.ones(w.N, bool) if margin is None else margin >= 1e-3
+    for p, y in zip(w.projections, hy):
+        ref, _ = oracle.apply(w.inputs[p.x_key], p.y, p.A, p.B, r_ref)
+        assert_close(y.float().numpy().astype(np.float64)[keep], ref[keep], what=f"forward_host {name}/{p.name}")
+    assert int(status.item()) == 0
