@@ -20,7 +20,7 @@
 // so that every global store instruction writes full 128-byte lines.
 //
 // Occupancy.  A call with few tiles (N / 128 of them) cannot fill 148 SMs, so a tile may be shared by a
-// thread-block cluster of S = 2 or 4 CTAs: CTA q shrinks over the q-th slice of d_in, the S partial T
+// thread-block cluster of S = 2, 3 or 4 CTAs: CTA q shrinks over the q-th slice of d_in, the S partial T
 // tiles (fp32) are exchanged through distributed shared memory and summed in rank order by every CTA (so
 // all of them hold the same bits), and CTA q then expands into the q-th slice of d_out.  x, y, A_c and B_c
 // are still read exactly once per tile.  The exchange uses mbarriers with remote arrives (bounded waits);
@@ -475,10 +475,12 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 for (int i = 0; i < 8; ++i)
                     op[i] = *reinterpret_cast<const uint4*>(
                         ytile + swizzle_offset((uint32_t)((et >> 3) + 16 * i) * 128u + piece * 16, 3));
+                if (et == 0) MOLORA_TR(2, it, 7);
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     if (otok[i] >= 0) stg128(dstc + (int64_t)otok[i] * pj.ldy, op[i]);
             }
+            if (et == 0) MOLORA_TR(2, it, 4);
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
             if (et == 0) mbar_arrive(bar(&ctrl->empty[s]));   // the stage may be refilled
             if (et == 0) MOLORA_TR(2, it, 6);
@@ -573,7 +575,7 @@ static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, int split, cuda
 template <int R>
 static int max_active_clusters(int split)
 {
-    static int cache[kMaxSplit + 1] = {0, 0, 0, 0, 0};
+    static int cache[kMaxSplit + 1] = {};
     if (cache[split] == 0) {
         cudaFuncSetAttribute(apply_umma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<R>::kSmemBytes);
         cudaLaunchConfig_t cfg = {};
@@ -605,14 +607,14 @@ static int choose_split_for_rank(const UmmaParams& prm, int64_t N)
         best = std::max(1, std::min(atoi(env), kMaxSplit));
     } else {
         double best_cost = 1e30;
-        for (int split = 1; split <= kMaxSplit; split *= 2) {
+        for (int split = 1; split <= kMaxSplit; ++split) {    // cluster sizes need not be powers of two
             const int resident = max_active_clusters<R>(split);
             const double waves = (double)((tiles + resident - 1) / resident);
             const double cost = waves * (1.0 / split + 0.15 + (split > 1 ? 0.10 : 0.0));
             if (cost < best_cost - 1e-9) { best_cost = cost; best = split; }
         }
     }
-    while (best > 1 && min_kx / best < 4) best /= 2;         // keep at least four chunks of d_in per CTA
+    while (best > 1 && min_kx / best < 4) --best;            // keep at least four chunks of d_in per CTA
     return best;
 }
 
