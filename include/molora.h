@@ -94,6 +94,28 @@ molora_status_t molora_route_gate(const void *x, molora_dtype_t xdt, int64_t N, 
                                   size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * The same gate for callers that cannot provide a workspace.  (The paper has no counterpart: this entry point
+ * exists for integration reasons only.)  Some hosts of this library may not allocate device memory at the
+ * point where they route tokens -- code running between the capture and replay of a fixed-address serving
+ * graph, plug-ins that are handed tensors but no allocator, allocation-free real-time loops -- and so cannot
+ * supply molora_route_gate's `ws`.  This variant keeps the scratch inside the library instead: a fixed 2 MiB
+ * device array that every GPU loading the library holds until the process exits.
+ *   - Same arguments, results and errors as molora_route_gate, without ws / ws_bytes.
+ *   - Limit: molora_route_gate_workspace_bytes(xdt, d, C) must not exceed 2 MiB (2 097 152 bytes); e.g.
+ *     bf16 x with C <= 16 up to d = 19 328, with C <= 32 up to d = 8 704.  Larger gates are refused with
+ *     MOLORA_ERR_WORKSPACE and nothing is enqueued.  Calls that need no scratch (fp32 x, or C <= 4) always fit.
+ *   - It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the array's device address (with that device current); make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the previous call wrote.  The kernels
+ *     rewrite every byte they later read, so nothing has to be cleared between calls -- but two calls that
+ *     overlap on the GPU (different streams, or graph branches) race on it: serialise them.
+ */
+molora_status_t molora_route_gate_noalloc(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx,
+                                          const float *G, const float *bias, int32_t C, int32_t *r_out,
+                                          float *logits_out, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Grouping (Section 3.3 steps 1-3; Algorithm 2; Table 10 "histogram"):
  *     counts[c]    = |{ i : r[i] = c }|
  *     offsets[0]   = 0,  offsets[c+1] = offsets[c] + counts[c]

@@ -72,6 +72,8 @@ def load_library():
     lib.molora_route_gate_workspace_bytes.restype = sz
     lib.molora_route_gate_workspace_bytes.argtypes = [ctypes.c_int, i32, i32]
     lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp]
+    lib.molora_route_gate_noalloc.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp]
+    lib.molora_route_gate_noalloc.restype = ctypes.c_int
     lib.molora_group_workspace_bytes.restype = sz
     lib.molora_group_workspace_bytes.argtypes = [i64, i32]
     lib.molora_group.argtypes = [vp, i64, i32, vp, vp, vp, vp, sz, vp, vp]
@@ -179,6 +181,25 @@ def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Ten
     _check("molora_route_gate", lib.molora_route_gate(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(G), _ptr(bias), C,
                                                       _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out), _ptr(ws),
                                                       ws_bytes, _stream(stream)))
+    return r_out
+
+
+def molora_route_gate_noalloc(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                              r_out: Optional[torch.Tensor] = None, logits_out: Optional[torch.Tensor] = None,
+                              stream=None) -> torch.Tensor:
+    """The gate without a caller workspace: its scratch is a fixed 2 MiB array inside the library (so gates whose
+    split weights need more are refused), for callers that cannot allocate device memory where they route.
+    Pass ``r_out`` to keep this binding allocation-free as well.  Calls that overlap on the GPU race on the array."""
+    lib = load_library()
+    N, d, ldx = _matrix(x, "x")
+    if G.dtype != torch.float32 or not G.is_cuda or not G.is_contiguous() or G.dim() != 2 or G.shape[0] != d:
+        raise ValueError("G: expected a contiguous fp32 CUDA tensor of shape [d, C]")
+    C = G.shape[1]
+    if r_out is None:
+        r_out = torch.empty(N, dtype=torch.int32, device=x.device)
+    _check("molora_route_gate_noalloc", lib.molora_route_gate_noalloc(
+        _ptr(x), _dtype_code(x), N, d, ldx, _ptr(G), _ptr(bias), C, _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
+        _stream(stream)))
     return r_out
 
 

@@ -14,6 +14,7 @@
 // once per call by a small preparation kernel that writes the exact shared-memory image of every k chunk into
 // the caller's workspace; the gate CTAs then only copy images (cp.async, double buffered).
 #include <algorithm>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -233,3 +234,54 @@ molora_status_t launch_route_gate_mma(const void* x, int64_t N, int32_t d, int64
 }
 
 }  // namespace molora
+
+// ------------------------------------------------------------------------------------------------
+// molora_route_gate_noalloc: the gate for callers that cannot hand the library a workspace.
+//
+// The split gate weights normally go to caller-provided scratch.  Here they go to a fixed array that is
+// part of the library image: every GPU that loads the library holds these 2 MiB until the process exits.
+// In host code the array's name is only a handle; the device address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and is what the kernels receive.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kNoAllocScratchBytes = 2u << 20;
+static __device__ __align__(256) unsigned char g_gate_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_scratch_ptr[kMaxDevices] = {};
+std::mutex g_scratch_mutex;
+
+// Device address of the scratch array on the current device (looked up on the first call per device).
+molora_status_t scratch_for_current_device(void** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MOLORA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_gate_scratch) != cudaSuccess || p == nullptr) return MOLORA_ERR_CUDA;
+        g_scratch_ptr[dev] = p;
+    }
+    *out = g_scratch_ptr[dev];
+    return MOLORA_OK;
+}
+
+}  // namespace
+
+extern "C" molora_status_t molora_route_gate_noalloc(const void* x, molora_dtype_t xdt, int64_t N, int32_t d,
+                                                     int64_t ldx, const float* G, const float* bias, int32_t C,
+                                                     int32_t* r_out, float* logits_out, void* stream)
+{
+    if (d <= 0 || C < 1) return MOLORA_ERR_INVALID_ARG;
+    if (C > 32) return MOLORA_ERR_UNSUPPORTED;
+    const size_t need = molora_route_gate_workspace_bytes(xdt, d, C);
+    if (need > kNoAllocScratchBytes) return MOLORA_ERR_WORKSPACE;     // d * C too large for the built-in scratch
+    void* scratch = nullptr;
+    if (need > 0) {
+        const molora_status_t st = scratch_for_current_device(&scratch);
+        if (st != MOLORA_OK) return st;
+    }
+    return molora_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, scratch, need > 0 ? kNoAllocScratchBytes : 0,
+                             stream);
+}
