@@ -208,7 +208,7 @@ def run_ours(args):
     del probe
     w, sets, shared = build_sets(W, torch, name, n_sets, rank)
     N, C = w.N, w.C
-    stream = torch.cuda.current_stream()
+    stream = torch.cuda.Stream()      # every call of the timed region is enqueued (or captured) on this stream
 
     # per-set routing/grouping outputs (fixed addresses, as a serving stack would keep them)
     for s in sets:
@@ -238,34 +238,77 @@ def run_ours(args):
             ev[1].record(stream)
 
     # ------------------------------------------------------------------ warm-up, then the timed region
-    for i in range(max(3, args.warmup)):
-        step(sets[i % n_sets])
-    torch.cuda.synchronize()
-    clocks = Clocks(local)
-    clocks.start()
     K = args.steps
-    ev_every = max(1, K // 2000)                                   # bound the number of event pairs
-    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) if k % ev_every == 0 else None
-             for k in range(K)]
+    W0 = max(3, args.warmup)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
-    t0.record(stream)
-    for k in range(K):
-        step(sets[(args.warmup + k) % n_sets], pairs[k])
-    t1.record(stream)
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    total_ms = t0.elapsed_time(t1)
-    # keep the GPU busy a little longer (untimed) if the region was too short for the clock sampler
-    t_end = time.time() + (0.25 if total_ms < 250 else 0.0)
-    while time.time() < t_end:
-        step(sets[0])
-    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for i in range(W0):
+            step(sets[i % n_sets])
+        torch.cuda.synchronize()
+        if args.launch == "graph":
+            # The paper replays this path from a CUDA graph (fixed addresses, no host work between kernels); so does
+            # the bench: K steps are captured in chunks and replayed, which removes the Python/driver launch cost
+            # from a step that lasts tens of microseconds.  A second set of graphs holds only the apply calls over
+            # the same buffer rotation; its replay time / K is the kernel time used for the roofline.
+            CH = min(K, 512)
+
+            def capture(fn, first, n):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    for k in range(first, first + n):
+                        fn(sets[k % n_sets])
+                return g
+
+            reps, rem = divmod(K, CH)
+            g_full, g_rem = capture(step, W0, CH), (capture(step, W0 + reps * CH, rem) if rem else None)
+            a_full = capture(lambda s_: s_["calls"][2](), W0, CH)
+            a_rem = capture(lambda s_: s_["calls"][2](), W0 + reps * CH, rem) if rem else None
+            g_full.replay()
+            torch.cuda.synchronize()
+        clocks = Clocks(local)
+        clocks.start()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if args.launch == "graph":
+            t0.record(stream)
+            for _ in range(reps):
+                g_full.replay()
+            if g_rem is not None:
+                g_rem.replay()
+            t1.record(stream)
+            torch.cuda.synchronize()
+            total_ms = t0.elapsed_time(t1)
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            for _ in range(reps):
+                a_full.replay()
+            if a_rem is not None:
+                a_rem.replay()
+            a1.record(stream)
+            torch.cuda.synchronize()
+            apply_ms = a0.elapsed_time(a1) / K
+            kernel_timing = "apply-only graphs over the same buffer rotation, CUDA events around K launches"
+        else:
+            ev_every = max(1, K // 2000)                               # bound the number of event pairs
+            pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                     if k % ev_every == 0 else None for k in range(K)]
+            t0.record(stream)
+            for k in range(K):
+                step(sets[(W0 + k) % n_sets], pairs[k])
+            t1.record(stream)
+            torch.cuda.synchronize()
+            total_ms = t0.elapsed_time(t1)
+            apply_ms = float(np.mean([a.elapsed_time(b) for p in pairs if p is not None for a, b in [p]]))
+            kernel_timing = "CUDA event pair around every apply call (includes host launch gaps)"
+        if dist is not None:
+            dist.barrier()
+        # keep the GPU busy a little longer (untimed) if the region was too short for the clock sampler
+        t_end = time.time() + (0.25 if total_ms < 250 else 0.0)
+        while time.time() < t_end:
+            step(sets[0])
+        torch.cuda.synchronize()
     clk = clocks.stop()
-    apply_ms = float(np.mean([a.elapsed_time(b) for p in pairs if p is not None for a, b in [p]]))
 
     if dist is not None:
         t = torch.tensor([total_ms], device="cuda")
@@ -289,14 +332,15 @@ def run_ours(args):
                 f"{p.name} {p.d_in}->{p.d_out} r{p.rank}" for p in w.projections) + f", router={w.router}",
                 "tokens_per_step_per_gpu": N, "buffer_sets": n_sets,
                 "l2": f"rotation over {n_sets} buffer sets ({n_sets * per_set / 1e6:.0f} MB > 126 MB L2)",
-                "launch": "eager, one C-ABI call per stage"},
+                "launch": ("CUDA graph replay of the C-ABI calls (one call per stage)" if args.launch == "graph"
+                           else "eager, one C-ABI call per stage")},
             "gpu_launches": launches_per_step * K,
             "clocks": clk,
             "e2e": e2e,
             "roofline": {"bound": "hbm", "kernel": "molora_apply (grouped shrink+expand)", "achieved": achieved,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                          "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES.get(name),
-                         "algorithmic_bytes": step_bytes, "kernel_ms": apply_ms,
+                         "algorithmic_bytes": step_bytes, "kernel_ms": apply_ms, "kernel_timing": kernel_timing,
                          "algorithmic_tflops": step_flops / (apply_ms * 1e-3) / 1e12},
             "cpu_baseline": None if args.profile else cpu_baseline(name),
         }
@@ -455,6 +499,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c5-iid"])
+    ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
+                    help="replay the timed steps from CUDA graphs (default) or launch them one by one")
     ap.add_argument("--max-sets", type=int, default=32)
     ap.add_argument("--e2e-steps", type=int, default=50)
     ap.add_argument("--profile", action="store_true",

@@ -105,21 +105,31 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // Split the projections by eligibility for the tensor-core kernel.  For eligible ones both kernels are
     // enqueued and each segment is taken by exactly one of them, chosen on the device from its row count.
-    molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
-    int n_tc = 0, n_cc = 0;
+    molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], dc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
+    int n_tc = 0, n_dc = 0, n_cc = 0;
     for (int i = 0; i < P; ++i) {
         if (N >= kUmmaMinTokens && umma_eligible(projs[i], dt)) tc[n_tc++] = projs[i];
+        else if (decode_eligible(projs[i], dt)) dc[n_dc++] = projs[i];
         else cc[n_cc++] = projs[i];
     }
     molora_status_t st = MOLORA_OK;
     if (n_tc > 0) {
         // With few adapters an under-filled 128-row tile is cheap, so the tensor-core kernel takes every segment
         // and the second launch is saved; with many adapters (up to 256 composite targets) tiny segments are
-        // the norm and go to the CUDA-core kernel instead.
+        // the norm and go to the small-tile kernel instead.
         const int32_t min_rows = C <= kUmmaAllSegmentsMaxC ? 1 : kUmmaMinRows;
         st = launch_apply_umma(tc, n_tc, N, C, offsets, perm, dev_status, min_rows, s);
-        if (st == MOLORA_OK && min_rows > 1) st = launch_apply_rowtile(tc, n_tc, dt, N, C, offsets, perm, min_rows, s);
+        if (st == MOLORA_OK && min_rows > 1) {
+            molora_proj_desc_t small_dc[MOLORA_MAX_PROJECTIONS], small_cc[MOLORA_MAX_PROJECTIONS];
+            int a = 0, b = 0;
+            for (int i = 0; i < n_tc; ++i) {
+                if (decode_eligible(tc[i], dt)) small_dc[a++] = tc[i]; else small_cc[b++] = tc[i];
+            }
+            if (a > 0) st = launch_apply_decode(small_dc, a, N, C, offsets, perm, min_rows, s);
+            if (st == MOLORA_OK && b > 0) st = launch_apply_rowtile(small_cc, b, dt, N, C, offsets, perm, min_rows, s);
+        }
     }
+    if (st == MOLORA_OK && n_dc > 0) st = launch_apply_decode(dc, n_dc, N, C, offsets, perm, INT32_MAX, s);
     if (st == MOLORA_OK && n_cc > 0) st = launch_apply_rowtile(cc, n_cc, dt, N, C, offsets, perm, INT32_MAX, s);
     return st;
 }

@@ -127,6 +127,27 @@ __device__ __forceinline__ bool find_tile(const int32_t* __restrict__ offsets, i
     return false;
 }
 
+// Same lookup on a copy of offsets[0..C] that already sits in shared memory (one memory round trip for the
+// whole table instead of one per segment scanned).
+__device__ __forceinline__ bool find_tile_smem(const int32_t* offs, int C, int tile_rows, int tile, int min_rows,
+                                               int max_rows, int& seg, int& row0, int& rows)
+{
+    int base = 0;
+    for (int c = 0; c < C; ++c) {
+        const int prev = offs[c], next = offs[c + 1];
+        const int n = next - prev;
+        const int tiles = (n >= min_rows && n < max_rows) ? (n + tile_rows - 1) / tile_rows : 0;
+        if (tile < base + tiles) {
+            seg = c;
+            row0 = prev + (tile - base) * tile_rows;
+            rows = min(tile_rows, next - row0);
+            return true;
+        }
+        base += tiles;
+    }
+    return false;
+}
+
 // Host launchers implemented in the .cu files (stream already unwrapped).
 molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M, int32_t* r_out,
                                    uint32_t* dev_status, cudaStream_t s);
@@ -152,6 +173,12 @@ bool umma_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                   const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
                                   cudaStream_t s);
+
+// mma.sync path for decode-sized calls (bf16, rank 16/32/64, d_in and d_out multiples of 32); takes the segments
+// with fewer than max_rows rows.
+bool decode_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
+molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
+                                    const int32_t* offsets, const int32_t* perm, int32_t max_rows, cudaStream_t s);
 
 // Path selection: a segment goes to the tensor-core kernel when it has at least kUmmaMinRows rows and the call
 // has at least kUmmaMinTokens tokens (known on the host); everything else runs on the CUDA-core kernel.

@@ -93,11 +93,16 @@ __global__ void __launch_bounds__(WARPS * 32) route_gate_mma_kernel(const __nv_b
     const __nv_bfloat16* xa = x + rowA * ldx + q * 8;
     const __nv_bfloat16* xb = x + rowB * ldx + q * 8;
 
-    float acc[NT][4];
+    // one accumulator fragment per (n-tile, term, k-step parity): independent MMA chains hide the MMA latency
+    float acc3[NT][3][2][4];
 #pragma unroll
     for (int n = 0; n < NT; ++n)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[n][i] = 0.f;
+        for (int t = 0; t < 3; ++t)
+#pragma unroll
+            for (int s = 0; s < 2; ++s)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc3[n][t][s][i] = 0.f;
 
     const int chunks = (d + KC - 1) / KC;
     auto copy_image = [&](int buf, int ch) {
@@ -161,7 +166,7 @@ __global__ void __launch_bounds__(WARPS * 32) route_gate_mma_kernel(const __nv_b
                             for (int t = 0; t < 3; ++t) {
                                 const uint2 bb =
                                     *reinterpret_cast<const uint2*>(&Gs[buf][t][n * 8 + g][b * 32 + s * 16 + q * 4]);
-                                mma_bf16_16816(acc[n], a, bb.x, bb.y);
+                                mma_bf16_16816(acc3[n][t][s], a, bb.x, bb.y);
                             }
                         }
                     }
@@ -170,6 +175,15 @@ __global__ void __launch_bounds__(WARPS * 32) route_gate_mma_kernel(const __nv_b
             }
         }
     }
+
+    // fold the partial fragments in a fixed order: ((lo + mid) + hi), even k-steps then odd
+    float acc[NT][4];
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            acc[n][i] = ((acc3[n][2][0][i] + acc3[n][2][1][i]) + (acc3[n][1][0][i] + acc3[n][1][1][i])) +
+                        (acc3[n][0][0][i] + acc3[n][0][1][i]);
 
     // fragment -> logits: acc[n][0..1] = (row g, c = 8n + 2q, +1), acc[n][2..3] = (row g + 8, same columns)
 #pragma unroll

@@ -344,3 +344,20 @@ def test_forward_host_matches_oracle(name):
         ref, _ = oracle.apply(w.inputs[p.x_key], p.y, p.A, p.B, r_ref)
         assert_close(y.float().numpy().astype(np.float64)[keep], ref[keep], what=f"forward_host {name}/{p.name}")
     assert int(status.item()) == 0
+
+
+# ------------------------------------------------------------------ decode path (N < 1024, 32-row tiles on mma.sync)
+@pytest.mark.parametrize("rank", [16, 32, 64])
+def test_decode_path_segment_size_sweep(rank):
+    sizes = [0, 1, 7, 15, 16, 17, 31, 32, 33, 47, 64, 65, 97]
+    r = W.segment_sizes_routing(sizes)
+    assert r.size < 1024
+    w = W.random_problem(300 + rank, r.size, len(sizes), 1024, 320, rank, "bf16", r=r)
+    run_and_check(w, scale=0.5)
+
+
+@pytest.mark.parametrize("N,C,d_in,d_out,rank", [(1, 1, 32, 32, 16), (256, 8, 2048, 6144, 16), (100, 2, 6144, 2048, 32),
+                                                 (700, 3, 256, 1024, 64), (64, 64, 512, 96, 16)])
+def test_decode_path_shapes(N, C, d_in, d_out, rank):
+    w = W.random_problem(N + rank + 7, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.1 if N > 10 else 0.0)
+    run_and_check(w)
