@@ -110,12 +110,14 @@ def build_sets(W, torch, name, n_sets, rank):
             return torch.from_numpy(W.bf16_bits(a)).cuda().view(torch.bfloat16)
         return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
 
+    from paper_2603_15965_b200.shard import rank_batches
+    batches = rank_batches(rank, max(1, int(os.environ.get("WORLD_SIZE", "1"))), n_sets)   # disjoint across ranks
     sets, w0 = [], None
     for b in range(n_sets):
         if name == "c2":
-            w = W.get("c2", batch=rank * n_sets + b)
+            w = W.get("c2", batch=batches[b])
         elif name == "c3":
-            w = W.get("c3", layer=rank * n_sets + b)
+            w = W.get("c3", layer=batches[b])
         else:
             w = W.get(name) if b == 0 else None
         if w is None:   # large configs: clone batch 0 into distinct buffers (same values, distinct addresses)
@@ -178,6 +180,7 @@ def run_ours(args):
     import torch
     import paper_2603_15965_b200 as M
     import paper_2603_15965_b200.binding  # noqa: F401
+    from paper_2603_15965_b200 import shard
     from paper_2603_15965_b200 import workloads as W
     from paper_2603_15965_b200.binding import pack_proj_descs
     from paper_2603_15965_b200.build import build_library
@@ -310,12 +313,9 @@ def run_ours(args):
         torch.cuda.synchronize()
     clk = clocks.stop()
 
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = shard.max_over_ranks(total_ms, dist, device="cuda")     # the slowest rank defines the step
     ms_per_step = total_ms / K
-    value = world * N / (ms_per_step * 1e-3)
+    value = shard.aggregate_tokens_per_s(N, world, ms_per_step)
 
     # ------------------------------------------------------------------ end to end with host buffers
     e2e = None if args.profile else run_e2e(args, torch, M, w, sets, shared, world, dist)
