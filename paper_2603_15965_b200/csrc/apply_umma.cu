@@ -164,7 +164,13 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     if (pj.rank != R) return;
     int seg, row0, rows;
     const uint32_t S = cluster_nctarank(), crank = cluster_ctarank();   // CTAs sharing this tile, and my slice
-    if (!find_tile(prm.offsets, prm.C, kTileM, blockIdx.x / S, prm.min_rows, INT32_MAX, seg, row0, rows)) return;
+    {
+        // bring the segment table on chip in one memory round trip, then look the tile up there
+        __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
+        for (int i = threadIdx.x; i <= prm.C; i += kUmmaThreads) offs_s[i] = __ldg(prm.offsets + i);
+        __syncthreads();
+        if (!find_tile_smem(offs_s, prm.C, kTileM, blockIdx.x / S, prm.min_rows, INT32_MAX, seg, row0, rows)) return;
+    }
 
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
