@@ -47,6 +47,7 @@ struct DecodeParams {
     const int32_t* offsets;
     const int32_t* perm;
     int32_t N;
+    int32_t passes;                       // expand passes per CTA: a cluster covers S * passes * (8 warps * GD * 32) columns
     int32_t P, C, max_rows;               // segments with at least max_rows rows belong to the tensor-core kernel
 #ifdef MOLORA_TRACE
     long long* trace;                     // development builds only: clock64 stamps per CTA
@@ -61,8 +62,18 @@ struct DecodeParams {
             if (cta < 2048) prm.trace[cta * 16 + (slot)] = (slot) == 0 ? (long long)clock64() : (long long)clock64(); \
         }                                                                                              \
     } while (0)
+#define DEC_GT(slot)                                                                                   \
+    do {                                                                                               \
+        if (prm.trace != nullptr && threadIdx.x == 0) {                                                \
+            const int cta = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;            \
+            long long t_;                                                                              \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                     \
+            if (cta < 2048) prm.trace[cta * 16 + (slot)] = t_;                                         \
+        }                                                                                              \
+    } while (0)
 #else
 #define DEC_TR(slot) do { } while (0)
+#define DEC_GT(slot) do { } while (0)
 #endif
 
 __device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
@@ -112,12 +123,13 @@ __global__ void __launch_bounds__(kDecThreads, 2) apply_decode_kernel(const __gr
     constexpr int kDecKD = Cfg::KD, kDecGD = Cfg::GD, kDecColsPerCta = Cfg::COLS_PER_CTA;
 
     DEC_TR(0);
+    DEC_GT(14);
     const molora_proj_desc_t& pd = prm.p[blockIdx.y];
     if (pd.rank != R) return;
     const uint32_t S = cluster_nctarank(), crank = cluster_ctarank();
     // blockIdx.z selects the cluster's slice of d_out (S * 768 columns); projections with fewer slices leave early
     const int ngroups = pd.d_out / 32;
-    const int G0 = (int)blockIdx.z * (int)S * (kDecColsPerCta / 32);
+    const int G0 = (int)blockIdx.z * (int)S * prm.passes * (kDecColsPerCta / 32);
     if (G0 >= ngroups) return;
     // One memory round trip brings the segment table and (for small calls) the whole permutation on chip.
     __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
@@ -196,7 +208,7 @@ __global__ void __launch_bounds__(kDecThreads, 2) apply_decode_kernel(const __gr
 
     DEC_TR(2);
     // my output groups: CTA q owns a contiguous run of groups, its warps interleave inside it
-    const int G1 = min(ngroups, G0 + (int)S * (kDecColsPerCta / 32));
+    const int G1 = min(ngroups, G0 + (int)S * prm.passes * (kDecColsPerCta / 32));
     const int per_cta = (G1 - G0 + (int)S - 1) / (int)S;
     const int g_lo = G0 + (int)crank * per_cta, g_hi = min(G1, g_lo + per_cta);
 
@@ -397,7 +409,28 @@ __global__ void __launch_bounds__(kDecThreads, 2) apply_decode_kernel(const __gr
         const int grp = g_lo + warp + j * kDecWarps;
         if (grp < g_hi) expand_group(j, grp, yv[j]);
     }
+    // wide projections: further passes of GD groups per warp, one extra memory round trip each
+    for (int gbase = g_lo + warp + kDecGD * kDecWarps; gbase < g_hi; gbase += kDecGD * kDecWarps) {
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < kDecGD; ++j) {
+            const int grp = gbase + j * kDecWarps;
+            if (grp < g_hi) {
+                stage_B(j, grp);
+                load_y(yv[j], grp);
+            }
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < kDecGD; ++j) {
+            const int grp = gbase + j * kDecWarps;
+            if (grp < g_hi) expand_group(j, grp, yv[j]);
+        }
+    }
     DEC_TR(13);
+    DEC_GT(15);
 }
 
 bool decode_eligible(const molora_proj_desc_t& p, molora_dtype_t dt)
@@ -427,7 +460,7 @@ static cudaError_t decode_launch(const DecodeParams& prm, int64_t N, int split, 
     int max_dout = 0;
     for (int i = 0; i < prm.P; ++i)
         if (prm.p[i].rank == R) max_dout = std::max(max_dout, prm.p[i].d_out);
-    const int nslices = ceil_div(max_dout, split * DecCfg<R>::COLS_PER_CTA);     // clusters along d_out (grid.z)
+    const int nslices = ceil_div(max_dout, split * prm.passes * DecCfg<R>::COLS_PER_CTA);   // clusters along d_out (grid.z)
     cfg.gridDim = dim3((unsigned)(tiles * split), (unsigned)prm.P, (unsigned)nslices);
     cfg.blockDim = dim3(kDecThreads, 1, 1);
     cfg.dynamicSmemBytes = decode_smem_bytes<R>();
@@ -464,11 +497,14 @@ molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, 
 #ifdef MOLORA_TRACE
     prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
 #endif
-    // CTAs per tile along d_in: up to 4 while every warp still gets a k block
-    int split = kDecMaxSplit;
-    const char* env = getenv("MOLORA_DECODE_SPLIT");                  // tuning override
+    // CTAs per tile along d_in: 3 (one wave of CTAs for a 256-token layer of 7 projections), fewer while a warp
+    // would be left without a k block; wide projections take up to 3 expand passes per CTA instead of more CTAs.
+    int split = 3;
+    const char* env = getenv("MOLORA_DECODE_SPLIT");                  // tuning overrides
     if (env != nullptr) split = std::max(1, std::min(atoi(env), kDecMaxSplit));
     while (split > 1 && min_kb / split < kDecWarps) --split;
+    const char* envp = getenv("MOLORA_DECODE_PASSES");
+    prm.passes = envp != nullptr ? std::max(1, atoi(envp)) : 3;
     cudaError_t e = cudaSuccess;
     if (has[0] && e == cudaSuccess) e = decode_launch<16>(prm, N, split, s);
     if (has[1] && e == cudaSuccess) e = decode_launch<32>(prm, N, split, s);
