@@ -73,6 +73,7 @@ struct UmmaParams {
     const int32_t* perm;
     uint32_t* dev_status;
     int32_t P, C, min_rows;
+    int32_t tile_rows;    // positions per tile: 128, or fewer (the MMA tile stays 128 lanes) to spread a small call over more SMs
 #ifdef MOLORA_TRACE
     long long* trace;     // development builds only: clock64 stamps of CTA 0, [role][iteration][slot]
 #endif
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
         for (int i = threadIdx.x; i <= prm.C; i += kUmmaThreads) offs_s[i] = __ldg(prm.offsets + i);
         __syncthreads();
-        if (!find_tile_smem(offs_s, prm.C, kTileM, blockIdx.x / S, prm.min_rows, INT32_MAX, seg, row0, rows)) return;
+        if (!find_tile_smem(offs_s, prm.C, prm.tile_rows, blockIdx.x / S, prm.min_rows, INT32_MAX, seg, row0, rows)) return;
     }
 
     const uint32_t raw = smem_u32(smem_raw);
@@ -543,6 +544,11 @@ bool umma_eligible(const molora_proj_desc_t& p, molora_dtype_t dt)
            (p.d_out % kChunkCols) == 0;
 }
 
+struct UmmaPlan {
+    int split;       // CTAs per tile (cluster size)
+    int tile_rows;   // positions per tile
+};
+
 template <int R>
 static void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int64_t tiles, int P, int split,
                                cudaStream_t s)
@@ -560,8 +566,10 @@ static void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* att
 }
 
 template <int R>
-static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, int split, cudaStream_t s)
+static cudaError_t umma_launch(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStream_t s)
 {
+    const int split = plan.split;
+    prm.tile_rows = plan.tile_rows;
     using Cfg = UmmaCfg<R>;
     static bool configured = false;
     if (!configured) {
@@ -570,7 +578,7 @@ static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, int split, cuda
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const int64_t tiles = ceil_div64(N, kTileM) + prm.C;
+    const int64_t tiles = ceil_div64(N, prm.tile_rows) + prm.C;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     fill_launch_config<R>(cfg, attr, tiles, prm.P, split, s);
@@ -598,29 +606,46 @@ static int max_active_clusters(int split)
 // a cluster of 2 or 4 CTAs.  Pick the split with the smallest estimated time: waves of resident clusters times
 // (work per CTA, which shrinks with the split, plus a fixed per-CTA cost and the cost of the exchange).
 template <int R>
-static int choose_split_for_rank(const UmmaParams& prm, int64_t N)
+static UmmaPlan choose_split_for_rank(const UmmaParams& prm, int64_t N)
 {
-    int min_kx = INT32_MAX;
-    int64_t tiles = 0;
+    int min_kx = INT32_MAX, nproj = 0;
     for (int i = 0; i < prm.P; ++i) {
         if (prm.p[i].rank != R) continue;
         min_kx = std::min(min_kx, prm.p[i].d_in / kChunkCols);
-        tiles += ceil_div64(N, kTileM) + prm.C / 2;           // expected: every segment ends in a partial tile
+        ++nproj;
     }
-    const char* env = getenv("MOLORA_UMMA_SPLIT");          // tuning override
-    int best = 1;
-    if (env != nullptr) {
-        best = std::max(1, std::min(atoi(env), kMaxSplit));
+    // expected tiles: every segment ends in a partial tile
+    auto tiles_for = [&](int rows) { return (ceil_div64(N, rows) + prm.C / 2) * nproj; };
+    auto cost_for = [&](int rows, int split, double& waves) {
+        const int resident = max_active_clusters<R>(split);
+        waves = (double)((tiles_for(rows) + resident - 1) / resident);
+        return waves * ((rows / 128.0) / split + 0.15 + (split > 1 ? 0.10 : 0.0));
+    };
+    UmmaPlan best = {1, kTileM};
+    const char* env = getenv("MOLORA_UMMA_SPLIT");          // tuning overrides
+    const char* envr = getenv("MOLORA_UMMA_TILE_ROWS");
+    if (env != nullptr || envr != nullptr) {
+        if (env != nullptr) best.split = std::max(1, std::min(atoi(env), kMaxSplit));
+        if (envr != nullptr) best.tile_rows = std::max(32, std::min(atoi(envr), kTileM));
     } else {
-        double best_cost = 1e30;
+        double best_cost = 1e30, best_waves = 0;
         for (int split = 1; split <= kMaxSplit; ++split) {    // cluster sizes need not be powers of two
-            const int resident = max_active_clusters<R>(split);
-            const double waves = (double)((tiles + resident - 1) / resident);
-            const double cost = waves * (1.0 / split + 0.15 + (split > 1 ? 0.10 : 0.0));
-            if (cost < best_cost - 1e-9) { best_cost = cost; best = split; }
+            double waves;
+            const double cost = cost_for(kTileM, split, waves);
+            if (cost < best_cost - 1e-9) { best_cost = cost; best_waves = waves; best = {split, kTileM}; }
+        }
+        // A call that does not even fill one wave can use shorter tiles (the MMA tile keeps 128 lanes, the extra
+        // lanes idle) to put more SMs to work, as long as everything still fits in one wave.
+        if (best_waves <= 1.0 && tiles_for(kTileM) * best.split < 0.85 * 148) {
+            for (int rows = 96; rows >= 64; rows -= 32)
+                for (int split = 1; split <= kMaxSplit; ++split) {
+                    double waves;
+                    const double cost = cost_for(rows, split, waves);
+                    if (waves <= 1.0 && cost < best_cost - 1e-9) { best_cost = cost; best = {split, rows}; }
+                }
         }
     }
-    while (best > 1 && min_kx / best < 4) --best;            // keep at least four chunks of d_in per CTA
+    while (best.split > 1 && min_kx / best.split < 4) --best.split;   // keep at least four chunks of d_in per CTA
     return best;
 }
 
@@ -631,8 +656,15 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
     if (N == 0 || P == 0) return MOLORA_OK;
     UmmaParams prm;
     bool has[3] = {false, false, false};
+    // CTAs are dispatched projection by projection (blockIdx.y): put the projections that move the most bytes
+    // per tile first, so that the last, partly filled wave consists of the cheap tiles.
+    int order[MOLORA_MAX_PROJECTIONS];
+    for (int i = 0; i < P; ++i) order[i] = i;
+    std::stable_sort(order, order + P, [&](int a, int b) {
+        return (int64_t)projs[a].d_in + 2 * (int64_t)projs[a].d_out > (int64_t)projs[b].d_in + 2 * (int64_t)projs[b].d_out;
+    });
     for (int i = 0; i < P; ++i) {
-        const molora_proj_desc_t& d = projs[i];
+        const molora_proj_desc_t& d = projs[order[i]];
         UmmaProj& u = prm.p[i];
         const CUtensorMapSwizzle wswz = d.rank == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
                                         : d.rank == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
@@ -657,6 +689,7 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
     prm.P = P;
     prm.C = C;
     prm.min_rows = min_rows;
+    prm.tile_rows = kTileM;
 #ifdef MOLORA_TRACE
     prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
 #endif
