@@ -173,6 +173,16 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t *projs, int32_t P,
                                      uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Failure-detection self-test.  Every device-side wait of the tensor-core apply kernel (on an mbarrier that a
+ * producer warp, the tensor core or a peer CTA of the cluster completes) is bounded: a waiter that gives up sets
+ * MOLORA_DEV_TIMEOUT in the status word and an abort flag after which all waits of the CTA fall through, so the
+ * kernel returns and the context stays usable.  This entry point exercises exactly that code on a barrier that
+ * nothing ever completes, with a limit of `limit_cycles` SM cycles (1 .. 2e9): afterwards *dev_status has
+ * MOLORA_DEV_TIMEOUT set, result[0] == 1 (abort flag raised) and result[1] == 1 (a second wait fell through).
+ * dev_status: device uint32; result: device int32[2].  Nothing faults, traps or spins without bound. */
+molora_status_t molora_selftest_bounded_wait(uint32_t *dev_status, int64_t limit_cycles, int32_t *result, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * The whole path on HOST activations (one layer: route -> group -> apply for P projections), for callers
  * whose activations live in host memory.  Everything is enqueued on `stream` in this order: host-to-device
  * copies of the routing source and of every distinct x and every y into `arena`, the router, the grouping,

@@ -74,6 +74,8 @@ def load_library():
     lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp]
     lib.molora_route_gate_noalloc.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp]
     lib.molora_route_gate_noalloc.restype = ctypes.c_int
+    lib.molora_selftest_bounded_wait.argtypes = [vp, i64, vp, vp]
+    lib.molora_selftest_bounded_wait.restype = ctypes.c_int
     lib.molora_group_workspace_bytes.restype = sz
     lib.molora_group_workspace_bytes.argtypes = [i64, i32]
     lib.molora_group.argtypes = [vp, i64, i32, vp, vp, vp, vp, sz, vp, vp]
@@ -201,6 +203,17 @@ def molora_route_gate_noalloc(x: torch.Tensor, G: torch.Tensor, bias: Optional[t
         _ptr(x), _dtype_code(x), N, d, ldx, _ptr(G), _ptr(bias), C, _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
         _stream(stream)))
     return r_out
+
+
+def molora_selftest_bounded_wait(limit_cycles: int = 200000, stream=None) -> Tuple[int, int, int]:
+    """Run the bounded-wait self-test; returns (status word, abort flag, second wait fell through)."""
+    lib = load_library()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    result = torch.zeros(2, dtype=torch.int32, device="cuda")
+    _check("molora_selftest_bounded_wait", lib.molora_selftest_bounded_wait(_ptr(status), int(limit_cycles), _ptr(result),
+                                                                            _stream(stream)))
+    torch.cuda.synchronize()
+    return int(status.item()), int(result[0].item()), int(result[1].item())
 
 
 def molora_group_workspace_bytes(N: int, C: int) -> int:

@@ -153,6 +153,13 @@ molora_status_t molora_apply(const void* x, int64_t ldx, void* y, int64_t ldy, m
     return molora_apply_batched(&p, 1, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, stream);
 }
 
+molora_status_t molora_selftest_bounded_wait(uint32_t* dev_status, int64_t limit_cycles, int32_t* result, void* stream)
+{
+    if (dev_status == nullptr || result == nullptr || limit_cycles < 1 || limit_cycles > 2000000000LL)
+        return MOLORA_ERR_INVALID_ARG;
+    return launch_bounded_wait_selftest(dev_status, limit_cycles, result, static_cast<cudaStream_t>(stream));
+}
+
 // ---------------------------------------------------------------------------------------------- host-buffer path
 namespace {
 

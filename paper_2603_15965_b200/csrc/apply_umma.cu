@@ -123,14 +123,15 @@ struct Ctrl {                         // lives in shared memory after the tiles
 static_assert(sizeof(Ctrl) <= 1024, "control block must fit its slot");
 
 // Bounded wait on an mbarrier phase.  Falls through once the CTA has aborted.
-__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* dev_status)
+__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* dev_status,
+                                         long long limit = kTimeoutCycles)
 {
     if (mbar_try_wait(bar, parity)) return;
     if (*abort_flag) return;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (*abort_flag) return;
-        if (clock64() - t0 > kTimeoutCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             if (dev_status != nullptr) atomicOr(dev_status, MOLORA_DEV_TIMEOUT);
             return;
@@ -503,6 +504,36 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     if (S > 1) cluster_sync_all();     // no CTA retires while a peer could still touch its shared memory
     if (tid == 0) MOLORA_TR(3, 0, 5);
     MOLORA_TR_CTA(1);
+}
+
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing ever arrives on, with a limit of
+// `limit_cycles`.  The wait must give up, raise the abort flag and MOLORA_DEV_TIMEOUT, and the kernel must return
+// normally (no trap, no hang): this is the exit every pipeline role takes if a peer never shows up.
+__global__ void bounded_wait_selftest_kernel(uint32_t* dev_status, long long limit_cycles, int32_t* result)
+{
+    __shared__ uint64_t never;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&never), 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    wait_bar(smem_u32(&never), 0, &abort_flag, dev_status, limit_cycles);
+    __syncthreads();
+    // a second wait after the abort must fall through at once
+    const long long t0 = clock64();
+    wait_bar(smem_u32(&never), 0, &abort_flag, dev_status, limit_cycles);
+    if (threadIdx.x == 0) {
+        result[0] = abort_flag;
+        result[1] = (clock64() - t0) < limit_cycles ? 1 : 0;
+    }
+}
+
+molora_status_t launch_bounded_wait_selftest(uint32_t* dev_status, int64_t limit_cycles, int32_t* result, cudaStream_t s)
+{
+    bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(dev_status, limit_cycles, result);
+    return cuda_ok(cudaGetLastError());
 }
 
 // ------------------------------------------------------------------------------------------------ host side

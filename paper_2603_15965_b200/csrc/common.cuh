@@ -180,6 +180,8 @@ bool decode_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
 molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                     const int32_t* offsets, const int32_t* perm, int32_t max_rows, cudaStream_t s);
 
+molora_status_t launch_bounded_wait_selftest(uint32_t* dev_status, int64_t limit_cycles, int32_t* result, cudaStream_t s);
+
 // Path selection: a segment goes to the tensor-core kernel when it has at least kUmmaMinRows rows and the call
 // has at least kUmmaMinTokens tokens (known on the host); everything else runs on the CUDA-core kernel.
 constexpr int32_t kUmmaMinRows = 32;

@@ -361,3 +361,13 @@ def test_decode_path_segment_size_sweep(rank):
 def test_decode_path_shapes(N, C, d_in, d_out, rank):
     w = W.random_problem(N + rank + 7, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.1 if N > 10 else 0.0)
     run_and_check(w)
+
+
+# ------------------------------------------------------------------ failure detection: bounded device-side waits
+def test_bounded_wait_gives_up_cleanly_and_context_stays_usable():
+    # a wait on a barrier that nothing completes must time out (here after 2e5 cycles ~ 0.1 ms), report it in the
+    # status word and let the kernel return; the context must then still run work correctly
+    status, aborted, fell_through = M.molora_selftest_bounded_wait(200000)
+    assert status & 4 and aborted == 1 and fell_through == 1
+    w = W.random_problem(31, 1100, 3, 128, 128, 16, "bf16")
+    run_and_check(w)
