@@ -85,8 +85,9 @@ molora_status_t molora_route_vocab(const int32_t *ids, int64_t N, const int32_t 
  * r_out    device int32[N]
  * logits_out  device fp32 [N, C] or NULL (the logits as the kernel accumulated them, fp32)
  * ws, ws_bytes  device scratch of at least molora_route_gate_workspace_bytes(xdt, d, C) bytes, 16-byte aligned
- *               (NULL when that is 0).  For bf16 x and C > 4 the kernel runs on the tensor cores and keeps there a
- *               three-term bf16 split of G (hi + mid + lo = 24 mantissa bits), rebuilt on every call.
+ *               (NULL when that is 0).  For bf16 x and C > 4 the kernel runs on the tensor cores (tcgen05 when N >= 1024
+ *               and d is a multiple of 64, mma.sync otherwise) and keeps there a three-term bf16 split of G
+ *               (hi + mid + lo = 24 mantissa bits), rebuilt on every call.
  * Products are exact in fp32 for bf16 x; accumulation is fp32 in a fixed, token-independent order. */
 size_t molora_route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
 molora_status_t molora_route_gate(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float *G,

@@ -38,7 +38,9 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "pipeline.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace molora {
 
@@ -57,7 +59,6 @@ constexpr int kTileBytes = kTileM * 128;    // 16 KB: X or Y chunk
 constexpr int kDBufs = 4;                   // expand accumulators in flight (64 TMEM columns each)
 constexpr int kTmemCols = 512;
 constexpr int kMaxSplit = 4;                // largest cluster a tile is split over
-constexpr long long kTimeoutCycles = 2000000000LL;
 
 struct UmmaProj {
     CUtensorMap tm_a, tm_b;
@@ -121,40 +122,6 @@ struct Ctrl {                         // lives in shared memory after the tiles
     alignas(16) int32_t rows[kTileM];
 };
 static_assert(sizeof(Ctrl) <= 1024, "control block must fit its slot");
-
-// Bounded wait on an mbarrier phase.  Falls through once the CTA has aborted.
-__device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* dev_status,
-                                         long long limit = kTimeoutCycles)
-{
-    if (mbar_try_wait(bar, parity)) return;
-    if (*abort_flag) return;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (*abort_flag) return;
-        if (clock64() - t0 > limit) {
-            *abort_flag = 1;
-            if (dev_status != nullptr) atomicOr(dev_status, MOLORA_DEV_TIMEOUT);
-            return;
-        }
-    }
-}
-
-// Same, for a barrier that CTAs of the cluster arrive on remotely (acquire at cluster scope).
-__device__ __forceinline__ void wait_bar_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                                 uint32_t* dev_status)
-{
-    if (mbar_try_wait_cluster(bar, parity)) return;
-    if (*abort_flag) return;
-    const long long t0 = clock64();
-    while (!mbar_try_wait_cluster(bar, parity)) {
-        if (*abort_flag) return;
-        if (clock64() - t0 > kTimeoutCycles) {
-            *abort_flag = 1;
-            if (dev_status != nullptr) atomicOr(dev_status, MOLORA_DEV_TIMEOUT);
-            return;
-        }
-    }
-}
 
 template <int R>
 __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __grid_constant__ UmmaParams prm)
@@ -537,38 +504,6 @@ molora_status_t launch_bounded_wait_selftest(uint32_t* dev_status, int64_t limit
 }
 
 // ------------------------------------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = []() -> EncodeTiledFn {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// 2-D bf16 tensor map: `cols` contiguous elements per row, `rows` rows of pitch `ld` elements.
-static bool make_map(CUtensorMap* m, const void* ptr, uint64_t cols, uint64_t rows, uint64_t ld, uint32_t box_cols,
-                     uint32_t box_rows, CUtensorMapSwizzle swz)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (fn == nullptr) return false;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {ld * 2};
-    const cuuint32_t box[2] = {box_cols, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 bool umma_eligible(const molora_proj_desc_t& p, molora_dtype_t dt)
 {
     return dt == MOLORA_BF16 && (p.rank == 16 || p.rank == 32 || p.rank == 64) && (p.d_in % kChunkCols) == 0 &&
@@ -699,8 +634,8 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
         UmmaProj& u = prm.p[i];
         const CUtensorMapSwizzle wswz = d.rank == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
                                         : d.rank == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-        bool ok = make_map(&u.tm_a, d.A, d.rank, (uint64_t)C * d.d_in, d.rank, d.rank, kChunkCols, wswz);
-        ok = ok && make_map(&u.tm_b, d.B, d.d_out, (uint64_t)C * d.rank, d.d_out, kChunkCols, d.rank,
+        bool ok = make_tensor_map_bf16_2d(&u.tm_a, d.A, d.rank, (uint64_t)C * d.d_in, d.rank, d.rank, kChunkCols, wswz);
+        ok = ok && make_tensor_map_bf16_2d(&u.tm_b, d.B, d.d_out, (uint64_t)C * d.rank, d.d_out, kChunkCols, d.rank,
                             CU_TENSOR_MAP_SWIZZLE_128B);
         if (!ok) return MOLORA_ERR_CUDA;
         u.x = static_cast<const __nv_bfloat16*>(d.x);

@@ -151,6 +151,12 @@ __device__ __forceinline__ bool find_tile_smem(const int32_t* offs, int C, int t
 // Host launchers implemented in the .cu files (stream already unwrapped).
 molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M, int32_t* r_out,
                                    uint32_t* dev_status, cudaStream_t s);
+// tcgen05 gate (bf16 activations, C > 4, d a multiple of 64, at least 1024 tokens).
+bool gate_umma_eligible(int64_t N, int32_t d, int32_t C);
+size_t route_gate_umma_workspace_bytes(int32_t d, int32_t C);
+molora_status_t launch_route_gate_umma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
+                                       const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
+                                       cudaStream_t s);
 size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
 molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
                                   const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,

@@ -328,7 +328,9 @@ static molora_status_t gate_dispatch(const void* x, int64_t N, int d, int64_t ld
 
 size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
 {
-    return xdt == MOLORA_BF16 ? route_gate_mma_workspace_bytes(d, C) : 0;
+    if (xdt != MOLORA_BF16) return 0;
+    const size_t a = route_gate_mma_workspace_bytes(d, C), b = route_gate_umma_workspace_bytes(d, C);
+    return a > b ? a : b;      // which kernel runs depends on N, which this query does not know
 }
 
 molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
@@ -336,6 +338,8 @@ molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, 
                                   cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
+    if (xdt == MOLORA_BF16 && gate_umma_eligible(N, d, C))
+        return launch_route_gate_umma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
     if (xdt == MOLORA_BF16 && C > 4) return launch_route_gate_mma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
     if (xdt == MOLORA_BF16) return gate_dispatch<__nv_bfloat16>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
     return gate_dispatch<float>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);

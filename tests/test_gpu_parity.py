@@ -371,3 +371,24 @@ def test_bounded_wait_gives_up_cleanly_and_context_stays_usable():
     assert status & 4 and aborted == 1 and fell_through == 1
     w = W.random_problem(31, 1100, 3, 128, 128, 16, "bf16")
     run_and_check(w)
+
+
+@pytest.mark.parametrize("N,d,C", [(1024, 64, 5), (1500, 4096, 16), (2049, 2048, 8), (1100, 512, 32), (1300, 1024, 17)])
+def test_route_gate_tensor_core_paths(N, d, C):
+    # at least 1024 tokens and C > 4: the tcgen05 gate; logits and argmax against the oracle, bias included
+    rng = np.random.default_rng(N + d + C)
+    x = W.round_to_bf16(rng.standard_normal((N, d), dtype=np.float32))
+    G = (rng.standard_normal((d, C)) * d ** -0.5).astype(np.float32)
+    bias = (rng.standard_normal(C) * 0.1).astype(np.float32)
+    r_ref, z_ref, margin = oracle.route_gate(x, G, bias)
+    logits = torch.empty(N, C, dtype=torch.float32, device="cuda")
+    r = M.molora_route_gate(dev_tensor(x, "bf16"), dev_tensor(G, "f32"), dev_tensor(bias, "f32"), logits_out=logits)
+    assert_close(to_f64(logits), z_ref, 1e-4, 1e-4, what="gate logits")
+    keep = margin >= 1e-3
+    assert np.array_equal(r.cpu().numpy()[keep], r_ref[keep])
+    # unit vectors read rows of G exactly (hi + mid + lo reconstructs every fp32 value)
+    if d <= 1024:
+        eye = np.zeros((N, d), np.float32)
+        eye[np.arange(N), np.arange(N) % d] = 1.0
+        M.molora_route_gate(dev_tensor(eye, "bf16"), dev_tensor(G, "f32"), logits_out=logits)
+        assert np.array_equal(logits.cpu().numpy(), G[np.arange(N) % d])
