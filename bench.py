@@ -30,7 +30,7 @@ METRIC = "routed_lora_tokens_per_s"
 UNIT = "tokens/s"
 L2_BYTES = 126e6
 # dram__bytes_read.sum + dram__bytes_write.sum per apply launch from the committed ncu capture (profiles/), by workload
-NCU_TRAFFIC_BYTES = {"c2": 34.13e6, "c3": 26.78e6, "c5": 605.3e6}
+NCU_TRAFFIC_BYTES = {"c2": 34.13e6, "c3": 27.09e6, "c5": 605.3e6}
 
 
 def measured_peaks():
@@ -171,8 +171,10 @@ def marshal_step(lib, w, s, shared, stream_handle):
     group = partial(lib.molora_group, vp(r.data_ptr()), i64(N), i32(C), vp(s["counts"].data_ptr()),
                     vp(s["offsets"].data_ptr()), vp(s["perm"].data_ptr()), None, ctypes.c_size_t(0), None, st)
     arr, n, c, dt = s["packed"]
+    aws = shared.get("apply_ws")
     apply = partial(lib.molora_apply_batched, arr, i32(len(arr)), dt, i64(n), i32(c), vp(s["offsets"].data_ptr()),
-                    vp(s["perm"].data_ptr()), None, ctypes.c_size_t(0), vp(shared["status"].data_ptr()), st)
+                    vp(s["perm"].data_ptr()), vp(aws.data_ptr()) if aws is not None else None,
+                    ctypes.c_size_t(aws.numel() if aws is not None else 0), vp(shared["status"].data_ptr()), st)
     return route, group, apply
 
 
@@ -222,7 +224,12 @@ def run_ours(args):
         s["packed"] = pack_proj_descs([M.ProjDesc(s["x"][p.x_key], y, A, B, 1.0) for p, y, A, B in
                                                  zip(w.projections, s["y"], s["A"], s["B"])])
     gate_launches = 0 if w.router == "given" else (2 if (w.router == "gate" and shared["gate_ws"] is not None) else 1)
-    launches_per_step = gate_launches + 1 + len({p.rank for p in w.projections})
+    # scratch of the apply (partial shrink results of the two-launch small-tile path); one buffer serves every set
+    from paper_2603_15965_b200.binding import molora_apply_batched_workspace_bytes
+    need = molora_apply_batched_workspace_bytes(sets[0]["packed"][0], N, C)
+    shared["apply_ws"] = torch.empty(need, dtype=torch.uint8, device="cuda") if need else None
+    apply_launches = (2 if need else 1) * len({p.rank for p in w.projections})
+    launches_per_step = gate_launches + 1 + apply_launches
     for s in sets:
         s["calls"] = marshal_step(lib, w, s, shared, stream.cuda_stream)
 

@@ -145,7 +145,10 @@ molora_status_t molora_group(const int32_t *r, int64_t N, int32_t C, int32_t *co
  * y   device [N, d_out] of type dt, pitch ldy;  in: base projection x W, out: h
  * A   device [C, d_in, rank] of type dt, dense;  B  device [C, rank, d_out] of type dt, dense
  * offsets, perm   device outputs of molora_group for the same N, C (read on the device only)
- * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes (NULL if that is 0)
+ * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes, 16-byte aligned (NULL if
+ *                 that is 0).  Only the small-tile path writes it (fp32 partial shrink results [slice][N][rank]):
+ *                 calls below 1024 tokens and, with more than 64 adapters, the short segments of larger calls.
+ *                 MOLORA_ERR_WORKSPACE if that path is needed and ws is NULL, misaligned or too small.
  * dev_status      device uint32 or NULL; MOLORA_DEV_TIMEOUT is OR-ed in if a bounded wait inside the
  *                 tensor-core kernel gave up (the kernel then returns without hanging; y is incomplete)
  * The kernel variant (CUDA-core path for small segments, tensor-core tiles for large ones) is chosen on
@@ -157,8 +160,9 @@ molora_status_t molora_apply(const void *x, int64_t ldx, void *y, int64_t ldy, m
                              uint32_t *dev_status, void *stream);
 
 /* Same operation for P projections that share N, C, offsets and perm (the projections of one layer),
- * enqueued as one launch.  `projs` is a HOST array of P descriptors (1 <= P <= MOLORA_MAX_PROJECTIONS),
- * copied at enqueue time; the pointers inside are device pointers with the meaning given above. */
+ * enqueued as one launch per kernel variant.  `projs` is a HOST array of P descriptors (1 <= P <=
+ * MOLORA_MAX_PROJECTIONS), copied at enqueue time; the pointers inside are device pointers with the meaning
+ * given above.  ws needs the SUM of molora_apply_workspace_bytes(N, C, d_in, d_out, rank) over the projections. */
 typedef struct {
     const void *x;
     int64_t ldx;

@@ -304,11 +304,20 @@ def pack_proj_descs(projs: Sequence[ProjDesc]):
     return arr, N, C, dt
 
 
+def molora_apply_batched_workspace_bytes(arr, N: int, C: int) -> int:
+    """Scratch a batched apply needs: the sum of molora_apply_workspace_bytes over its projections."""
+    return sum(molora_apply_workspace_bytes(N, C, d.d_in, d.d_out, d.rank) for d in arr)
+
+
 def molora_apply_batched(projs, offsets: torch.Tensor, perm: torch.Tensor, ws: Optional[torch.Tensor] = None,
                          dev_status: Optional[torch.Tensor] = None, stream=None, packed=None) -> None:
     """One launch for the projections of a layer (shared N, C, offsets, perm).  ``projs``: ProjDesc list."""
     lib = load_library()
     arr, N, C, dt = packed if packed is not None else pack_proj_descs(projs)
+    if ws is None:
+        need = molora_apply_batched_workspace_bytes(arr, N, C)
+        if need > 0:
+            ws = torch.empty(need, dtype=torch.uint8, device=offsets.device)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_apply_batched", lib.molora_apply_batched(arr, len(arr), dt, N, C, _ptr(offsets), _ptr(perm),
                                                             _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))

@@ -2,7 +2,21 @@
 // allocates, or synchronises.
 #include "common.cuh"
 
+#include <cstdlib>
+#include <cstring>
+
 using namespace molora;
+
+namespace molora {
+bool chained_launch_enabled()
+{
+    static const bool on = [] {
+        const char* v = std::getenv("MOLORA_CHAINED_LAUNCH");
+        return v == nullptr || std::strcmp(v, "0") != 0;
+    }();
+    return on;
+}
+}  // namespace molora
 
 namespace {
 
@@ -82,17 +96,21 @@ molora_status_t molora_group(const int32_t* r, int64_t N, int32_t C, int32_t* co
     return launch_group(r, N, C, counts, offsets, perm, ws, ws_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
-size_t molora_apply_workspace_bytes(int64_t /*N*/, int32_t /*C*/, int32_t /*d_in*/, int32_t /*d_out*/, int32_t /*rank*/)
+size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t d_out, int32_t rank)
 {
-    return 0;
+    // Only the two-launch small-tile path needs scratch (its partial shrink results).  It serves calls below
+    // kUmmaMinTokens tokens and, with more than kUmmaAllSegmentsMaxC adapters, the short segments of larger calls;
+    // the element type is not known here, so the figure assumes bf16 (fp32 calls need none).
+    if (N <= 0 || d_in <= 0 || d_out <= 0 || (rank != 16 && rank != 32 && rank != 64)) return 0;
+    if ((d_in % 32) != 0 || (d_out % 32) != 0) return 0;
+    if (N >= kUmmaMinTokens && C <= kUmmaAllSegmentsMaxC && (d_in % 64) == 0 && (d_out % 64) == 0) return 0;
+    return decode_workspace_bytes(N, d_in, rank);
 }
 
 molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
                                      int32_t C, const int32_t* offsets, const int32_t* perm, void* ws, size_t ws_bytes,
                                      uint32_t* dev_status, void* stream)
 {
-    (void)ws;
-    (void)ws_bytes;
     if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS) return MOLORA_ERR_INVALID_ARG;
     if (N < 0 || N >= INT32_MAX || C < 1) return MOLORA_ERR_INVALID_ARG;
     if (C > MOLORA_MAX_ADAPTERS) return MOLORA_ERR_UNSUPPORTED;
@@ -125,11 +143,11 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
             for (int i = 0; i < n_tc; ++i) {
                 if (decode_eligible(tc[i], dt)) small_dc[a++] = tc[i]; else small_cc[b++] = tc[i];
             }
-            if (a > 0) st = launch_apply_decode(small_dc, a, N, C, offsets, perm, min_rows, s);
+            if (a > 0) st = launch_apply_decode(small_dc, a, N, C, offsets, perm, min_rows, ws, ws_bytes, dev_status, s);
             if (st == MOLORA_OK && b > 0) st = launch_apply_rowtile(small_cc, b, dt, N, C, offsets, perm, min_rows, s);
         }
     }
-    if (st == MOLORA_OK && n_dc > 0) st = launch_apply_decode(dc, n_dc, N, C, offsets, perm, INT32_MAX, s);
+    if (st == MOLORA_OK && n_dc > 0) st = launch_apply_decode(dc, n_dc, N, C, offsets, perm, INT32_MAX, ws, ws_bytes, dev_status, s);
     if (st == MOLORA_OK && n_cc > 0) st = launch_apply_rowtile(cc, n_cc, dt, N, C, offsets, perm, INT32_MAX, s);
     return st;
 }
@@ -164,7 +182,7 @@ molora_status_t molora_selftest_bounded_wait(uint32_t* dev_status, int64_t limit
 namespace {
 
 struct HostPlan {          // byte offsets into the arena
-    size_t ids, r, counts, offsets, perm, gate_ws, x[MOLORA_MAX_PROJECTIONS], y[MOLORA_MAX_PROJECTIONS], total;
+    size_t ids, r, counts, offsets, perm, gate_ws, apply_ws, apply_ws_bytes, x[MOLORA_MAX_PROJECTIONS], y[MOLORA_MAX_PROJECTIONS], total;
     int x_owner[MOLORA_MAX_PROJECTIONS];   // first projection with the same x_host (its staged copy is shared)
 };
 
@@ -187,6 +205,11 @@ bool plan_host(const molora_host_proj_t* projs, int32_t P, molora_dtype_t dt, in
         if (gate_proj < 0 || gate_proj >= P) return false;
         off = align256(off + route_gate_workspace_bytes(dt, projs[gate_proj].d_in, C));
     }
+    pl.apply_ws = off;
+    pl.apply_ws_bytes = 0;
+    for (int i = 0; i < P; ++i)
+        pl.apply_ws_bytes += molora_apply_workspace_bytes(N, C, projs[i].d_in, projs[i].d_out, projs[i].rank);
+    off = align256(off + pl.apply_ws_bytes);
     for (int i = 0; i < P; ++i) {
         pl.x_owner[i] = i;
         for (int j = 0; j < i; ++j)
@@ -275,7 +298,8 @@ molora_status_t molora_forward_host(molora_router_t router, const int32_t* route
     int32_t* perm = reinterpret_cast<int32_t*>(base + pl.perm);
     st = launch_group(r, N, C, reinterpret_cast<int32_t*>(base + pl.counts), offsets, perm, nullptr, 0, dev_status, s);
     if (st != MOLORA_OK) return st;
-    st = molora_apply_batched(dev, P, dt, N, C, offsets, perm, nullptr, 0, dev_status, stream);
+    st = molora_apply_batched(dev, P, dt, N, C, offsets, perm, pl.apply_ws_bytes > 0 ? base + pl.apply_ws : nullptr,
+                              pl.apply_ws_bytes, dev_status, stream);
     if (st != MOLORA_OK) return st;
     // 5. results: device -> host
     for (int i = 0; i < P; ++i)

@@ -16,6 +16,7 @@
 // The intermediate t never leaves the chip.  Tiles are located on the device from `offsets`
 // (no host read of the histogram), so the grid is sized for the worst case and surplus CTAs exit.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 #include "warp_reduce.cuh"
 
 namespace molora {
@@ -42,6 +43,7 @@ __global__ void __launch_bounds__(kRowTileThreads, 1) apply_rowtile_kernel(const
     const molora_proj_desc_t& pd = prm.p[blockIdx.y];
     if (pd.rank != R) return;                // a launch of this instantiation serves the projections of rank R
 
+    ptx::grid_dependency_sync();             // offsets and perm come from the grouping kernel
     int seg, row0, rows;
     if (!find_tile(prm.offsets, prm.C, TM, blockIdx.x, 1, prm.max_rows, seg, row0, rows)) return;
 
@@ -145,8 +147,7 @@ static cudaError_t rowtile_launch(const ApplyBatchParams& prm, int64_t N, cudaSt
     const int64_t cap_rows = prm.max_rows == INT32_MAX ? N : (N < (int64_t)prm.C * prm.max_rows ? N : (int64_t)prm.C * prm.max_rows);
     const int64_t tiles = ceil_div64(cap_rows, TM) + prm.C;
     dim3 grid((unsigned)tiles, (unsigned)prm.P);
-    apply_rowtile_kernel<T, R><<<grid, kRowTileThreads, 0, s>>>(prm);
-    return cudaGetLastError();
+    return launch_chained(apply_rowtile_kernel<T, R>, grid, dim3(kRowTileThreads), 0, s, 1, prm);
 }
 
 template <typename T>

@@ -131,15 +131,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     MOLORA_TR_CTA(0);
     const UmmaProj& pj = prm.p[blockIdx.y];
     if (pj.rank != R) return;
-    int seg, row0, rows;
     const uint32_t S = cluster_nctarank(), crank = cluster_ctarank();   // CTAs sharing this tile, and my slice
-    {
-        // bring the segment table on chip in one memory round trip, then look the tile up there
-        __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
-        for (int i = threadIdx.x; i <= prm.C; i += kUmmaThreads) offs_s[i] = __ldg(prm.offsets + i);
-        __syncthreads();
-        if (!find_tile_smem(offs_s, prm.C, prm.tile_rows, blockIdx.x / S, prm.min_rows, INT32_MAX, seg, row0, rows)) return;
-    }
 
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -149,14 +141,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     volatile int* abort_flag = &ctrl->abort_flag;
     auto stage = [&](int s) { return base + (uint32_t)s * Cfg::kStageBytes; };
     auto bar = [&](const uint64_t* b) { return smem_u32(b); };
-
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int KXall = pj.d_in / kChunkCols, NYall = pj.d_out / kChunkCols;
-    const int kx0 = (int)(crank * KXall / S), KX = (int)((crank + 1) * KXall / S) - kx0;   // my slice of d_in
-    const int ny0 = (int)(crank * NYall / S), NY = (int)((crank + 1) * NYall / S) - ny0;   // my slice of d_out
-    const int total = KX + NY;
 
-    // ---------------------------------------------------------------- set-up
+    // ---------------------------------------------------------------- set-up, part 1: nothing read from memory
+    // (runs while the previous kernel of the stream may still be executing)
     if (tid == 0) MOLORA_TR(3, 0, 0);
     if (tid == 0) {
         prefetch_tensormap(&pj.tm_a);
@@ -180,10 +168,27 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
         tmem_relinquish();
     }
-    if (tid < kTileM) ctrl->rows[tid] = tid < rows ? __ldg(prm.perm + row0 + tid) : -1;
+    grid_dependency_sync();            // offsets and perm come from the grouping kernel; y from the base projection
+
+    // ---------------------------------------------------------------- set-up, part 2: which tile is mine
+    // bring the segment table on chip in one memory round trip, then look the tile up there
+    __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
+    for (int i = tid; i <= prm.C; i += kUmmaThreads) offs_s[i] = __ldg(prm.offsets + i);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    int seg, row0, rows;
+    if (!find_tile_smem(offs_s, prm.C, prm.tile_rows, blockIdx.x / S, prm.min_rows, INT32_MAX, seg, row0, rows)) {
+        // past the last tile (the grid is sized from an upper bound); the whole cluster takes this exit together
+        if (warp == kMmaWarp) tmem_dealloc(ctrl->tmem_base, kTmemCols);
+        return;
+    }
+    const int KXall = pj.d_in / kChunkCols, NYall = pj.d_out / kChunkCols;
+    const int kx0 = (int)(crank * KXall / S), KX = (int)((crank + 1) * KXall / S) - kx0;   // my slice of d_in
+    const int ny0 = (int)(crank * NYall / S), NY = (int)((crank + 1) * NYall / S) - ny0;   // my slice of d_out
+    const int total = KX + NY;
+    if (tid < kTileM) ctrl->rows[tid] = tid < rows ? __ldg(prm.perm + row0 + tid) : -1;
+    __syncthreads();
     if (tid == 0) MOLORA_TR(3, 0, 1);
     if (S > 1) cluster_sync_all();     // every CTA of the cluster is running and has initialised its barriers
     if (tid == 0) MOLORA_TR(3, 0, 2);
@@ -546,8 +551,13 @@ static cudaError_t umma_launch(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStr
     }
     const int64_t tiles = ceil_div64(N, prm.tile_rows) + prm.C;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     fill_launch_config<R>(cfg, attr, tiles, prm.P, split, s);
+    if (chained_launch_enabled()) {
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 2;
+    }
     return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R>, prm);
 }
 

@@ -180,11 +180,14 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
                                   const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
                                   cudaStream_t s);
 
-// mma.sync path for decode-sized calls (bf16, rank 16/32/64, d_in and d_out multiples of 32); takes the segments
-// with fewer than max_rows rows.
+// mma.sync path for decode-sized calls (bf16, rank 16/32/64, d_in and d_out multiples of 32): a shrink launch and
+// an expand launch; takes the segments with fewer than max_rows rows.  The workspace holds the fp32 partial
+// shrink results: the sum of decode_workspace_bytes over the projections.
 bool decode_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
+size_t decode_workspace_bytes(int64_t N, int32_t d_in, int32_t rank);
 molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
-                                    const int32_t* offsets, const int32_t* perm, int32_t max_rows, cudaStream_t s);
+                                    const int32_t* offsets, const int32_t* perm, int32_t max_rows, void* ws,
+                                    size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
 
 molora_status_t launch_bounded_wait_selftest(uint32_t* dev_status, int64_t limit_cycles, int32_t* result, cudaStream_t s);
 
@@ -193,6 +196,37 @@ molora_status_t launch_bounded_wait_selftest(uint32_t* dev_status, int64_t limit
 constexpr int32_t kUmmaMinRows = 32;
 constexpr int64_t kUmmaMinTokens = 1024;
 constexpr int32_t kUmmaAllSegmentsMaxC = 64;   // up to this many adapters the tensor-core kernel takes all segments
+
+// Launch with programmatic stream serialization (the kernel calls ptx::grid_dependency_sync() after its
+// on-chip set-up) and, when cluster_x > 1, a cluster of that many CTAs along x.
+bool chained_launch_enabled();   // false when MOLORA_CHAINED_LAUNCH=0 (plain stream order, for comparisons)
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                  unsigned cluster_x, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    unsigned n = 0;
+    if (cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (chained_launch_enabled()) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 inline molora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? MOLORA_OK : MOLORA_ERR_CUDA; }
 

@@ -60,6 +60,7 @@ __global__ void __launch_bounds__(kGroupThreads) group_cluster_kernel(const int3
 
     for (int c = lane; c < C; c += 32) hist[warp][c] = 0;
     __syncwarp();
+    ptx::grid_dependency_sync();   // r is the router's output
 
     bool bad = false;
     for (int64_t i0 = begin; i0 < end; i0 += 32) {
@@ -160,19 +161,8 @@ molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* co
     // one CTA per ~1024 tokens (one 32-token step per warp), at most 8 CTAs
     int split = 1;
     while (split < kGroupMaxCluster && (int64_t)split * 1024 < N) split *= 2;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)split, 1, 1);
-    cfg.blockDim = dim3(kGroupThreads, 1, 1);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)split;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cuda_ok(cudaLaunchKernelEx(&cfg, group_cluster_kernel, r, N, C, counts, offsets, perm, dev_status));
+    return cuda_ok(launch_chained(group_cluster_kernel, dim3((unsigned)split), dim3(kGroupThreads), 0, s, (unsigned)split,
+                                  r, N, C, counts, offsets, perm, dev_status));
 }
 
 }  // namespace molora

@@ -1,5 +1,6 @@
 // Routers: vocabulary-range routing (Definition 3.1) and the linear gate with top-1 argmax (Eq. 8, k = 1).
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 #include "warp_reduce.cuh"
 
 namespace molora {
@@ -15,6 +16,7 @@ __global__ void __launch_bounds__(256) route_vocab_kernel(const int32_t* __restr
                                                           int32_t* __restrict__ r_out, uint32_t* dev_status)
 {
     __shared__ int32_t b[MOLORA_MAX_ADAPTERS + 1];
+    ptx::grid_dependency_sync();
     for (int i = threadIdx.x; i <= M; i += blockDim.x) b[i] = __ldg(breaks + i);
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -49,8 +51,8 @@ molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t*
     const int threads = 256;
     const int64_t want = ceil_div64(N, threads);
     const int blocks = (int)(want < 148 * 8 ? want : 148 * 8);
-    route_vocab_kernel<<<blocks, threads, 0, s>>>(ids, N, breaks, M, r_out, dev_status);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(launch_chained(route_vocab_kernel, dim3(blocks), dim3(threads), 0, s, 1, ids, N, breaks, M, r_out,
+                                  dev_status));
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -75,6 +77,7 @@ __global__ void __launch_bounds__(256) route_gate_kernel(const T* __restrict__ x
     __shared__ float zs[WARPS][TOK][CP];
 
     const int warp = threadIdx.x >> 5, lane = lane_id();
+    ptx::grid_dependency_sync();
     const int64_t tok0 = ((int64_t)blockIdx.x * WARPS + warp) * TOK;
 
     float acc[TOK][CP];
@@ -171,6 +174,7 @@ __global__ void __launch_bounds__(128) route_gate_resident_kernel(const T* __res
     constexpr int BATCH = 8;                       // 16-byte vectors per token kept in flight per lane
     extern __shared__ __align__(16) float Gres[];  // [chunks][32 lanes][LANE_STRIDE]
     const int chunks = (d + KC - 1) / KC;
+    ptx::grid_dependency_sync();
     if (C == CP && (d % KC) == 0) {
         // G rows are CP floats = whole 16-byte vectors: copy them as they are (coalesced float4 loads)
         constexpr int V = CP / 4;
@@ -294,9 +298,8 @@ static molora_status_t gate_resident_launch(const void* x, int64_t N, int d, int
     int tpw = 8;
     while (tpw > 2 && ceil_div64(N, 4 * tpw) < 148) tpw /= 2;
     const int64_t blocks = ceil_div64(N, 4 * tpw);
-    route_gate_resident_kernel<T, CP><<<(unsigned)blocks, 128, smem, s>>>(static_cast<const T*>(x), N, d, ldx, G, bias,
-                                                                         C, r_out, logits_out, tpw);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(launch_chained(route_gate_resident_kernel<T, CP>, dim3((unsigned)blocks), dim3(128), smem, s, 1,
+                                  static_cast<const T*>(x), N, d, ldx, G, bias, C, r_out, logits_out, tpw));
 }
 
 template <typename T, int CP, int TOK>
@@ -304,9 +307,8 @@ static molora_status_t gate_launch(const void* x, int64_t N, int d, int64_t ldx,
                                    int C, int32_t* r_out, float* logits_out, cudaStream_t s)
 {
     const int64_t blocks = ceil_div64(N, 8 * TOK);
-    route_gate_kernel<T, CP, TOK><<<(unsigned)blocks, 256, 0, s>>>(static_cast<const T*>(x), N, d, ldx, G, bias, C,
-                                                                   r_out, logits_out);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(launch_chained(route_gate_kernel<T, CP, TOK>, dim3((unsigned)blocks), dim3(256), 0, s, 1,
+                                  static_cast<const T*>(x), N, d, ldx, G, bias, C, r_out, logits_out));
 }
 
 template <typename T>

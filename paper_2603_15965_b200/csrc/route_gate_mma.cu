@@ -17,6 +17,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace molora {
 
@@ -54,6 +55,7 @@ __global__ void __launch_bounds__(256) gate_split_kernel(const float* __restrict
     using Img = GateImage<NT, KC>;
     const int chunks = (d + KC - 1) / KC;
     const int64_t total = (int64_t)chunks * KC * Img::CP;
+    ptx::grid_dependency_sync();     // an earlier gate call may still be reading the images this kernel rewrites
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int c = (int)(e % Img::CP);
         const int64_t k = e / Img::CP;
@@ -86,6 +88,7 @@ __global__ void __launch_bounds__(WARPS * 32) route_gate_mma_kernel(const __nv_b
     __shared__ __align__(16) __nv_bfloat16 Gs[IB][3][CP][ROW];        // [buffer][term][c][k']
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    ptx::grid_dependency_sync();     // the weight images come from gate_split_kernel
     const int g = lane >> 2, q = lane & 3;
     const int64_t tok0 = ((int64_t)blockIdx.x * WARPS + warp) * 16;
     const int64_t rowA = tok0 + g < N ? tok0 + g : N - 1;             // tail rows recompute the last token
@@ -222,11 +225,14 @@ static molora_status_t gate_mma_launch(const void* x, int64_t N, int d, int64_t 
     __nv_bfloat16* img = static_cast<__nv_bfloat16*>(ws);
     const int chunks = (d + KC - 1) / KC;
     const int64_t elems = (int64_t)chunks * KC * NT * 8;
-    gate_split_kernel<NT, KC><<<(unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4), 256, 0, s>>>(G, d, C, img);
+    if (cudaError_t e = launch_chained(gate_split_kernel<NT, KC>,
+                                       dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)), dim3(256), 0, s,
+                                       1, G, d, C, img);
+        e != cudaSuccess)
+        return MOLORA_ERR_CUDA;
     const int64_t blocks = ceil_div64(N, 16 * WARPS);
-    route_gate_mma_kernel<NT, WARPS, KC><<<(unsigned)blocks, WARPS * 32, 0, s>>>(static_cast<const __nv_bfloat16*>(x), N,
-                                                                                d, ldx, img, bias, C, r_out, logits_out);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(launch_chained(route_gate_mma_kernel<NT, WARPS, KC>, dim3((unsigned)blocks), dim3(WARPS * 32), 0, s, 1,
+                                  static_cast<const __nv_bfloat16*>(x), N, d, ldx, img, bias, C, r_out, logits_out));
 }
 
 size_t route_gate_mma_workspace_bytes(int32_t d, int32_t C)

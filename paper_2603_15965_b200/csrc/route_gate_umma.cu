@@ -54,9 +54,10 @@ template <int CP>
 __global__ void __launch_bounds__(256) gate_umma_split_kernel(const float* __restrict__ G, int d, int C,
                                                               __nv_bfloat16* __restrict__ img)
 {
-    // the gate kernel that follows is launched programmatically: it may start its set-up and its x loads now and
-    // waits (griddepcontrol.wait) only before it reads the images written here
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // An earlier gate call may still be reading the images this kernel rewrites: wait for it.  The gate kernel
+    // that follows is launched programmatically: from here on it may run its set-up and its x loads, and it
+    // waits only before it reads the images written here.
+    grid_dependency_sync();
     const int64_t total = (int64_t)d * CP;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int c = (int)(e % CP);
@@ -128,7 +129,7 @@ __global__ void __launch_bounds__(kGuThreads, 1) route_gate_umma_kernel(const __
                 mbar_arrive_expect_tx(fb, (uint32_t)STAGE);
                 tma_load_2d(stage(s), &prm.tm_x, kc * 64, (int)tok0, fb);          // rows past N are zero-filled
                 if (!images_ready) {           // the preparation kernel (previous launch) has completed and flushed
-                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    grid_dependency_sync();
                     images_ready = true;
                 }
                 tma_load_2d(stage(s) + kGuTileBytes, &prm.tm_g, 0, kc * NP, fb);
@@ -234,7 +235,9 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
     prm.d = d;
     prm.C = C;
     const int64_t elems = (int64_t)d * CP;
-    gate_umma_split_kernel<CP><<<(unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4), 256, 0, s>>>(G, d, C, img);
+    if (launch_chained(gate_umma_split_kernel<CP>, dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)),
+                       dim3(256), 0, s, 1, G, d, C, img) != cudaSuccess)
+        return MOLORA_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(tiles * split), 1, 1);
     cfg.blockDim = dim3(kGuThreads, 1, 1);
@@ -248,7 +251,7 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // overlap with the tail of the preparation kernel
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cfg.numAttrs = chained_launch_enabled() ? 2 : 1;
     return cuda_ok(cudaLaunchKernelEx(&cfg, route_gate_umma_kernel<CP>, prm));
 }
 

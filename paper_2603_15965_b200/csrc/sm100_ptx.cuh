@@ -145,6 +145,19 @@ __device__ __forceinline__ void tma_scatter4(const void* tmap, uint32_t src, int
         ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(src), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
         : "memory");
 }
+// Linear bulk copies (no tensor map): `bytes` is a multiple of 16, both addresses are 16-byte aligned.
+// global -> shared memory of this CTA, completion counted in bytes on an mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* gsrc, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(gsrc), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// shared memory of this CTA -> global (bulk async group)
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_group_read()
@@ -257,6 +270,21 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, int a_mn_maj
            | (1u << 10)                   // B format: bf16
            | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) |
            ((uint32_t)(M >> 4) << 24);
+}
+
+// ---- programmatic dependent launch -----------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may start while its predecessor in the
+// stream still runs.  grid_dependency_wait() returns once the predecessor has completed and its writes are
+// visible; nothing the predecessor may write, and nothing it may still read that this kernel writes, is touched
+// before it.  grid_dependency_trigger() lets the successor start its own prologue.  Every kernel of this
+// library triggers only after its own wait, so a kernel that starts early knows that everything before its
+// predecessor has completed.  Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_sync()
+{
+    grid_dependency_wait();
+    grid_dependency_trigger();
 }
 
 }  // namespace ptx

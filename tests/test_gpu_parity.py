@@ -346,7 +346,7 @@ def test_forward_host_matches_oracle(name):
     assert int(status.item()) == 0
 
 
-# ------------------------------------------------------------------ decode path (N < 1024, 32-row tiles on mma.sync)
+# ------------------------------------------------------------------ decode path (N < 1024: shrink launch + expand launch)
 @pytest.mark.parametrize("rank", [16, 32, 64])
 def test_decode_path_segment_size_sweep(rank):
     sizes = [0, 1, 7, 15, 16, 17, 31, 32, 33, 47, 64, 65, 97]
@@ -357,7 +357,10 @@ def test_decode_path_segment_size_sweep(rank):
 
 
 @pytest.mark.parametrize("N,C,d_in,d_out,rank", [(1, 1, 32, 32, 16), (256, 8, 2048, 6144, 16), (100, 2, 6144, 2048, 32),
-                                                 (700, 3, 256, 1024, 64), (64, 64, 512, 96, 16)])
+                                                 (700, 3, 256, 1024, 64), (64, 64, 512, 96, 16),
+                                                 (200, 4, 16384, 64, 32),     # slices longer than one staging pass
+                                                 (300, 5, 32, 1536, 64),      # three column slices, one k block
+                                                 (90, 3, 2080, 1056, 16)])    # ragged last slices (multiples of 32 only)
 def test_decode_path_shapes(N, C, d_in, d_out, rank):
     w = W.random_problem(N + rank + 7, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.1 if N > 10 else 0.0)
     run_and_check(w)
