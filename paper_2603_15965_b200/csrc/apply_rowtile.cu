@@ -147,7 +147,7 @@ static cudaError_t rowtile_launch(const ApplyBatchParams& prm, int64_t N, cudaSt
     const int64_t cap_rows = prm.max_rows == INT32_MAX ? N : (N < (int64_t)prm.C * prm.max_rows ? N : (int64_t)prm.C * prm.max_rows);
     const int64_t tiles = ceil_div64(cap_rows, TM) + prm.C;
     dim3 grid((unsigned)tiles, (unsigned)prm.P);
-    return launch_chained(apply_rowtile_kernel<T, R>, grid, dim3(kRowTileThreads), 0, s, 1, prm);
+    return launch_kernel(apply_rowtile_kernel<T, R>, grid, dim3(kRowTileThreads), 0, s, 1, false, prm);
 }
 
 template <typename T>

@@ -502,9 +502,9 @@ static cudaError_t twophase_launch(const TwoPhaseParams& prm, int64_t N, cudaStr
     }
     const unsigned grid_s = (unsigned)std::min<int64_t>(tiles * su.start[prm.P], wave[0]);
     const unsigned grid_e = (unsigned)std::min<int64_t>(tiles * eu.start[prm.P], wave[1]);
-    cudaError_t e = launch_chained(shrink_kernel<R>, dim3(grid_s), dim3(kTpThreads), Cfg::SHRINK_SMEM, s, 1, prm, su);
+    cudaError_t e = launch_kernel(shrink_kernel<R>, dim3(grid_s), dim3(kTpThreads), Cfg::SHRINK_SMEM, s, 1, false, prm, su);
     if (e != cudaSuccess) return e;
-    return launch_chained(expand_kernel<R>, dim3(grid_e), dim3(kTpThreads), Cfg::EXPAND_SMEM, s, 1, prm, eu);
+    return launch_kernel(expand_kernel<R>, dim3(grid_e), dim3(kTpThreads), Cfg::EXPAND_SMEM, s, 1, true, prm, eu);
 }
 
 molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,

@@ -111,8 +111,12 @@ struct UmmaCfg {
     static constexpr int kTBytes = kTileM * kTRowBytes;
     static constexpr int kSwzBits = R == 64 ? 3 : R == 32 ? 2 : 1;    // swizzle width of R*2-byte rows
     static constexpr uint32_t kWLayout = swizzle_layout_type(static_cast<Swizzle>(kSwzBits));
+    // partial T rows received from the cluster peers: (S - 1) * ceil(128 / S) rows of R fp32: 64, 86, 96 rows for
+    // S = 2, 3, 4.  Rank 64 stops at S = 3 (shared memory).
+    static constexpr int kMaxSplitR = R == 64 ? 3 : kMaxSplit;
+    static constexpr int kRecvBytes = (R == 64 ? 86 : 96) * R * 4;
     static constexpr int kCtrlBytes = 1024;
-    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kTBytes + kCtrlBytes;
+    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kTBytes + kRecvBytes + kCtrlBytes;
 };
 
 struct Ctrl {                         // lives in shared memory after the tiles
@@ -137,7 +141,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     const uint32_t base = (raw + 1023u) & ~1023u;
     const uint32_t thi = base + Cfg::kStages * Cfg::kStageBytes;
     const uint32_t tlo = thi + Cfg::kTBytes;
-    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw + (tlo + Cfg::kTBytes - raw));
+    const uint32_t recv = tlo + Cfg::kTBytes;
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw + (recv + Cfg::kRecvBytes - raw));
     volatile int* abort_flag = &ctrl->abort_flag;
     auto stage = [&](int s) { return base + (uint32_t)s * Cfg::kStageBytes; };
     auto bar = [&](const uint64_t* b) { return smem_u32(b); };
@@ -190,7 +195,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     if (tid < kTileM) ctrl->rows[tid] = tid < rows ? __ldg(prm.perm + row0 + tid) : -1;
     __syncthreads();
     if (tid == 0) MOLORA_TR(3, 0, 1);
-    if (S > 1) cluster_sync_all();     // every CTA of the cluster is running and has initialised its barriers
+    // "I am running and my barriers are initialised": the matching wait comes right before the first access to
+    // a peer's shared memory (the T exchange), so the cluster barrier costs nothing here
+    if (S > 1) cluster_arrive();
     if (tid == 0) MOLORA_TR(3, 0, 2);
     const uint32_t tmem = ctrl->tmem_base;
     const uint32_t tmem_T = tmem;                               // columns [0, R)
@@ -335,70 +342,100 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 #pragma unroll
             for (int c = 0; c < R / 16; ++c) tmem_ld_x16(tmem_T + lane_addr + c * 16, tv + c * 16);
             tmem_wait_ld();
+            bool t_published = false;
             if (S > 1) {
-                // Exchange the partial T tiles.  Mine goes to the (still unused) T_hi/T_lo region as
-                // [R/4][128] float4, so a warp touches 512 contiguous bytes per access, locally and remotely.
+                // Exchange of the partial T tiles in two pushes through distributed shared memory.  CTA o owns the
+                // tile rows [o*128/S, (o+1)*128/S): (1) every CTA sends its partial of a row to the row's owner;
+                // (2) the owner sums the partials in rank order (the same bits whoever computes them), scales,
+                // splits into bf16 hi + lo and writes the finished row into the T_hi / T_lo tiles of every CTA.
+                // Nothing is ever read from a peer, and after step 2 nobody touches this CTA's memory again, so
+                // the CTAs of a cluster retire independently.
+                const int rows_max = (kTileM + (int)S - 1) / (int)S;
+                int owner = 0;
 #pragma unroll
-                for (int c4 = 0; c4 < R / 4; ++c4)
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(thi + (uint32_t)(c4 * kTileM + row) * 16u),
-                                 "r"(tv[4 * c4]), "r"(tv[4 * c4 + 1]), "r"(tv[4 * c4 + 2]), "r"(tv[4 * c4 + 3]) : "memory");
-                __syncwarp();                                   // the warp's rows are written; lane q2 tells CTA q2
+                for (int o = 1; o < kMaxSplit; ++o)
+                    if ((uint32_t)o < S && row >= o * kTileM / (int)S) owner = o;
+                const int own_lo = owner * kTileM / (int)S;
+                cluster_wait();                                 // every peer is running, its barriers initialised
+                if ((uint32_t)owner != crank) {
+                    const uint32_t slot = crank < (uint32_t)owner ? crank : crank - 1;      // my slot at the owner
+                    const uint32_t dst = map_to_cta(recv, (uint32_t)owner) + slot * (uint32_t)(rows_max * R * 4);
+#pragma unroll
+                    for (int c4 = 0; c4 < R / 4; ++c4)
+                        st_cluster_u32x4(dst + (uint32_t)(c4 * rows_max + (row - own_lo)) * 16u, tv[4 * c4], tv[4 * c4 + 1],
+                                         tv[4 * c4 + 2], tv[4 * c4 + 3]);
+                }
+                __syncwarp();                                   // the warp's rows are sent; lane q2 tells CTA q2
                 if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
                 if (et == 0) MOLORA_TR(3, 2, 2);
                 wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
                 if (et == 0) MOLORA_TR(3, 2, 3);
+                if ((uint32_t)owner == crank) {
+                    // sum in rank order, in place: lower ranks' partials, mine (registers), higher ranks'
 #pragma unroll
-                for (int e = 0; e < R; ++e) tv[e] = 0u;
-                if (!*abort_flag) {
-                    // Sum in rank order (every CTA of the cluster gets the same bits).  Loads of one 16-column
-                    // slab from all peers are issued together so that their latencies overlap.
-                    uint32_t rbase[kMaxSplit];
-#pragma unroll
-                    for (int q2 = 0; q2 < kMaxSplit; ++q2) rbase[q2] = map_to_cta(thi, (uint32_t)q2 < S ? q2 : 0);
-#pragma unroll
-                    for (int slab = 0; slab < R / 16; ++slab) {
-                        float4 v[kMaxSplit][4];
-#pragma unroll
-                        for (int q2 = 0; q2 < kMaxSplit; ++q2)
-                            if ((uint32_t)q2 < S) {
-#pragma unroll
-                                for (int c = 0; c < 4; ++c)
-                                    v[q2][c] = ld_cluster_f32x4(rbase[q2] + (uint32_t)((slab * 4 + c) * kTileM + row) * 16u);
+                    for (int c4 = 0; c4 < R / 4; ++c4) {
+                        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (uint32_t q2 = 0; q2 < S; ++q2) {
+                            float4 v;
+                            if (q2 == crank) {
+                                v = make_float4(__uint_as_float(tv[4 * c4]), __uint_as_float(tv[4 * c4 + 1]),
+                                                __uint_as_float(tv[4 * c4 + 2]), __uint_as_float(tv[4 * c4 + 3]));
+                            } else {
+                                const uint32_t src = recv + (q2 < crank ? q2 : q2 - 1) * (uint32_t)(rows_max * R * 4);
+                                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                                             : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                                             : "r"(src + (uint32_t)(c4 * rows_max + (row - own_lo)) * 16u)
+                                             : "memory");
                             }
+                            a.x += v.x;
+                            a.y += v.y;
+                            a.z += v.z;
+                            a.w += v.w;
+                        }
+                        tv[4 * c4] = __float_as_uint(a.x);
+                        tv[4 * c4 + 1] = __float_as_uint(a.y);
+                        tv[4 * c4 + 2] = __float_as_uint(a.z);
+                        tv[4 * c4 + 3] = __float_as_uint(a.w);
+                    }
 #pragma unroll
-                        for (int q2 = 0; q2 < kMaxSplit; ++q2)
-                            if ((uint32_t)q2 < S) {
+                    for (int c8 = 0; c8 < R / 8; ++c8) {
+                        float hi[8], lo[8];
 #pragma unroll
-                                for (int c = 0; c < 4; ++c) {
-                                    const int e = (slab * 4 + c) * 4;
-                                    tv[e + 0] = __float_as_uint(__uint_as_float(tv[e + 0]) + v[q2][c].x);
-                                    tv[e + 1] = __float_as_uint(__uint_as_float(tv[e + 1]) + v[q2][c].y);
-                                    tv[e + 2] = __float_as_uint(__uint_as_float(tv[e + 2]) + v[q2][c].z);
-                                    tv[e + 3] = __float_as_uint(__uint_as_float(tv[e + 3]) + v[q2][c].w);
-                                }
-                            }
+                        for (int e = 0; e < 8; ++e) {
+                            const float t = __uint_as_float(tv[c8 * 8 + e]) * pj.scale;
+                            hi[e] = __bfloat162float(__float2bfloat16_rn(t));
+                            lo[e] = t - hi[e];
+                        }
+                        const uint32_t off = swizzle_offset((uint32_t)row * Cfg::kTRowBytes + c8 * 16, Cfg::kSwzBits);
+                        const uint4 h = pack<__nv_bfloat16>(hi), l = pack<__nv_bfloat16>(lo);
+                        for (uint32_t q2 = 0; q2 < S; ++q2) {
+                            st_cluster_u32x4(map_to_cta(thi + off, q2), h.x, h.y, h.z, h.w);
+                            st_cluster_u32x4(map_to_cta(tlo + off, q2), l.x, l.y, l.z, l.w);
+                        }
                     }
                 }
-                // nobody may overwrite its partial (with T_hi/T_lo) before every CTA has read it
-                __syncwarp();
+                __syncwarp();                                   // the warp's rows are published everywhere
                 if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_free), (uint32_t)lane));
                 if (et == 0) MOLORA_TR(3, 2, 4);
-                wait_bar_cluster(bar(&ctrl->part_free), 0, abort_flag, prm.dev_status);
+                wait_bar_cluster(bar(&ctrl->part_free), 0, abort_flag, prm.dev_status);   // all 128 rows of T are here
                 if (et == 0) MOLORA_TR(3, 2, 5);
+                t_published = true;
             }
+            if (!t_published) {
 #pragma unroll
-            for (int c8 = 0; c8 < R / 8; ++c8) {
-                float hi[8], lo[8];
+                for (int c8 = 0; c8 < R / 8; ++c8) {
+                    float hi[8], lo[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const float t = __uint_as_float(tv[c8 * 8 + e]) * pj.scale;
-                    hi[e] = __bfloat162float(__float2bfloat16_rn(t));
-                    lo[e] = t - hi[e];
+                    for (int e = 0; e < 8; ++e) {
+                        const float t = __uint_as_float(tv[c8 * 8 + e]) * pj.scale;
+                        hi[e] = __bfloat162float(__float2bfloat16_rn(t));
+                        lo[e] = t - hi[e];
+                    }
+                    const uint32_t off = swizzle_offset((uint32_t)row * Cfg::kTRowBytes + c8 * 16, Cfg::kSwzBits);
+                    const uint4 h = pack<__nv_bfloat16>(hi), l = pack<__nv_bfloat16>(lo);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(thi + off), "r"(h.x), "r"(h.y), "r"(h.z), "r"(h.w) : "memory");
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(tlo + off), "r"(l.x), "r"(l.y), "r"(l.z), "r"(l.w) : "memory");
                 }
-                const uint32_t off = swizzle_offset((uint32_t)row * Cfg::kTRowBytes + c8 * 16, Cfg::kSwzBits);
-                const uint4 h = pack<__nv_bfloat16>(hi), l = pack<__nv_bfloat16>(lo);
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(thi + off), "r"(h.x), "r"(h.y), "r"(h.z), "r"(h.w) : "memory");
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(tlo + off), "r"(l.x), "r"(l.y), "r"(l.z), "r"(l.w) : "memory");
             }
             fence_proxy_async_smem();
             tc_fence_before();
@@ -473,7 +510,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     __syncthreads();
     if (tid == 0) MOLORA_TR(3, 0, 4);
     if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
-    if (S > 1) cluster_sync_all();     // no CTA retires while a peer could still touch its shared memory
+    // threads that took no part in the exchange complete the start-up cluster barrier here (it has long been
+    // passed); no closing barrier is needed, see the exchange
+    if (S > 1 && !(warp >= kEpiWarp0 && warp < kEpiWarp0 + 4)) cluster_wait();
     if (tid == 0) MOLORA_TR(3, 0, 5);
     MOLORA_TR_CTA(1);
 }
@@ -551,13 +590,8 @@ static cudaError_t umma_launch(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStr
     }
     const int64_t tiles = ceil_div64(N, prm.tile_rows) + prm.C;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     fill_launch_config<R>(cfg, attr, tiles, prm.P, split, s);
-    if (chained_launch_enabled()) {
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.numAttrs = 2;
-    }
     return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R>, prm);
 }
 
@@ -601,11 +635,11 @@ static UmmaPlan choose_split_for_rank(const UmmaParams& prm, int64_t N)
     const char* env = getenv("MOLORA_UMMA_SPLIT");          // tuning overrides
     const char* envr = getenv("MOLORA_UMMA_TILE_ROWS");
     if (env != nullptr || envr != nullptr) {
-        if (env != nullptr) best.split = std::max(1, std::min(atoi(env), kMaxSplit));
+        if (env != nullptr) best.split = std::max(1, std::min(atoi(env), UmmaCfg<R>::kMaxSplitR));
         if (envr != nullptr) best.tile_rows = std::max(32, std::min(atoi(envr), kTileM));
     } else {
         double best_cost = 1e30, best_waves = 0;
-        for (int split = 1; split <= kMaxSplit; ++split) {    // cluster sizes need not be powers of two
+        for (int split = 1; split <= UmmaCfg<R>::kMaxSplitR; ++split) {    // cluster sizes need not be powers of two
             double waves;
             const double cost = cost_for(kTileM, split, waves);
             if (cost < best_cost - 1e-9) { best_cost = cost; best_waves = waves; best = {split, kTileM}; }
@@ -614,7 +648,7 @@ static UmmaPlan choose_split_for_rank(const UmmaParams& prm, int64_t N)
         // lanes idle) to put more SMs to work, as long as everything still fits in one wave.
         if (best_waves <= 1.0 && tiles_for(kTileM) * best.split < 0.85 * 148) {
             for (int rows = 96; rows >= 64; rows -= 32)
-                for (int split = 1; split <= kMaxSplit; ++split) {
+                for (int split = 1; split <= UmmaCfg<R>::kMaxSplitR; ++split) {
                     double waves;
                     const double cost = cost_for(rows, split, waves);
                     if (waves <= 1.0 && cost < best_cost - 1e-9) { best_cost = cost; best = {split, rows}; }

@@ -197,12 +197,15 @@ constexpr int32_t kUmmaMinRows = 32;
 constexpr int64_t kUmmaMinTokens = 1024;
 constexpr int32_t kUmmaAllSegmentsMaxC = 64;   // up to this many adapters the tensor-core kernel takes all segments
 
-// Launch with programmatic stream serialization (the kernel calls ptx::grid_dependency_sync() after its
-// on-chip set-up) and, when cluster_x > 1, a cluster of that many CTAs along x.
-bool chained_launch_enabled();   // false when MOLORA_CHAINED_LAUNCH=0 (plain stream order, for comparisons)
+// Launch helper: a cluster of cluster_x CTAs along x when cluster_x > 1, and, when under_predecessor is set,
+// programmatic stream serialization: the kernel may start while the previous kernel of the stream still runs and
+// calls ptx::grid_dependency_wait() before it touches what that kernel writes.  Used only between the two
+// launches of one call (weight split -> tcgen05 gate, decode shrink -> expand), where the predecessor is known;
+// across calls the kernels run in plain stream order (chaining them was measured: no gain on any workload).
+bool chained_launch_enabled();   // false when MOLORA_CHAINED_LAUNCH=0 (plain stream order everywhere, for comparisons)
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
-                                  unsigned cluster_x, Args&&... args)
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                 unsigned cluster_x, bool under_predecessor, Args&&... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -218,7 +221,7 @@ inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 bloc
         attr[n].val.clusterDim.z = 1;
         ++n;
     }
-    if (chained_launch_enabled()) {
+    if (under_predecessor && chained_launch_enabled()) {
         attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n].val.programmaticStreamSerializationAllowed = 1;
         ++n;

@@ -51,7 +51,7 @@ molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t*
     const int threads = 256;
     const int64_t want = ceil_div64(N, threads);
     const int blocks = (int)(want < 148 * 8 ? want : 148 * 8);
-    return cuda_ok(launch_chained(route_vocab_kernel, dim3(blocks), dim3(threads), 0, s, 1, ids, N, breaks, M, r_out,
+    return cuda_ok(launch_kernel(route_vocab_kernel, dim3(blocks), dim3(threads), 0, s, 1, false, ids, N, breaks, M, r_out,
                                   dev_status));
 }
 
@@ -298,7 +298,7 @@ static molora_status_t gate_resident_launch(const void* x, int64_t N, int d, int
     int tpw = 8;
     while (tpw > 2 && ceil_div64(N, 4 * tpw) < 148) tpw /= 2;
     const int64_t blocks = ceil_div64(N, 4 * tpw);
-    return cuda_ok(launch_chained(route_gate_resident_kernel<T, CP>, dim3((unsigned)blocks), dim3(128), smem, s, 1,
+    return cuda_ok(launch_kernel(route_gate_resident_kernel<T, CP>, dim3((unsigned)blocks), dim3(128), smem, s, 1, false,
                                   static_cast<const T*>(x), N, d, ldx, G, bias, C, r_out, logits_out, tpw));
 }
 
@@ -307,7 +307,7 @@ static molora_status_t gate_launch(const void* x, int64_t N, int d, int64_t ldx,
                                    int C, int32_t* r_out, float* logits_out, cudaStream_t s)
 {
     const int64_t blocks = ceil_div64(N, 8 * TOK);
-    return cuda_ok(launch_chained(route_gate_kernel<T, CP, TOK>, dim3((unsigned)blocks), dim3(256), 0, s, 1,
+    return cuda_ok(launch_kernel(route_gate_kernel<T, CP, TOK>, dim3((unsigned)blocks), dim3(256), 0, s, 1, false,
                                   static_cast<const T*>(x), N, d, ldx, G, bias, C, r_out, logits_out));
 }
 

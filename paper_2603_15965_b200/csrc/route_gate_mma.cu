@@ -225,13 +225,13 @@ static molora_status_t gate_mma_launch(const void* x, int64_t N, int d, int64_t 
     __nv_bfloat16* img = static_cast<__nv_bfloat16*>(ws);
     const int chunks = (d + KC - 1) / KC;
     const int64_t elems = (int64_t)chunks * KC * NT * 8;
-    if (cudaError_t e = launch_chained(gate_split_kernel<NT, KC>,
+    if (cudaError_t e = launch_kernel(gate_split_kernel<NT, KC>,
                                        dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)), dim3(256), 0, s,
-                                       1, G, d, C, img);
+                                      1, false, G, d, C, img);
         e != cudaSuccess)
         return MOLORA_ERR_CUDA;
     const int64_t blocks = ceil_div64(N, 16 * WARPS);
-    return cuda_ok(launch_chained(route_gate_mma_kernel<NT, WARPS, KC>, dim3((unsigned)blocks), dim3(WARPS * 32), 0, s, 1,
+    return cuda_ok(launch_kernel(route_gate_mma_kernel<NT, WARPS, KC>, dim3((unsigned)blocks), dim3(WARPS * 32), 0, s, 1, true,
                                   static_cast<const __nv_bfloat16*>(x), N, d, ldx, img, bias, C, r_out, logits_out));
 }
 

@@ -235,8 +235,8 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
     prm.d = d;
     prm.C = C;
     const int64_t elems = (int64_t)d * CP;
-    if (launch_chained(gate_umma_split_kernel<CP>, dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)),
-                       dim3(256), 0, s, 1, G, d, C, img) != cudaSuccess)
+    if (launch_kernel(gate_umma_split_kernel<CP>, dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)),
+                       dim3(256), 0, s, 1, false, G, d, C, img) != cudaSuccess)
         return MOLORA_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(tiles * split), 1, 1);
