@@ -14,6 +14,10 @@
 //   4. second walk: position = seg[c] + lower[c] + hist[w][c] + (rank of the lane inside its group);
 //      the group leader then advances hist[w][c].
 // A final cluster barrier keeps every CTA's shared memory alive until all peers have read it.
+#include <stdlib.h>
+
+#include <algorithm>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -24,6 +28,7 @@ using namespace ptx;
 constexpr int kGroupThreads = 1024;
 constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kGroupMaxCluster = 8;
+constexpr int kGroupCached = 4;      // 32-token steps of a warp kept in registers
 
 // Lanes that hold the same routed adapter as this lane (0 for unrouted lanes are never used).
 __device__ __forceinline__ unsigned peers_of(int v, bool routed, int C)
@@ -46,7 +51,7 @@ __global__ void __launch_bounds__(kGroupThreads) group_cluster_kernel(const int3
                                                                      int32_t* __restrict__ perm, uint32_t* dev_status)
 {
     __shared__ int hist[kGroupWarps][MOLORA_MAX_ADAPTERS];
-    __shared__ int tot[MOLORA_MAX_ADAPTERS];          // this CTA's histogram (read by the peers)
+    __shared__ int tot_all[kGroupMaxCluster][MOLORA_MAX_ADAPTERS];   // every CTA's histogram, pushed by its owner
     __shared__ int seg[MOLORA_MAX_ADAPTERS + 1];      // global exclusive prefix of counts
     __shared__ int lower[MOLORA_MAX_ADAPTERS];        // tokens of adapter c in lower-ranked CTAs
     const int warp = threadIdx.x >> 5, lane = lane_id();
@@ -58,14 +63,35 @@ __global__ void __launch_bounds__(kGroupThreads) group_cluster_kernel(const int3
     const int64_t begin = begin0 < N ? begin0 : N;
     const int64_t end = begin + chunk < N ? begin + chunk : N;
 
+    if (S > 1) cluster_arrive_relaxed();   // "I am running"; waited for before the first write to a peer
     for (int c = lane; c < C; c += 32) hist[warp][c] = 0;
     __syncwarp();
     ptx::grid_dependency_sync();   // r is the router's output
 
+    // the first kGroupCached steps of the warp's tokens stay in registers for both passes (all loads in flight at once)
+    int vreg[kGroupCached];
+#pragma unroll
+    for (int j = 0; j < kGroupCached; ++j) {
+        const int64_t i = begin + j * 32 + lane;
+        vreg[j] = i < end ? __ldg(r + i) : -1;
+    }
+    auto route_of = [&](int64_t i0) {
+        const int64_t j = (i0 - begin) >> 5;
+        int v = -1;
+        if (j < kGroupCached) {
+#pragma unroll
+            for (int jj = 0; jj < kGroupCached; ++jj)
+                if (jj == j) v = vreg[jj];
+        } else {
+            const int64_t i = i0 + lane;
+            v = i < end ? __ldg(r + i) : -1;
+        }
+        return v;
+    };
+
     bool bad = false;
     for (int64_t i0 = begin; i0 < end; i0 += 32) {
-        const int64_t i = i0 + lane;
-        const int v = i < end ? __ldg(r + i) : -1;
+        const int v = route_of(i0);
         const bool routed = v >= 0 && v < C;
         bad |= (v < -1) || (v >= C);
         const unsigned peers = peers_of(v, routed, C);
@@ -83,22 +109,32 @@ __global__ void __launch_bounds__(kGroupThreads) group_cluster_kernel(const int3
             hist[w][c] = run;
             run += t;
         }
-        tot[c] = run;
+        if (S == 1) tot_all[0][c] = run;
+        else tot_all[crank][c] = run;      // published to the peers below
     }
-    if (S > 1) cluster_sync_all(); else __syncthreads();
+    if (S > 1) {
+        // push my histogram into every peer's table; one cluster barrier makes all tables complete and visible.
+        // Nothing is read from a peer afterwards, so the CTAs retire independently.
+        __syncthreads();
+        cluster_wait();                    // every peer is running
+        for (int c = threadIdx.x; c < C; c += kGroupThreads) {
+            const int mine = tot_all[crank][c];
+            for (uint32_t q = 0; q < S; ++q)
+                if (q != crank)
+                    asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(map_to_cta(smem_u32(&tot_all[crank][c]), q)), "r"(mine) : "memory");
+        }
+        cluster_sync_all();
+    } else {
+        __syncthreads();
+    }
 
     // global histogram and the part that precedes this CTA
     for (int c = threadIdx.x; c < C; c += kGroupThreads) {
         int all = 0, low = 0;
-        if (S > 1) {
-            for (uint32_t q = 0; q < S; ++q) {
-                int t;
-                asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(t) : "r"(map_to_cta(smem_u32(&tot[c]), q)) : "memory");
-                all += t;
-                if (q < crank) low += t;
-            }
-        } else {
-            all = tot[c];
+        for (uint32_t q = 0; q < S; ++q) {
+            const int t = tot_all[q][c];
+            all += t;
+            if (q < crank) low += t;
         }
         lower[c] = low;
         seg[c + 1] = all;      // shifted by one: turned into the prefix below
@@ -138,7 +174,7 @@ __global__ void __launch_bounds__(kGroupThreads) group_cluster_kernel(const int3
     // stable scatter
     for (int64_t i0 = begin; i0 < end; i0 += 32) {
         const int64_t i = i0 + lane;
-        const int v = i < end ? __ldg(r + i) : -1;
+        const int v = route_of(i0);
         const bool routed = v >= 0 && v < C;
         const unsigned peers = peers_of(v, routed, C);
         if (routed) {
@@ -150,7 +186,6 @@ __global__ void __launch_bounds__(kGroupThreads) group_cluster_kernel(const int3
         __syncwarp();
     }
     if (dev_status != nullptr && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(dev_status, MOLORA_DEV_BAD_ROUTE);
-    if (S > 1) cluster_sync_all();    // peers may still be reading tot[]
 }
 
 size_t group_workspace_bytes(int64_t /*N*/, int32_t /*C*/) { return 0; }
@@ -161,6 +196,7 @@ molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* co
     // one CTA per ~1024 tokens (one 32-token step per warp), at most 8 CTAs
     int split = 1;
     while (split < kGroupMaxCluster && (int64_t)split * 1024 < N) split *= 2;
+    if (const char* e = getenv("MOLORA_GROUP_SPLIT")) split = std::max(1, std::min(atoi(e), kGroupMaxCluster));
     return cuda_ok(launch_kernel(group_cluster_kernel, dim3((unsigned)split), dim3(kGroupThreads), 0, s, (unsigned)split, false,
                                   r, N, C, counts, offsets, perm, dev_status));
 }
