@@ -56,3 +56,21 @@ def test_invalid_arguments_are_refused_before_any_launch():
     assert apply(A=None) == 1
     assert apply(ldy=32) == 1
     assert apply(N=-3) == 1
+
+
+def test_apply_workspace_sizes_and_refusal_without_it():
+    lib = M.load_library()
+    fake = ctypes.c_void_p(0x1000)
+    # the two-launch small-tile path keeps fp32 partial shrink results [slice][N][rank] in the workspace:
+    # 256 tokens, d_in 2048, rank 16 -> 2 slices of 1024 columns -> 2 * 256 * 16 * 4 bytes
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 2 * 256 * 16 * 4
+    assert M.molora_apply_workspace_bytes(256, 8, 6144, 2048, 16) == 6 * 256 * 16 * 4
+    # prefill-sized calls with few adapters run on the tcgen05 kernel alone; rank 8 and fp32-only shapes need none
+    assert M.molora_apply_workspace_bytes(4096, 4, 2048, 2048, 16) == 0
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 8) == 0
+    assert M.molora_apply_workspace_bytes(256, 8, 2040, 2048, 16) == 0
+    # with more than 64 adapters the short segments of a large call take the small-tile path
+    assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 16) > 0
+    # a decode-sized bf16 call without its workspace is refused before anything is enqueued
+    st = lib.molora_apply(fake, 64, fake, 64, M.BF16, 4, 64, 64, 16, fake, fake, 2, fake, fake, 1.0, None, 0, None, None)
+    assert st == 3
