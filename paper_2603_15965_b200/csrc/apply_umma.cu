@@ -67,6 +67,7 @@ struct UmmaProj {
     int64_t ldx, ldy;
     int32_t d_in, d_out, rank;
     float scale;
+    int32_t wide_store;     // y rows are 32-byte aligned: the copy-out uses 256-bit stores
 };
 struct UmmaParams {
     UmmaProj p[MOLORA_MAX_PROJECTIONS];
@@ -448,6 +449,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         int otok[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) otok[i] = ctrl->rows[(et >> 3) + 16 * i];
+        int wtok[4];                                    // 256-bit variant: rows (et >> 2) + 32 i
+#pragma unroll
+        for (int i = 0; i < 4; ++i) wtok[i] = ctrl->rows[(et >> 2) + 32 * i];
         for (int nc = group; nc < NY; nc += kEpiGroups) {
             const int it = KX + nc;
             const int s = it % Cfg::kStages;
@@ -486,16 +490,33 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
             if (et == 0) MOLORA_TR(2, it, 5);
             if (!*abort_flag) {
-                __nv_bfloat16* dstc = pj.y + (ny0 + nc) * kChunkCols + piece * 8;
-                uint4 op[8];
+                if (pj.wide_store) {
+                    // 32 bytes per lane: four lanes cover a 128-byte row segment, a warp instruction eight rows
+                    const int p32 = et & 3;
+                    __nv_bfloat16* dstc = pj.y + (ny0 + nc) * kChunkCols + p32 * 16;
+                    uint4 lo4[4], hi4[4];
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    op[i] = *reinterpret_cast<const uint4*>(
-                        ytile + swizzle_offset((uint32_t)((et >> 3) + 16 * i) * 128u + piece * 16, 3));
-                if (et == 0) MOLORA_TR(2, it, 7);
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t r = (uint32_t)((et >> 2) + 32 * i);
+                        lo4[i] = *reinterpret_cast<const uint4*>(ytile + swizzle_offset(r * 128u + p32 * 32, 3));
+                        hi4[i] = *reinterpret_cast<const uint4*>(ytile + swizzle_offset(r * 128u + p32 * 32 + 16, 3));
+                    }
+                    if (et == 0) MOLORA_TR(2, it, 7);
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (otok[i] >= 0) stg128(dstc + (int64_t)otok[i] * pj.ldy, op[i]);
+                    for (int i = 0; i < 4; ++i)
+                        if (wtok[i] >= 0) stg256(dstc + (int64_t)wtok[i] * pj.ldy, lo4[i], hi4[i]);
+                } else {
+                    __nv_bfloat16* dstc = pj.y + (ny0 + nc) * kChunkCols + piece * 8;
+                    uint4 op[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        op[i] = *reinterpret_cast<const uint4*>(
+                            ytile + swizzle_offset((uint32_t)((et >> 3) + 16 * i) * 128u + piece * 16, 3));
+                    if (et == 0) MOLORA_TR(2, it, 7);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        if (otok[i] >= 0) stg128(dstc + (int64_t)otok[i] * pj.ldy, op[i]);
+                }
             }
             if (et == 0) MOLORA_TR(2, it, 4);
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
@@ -690,6 +711,7 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
         u.d_out = d.d_out;
         u.rank = d.rank;
         u.scale = d.scale;
+        u.wide_store = ((reinterpret_cast<uintptr_t>(d.y) & 31u) == 0 && ((d.ldy * 2) % 32) == 0) ? 1 : 0;
         has[d.rank == 16 ? 0 : d.rank == 32 ? 1 : 2] = true;
     }
     for (int i = P; i < MOLORA_MAX_PROJECTIONS; ++i) prm.p[i].rank = 0;

@@ -49,6 +49,13 @@ __device__ __forceinline__ uint4 ld128_rw_stream(const void* p)
     return v;
 }
 __device__ __forceinline__ void stg128(void* p, uint4 v) { *reinterpret_cast<uint4*>(p) = v; }
+// 256-bit store (sm_100): p is 32-byte aligned
+__device__ __forceinline__ void stg256(void* p, uint4 a, uint4 b)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x),
+                 "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+}
 
 // bf16 pair packed in a 32-bit word -> two fp32 (exact: bf16 is the top half of an fp32).
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t w) { return __uint_as_float(w << 16); }
