@@ -114,9 +114,12 @@ struct UmmaCfg {
     static constexpr uint32_t kWLayout = swizzle_layout_type(static_cast<Swizzle>(kSwzBits));
     // partial T rows received from the cluster peers: (S - 1) * ceil(128 / S) rows of R fp32: 64, 86, 96 rows for
     // S = 2, 3, 4.  Rank 64 stops at S = 3 (shared memory).
+    // Ranks 16 and 32 have room for the whole partial of every peer ((S - 1) * 128 rows): one push, every CTA sums
+    // for itself.
     static constexpr int kMaxSplitR = R == 64 ? 3 : kMaxSplit;
-    static constexpr int kRecvBytes = (R == 64 ? 86 : 96) * R * 4;
-    static constexpr int kCtrlBytes = 1024;
+    static constexpr bool kOnePush = R != 64;
+    static constexpr int kRecvBytes = kOnePush ? (kMaxSplit - 1) * kTileM * R * 4 : 86 * R * 4;
+    static constexpr int kCtrlBytes = 768;
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kTBytes + kRecvBytes + kCtrlBytes;
 };
 
@@ -126,7 +129,7 @@ struct Ctrl {                         // lives in shared memory after the tiles
     int abort_flag;
     alignas(16) int32_t rows[kTileM];
 };
-static_assert(sizeof(Ctrl) <= 1024, "control block must fit its slot");
+static_assert(sizeof(Ctrl) <= 768, "control block must fit its slot");
 
 template <int R>
 __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __grid_constant__ UmmaParams prm)
@@ -344,7 +347,55 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             for (int c = 0; c < R / 16; ++c) tmem_ld_x16(tmem_T + lane_addr + c * 16, tv + c * 16);
             tmem_wait_ld();
             bool t_published = false;
-            if (S > 1) {
+            if (Cfg::kOnePush && S > 1) {
+                // Exchange of the partial T tiles in one push through distributed shared memory: every CTA writes its
+                // partial into its slot at every peer, one barrier round, and every CTA sums all partials itself in
+                // rank order (the same bits in every CTA).  Nothing is read from a peer and nobody touches this CTA's
+                // memory afterwards, so the CTAs of a cluster retire independently.
+                cluster_wait();                                 // every peer is running, its barriers initialised
+                for (uint32_t q2 = 0; q2 < S; ++q2) {
+                    if (q2 == crank) continue;
+                    const uint32_t slot = crank < q2 ? crank : crank - 1;                   // my slot at CTA q2
+                    const uint32_t dst = map_to_cta(recv, q2) + slot * (uint32_t)(kTileM * R * 4);
+#pragma unroll
+                    for (int c4 = 0; c4 < R / 4; ++c4)
+                        st_cluster_u32x4(dst + (uint32_t)(c4 * kTileM + row) * 16u, tv[4 * c4], tv[4 * c4 + 1], tv[4 * c4 + 2],
+                                         tv[4 * c4 + 3]);
+                }
+                __syncwarp();                                   // the warp's rows are sent; lane q2 tells CTA q2
+                if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
+                if (et == 0) MOLORA_TR(3, 2, 2);
+                wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
+                if (et == 0) MOLORA_TR(3, 2, 3);
+#pragma unroll
+                for (int c4 = 0; c4 < R / 4; ++c4) {            // rank order, in place
+                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (uint32_t q2 = 0; q2 < S; ++q2) {
+                        float4 v;
+                        if (q2 == crank) {
+                            v = make_float4(__uint_as_float(tv[4 * c4]), __uint_as_float(tv[4 * c4 + 1]),
+                                            __uint_as_float(tv[4 * c4 + 2]), __uint_as_float(tv[4 * c4 + 3]));
+                        } else {
+                            const uint32_t src = recv + (q2 < crank ? q2 : q2 - 1) * (uint32_t)(kTileM * R * 4);
+                            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                                         : "r"(src + (uint32_t)(c4 * kTileM + row) * 16u)
+                                         : "memory");
+                        }
+                        a.x += v.x;
+                        a.y += v.y;
+                        a.z += v.z;
+                        a.w += v.w;
+                    }
+                    tv[4 * c4] = __float_as_uint(a.x);
+                    tv[4 * c4 + 1] = __float_as_uint(a.y);
+                    tv[4 * c4 + 2] = __float_as_uint(a.z);
+                    tv[4 * c4 + 3] = __float_as_uint(a.w);
+                }
+                if (et == 0) MOLORA_TR(3, 2, 4);
+                if (et == 0) MOLORA_TR(3, 2, 5);
+                // tv now holds the full T row: the local conversion below finishes it
+            } else if (S > 1) {
                 // Exchange of the partial T tiles in two pushes through distributed shared memory.  CTA o owns the
                 // tile rows [o*128/S, (o+1)*128/S): (1) every CTA sends its partial of a row to the row's owner;
                 // (2) the owner sums the partials in rank order (the same bits whoever computes them), scales,
