@@ -152,9 +152,17 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     auto bar = [&](const uint64_t* b) { return smem_u32(b); };
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // ---------------------------------------------------------------- set-up, part 1: nothing read from memory
-    // (runs while the previous kernel of the stream may still be executing)
+    // ---------------------------------------------------------------- set-up
+    // The segment table is requested first; barriers and TMEM are set up while it is on its way.
     if (tid == 0) MOLORA_TR(3, 0, 0);
+    grid_dependency_sync();            // offsets and perm come from the grouping kernel; y from the base projection
+    __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
+    int32_t offs_v[(MOLORA_MAX_ADAPTERS + kUmmaThreads) / kUmmaThreads];
+#pragma unroll
+    for (int j = 0; j < (MOLORA_MAX_ADAPTERS + kUmmaThreads) / kUmmaThreads; ++j) {
+        const int i = tid + j * kUmmaThreads;
+        offs_v[j] = i <= prm.C ? __ldg(prm.offsets + i) : 0;
+    }
     if (tid == 0) {
         prefetch_tensormap(&pj.tm_a);
         prefetch_tensormap(&pj.tm_b);
@@ -177,12 +185,12 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
         tmem_relinquish();
     }
-    grid_dependency_sync();            // offsets and perm come from the grouping kernel; y from the base projection
-
-    // ---------------------------------------------------------------- set-up, part 2: which tile is mine
-    // bring the segment table on chip in one memory round trip, then look the tile up there
-    __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
-    for (int i = tid; i <= prm.C; i += kUmmaThreads) offs_s[i] = __ldg(prm.offsets + i);
+    // which tile is mine: the segment table goes on chip, then the tile is looked up there
+#pragma unroll
+    for (int j = 0; j < (MOLORA_MAX_ADAPTERS + kUmmaThreads) / kUmmaThreads; ++j) {
+        const int i = tid + j * kUmmaThreads;
+        if (i <= prm.C) offs_s[i] = offs_v[j];
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -201,7 +209,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     if (tid == 0) MOLORA_TR(3, 0, 1);
     // "I am running and my barriers are initialised": the matching wait comes right before the first access to
     // a peer's shared memory (the T exchange), so the cluster barrier costs nothing here
-    if (S > 1) cluster_arrive();
+    if (S > 1) cluster_arrive_relaxed();      // (the barrier initialisation was released by fence_mbar_init)
     if (tid == 0) MOLORA_TR(3, 0, 2);
     const uint32_t tmem = ctrl->tmem_base;
     const uint32_t tmem_T = tmem;                               // columns [0, R)
@@ -232,7 +240,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         uint32_t ph = 1;                                        // parity of the "empty" phase to wait for
         for (int it = 0; it < total; ++it) {
             if (tid == 0) MOLORA_TR(0, it, 0);
-            wait_bar(bar(&ctrl->empty[s]), ph, abort_flag, prm.dev_status);
+            if (it >= Cfg::kStages) wait_bar(bar(&ctrl->empty[s]), ph, abort_flag, prm.dev_status);   // first round: all free
             if (tid == 0) MOLORA_TR(0, it, 1);
             const uint32_t dst = stage(s);
             if (!*abort_flag) {
@@ -260,7 +268,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             int s = 0;
             uint32_t ph = 1;
             for (int it = 0; it < total; ++it) {
-                wait_bar(bar(&ctrl->empty[s]), ph, abort_flag, prm.dev_status);
+                if (it >= Cfg::kStages) wait_bar(bar(&ctrl->empty[s]), ph, abort_flag, prm.dev_status);
                 if (*abort_flag) break;
                 const uint32_t fb = bar(&ctrl->full[s]);
                 mbar_arrive_expect_tx(fb, (uint32_t)Cfg::kWBytes);
