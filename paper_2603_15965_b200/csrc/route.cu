@@ -1,4 +1,6 @@
 // Routers: vocabulary-range routing (Definition 3.1) and the linear gate with top-1 argmax (Eq. 8, k = 1).
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 #include "warp_reduce.cuh"
@@ -277,6 +279,118 @@ __global__ void __launch_bounds__(128) route_gate_resident_kernel(const T* __res
     }
 }
 
+// Small calls (at most four tokens per warp, rows of at most eight 16-byte vectors per lane): latency decides, so
+// a warp requests ALL of its activations first (up to 16 KB in flight per warp), while the CTA's copy of G is still
+// on its way into shared memory, and only then starts the FMAs.  Same layout of G and the same summation order per
+// token as route_gate_resident_kernel.
+template <typename T, int CP, int TPW>
+__global__ void __launch_bounds__(128) route_gate_resident_burst_kernel(const T* __restrict__ x, int64_t N, int d,
+                                                                        int64_t ldx, const float* __restrict__ G,
+                                                                        const float* __restrict__ bias, int C,
+                                                                        int32_t* __restrict__ r_out,
+                                                                        float* __restrict__ logits_out)
+{
+    constexpr int VEC = VecTraits<T>::kElems;
+    constexpr int KC = 32 * VEC;
+    constexpr int LANE_STRIDE = VEC * CP + 4;
+    constexpr int MAXCH = 8;                       // chunks per row (the launcher guarantees d <= MAXCH * KC)
+    extern __shared__ __align__(16) float Gres[];  // [chunks][32 lanes][LANE_STRIDE]
+    const int chunks = (d + KC - 1) / KC;
+    const int warp = threadIdx.x >> 5, lane = lane_id();
+    ptx::grid_dependency_sync();
+
+    // ---- all activations of my tokens
+    const int64_t wtok0 = ((int64_t)blockIdx.x * 4 + warp) * TPW;
+    uint4 v[TPW][MAXCH];
+#pragma unroll
+    for (int t = 0; t < TPW; ++t) {
+        const int64_t i = wtok0 + t < N ? wtok0 + t : N - 1;          // tail tokens recompute the last one
+        const T* xi = x + i * ldx + lane * VEC;
+#pragma unroll
+        for (int b = 0; b < MAXCH; ++b)
+            v[t][b] = (b * KC + lane * VEC < d) ? ldg128_stream(xi + b * KC) : make_uint4(0, 0, 0, 0);
+    }
+    // ---- G into shared memory
+    if (C == CP && (d % KC) == 0) {
+        constexpr int V = CP / 4;
+        for (int e = threadIdx.x; e < d * V; e += blockDim.x) {
+            const int k = e / V, vv = e - k * V;
+            const int ch = k / KC, kk = k - ch * KC;
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(
+                &Gres[(ch * 32 + kk / VEC) * LANE_STRIDE + (kk % VEC) * CP + vv * 4]);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(reinterpret_cast<const float4*>(G) + e)
+                         : "memory");
+        }
+        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+    } else {
+        for (int e = threadIdx.x; e < chunks * KC * CP; e += blockDim.x) {
+            const int k = e / CP, c = e - k * CP;
+            const float g = (k < d && c < C) ? __ldg(G + (int64_t)k * C + c) : 0.f;
+            const int ch = k / KC, kk = k - ch * KC;
+            Gres[(ch * 32 + kk / VEC) * LANE_STRIDE + (kk % VEC) * CP + c] = g;
+        }
+    }
+    __syncthreads();
+    if (wtok0 >= N) return;
+
+    float acc[TPW][CP];
+#pragma unroll
+    for (int t = 0; t < TPW; ++t)
+#pragma unroll
+        for (int c = 0; c < CP; ++c) acc[t][c] = 0.f;
+#pragma unroll
+    for (int b = 0; b < MAXCH; ++b) {
+        if (b < chunks) {
+            float f[TPW][VEC];
+#pragma unroll
+            for (int t = 0; t < TPW; ++t) unpack<T>(v[t][b], f[t]);
+            const float* g = Gres + (b * 32 + lane) * LANE_STRIDE;
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) {
+#pragma unroll
+                for (int c4 = 0; c4 < CP; c4 += 4) {
+                    const float4 gv = *reinterpret_cast<const float4*>(g + j * CP + c4);
+#pragma unroll
+                    for (int t = 0; t < TPW; ++t) {
+                        acc[t][c4 + 0] = fmaf(f[t][j], gv.x, acc[t][c4 + 0]);
+                        acc[t][c4 + 1] = fmaf(f[t][j], gv.y, acc[t][c4 + 1]);
+                        acc[t][c4 + 2] = fmaf(f[t][j], gv.z, acc[t][c4 + 2]);
+                        acc[t][c4 + 3] = fmaf(f[t][j], gv.w, acc[t][c4 + 3]);
+                    }
+                }
+            }
+        }
+    }
+    // finish the logits: plain butterfly sums
+#pragma unroll
+    for (int t = 0; t < TPW; ++t)
+#pragma unroll
+        for (int c = 0; c < CP; ++c) {
+            float z = acc[t][c];
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) z += __shfl_xor_sync(0xFFFFFFFFu, z, off);
+            acc[t][c] = z;
+        }
+    if (lane < TPW && wtok0 + lane < N) {
+        const int64_t i = wtok0 + lane;
+        float best = 0.f;
+        int arg = 0;
+#pragma unroll
+        for (int c = 0; c < CP; ++c) {
+            if (c < C) {
+                float z = 0.f;
+#pragma unroll
+                for (int t = 0; t < TPW; ++t)
+                    if (t == lane) z = acc[t][c];
+                if (bias != nullptr) z += __ldg(bias + c);
+                if (logits_out != nullptr) logits_out[i * C + c] = z;
+                if (c == 0 || z > best) { best = z; arg = c; }
+            }
+        }
+        r_out[i] = arg;
+    }
+}
+
 template <typename T, int CP>
 static molora_status_t gate_resident_launch(const void* x, int64_t N, int d, int64_t ldx, const float* G,
                                             const float* bias, int C, int32_t* r_out, float* logits_out,
@@ -298,6 +412,22 @@ static molora_status_t gate_resident_launch(const void* x, int64_t N, int d, int
     int tpw = 8;
     while (tpw > 2 && ceil_div64(N, 4 * tpw) < 148) tpw /= 2;
     const int64_t blocks = ceil_div64(N, 4 * tpw);
+    if (tpw <= 4 && chunks <= 8) {   // small call: the burst variant (every load of a warp in flight at once)
+        static bool configured_burst = false;
+        if (!configured_burst) {
+            if (cudaFuncSetAttribute(route_gate_resident_burst_kernel<T, CP, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     96 * 1024) != cudaSuccess ||
+                cudaFuncSetAttribute(route_gate_resident_burst_kernel<T, CP, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     96 * 1024) != cudaSuccess)
+                return MOLORA_ERR_CUDA;
+            configured_burst = true;
+        }
+        if (tpw == 4)
+            return cuda_ok(launch_kernel(route_gate_resident_burst_kernel<T, CP, 4>, dim3((unsigned)blocks), dim3(128), smem,
+                                         s, 1, false, static_cast<const T*>(x), N, d, ldx, G, bias, C, r_out, logits_out));
+        return cuda_ok(launch_kernel(route_gate_resident_burst_kernel<T, CP, 2>, dim3((unsigned)blocks), dim3(128), smem, s,
+                                     1, false, static_cast<const T*>(x), N, d, ldx, G, bias, C, r_out, logits_out));
+    }
     return cuda_ok(launch_kernel(route_gate_resident_kernel<T, CP>, dim3((unsigned)blocks), dim3(128), smem, s, 1, false,
                                   static_cast<const T*>(x), N, d, ldx, G, bias, C, r_out, logits_out, tpw));
 }
