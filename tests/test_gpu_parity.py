@@ -395,3 +395,23 @@ def test_route_gate_tensor_core_paths(N, d, C):
         eye[np.arange(N), np.arange(N) % d] = 1.0
         M.molora_route_gate(dev_tensor(eye, "bf16"), dev_tensor(G, "f32"), logits_out=logits)
         assert np.array_equal(logits.cpu().numpy(), G[np.arange(N) % d])
+
+
+# ------------------------------------------------------------------ seeded random shapes across every kernel path
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_all_paths(seed):
+    # token counts on both sides of the 1024-token path switch, adapter counts on both sides of the 64-adapter
+    # switch, ranks of every kernel, widths that are multiples of 8 / 32 / 64, skewed routing, unrouted tokens
+    rng = np.random.default_rng(1000 + seed)
+    N = int(rng.choice([1, 17, 130, 700, 1023, 1024, 1500, 2600]))
+    C = int(rng.choice([1, 2, 5, 8, 33, 70]))
+    rank = int(rng.choice([8, 16, 32, 64]))
+    step = int(rng.choice([8, 32, 64]))
+    d_in = step * int(rng.integers(1, 20))
+    d_out = step * int(rng.integers(1, 20))
+    dtype = "f32" if seed % 6 == 5 else "bf16"
+    p = rng.dirichlet(np.full(C, 0.5))                      # skewed segment sizes, some adapters nearly empty
+    r = rng.choice(C, size=N, p=p).astype(np.int32)
+    r[rng.random(N) < 0.05] = -1
+    w = W.random_problem(2000 + seed, N, C, d_in, d_out, rank, dtype, r=r)
+    run_and_check(w, scale=float(rng.choice([1.0, 0.5, 2.0])))
