@@ -415,3 +415,48 @@ def test_random_shapes_all_paths(seed):
     r[rng.random(N) < 0.05] = -1
     w = W.random_problem(2000 + seed, N, C, d_in, d_out, rank, dtype, r=r)
     run_and_check(w, scale=float(rng.choice([1.0, 0.5, 2.0])))
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_route_gate_random_shapes_all_kernels(seed):
+    # resident / burst / chunked CUDA-core kernels, mma.sync and tcgen05 gates: N around the switches at 1024 and
+    # ~2400 / ~4700 tokens, C around 4, 8, 16, 32, hidden sizes with and without whole 64-column chunks
+    rng = np.random.default_rng(500 + seed)
+    N = int(rng.choice([3, 200, 1023, 1025, 2500, 5000]))
+    C = int(rng.choice([1, 3, 4, 5, 8, 9, 16, 17, 32]))
+    d = int(rng.choice([8, 72, 256, 1024, 2048, 2056, 4096]))
+    dtype = "f32" if seed % 5 == 4 else "bf16"
+    x = rng.standard_normal((N, d), dtype=np.float32)
+    if dtype == "bf16":
+        x = W.round_to_bf16(x)
+    G = (rng.standard_normal((d, C)) * d ** -0.5).astype(np.float32)
+    bias = (rng.standard_normal(C) * 0.1).astype(np.float32) if seed % 2 else None
+    r_ref, z_ref, margin = oracle.route_gate(x, G, bias)
+    logits = torch.empty(N, C, dtype=torch.float32, device="cuda")
+    r = M.molora_route_gate(dev_tensor(x, dtype), dev_tensor(G, "f32"),
+                            dev_tensor(bias, "f32") if bias is not None else None, logits_out=logits)
+    assert_close(to_f64(logits), z_ref, 1e-4, 1e-4, what="gate logits")
+    keep = margin >= 1e-3
+    assert np.array_equal(r.cpu().numpy()[keep], r_ref[keep])
+
+
+@pytest.mark.parametrize("N", [300, 1400])
+def test_batched_apply_mixed_ranks_and_paths(N):
+    # one batched call whose projections need different kernels: ranks 16 / 64 (tensor-core or two-launch path),
+    # rank 8 and a width that is only a multiple of 8 (CUDA-core path); shared routing
+    rng = np.random.default_rng(N)
+    C = 6
+    r = rng.integers(0, C, size=N).astype(np.int32)
+    r[rng.random(N) < 0.1] = -1
+    shapes = [(256, 512, 16), (512, 128, 64), (128, 192, 8), (200, 264, 32), (256, 96, 32)]
+    ws = [W.random_problem(7000 + i, N, C, di, do, rk, "bf16", r=r) for i, (di, do, rk) in enumerate(shapes)]
+    counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), C)
+    xs = [dev_tensor(w.inputs["x"], "bf16") for w in ws]
+    ys = [dev_tensor(w.projections[0].y, "bf16") for w in ws]
+    As = [dev_tensor(w.projections[0].A, "bf16") for w in ws]
+    Bs = [dev_tensor(w.projections[0].B, "bf16") for w in ws]
+    M.molora_apply_batched([M.ProjDesc(x, y, A, B, 1.0) for x, y, A, B in zip(xs, ys, As, Bs)], offsets, perm)
+    for w, y in zip(ws, ys):
+        p = w.projections[0]
+        ref, _ = oracle.apply(w.inputs["x"], p.y, p.A, p.B, r)
+        assert_close(to_f64(y), ref, what=f"mixed batch {p.d_in}->{p.d_out} r{p.rank}")
