@@ -228,7 +228,10 @@ def run_ours(args):
     from paper_2603_15965_b200.binding import molora_apply_batched_workspace_bytes
     need = molora_apply_batched_workspace_bytes(sets[0]["packed"][0], N, C)
     shared["apply_ws"] = torch.empty(need, dtype=torch.uint8, device="cuda") if need else None
-    apply_launches = (2 if need else 1) * len({p.rank for p in w.projections})
+    # launches of the apply: one per rank on the tensor-core path, shrink + expand on the small-tile path (which is the
+    # one that asks for a workspace)
+    apply_launches = sum(2 if any(M.molora_apply_workspace_bytes(N, C, p.d_in, p.d_out, p.rank) > 0
+                                  for p in w.projections if p.rank == rk) else 1 for rk in {p.rank for p in w.projections})
     launches_per_step = gate_launches + 1 + apply_launches
     for s in sets:
         s["calls"] = marshal_step(lib, w, s, shared, stream.cuda_stream)
@@ -442,6 +445,9 @@ def oracle_sample(name):
         return W.get("c3"), "the whole step: 256 tokens, group + 7 applies"
     if name == "c4":
         return W.get("c4", n_tokens=512), "512 of 8192 tokens, gate + group + 7 applies"
+    if name.startswith("f9-") or name.startswith("t9-"):
+        w = W.get(name)
+        return w, f"the whole step: {w.N} tokens, group + apply"
     w = W.c5_multimodal(n_seqs=1, seq_len=2048, iid=name == "c5-iid")
     return w, "2048 of 16384 tokens (one sequence), vocab route + group + 2 applies"
 
@@ -505,7 +511,9 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c5-iid"])
+    from paper_2603_15965_b200.workloads import SWEEP_NAMES
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c5-iid", *SWEEP_NAMES],
+                    help="c2 (default, the headline configuration) .. c5; f9-<N> / t9-<skew>: batch and skew sweeps")
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="replay the timed steps from CUDA graphs (default) or launch them one by one")
     ap.add_argument("--max-sets", type=int, default=32)

@@ -147,7 +147,8 @@ molora_status_t molora_group(const int32_t *r, int64_t N, int32_t C, int32_t *co
  * offsets, perm   device outputs of molora_group for the same N, C (read on the device only)
  * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes, 16-byte aligned (NULL if
  *                 that is 0).  Only the small-tile path writes it (fp32 partial shrink results [slice][N][rank]):
- *                 calls below 1024 tokens and, with more than 64 adapters, the short segments of larger calls.
+ *                 calls below 3072 / 1792 / 1280 tokens (rank 16 / 32 / 64) and, with more than 64 adapters, the short segments
+ *                 of larger calls.
  *                 MOLORA_ERR_WORKSPACE if that path is needed and ws is NULL, misaligned or too small.
  * dev_status      device uint32 or NULL; MOLORA_DEV_TIMEOUT is OR-ed in if a bounded wait inside the
  *                 tensor-core kernel gave up (the kernel then returns without hanging; y is incomplete)

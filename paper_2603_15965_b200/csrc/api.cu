@@ -21,14 +21,15 @@ bool chained_launch_enabled()
 
 namespace {
 
-// Calls with fewer tokens than this run on the two-launch small-tile path (tuning override: MOLORA_UMMA_MIN_TOKENS).
-int64_t umma_min_tokens()
+// Calls with fewer tokens than this run on the two-launch small-tile path (tuning override for every rank:
+// MOLORA_UMMA_MIN_TOKENS).
+int64_t umma_min_tokens(int32_t rank)
 {
-    static const int64_t v = [] {
+    static const int64_t forced = [] {
         const char* e = std::getenv("MOLORA_UMMA_MIN_TOKENS");
-        return e != nullptr ? std::max<int64_t>(1, std::atoll(e)) : kUmmaMinTokens;
+        return e != nullptr ? std::max<int64_t>(1, std::atoll(e)) : (int64_t)0;
     }();
-    return v;
+    return forced > 0 ? forced : umma_min_tokens_for_rank(rank);
 }
 
 bool rank_supported(int r) { return r == 8 || r == 16 || r == 32 || r == 64; }
@@ -114,7 +115,7 @@ size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t 
     // the element type is not known here, so the figure assumes bf16 (fp32 calls need none).
     if (N <= 0 || d_in <= 0 || d_out <= 0 || (rank != 16 && rank != 32 && rank != 64)) return 0;
     if ((d_in % 32) != 0 || (d_out % 32) != 0) return 0;
-    if (N >= umma_min_tokens() && C <= kUmmaAllSegmentsMaxC && (d_in % 64) == 0 && (d_out % 64) == 0) return 0;
+    if (N >= umma_min_tokens(rank) && C <= kUmmaAllSegmentsMaxC && (d_in % 64) == 0 && (d_out % 64) == 0) return 0;
     return decode_workspace_bytes(N, d_in, rank);
 }
 
@@ -137,7 +138,7 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
     molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], dc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
     int n_tc = 0, n_dc = 0, n_cc = 0;
     for (int i = 0; i < P; ++i) {
-        if (N >= umma_min_tokens() && umma_eligible(projs[i], dt)) tc[n_tc++] = projs[i];
+        if (N >= umma_min_tokens(projs[i].rank) && umma_eligible(projs[i], dt)) tc[n_tc++] = projs[i];
         else if (decode_eligible(projs[i], dt)) dc[n_dc++] = projs[i];
         else cc[n_cc++] = projs[i];
     }

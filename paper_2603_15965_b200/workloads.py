@@ -86,7 +86,7 @@ class Workload:
 
 def _rng(cfg_index: int, stream: int) -> np.random.Generator:
     """Child stream ``stream`` of configuration ``cfg_index`` (0 = routing source + weights, 1+b = batch b)."""
-    ss = np.random.SeedSequence(ROOT_SEED).spawn(5)[cfg_index]
+    ss = np.random.SeedSequence(ROOT_SEED).spawn(9)[cfg_index]      # children 0..4: c1..c5; 7, 8: the sweeps
     return np.random.default_rng(ss.spawn(stream + 1)[stream])
 
 
@@ -255,9 +255,51 @@ def segment_sizes_routing(sizes) -> np.ndarray:
     return np.asarray(out, dtype=np.int32)
 
 
+# ----------------------------------------------------------------------------- sweeps (Figure 9, Table 9 conditions)
+F9_BATCHES = (64, 128, 256, 512, 1024, 2048)
+T9_SKEWS = {"uniform": (0.25, 0.25, 0.25, 0.25), "80": (0.80, 0.10, 0.05, 0.05), "95": (0.95, 0.02, 0.02, 0.01)}
+
+
+def f9_batch(n_tokens: int) -> Workload:
+    """Batch sweep at the conditions of the paper's kernel study (Figure 9): one projection 4096->4096, rank 64,
+    8 adapters chosen uniformly at random, bf16; n_tokens in F9_BATCHES locates the crossover between the
+    small-tile and the tensor-core path."""
+    wrng, rng = _rng(7, 0), _rng(7, 1 + (F9_BATCHES.index(n_tokens) if n_tokens in F9_BATCHES else len(F9_BATCHES)))
+    N, C, d, rank = n_tokens, 8, 4096, 64
+    A, B = _adapters(wrng, C, d, d, rank, True)
+    r = rng.integers(0, C, size=N).astype(np.int32)
+    return Workload(name=f"f9-{N}", N=N, C=C, dtype="bf16", router="given", inputs={"x": _normal(rng, (N, d), 1.0, True)},
+                    projections=[Projection("proj", "x", d, d, rank, A, B, _normal(rng, (N, d), 1.0, True))], r=r,
+                    seq_id=np.arange(N, dtype=np.int32))
+
+
+def t9_skew(kind: str, n_tokens: int = 2048) -> Workload:
+    """Adapter-load skew at the conditions of Table 9: 4 adapters with the given load split (uniform, 80/10/5/5,
+    95/2/2/1), one projection 4096->4096, rank 64, bf16.  Segment sizes are exact (largest-remainder rounding),
+    token order is shuffled."""
+    wrng, rng = _rng(8, 0), _rng(8, 1)
+    N, C, d, rank = n_tokens, 4, 4096, 64
+    share = np.asarray(T9_SKEWS[kind])
+    sizes = np.floor(share * N).astype(int)
+    sizes[: N - sizes.sum()] += 1
+    r = np.repeat(np.arange(C, dtype=np.int32), sizes)
+    rng.shuffle(r)
+    A, B = _adapters(wrng, C, d, d, rank, True)
+    return Workload(name=f"t9-{kind}", N=N, C=C, dtype="bf16", router="given", inputs={"x": _normal(rng, (N, d), 1.0, True)},
+                    projections=[Projection("proj", "x", d, d, rank, A, B, _normal(rng, (N, d), 1.0, True))], r=r,
+                    seq_id=np.arange(N, dtype=np.int32))
+
+
+SWEEP_NAMES = tuple(f"f9-{n}" for n in F9_BATCHES) + tuple(f"t9-{k}" for k in T9_SKEWS)
+
+
 def get(name: str, **kw) -> Workload:
     table = {"c1": c1_tiny_vocab, "c2": c2_prefill_1p7b, "c3": c3_decode_1p7b, "c4": c4_prefill_8b,
              "c5": c5_multimodal}
     if name == "c5-iid":
         return c5_multimodal(iid=True, **kw)
+    if name.startswith("f9-"):
+        return f9_batch(int(name[3:]))
+    if name.startswith("t9-"):
+        return t9_skew(name[3:], **kw)
     return table[name](**kw)

@@ -65,8 +65,10 @@ def test_apply_workspace_sizes_and_refusal_without_it():
     # 256 tokens, d_in 2048, rank 16 -> 2 slices of 1024 columns -> 2 * 256 * 16 * 4 bytes
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 2 * 256 * 16 * 4
     assert M.molora_apply_workspace_bytes(256, 8, 6144, 2048, 16) == 6 * 256 * 16 * 4
-    # prefill-sized calls with few adapters run on the tcgen05 kernel alone; rank 8 and fp32-only shapes need none
+    # prefill-sized calls with few adapters run on the tcgen05 kernel alone (from 3072 / 1792 / 1280 tokens for ranks
+    # 16 / 32 / 64); rank 8 and fp32-only shapes need none
     assert M.molora_apply_workspace_bytes(4096, 4, 2048, 2048, 16) == 0
+    assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 16) > 0 and M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 64) == 0
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 8) == 0
     assert M.molora_apply_workspace_bytes(256, 8, 2040, 2048, 16) == 0
     # with more than 64 adapters the short segments of a large call take the small-tile path

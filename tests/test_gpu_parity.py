@@ -268,26 +268,28 @@ def test_kpass_per_sequence_baseline_matches_single_pass():
     assert_close(to_f64(out), to_f64(y1), what="k-pass vs one pass")
 
 
-# ------------------------------------------------------------------ tensor-core path (N >= 1024, segments >= 32 rows)
+# ------------------------------------------------------------------ tensor-core path (token counts above the path switch:
+# 3072 tokens for rank 16, 1792 for rank 32, 1280 for rank 64)
 @pytest.mark.parametrize("rank", [16, 32, 64])
 def test_tensor_path_segment_size_sweep(rank):
     # segment sizes straddle the 32-row path threshold, the 4-row gather groups and the 128-row tile
-    sizes = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 130, 131, 255, 256, 257, 300]
+    sizes = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 130, 131, 255, 256, 257, 300, 385, 700]
     r = W.segment_sizes_routing(sizes)
-    assert r.size >= 1024
+    assert r.size >= 3072
     w = W.random_problem(200 + rank, r.size, len(sizes), 256, 320, rank, "bf16", r=r)
     run_and_check(w)
 
 
-@pytest.mark.parametrize("N,C,d_in,d_out,rank", [(1024, 1, 64, 64, 16), (1500, 3, 2048, 1024, 16),
-                                                 (1100, 2, 6144, 2048, 32), (2048, 4, 128, 6144, 64)])
+@pytest.mark.parametrize("N,C,d_in,d_out,rank", [(3072, 1, 64, 64, 16), (3300, 3, 2048, 1024, 16),
+                                                 (1800, 2, 6144, 2048, 32), (2048, 4, 128, 6144, 64),
+                                                 (1280, 5, 4096, 256, 64)])
 def test_tensor_path_shapes(N, C, d_in, d_out, rank):
     w = W.random_problem(N + rank, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.05)
     run_and_check(w, scale=0.75)
 
 
 def test_tensor_path_selector_exact_and_status_clean():
-    N, C, d_in, d_out, rank = 1200, 2, 128, 192, 16
+    N, C, d_in, d_out, rank = 3200, 2, 128, 192, 16
     rng = np.random.default_rng(6)
     x = rng.integers(-8, 9, size=(N, d_in)).astype(np.float32)
     y = rng.integers(-8, 9, size=(N, d_out)).astype(np.float32)
@@ -400,10 +402,10 @@ def test_route_gate_tensor_core_paths(N, d, C):
 # ------------------------------------------------------------------ seeded random shapes across every kernel path
 @pytest.mark.parametrize("seed", range(24))
 def test_random_shapes_all_paths(seed):
-    # token counts on both sides of the 1024-token path switch, adapter counts on both sides of the 64-adapter
+    # token counts on both sides of the per-rank path switches (1280 / 1792 / 3072 tokens), adapter counts on both sides of the 64-adapter
     # switch, ranks of every kernel, widths that are multiples of 8 / 32 / 64, skewed routing, unrouted tokens
     rng = np.random.default_rng(1000 + seed)
-    N = int(rng.choice([1, 17, 130, 700, 1023, 1024, 1500, 2600]))
+    N = int(rng.choice([1, 17, 130, 700, 1279, 1280, 1792, 2600, 3071, 3072, 3500]))
     C = int(rng.choice([1, 2, 5, 8, 33, 70]))
     rank = int(rng.choice([8, 16, 32, 64]))
     step = int(rng.choice([8, 32, 64]))
