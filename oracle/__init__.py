@@ -40,6 +40,7 @@ def _load():
                                                                 ctypes.c_int64))
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_route_vocab.argtypes = [i32p, ctypes.c_int64, i32p, ctypes.c_int32, i32p]
+        lib.oracle_route_composite.argtypes = [i32p, i32p, ctypes.c_int64, i32p, ctypes.c_int32, ctypes.c_int32, i32p]
         lib.oracle_route_gate.argtypes = [f32p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, f32p, f32p,
                                           ctypes.c_int32, i32p, f64p, f64p]
         lib.oracle_group.argtypes = [i32p, ctypes.c_int64, ctypes.c_int32, i32p, i32p, i32p]
@@ -75,6 +76,20 @@ def route_vocab(ids, breaks) -> np.ndarray:
                                     breaks.shape[0] - 1, _p(r, ctypes.c_int32))
     if rc:
         raise ValueError("oracle_route_vocab: invalid arguments")
+    return r
+
+
+def route_composite(ids, adapter, breaks, n_adapters: int) -> np.ndarray:
+    """Definition 3.2 / Algorithm 1: r[t] = adapter[t] * M + m(ids[t]); -1 if the id is in no range or the adapter
+    index is outside [0, n_adapters)."""
+    ids, adapter, breaks = _i32(ids), _i32(adapter), _i32(breaks)
+    assert adapter.shape == ids.shape
+    r = np.empty(ids.shape[0], dtype=np.int32)
+    rc = _load().oracle_route_composite(_p(ids, ctypes.c_int32), _p(adapter, ctypes.c_int32), ids.shape[0],
+                                        _p(breaks, ctypes.c_int32), breaks.shape[0] - 1, int(n_adapters),
+                                        _p(r, ctypes.c_int32))
+    if rc:
+        raise ValueError("oracle_route_composite: invalid arguments")
     return r
 
 

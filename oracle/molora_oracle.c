@@ -52,6 +52,24 @@ int oracle_route_vocab(const int32_t *ids, int64_t N, const int32_t *breaks, int
     return 0;
 }
 
+/* Compositional routing (Definition 3.2, Algorithm 1 lines 4-6): a <- adapter index of the token from the request
+ * metadata, m <- FindModality(v, b), c <- a * |M| + m.  A token whose id lies in no range, or whose adapter index
+ * is outside [0, n_adapters), is unrouted (-1). */
+int oracle_route_composite(const int32_t *ids, const int32_t *adapter, int64_t N, const int32_t *breaks, int32_t M,
+                           int32_t n_adapters, int32_t *r)
+{
+    if (N < 0 || M <= 0 || n_adapters <= 0) return 1;
+    for (int64_t t = 0; t < N; ++t) {
+        const int32_t a = adapter[t];
+        int32_t m = -1;
+        for (int32_t j = 0; j < M; ++j) {
+            if (breaks[j] <= ids[t] && ids[t] < breaks[j + 1]) { m = j; break; }
+        }
+        r[t] = (m >= 0 && a >= 0 && a < n_adapters) ? a * M + m : -1;
+    }
+    return 0;
+}
+
 /* Linear gate with top-1 selection (Eq. 8 with k = 1; the gate of Theorem 3.4 / Table 10 is
  * softmax(W x + b)).  Softmax is monotone, so the winner is the argmax of the raw logits
  * z[i][c] = sum_k x[i][k] * G[k][c] (+ bias[c]); with a single kept logit the softmax weight is 1.

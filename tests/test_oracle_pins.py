@@ -87,6 +87,26 @@ def test_composite_target_range(golden_dir):
     assert np.unique(c).size == int(g["composite_targets"][0]) and c.min() == 0 and c.max() == 255
 
 
+def test_composite_routing_pins():
+    # Definition 3.2 / Algorithm 1: c = a * |M| + m.  Pins: adapter 0 reduces to vocabulary routing; the pair (a, m)
+    # is recovered by divmod; every one of the |A| * |M| targets of Example 3.3 is hit exactly once by one token per
+    # (a, m); an id outside every range or an adapter outside [0, |A|) is unrouted.
+    breaks = np.array([0, 100, 250, 251, 1000], np.int32)            # four ranges, one of a single id
+    rng = np.random.default_rng(5)
+    ids = rng.integers(0, 1000, size=500).astype(np.int32)
+    m = oracle.route_vocab(ids, breaks)
+    assert np.array_equal(oracle.route_composite(ids, np.zeros_like(ids), breaks, 64), m)
+    a = rng.integers(0, 64, size=500).astype(np.int32)
+    c = oracle.route_composite(ids, a, breaks, 64)
+    assert np.array_equal(c // 4, a) and np.array_equal(c % 4, m)
+    one_id_per_range = np.array([0, 100, 250, 251], np.int32)
+    aa, mm = np.meshgrid(np.arange(64, dtype=np.int32), np.arange(4), indexing="ij")
+    c = oracle.route_composite(one_id_per_range[mm.ravel()], aa.ravel(), breaks, 64)
+    assert np.array_equal(np.sort(c), np.arange(256))
+    c = oracle.route_composite(np.array([5, 1000, 5, -1], np.int32), np.array([3, 3, 64, 0], np.int32), breaks, 64)
+    assert c.tolist() == [12, -1, -1, -1]
+
+
 # ------------------------------------------------------------------ linear gate, top-1 (Eq. 8, k = 1)
 def test_gate_unit_vectors_read_rows_of_G():
     rng = np.random.default_rng(2)
