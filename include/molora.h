@@ -77,6 +77,17 @@ molora_status_t molora_route_vocab(const int32_t *ids, int64_t N, const int32_t 
                                    uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Router 1b: compositional routing (Definition 3.2; Algorithm 1 "Compositional Gating Kernel", lines 4-6): the
+ * modality of a token comes from its vocabulary index as above, its adapter from the request metadata, and the
+ * composite target indexes a weight stack of shape (n_adapters, M, d, r):
+ *     r_out[i] = adapter[i] * M + m(ids[i]);   -1 if ids[i] lies in no range or adapter[i] is outside [0, n_adapters).
+ * adapter  device int32[N]   adapter index of every token (constant inside a request); M * n_adapters <= 256
+ * The result feeds molora_group / molora_apply with C = n_adapters * M (Example 3.3: 64 x 4 = 256 targets).
+ * dev_status  MOLORA_DEV_ID_OUT_OF_RANGE is OR-ed in if any token is left unrouted.  Integer work, exact. */
+molora_status_t molora_route_composite(const int32_t *ids, const int32_t *adapter, int64_t N, const int32_t *breaks,
+                                       int32_t M, int32_t n_adapters, int32_t *r_out, uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Router 2: learned linear gate with top-1 selection (Eq. 8 with k = 1; gate form softmax(W x + b) of
  * Theorem 3.4 / Table 10).  Softmax is monotone and the weight of a single kept logit is 1, so
  *     z[i][c] = sum_k x[i][k] * G[k][c] (+ bias[c]),    r_out[i] = argmax_c z[i][c]  (lowest c on ties).

@@ -69,6 +69,7 @@ def load_library():
     lib.molora_status_string.restype = ctypes.c_char_p
     lib.molora_status_string.argtypes = [ctypes.c_int]
     lib.molora_route_vocab.argtypes = [vp, i64, vp, i32, vp, vp, vp]
+    lib.molora_route_composite.argtypes = [vp, vp, i64, vp, i32, i32, vp, vp, vp]
     lib.molora_route_gate_workspace_bytes.restype = sz
     lib.molora_route_gate_workspace_bytes.argtypes = [ctypes.c_int, i32, i32]
     lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp]
@@ -153,6 +154,23 @@ def molora_route_vocab(ids: torch.Tensor, breaks: torch.Tensor, r_out: Optional[
         r_out = torch.empty(N, dtype=torch.int32, device=ids.device)
     _check("molora_route_vocab", lib.molora_route_vocab(_ptr(ids), N, _ptr(breaks), M, _ptr(_i32_dev(r_out, "r_out")),
                                                         _ptr(dev_status), _stream(stream)))
+    return r_out
+
+
+def molora_route_composite(ids: torch.Tensor, adapter: torch.Tensor, breaks: torch.Tensor, n_adapters: int,
+                           r_out: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                           stream=None) -> torch.Tensor:
+    """r_out[i] = adapter[i] * M + m(ids[i]) (Definition 3.2 / Algorithm 1); -1 if the token is unrouted."""
+    lib = load_library()
+    _i32_dev(ids, "ids"), _i32_dev(adapter, "adapter"), _i32_dev(breaks, "breaks")
+    N, M = ids.numel(), breaks.numel() - 1
+    if adapter.numel() != N:
+        raise ValueError("adapter must hold one index per token")
+    if r_out is None:
+        r_out = torch.empty(N, dtype=torch.int32, device=ids.device)
+    _check("molora_route_composite", lib.molora_route_composite(_ptr(ids), _ptr(adapter), N, _ptr(breaks), M,
+                                                                int(n_adapters), _ptr(_i32_dev(r_out, "r_out")),
+                                                                _ptr(dev_status), _stream(stream)))
     return r_out
 
 

@@ -71,7 +71,17 @@ molora_status_t molora_route_vocab(const int32_t* ids, int64_t N, const int32_t*
     if (M < 1) return MOLORA_ERR_INVALID_ARG;
     if (M > MOLORA_MAX_ADAPTERS) return MOLORA_ERR_UNSUPPORTED;
     if (breaks == nullptr || (N > 0 && (ids == nullptr || r_out == nullptr))) return MOLORA_ERR_INVALID_ARG;
-    return launch_route_vocab(ids, N, breaks, M, r_out, dev_status, static_cast<cudaStream_t>(stream));
+    return launch_route_vocab(ids, N, breaks, M, nullptr, 0, r_out, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+molora_status_t molora_route_composite(const int32_t* ids, const int32_t* adapter, int64_t N, const int32_t* breaks,
+                                       int32_t M, int32_t n_adapters, int32_t* r_out, uint32_t* dev_status, void* stream)
+{
+    if (N < 0 || N >= INT32_MAX) return MOLORA_ERR_INVALID_ARG;
+    if (M < 1 || n_adapters < 1) return MOLORA_ERR_INVALID_ARG;
+    if ((int64_t)M * n_adapters > MOLORA_MAX_ADAPTERS) return MOLORA_ERR_UNSUPPORTED;
+    if (breaks == nullptr || (N > 0 && (ids == nullptr || adapter == nullptr || r_out == nullptr))) return MOLORA_ERR_INVALID_ARG;
+    return launch_route_vocab(ids, N, breaks, M, adapter, n_adapters, r_out, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 size_t molora_route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
@@ -298,7 +308,7 @@ molora_status_t molora_forward_host(molora_router_t router, const int32_t* route
     // 2. route
     molora_status_t st = MOLORA_OK;
     if (router == MOLORA_ROUTE_VOCAB) {
-        st = launch_route_vocab(ids, N, breaks_dev, M, r, dev_status, s);
+        st = launch_route_vocab(ids, N, breaks_dev, M, nullptr, 0, r, dev_status, s);
     } else if (router == MOLORA_ROUTE_GATE) {
         const molora_proj_desc_t& gp = dev[gate_proj];
         if ((gp.d_in % 8) != 0) return MOLORA_ERR_UNSUPPORTED;

@@ -156,8 +156,10 @@ __device__ __forceinline__ bool find_tile_smem(const int32_t* offs, int C, int t
 }
 
 // Host launchers implemented in the .cu files (stream already unwrapped).
-molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M, int32_t* r_out,
-                                   uint32_t* dev_status, cudaStream_t s);
+// adapter == nullptr: vocabulary routing; otherwise the compositional gate (r = adapter[i] * M + m)
+molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M,
+                                   const int32_t* adapter, int32_t n_adapters, int32_t* r_out, uint32_t* dev_status,
+                                   cudaStream_t s);
 // tcgen05 gate (bf16 activations, C > 4, d a multiple of 64, at least 1024 tokens).
 bool gate_umma_eligible(int64_t N, int32_t d, int32_t C);
 size_t route_gate_umma_workspace_bytes(int32_t d, int32_t C);

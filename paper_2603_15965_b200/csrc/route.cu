@@ -13,8 +13,11 @@ namespace molora {
 // (an empty range b_m == b_{m+1} can hold no id and is skipped by the count).  M-1 integer compares
 // per token, as the paper notes for Theorem 3.4; boundaries live in shared memory.
 // ------------------------------------------------------------------------------------------------
+// With `adapter` non-null the kernel is the compositional gate of Algorithm 1 (Definition 3.2): the modality m found
+// from the id is combined with the token's adapter index a (request metadata) into the composite target a * M + m.
 __global__ void __launch_bounds__(256) route_vocab_kernel(const int32_t* __restrict__ ids, int64_t N,
                                                           const int32_t* __restrict__ breaks, int M,
+                                                          const int32_t* __restrict__ adapter, int n_adapters,
                                                           int32_t* __restrict__ r_out, uint32_t* dev_status)
 {
     __shared__ int32_t b[MOLORA_MAX_ADAPTERS + 1];
@@ -38,7 +41,12 @@ __global__ void __launch_bounds__(256) route_vocab_kernel(const int32_t* __restr
             }
             m = lo - 1;
         }
-        const bool inside = (v >= b[0]) && (v < b[M]);
+        bool inside = (v >= b[0]) && (v < b[M]);
+        if (adapter != nullptr) {
+            const int32_t a = __ldg(adapter + i);
+            inside = inside && a >= 0 && a < n_adapters;
+            m += a * M;
+        }
         r_out[i] = inside ? m : -1;
         any_bad |= !inside;
     }
@@ -46,15 +54,16 @@ __global__ void __launch_bounds__(256) route_vocab_kernel(const int32_t* __restr
         atomicOr(dev_status, MOLORA_DEV_ID_OUT_OF_RANGE);
 }
 
-molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M, int32_t* r_out,
-                                   uint32_t* dev_status, cudaStream_t s)
+molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M,
+                                   const int32_t* adapter, int32_t n_adapters, int32_t* r_out, uint32_t* dev_status,
+                                   cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
     const int threads = 256;
     const int64_t want = ceil_div64(N, threads);
     const int blocks = (int)(want < 148 * 8 ? want : 148 * 8);
-    return cuda_ok(launch_kernel(route_vocab_kernel, dim3(blocks), dim3(threads), 0, s, 1, false, ids, N, breaks, M, r_out,
-                                  dev_status));
+    return cuda_ok(launch_kernel(route_vocab_kernel, dim3(blocks), dim3(threads), 0, s, 1, false, ids, N, breaks, M, adapter,
+                                  n_adapters, r_out, dev_status));
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -66,6 +66,36 @@ def test_route_vocab_boundaries_empty_ranges_and_status():
     assert np.array_equal(r.cpu().numpy(), oracle.route_vocab(inside, breaks)) and int(status.item()) == 0
 
 
+def test_route_composite_example_3_3_end_to_end():
+    # 64 adapters x 4 modalities = 256 composite targets (Example 3.3): routing bit-exact against the oracle, then the
+    # whole path (group + apply over C = 256) against the oracle's apply on the oracle's routing
+    breaks = np.array([0, 4000, 6000, 7000, 8000], np.int32)
+    rng = np.random.default_rng(33)
+    N, n_adapters, n_mod = 2000, 64, 4
+    ids = rng.integers(-50, 8100, size=N).astype(np.int32)                  # a few ids outside every range
+    seq_adapter = rng.integers(0, n_adapters, size=40).astype(np.int32)     # 40 requests of 50 tokens, one adapter each
+    adapter = np.repeat(seq_adapter, 50)
+    adapter[7] = 64                                                         # an adapter index outside [0, 64)
+    r_ref = oracle.route_composite(ids, adapter, breaks, n_adapters)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    r = M_route_composite(ids, adapter, breaks, n_adapters, status)
+    assert np.array_equal(r.cpu().numpy(), r_ref)
+    assert (int(status.item()) & 1) == 1 and r_ref[7] == -1
+    C = n_adapters * n_mod
+    w = W.random_problem(91, N, C, 256, 128, 16, "bf16", r=r_ref)
+    counts, offsets, perm = M.molora_group(r, C)
+    p = w.projections[0]
+    y = dev_tensor(p.y, "bf16")
+    M.molora_apply(dev_tensor(w.inputs["x"], "bf16"), y, dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), offsets, perm)
+    ref, _ = oracle.apply(w.inputs["x"], p.y, p.A, p.B, r_ref)
+    assert_close(to_f64(y), ref, what="composite routing, 256 targets")
+
+
+def M_route_composite(ids, adapter, breaks, n_adapters, status):
+    return M.molora_route_composite(dev_tensor(ids, "i"), dev_tensor(adapter, "i"), dev_tensor(breaks, "i"), n_adapters,
+                                    dev_status=status)
+
+
 def test_route_vocab_many_ranges():
     rng = np.random.default_rng(1)
     breaks = np.concatenate([[0], np.sort(rng.integers(1, 100000, size=255)), [100000]]).astype(np.int32)
