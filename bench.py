@@ -314,6 +314,25 @@ def run_ours(args):
             total_ms = t0.elapsed_time(t1)
             apply_ms = float(np.mean([a.elapsed_time(b) for p in pairs if p is not None for a, b in [p]]))
             kernel_timing = "CUDA event pair around every apply call (includes host launch gaps)"
+        # latency of a single step replayed on its own (one graph per buffer set, one event pair per replay): the
+        # distribution the paper reports for graph replay (median, P99, coefficient of variation)
+        latency = None
+        if args.launch == "graph" and not args.profile:
+            singles = [capture(step, i, 1) for i in range(min(n_sets, 8))]
+            n_lat = 400
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
+            for i in range(16):
+                singles[i % len(singles)].replay()
+            torch.cuda.synchronize()
+            for i, (e0, e1) in enumerate(evs):
+                e0.record(stream)
+                singles[i % len(singles)].replay()
+                e1.record(stream)
+            torch.cuda.synchronize()
+            lat = np.sort(np.array([e0.elapsed_time(e1) * 1e3 for e0, e1 in evs]))
+            latency = {"p50_us": float(lat[len(lat) // 2]), "p99_us": float(lat[int(len(lat) * 0.99) - 1]),
+                       "cv": float(lat.std() / lat.mean()), "samples": n_lat,
+                       "note": "one step per CUDA-graph replay, event pair around each replay (includes the graph launch)"}
         if dist is not None:
             dist.barrier()
         # keep the GPU busy a little longer (untimed) if the region was too short for the clock sampler
@@ -335,7 +354,7 @@ def run_ours(args):
         peaks = measured_peaks()
         achieved = step_bytes / (apply_ms * 1e-3) / 1e9
         out = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "metric": METRIC, "value": value, "unit": UNIT, "latency": latency, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": f"{name}: N={N} tokens/GPU, C={C}, " + ", ".join(
