@@ -27,7 +27,7 @@ def build(force: bool = False) -> str:
     """Compile the oracle with gcc (no fast-math: summation order is part of the definition)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + f".{os.getpid()}.tmp"
-        subprocess.run(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC], check=True)
+        subprocess.run(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"], check=True)
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -41,6 +41,8 @@ def _load():
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_route_vocab.argtypes = [i32p, ctypes.c_int64, i32p, ctypes.c_int32, i32p]
         lib.oracle_route_composite.argtypes = [i32p, i32p, ctypes.c_int64, i32p, ctypes.c_int32, ctypes.c_int32, i32p]
+        lib.oracle_route_mlp.argtypes = [f32p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, f32p, f32p, ctypes.c_int32, f32p,
+                                         f32p, ctypes.c_int32, i32p, f64p, f64p, f64p]
         lib.oracle_route_gate.argtypes = [f32p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, f32p, f32p,
                                           ctypes.c_int32, i32p, f64p, f64p]
         lib.oracle_group.argtypes = [i32p, ctypes.c_int64, ctypes.c_int32, i32p, i32p, i32p]
@@ -91,6 +93,27 @@ def route_composite(ids, adapter, breaks, n_adapters: int) -> np.ndarray:
     if rc:
         raise ValueError("oracle_route_composite: invalid arguments")
     return r
+
+
+def route_mlp(x, W1, b1, W2, b2, return_hidden: bool = False):
+    """The paper's router (Eq. 9), top-1: g(x) = W2 GELU(W1 x + b1) + b2 with W1 [d, H], W2 [H, C] (input-major) and
+    the exact erf GELU.  Returns (r, logits z [N, C] fp64, margin top1 - top2 [N]) (+ hidden [N, H] if asked)."""
+    x, W1, W2 = _f32(x), _f32(W1), _f32(W2)
+    N, d = x.shape
+    H, C = W2.shape
+    assert W1.shape == (d, H) and H <= 1024
+    b1 = None if b1 is None else _f32(b1)
+    b2 = None if b2 is None else _f32(b2)
+    r = np.empty(N, dtype=np.int32)
+    z = np.empty((N, C), dtype=np.float64)
+    margin = np.empty(N, dtype=np.float64)
+    h = np.empty((N, H), dtype=np.float64)
+    rc = _load().oracle_route_mlp(_p(x, ctypes.c_float), N, d, d, _p(W1, ctypes.c_float), _p(b1, ctypes.c_float), H,
+                                  _p(W2, ctypes.c_float), _p(b2, ctypes.c_float), C, _p(r, ctypes.c_int32),
+                                  _p(z, ctypes.c_double), _p(margin, ctypes.c_double), _p(h, ctypes.c_double))
+    if rc:
+        raise ValueError("oracle_route_mlp: invalid arguments")
+    return (r, z, margin, h) if return_hidden else (r, z, margin)
 
 
 def route_gate(x, G, bias=None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:

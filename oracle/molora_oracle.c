@@ -20,6 +20,7 @@
  * closed forms, the grouping example of Figure 2, upper_bound for vocabulary routing, exhaustive
  * routings on integer data, permutation equivariance, the N vs K*N work count of Theorem 3.6).
  */
+#include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -87,6 +88,41 @@ int oracle_route_gate(const float *x, int64_t N, int32_t d, int64_t ldx, const f
             double z = 0.0;
             for (int32_t k = 0; k < d; ++k) z += (double)x[i * ldx + k] * (double)G[(int64_t)k * C + c];
             if (bias) z += (double)bias[c];
+            if (z_out) z_out[i * C + c] = z;
+            if (arg < 0) { best = z; arg = c; second = -1e300; }
+            else if (z > best) { second = best; best = z; arg = c; }
+            else if (z > second) { second = z; }
+        }
+        r[i] = arg;
+        if (margin_out) margin_out[i] = (C > 1) ? best - second : 1e300;
+    }
+    return 0;
+}
+
+/* The paper's router (Eq. 9): g(x) = W2 GELU(W1 x + b1) + b2, a 2-layer MLP with hidden width H (64 in Eq. 9, 128 in
+ * the 2560 -> 128 -> 4 variant of the appendix), followed by top-1 selection as in oracle_route_gate.  GELU is the
+ * exact form t * Phi(t) = t * (1 + erf(t / sqrt 2)) / 2.  Weights are stored input-major: W1[d][H], W2[H][C].
+ * z_out (optional) receives the logits, h_out (optional) the hidden activations after GELU. */
+int oracle_route_mlp(const float *x, int64_t N, int32_t d, int64_t ldx, const float *W1, const float *b1, int32_t H,
+                     const float *W2, const float *b2, int32_t C, int32_t *r, double *z_out, double *margin_out,
+                     double *h_out)
+{
+    if (N < 0 || d <= 0 || H <= 0 || C <= 0 || ldx < d) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < N; ++i) {
+        double h[1024];
+        if (H > 1024) continue;
+        for (int32_t j = 0; j < H; ++j) {
+            double t = b1 ? (double)b1[j] : 0.0;
+            for (int32_t k = 0; k < d; ++k) t += (double)W1[(int64_t)k * H + j] * (double)x[i * ldx + k];
+            h[j] = 0.5 * t * (1.0 + erf(t / sqrt(2.0)));
+            if (h_out) h_out[i * H + j] = h[j];
+        }
+        double best = 0.0, second = 0.0;
+        int32_t arg = -1;
+        for (int32_t c = 0; c < C; ++c) {
+            double z = b2 ? (double)b2[c] : 0.0;
+            for (int32_t j = 0; j < H; ++j) z += (double)W2[(int64_t)j * C + c] * h[j];
             if (z_out) z_out[i * C + c] = z;
             if (arg < 0) { best = z; arg = c; second = -1e300; }
             else if (z > best) { second = best; best = z; arg = c; }

@@ -28,6 +28,48 @@ def _small(seed, N=37, C=3, d_in=24, d_out=40, rank=4, dtype="f32", **kw):
     return W.random_problem(seed, N, C, d_in, d_out, rank, dtype, **kw)
 
 
+# ------------------------------------------------------------------ the paper's router (Eq. 9): 2-layer MLP, GELU
+def test_mlp_router_pins():
+    from scipy.stats import norm
+    rng = np.random.default_rng(9)
+    d, H, C, N = 10, 6, 4, 50
+    x = rng.standard_normal((N, d)).astype(np.float32)
+    W1 = rng.standard_normal((d, H)).astype(np.float32)
+    b1 = rng.standard_normal(H).astype(np.float32)
+    W2 = rng.standard_normal((H, C)).astype(np.float32)
+    b2 = rng.standard_normal(C).astype(np.float32)
+    r, z, margin, h = oracle.route_mlp(x, W1, b1, W2, b2, return_hidden=True)
+    # hidden layer: GELU(t) = t * Phi(t) with Phi from an independent routine (the normal CDF), t by library matmul
+    t = x.astype(np.float64) @ W1.astype(np.float64) + b1
+    assert np.allclose(h, t * norm.cdf(t), rtol=1e-12, atol=1e-14)
+    # output layer, argmax with lowest index on ties, margin = top1 - top2
+    zz = h @ W2.astype(np.float64) + b2
+    assert np.allclose(z, zz, rtol=1e-12, atol=1e-13)
+    assert np.array_equal(r, np.argmax(zz, axis=1))
+    srt = np.sort(zz, axis=1)
+    assert np.allclose(margin, srt[:, -1] - srt[:, -2], rtol=1e-12, atol=1e-13)
+    # unit vectors read rows of W1 (catches a transposed first layer); W2 = identity exposes the hidden layer
+    _, z1, _, h1 = oracle.route_mlp(np.eye(d, dtype=np.float32), W1, None, np.eye(H, dtype=np.float32), None,
+                                    return_hidden=True)
+    assert np.allclose(h1, W1 * norm.cdf(W1.astype(np.float64)), rtol=1e-12, atol=1e-14) and np.array_equal(z1, h1)
+    # closed forms: GELU(0) = 0, and far in the positive tail GELU is the identity, so the MLP collapses to the
+    # (already pinned) linear gate with G = W1 W2 and bias = b1 W2 + b2
+    r0, z0, _ = oracle.route_mlp(np.zeros((3, d), np.float32), W1, None, W2, b2)
+    assert np.allclose(z0, np.broadcast_to(b2.astype(np.float64), (3, C)))
+    big = (np.abs(W1) + 1.0).astype(np.float32)
+    xb = (np.abs(x) + 1.0).astype(np.float32)
+    bb = np.full(H, 40.0, np.float32)                              # pre-activations >= 40: Phi(t) == 1 in fp64
+    rb, zb, _ = oracle.route_mlp(xb, big, bb, W2, b2)
+    G = (big.astype(np.float64) @ W2.astype(np.float64))
+    lin = xb.astype(np.float64) @ G + (bb.astype(np.float64) @ W2.astype(np.float64) + b2)
+    assert np.allclose(zb, lin, rtol=1e-12) and np.array_equal(rb, np.argmax(lin, axis=1))
+    # ties go to the lowest index: two identical output columns
+    W2t = W2.copy(); W2t[:, 3] = W2t[:, 1]
+    b2t = b2.copy(); b2t[3] = b2t[1]
+    rt, zt, mt = oracle.route_mlp(x, W1, b1, W2t, b2t)
+    assert not np.any(rt == 3) and np.all(mt[(rt == 1)] == 0.0)
+
+
 # ------------------------------------------------------------------ grouping (Section 3.3, Figure 2)
 def test_group_matches_figure2_example(golden_dir):
     g = _read_golden(os.path.join(golden_dir, "fig2_grouping.txt"))
