@@ -106,6 +106,24 @@ molora_status_t molora_route_gate(const void *x, molora_dtype_t xdt, int64_t N, 
                                   size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Router 3: the paper's learned router (Eq. 9), a 2-layer MLP with GELU, followed by top-1 selection:
+ *     g(x_i) = W2 GELU(W1 x_i + b1) + b2,    r_out[i] = argmax_c g(x_i)[c]  (lowest c on ties)
+ * with the exact GELU(t) = t (1 + erf(t / sqrt 2)) / 2.
+ * x        device [N, d] of type xdt, row pitch ldx >= d elements; d a multiple of 8; never written
+ * W1       device fp32 [d, H] row-major (input-major);  b1  device fp32 [H] or NULL;  1 <= H <= 128 (the paper: 64, 128)
+ * W2       device fp32 [H, C] row-major;                b2  device fp32 [C] or NULL;  1 <= C <= 32
+ * r_out    device int32[N];  logits_out  device fp32 [N, C] or NULL
+ * ws, ws_bytes  device scratch of at least molora_route_mlp_workspace_bytes(xdt, d, H, C) bytes, 16-byte aligned (NULL
+ *               when that is 0): for bf16 x and d a multiple of 64 the first layer runs on the tensor cores with a
+ *               three-term bf16 split of W1 kept there (rebuilt on every call); MOLORA_ERR_WORKSPACE if it is
+ *               needed (at least 128 tokens) and missing.
+ * Products of the first layer are exact in fp32 for bf16 x; accumulation, GELU and the second layer are fp32. */
+size_t molora_route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H, int32_t C);
+molora_status_t molora_route_mlp(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float *W1,
+                                 const float *b1, int32_t H, const float *W2, const float *b2, int32_t C, int32_t *r_out,
+                                 float *logits_out, void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * The same gate for callers that cannot provide a workspace.  (The paper has no counterpart: this entry point
  * exists for integration reasons only.)  Some hosts of this library may not allocate device memory at the
  * point where they route tokens -- code running between the capture and replay of a fixed-address serving

@@ -70,6 +70,9 @@ def load_library():
     lib.molora_status_string.argtypes = [ctypes.c_int]
     lib.molora_route_vocab.argtypes = [vp, i64, vp, i32, vp, vp, vp]
     lib.molora_route_composite.argtypes = [vp, vp, i64, vp, i32, i32, vp, vp, vp]
+    lib.molora_route_mlp_workspace_bytes.restype = sz
+    lib.molora_route_mlp_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i32]
+    lib.molora_route_mlp.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
     lib.molora_route_gate_workspace_bytes.restype = sz
     lib.molora_route_gate_workspace_bytes.argtypes = [ctypes.c_int, i32, i32]
     lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp]
@@ -171,6 +174,34 @@ def molora_route_composite(ids: torch.Tensor, adapter: torch.Tensor, breaks: tor
     _check("molora_route_composite", lib.molora_route_composite(_ptr(ids), _ptr(adapter), N, _ptr(breaks), M,
                                                                 int(n_adapters), _ptr(_i32_dev(r_out, "r_out")),
                                                                 _ptr(dev_status), _stream(stream)))
+    return r_out
+
+
+def molora_route_mlp_workspace_bytes(xdt: int, d: int, H: int, C: int) -> int:
+    return int(load_library().molora_route_mlp_workspace_bytes(xdt, d, H, C))
+
+
+def molora_route_mlp(x: torch.Tensor, W1: torch.Tensor, b1: Optional[torch.Tensor], W2: torch.Tensor,
+                     b2: Optional[torch.Tensor], r_out: Optional[torch.Tensor] = None,
+                     logits_out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
+                     stream=None) -> torch.Tensor:
+    """r_out[i] = argmax_c (W2 GELU(W1 x_i + b1) + b2)[c] (Eq. 9, top-1); W1 [d, H], W2 [H, C] fp32."""
+    lib = load_library()
+    N, d, ldx = _matrix(x, "x")
+    if W1.dtype != torch.float32 or W2.dtype != torch.float32 or not W1.is_contiguous() or not W2.is_contiguous():
+        raise ValueError("W1 [d, H] and W2 [H, C] must be dense fp32 tensors")
+    H, C = W2.shape
+    if tuple(W1.shape) != (d, H):
+        raise ValueError("W1 must be [d, H]")
+    if r_out is None:
+        r_out = torch.empty(N, dtype=torch.int32, device=x.device)
+    need = molora_route_mlp_workspace_bytes(_dtype_code(x), d, H, C)
+    if ws is None and need > 0:
+        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check("molora_route_mlp", lib.molora_route_mlp(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(W1), _ptr(b1), H, _ptr(W2),
+                                                    _ptr(b2), C, _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
+                                                    _ptr(ws), ws_bytes, _stream(stream)))
     return r_out
 
 

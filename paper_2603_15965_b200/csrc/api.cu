@@ -104,6 +104,26 @@ molora_status_t molora_route_gate(const void* x, molora_dtype_t xdt, int64_t N, 
     return launch_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, ws, static_cast<cudaStream_t>(stream));
 }
 
+size_t molora_route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H, int32_t C)
+{
+    if (d <= 0 || H < 1 || H > 128 || C < 1 || C > 32) return 0;
+    return route_mlp_workspace_bytes(xdt, d, H);
+}
+
+molora_status_t molora_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
+                                 const float* b1, int32_t H, const float* W2, const float* b2, int32_t C, int32_t* r_out,
+                                 float* logits_out, void* ws, size_t ws_bytes, void* stream)
+{
+    if (N < 0 || N >= INT32_MAX || d <= 0 || H < 1 || C < 1) return MOLORA_ERR_INVALID_ARG;
+    if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
+    if ((d % 8) != 0 || (ldx % 8) != 0 || H > 128 || C > 32) return MOLORA_ERR_UNSUPPORTED;
+    if (ldx < d) return MOLORA_ERR_INVALID_ARG;
+    if (W1 == nullptr || W2 == nullptr || (N > 0 && (x == nullptr || r_out == nullptr))) return MOLORA_ERR_INVALID_ARG;
+    if (N > 0 && !aligned16(x)) return MOLORA_ERR_INVALID_ARG;
+    return launch_route_mlp(x, xdt, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, ws_bytes,
+                            static_cast<cudaStream_t>(stream));
+}
+
 size_t molora_group_workspace_bytes(int64_t N, int32_t C) { return group_workspace_bytes(N, C); }
 
 molora_status_t molora_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,

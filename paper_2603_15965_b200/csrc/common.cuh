@@ -176,6 +176,12 @@ size_t route_gate_mma_workspace_bytes(int32_t d, int32_t C);
 molora_status_t launch_route_gate_mma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
                                       const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
                                       cudaStream_t s);
+// The paper's MLP router (Eq. 9).  The tensor-core path (bf16 x, d a multiple of 64, at least 128 tokens) needs
+// route_mlp_workspace_bytes(...) bytes for the split first-layer weights.
+size_t route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H);
+molora_status_t launch_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
+                                 const float* b1, int32_t H, const float* W2, const float* b2, int32_t C, int32_t* r_out,
+                                 float* logits_out, void* ws, size_t ws_bytes, cudaStream_t s);
 size_t group_workspace_bytes(int64_t N, int32_t C);
 molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
                              void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);

@@ -10,7 +10,7 @@ def test_library_builds_loads_and_exports_header_symbols():
     build_library()
     lib = M.load_library()
     names = M.exported_symbols()
-    assert {"molora_route_vocab", "molora_route_composite", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched",
+    assert {"molora_route_vocab", "molora_route_composite", "molora_route_mlp", "molora_route_mlp_workspace_bytes", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched",
             "molora_group_workspace_bytes", "molora_apply_workspace_bytes", "molora_route_gate_workspace_bytes",
             "molora_version",
             "molora_status_string"} <= set(names)
@@ -32,6 +32,13 @@ def test_invalid_arguments_are_refused_before_any_launch():
     # compositional routing: more than 256 composite targets, null adapter indices
     assert lib.molora_route_composite(fake, fake, 4, fake, 4, 65, fake, None, None) == 2
     assert lib.molora_route_composite(fake, None, 4, fake, 4, 64, fake, None, None) == 1
+    # MLP router: hidden width and adapter count limits, tensor-core path without its workspace
+    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, fake, None, 129, fake, None, 4, fake, None, None, 0, None) == 2
+    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, fake, None, 64, fake, None, 33, fake, None, None, 0, None) == 2
+    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, None, None, 64, fake, None, 4, fake, None, None, 0, None) == 1
+    assert M.molora_route_mlp_workspace_bytes(M.BF16, 2560, 128, 4) == 2560 * 3 * 128 * 2
+    assert M.molora_route_mlp_workspace_bytes(M.F32, 2560, 128, 4) == 0
+    assert lib.molora_route_mlp(fake, M.BF16, 128, 64, 64, fake, None, 64, fake, None, 4, fake, None, None, 0, None) == 3
     # gate: d not a multiple of 8, C too large, pitch too small
     assert lib.molora_route_gate(fake, M.BF16, 4, 12, 16, fake, None, 4, fake, None, None, 0, None) == 2
     assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 33, fake, None, None, 0, None) == 2

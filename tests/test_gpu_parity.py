@@ -492,3 +492,50 @@ def test_batched_apply_mixed_ranks_and_paths(N):
         p = w.projections[0]
         ref, _ = oracle.apply(w.inputs["x"], p.y, p.A, p.B, r)
         assert_close(to_f64(y), ref, what=f"mixed batch {p.d_in}->{p.d_out} r{p.rank}")
+
+
+# ------------------------------------------------------------------ the paper's MLP router (Eq. 9)
+@pytest.mark.parametrize("dtype,N,d,H,C", [("bf16", 4096, 2048, 64, 4),      # c2-sized, Eq. 9's hidden width
+                                           ("bf16", 1000, 2560, 128, 4),     # the 2560 -> 128 -> 4 variant, ragged tile
+                                           ("bf16", 300, 512, 48, 9),        # hidden width below the padded 64
+                                           ("bf16", 128, 64, 100, 32),       # one chunk, hidden width below 128
+                                           ("bf16", 50, 2048, 64, 4),        # small call: CUDA-core kernel
+                                           ("bf16", 700, 72, 16, 3),         # d not a multiple of 64
+                                           ("f32", 200, 264, 64, 5)])
+def test_route_mlp_logits_and_argmax(dtype, N, d, H, C):
+    rng = np.random.default_rng(N + d + H + C)
+    x = rng.standard_normal((N, d), dtype=np.float32)
+    if dtype == "bf16":
+        x = W.round_to_bf16(x)
+    W1 = (rng.standard_normal((d, H)) * d ** -0.5).astype(np.float32)
+    b1 = (rng.standard_normal(H) * 0.2).astype(np.float32)
+    W2 = (rng.standard_normal((H, C)) * H ** -0.5).astype(np.float32)
+    b2 = (rng.standard_normal(C) * 0.1).astype(np.float32)
+    r_ref, z_ref, margin = oracle.route_mlp(x, W1, b1, W2, b2)
+    logits = torch.empty(N, C, dtype=torch.float32, device="cuda")
+    r = M.molora_route_mlp(dev_tensor(x, dtype), dev_tensor(W1, "f32"), dev_tensor(b1, "f32"), dev_tensor(W2, "f32"),
+                           dev_tensor(b2, "f32"), logits_out=logits)
+    assert_close(to_f64(logits), z_ref, 1e-4, 1e-4, what="MLP router logits")
+    keep = margin >= 1e-3
+    assert (~keep).sum() <= max(4, N // 100)
+    assert np.array_equal(r.cpu().numpy()[keep], r_ref[keep])
+
+
+def test_route_mlp_feeds_group_and_apply():
+    # route (MLP) -> group -> apply against the oracle on the oracle's routing
+    rng = np.random.default_rng(77)
+    N, d, H, C = 1500, 256, 64, 4
+    w = W.random_problem(78, N, C, d, 192, 16, "bf16")
+    W1 = (rng.standard_normal((d, H)) * d ** -0.5).astype(np.float32)
+    W2 = rng.standard_normal((H, C)).astype(np.float32)
+    r_ref, _, margin = oracle.route_mlp(w.inputs["x"], W1, None, W2, None)
+    x = dev_tensor(w.inputs["x"], "bf16")
+    r = M.molora_route_mlp(x, dev_tensor(W1, "f32"), None, dev_tensor(W2, "f32"), None)
+    keep = margin >= 1e-3
+    assert np.array_equal(r.cpu().numpy()[keep], r_ref[keep])
+    counts, offsets, perm = M.molora_group(r, C)
+    p = w.projections[0]
+    y = dev_tensor(p.y, "bf16")
+    M.molora_apply(x, y, dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), offsets, perm)
+    ref, _ = oracle.apply(w.inputs["x"], p.y, p.A, p.B, r_ref)
+    assert_close(to_f64(y)[keep], ref[keep], what="MLP-routed apply")
