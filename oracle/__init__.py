@@ -41,6 +41,10 @@ def _load():
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_route_vocab.argtypes = [i32p, ctypes.c_int64, i32p, ctypes.c_int32, i32p]
         lib.oracle_route_composite.argtypes = [i32p, i32p, ctypes.c_int64, i32p, ctypes.c_int32, ctypes.c_int32, i32p]
+        lib.oracle_topk_softmax.argtypes = [f64p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, i32p, f64p]
+        lib.oracle_apply_topk.argtypes = [f32p, ctypes.c_int64, f32p, ctypes.c_int64, f32p, f32p, i32p, f64p, ctypes.c_int32,
+                                          ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                          ctypes.c_double, f64p]
         lib.oracle_route_mlp.argtypes = [f32p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, f32p, f32p, ctypes.c_int32, f32p,
                                          f32p, ctypes.c_int32, i32p, f64p, f64p, f64p]
         lib.oracle_route_gate.argtypes = [f32p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, f32p, f32p,
@@ -114,6 +118,37 @@ def route_mlp(x, W1, b1, W2, b2, return_hidden: bool = False):
     if rc:
         raise ValueError("oracle_route_mlp: invalid arguments")
     return (r, z, margin, h) if return_hidden else (r, z, margin)
+
+
+def topk_softmax(z, k: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. 8: the k largest logits of every token (ties: lowest index first) and the softmax over them.
+    Returns (idx int32 [k, N], w fp64 [k, N]), slot 0 = the largest logit."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    N, C = z.shape
+    idx = np.empty((k, N), dtype=np.int32)
+    w = np.empty((k, N), dtype=np.float64)
+    rc = _load().oracle_topk_softmax(_p(z, ctypes.c_double), N, C, int(k), _p(idx, ctypes.c_int32), _p(w, ctypes.c_double))
+    if rc:
+        raise ValueError("oracle_topk_softmax: invalid arguments")
+    return idx, w
+
+
+def apply_topk(x, y, A, B, idx, w, scale: float = 1.0) -> np.ndarray:
+    """Eq. 8: h_i = y_i + scale * sum_j w[j, i] x_i A[idx[j, i]] B[idx[j, i]] in fp64."""
+    x, y, A, B = _f32(x), _f32(y), _f32(A), _f32(B)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    k, N = idx.shape
+    C, d_in, rank = A.shape
+    d_out = B.shape[2]
+    assert x.shape == (N, d_in) and y.shape == (N, d_out) and B.shape == (C, rank, d_out) and w.shape == (k, N)
+    h = np.empty((N, d_out), dtype=np.float64)
+    rc = _load().oracle_apply_topk(_p(x, ctypes.c_float), d_in, _p(y, ctypes.c_float), d_out, _p(A, ctypes.c_float),
+                                   _p(B, ctypes.c_float), _p(idx, ctypes.c_int32), _p(w, ctypes.c_double), k, N, d_in,
+                                   d_out, rank, C, float(scale), _p(h, ctypes.c_double))
+    if rc:
+        raise ValueError("oracle_apply_topk: invalid arguments")
+    return h
 
 
 def route_gate(x, G, bias=None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:

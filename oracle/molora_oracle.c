@@ -199,6 +199,58 @@ int oracle_apply(const float *x, int64_t ldx, const float *y, int64_t ldy, const
     return 0;
 }
 
+/* Top-k weighted routing (Eq. 8): from the logits z_i the k largest are kept (ties: lowest index first), and
+ * w_i = softmax over the kept logits.  idx and w are slot-major: idx[j * N + i] is the j-th choice of token i
+ * (j = 0 the largest logit).  k <= C. */
+int oracle_topk_softmax(const double *z, int64_t N, int32_t C, int32_t k, int32_t *idx, double *w)
+{
+    if (N < 0 || C <= 0 || k <= 0 || k > C) return 1;
+    for (int64_t i = 0; i < N; ++i) {
+        const double *zi = z + i * (int64_t)C;
+        for (int32_t j = 0; j < k; ++j) {
+            int32_t best = -1;
+            for (int32_t c = 0; c < C; ++c) {
+                int taken = 0;
+                for (int32_t q = 0; q < j; ++q) taken |= idx[(int64_t)q * N + i] == c;
+                if (taken) continue;
+                if (best < 0 || zi[c] > zi[best]) best = c;
+            }
+            idx[(int64_t)j * N + i] = best;
+        }
+        const double zmax = zi[idx[i]];
+        double den = 0.0;
+        for (int32_t j = 0; j < k; ++j) den += exp(zi[idx[(int64_t)j * N + i]] - zmax);
+        for (int32_t j = 0; j < k; ++j) w[(int64_t)j * N + i] = exp(zi[idx[(int64_t)j * N + i]] - zmax) / den;
+    }
+    return 0;
+}
+
+/* Eq. 8, second half: h_i = y_i + scale * sum_j w_ij x_i A^(r_ij) B^(r_ij) over the k kept adapters of token i
+ * (slot-major idx, w as above; an index outside [0, C) contributes nothing). */
+int oracle_apply_topk(const float *x, int64_t ldx, const float *y, int64_t ldy, const float *A, const float *B,
+                      const int32_t *idx, const double *w, int32_t k, int64_t N, int32_t d_in, int32_t d_out,
+                      int32_t rank, int32_t C, double scale, double *h)
+{
+    if (N < 0 || d_in <= 0 || d_out <= 0 || rank <= 0 || C <= 0 || k <= 0 || ldx < d_in || ldy < d_out) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < N; ++i) {
+        double *hi = h + i * (int64_t)d_out;
+        for (int32_t o = 0; o < d_out; ++o) hi[o] = (double)y[i * ldy + o];
+        for (int32_t j = 0; j < k; ++j) {
+            const int32_t c = idx[(int64_t)j * N + i];
+            if (c < 0 || c >= C) continue;
+            const float *Ac = A + (int64_t)c * d_in * rank, *Bc = B + (int64_t)c * rank * d_out;
+            for (int32_t q = 0; q < rank; ++q) {
+                double t = 0.0;
+                for (int32_t kk = 0; kk < d_in; ++kk) t += (double)x[i * ldx + kk] * (double)Ac[(int64_t)kk * rank + q];
+                t *= scale * w[(int64_t)j * N + i];
+                for (int32_t o = 0; o < d_out; ++o) hi[o] += t * (double)Bc[(int64_t)q * d_out + o];
+            }
+        }
+    }
+    return 0;
+}
+
 /* Per-sequence routing served as K passes (Eq. 1 applied once per adapter, Theorem 3.6): pass k runs
  * the dense single-adapter LoRA of adapter k over ALL N tokens, then only rows with r[i] == k are kept.
  * Work is K*N token-adapter products.  The result must equal oracle_apply() bit for bit. */

@@ -28,6 +28,47 @@ def _small(seed, N=37, C=3, d_in=24, d_out=40, rank=4, dtype="f32", **kw):
     return W.random_problem(seed, N, C, d_in, d_out, rank, dtype, **kw)
 
 
+# ------------------------------------------------------------------ top-k weighted routing (Eq. 8)
+def test_topk_softmax_and_weighted_apply_pins():
+    rng = np.random.default_rng(21)
+    N, C, d_in, d_out, rank = 40, 5, 12, 9, 3
+    z = rng.standard_normal((N, C))
+    # k = 1: the argmax with weight exactly 1 (the case the hot path serves)
+    i1, w1 = oracle.topk_softmax(z, 1)
+    assert np.array_equal(i1[0], np.argmax(z, axis=1)) and np.all(w1 == 1.0)
+    # k = 2: the two largest in order, weights in closed form: w_top = sigmoid(z_top - z_second), sum 1
+    i2, w2 = oracle.topk_softmax(z, 2)
+    order = np.argsort(-z, axis=1, kind="stable")
+    assert np.array_equal(i2[0], order[:, 0]) and np.array_equal(i2[1], order[:, 1])
+    gap = z[np.arange(N), i2[0]] - z[np.arange(N), i2[1]]
+    assert np.allclose(w2[0], 1.0 / (1.0 + np.exp(-gap)), rtol=1e-13) and np.allclose(w2.sum(axis=0), 1.0, rtol=1e-13)
+    # k = C: the full softmax (library routine), permuted into descending order
+    from scipy.special import softmax
+    i5, w5 = oracle.topk_softmax(z, C)
+    assert np.allclose(w5.T, np.take_along_axis(softmax(z, axis=1), i5.T.astype(np.int64), axis=1), rtol=1e-12)
+    # ties: equal logits are taken lowest index first
+    it, wt = oracle.topk_softmax(np.array([[1.0, 3.0, 3.0, 0.0]]), 2)
+    assert it[:, 0].tolist() == [1, 2] and np.allclose(wt[:, 0], [0.5, 0.5])
+    # weighted apply: against library matmul per token; k = 1 with weight 1 equals the per-token apply of Eq. 2
+    x = rng.standard_normal((N, d_in)).astype(np.float32)
+    y = rng.standard_normal((N, d_out)).astype(np.float32)
+    A = rng.standard_normal((C, d_in, rank)).astype(np.float32)
+    B = rng.standard_normal((C, rank, d_out)).astype(np.float32)
+    h = oracle.apply_topk(x, y, A, B, i2, w2, scale=0.5)
+    ref = y.astype(np.float64).copy()
+    for i in range(N):
+        for j in range(2):
+            c = i2[j, i]
+            ref[i] += 0.5 * w2[j, i] * (x[i].astype(np.float64) @ A[c].astype(np.float64) @ B[c].astype(np.float64))
+    assert np.allclose(h, ref, rtol=1e-12, atol=1e-12)
+    h1 = oracle.apply_topk(x, y, A, B, i1, w1)
+    ref1, _ = oracle.apply(x, y, A, B, i1[0])
+    assert np.allclose(h1, ref1, rtol=1e-13, atol=1e-13)
+    # swapping the two slots (with their weights) changes nothing: the sum over the kept set is order-free up to rounding
+    hs = oracle.apply_topk(x, y, A, B, i2[::-1], w2[::-1], scale=0.5)
+    assert np.allclose(hs, h, rtol=1e-12, atol=1e-12)
+
+
 # ------------------------------------------------------------------ the paper's router (Eq. 9): 2-layer MLP, GELU
 def test_mlp_router_pins():
     from scipy.stats import norm
