@@ -202,10 +202,31 @@ typedef struct {
     const void *B;
     int32_t d_in, d_out, rank;
     float scale;
+    const float *row_scale; /* device fp32[N] or NULL: extra factor per TOKEN on its delta (the routing weight w_ij of
+                               top-k routing, Eq. 8); NULL means 1 */
 } molora_proj_desc_t;
 molora_status_t molora_apply_batched(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N,
                                      int32_t C, const int32_t *offsets, const int32_t *perm, void *ws, size_t ws_bytes,
                                      uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Top-k weighted routing (Eq. 8): w_i = softmax(TopK(z_i, k)), delta h_i = sum_j w_ij x_i A^(j) B^(j).
+ * molora_topk_softmax turns router logits (logits_out of molora_route_gate / molora_route_mlp) into the k kept
+ * adapters per token and their weights:
+ *   logits   device fp32 [N, C], 1 <= k <= C <= 32
+ *   idx_out  device int32 [k, N] slot-major: idx_out[j*N + i] = the j-th choice of token i (j = 0: largest logit;
+ *            equal logits: lowest index first);  w_out  device fp32 [k, N], softmax over the k kept logits
+ * molora_apply_topk applies the k choices as k passes of (group, apply) with the weights as per-token factors: within
+ * a pass every row of y is touched by one adapter only, so there are no conflicting updates and the result is
+ * deterministic; y is rounded to its storage type once per pass.
+ *   projs    HOST array of P descriptors as for molora_apply_batched (their row_scale is ignored)
+ *   ws       device scratch of at least molora_apply_topk_workspace_bytes(projs, P, N, C) bytes, 256-byte aligned */
+molora_status_t molora_topk_softmax(const float *logits, int64_t N, int32_t C, int32_t k, int32_t *idx_out, float *w_out,
+                                    void *stream);
+size_t molora_apply_topk_workspace_bytes(const molora_proj_desc_t *projs, int32_t P, int64_t N, int32_t C);
+molora_status_t molora_apply_topk(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C,
+                                  int32_t k, const int32_t *idx, const float *w, void *ws, size_t ws_bytes,
+                                  uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Failure-detection self-test.  Every device-side wait of the tensor-core apply kernel (on an mbarrier that a

@@ -40,7 +40,7 @@ class _HostProjC(ctypes.Structure):
 class _ProjDescC(ctypes.Structure):
     _fields_ = [("x", ctypes.c_void_p), ("ldx", ctypes.c_int64), ("y", ctypes.c_void_p), ("ldy", ctypes.c_int64),
                 ("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32),
-                ("rank", ctypes.c_int32), ("scale", ctypes.c_float)]
+                ("rank", ctypes.c_int32), ("scale", ctypes.c_float), ("row_scale", ctypes.c_void_p)]
 
 
 def lib_path() -> str:
@@ -70,6 +70,10 @@ def load_library():
     lib.molora_status_string.argtypes = [ctypes.c_int]
     lib.molora_route_vocab.argtypes = [vp, i64, vp, i32, vp, vp, vp]
     lib.molora_route_composite.argtypes = [vp, vp, i64, vp, i32, i32, vp, vp, vp]
+    lib.molora_topk_softmax.argtypes = [vp, i64, i32, i32, vp, vp, vp]
+    lib.molora_apply_topk_workspace_bytes.restype = sz
+    lib.molora_apply_topk_workspace_bytes.argtypes = [vp, i32, i64, i32]
+    lib.molora_apply_topk.argtypes = [vp, i32, ctypes.c_int, i64, i32, i32, vp, vp, vp, sz, vp, vp]
     lib.molora_route_mlp_workspace_bytes.restype = sz
     lib.molora_route_mlp_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i32]
     lib.molora_route_mlp.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
@@ -329,6 +333,7 @@ class ProjDesc:
     A: torch.Tensor
     B: torch.Tensor
     scale: float = 1.0
+    row_scale: Optional[torch.Tensor] = None     # fp32 [N]: extra per-token factor on the delta (top-k routing weights)
 
 
 def pack_proj_descs(projs: Sequence[ProjDesc]):
@@ -348,8 +353,11 @@ def pack_proj_descs(projs: Sequence[ProjDesc]):
             N, C, dt = n, c, _dtype_code(p.x)
         elif (N, C, dt) != (n, c, _dtype_code(p.x)):
             raise ValueError("all projections of a batched apply share N, C and the element type")
+        rs = getattr(p, "row_scale", None)
+        if rs is not None and (rs.dtype != torch.float32 or rs.numel() != n or not rs.is_contiguous()):
+            raise ValueError("row_scale must be a dense fp32 tensor with one factor per token")
         arr[i] = _ProjDescC(p.x.data_ptr(), ldx, p.y.data_ptr(), ldy, p.A.data_ptr(), p.B.data_ptr(), d_in, d_out,
-                            rank, float(p.scale))
+                            rank, float(p.scale), rs.data_ptr() if rs is not None else None)
     return arr, N, C, dt
 
 
@@ -370,6 +378,36 @@ def molora_apply_batched(projs, offsets: torch.Tensor, perm: torch.Tensor, ws: O
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_apply_batched", lib.molora_apply_batched(arr, len(arr), dt, N, C, _ptr(offsets), _ptr(perm),
                                                             _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
+
+
+def molora_topk_softmax(logits: torch.Tensor, k: int, stream=None):
+    """Eq. 8: the k largest logits per token (ties: lowest index first) and the softmax over them.
+    Returns (idx int32 [k, N], w fp32 [k, N]), slot 0 = the largest logit."""
+    lib = load_library()
+    if logits.dtype != torch.float32 or logits.dim() != 2 or not logits.is_contiguous():
+        raise ValueError("logits must be a dense fp32 [N, C] tensor")
+    N, C = logits.shape
+    idx = torch.empty(k, N, dtype=torch.int32, device=logits.device)
+    w = torch.empty(k, N, dtype=torch.float32, device=logits.device)
+    _check("molora_topk_softmax", lib.molora_topk_softmax(_ptr(logits), N, C, int(k), _ptr(idx), _ptr(w), _stream(stream)))
+    return idx, w
+
+
+def molora_apply_topk(projs, idx: torch.Tensor, w: torch.Tensor, C: int, ws: Optional[torch.Tensor] = None,
+                      dev_status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Eq. 8: y_i += sum_j w[j, i] * scale * (x_i A[idx[j, i]]) B[idx[j, i]] as k passes of (group, apply)."""
+    lib = load_library()
+    arr, N, C_, dt = pack_proj_descs(projs)
+    if C_ != C or idx.dtype != torch.int32 or w.dtype != torch.float32 or tuple(idx.shape) != tuple(w.shape) or idx.shape[1] != N:
+        raise ValueError("idx int32 [k, N] and w fp32 [k, N] must match the projections")
+    k = idx.shape[0]
+    need = int(lib.molora_apply_topk_workspace_bytes(arr, len(arr), N, C))
+    if ws is None:
+        ws = torch.empty(need + 256, dtype=torch.uint8, device=idx.device)
+    off = (-ws.data_ptr()) % 256
+    _check("molora_apply_topk", lib.molora_apply_topk(arr, len(arr), dt, N, C, k, _ptr(idx.contiguous()), _ptr(w.contiguous()),
+                                                      ctypes.c_void_p(ws.data_ptr() + off), ws.numel() - off,
+                                                      _ptr(dev_status), _stream(stream)))
 
 
 ROUTE_VOCAB, ROUTE_GATE, ROUTE_GIVEN = 0, 1, 2

@@ -210,7 +210,71 @@ molora_status_t molora_apply(const void* x, int64_t ldx, void* y, int64_t ldy, m
     p.d_out = d_out;
     p.rank = rank;
     p.scale = scale;
+    p.row_scale = nullptr;
     return molora_apply_batched(&p, 1, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, stream);
+}
+
+molora_status_t molora_topk_softmax(const float* logits, int64_t N, int32_t C, int32_t k, int32_t* idx_out, float* w_out,
+                                    void* stream)
+{
+    if (N < 0 || N >= INT32_MAX || C < 1 || k < 1 || k > C) return MOLORA_ERR_INVALID_ARG;
+    if (C > 32) return MOLORA_ERR_UNSUPPORTED;
+    if (N > 0 && (logits == nullptr || idx_out == nullptr || w_out == nullptr)) return MOLORA_ERR_INVALID_ARG;
+    return launch_topk_softmax(logits, N, C, k, idx_out, w_out, static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+struct TopkPlan {
+    size_t counts, offsets, perm, apply_ws, apply_ws_bytes, total;
+};
+TopkPlan plan_topk(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C)
+{
+    auto a256 = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    TopkPlan pl;
+    size_t off = 0;
+    pl.counts = off;   off = a256(off + sizeof(int32_t) * (size_t)C);
+    pl.offsets = off;  off = a256(off + sizeof(int32_t) * (size_t)(C + 1));
+    pl.perm = off;     off = a256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
+    pl.apply_ws = off;
+    pl.apply_ws_bytes = 0;
+    for (int i = 0; i < P; ++i)
+        pl.apply_ws_bytes += molora_apply_workspace_bytes(N, C, projs[i].d_in, projs[i].d_out, projs[i].rank);
+    pl.total = a256(off + pl.apply_ws_bytes);
+    return pl;
+}
+}  // namespace
+
+size_t molora_apply_topk_workspace_bytes(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C)
+{
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 0 || C < 1) return 0;
+    return plan_topk(projs, P, N, C).total;
+}
+
+molora_status_t molora_apply_topk(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C,
+                                  int32_t k, const int32_t* idx, const float* w, void* ws, size_t ws_bytes,
+                                  uint32_t* dev_status, void* stream)
+{
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 0 || C < 1 || k < 1 || k > C) return MOLORA_ERR_INVALID_ARG;
+    if (N > 0 && (idx == nullptr || w == nullptr)) return MOLORA_ERR_INVALID_ARG;
+    const TopkPlan pl = plan_topk(projs, P, N, C);
+    if (ws == nullptr || ws_bytes < pl.total || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return MOLORA_ERR_WORKSPACE;
+    char* base = static_cast<char*>(ws);
+    int32_t* counts = reinterpret_cast<int32_t*>(base + pl.counts);
+    int32_t* offsets = reinterpret_cast<int32_t*>(base + pl.offsets);
+    int32_t* perm = reinterpret_cast<int32_t*>(base + pl.perm);
+    molora_proj_desc_t pass[MOLORA_MAX_PROJECTIONS];
+    for (int32_t j = 0; j < k; ++j) {               // one (group, apply) pass per kept adapter slot
+        molora_status_t st = molora_group(idx + (int64_t)j * N, N, C, counts, offsets, perm, nullptr, 0, dev_status, stream);
+        if (st != MOLORA_OK) return st;
+        for (int i = 0; i < P; ++i) {
+            pass[i] = projs[i];
+            pass[i].row_scale = w + (int64_t)j * N;
+        }
+        st = molora_apply_batched(pass, P, dt, N, C, offsets, perm, pl.apply_ws_bytes > 0 ? base + pl.apply_ws : nullptr,
+                                  pl.apply_ws_bytes, dev_status, stream);
+        if (st != MOLORA_OK) return st;
+    }
+    return MOLORA_OK;
 }
 
 molora_status_t molora_selftest_bounded_wait(uint32_t* dev_status, int64_t limit_cycles, int32_t* result, void* stream)
@@ -305,6 +369,7 @@ molora_status_t molora_forward_host(molora_router_t router, const int32_t* route
         dev[i].d_out = projs[i].d_out;
         dev[i].rank = projs[i].rank;
         dev[i].scale = projs[i].scale;
+        dev[i].row_scale = nullptr;
         const molora_status_t st = check_proj(dev[i], dt);
         if (st != MOLORA_OK) return st;
     }

@@ -95,7 +95,9 @@ __global__ void __launch_bounds__(kRowTileThreads, 1) apply_rowtile_kernel(const
         float s = 0.f;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) s += partial[w][tid];
-        t_s[tid] = s * pd.scale;               // fold the LoRA scale into t once
+        // fold the LoRA scale (and the token's routing weight, if given) into t once: t_s is [TM][R], row m = tid / R
+        const float rs = pd.row_scale != nullptr ? __ldg(pd.row_scale + row_s[tid / R]) : 1.f;
+        t_s[tid] = s * pd.scale * rs;
     }
     __syncthreads();
 

@@ -353,6 +353,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
         {
             const int KS = prm.ks[proj];
             const float scale = prm.p[proj].scale;
+            const float* rscale = prm.p[proj].row_scale;
             const float* part = prm.tws + prm.t_off[proj] + (int64_t)t.row0 * R;
             const int64_t slice_stride = (int64_t)prm.N * R;
             for (int e4 = tid; e4 < Cfg::TFLOATS / 4; e4 += kTpThreads) {
@@ -366,7 +367,9 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
                         s.w += v.w;
                     }
                 }
-                *reinterpret_cast<float4*>(&tfin[e4 * 4]) = make_float4(s.x * scale, s.y * scale, s.z * scale, s.w * scale);
+                float sc = scale;                   // times the token's routing weight, if the caller passes per-token factors
+                if (rscale != nullptr && e4 * 4 < t.rows * R) sc *= __ldg(rscale + tp_token(prm, perm_s, t.row0 + e4 * 4 / R));
+                *reinterpret_cast<float4*>(&tfin[e4 * 4]) = make_float4(s.x * sc, s.y * sc, s.z * sc, s.w * sc);
             }
         }
         wait_bar(bar, parity, &abort_s, prm.dev_status);

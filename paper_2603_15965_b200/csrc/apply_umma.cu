@@ -67,6 +67,7 @@ struct UmmaProj {
     int64_t ldx, ldy;
     int32_t d_in, d_out, rank;
     float scale;
+    const float* row_scale;  // per-token factor on the delta (top-k routing weights) or NULL
     int32_t wide_store;     // y rows are 32-byte aligned: the copy-out uses 256-bit stores
 };
 struct UmmaParams {
@@ -354,6 +355,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 #pragma unroll
             for (int c = 0; c < R / 16; ++c) tmem_ld_x16(tmem_T + lane_addr + c * 16, tv + c * 16);
             tmem_wait_ld();
+            // LoRA scale times the token's routing weight (1 unless the caller passes per-token factors)
+            const int my_tok = ctrl->rows[row];
+            const float tscale = pj.scale * ((pj.row_scale != nullptr && my_tok >= 0) ? __ldg(pj.row_scale + my_tok) : 1.f);
             bool t_published = false;
             if (Cfg::kOnePush && S > 1) {
                 // Exchange of the partial T tiles in one push through distributed shared memory: every CTA writes its
@@ -462,7 +466,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                         float hi[8], lo[8];
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
-                            const float t = __uint_as_float(tv[c8 * 8 + e]) * pj.scale;
+                            const float t = __uint_as_float(tv[c8 * 8 + e]) * tscale;
                             hi[e] = __bfloat162float(__float2bfloat16_rn(t));
                             lo[e] = t - hi[e];
                         }
@@ -487,7 +491,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                     float hi[8], lo[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        const float t = __uint_as_float(tv[c8 * 8 + e]) * pj.scale;
+                        const float t = __uint_as_float(tv[c8 * 8 + e]) * tscale;
                         hi[e] = __bfloat162float(__float2bfloat16_rn(t));
                         lo[e] = t - hi[e];
                     }
@@ -770,6 +774,7 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
         u.d_out = d.d_out;
         u.rank = d.rank;
         u.scale = d.scale;
+        u.row_scale = d.row_scale;
         u.wide_store = ((reinterpret_cast<uintptr_t>(d.y) & 31u) == 0 && ((d.ldy * 2) % 32) == 0) ? 1 : 0;
         has[d.rank == 16 ? 0 : d.rank == 32 ? 1 : 2] = true;
     }

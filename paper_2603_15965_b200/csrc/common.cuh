@@ -182,6 +182,9 @@ size_t route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H);
 molora_status_t launch_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
                                  const float* b1, int32_t H, const float* W2, const float* b2, int32_t C, int32_t* r_out,
                                  float* logits_out, void* ws, size_t ws_bytes, cudaStream_t s);
+// Top-k selection and softmax over router logits (Eq. 8); idx / w slot-major [k][N].
+molora_status_t launch_topk_softmax(const float* logits, int64_t N, int32_t C, int32_t k, int32_t* idx_out, float* w_out,
+                                    cudaStream_t s);
 size_t group_workspace_bytes(int64_t N, int32_t C);
 molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
                              void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);

@@ -467,6 +467,57 @@ static molora_status_t gate_dispatch(const void* x, int64_t N, int d, int64_t ld
     return gate_launch<T, 32, 2>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);   // C <= 32 checked by the caller
 }
 
+// ------------------------------------------------------------------------------------------------
+// Top-k weighted routing (Eq. 8): per token the k largest logits (equal logits: lowest index first) and the softmax
+// over the kept ones.  One thread per token, C <= 32 logits in registers; k passes of a masked argmax.
+__global__ void __launch_bounds__(256) topk_softmax_kernel(const float* __restrict__ logits, int64_t N, int C, int k,
+                                                           int32_t* __restrict__ idx_out, float* __restrict__ w_out)
+{
+    ptx::grid_dependency_sync();
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    float z[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) z[c] = c < C ? __ldg(logits + i * C + c) : 0.f;
+    uint32_t taken = 0;
+    float zmax = 0.f, den = 0.f;
+    float kept[32];
+    for (int j = 0; j < k; ++j) {
+        int best = -1;
+        float bz = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            if (c < C && !((taken >> c) & 1u) && (best < 0 || z[c] > bz)) {
+                best = c;
+                bz = z[c];
+            }
+        }
+        taken |= 1u << best;
+        idx_out[(int64_t)j * N + i] = best;
+        if (j == 0) zmax = bz;
+        const float e = expf(bz - zmax);
+#pragma unroll
+        for (int q = 0; q < 32; ++q)
+            if (q == j) kept[q] = e;
+        den += e;
+    }
+    for (int j = 0; j < k; ++j) {
+        float e = 0.f;
+#pragma unroll
+        for (int q = 0; q < 32; ++q)
+            if (q == j) e = kept[q];
+        w_out[(int64_t)j * N + i] = e / den;
+    }
+}
+
+molora_status_t launch_topk_softmax(const float* logits, int64_t N, int32_t C, int32_t k, int32_t* idx_out, float* w_out,
+                                    cudaStream_t s)
+{
+    if (N == 0) return MOLORA_OK;
+    return cuda_ok(launch_kernel(topk_softmax_kernel, dim3((unsigned)ceil_div64(N, 256)), dim3(256), 0, s, 1, false, logits, N,
+                                 (int)C, (int)k, idx_out, w_out));
+}
+
 size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
 {
     if (xdt != MOLORA_BF16) return 0;

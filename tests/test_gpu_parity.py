@@ -539,3 +539,43 @@ def test_route_mlp_feeds_group_and_apply():
     M.molora_apply(x, y, dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), offsets, perm)
     ref, _ = oracle.apply(w.inputs["x"], p.y, p.A, p.B, r_ref)
     assert_close(to_f64(y)[keep], ref[keep], what="MLP-routed apply")
+
+
+# ------------------------------------------------------------------ top-k weighted routing (Eq. 8, the paper's k = 2)
+@pytest.mark.parametrize("N,C,k,d_in,d_out,rank", [(300, 4, 2, 256, 192, 16),     # small-tile path
+                                                   (3300, 4, 2, 512, 256, 16),    # tensor-core path
+                                                   (200, 6, 3, 128, 96, 8),       # CUDA-core path (rank 8)
+                                                   (500, 5, 1, 64, 64, 32)])      # k = 1: weight exactly 1
+def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank):
+    rng = np.random.default_rng(N + C + k)
+    w_ = W.random_problem(500 + N, N, C, d_in, d_out, rank, "bf16")
+    p = w_.projections[0]
+    x_np = w_.inputs["x"]
+    G = (rng.standard_normal((d_in, C)) * d_in ** -0.5).astype(np.float32)
+    # router logits on the GPU, then top-k + softmax on the GPU; oracle side from its own logits
+    logits = torch.empty(N, C, dtype=torch.float32, device="cuda")
+    x = dev_tensor(x_np, "bf16")
+    M.molora_route_gate(x, dev_tensor(G, "f32"), logits_out=logits)
+    idx, wt = M.molora_topk_softmax(logits, k)
+    _, z_ref, _ = oracle.route_gate(x_np, G)
+    idx_ref, w_ref = oracle.topk_softmax(z_ref, k)
+    srt = np.sort(z_ref, axis=1)[:, ::-1]
+    gaps = srt[:, :k] - srt[:, 1:k + 1] if k < C else srt[:, :k - 1] - srt[:, 1:k]
+    keep = np.all(gaps >= 1e-3, axis=1)                       # tokens whose kept set and order are unambiguous
+    assert (~keep).sum() <= max(6, N // 50)
+    assert np.array_equal(idx.cpu().numpy()[:, keep], idx_ref[:, keep])
+    assert np.allclose(wt.cpu().numpy()[:, keep], w_ref[:, keep], rtol=1e-4, atol=1e-5)
+    assert np.allclose(wt.cpu().numpy().sum(axis=0), 1.0, atol=1e-5)
+    # weighted apply in k passes against the oracle's weighted sum
+    y = dev_tensor(p.y, "bf16")
+    M.molora_apply_topk([M.ProjDesc(x, y, dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), 1.0)], idx, wt, C)
+    ref = oracle.apply_topk(x_np, p.y, p.A, p.B, idx_ref, w_ref)
+    # y is rounded to bf16 after every pass: besides the usual bound, half a bf16 ulp (2^-9 relative) of each
+    # intermediate result h after passes 1 .. k-1 (which can be much larger than the final value when slots cancel)
+    got, err = to_f64(y), None
+    slack = np.zeros_like(ref)
+    for j in range(1, k):
+        slack += 2.0 ** -9 * np.abs(oracle.apply_topk(x_np, p.y, p.A, p.B, idx_ref[:j], w_ref[:j]))
+    err = np.abs(got - ref)
+    bound = 1e-3 + 2e-2 * np.abs(ref) + slack
+    assert np.all(err[keep] <= bound[keep]), f"top-{k} weighted apply: worst ratio {(err / bound)[keep].max():.3f}"
