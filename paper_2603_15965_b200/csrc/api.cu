@@ -21,15 +21,42 @@ bool chained_launch_enabled()
 
 namespace {
 
-// Calls with fewer tokens than this run on the two-launch small-tile path (tuning override for every rank:
-// MOLORA_UMMA_MIN_TOKENS).
-int64_t umma_min_tokens(int32_t rank)
+// ---- path selection (bf16, ranks 16 / 32 / 64; everything else runs on the CUDA-core row-tile kernel)
+// Three kernels cover the bf16 calls: the tcgen05 kernel (128-row tiles, clusters), the single-launch streaming
+// kernel (32-row tiles, one CTA per item) and the two-launch small-tile kernels.  Measured on B200 (2048- and
+// 4096-wide projections, 4-128 adapters, 1-7 projections per call):
+//   rank 16  streaming wins until the projections of the call move ~150 MB (x once, y twice), tcgen05 above;
+//   rank 32  two-launch below 1024 tokens (a tie with streaming), streaming until ~60 MB, tcgen05 above;
+//   rank 64  two-launch below 1280 tokens, tcgen05 above (the streaming kernel has only two stages there).
+// MOLORA_UMMA_MIN_TOKENS=n forces "tcgen05 from n tokens" and MOLORA_SMALL_PATH=stream|twophase forces the kernel used
+// below it, for measurements and for tests that target one kernel.
+int64_t forced_umma_min_tokens()
 {
-    static const int64_t forced = [] {
-        const char* e = std::getenv("MOLORA_UMMA_MIN_TOKENS");
-        return e != nullptr ? std::max<int64_t>(1, std::atoll(e)) : (int64_t)0;
-    }();
-    return forced > 0 ? forced : umma_min_tokens_for_rank(rank);
+    const char* e = std::getenv("MOLORA_UMMA_MIN_TOKENS");   // read per call: tests switch it
+    return e != nullptr && e[0] != '\0' ? std::max<int64_t>(1, std::atoll(e)) : (int64_t)0;
+}
+constexpr double kUmmaMinBytesR16 = 150e6, kUmmaMinBytesR32 = 60e6;
+constexpr int64_t kUmmaMinTokensR64 = 1280, kStreamMinTokensR32 = 1024;
+
+double proj_bytes(int64_t N, int32_t d_in, int32_t d_out) { return (double)N * ((double)d_in + 2.0 * d_out) * 2.0; }
+
+// group_bytes: bytes moved by all projections of this rank in the call
+bool use_umma(int32_t rank, int64_t N, double group_bytes)
+{
+    if (const int64_t forced = forced_umma_min_tokens()) return N >= forced;
+    if (N < kUmmaMinTokens) return false;
+    if (rank == 16) return group_bytes >= kUmmaMinBytesR16;
+    if (rank == 32) return group_bytes >= kUmmaMinBytesR32;
+    return N >= kUmmaMinTokensR64;
+}
+// the kernel for what the tcgen05 kernel does not take
+bool small_path_is_stream(int32_t rank, int64_t N)
+{
+    if (const char* e = std::getenv("MOLORA_SMALL_PATH")) {
+        if (e[0] == 's') return true;
+        if (e[0] == 't') return false;
+    }
+    return rank == 16 || (rank == 32 && N >= kStreamMinTokensR32);
 }
 
 bool rank_supported(int r) { return r == 8 || r == 16 || r == 32 || r == 64; }
@@ -140,12 +167,16 @@ molora_status_t molora_group(const int32_t* r, int64_t N, int32_t C, int32_t* co
 
 size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t d_out, int32_t rank)
 {
-    // Only the two-launch small-tile path needs scratch (its partial shrink results).  It serves calls below
-    // kUmmaMinTokens tokens and, with more than kUmmaAllSegmentsMaxC adapters, the short segments of larger calls;
-    // the element type is not known here, so the figure assumes bf16 (fp32 calls need none).
+    // Only the two-launch small-tile kernels need scratch (their partial shrink results); see the path selection at
+    // the top of this file.  The element type is not known here, so the figure assumes bf16 (fp32 calls need none).
     if (N <= 0 || d_in <= 0 || d_out <= 0 || (rank != 16 && rank != 32 && rank != 64)) return 0;
     if ((d_in % 32) != 0 || (d_out % 32) != 0) return 0;
-    if (N >= umma_min_tokens(rank) && C <= kUmmaAllSegmentsMaxC && (d_in % 64) == 0 && (d_out % 64) == 0) return 0;
+    if (small_path_is_stream(rank, N)) return 0;
+    // two-launch kernels: needed unless the tcgen05 kernel is certain to take every segment (for ranks 16 and 32 that
+    // depends on the other projections of the call, which are not known here)
+    const int64_t forced = forced_umma_min_tokens();
+    const bool umma_certain = forced > 0 ? N >= forced : (rank == 64 && N >= kUmmaMinTokensR64);
+    if (umma_certain && C <= kUmmaAllSegmentsMaxC && (d_in % 64) == 0 && (d_out % 64) == 0) return 0;
     return decode_workspace_bytes(N, d_in, rank);
 }
 
@@ -163,32 +194,44 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
         if (st != MOLORA_OK) return st;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // Split the projections by eligibility for the tensor-core kernel.  For eligible ones both kernels are
-    // enqueued and each segment is taken by exactly one of them, chosen on the device from its row count.
-    molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], dc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
-    int n_tc = 0, n_dc = 0, n_cc = 0;
+    // Split the projections by kernel.  For projections of the tcgen05 kernel with many adapters both it and a
+    // small-tile kernel are enqueued and each segment is taken by exactly one of them, chosen on the device from
+    // its row count.
+    double group_bytes[3] = {0.0, 0.0, 0.0};       // ranks 16, 32, 64
+    auto group_of = [](int32_t rank) { return rank == 16 ? 0 : rank == 32 ? 1 : 2; };
+    for (int i = 0; i < P; ++i)
+        if (umma_eligible(projs[i], dt)) group_bytes[group_of(projs[i].rank)] += proj_bytes(N, projs[i].d_in, projs[i].d_out);
+    molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], sc[MOLORA_MAX_PROJECTIONS], dc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
+    int n_tc = 0, n_sc = 0, n_dc = 0, n_cc = 0;
     for (int i = 0; i < P; ++i) {
-        if (N >= umma_min_tokens(projs[i].rank) && umma_eligible(projs[i], dt)) tc[n_tc++] = projs[i];
-        else if (decode_eligible(projs[i], dt)) dc[n_dc++] = projs[i];
-        else cc[n_cc++] = projs[i];
+        const int32_t rank = projs[i].rank;
+        if (umma_eligible(projs[i], dt) && use_umma(rank, N, group_bytes[group_of(rank)])) tc[n_tc++] = projs[i];
+        else if (decode_eligible(projs[i], dt)) {
+            if (small_path_is_stream(rank, N)) sc[n_sc++] = projs[i];
+            else dc[n_dc++] = projs[i];
+        } else cc[n_cc++] = projs[i];
     }
     molora_status_t st = MOLORA_OK;
     if (n_tc > 0) {
         // With few adapters an under-filled 128-row tile is cheap, so the tensor-core kernel takes every segment
         // and the second launch is saved; with many adapters (up to 256 composite targets) tiny segments are
-        // the norm and go to the small-tile kernel instead.
+        // the norm and go to a small-tile kernel instead.
         const int32_t min_rows = C <= kUmmaAllSegmentsMaxC ? 1 : kUmmaMinRows;
         st = launch_apply_umma(tc, n_tc, N, C, offsets, perm, dev_status, min_rows, s);
         if (st == MOLORA_OK && min_rows > 1) {
-            molora_proj_desc_t small_dc[MOLORA_MAX_PROJECTIONS], small_cc[MOLORA_MAX_PROJECTIONS];
-            int a = 0, b = 0;
+            molora_proj_desc_t small_sc[MOLORA_MAX_PROJECTIONS], small_dc[MOLORA_MAX_PROJECTIONS], small_cc[MOLORA_MAX_PROJECTIONS];
+            int a = 0, b = 0, c = 0;
             for (int i = 0; i < n_tc; ++i) {
-                if (decode_eligible(tc[i], dt)) small_dc[a++] = tc[i]; else small_cc[b++] = tc[i];
+                if (!decode_eligible(tc[i], dt)) small_cc[c++] = tc[i];
+                else if (small_path_is_stream(tc[i].rank, N)) small_sc[a++] = tc[i];
+                else small_dc[b++] = tc[i];
             }
-            if (a > 0) st = launch_apply_decode(small_dc, a, N, C, offsets, perm, min_rows, ws, ws_bytes, dev_status, s);
-            if (st == MOLORA_OK && b > 0) st = launch_apply_rowtile(small_cc, b, dt, N, C, offsets, perm, min_rows, s);
+            if (a > 0) st = launch_apply_stream(small_sc, a, N, C, offsets, perm, min_rows, dev_status, s);
+            if (st == MOLORA_OK && b > 0) st = launch_apply_decode(small_dc, b, N, C, offsets, perm, min_rows, ws, ws_bytes, dev_status, s);
+            if (st == MOLORA_OK && c > 0) st = launch_apply_rowtile(small_cc, c, dt, N, C, offsets, perm, min_rows, s);
         }
     }
+    if (st == MOLORA_OK && n_sc > 0) st = launch_apply_stream(sc, n_sc, N, C, offsets, perm, INT32_MAX, dev_status, s);
     if (st == MOLORA_OK && n_dc > 0) st = launch_apply_decode(dc, n_dc, N, C, offsets, perm, INT32_MAX, ws, ws_bytes, dev_status, s);
     if (st == MOLORA_OK && n_cc > 0) st = launch_apply_rowtile(cc, n_cc, dt, N, C, offsets, perm, INT32_MAX, s);
     return st;

@@ -202,6 +202,10 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
 // an expand launch; takes the segments with fewer than max_rows rows.  The workspace holds the fp32 partial
 // shrink results: the sum of decode_workspace_bytes over the projections.
 bool decode_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
+// Single-launch streaming kernel for calls below the tcgen05 crossover (bf16, ranks 16 / 32 / 64, no workspace).
+molora_status_t launch_apply_stream(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
+                                    const int32_t* offsets, const int32_t* perm, int32_t max_rows, uint32_t* dev_status,
+                                    cudaStream_t s);
 size_t decode_workspace_bytes(int64_t N, int32_t d_in, int32_t rank);
 molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                     const int32_t* offsets, const int32_t* perm, int32_t max_rows, void* ws,
@@ -212,11 +216,7 @@ molora_status_t launch_bounded_wait_selftest(uint32_t* dev_status, int64_t limit
 // Path selection: a segment goes to the tensor-core kernel when it has at least kUmmaMinRows rows and the call
 // has at least kUmmaMinTokens tokens (known on the host); everything else runs on the CUDA-core kernel.
 constexpr int32_t kUmmaMinRows = 32;
-// Calls with fewer tokens run on the two-launch small-tile path.  Measured crossovers on B200 (one projection, d =
-// 2048 and 4096, 4-8 adapters): rank 16 -- the small-tile path wins up to ~3000 tokens, rank 32 up to ~1800, rank 64
-// up to ~1300 (the tensor-core kernel pays a fixed ~0.5 us per 64-column chunk and CTA until all SMs are busy).
 constexpr int64_t kUmmaMinTokens = 1024;     // below this no projection uses the tensor-core kernel
-inline int64_t umma_min_tokens_for_rank(int32_t rank) { return rank <= 16 ? 3072 : rank <= 32 ? 1792 : 1280; }
 constexpr int32_t kUmmaAllSegmentsMaxC = 64;   // up to this many adapters the tensor-core kernel takes all segments
 
 // Launch helper: a cluster of cluster_x CTAs along x when cluster_x > 1, and, when under_predecessor is set,

@@ -69,21 +69,32 @@ def test_invalid_arguments_are_refused_before_any_launch():
     assert apply(N=-3) == 1
 
 
-def test_apply_workspace_sizes_and_refusal_without_it():
+def test_apply_workspace_sizes_and_refusal_without_it(monkeypatch):
+    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH"):
+        monkeypatch.delenv(k, raising=False)
     lib = M.load_library()
     fake = ctypes.c_void_p(0x1000)
-    # the two-launch small-tile path keeps fp32 partial shrink results [slice][N][rank] in the workspace:
-    # 256 tokens, d_in 2048, rank 16 -> 2 slices of 1024 columns -> 2 * 256 * 16 * 4 bytes
-    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 2 * 256 * 16 * 4
-    assert M.molora_apply_workspace_bytes(256, 8, 6144, 2048, 16) == 6 * 256 * 16 * 4
-    # prefill-sized calls with few adapters run on the tcgen05 kernel alone (from 3072 / 1792 / 1280 tokens for ranks
-    # 16 / 32 / 64); rank 8 and fp32-only shapes need none
+    # only the two-launch small-tile kernels need scratch: fp32 partial shrink results [slice][N][rank].  They serve
+    # rank 32 below 1024 tokens and rank 64 below 1280 tokens:
+    # 256 tokens, d_in 2048, rank 32 -> 4 slices of 512 columns -> 4 * 256 * 32 * 4 bytes
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 32) == 4 * 256 * 32 * 4
+    assert M.molora_apply_workspace_bytes(256, 8, 6144, 2048, 32) == 12 * 256 * 32 * 4
+    assert M.molora_apply_workspace_bytes(1024, 8, 2048, 2048, 64) > 0
+    # rank 16 (streaming or tcgen05 kernel), rank 32 from 1024 tokens, rank 64 from 1280 tokens with few adapters, rank 8
+    # and fp32-only shapes need none
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 0
     assert M.molora_apply_workspace_bytes(4096, 4, 2048, 2048, 16) == 0
-    assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 16) > 0 and M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 64) == 0
+    assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 32) == 0
+    assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 64) == 0
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 8) == 0
-    assert M.molora_apply_workspace_bytes(256, 8, 2040, 2048, 16) == 0
-    # with more than 64 adapters the short segments of a large call take the small-tile path
-    assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 16) > 0
-    # a decode-sized bf16 call without its workspace is refused before anything is enqueued
-    st = lib.molora_apply(fake, 64, fake, 64, M.BF16, 4, 64, 64, 16, fake, fake, 2, fake, fake, 1.0, None, 0, None, None)
+    assert M.molora_apply_workspace_bytes(256, 8, 2040, 2048, 32) == 0
+    # with more than 64 adapters the short segments of a large rank-64 call take the two-launch kernels
+    assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 64) > 0
+    assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 16) == 0
+    # the two-launch kernels can be forced for every rank, and then ask for their scratch
+    monkeypatch.setenv("MOLORA_SMALL_PATH", "twophase")
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 2 * 256 * 16 * 4
+    monkeypatch.delenv("MOLORA_SMALL_PATH")
+    # a call for the two-launch kernels without its workspace is refused before anything is enqueued
+    st = lib.molora_apply(fake, 64, fake, 64, M.BF16, 4, 64, 64, 32, fake, fake, 2, fake, fake, 1.0, None, 0, None, None)
     assert st == 3

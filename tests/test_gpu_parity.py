@@ -15,6 +15,23 @@ from _harness import (assert_close, dev_tensor, gpu_route, oracle_route, run_and
 
 pytestmark = pytest.mark.gpu
 
+# The bf16 apply has three kernels for ranks 16 / 32 / 64 (tcgen05, single-launch streaming, two-launch small-tile);
+# the library picks one from rank, token count and bytes.  These settings force one so that every kernel is checked
+# on every shape class, whatever the default choice is.
+KERNEL_MODES = {
+    "default": {},
+    "tcgen05": {"MOLORA_UMMA_MIN_TOKENS": "1024"},                                  # tcgen05 from 1024 tokens
+    "stream": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "stream"},
+    "twophase": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "twophase"},
+}
+
+
+def force_kernel(monkeypatch, mode):
+    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH"):
+        monkeypatch.delenv(k, raising=False)
+    for k, v in KERNEL_MODES[mode].items():
+        monkeypatch.setenv(k, v)
+
 
 # ------------------------------------------------------------------ the five configurations
 def test_c1_tiny_vocab_full():
@@ -298,10 +315,10 @@ def test_kpass_per_sequence_baseline_matches_single_pass():
     assert_close(to_f64(out), to_f64(y1), what="k-pass vs one pass")
 
 
-# ------------------------------------------------------------------ tensor-core path (token counts above the path switch:
-# 3072 tokens for rank 16, 1792 for rank 32, 1280 for rank 64)
+# ------------------------------------------------------------------ tensor-core path (forced from 1024 tokens)
 @pytest.mark.parametrize("rank", [16, 32, 64])
-def test_tensor_path_segment_size_sweep(rank):
+def test_tensor_path_segment_size_sweep(rank, monkeypatch):
+    force_kernel(monkeypatch, "tcgen05")
     # segment sizes straddle the 32-row path threshold, the 4-row gather groups and the 128-row tile
     sizes = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 130, 131, 255, 256, 257, 300, 385, 700]
     r = W.segment_sizes_routing(sizes)
@@ -313,12 +330,14 @@ def test_tensor_path_segment_size_sweep(rank):
 @pytest.mark.parametrize("N,C,d_in,d_out,rank", [(3072, 1, 64, 64, 16), (3300, 3, 2048, 1024, 16),
                                                  (1800, 2, 6144, 2048, 32), (2048, 4, 128, 6144, 64),
                                                  (1280, 5, 4096, 256, 64)])
-def test_tensor_path_shapes(N, C, d_in, d_out, rank):
+def test_tensor_path_shapes(N, C, d_in, d_out, rank, monkeypatch):
+    force_kernel(monkeypatch, "tcgen05")
     w = W.random_problem(N + rank, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.05)
     run_and_check(w, scale=0.75)
 
 
-def test_tensor_path_selector_exact_and_status_clean():
+def test_tensor_path_selector_exact_and_status_clean(monkeypatch):
+    force_kernel(monkeypatch, "tcgen05")
     N, C, d_in, d_out, rank = 3200, 2, 128, 192, 16
     rng = np.random.default_rng(6)
     x = rng.integers(-8, 9, size=(N, d_in)).astype(np.float32)
@@ -378,9 +397,11 @@ def test_forward_host_matches_oracle(name):
     assert int(status.item()) == 0
 
 
-# ------------------------------------------------------------------ decode path (N < 1024: shrink launch + expand launch)
+# ------------------------------------------------------------------ small-tile kernels: single-launch streaming and two-launch
+@pytest.mark.parametrize("mode", ["stream", "twophase"])
 @pytest.mark.parametrize("rank", [16, 32, 64])
-def test_decode_path_segment_size_sweep(rank):
+def test_decode_path_segment_size_sweep(rank, mode, monkeypatch):
+    force_kernel(monkeypatch, mode)
     sizes = [0, 1, 7, 15, 16, 17, 31, 32, 33, 47, 64, 65, 97]
     r = W.segment_sizes_routing(sizes)
     assert r.size < 1024
@@ -392,8 +413,12 @@ def test_decode_path_segment_size_sweep(rank):
                                                  (700, 3, 256, 1024, 64), (64, 64, 512, 96, 16),
                                                  (200, 4, 16384, 64, 32),     # slices longer than one staging pass
                                                  (300, 5, 32, 1536, 64),      # three column slices, one k block
-                                                 (90, 3, 2080, 1056, 16)])    # ragged last slices (multiples of 32 only)
-def test_decode_path_shapes(N, C, d_in, d_out, rank):
+                                                 (90, 3, 2080, 1056, 16),     # ragged last slices (multiples of 32 only)
+                                                 (1500, 3, 1056, 2592, 16),   # more tiles than CTAs x items, ragged chunks
+                                                 (5000, 4, 512, 512, 32)])    # several items per persistent CTA
+@pytest.mark.parametrize("mode", ["stream", "twophase"])
+def test_decode_path_shapes(N, C, d_in, d_out, rank, mode, monkeypatch):
+    force_kernel(monkeypatch, mode)
     w = W.random_problem(N + rank + 7, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.1 if N > 10 else 0.0)
     run_and_check(w)
 
@@ -430,12 +455,15 @@ def test_route_gate_tensor_core_paths(N, d, C):
 
 
 # ------------------------------------------------------------------ seeded random shapes across every kernel path
+@pytest.mark.parametrize("mode", ["default", "tcgen05", "stream", "twophase"])
 @pytest.mark.parametrize("seed", range(24))
-def test_random_shapes_all_paths(seed):
-    # token counts on both sides of the per-rank path switches (1280 / 1792 / 3072 tokens), adapter counts on both sides of the 64-adapter
-    # switch, ranks of every kernel, widths that are multiples of 8 / 32 / 64, skewed routing, unrouted tokens
+def test_random_shapes_all_paths(seed, mode, monkeypatch):
+    # token counts on both sides of the path switches (1024 / 1280 tokens), adapter counts on both sides of the
+    # 64-adapter switch, ranks of every kernel, widths that are multiples of 8 / 32 / 64, skewed routing, unrouted
+    # tokens; every shape with the default kernel choice and with each bf16 kernel forced
+    force_kernel(monkeypatch, mode)
     rng = np.random.default_rng(1000 + seed)
-    N = int(rng.choice([1, 17, 130, 700, 1279, 1280, 1792, 2600, 3071, 3072, 3500]))
+    N = int(rng.choice([1, 17, 130, 700, 1023, 1024, 1279, 1280, 1792, 2600, 3072, 3500]))
     C = int(rng.choice([1, 2, 5, 8, 33, 70]))
     rank = int(rng.choice([8, 16, 32, 64]))
     step = int(rng.choice([8, 32, 64]))
@@ -472,10 +500,12 @@ def test_route_gate_random_shapes_all_kernels(seed):
     assert np.array_equal(r.cpu().numpy()[keep], r_ref[keep])
 
 
+@pytest.mark.parametrize("mode", ["default", "tcgen05"])
 @pytest.mark.parametrize("N", [300, 1400])
-def test_batched_apply_mixed_ranks_and_paths(N):
-    # one batched call whose projections need different kernels: ranks 16 / 64 (tensor-core or two-launch path),
-    # rank 8 and a width that is only a multiple of 8 (CUDA-core path); shared routing
+def test_batched_apply_mixed_ranks_and_paths(N, mode, monkeypatch):
+    # one batched call whose projections need different kernels: ranks 16 / 32 / 64 (tcgen05, streaming or two-launch
+    # kernels), rank 8 and a width that is only a multiple of 8 (CUDA-core kernel); shared routing
+    force_kernel(monkeypatch, mode)
     rng = np.random.default_rng(N)
     C = 6
     r = rng.integers(0, C, size=N).astype(np.int32)
@@ -542,11 +572,13 @@ def test_route_mlp_feeds_group_and_apply():
 
 
 # ------------------------------------------------------------------ top-k weighted routing (Eq. 8, the paper's k = 2)
-@pytest.mark.parametrize("N,C,k,d_in,d_out,rank", [(300, 4, 2, 256, 192, 16),     # small-tile path
-                                                   (3300, 4, 2, 512, 256, 16),    # tensor-core path
-                                                   (200, 6, 3, 128, 96, 8),       # CUDA-core path (rank 8)
-                                                   (500, 5, 1, 64, 64, 32)])      # k = 1: weight exactly 1
-def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank):
+@pytest.mark.parametrize("N,C,k,d_in,d_out,rank,mode", [(300, 4, 2, 256, 192, 16, "stream"),
+                                                        (300, 4, 2, 256, 192, 16, "twophase"),
+                                                        (3300, 4, 2, 512, 256, 16, "tcgen05"),
+                                                        (200, 6, 3, 128, 96, 8, "default"),      # CUDA-core kernel (rank 8)
+                                                        (500, 5, 1, 64, 64, 32, "default")])     # k = 1: weight exactly 1
+def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode, monkeypatch):
+    force_kernel(monkeypatch, mode)
     rng = np.random.default_rng(N + C + k)
     w_ = W.random_problem(500 + N, N, C, d_in, d_out, rank, "bf16")
     p = w_.projections[0]
