@@ -175,14 +175,16 @@ molora_status_t molora_group(const int32_t *r, int64_t N, int32_t C, int32_t *co
  * A   device [C, d_in, rank] of type dt, dense;  B  device [C, rank, d_out] of type dt, dense
  * offsets, perm   device outputs of molora_group for the same N, C (read on the device only)
  * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes, 16-byte aligned (NULL if
- *                 that is 0).  Only the small-tile path writes it (fp32 partial shrink results [slice][N][rank]):
- *                 calls below 3072 / 1792 / 1280 tokens (rank 16 / 32 / 64) and, with more than 64 adapters, the short segments
- *                 of larger calls.
- *                 MOLORA_ERR_WORKSPACE if that path is needed and ws is NULL, misaligned or too small.
- * dev_status      device uint32 or NULL; MOLORA_DEV_TIMEOUT is OR-ed in if a bounded wait inside the
- *                 tensor-core kernel gave up (the kernel then returns without hanging; y is incomplete)
- * The kernel variant (CUDA-core path for small segments, tensor-core tiles for large ones) is chosen on
- * the device from the segment sizes; the paper picks its tile shape from the histogram too (Eq. 12-13). */
+ *                 that is 0).  Only the two-launch small-tile kernels write it (fp32 partial shrink results
+ *                 [slice][N][rank]): bf16 calls of rank 32 below 1024 tokens and of rank 64 below 1280 tokens and, with
+ *                 more than 64 adapters, the short segments of larger rank-64 calls.
+ *                 MOLORA_ERR_WORKSPACE if those kernels are needed and ws is NULL, misaligned or too small.
+ * dev_status      device uint32 or NULL; MOLORA_DEV_TIMEOUT is OR-ed in if a bounded wait inside a kernel gave
+ *                 up (the kernel then returns without hanging; y is incomplete)
+ * The kernel variant is chosen per call on the host from rank, token count and bytes (tcgen05 tiles of 128 rows
+ * for large calls, a single-launch streaming kernel with 32-row tiles below that, CUDA cores for fp32 storage,
+ * rank 8 and odd widths) and per segment on the device from the segment sizes; the paper picks its tile shape
+ * from the histogram too (Eq. 12-13). */
 size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t d_out, int32_t rank);
 molora_status_t molora_apply(const void *x, int64_t ldx, void *y, int64_t ldy, molora_dtype_t dt, int64_t N,
                              int32_t d_in, int32_t d_out, int32_t rank, const void *A, const void *B, int32_t C,
