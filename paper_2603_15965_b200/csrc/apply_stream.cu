@@ -40,7 +40,6 @@ constexpr int kFsWarps = 8;               // compute warps
 constexpr int kFsCopyWarps = 4;            // each moves 8 rows of the tile and a quarter of the weight rows
 constexpr int kFsThreads = (kFsWarps + kFsCopyWarps) * 32;
 constexpr int kFsPermCache = 4096;        // calls with at most this many tokens keep perm in shared memory
-constexpr int kFsBulkPiece = 8192;        // largest single bulk copy issued for a contiguous region
 
 struct StreamParams {
     molora_proj_desc_t p[MOLORA_MAX_PROJECTIONS];
@@ -115,8 +114,8 @@ struct FsItem {
     int ne;         // expand chunks
     int col0;       // first output column
 };
-__device__ __forceinline__ FsItem fs_item(const StreamParams& prm, const FsUnits& units, const int32_t* offs_s, int T,
-                                          int item, int CH)
+__device__ __forceinline__ FsItem fs_item(const StreamParams& prm, const FsUnits& units, const int32_t* offs_s,
+                                          const int32_t* tstart_s, int T, int item, int CH)
 {
     FsItem it;
     const int unit = item / T, tile = item - unit * T;
@@ -128,7 +127,7 @@ __device__ __forceinline__ FsItem fs_item(const StreamParams& prm, const FsUnits
     it.seg = 0;
     it.row0 = 0;
     it.rows = 1;
-    find_tile_smem(offs_s, prm.C, kFsRows, tile, 1, prm.max_rows, it.seg, it.row0, it.rows);
+    find_tile_bisect(offs_s, tstart_s, prm.C, kFsRows, tile, it.seg, it.row0, it.rows);
     const molora_proj_desc_t& pd = prm.p[it.proj];
     it.nks = (pd.d_in + CH - 1) / CH;
     it.col0 = slice * prm.och[it.proj] * CH;
@@ -149,6 +148,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
     using Cfg = FsCfg<R>;
     constexpr int NS = Cfg::NSTAGE;
     __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
+    __shared__ int32_t tstart_s[MOLORA_MAX_ADAPTERS + 1];
     __shared__ int32_t perm_s[kFsPermCache];
     __shared__ __align__(8) uint64_t full_s[NS], done_s[NS];
     __shared__ unsigned long long st_dst[NS][kFsRows];   // expand job in the stage: where its y rows go back to
@@ -172,11 +172,11 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
     if (prm.N <= kFsPermCache)
         for (int i = tid; i < prm.N; i += kFsThreads) perm_s[i] = __ldg(prm.perm + i);
     __syncthreads();
-    int T = 0;
-    for (int c = 0; c < prm.C; ++c) {
-        const int n = offs_s[c + 1] - offs_s[c];
-        if (n >= 1 && n < prm.max_rows) T += (n + kFsRows - 1) / kFsRows;
-    }
+    // tiles of the segments before each segment (those with 1 <= rows < max_rows own tiles here), so that an item finds
+    // its tile by bisection instead of a walk over all segments
+    if (warp == 0) tile_starts(offs_s, prm.C, kFsRows, 1, prm.max_rows, tstart_s);
+    __syncthreads();
+    const int T = tstart_s[prm.C];
     const int nitems = T * units.start[prm.P];
     if (warp == 0) FS_GT(1);
     const uint32_t stage0 = smem_u32(dsm);
@@ -205,7 +205,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
         };
         uint32_t g = 0;                        // jobs issued so far; job k lives in stage k % NS
         for (int item = blockIdx.x; item < nitems && !abort_s; item += (int)gridDim.x) {
-            const FsItem it = fs_item(prm, units, offs_s, T, item, Cfg::CH);
+            const FsItem it = fs_item(prm, units, offs_s, tstart_s, T, item, Cfg::CH);
             const molora_proj_desc_t& pd = prm.p[it.proj];
             const bool rowlane = lane < 8 && myrow < it.rows;
             const int64_t tok = rowlane ? fs_token(prm, perm_s, it.row0 + myrow) : 0;
@@ -274,7 +274,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
     const int g4 = lane >> 2, q = lane & 3;
     uint32_t g = 0;
     for (int item = blockIdx.x; item < nitems; item += (int)gridDim.x) {
-        const FsItem it = fs_item(prm, units, offs_s, T, item, Cfg::CH);
+        const FsItem it = fs_item(prm, units, offs_s, tstart_s, T, item, Cfg::CH);
         const molora_proj_desc_t& pd = prm.p[it.proj];
         const bool two = it.rows > 16;         // the second 16-row MMA tile holds valid rows
 

@@ -125,19 +125,16 @@ struct TpCfg {
 
 // Segment table and (for small calls) the permutation on chip in one memory round trip.  Returns the number of
 // tiles of the segments that belong to this path (1 <= rows < max_rows): work items are (tile, unit) pairs.
-__device__ __forceinline__ int tp_load_tables(const TwoPhaseParams& prm, int32_t* offs_s, int32_t* perm_s)
+__device__ __forceinline__ int tp_load_tables(const TwoPhaseParams& prm, int32_t* offs_s, int32_t* tstart_s, int32_t* perm_s)
 {
     const int tid = threadIdx.x;
     for (int i = tid; i <= prm.C; i += kTpThreads) offs_s[i] = __ldg(prm.offsets + i);
     if (prm.N <= kTpPermCache)
         for (int i = tid; i < prm.N; i += kTpThreads) perm_s[i] = __ldg(prm.perm + i);
     __syncthreads();
-    int tiles = 0;
-    for (int c = 0; c < prm.C; ++c) {
-        const int n = offs_s[c + 1] - offs_s[c];
-        if (n >= 1 && n < prm.max_rows) tiles += (n + kTpRows - 1) / kTpRows;
-    }
-    return tiles;
+    if (tid < 32) tile_starts(offs_s, prm.C, kTpRows, 1, prm.max_rows, tstart_s);
+    __syncthreads();
+    return tstart_s[prm.C];
 }
 struct TpTile {
     int seg, row0, rows;
@@ -163,6 +160,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
     using Cfg = TpCfg<R>;
     constexpr int NT = R / 8;                      // n8 tiles
     __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
+    __shared__ int32_t tstart_s[MOLORA_MAX_ADAPTERS + 1];
     __shared__ int32_t perm_s[kTpPermCache];
     __shared__ __align__(8) uint64_t bar_s;
     __shared__ int abort_s;
@@ -179,7 +177,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
     TP_GT(0, 0);
     grid_dependency_sync();                        // offsets and perm come from the grouping kernel
     TP_GT(0, 1);
-    const int T = tp_load_tables(prm, offs_s, perm_s);
+    const int T = tp_load_tables(prm, offs_s, tstart_s, perm_s);
     const int nitems = T * units.start[prm.P];
     TP_GT(0, 2);
 
@@ -194,7 +192,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
         int proj, ks;
         tp_unit(units, prm.P, unit, proj, ks);
         TpTile t;
-        find_tile_smem(offs_s, prm.C, kTpRows, tile, 1, prm.max_rows, t.seg, t.row0, t.rows);
+        find_tile_bisect(offs_s, tstart_s, prm.C, kTpRows, tile, t.seg, t.row0, t.rows);
         const molora_proj_desc_t& pd = prm.p[proj];
         const bool two = t.rows > 16;              // second 16-row MMA tile holds valid rows
         const int kblocks = pd.d_in / 32, KS = prm.ks[proj];
@@ -292,6 +290,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
     using Cfg = TpCfg<R>;
     constexpr int KB = R / 16;                     // k16 blocks
     __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
+    __shared__ int32_t tstart_s[MOLORA_MAX_ADAPTERS + 1];
     __shared__ int32_t perm_s[kTpPermCache];
     __shared__ __align__(8) uint64_t bar_s;
     __shared__ int abort_s;
@@ -307,7 +306,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
     }
     // Nothing read before the dependency wait below is written by the shrink kernel (see the file header).
     TP_GT(1, 0);
-    const int T = tp_load_tables(prm, offs_s, perm_s);
+    const int T = tp_load_tables(prm, offs_s, tstart_s, perm_s);
     const int nitems = T * units.start[prm.P];
 
     const uint32_t ys = smem_u32(dsm), bs = ys + Cfg::YBYTES;
@@ -323,7 +322,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
         const int unit = item / T, tile = item - unit * T;
         int slice;
         tp_unit(units, prm.P, unit, proj, slice);
-        find_tile_smem(offs_s, prm.C, kTpRows, tile, 1, prm.max_rows, t.seg, t.row0, t.rows);
+        find_tile_bisect(offs_s, tstart_s, prm.C, kTpRows, tile, t.seg, t.row0, t.rows);
         const molora_proj_desc_t& pd = prm.p[proj];
         const int col0 = slice * Cfg::COLS;
         ncols = min(Cfg::COLS, pd.d_out - col0);

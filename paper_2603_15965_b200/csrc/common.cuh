@@ -155,6 +155,52 @@ __device__ __forceinline__ bool find_tile_smem(const int32_t* offs, int C, int t
     return false;
 }
 
+// Bisection form of the lookup for kernels that decode many items per CTA.  tile_starts() (one warp, after
+// offs[0..C] is in shared memory; eight consecutive segments per lane) fills tstart[c] = number of tiles owned by
+// the segments before c, tstart[C] = all tiles; find_tile_bisect() then costs log2(C) shared-memory reads.
+__device__ __forceinline__ void tile_starts(const int32_t* offs, int C, int tile_rows, int min_rows, int max_rows,
+                                            int32_t* tstart)
+{
+    const int lane = threadIdx.x & 31;
+    int cnt[8], sum = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int c = lane * 8 + j;
+        const int n = c < C ? offs[c + 1] - offs[c] : 0;
+        cnt[j] = (n >= min_rows && n < max_rows) ? (n + tile_rows - 1) / tile_rows : 0;
+        sum += cnt[j];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    int run = incl - sum;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int c = lane * 8 + j;
+        if (c <= C) tstart[c] = run;
+        run += cnt[j];
+    }
+    if (lane == 31 && C == MOLORA_MAX_ADAPTERS) tstart[MOLORA_MAX_ADAPTERS] = run;
+}
+// requires 0 <= tile < tstart[C]
+__device__ __forceinline__ void find_tile_bisect(const int32_t* offs, const int32_t* tstart, int C, int tile_rows,
+                                                 int tile, int& seg, int& row0, int& rows)
+{
+    int lo = 0, hi = C;                    // invariant: tstart[lo] <= tile < tstart[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (tstart[mid] <= tile) lo = mid;
+        else hi = mid;
+    }
+    // lo is the last segment whose first tile is <= tile; segments that own no tile share their successor's start
+    seg = lo;
+    row0 = offs[lo] + (tile - tstart[lo]) * tile_rows;
+    rows = min(tile_rows, offs[lo + 1] - row0);
+}
+
 // Host launchers implemented in the .cu files (stream already unwrapped).
 // adapter == nullptr: vocabulary routing; otherwise the compositional gate (r = adapter[i] * M + m)
 molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M,
