@@ -175,7 +175,12 @@ def marshal_step(lib, w, s, shared, stream_handle):
     apply = partial(lib.molora_apply_batched, arr, i32(len(arr)), dt, i64(n), i32(c), vp(s["offsets"].data_ptr()),
                     vp(s["perm"].data_ptr()), vp(aws.data_ptr()) if aws is not None else None,
                     ctypes.c_size_t(aws.numel() if aws is not None else 0), vp(shared["status"].data_ptr()), st)
-    return route, group, apply
+    # the same two stages as ONE call (a single launch where the library can fuse them)
+    group_apply = partial(lib.molora_group_apply_batched, vp(r.data_ptr()), i64(N), i32(C), vp(s["counts"].data_ptr()),
+                          vp(s["offsets"].data_ptr()), vp(s["perm"].data_ptr()), arr, i32(len(arr)), dt,
+                          vp(aws.data_ptr()) if aws is not None else None,
+                          ctypes.c_size_t(aws.numel() if aws is not None else 0), vp(shared["status"].data_ptr()), st)
+    return route, group, apply, group_apply
 
 
 def run_ours(args):
@@ -232,21 +237,33 @@ def run_ours(args):
     # one that asks for a workspace)
     apply_launches = sum(2 if any(M.molora_apply_workspace_bytes(N, C, p.d_in, p.d_out, p.rank) > 0
                                   for p in w.projections if p.rank == rk) else 1 for rk in {p.rank for p in w.projections})
-    launches_per_step = gate_launches + 1 + apply_launches
+    # grouping + apply are one C-ABI call; it is one launch when the library fuses them (every projection on the
+    # streaming kernel), otherwise the grouping launch followed by the apply launches
+    arr0, n0, c0, dt0 = sets[0]["packed"]
+    fused = bool(lib.molora_group_apply_is_one_launch(arr0, len(arr0), dt0, n0))
+    launches_per_step = gate_launches + (1 if fused else 1 + apply_launches)
     for s in sets:
         s["calls"] = marshal_step(lib, w, s, shared, stream.cuda_stream)
 
     def step(s, ev=None):
-        """route -> group -> apply on buffer set s: three C-ABI calls with pre-marshalled arguments."""
-        route, group, apply = s["calls"]
+        """route -> group + apply on buffer set s: two C-ABI calls with pre-marshalled arguments."""
+        route, group, apply, group_apply = s["calls"]
         if route is not None and route() != 0:
             raise RuntimeError("molora_route_* refused the call")
-        if group() != 0:
-            raise RuntimeError("molora_group refused the call")
-        if ev is not None:
-            ev[0].record(stream)
-        if apply() != 0:
-            raise RuntimeError("molora_apply_batched refused the call")
+        if fused or ev is None:
+            if ev is not None:
+                ev[0].record(stream)
+            if group_apply() != 0:
+                raise RuntimeError("molora_group_apply_batched refused the call")
+        else:
+            # eager timing of a call the library does not fuse: the same two calls it makes, taken apart so that the
+            # apply kernels can be bracketed by events
+            if group() != 0:
+                raise RuntimeError("molora_group refused the call")
+            if ev is not None:
+                ev[0].record(stream)
+            if apply() != 0:
+                raise RuntimeError("molora_apply_batched refused the call")
         if ev is not None:
             ev[1].record(stream)
 
@@ -274,8 +291,9 @@ def run_ours(args):
 
             reps, rem = divmod(K, CH)
             g_full, g_rem = capture(step, W0, CH), (capture(step, W0 + reps * CH, rem) if rem else None)
-            a_full = capture(lambda s_: s_["calls"][2](), W0, CH)
-            a_rem = capture(lambda s_: s_["calls"][2](), W0 + reps * CH, rem) if rem else None
+            kcall = 3 if fused else 2          # the dominant kernel: grouping + apply in one launch, or the apply
+            a_full = capture(lambda s_: s_["calls"][kcall](), W0, CH)
+            a_rem = capture(lambda s_: s_["calls"][kcall](), W0 + reps * CH, rem) if rem else None
             g_full.replay()
             torch.cuda.synchronize()
         clocks = Clocks(local)
@@ -361,12 +379,13 @@ def run_ours(args):
                 f"{p.name} {p.d_in}->{p.d_out} r{p.rank}" for p in w.projections) + f", router={w.router}",
                 "tokens_per_step_per_gpu": N, "buffer_sets": n_sets,
                 "l2": f"rotation over {n_sets} buffer sets ({n_sets * per_set / 1e6:.0f} MB > 126 MB L2)",
-                "launch": ("CUDA graph replay of the C-ABI calls (one call per stage)" if args.launch == "graph"
+                "launch": ("CUDA graph replay of the C-ABI calls (route, then group + apply)" if args.launch == "graph"
                            else "eager, one C-ABI call per stage")},
             "gpu_launches": launches_per_step * K,
             "clocks": clk,
             "e2e": e2e,
-            "roofline": {"bound": "hbm", "kernel": "molora_apply (grouped shrink+expand)", "achieved": achieved,
+            "roofline": {"bound": "hbm", "kernel": ("molora_group_apply_batched (grouping + grouped shrink+expand, one launch)" if fused
+                                                    else "molora_apply (grouped shrink+expand)"), "achieved": achieved,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                          "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES.get(name),
                          "algorithmic_bytes": step_bytes, "kernel_ms": apply_ms, "kernel_timing": kernel_timing,

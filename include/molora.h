@@ -211,6 +211,21 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t *projs, int32_t P,
                                      int32_t C, const int32_t *offsets, const int32_t *perm, void *ws, size_t ws_bytes,
                                      uint32_t *dev_status, void *stream);
 
+/* Grouping and grouped application of one layer in one call (Section 3.3 steps 1-4, Algorithm 2): exactly
+ * molora_group(r, ...) followed by molora_apply_batched(projs, ...) on its outputs, with the arguments, results
+ * (counts, offsets and perm are written, bit-equal to molora_group's), status bits and error behaviour of those two
+ * calls; ws / ws_bytes as for molora_apply_batched.  When every projection of the call runs on the single-launch
+ * streaming kernel with one rank (bf16, at most 4096 tokens, below the tcgen05 crossover) the whole call is ONE
+ * launch: every CTA builds the grouping in its shared memory before its first copy request, which saves the
+ * grouping launch; otherwise the two launches are enqueued in stream order. */
+molora_status_t molora_group_apply_batched(const int32_t *r, int64_t N, int32_t C, int32_t *counts, int32_t *offsets,
+                                           int32_t *perm, const molora_proj_desc_t *projs, int32_t P,
+                                           molora_dtype_t dt, void *ws, size_t ws_bytes, uint32_t *dev_status,
+                                           void *stream);
+/* 1 if that call is a single launch for these projections (host array, as above) and this token count, else 0;
+ * pure host arithmetic, for callers that count launches. */
+int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N);
+
 /* ---------------------------------------------------------------------------------------------
  * Top-k weighted routing (Eq. 8): w_i = softmax(TopK(z_i, k)), delta h_i = sum_j w_ij x_i A^(j) B^(j).
  * molora_topk_softmax turns router logits (logits_out of molora_route_gate / molora_route_mlp) into the k kept

@@ -93,6 +93,11 @@ def load_library():
                                  vp, vp]
     lib.molora_apply_batched.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64, i32, vp, vp, vp, sz, vp,
                                          vp]
+    lib.molora_group_apply_batched.argtypes = [vp, i64, i32, vp, vp, vp, ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, vp,
+                                               sz, vp, vp]
+    lib.molora_group_apply_batched.restype = ctypes.c_int
+    lib.molora_group_apply_is_one_launch.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64]
+    lib.molora_group_apply_is_one_launch.restype = i32
     lib.molora_forward_host_arena_bytes.restype = sz
     lib.molora_forward_host_arena_bytes.argtypes = [ctypes.POINTER(_HostProjC), i32, ctypes.c_int, i64, i32, ctypes.c_int,
                                                     i32]
@@ -378,6 +383,33 @@ def molora_apply_batched(projs, offsets: torch.Tensor, perm: torch.Tensor, ws: O
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_apply_batched", lib.molora_apply_batched(arr, len(arr), dt, N, C, _ptr(offsets), _ptr(perm),
                                                             _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
+
+
+def molora_group_apply_batched(r: torch.Tensor, projs, C: Optional[int] = None, counts: Optional[torch.Tensor] = None,
+                               offsets: Optional[torch.Tensor] = None, perm: Optional[torch.Tensor] = None,
+                               ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None, stream=None,
+                               packed=None) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """molora_group followed by molora_apply_batched as one call (one launch where the library can fuse them).
+    Returns (counts, offsets, perm) as molora_group does."""
+    lib = load_library()
+    _i32_dev(r, "r")
+    arr, N, C_, dt = packed if packed is not None else pack_proj_descs(projs)
+    C = C_ if C is None else C
+    if r.numel() != N or C != C_:
+        raise ValueError("r must hold one routing decision per token of the projections")
+    dev = r.device
+    counts = torch.empty(C, dtype=torch.int32, device=dev) if counts is None else _i32_dev(counts, "counts")
+    offsets = torch.empty(C + 1, dtype=torch.int32, device=dev) if offsets is None else _i32_dev(offsets, "offsets")
+    perm = torch.empty(max(N, 1), dtype=torch.int32, device=dev) if perm is None else _i32_dev(perm, "perm")
+    if ws is None:
+        need = molora_apply_batched_workspace_bytes(arr, N, C)
+        if need > 0:
+            ws = torch.empty(need, dtype=torch.uint8, device=dev)
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check("molora_group_apply_batched",
+           lib.molora_group_apply_batched(_ptr(r), N, C, _ptr(counts), _ptr(offsets), _ptr(perm), arr, len(arr), dt, _ptr(ws),
+                                          ws_bytes, _ptr(dev_status), _stream(stream)))
+    return counts, offsets, perm
 
 
 def molora_topk_softmax(logits: torch.Tensor, k: int, stream=None):

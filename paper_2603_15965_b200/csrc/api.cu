@@ -237,6 +237,48 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
     return st;
 }
 
+// every projection on the streaming kernel, one rank, few enough tokens for the CTA-local grouping
+static bool group_apply_fuses(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
+{
+    bool fused = dt == MOLORA_BF16 && group_apply_stream_eligible(N);
+    double bytes = 0.0;
+    for (int i = 0; i < P && fused; ++i) {
+        fused = projs[i].rank == projs[0].rank && decode_eligible(projs[i], dt) && small_path_is_stream(projs[i].rank, N);
+        if (umma_eligible(projs[i], dt)) bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
+    }
+    return fused && !use_umma(projs[0].rank, N, bytes);
+}
+
+int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
+{
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 1) return 0;
+    return group_apply_fuses(projs, P, dt, N) ? 1 : 0;
+}
+
+molora_status_t molora_group_apply_batched(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets,
+                                           int32_t* perm, const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt,
+                                           void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream)
+{
+    // argument checks of both halves first: nothing is enqueued if either would refuse
+    if (N < 0 || N >= INT32_MAX || C < 1) return MOLORA_ERR_INVALID_ARG;
+    if (C > MOLORA_MAX_ADAPTERS) return MOLORA_ERR_UNSUPPORTED;
+    if (counts == nullptr || offsets == nullptr) return MOLORA_ERR_INVALID_ARG;
+    if (N > 0 && (r == nullptr || perm == nullptr)) return MOLORA_ERR_INVALID_ARG;
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS) return MOLORA_ERR_INVALID_ARG;
+    if (dt != MOLORA_F32 && dt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
+    for (int i = 0; i < P; ++i) {
+        const molora_status_t st = check_proj(projs[i], dt);
+        if (st != MOLORA_OK) return st;
+    }
+    // One launch when every projection of the call runs on the streaming kernel with one rank: its CTAs do the
+    // grouping themselves.  Otherwise the two calls, in stream order.
+    if (group_apply_fuses(projs, P, dt, N))
+        return launch_group_apply_stream(r, projs, P, N, C, counts, offsets, perm, dev_status, static_cast<cudaStream_t>(stream));
+    const molora_status_t st = molora_group(r, N, C, counts, offsets, perm, nullptr, 0, dev_status, stream);
+    if (st != MOLORA_OK) return st;
+    return molora_apply_batched(projs, P, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, stream);
+}
+
 molora_status_t molora_apply(const void* x, int64_t ldx, void* y, int64_t ldy, molora_dtype_t dt, int64_t N,
                              int32_t d_in, int32_t d_out, int32_t rank, const void* A, const void* B, int32_t C,
                              const int32_t* offsets, const int32_t* perm, float scale, void* ws, size_t ws_bytes,
@@ -307,14 +349,13 @@ molora_status_t molora_apply_topk(const molora_proj_desc_t* projs, int32_t P, mo
     int32_t* perm = reinterpret_cast<int32_t*>(base + pl.perm);
     molora_proj_desc_t pass[MOLORA_MAX_PROJECTIONS];
     for (int32_t j = 0; j < k; ++j) {               // one (group, apply) pass per kept adapter slot
-        molora_status_t st = molora_group(idx + (int64_t)j * N, N, C, counts, offsets, perm, nullptr, 0, dev_status, stream);
-        if (st != MOLORA_OK) return st;
         for (int i = 0; i < P; ++i) {
             pass[i] = projs[i];
             pass[i].row_scale = w + (int64_t)j * N;
         }
-        st = molora_apply_batched(pass, P, dt, N, C, offsets, perm, pl.apply_ws_bytes > 0 ? base + pl.apply_ws : nullptr,
-                                  pl.apply_ws_bytes, dev_status, stream);
+        const molora_status_t st = molora_group_apply_batched(idx + (int64_t)j * N, N, C, counts, offsets, perm, pass, P, dt,
+                                                              pl.apply_ws_bytes > 0 ? base + pl.apply_ws : nullptr,
+                                                              pl.apply_ws_bytes, dev_status, stream);
         if (st != MOLORA_OK) return st;
     }
     return MOLORA_OK;
@@ -446,10 +487,9 @@ molora_status_t molora_forward_host(molora_router_t router, const int32_t* route
     // 3. group, 4. apply
     int32_t* offsets = reinterpret_cast<int32_t*>(base + pl.offsets);
     int32_t* perm = reinterpret_cast<int32_t*>(base + pl.perm);
-    st = launch_group(r, N, C, reinterpret_cast<int32_t*>(base + pl.counts), offsets, perm, nullptr, 0, dev_status, s);
-    if (st != MOLORA_OK) return st;
-    st = molora_apply_batched(dev, P, dt, N, C, offsets, perm, pl.apply_ws_bytes > 0 ? base + pl.apply_ws : nullptr,
-                              pl.apply_ws_bytes, dev_status, stream);
+    st = molora_group_apply_batched(r, N, C, reinterpret_cast<int32_t*>(base + pl.counts), offsets, perm, dev, P, dt,
+                                    pl.apply_ws_bytes > 0 ? base + pl.apply_ws : nullptr, pl.apply_ws_bytes, dev_status,
+                                    stream);
     if (st != MOLORA_OK) return st;
     // 5. results: device -> host
     for (int i = 0; i < P; ++i)

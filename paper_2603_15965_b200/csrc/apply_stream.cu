@@ -39,6 +39,7 @@ constexpr int kFsRows = 32;               // positions per tile (two 16-row MMA 
 constexpr int kFsWarps = 8;               // compute warps
 constexpr int kFsCopyWarps = 4;            // each moves 8 rows of the tile and a quarter of the weight rows
 constexpr int kFsThreads = (kFsWarps + kFsCopyWarps) * 32;
+constexpr int kFsGroupSmemMaxC = 32;       // grouping variant: adapters handled by the per-thread count table
 constexpr int kFsPermCache = 4096;        // calls with at most this many tokens keep perm in shared memory
 
 struct StreamParams {
@@ -48,6 +49,11 @@ struct StreamParams {
     const int32_t* perm;
     uint32_t* dev_status;
     int32_t N, P, C, max_rows;                // segments with at least max_rows rows belong to the tcgen05 kernel
+    // grouping variant only: the routing decisions and where counts / offsets / perm are written (as by molora_group)
+    const int32_t* r;
+    int32_t* counts_out;
+    int32_t* offsets_out;
+    int32_t* perm_out;
 #ifdef MOLORA_TRACE
     long long* trace;                         // development builds only: globaltimer stamps per CTA
 #endif
@@ -141,7 +147,12 @@ __device__ __forceinline__ int fs_token(const StreamParams& prm, const int32_t* 
 
 }  // namespace
 
-template <int R>
+// GROUP: the call starts from the routing decisions r instead of offsets / perm (at most kFsPermCache tokens).  Every
+// CTA then runs the whole grouping (Section 3.3 steps 1-3: histogram, exclusive scan, stable permutation -- the
+// algorithm of group_cluster_kernel on one CTA) into its own shared memory before its first copy request, which
+// replaces the table load and saves the grouping launch; the CTAs also write counts, offsets and perm out, bit-equal
+// to molora_group's, each a slice of perm.
+template <int R, bool GROUP>
 __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __grid_constant__ StreamParams prm,
                                                                     const __grid_constant__ FsUnits units)
 {
@@ -167,11 +178,184 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
         abort_s = 0;
         fence_mbar_init();
     }
-    // segment table and (small calls) the permutation on chip in one memory round trip
-    for (int i = tid; i <= prm.C; i += kFsThreads) offs_s[i] = __ldg(prm.offsets + i);
-    if (prm.N <= kFsPermCache)
-        for (int i = tid; i < prm.N; i += kFsThreads) perm_s[i] = __ldg(prm.perm + i);
-    __syncthreads();
+    if constexpr (GROUP) {
+        constexpr int NW = kFsThreads / 32;
+      if (prm.C <= kFsGroupSmemMaxC) {
+        // Up to 32 adapters: every thread owns a contiguous run of tokens and counts it into its own column of a
+        // [adapter][thread] table in shared memory (the ring is idle; consecutive threads hit consecutive banks); a warp
+        // per adapter turns the table into exclusive prefixes over the threads, and every thread then writes its run
+        // out in token order -- stable by construction, no atomics.
+        constexpr int TPT = (kFsPermCache + kFsThreads - 1) / kFsThreads;      // tokens per thread
+        constexpr int LPT = kFsThreads / 32;                                   // table entries per lane in the scan
+        int* cnt_s = reinterpret_cast<int*>(dsm);                              // [C][kFsThreads]
+        int* tot_s = cnt_s + kFsGroupSmemMaxC * kFsThreads;                    // [C] adapter totals
+        const int C = prm.C, N = prm.N;
+        const int per = (N + kFsThreads - 1) / kFsThreads;
+        const int b0 = min(tid * per, N), e0 = min(b0 + per, N);
+        int v[TPT];
+        bool bad = false;
+#pragma unroll
+        for (int j = 0; j < TPT; ++j) {
+            const int raw = b0 + j < e0 ? __ldg(prm.r + b0 + j) : -1;
+            bad |= (raw < -1) || (raw >= C);
+            v[j] = (raw >= 0 && raw < C) ? raw : -1;
+        }
+        for (int c = 0; c < C; ++c) cnt_s[c * kFsThreads + tid] = 0;
+#pragma unroll
+        for (int j = 0; j < TPT; ++j)
+            if (v[j] >= 0) cnt_s[v[j] * kFsThreads + tid] += 1;
+        __syncthreads();
+        for (int c = warp; c < C; c += NW) {           // exclusive prefix over the threads, lane = LPT consecutive threads
+            int* row = cnt_s + c * kFsThreads + lane * LPT;
+            int loc[LPT], sum = 0;
+#pragma unroll
+            for (int k = 0; k < LPT; ++k) {
+                loc[k] = row[k];
+                sum += loc[k];
+            }
+            int incl = sum;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += up;
+            }
+            int run = incl - sum;
+#pragma unroll
+            for (int k = 0; k < LPT; ++k) {
+                row[k] = run;
+                run += loc[k];
+            }
+            if (lane == 31) tot_s[c] = incl;
+        }
+        __syncthreads();
+        if (warp == 0) {                               // offsets: exclusive prefix of the totals (C <= 32: one per lane)
+            const int mine = lane < C ? tot_s[lane] : 0;
+            int incl = mine;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += up;
+            }
+            if (lane < C) offs_s[lane] = incl - mine;
+            if (lane == C - 1) offs_s[C] = incl;
+            if (blockIdx.x == 0 && lane < C) prm.counts_out[lane] = mine;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < TPT; ++j)
+            if (v[j] >= 0) {
+                int* slot = cnt_s + v[j] * kFsThreads + tid;
+                const int k = *slot;
+                *slot = k + 1;
+                perm_s[offs_s[v[j]] + k] = b0 + j;
+            }
+        if (blockIdx.x == 0 && prm.dev_status != nullptr && __any_sync(0xFFFFFFFFu, bad) && lane == 0)
+            atomicOr(prm.dev_status, MOLORA_DEV_BAD_ROUTE);
+        __syncthreads();
+        if (blockIdx.x == 0)
+            for (int c = tid; c <= C; c += kFsThreads) prm.offsets_out[c] = offs_s[c];
+      } else {
+        constexpr int STEPS = (kFsPermCache + NW * 32 - 1) / (NW * 32);      // 32-token steps of a warp
+        int(*hist)[MOLORA_MAX_ADAPTERS] = reinterpret_cast<int(*)[MOLORA_MAX_ADAPTERS]>(dsm);   // [warp][adapter]; the ring is idle
+        const int C = prm.C, N = prm.N;
+        const unsigned lt_mask = (1u << lane) - 1u;
+        const int chunk = ((N + NW - 1) / NW + 31) / 32 * 32;                // tokens of a warp: ascending token order
+        const int begin = min(warp * chunk, N), end = min(begin + chunk, N);
+        int vreg[STEPS];
+#pragma unroll
+        for (int j = 0; j < STEPS; ++j) {
+            const int i = begin + j * 32 + lane;
+            vreg[j] = i < end ? __ldg(prm.r + i) : -1;
+        }
+        for (int c = lane; c < C; c += 32) hist[warp][c] = 0;
+        __syncwarp();
+        bool bad = false;
+#pragma unroll
+        for (int j = 0; j < STEPS; ++j) {
+            if (begin + j * 32 < end) {
+                const int v = vreg[j];
+                const bool routed = v >= 0 && v < C;
+                bad |= (v < -1) || (v >= C);
+                const unsigned peers = peers_of(v, routed, C);
+                if (routed && lane == __ffs(peers) - 1) hist[warp][v] += __popc(peers);
+                __syncwarp();
+            }
+        }
+        __syncthreads();
+        // exclusive prefix over the warps, per adapter; the totals are the histogram
+        for (int c = tid; c < C; c += kFsThreads) {
+            int run = 0;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const int t = hist[w][c];
+                hist[w][c] = run;
+                run += t;
+            }
+            tstart_s[c] = run;                 // counts, until the tile prefix replaces them below
+        }
+        __syncthreads();
+        if (warp == 0) {                       // exclusive prefix over adapters, eight consecutive adapters per lane
+            int local[8], sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int c = lane * 8 + j;
+                local[j] = c < C ? tstart_s[c] : 0;
+                sum += local[j];
+            }
+            if (blockIdx.x == 0) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (lane * 8 + j < C) prm.counts_out[lane * 8 + j] = local[j];
+            }
+            int incl = sum;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += up;
+            }
+            int run = incl - sum;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int c = lane * 8 + j;
+                if (c <= C) offs_s[c] = run;
+                run += local[j];
+            }
+            if (lane == 31 && C == MOLORA_MAX_ADAPTERS) offs_s[MOLORA_MAX_ADAPTERS] = run;
+        }
+        __syncthreads();
+        // stable scatter into the CTA's copy of perm
+#pragma unroll
+        for (int j = 0; j < STEPS; ++j) {
+            if (begin + j * 32 < end) {
+                const int v = vreg[j];
+                const bool routed = v >= 0 && v < C;
+                const unsigned peers = peers_of(v, routed, C);
+                if (routed) perm_s[offs_s[v] + hist[warp][v] + __popc(peers & lt_mask)] = begin + j * 32 + lane;
+                __syncwarp();
+                if (routed && lane == __ffs(peers) - 1) hist[warp][v] += __popc(peers);
+                __syncwarp();
+            }
+        }
+        if (blockIdx.x == 0) {
+            for (int c = tid; c <= C; c += kFsThreads) prm.offsets_out[c] = offs_s[c];
+            if (prm.dev_status != nullptr && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(prm.dev_status, MOLORA_DEV_BAD_ROUTE);
+        }
+        __syncthreads();
+      }
+        {   // my slice of perm
+            const int C = prm.C;
+            const int total = offs_s[C];
+            const int per = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+            const int lo = (int)blockIdx.x * per, hi = min(lo + per, total);
+            for (int i = lo + tid; i < hi; i += kFsThreads) prm.perm_out[i] = perm_s[i];
+        }
+    } else {
+        // segment table and (small calls) the permutation on chip in one memory round trip
+        for (int i = tid; i <= prm.C; i += kFsThreads) offs_s[i] = __ldg(prm.offsets + i);
+        if (prm.N <= kFsPermCache)
+            for (int i = tid; i < prm.N; i += kFsThreads) perm_s[i] = __ldg(prm.perm + i);
+        __syncthreads();
+    }
     // tiles of the segments before each segment (those with 1 <= rows < max_rows own tiles here), so that an item finds
     // its tile by bisection instead of a walk over all segments
     if (warp == 0) tile_starts(offs_s, prm.C, kFsRows, 1, prm.max_rows, tstart_s);
@@ -468,18 +652,18 @@ bool stream_eligible(const molora_proj_desc_t& p, molora_dtype_t dt)
     return dt == MOLORA_BF16 && (p.rank == 16 || p.rank == 32 || p.rank == 64) && (p.d_in % 32) == 0 && (p.d_out % 32) == 0;
 }
 
-template <int R>
+template <int R, bool GROUP>
 static cudaError_t stream_launch(StreamParams prm, int64_t N, cudaStream_t s)
 {
     using Cfg = FsCfg<R>;
     static int slots = 0;                          // resident CTAs on this device: the size of a wave
     if (slots == 0) {
-        cudaError_t e = cudaFuncSetAttribute(apply_stream_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+        cudaError_t e = cudaFuncSetAttribute(apply_stream_kernel<R, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
         if (e != cudaSuccess) return e;
         int dev = 0, sms = 0, occ = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, apply_stream_kernel<R>, kFsThreads, Cfg::SMEM);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, apply_stream_kernel<R, GROUP>, kFsThreads, Cfg::SMEM);
         slots = std::max(1, sms * occ);
     }
     // every segment adds at most one partial tile; with a row cap only min(N, C * cap) rows can come here
@@ -516,7 +700,35 @@ static cudaError_t stream_launch(StreamParams prm, int64_t N, cudaStream_t s)
         u.start[i + 1] = u.start[i] + (slices[i] > 0 ? ceil_div(chunks[i], prm.och[i]) : 0);
     }
     const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(tiles_max * u.start[prm.P], slots));
-    return launch_kernel(apply_stream_kernel<R>, dim3(grid), dim3(kFsThreads), Cfg::SMEM, s, 1, false, prm, u);
+    return launch_kernel(apply_stream_kernel<R, GROUP>, dim3(grid), dim3(kFsThreads), Cfg::SMEM, s, 1, false, prm, u);
+}
+
+static molora_status_t stream_enqueue(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C, StreamParams& prm,
+                                      bool group, cudaStream_t s)
+{
+    bool has[3] = {false, false, false};
+    for (int i = 0; i < MOLORA_MAX_PROJECTIONS; ++i) {
+        prm.p[i] = i < P ? projs[i] : molora_proj_desc_t{};
+        prm.och[i] = 0;
+        if (i < P) has[projs[i].rank == 16 ? 0 : projs[i].rank == 32 ? 1 : 2] = true;
+    }
+    prm.P = P;
+    prm.C = C;
+    prm.N = (int32_t)N;
+#ifdef MOLORA_TRACE
+    prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
+#endif
+    cudaError_t e = cudaSuccess;
+    if (group) {                                   // one rank only (checked by the caller): one launch does it all
+        if (has[0]) e = stream_launch<16, true>(prm, N, s);
+        else if (has[1]) e = stream_launch<32, true>(prm, N, s);
+        else e = stream_launch<64, true>(prm, N, s);
+        return cuda_ok(e);
+    }
+    if (has[0] && e == cudaSuccess) e = stream_launch<16, false>(prm, N, s);
+    if (has[1] && e == cudaSuccess) e = stream_launch<32, false>(prm, N, s);
+    if (has[2] && e == cudaSuccess) e = stream_launch<64, false>(prm, N, s);
+    return cuda_ok(e);
 }
 
 molora_status_t launch_apply_stream(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
@@ -525,27 +737,31 @@ molora_status_t launch_apply_stream(const molora_proj_desc_t* projs, int32_t P, 
 {
     if (N == 0 || P == 0) return MOLORA_OK;
     StreamParams prm;
-    bool has[3] = {false, false, false};
-    for (int i = 0; i < MOLORA_MAX_PROJECTIONS; ++i) {
-        prm.p[i] = i < P ? projs[i] : molora_proj_desc_t{};
-        prm.och[i] = 0;
-        if (i < P) has[projs[i].rank == 16 ? 0 : projs[i].rank == 32 ? 1 : 2] = true;
-    }
     prm.offsets = offsets;
     prm.perm = perm;
     prm.dev_status = dev_status;
-    prm.P = P;
-    prm.C = C;
     prm.max_rows = max_rows;
-    prm.N = (int32_t)N;
-#ifdef MOLORA_TRACE
-    prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
-#endif
-    cudaError_t e = cudaSuccess;
-    if (has[0] && e == cudaSuccess) e = stream_launch<16>(prm, N, s);
-    if (has[1] && e == cudaSuccess) e = stream_launch<32>(prm, N, s);
-    if (has[2] && e == cudaSuccess) e = stream_launch<64>(prm, N, s);
-    return cuda_ok(e);
+    prm.r = nullptr;
+    prm.counts_out = prm.offsets_out = prm.perm_out = nullptr;
+    return stream_enqueue(projs, P, N, C, prm, false, s);
+}
+
+bool group_apply_stream_eligible(int64_t N) { return N >= 1 && N <= kFsPermCache; }
+
+molora_status_t launch_group_apply_stream(const int32_t* r, const molora_proj_desc_t* projs, int32_t P, int64_t N,
+                                          int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                          uint32_t* dev_status, cudaStream_t s)
+{
+    StreamParams prm;
+    prm.offsets = nullptr;
+    prm.perm = nullptr;
+    prm.dev_status = dev_status;
+    prm.max_rows = INT32_MAX;
+    prm.r = r;
+    prm.counts_out = counts;
+    prm.offsets_out = offsets;
+    prm.perm_out = perm;
+    return stream_enqueue(projs, P, N, C, prm, true, s);
 }
 
 }  // namespace molora

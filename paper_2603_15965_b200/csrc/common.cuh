@@ -155,6 +155,21 @@ __device__ __forceinline__ bool find_tile_smem(const int32_t* offs, int C, int t
     return false;
 }
 
+// Lanes that hold the same routed adapter as this lane (the value for unrouted lanes is never used); shared by the grouping kernels.
+__device__ __forceinline__ unsigned peers_of(int v, bool routed, int C)
+{
+    if (C <= 8) {   // a few ballots are cheaper than a match
+        unsigned mine = 0;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, routed && v == c);
+            if (v == c) mine = m;
+        }
+        return mine;
+    }
+    return __match_any_sync(0xFFFFFFFFu, routed ? v : -1);
+}
+
 // Bisection form of the lookup for kernels that decode many items per CTA.  tile_starts() (one warp, after
 // offs[0..C] is in shared memory; eight consecutive segments per lane) fills tstart[c] = number of tiles owned by
 // the segments before c, tstart[C] = all tiles; find_tile_bisect() then costs log2(C) shared-memory reads.
@@ -252,6 +267,12 @@ bool decode_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
 molora_status_t launch_apply_stream(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                     const int32_t* offsets, const int32_t* perm, int32_t max_rows, uint32_t* dev_status,
                                     cudaStream_t s);
+// The same kernel started from the routing decisions r: grouping (counts, offsets, perm as molora_group writes them)
+// and apply in one launch; all projections of one rank, at most 4096 tokens.
+bool group_apply_stream_eligible(int64_t N);
+molora_status_t launch_group_apply_stream(const int32_t* r, const molora_proj_desc_t* projs, int32_t P, int64_t N,
+                                          int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                          uint32_t* dev_status, cudaStream_t s);
 size_t decode_workspace_bytes(int64_t N, int32_t d_in, int32_t rank);
 molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                     const int32_t* offsets, const int32_t* perm, int32_t max_rows, void* ws,

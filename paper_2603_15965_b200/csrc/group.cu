@@ -30,21 +30,6 @@ constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kGroupMaxCluster = 8;
 constexpr int kGroupCached = 4;      // 32-token steps of a warp kept in registers
 
-// Lanes that hold the same routed adapter as this lane (0 for unrouted lanes are never used).
-__device__ __forceinline__ unsigned peers_of(int v, bool routed, int C)
-{
-    if (C <= 8) {   // a few ballots are cheaper than a match
-        unsigned mine = 0;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const unsigned m = __ballot_sync(0xFFFFFFFFu, routed && v == c);
-            if (v == c) mine = m;
-        }
-        return mine;
-    }
-    return __match_any_sync(0xFFFFFFFFu, routed ? v : -1);
-}
-
 __global__ void __launch_bounds__(kGroupThreads) group_cluster_kernel(const int32_t* __restrict__ r, int64_t N, int C,
                                                                      int32_t* __restrict__ counts,
                                                                      int32_t* __restrict__ offsets,

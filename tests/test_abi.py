@@ -11,7 +11,7 @@ def test_library_builds_loads_and_exports_header_symbols():
     lib = M.load_library()
     names = M.exported_symbols()
     assert {"molora_route_vocab", "molora_route_composite", "molora_route_mlp", "molora_route_mlp_workspace_bytes", "molora_topk_softmax", "molora_apply_topk",
-            "molora_apply_topk_workspace_bytes", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched",
+            "molora_apply_topk_workspace_bytes", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched", "molora_group_apply_batched",
             "molora_group_workspace_bytes", "molora_apply_workspace_bytes", "molora_route_gate_workspace_bytes",
             "molora_version",
             "molora_status_string"} <= set(names)

@@ -611,3 +611,62 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode, monk
     err = np.abs(got - ref)
     bound = 1e-3 + 2e-2 * np.abs(ref) + slack
     assert np.all(err[keep] <= bound[keep]), f"top-{k} weighted apply: worst ratio {(err / bound)[keep].max():.3f}"
+
+
+# ------------------------------------------------------------------ grouping + apply in one call (one launch where fused)
+@pytest.mark.parametrize("N,C,shapes,mode", [
+    (4096, 4, [(2048, 2048, 16)], "default"),                                   # c2's apply: fused, the largest fused size
+    (256, 8, [(2048, 2048, 16), (2048, 1024, 16), (6144, 2048, 16)], "default"),  # a decode layer's shapes: fused, 3 projections
+    (1, 1, [(32, 32, 16)], "default"), (33, 256, [(64, 96, 16)], "default"),    # one token; more adapters than tokens
+    (1500, 5, [(512, 320, 32)], "default"),                                     # rank 32 streaming: fused
+    (700, 70, [(256, 512, 16)], "default"),                                     # many adapters, match_any grouping
+    (4097, 4, [(256, 256, 16)], "default"),                                     # one token too many: two launches
+    (600, 3, [(256, 256, 16), (256, 128, 64)], "default"),                      # mixed ranks: two launches
+    (300, 4, [(128, 192, 8)], "default"),                                       # CUDA-core apply: two launches
+    (900, 6, [(512, 512, 16)], "twophase"),                                     # two-launch apply forced: group + 2
+])
+def test_group_apply_one_call_matches_oracle_and_group(N, C, shapes, mode, monkeypatch):
+    force_kernel(monkeypatch, mode)
+    rng = np.random.default_rng(N * 31 + C)
+    p = rng.dirichlet(np.full(C, 0.6))
+    r = rng.choice(C, size=N, p=p).astype(np.int32)
+    if N > 10:
+        r[rng.random(N) < 0.07] = -1
+    ws = [W.random_problem(8100 + i, N, C, di, do, rk, "bf16", r=r) for i, (di, do, rk) in enumerate(shapes)]
+    xs = [dev_tensor(w.inputs["x"], "bf16") for w in ws]
+    ys = [dev_tensor(w.projections[0].y, "bf16") for w in ws]
+    As = [dev_tensor(w.projections[0].A, "bf16") for w in ws]
+    Bs = [dev_tensor(w.projections[0].B, "bf16") for w in ws]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # poison the outputs: everything the call must write is checked below
+    counts = torch.full((C,), -7, dtype=torch.int32, device="cuda")
+    offsets = torch.full((C + 1,), -7, dtype=torch.int32, device="cuda")
+    perm = torch.full((N,), -7, dtype=torch.int32, device="cuda")
+    M.molora_group_apply_batched(dev_tensor(r, "i"), [M.ProjDesc(x, y, A, B, 1.0) for x, y, A, B in zip(xs, ys, As, Bs)],
+                                 counts=counts, offsets=offsets, perm=perm, dev_status=status)
+    c_ref, o_ref, p_ref = oracle.group(r, C)
+    assert np.array_equal(counts.cpu().numpy(), c_ref)
+    assert np.array_equal(offsets.cpu().numpy(), o_ref)
+    assert np.array_equal(perm.cpu().numpy()[: o_ref[-1]], p_ref)
+    assert int(status.item()) == 0
+    for w, y in zip(ws, ys):
+        pr = w.projections[0]
+        ref, _ = oracle.apply(w.inputs["x"], pr.y, pr.A, pr.B, r)
+        assert_close(to_f64(y), ref, what=f"group+apply {pr.d_in}->{pr.d_out} r{pr.rank}")
+
+
+def test_group_apply_one_call_flags_bad_routes():
+    N, C = 500, 4
+    rng = np.random.default_rng(77)
+    r = rng.integers(0, C, size=N).astype(np.int32)
+    r[[3, 250]] = [C, -5]                       # outside [-1, C): unrouted, flagged
+    w = W.random_problem(8200, N, C, 256, 256, 16, "bf16", r=np.where((r >= 0) & (r < C), r, -1).astype(np.int32))
+    pr = w.projections[0]
+    x, y = dev_tensor(w.inputs["x"], "bf16"), dev_tensor(pr.y, "bf16")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    counts, offsets, perm = M.molora_group_apply_batched(dev_tensor(r, "i"), [M.ProjDesc(x, y, dev_tensor(pr.A, "bf16"), dev_tensor(pr.B, "bf16"), 1.0)],
+                                                         dev_status=status)
+    assert int(status.item()) & 2                # MOLORA_DEV_BAD_ROUTE
+    ref, _ = oracle.apply(w.inputs["x"], pr.y, pr.A, pr.B, w.r)
+    assert_close(to_f64(y), ref, what="bad routes are unrouted")
+    assert int(offsets.cpu().numpy()[-1]) == N - 2
