@@ -30,7 +30,7 @@ METRIC = "routed_lora_tokens_per_s"
 UNIT = "tokens/s"
 L2_BYTES = 126e6
 # dram__bytes_read.sum + dram__bytes_write.sum per apply launch from the committed ncu capture (profiles/), by workload
-NCU_TRAFFIC_BYTES = {"c2": 34.13e6, "c3": 26.77e6, "c5": 615.3e6}
+NCU_TRAFFIC_BYTES = {"c2": 34.17e6, "c3": 26.81e6, "c5": 615.3e6}
 
 
 def measured_peaks():
