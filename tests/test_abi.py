@@ -98,3 +98,41 @@ def test_apply_workspace_sizes_and_refusal_without_it(monkeypatch):
     # a call for the two-launch kernels without its workspace is refused before anything is enqueued
     st = lib.molora_apply(fake, 64, fake, 64, M.BF16, 4, 64, 64, 32, fake, fake, 2, fake, fake, 1.0, None, 0, None, None)
     assert st == 3
+
+
+def _desc(d_in, d_out, rank):
+    from paper_2603_15965_b200.binding import _ProjDescC
+    return _ProjDescC(0x1000, d_in, 0x2000, d_out, 0x3000, 0x4000, d_in, d_out, rank, 1.0, None)
+
+
+def test_group_apply_one_call_launch_count_and_refusals(monkeypatch):
+    """Host arithmetic only: when molora_group_apply_batched is one launch, and that it validates both halves."""
+    from paper_2603_15965_b200.binding import _ProjDescC
+    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH"):
+        monkeypatch.delenv(k, raising=False)
+    lib = M.load_library()
+
+    def one_launch(shapes, N, dt=M.BF16):
+        arr = (_ProjDescC * len(shapes))(*[_desc(*s) for s in shapes])
+        return int(lib.molora_group_apply_is_one_launch(arr, len(shapes), dt, N))
+
+    assert one_launch([(2048, 2048, 16)], 4096) == 1                    # c2's apply
+    assert one_launch([(2048, 2048, 16)] * 4 + [(2048, 6144, 16)] * 2 + [(6144, 2048, 16)], 256) == 1   # a decode layer
+    assert one_launch([(2048, 2048, 16)], 4097) == 0                    # more tokens than a CTA groups on its own
+    assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 0   # rank 32 streams from 1024 tokens
+    assert one_launch([(2048, 2048, 64)], 512) == 0                     # rank 64: two-launch kernels / tcgen05
+    assert one_launch([(2048, 2048, 16), (2048, 2048, 32)], 2048) == 0  # two ranks: two apply launches
+    assert one_launch([(2048, 2048, 16)] * 8, 4096) == 0                # 400 MB: above the tcgen05 crossover
+    assert one_launch([(2048, 2048, 16)], 4096, M.F32) == 0             # fp32 storage: CUDA-core kernel
+    assert one_launch([(2048, 2040, 16)], 256) == 0                     # width not a multiple of 32: CUDA-core kernel
+    monkeypatch.setenv("MOLORA_SMALL_PATH", "twophase")
+    assert one_launch([(2048, 2048, 16)], 4096) == 0
+    monkeypatch.delenv("MOLORA_SMALL_PATH")
+    # refusals before any launch: null outputs, too many adapters, no projections, unsupported rank
+    fake = ctypes.c_void_p(0x1000)
+    arr = (_ProjDescC * 1)(_desc(64, 64, 16))
+    assert lib.molora_group_apply_batched(fake, 8, 4, None, fake, fake, arr, 1, M.BF16, None, 0, None, None) == 1
+    assert lib.molora_group_apply_batched(fake, 8, 257, fake, fake, fake, arr, 1, M.BF16, None, 0, None, None) == 2
+    assert lib.molora_group_apply_batched(fake, 8, 4, fake, fake, fake, arr, 0, M.BF16, None, 0, None, None) == 1
+    bad = (_ProjDescC * 1)(_desc(64, 64, 12))
+    assert lib.molora_group_apply_batched(fake, 8, 4, fake, fake, fake, bad, 1, M.BF16, None, 0, None, None) != 0
