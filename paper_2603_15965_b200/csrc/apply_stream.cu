@@ -35,11 +35,12 @@ namespace molora {
 
 using namespace ptx;
 
-constexpr int kFsRows = 32;               // positions per tile (two 16-row MMA tiles)
+constexpr int kFsMaxRows = 32;            // most positions of a tile (two 16-row MMA tiles)
 constexpr int kFsWarps = 8;               // compute warps
 constexpr int kFsCopyWarps = 4;            // each moves 8 rows of the tile and a quarter of the weight rows
 constexpr int kFsThreads = (kFsWarps + kFsCopyWarps) * 32;
 constexpr int kFsGroupSmemMaxC = 32;       // grouping variant: adapters handled by the per-thread count table
+constexpr double kFsShortFill = 1.25;     // rank 16: short tiles while (16-row tiles x projections) <= this x SMs
 constexpr int kFsPermCache = 4096;        // calls with at most this many tokens keep perm in shared memory
 
 struct StreamParams {
@@ -75,16 +76,25 @@ struct FsUnits {
     int32_t start[MOLORA_MAX_PROJECTIONS + 1];
 };
 
-template <int R>
+// SHORT (rank 16 only): 16-row tiles and 1024-column chunks instead of 32 rows and 512 columns.
+template <int R, bool SHORT>
 struct FsCfg {
-    static constexpr int CH = 512;                               // columns of a chunk (of d_in or of d_out)
-    static constexpr int NSTAGE = R == 16 ? 4 : R == 32 ? 3 : 2;
+    static_assert(!SHORT || R == 16, "the short tile exists for rank 16");
+    // The SM accepts one bulk-copy request per ~25 cycles whatever its size, so 1 KB requests cap an SM at ~40 B/cycle
+    // and an item with a long reduction is bound by them.  The short tile moves 2 KB per request and needs fewer
+    // output slices (each of which recomputes the shrink) to fill the SMs of a small call; it reads the weight chunks
+    // twice as often per row, which costs more than it saves once every SM has several tiles.
+    static constexpr int ROWS = SHORT ? 16 : 32;                 // positions per tile
+    static constexpr int MT = ROWS / 16;                         // 16-row MMA tiles
+    static constexpr int RPW = ROWS / kFsCopyWarps;              // rows of the tile a copy warp moves
+    static constexpr int CH = SHORT ? 1024 : 512;                // columns of a chunk (of d_in or of d_out)
+    static constexpr int NSTAGE = SHORT ? 3 : R == 16 ? 4 : R == 32 ? 3 : 2;
     static constexpr int RP = CH * 2 + 16;                       // pitch of a staged x / y / B_c row: 16 bytes of padding
-    static constexpr int ROWBYTES = kFsRows * RP;                //   keep the 8 rows of an ldmatrix in distinct banks
+    static constexpr int ROWBYTES = ROWS * RP;                //   keep the 8 rows of an ldmatrix in distinct banks
     static constexpr int ABYTES = CH * R * 2;                    // the chunk's rows of A_c, dense [k][R]
     static constexpr int BBYTES = R * RP;
     static constexpr int STAGE = ROWBYTES + (ABYTES > BBYTES ? ABYTES : BBYTES);
-    static constexpr int TFLOATS = kFsRows * R;                  // one fp32 copy of t
+    static constexpr int TFLOATS = ROWS * R;                  // one fp32 copy of t
     static constexpr int SMEM = NSTAGE * STAGE + TFLOATS * 4 + 16;
     static_assert(kFsWarps * TFLOATS * 4 <= STAGE, "the per-warp partials are summed through one stage");
 };
@@ -121,7 +131,7 @@ struct FsItem {
     int col0;       // first output column
 };
 __device__ __forceinline__ FsItem fs_item(const StreamParams& prm, const FsUnits& units, const int32_t* offs_s,
-                                          const int32_t* tstart_s, int T, int item, int CH)
+                                          const int32_t* tstart_s, int T, int item, int CH, int ROWS)
 {
     FsItem it;
     const int unit = item / T, tile = item - unit * T;
@@ -133,7 +143,7 @@ __device__ __forceinline__ FsItem fs_item(const StreamParams& prm, const FsUnits
     it.seg = 0;
     it.row0 = 0;
     it.rows = 1;
-    find_tile_bisect(offs_s, tstart_s, prm.C, kFsRows, tile, it.seg, it.row0, it.rows);
+    find_tile_bisect(offs_s, tstart_s, prm.C, ROWS, tile, it.seg, it.row0, it.rows);
     const molora_proj_desc_t& pd = prm.p[it.proj];
     it.nks = (pd.d_in + CH - 1) / CH;
     it.col0 = slice * prm.och[it.proj] * CH;
@@ -152,17 +162,17 @@ __device__ __forceinline__ int fs_token(const StreamParams& prm, const int32_t* 
 // algorithm of group_cluster_kernel on one CTA) into its own shared memory before its first copy request, which
 // replaces the table load and saves the grouping launch; the CTAs also write counts, offsets and perm out, bit-equal
 // to molora_group's, each a slice of perm.
-template <int R, bool GROUP>
+template <int R, bool GROUP, bool SHORT>
 __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __grid_constant__ StreamParams prm,
                                                                     const __grid_constant__ FsUnits units)
 {
-    using Cfg = FsCfg<R>;
+    using Cfg = FsCfg<R, SHORT>;
     constexpr int NS = Cfg::NSTAGE;
     __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
     __shared__ int32_t tstart_s[MOLORA_MAX_ADAPTERS + 1];
     __shared__ int32_t perm_s[kFsPermCache];
     __shared__ __align__(8) uint64_t full_s[NS], done_s[NS];
-    __shared__ unsigned long long st_dst[NS][kFsRows];   // expand job in the stage: where its y rows go back to
+    __shared__ unsigned long long st_dst[NS][kFsMaxRows];   // expand job in the stage: where its y rows go back to
     __shared__ uint32_t st_bytes[kFsCopyWarps][NS];      // bytes per row to store (0: a shrink job, nothing to store)
     __shared__ int st_rows[kFsCopyWarps][NS];
     __shared__ int abort_s;
@@ -358,7 +368,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
     }
     // tiles of the segments before each segment (those with 1 <= rows < max_rows own tiles here), so that an item finds
     // its tile by bisection instead of a walk over all segments
-    if (warp == 0) tile_starts(offs_s, prm.C, kFsRows, 1, prm.max_rows, tstart_s);
+    if (warp == 0) tile_starts(offs_s, prm.C, Cfg::ROWS, 1, prm.max_rows, tstart_s);
     __syncthreads();
     const int T = tstart_s[prm.C];
     const int nitems = T * units.start[prm.P];
@@ -368,18 +378,19 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
 
     if (warp >= kFsWarps) {
         // ------------------------------------------------------------------------------------------ copy warps
-        // Copy warp w owns rows 8w .. 8w+7 of the tile (lanes 0-7, one bulk request each) and a quarter of the
+        // Copy warp w owns RPW consecutive rows of the tile (its first RPW lanes, one bulk request each) and a quarter of the
         // weight rows (lanes 8 ..); the four warps run the same job list without talking to one another -- each
         // arrives once per job on the stage's "full" barrier with the bytes it requested.
         const int cw = warp - kFsWarps;
-        const int myrow = cw * 8 + (lane & 7);
+        constexpr int RPW = Cfg::RPW;
+        const int myrow = cw * RPW + (lane % RPW);
         // the stage's previous job is finished: write back my y rows if it was an expand chunk
         auto retire = [&](uint32_t k) {
             const uint32_t s = k % NS;
             wait_bar(smem_u32(&done_s[s]), (k / NS) & 1u, &abort_s, prm.dev_status);
             const uint32_t nb = st_bytes[cw][s];
             if (nb != 0 && !abort_s) {
-                if (lane < 8 && myrow < st_rows[cw][s])
+                if (lane < RPW && myrow < st_rows[cw][s])
                     bulk_store(reinterpret_cast<void*>(st_dst[s][myrow]), stage0 + s * Cfg::STAGE + myrow * Cfg::RP, nb);
                 bulk_commit_group();
                 bulk_wait_group_read<0>();     // the stage may be overwritten
@@ -389,15 +400,15 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
         };
         uint32_t g = 0;                        // jobs issued so far; job k lives in stage k % NS
         for (int item = blockIdx.x; item < nitems && !abort_s; item += (int)gridDim.x) {
-            const FsItem it = fs_item(prm, units, offs_s, tstart_s, T, item, Cfg::CH);
+            const FsItem it = fs_item(prm, units, offs_s, tstart_s, T, item, Cfg::CH, Cfg::ROWS);
             const molora_proj_desc_t& pd = prm.p[it.proj];
-            const bool rowlane = lane < 8 && myrow < it.rows;
+            const bool rowlane = lane < RPW && myrow < it.rows;
             const int64_t tok = rowlane ? fs_token(prm, perm_s, it.row0 + myrow) : 0;
             const char* xrow = static_cast<const char*>(pd.x) + tok * pd.ldx * 2;
             char* yrow = static_cast<char*>(pd.y) + tok * pd.ldy * 2 + (int64_t)it.col0 * 2;
             const char* Ac = static_cast<const char*>(pd.A) + (int64_t)it.seg * pd.d_in * R * 2;
             const char* Bc = static_cast<const char*>(pd.B) + ((int64_t)it.seg * R * pd.d_out + it.col0) * 2;
-            const int myrows = max(0, min(8, it.rows - cw * 8));
+            const int myrows = max(0, min(RPW, it.rows - cw * RPW));
             for (int j = 0; j < it.nks + it.ne; ++j, ++g) {
                 const uint32_t s = g % NS;
                 if (g >= (uint32_t)NS) retire(g - NS);
@@ -416,7 +427,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                     }
                     __syncwarp();
                     if (rowlane) bulk_load(sb + myrow * Cfg::RP, xrow + (int64_t)k0 * 2, xbytes, bar);
-                    if (lane == 8) bulk_load(sb + Cfg::ROWBYTES + cw * aq, Ac + (int64_t)k0 * R * 2 + cw * aq, aq, bar);
+                    if (lane == RPW) bulk_load(sb + Cfg::ROWBYTES + cw * aq, Ac + (int64_t)k0 * R * 2 + cw * aq, aq, bar);
                 } else {
                     const int c0 = (j - it.nks) * Cfg::CH, nc = min(Cfg::CH, pd.d_out - it.col0 - c0);
                     const uint32_t rowbytes = (uint32_t)nc * 2u;
@@ -428,8 +439,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                     }
                     __syncwarp();
                     if (rowlane) bulk_load(sb + myrow * Cfg::RP, yrow + (int64_t)c0 * 2, rowbytes, bar);
-                    if (lane >= 8 && lane < 8 + R / kFsCopyWarps) {
-                        const int k = cw * (R / kFsCopyWarps) + lane - 8;
+                    if (lane >= RPW && lane < RPW + R / kFsCopyWarps) {
+                        const int k = cw * (R / kFsCopyWarps) + lane - RPW;
                         bulk_load(sb + Cfg::ROWBYTES + k * Cfg::RP, Bc + ((int64_t)k * pd.d_out + c0) * 2, rowbytes, bar);
                     }
                 }
@@ -455,17 +466,18 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
     // ---------------------------------------------------------------------------------------------- compute warps
     constexpr int NT = R / 8;                  // n8 tiles of t
     constexpr int KB = R / 16;                 // k16 blocks of the expand
+    constexpr int MT = Cfg::MT;
     const int g4 = lane >> 2, q = lane & 3;
     uint32_t g = 0;
     for (int item = blockIdx.x; item < nitems; item += (int)gridDim.x) {
-        const FsItem it = fs_item(prm, units, offs_s, tstart_s, T, item, Cfg::CH);
+        const FsItem it = fs_item(prm, units, offs_s, tstart_s, T, item, Cfg::CH, Cfg::ROWS);
         const molora_proj_desc_t& pd = prm.p[it.proj];
-        const bool two = it.rows > 16;         // the second 16-row MMA tile holds valid rows
+        const bool two = MT == 2 && it.rows > 16;   // the second 16-row MMA tile holds valid rows
 
         // ---- shrink: t = x A_c, fp32 partial per warp
-        float acc[2][NT][4];
+        float acc[MT][NT][4];
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
+        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
             for (int n = 0; n < NT; ++n)
 #pragma unroll
@@ -485,7 +497,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                     for (int n16 = 0; n16 < NT / 2; ++n16)
                         fs_ldsm_t(bf[n16], as + (b * 32 + h * 16 + (m & 1) * 8 + (lane & 7)) * (R * 2) + (n16 * 16 + (m >> 1) * 8) * 2);
 #pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {
+                    for (int mt = 0; mt < MT; ++mt) {
                         if (mt == 0 || two) {
                             uint32_t a[4];
                             fs_ldsm(a, xs + (mt * 16 + (lane & 15)) * Cfg::RP + (b * 32 + h * 16 + (lane >> 4) * 8) * 2);
@@ -508,7 +520,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                 float* tpart = tparts + warp * Cfg::TFLOATS;
                 fs_compute_sync();                 // every warp has finished reading the stage (and the previous item's t)
 #pragma unroll
-                for (int mt = 0; mt < 2; ++mt)
+                for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                     for (int n = 0; n < NT; ++n) {
                         const int c = n * 8 + 2 * q;
@@ -541,9 +553,9 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
         }
 
         // ---- A fragments of t: bf16 hi and lo parts
-        uint32_t thi[2][KB][4], tlo[2][KB][4];
+        uint32_t thi[MT][KB][4], tlo[MT][KB][4];
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
+        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
@@ -569,14 +581,14 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             constexpr int GI = R == 64 ? 1 : 2;
             const int ngroups = ncols / 32;
             for (int grp0 = warp; grp0 < ngroups; grp0 += GI * kFsWarps) {
-                uint32_t yv[GI][2][2][4];
-                float d[GI][2][4][4];
+                uint32_t yv[GI][MT][2][4];
+                float d[GI][MT][4][4];
 #pragma unroll
                 for (int gi = 0; gi < GI; ++gi) {
                     const int grp = grp0 + gi * kFsWarps;
                     if (grp < ngroups) {
 #pragma unroll
-                        for (int mt = 0; mt < 2; ++mt)
+                        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                             for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -585,7 +597,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                                         ysp + (mt * 16 + g4 + 8 * h) * Cfg::RP + (grp * 32 + nt * 8 + 2 * q) * 2);
                     }
 #pragma unroll
-                    for (int mt = 0; mt < 2; ++mt)
+                    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                         for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
@@ -603,7 +615,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                             for (int p2 = 0; p2 < 2; ++p2)
                                 fs_ldsm_t(bf[p2], bs + (kb * 16 + (m & 1) * 8 + (lane & 7)) * Cfg::RP + (grp * 32 + p2 * 16 + (m >> 1) * 8) * 2);
 #pragma unroll
-                            for (int mt = 0; mt < 2; ++mt) {
+                            for (int mt = 0; mt < MT; ++mt) {
                                 if (mt == 0 || two) {
 #pragma unroll
                                     for (int p2 = 0; p2 < 2; ++p2) {
@@ -626,7 +638,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                     const int grp = grp0 + gi * kFsWarps;
                     if (grp < ngroups) {
 #pragma unroll
-                        for (int mt = 0; mt < 2; ++mt)
+                        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                             for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -652,23 +664,23 @@ bool stream_eligible(const molora_proj_desc_t& p, molora_dtype_t dt)
     return dt == MOLORA_BF16 && (p.rank == 16 || p.rank == 32 || p.rank == 64) && (p.d_in % 32) == 0 && (p.d_out % 32) == 0;
 }
 
-template <int R, bool GROUP>
+template <int R, bool GROUP, bool SHORT>
 static cudaError_t stream_launch(StreamParams prm, int64_t N, cudaStream_t s)
 {
-    using Cfg = FsCfg<R>;
+    using Cfg = FsCfg<R, SHORT>;
     static int slots = 0;                          // resident CTAs on this device: the size of a wave
     if (slots == 0) {
-        cudaError_t e = cudaFuncSetAttribute(apply_stream_kernel<R, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+        cudaError_t e = cudaFuncSetAttribute(apply_stream_kernel<R, GROUP, SHORT>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
         if (e != cudaSuccess) return e;
         int dev = 0, sms = 0, occ = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, apply_stream_kernel<R, GROUP>, kFsThreads, Cfg::SMEM);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, apply_stream_kernel<R, GROUP, SHORT>, kFsThreads, Cfg::SMEM);
         slots = std::max(1, sms * occ);
     }
     // every segment adds at most one partial tile; with a row cap only min(N, C * cap) rows can come here
     const int64_t cap_rows = prm.max_rows == INT32_MAX ? N : std::min<int64_t>(N, (int64_t)prm.C * prm.max_rows);
-    const int64_t tiles_max = ceil_div64(cap_rows, kFsRows) + prm.C;
+    const int64_t tiles_max = ceil_div64(cap_rows, Cfg::ROWS) + prm.C;
     // Output slices per projection: start with one item per (projection, tile); while the items certainly fit into
     // one wave, split the widest item once more (its shrink is then recomputed per slice).  A second round of
     // items costs more than the imbalance it removes.
@@ -700,7 +712,7 @@ static cudaError_t stream_launch(StreamParams prm, int64_t N, cudaStream_t s)
         u.start[i + 1] = u.start[i] + (slices[i] > 0 ? ceil_div(chunks[i], prm.och[i]) : 0);
     }
     const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(tiles_max * u.start[prm.P], slots));
-    return launch_kernel(apply_stream_kernel<R, GROUP>, dim3(grid), dim3(kFsThreads), Cfg::SMEM, s, 1, false, prm, u);
+    return launch_kernel(apply_stream_kernel<R, GROUP, SHORT>, dim3(grid), dim3(kFsThreads), Cfg::SMEM, s, 1, false, prm, u);
 }
 
 static molora_status_t stream_enqueue(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C, StreamParams& prm,
@@ -718,16 +730,28 @@ static molora_status_t stream_enqueue(const molora_proj_desc_t* projs, int32_t P
 #ifdef MOLORA_TRACE
     prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
 #endif
+    // rank 16: the short tile while its tiles of all projections (nearly) fit one wave of CTAs
+    int p16 = 0;
+    for (int i = 0; i < P; ++i) p16 += projs[i].rank == 16;
+    int sms = 148;
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    const int64_t cap_rows = prm.max_rows == INT32_MAX ? N : std::min<int64_t>(N, (int64_t)C * prm.max_rows);
+    bool short16 = (ceil_div64(cap_rows, 16) + C) * p16 <= (int64_t)(sms * kFsShortFill);
+    if (const char* e = getenv("MOLORA_STREAM_TILE")) short16 = atoi(e) == 16;
     cudaError_t e = cudaSuccess;
     if (group) {                                   // one rank only (checked by the caller): one launch does it all
-        if (has[0]) e = stream_launch<16, true>(prm, N, s);
-        else if (has[1]) e = stream_launch<32, true>(prm, N, s);
-        else e = stream_launch<64, true>(prm, N, s);
+        if (has[0]) e = short16 ? stream_launch<16, true, true>(prm, N, s) : stream_launch<16, true, false>(prm, N, s);
+        else if (has[1]) e = stream_launch<32, true, false>(prm, N, s);
+        else e = stream_launch<64, true, false>(prm, N, s);
         return cuda_ok(e);
     }
-    if (has[0] && e == cudaSuccess) e = stream_launch<16, false>(prm, N, s);
-    if (has[1] && e == cudaSuccess) e = stream_launch<32, false>(prm, N, s);
-    if (has[2] && e == cudaSuccess) e = stream_launch<64, false>(prm, N, s);
+    if (has[0] && e == cudaSuccess)
+        e = short16 ? stream_launch<16, false, true>(prm, N, s) : stream_launch<16, false, false>(prm, N, s);
+    if (has[1] && e == cudaSuccess) e = stream_launch<32, false, false>(prm, N, s);
+    if (has[2] && e == cudaSuccess) e = stream_launch<64, false, false>(prm, N, s);
     return cuda_ok(e);
 }
 

@@ -70,7 +70,7 @@ def test_invalid_arguments_are_refused_before_any_launch():
 
 
 def test_apply_workspace_sizes_and_refusal_without_it(monkeypatch):
-    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH"):
+    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH", "MOLORA_STREAM_TILE"):
         monkeypatch.delenv(k, raising=False)
     lib = M.load_library()
     fake = ctypes.c_void_p(0x1000)
@@ -108,7 +108,7 @@ def _desc(d_in, d_out, rank):
 def test_group_apply_one_call_launch_count_and_refusals(monkeypatch):
     """Host arithmetic only: when molora_group_apply_batched is one launch, and that it validates both halves."""
     from paper_2603_15965_b200.binding import _ProjDescC
-    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH"):
+    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH", "MOLORA_STREAM_TILE"):
         monkeypatch.delenv(k, raising=False)
     lib = M.load_library()
 

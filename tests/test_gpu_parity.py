@@ -22,12 +22,15 @@ KERNEL_MODES = {
     "default": {},
     "tcgen05": {"MOLORA_UMMA_MIN_TOKENS": "1024"},                                  # tcgen05 from 1024 tokens
     "stream": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "stream"},
+    # rank 16 has two tile shapes in the streaming kernel (16 rows x 1024 columns, 32 rows x 512 columns)
+    "stream-short": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "stream", "MOLORA_STREAM_TILE": "16"},
+    "stream-tall": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "stream", "MOLORA_STREAM_TILE": "32"},
     "twophase": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "twophase"},
 }
 
 
 def force_kernel(monkeypatch, mode):
-    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH"):
+    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH", "MOLORA_STREAM_TILE"):
         monkeypatch.delenv(k, raising=False)
     for k, v in KERNEL_MODES[mode].items():
         monkeypatch.setenv(k, v)
@@ -398,7 +401,7 @@ def test_forward_host_matches_oracle(name):
 
 
 # ------------------------------------------------------------------ small-tile kernels: single-launch streaming and two-launch
-@pytest.mark.parametrize("mode", ["stream", "twophase"])
+@pytest.mark.parametrize("mode", ["stream-short", "stream-tall", "twophase"])
 @pytest.mark.parametrize("rank", [16, 32, 64])
 def test_decode_path_segment_size_sweep(rank, mode, monkeypatch):
     force_kernel(monkeypatch, mode)
@@ -416,7 +419,7 @@ def test_decode_path_segment_size_sweep(rank, mode, monkeypatch):
                                                  (90, 3, 2080, 1056, 16),     # ragged last slices (multiples of 32 only)
                                                  (1500, 3, 1056, 2592, 16),   # more tiles than CTAs x items, ragged chunks
                                                  (5000, 4, 512, 512, 32)])    # several items per persistent CTA
-@pytest.mark.parametrize("mode", ["stream", "twophase"])
+@pytest.mark.parametrize("mode", ["stream-short", "stream-tall", "twophase"])
 def test_decode_path_shapes(N, C, d_in, d_out, rank, mode, monkeypatch):
     force_kernel(monkeypatch, mode)
     w = W.random_problem(N + rank + 7, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.1 if N > 10 else 0.0)
@@ -455,7 +458,7 @@ def test_route_gate_tensor_core_paths(N, d, C):
 
 
 # ------------------------------------------------------------------ seeded random shapes across every kernel path
-@pytest.mark.parametrize("mode", ["default", "tcgen05", "stream", "twophase"])
+@pytest.mark.parametrize("mode", ["default", "tcgen05", "stream-short", "stream-tall", "twophase"])
 @pytest.mark.parametrize("seed", range(24))
 def test_random_shapes_all_paths(seed, mode, monkeypatch):
     # token counts on both sides of the path switches (1024 / 1280 tokens), adapter counts on both sides of the
@@ -616,6 +619,7 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode, monk
 # ------------------------------------------------------------------ grouping + apply in one call (one launch where fused)
 @pytest.mark.parametrize("N,C,shapes,mode", [
     (4096, 4, [(2048, 2048, 16)], "default"),                                   # c2's apply: fused, the largest fused size
+    (4096, 4, [(512, 256, 16)], "stream-short"), (700, 9, [(512, 256, 16)], "stream-tall"),   # both rank-16 tile shapes, fused
     (256, 8, [(2048, 2048, 16), (2048, 1024, 16), (6144, 2048, 16)], "default"),  # a decode layer's shapes: fused, 3 projections
     (1, 1, [(32, 32, 16)], "default"), (33, 256, [(64, 96, 16)], "default"),    # one token; more adapters than tokens
     (1500, 5, [(512, 320, 32)], "default"),                                     # rank 32 streaming: fused
