@@ -319,7 +319,7 @@ def run_ours(args):
             a1.record(stream)
             torch.cuda.synchronize()
             apply_ms = a0.elapsed_time(a1) / K
-            kernel_timing = "apply-only graphs over the same buffer rotation, CUDA events around K launches"
+            kernel_timing = "graphs of the dominant kernel's call alone over the same buffer rotation, CUDA events around K launches"
         else:
             ev_every = max(1, K // 2000)                               # bound the number of event pairs
             pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
