@@ -358,12 +358,19 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
             for (int e4 = tid; e4 < Cfg::TFLOATS / 4; e4 += kTpThreads) {
                 float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (e4 * 4 < t.rows * R) {
-                    for (int k = 0; k < KS; ++k) {
-                        const float4 v = __ldcg(reinterpret_cast<const float4*>(part + k * slice_stride + e4 * 4));
-                        s.x += v.x;
-                        s.y += v.y;
-                        s.z += v.z;
-                        s.w += v.w;
+                    for (int k0 = 0; k0 < KS; k0 += 4) {           // four slices in flight at once, summed in slice order
+                        float4 v[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            if (k0 + k < KS) v[k] = __ldcg(reinterpret_cast<const float4*>(part + (k0 + k) * slice_stride + e4 * 4));
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            if (k0 + k < KS) {
+                                s.x += v[k].x;
+                                s.y += v[k].y;
+                                s.z += v[k].z;
+                                s.w += v[k].w;
+                            }
                     }
                 }
                 float sc = scale;                   // times the token's routing weight, if the caller passes per-token factors
