@@ -26,7 +26,8 @@ namespace {
 // kernel (32-row tiles, one CTA per item) and the two-launch small-tile kernels.  Measured on B200 (2048- and
 // 4096-wide projections, 4-128 adapters, 1-7 projections per call):
 //   rank 16  streaming wins until the projections of the call move ~150 MB (x once, y twice), tcgen05 above;
-//   rank 32  two-launch below 1024 tokens (a tie with streaming), streaming until ~60 MB, tcgen05 above;
+//   rank 32  streaming until ~60 MB, tcgen05 above (below 1024 tokens the two-launch pair ties for one projection
+//            and loses by a third for a layer's worth of them);
 //   rank 64  two-launch below 1280 tokens, tcgen05 above (the streaming kernel has only two stages there).
 // MOLORA_UMMA_MIN_TOKENS=n forces "tcgen05 from n tokens" and MOLORA_SMALL_PATH=stream|twophase forces the kernel used
 // below it, for measurements and for tests that target one kernel.
@@ -36,7 +37,7 @@ int64_t forced_umma_min_tokens()
     return e != nullptr && e[0] != '\0' ? std::max<int64_t>(1, std::atoll(e)) : (int64_t)0;
 }
 constexpr double kUmmaMinBytesR16 = 150e6, kUmmaMinBytesR32 = 60e6;
-constexpr int64_t kUmmaMinTokensR64 = 1280, kStreamMinTokensR32 = 1024;
+constexpr int64_t kUmmaMinTokensR64 = 1280;
 
 double proj_bytes(int64_t N, int32_t d_in, int32_t d_out) { return (double)N * ((double)d_in + 2.0 * d_out) * 2.0; }
 
@@ -56,7 +57,8 @@ bool small_path_is_stream(int32_t rank, int64_t N)
         if (e[0] == 's') return true;
         if (e[0] == 't') return false;
     }
-    return rank == 16 || (rank == 32 && N >= kStreamMinTokensR32);
+    (void)N;
+    return rank == 16 || rank == 32;
 }
 
 bool rank_supported(int r) { return r == 8 || r == 16 || r == 32 || r == 64; }

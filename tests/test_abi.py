@@ -75,19 +75,20 @@ def test_apply_workspace_sizes_and_refusal_without_it(monkeypatch):
     lib = M.load_library()
     fake = ctypes.c_void_p(0x1000)
     # only the two-launch small-tile kernels need scratch: fp32 partial shrink results [slice][N][rank].  They serve
-    # rank 32 below 1024 tokens and rank 64 below 1280 tokens:
-    # 256 tokens, d_in 2048, rank 32 -> 4 slices of 512 columns -> 4 * 256 * 32 * 4 bytes
-    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 32) == 4 * 256 * 32 * 4
-    assert M.molora_apply_workspace_bytes(256, 8, 6144, 2048, 32) == 12 * 256 * 32 * 4
+    # rank 64 below 1280 tokens:
+    # 256 tokens, d_in 2048, rank 64 -> 4 slices of 512 columns -> 4 * 256 * 64 * 4 bytes
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 64) == 4 * 256 * 64 * 4
+    assert M.molora_apply_workspace_bytes(256, 8, 6144, 2048, 64) == 12 * 256 * 64 * 4
     assert M.molora_apply_workspace_bytes(1024, 8, 2048, 2048, 64) > 0
-    # rank 16 (streaming or tcgen05 kernel), rank 32 from 1024 tokens, rank 64 from 1280 tokens with few adapters, rank 8
-    # and fp32-only shapes need none
+    # ranks 16 and 32 (streaming or tcgen05 kernel), rank 64 from 1280 tokens with few adapters, rank 8 and fp32-only
+    # shapes need none
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 0
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 32) == 0
     assert M.molora_apply_workspace_bytes(4096, 4, 2048, 2048, 16) == 0
     assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 32) == 0
     assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 64) == 0
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 8) == 0
-    assert M.molora_apply_workspace_bytes(256, 8, 2040, 2048, 32) == 0
+    assert M.molora_apply_workspace_bytes(256, 8, 2040, 2048, 64) == 0
     # with more than 64 adapters the short segments of a large rank-64 call take the two-launch kernels
     assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 64) > 0
     assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 16) == 0
@@ -96,7 +97,7 @@ def test_apply_workspace_sizes_and_refusal_without_it(monkeypatch):
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 2 * 256 * 16 * 4
     monkeypatch.delenv("MOLORA_SMALL_PATH")
     # a call for the two-launch kernels without its workspace is refused before anything is enqueued
-    st = lib.molora_apply(fake, 64, fake, 64, M.BF16, 4, 64, 64, 32, fake, fake, 2, fake, fake, 1.0, None, 0, None, None)
+    st = lib.molora_apply(fake, 64, fake, 64, M.BF16, 4, 64, 64, 64, fake, fake, 2, fake, fake, 1.0, None, 0, None, None)
     assert st == 3
 
 
@@ -119,7 +120,7 @@ def test_group_apply_one_call_launch_count_and_refusals(monkeypatch):
     assert one_launch([(2048, 2048, 16)], 4096) == 1                    # c2's apply
     assert one_launch([(2048, 2048, 16)] * 4 + [(2048, 6144, 16)] * 2 + [(6144, 2048, 16)], 256) == 1   # a decode layer
     assert one_launch([(2048, 2048, 16)], 4097) == 0                    # more tokens than a CTA groups on its own
-    assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 0   # rank 32 streams from 1024 tokens
+    assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 1   # rank 32 streams too
     assert one_launch([(2048, 2048, 64)], 512) == 0                     # rank 64: two-launch kernels / tcgen05
     assert one_launch([(2048, 2048, 16), (2048, 2048, 32)], 2048) == 0  # two ranks: two apply launches
     assert one_launch([(2048, 2048, 16)] * 8, 4096) == 0                # 400 MB: above the tcgen05 crossover
