@@ -176,8 +176,8 @@ molora_status_t molora_group(const int32_t *r, int64_t N, int32_t C, int32_t *co
  * offsets, perm   device outputs of molora_group for the same N, C (read on the device only)
  * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes, 16-byte aligned (NULL if
  *                 that is 0).  Only the two-launch small-tile kernels write it (fp32 partial shrink results
- *                 [slice][N][rank]): bf16 calls of rank 64 below 1280 tokens and, with more than 64 adapters, the
- *                 short segments of larger rank-64 calls.
+ *                 [slice][N][rank]): bf16 calls of rank 64 below 1280 tokens (with one or two rank-64 projections in
+ *                 the call) and, with more than 64 adapters, the short segments of larger rank-64 calls.
  *                 MOLORA_ERR_WORKSPACE if those kernels are needed and ws is NULL, misaligned or too small.
  * dev_status      device uint32 or NULL; MOLORA_DEV_TIMEOUT is OR-ed in if a bounded wait inside a kernel gave
  *                 up (the kernel then returns without hanging; y is incomplete)

@@ -28,7 +28,8 @@ namespace {
 //   rank 16  streaming wins until the projections of the call move ~150 MB (x once, y twice), tcgen05 above;
 //   rank 32  streaming until ~60 MB, tcgen05 above (below 1024 tokens the two-launch pair ties for one projection
 //            and loses by a third for a layer's worth of them);
-//   rank 64  two-launch below 1280 tokens, tcgen05 above (the streaming kernel has only two stages there).
+//   rank 64  below 1280 tokens the two-launch pair for one or two projections and the streaming kernel for more,
+//            tcgen05 above (the streaming kernel has only two stages at this rank).
 // MOLORA_UMMA_MIN_TOKENS=n forces "tcgen05 from n tokens" and MOLORA_SMALL_PATH=stream|twophase forces the kernel used
 // below it, for measurements and for tests that target one kernel.
 int64_t forced_umma_min_tokens()
@@ -50,15 +51,17 @@ bool use_umma(int32_t rank, int64_t N, double group_bytes)
     if (rank == 32) return group_bytes >= kUmmaMinBytesR32;
     return N >= kUmmaMinTokensR64;
 }
-// the kernel for what the tcgen05 kernel does not take
-bool small_path_is_stream(int32_t rank, int64_t N)
+// the kernel for what the tcgen05 kernel does not take; same_rank: projections of this rank in the call (0: unknown)
+bool small_path_is_stream(int32_t rank, int64_t N, int same_rank)
 {
     if (const char* e = std::getenv("MOLORA_SMALL_PATH")) {
         if (e[0] == 's') return true;
         if (e[0] == 't') return false;
     }
     (void)N;
-    return rank == 16 || rank == 32;
+    // rank 64: the two-launch pair for one or two projections (its split of the reduction over CTAs pays there);
+    // with a layer's worth of them its items no longer fit a wave and the streaming kernel is faster
+    return rank == 16 || rank == 32 || same_rank > 2;
 }
 
 bool rank_supported(int r) { return r == 8 || r == 16 || r == 32 || r == 64; }
@@ -173,7 +176,7 @@ size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t 
     // the top of this file.  The element type is not known here, so the figure assumes bf16 (fp32 calls need none).
     if (N <= 0 || d_in <= 0 || d_out <= 0 || (rank != 16 && rank != 32 && rank != 64)) return 0;
     if ((d_in % 32) != 0 || (d_out % 32) != 0) return 0;
-    if (small_path_is_stream(rank, N)) return 0;
+    if (small_path_is_stream(rank, N, 0)) return 0;
     // two-launch kernels: needed unless the tcgen05 kernel is certain to take every segment (for ranks 16 and 32 that
     // depends on the other projections of the call, which are not known here)
     const int64_t forced = forced_umma_min_tokens();
@@ -203,13 +206,16 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
     auto group_of = [](int32_t rank) { return rank == 16 ? 0 : rank == 32 ? 1 : 2; };
     for (int i = 0; i < P; ++i)
         if (umma_eligible(projs[i], dt)) group_bytes[group_of(projs[i].rank)] += proj_bytes(N, projs[i].d_in, projs[i].d_out);
+    int same_rank[3] = {0, 0, 0};                  // projections per rank that a small-tile kernel can take
+    for (int i = 0; i < P; ++i)
+        if (decode_eligible(projs[i], dt)) ++same_rank[group_of(projs[i].rank)];
     molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], sc[MOLORA_MAX_PROJECTIONS], dc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
     int n_tc = 0, n_sc = 0, n_dc = 0, n_cc = 0;
     for (int i = 0; i < P; ++i) {
         const int32_t rank = projs[i].rank;
         if (umma_eligible(projs[i], dt) && use_umma(rank, N, group_bytes[group_of(rank)])) tc[n_tc++] = projs[i];
         else if (decode_eligible(projs[i], dt)) {
-            if (small_path_is_stream(rank, N)) sc[n_sc++] = projs[i];
+            if (small_path_is_stream(rank, N, same_rank[group_of(rank)])) sc[n_sc++] = projs[i];
             else dc[n_dc++] = projs[i];
         } else cc[n_cc++] = projs[i];
     }
@@ -225,7 +231,7 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
             int a = 0, b = 0, c = 0;
             for (int i = 0; i < n_tc; ++i) {
                 if (!decode_eligible(tc[i], dt)) small_cc[c++] = tc[i];
-                else if (small_path_is_stream(tc[i].rank, N)) small_sc[a++] = tc[i];
+                else if (small_path_is_stream(tc[i].rank, N, same_rank[group_of(tc[i].rank)])) small_sc[a++] = tc[i];
                 else small_dc[b++] = tc[i];
             }
             if (a > 0) st = launch_apply_stream(small_sc, a, N, C, offsets, perm, min_rows, dev_status, s);
@@ -245,7 +251,7 @@ static bool group_apply_fuses(const molora_proj_desc_t* projs, int32_t P, molora
     bool fused = dt == MOLORA_BF16 && group_apply_stream_eligible(N);
     double bytes = 0.0;
     for (int i = 0; i < P && fused; ++i) {
-        fused = projs[i].rank == projs[0].rank && decode_eligible(projs[i], dt) && small_path_is_stream(projs[i].rank, N);
+        fused = projs[i].rank == projs[0].rank && decode_eligible(projs[i], dt) && small_path_is_stream(projs[i].rank, N, P);
         if (umma_eligible(projs[i], dt)) bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
     }
     return fused && !use_umma(projs[0].rank, N, bytes);
