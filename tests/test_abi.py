@@ -121,7 +121,9 @@ def test_group_apply_one_call_launch_count_and_refusals(monkeypatch):
     assert one_launch([(2048, 2048, 16)] * 4 + [(2048, 6144, 16)] * 2 + [(6144, 2048, 16)], 256) == 1   # a decode layer
     assert one_launch([(2048, 2048, 16)], 4097) == 0                    # more tokens than a CTA groups on its own
     assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 1   # rank 32 streams too
-    assert one_launch([(2048, 2048, 64)], 512) == 0                     # rank 64: two-launch kernels / tcgen05
+    assert one_launch([(2048, 2048, 64)], 512) == 0                     # rank 64, one projection: two-launch kernels
+    assert one_launch([(2048, 2048, 64)] * 3, 512) == 1                 # rank 64, a layer's projections: streaming kernel
+    assert one_launch([(2048, 2048, 64)] * 3, 2048) == 0                # rank 64 from 1280 tokens: tcgen05
     assert one_launch([(2048, 2048, 16), (2048, 2048, 32)], 2048) == 0  # two ranks: two apply launches
     assert one_launch([(2048, 2048, 16)] * 8, 4096) == 0                # 400 MB: above the tcgen05 crossover
     assert one_launch([(2048, 2048, 16)], 4096, M.F32) == 0             # fp32 storage: CUDA-core kernel

@@ -623,6 +623,7 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode, monk
     (256, 8, [(2048, 2048, 16), (2048, 1024, 16), (6144, 2048, 16)], "default"),  # a decode layer's shapes: fused, 3 projections
     (1, 1, [(32, 32, 16)], "default"), (33, 256, [(64, 96, 16)], "default"),    # one token; more adapters than tokens
     (1500, 5, [(512, 320, 32)], "default"),                                     # rank 32 streaming: fused
+    (300, 4, [(256, 320, 64), (512, 256, 64), (256, 256, 64)], "default"),       # three rank-64 projections: streaming, fused
     (700, 70, [(256, 512, 16)], "default"),                                     # many adapters, match_any grouping
     (4097, 4, [(256, 256, 16)], "default"),                                     # one token too many: two launches
     (600, 3, [(256, 256, 16), (256, 128, 64)], "default"),                      # mixed ranks: two launches
