@@ -237,11 +237,11 @@ def run_ours(args):
     # one that asks for a workspace)
     apply_launches = sum(2 if any(M.molora_apply_workspace_bytes(N, C, p.d_in, p.d_out, p.rank) > 0
                                   for p in w.projections if p.rank == rk) else 1 for rk in {p.rank for p in w.projections})
-    # grouping + apply are one C-ABI call; it is one launch when the library fuses them (every projection on the
-    # streaming kernel), otherwise the grouping launch followed by the apply launches
+    # grouping + apply are one C-ABI call; where the library fuses them (every projection on the streaming kernel or on
+    # the two-launch kernels) the apply kernels group on chip, otherwise the grouping launch precedes the apply launches
     arr0, n0, c0, dt0 = sets[0]["packed"]
-    fused = bool(lib.molora_group_apply_is_one_launch(arr0, len(arr0), dt0, n0))
-    launches_per_step = gate_launches + (1 if fused else 1 + apply_launches)
+    fused = bool(lib.molora_group_apply_skips_group_launch(arr0, len(arr0), dt0, n0))   # grouping inside the apply kernels
+    launches_per_step = gate_launches + (apply_launches if fused else 1 + apply_launches)
     for s in sets:
         s["calls"] = marshal_step(lib, w, s, shared, stream.cuda_stream)
 
@@ -384,7 +384,7 @@ def run_ours(args):
             "gpu_launches": launches_per_step * K,
             "clocks": clk,
             "e2e": e2e,
-            "roofline": {"bound": "hbm", "kernel": ("molora_group_apply_batched (grouping + grouped shrink+expand, one launch)" if fused
+            "roofline": {"bound": "hbm", "kernel": ("molora_group_apply_batched (grouping + grouped shrink+expand, no grouping launch)" if fused
                                                     else "molora_apply (grouped shrink+expand)"), "achieved": achieved,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                          "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES.get(name),

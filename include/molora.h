@@ -217,7 +217,8 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t *projs, int32_t P,
  * calls; ws / ws_bytes as for molora_apply_batched.  When every projection of the call runs on the single-launch
  * streaming kernel with one rank (bf16, at most 4096 tokens, below the tcgen05 crossover) the whole call is ONE
  * launch: every CTA builds the grouping in its shared memory before its first copy request, which saves the
- * grouping launch; otherwise the two launches are enqueued in stream order. */
+ * grouping launch; the two-launch small-tile kernels do the same for at most 1024 tokens; otherwise the grouping
+ * launch and the apply launches are enqueued in stream order. */
 molora_status_t molora_group_apply_batched(const int32_t *r, int64_t N, int32_t C, int32_t *counts, int32_t *offsets,
                                            int32_t *perm, const molora_proj_desc_t *projs, int32_t P,
                                            molora_dtype_t dt, void *ws, size_t ws_bytes, uint32_t *dev_status,
@@ -225,6 +226,9 @@ molora_status_t molora_group_apply_batched(const int32_t *r, int64_t N, int32_t 
 /* 1 if that call is a single launch for these projections (host array, as above) and this token count, else 0;
  * pure host arithmetic, for callers that count launches. */
 int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N);
+/* 1 if that call needs no separate grouping launch: the single launch above, or the two-launch small-tile kernels
+ * grouping on chip (bf16, one rank, at most 1024 tokens; their launches are then the two of molora_apply_batched). */
+int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N);
 
 /* ---------------------------------------------------------------------------------------------
  * Top-k weighted routing (Eq. 8): w_i = softmax(TopK(z_i, k)), delta h_i = sum_j w_ij x_i A^(j) B^(j).

@@ -98,6 +98,8 @@ def load_library():
     lib.molora_group_apply_batched.restype = ctypes.c_int
     lib.molora_group_apply_is_one_launch.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64]
     lib.molora_group_apply_is_one_launch.restype = i32
+    lib.molora_group_apply_skips_group_launch.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64]
+    lib.molora_group_apply_skips_group_launch.restype = i32
     lib.molora_forward_host_arena_bytes.restype = sz
     lib.molora_forward_host_arena_bytes.argtypes = [ctypes.POINTER(_HostProjC), i32, ctypes.c_int, i64, i32, ctypes.c_int,
                                                     i32]

@@ -245,22 +245,38 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
     return st;
 }
 
-// every projection on the streaming kernel, one rank, few enough tokens for the CTA-local grouping
-static bool group_apply_fuses(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
+// How molora_group_apply_batched runs: 1 = one launch (every projection on the streaming kernel, one rank, at most 4096
+// tokens), 2 = the two-launch kernels with the grouping inside (one rank, at most 1024 tokens), 0 = the grouping launch
+// followed by the apply launches.
+static int group_apply_mode(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
 {
-    bool fused = dt == MOLORA_BF16 && group_apply_stream_eligible(N);
+    if (dt != MOLORA_BF16 || N < 1) return 0;
     double bytes = 0.0;
-    for (int i = 0; i < P && fused; ++i) {
-        fused = projs[i].rank == projs[0].rank && decode_eligible(projs[i], dt) && small_path_is_stream(projs[i].rank, N, P);
+    bool same = true, stream = true, twophase = true;
+    for (int i = 0; i < P; ++i) {
+        same = same && projs[i].rank == projs[0].rank && decode_eligible(projs[i], dt);
+        if (!same) return 0;
+        const bool st = small_path_is_stream(projs[i].rank, N, P);
+        stream = stream && st;
+        twophase = twophase && !st;
         if (umma_eligible(projs[i], dt)) bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
     }
-    return fused && !use_umma(projs[0].rank, N, bytes);
+    if (use_umma(projs[0].rank, N, bytes)) return 0;
+    if (stream && group_apply_stream_eligible(N)) return 1;
+    if (twophase && group_apply_decode_eligible(N)) return 2;
+    return 0;
 }
 
 int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
 {
     if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 1) return 0;
-    return group_apply_fuses(projs, P, dt, N) ? 1 : 0;
+    return group_apply_mode(projs, P, dt, N) == 1 ? 1 : 0;
+}
+
+int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
+{
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 1) return 0;
+    return group_apply_mode(projs, P, dt, N) != 0 ? 1 : 0;
 }
 
 molora_status_t molora_group_apply_batched(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets,
@@ -278,10 +294,14 @@ molora_status_t molora_group_apply_batched(const int32_t* r, int64_t N, int32_t 
         const molora_status_t st = check_proj(projs[i], dt);
         if (st != MOLORA_OK) return st;
     }
-    // One launch when every projection of the call runs on the streaming kernel with one rank: its CTAs do the
-    // grouping themselves.  Otherwise the two calls, in stream order.
-    if (group_apply_fuses(projs, P, dt, N))
+    // When every projection of the call runs on the streaming kernel (or on the two-launch kernels) with one rank, the
+    // CTAs of those kernels do the grouping themselves.  Otherwise the two calls, in stream order.
+    const int mode = group_apply_mode(projs, P, dt, N);
+    if (mode == 1)
         return launch_group_apply_stream(r, projs, P, N, C, counts, offsets, perm, dev_status, static_cast<cudaStream_t>(stream));
+    if (mode == 2)
+        return launch_group_apply_decode(r, projs, P, N, C, counts, offsets, perm, ws, ws_bytes, dev_status,
+                                         static_cast<cudaStream_t>(stream));
     const molora_status_t st = molora_group(r, N, C, counts, offsets, perm, nullptr, 0, dev_status, stream);
     if (st != MOLORA_OK) return st;
     return molora_apply_batched(projs, P, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, stream);

@@ -28,6 +28,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "group_inline.cuh"
 #include "pipeline.cuh"
 #include "sm100_ptx.cuh"
 
@@ -39,7 +40,6 @@ constexpr int kFsMaxRows = 32;            // most positions of a tile (two 16-ro
 constexpr int kFsWarps = 8;               // compute warps
 constexpr int kFsCopyWarps = 4;            // each moves 8 rows of the tile and a quarter of the weight rows
 constexpr int kFsThreads = (kFsWarps + kFsCopyWarps) * 32;
-constexpr int kFsGroupSmemMaxC = 32;       // grouping variant: adapters handled by the per-thread count table
 constexpr double kFsShortFill = 1.25;     // rank 16: short tiles while (16-row tiles x projections) <= this x SMs
 constexpr int kFsPermCache = 4096;        // calls with at most this many tokens keep perm in shared memory
 
@@ -189,176 +189,9 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
         fence_mbar_init();
     }
     if constexpr (GROUP) {
-        constexpr int NW = kFsThreads / 32;
-      if (prm.C <= kFsGroupSmemMaxC) {
-        // Up to 32 adapters: every thread owns a contiguous run of tokens and counts it into its own column of a
-        // [adapter][thread] table in shared memory (the ring is idle; consecutive threads hit consecutive banks); a warp
-        // per adapter turns the table into exclusive prefixes over the threads, and every thread then writes its run
-        // out in token order -- stable by construction, no atomics.
-        constexpr int TPT = (kFsPermCache + kFsThreads - 1) / kFsThreads;      // tokens per thread
-        constexpr int LPT = kFsThreads / 32;                                   // table entries per lane in the scan
-        int* cnt_s = reinterpret_cast<int*>(dsm);                              // [C][kFsThreads]
-        int* tot_s = cnt_s + kFsGroupSmemMaxC * kFsThreads;                    // [C] adapter totals
-        const int C = prm.C, N = prm.N;
-        const int per = (N + kFsThreads - 1) / kFsThreads;
-        const int b0 = min(tid * per, N), e0 = min(b0 + per, N);
-        int v[TPT];
-        bool bad = false;
-#pragma unroll
-        for (int j = 0; j < TPT; ++j) {
-            const int raw = b0 + j < e0 ? __ldg(prm.r + b0 + j) : -1;
-            bad |= (raw < -1) || (raw >= C);
-            v[j] = (raw >= 0 && raw < C) ? raw : -1;
-        }
-        for (int c = 0; c < C; ++c) cnt_s[c * kFsThreads + tid] = 0;
-#pragma unroll
-        for (int j = 0; j < TPT; ++j)
-            if (v[j] >= 0) cnt_s[v[j] * kFsThreads + tid] += 1;
-        __syncthreads();
-        for (int c = warp; c < C; c += NW) {           // exclusive prefix over the threads, lane = LPT consecutive threads
-            int* row = cnt_s + c * kFsThreads + lane * LPT;
-            int loc[LPT], sum = 0;
-#pragma unroll
-            for (int k = 0; k < LPT; ++k) {
-                loc[k] = row[k];
-                sum += loc[k];
-            }
-            int incl = sum;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                if (lane >= off) incl += up;
-            }
-            int run = incl - sum;
-#pragma unroll
-            for (int k = 0; k < LPT; ++k) {
-                row[k] = run;
-                run += loc[k];
-            }
-            if (lane == 31) tot_s[c] = incl;
-        }
-        __syncthreads();
-        if (warp == 0) {                               // offsets: exclusive prefix of the totals (C <= 32: one per lane)
-            const int mine = lane < C ? tot_s[lane] : 0;
-            int incl = mine;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                if (lane >= off) incl += up;
-            }
-            if (lane < C) offs_s[lane] = incl - mine;
-            if (lane == C - 1) offs_s[C] = incl;
-            if (blockIdx.x == 0 && lane < C) prm.counts_out[lane] = mine;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int j = 0; j < TPT; ++j)
-            if (v[j] >= 0) {
-                int* slot = cnt_s + v[j] * kFsThreads + tid;
-                const int k = *slot;
-                *slot = k + 1;
-                perm_s[offs_s[v[j]] + k] = b0 + j;
-            }
-        if (blockIdx.x == 0 && prm.dev_status != nullptr && __any_sync(0xFFFFFFFFu, bad) && lane == 0)
-            atomicOr(prm.dev_status, MOLORA_DEV_BAD_ROUTE);
-        __syncthreads();
-        if (blockIdx.x == 0)
-            for (int c = tid; c <= C; c += kFsThreads) prm.offsets_out[c] = offs_s[c];
-      } else {
-        constexpr int STEPS = (kFsPermCache + NW * 32 - 1) / (NW * 32);      // 32-token steps of a warp
-        int(*hist)[MOLORA_MAX_ADAPTERS] = reinterpret_cast<int(*)[MOLORA_MAX_ADAPTERS]>(dsm);   // [warp][adapter]; the ring is idle
-        const int C = prm.C, N = prm.N;
-        const unsigned lt_mask = (1u << lane) - 1u;
-        const int chunk = ((N + NW - 1) / NW + 31) / 32 * 32;                // tokens of a warp: ascending token order
-        const int begin = min(warp * chunk, N), end = min(begin + chunk, N);
-        int vreg[STEPS];
-#pragma unroll
-        for (int j = 0; j < STEPS; ++j) {
-            const int i = begin + j * 32 + lane;
-            vreg[j] = i < end ? __ldg(prm.r + i) : -1;
-        }
-        for (int c = lane; c < C; c += 32) hist[warp][c] = 0;
-        __syncwarp();
-        bool bad = false;
-#pragma unroll
-        for (int j = 0; j < STEPS; ++j) {
-            if (begin + j * 32 < end) {
-                const int v = vreg[j];
-                const bool routed = v >= 0 && v < C;
-                bad |= (v < -1) || (v >= C);
-                const unsigned peers = peers_of(v, routed, C);
-                if (routed && lane == __ffs(peers) - 1) hist[warp][v] += __popc(peers);
-                __syncwarp();
-            }
-        }
-        __syncthreads();
-        // exclusive prefix over the warps, per adapter; the totals are the histogram
-        for (int c = tid; c < C; c += kFsThreads) {
-            int run = 0;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                const int t = hist[w][c];
-                hist[w][c] = run;
-                run += t;
-            }
-            tstart_s[c] = run;                 // counts, until the tile prefix replaces them below
-        }
-        __syncthreads();
-        if (warp == 0) {                       // exclusive prefix over adapters, eight consecutive adapters per lane
-            int local[8], sum = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int c = lane * 8 + j;
-                local[j] = c < C ? tstart_s[c] : 0;
-                sum += local[j];
-            }
-            if (blockIdx.x == 0) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (lane * 8 + j < C) prm.counts_out[lane * 8 + j] = local[j];
-            }
-            int incl = sum;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                if (lane >= off) incl += up;
-            }
-            int run = incl - sum;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int c = lane * 8 + j;
-                if (c <= C) offs_s[c] = run;
-                run += local[j];
-            }
-            if (lane == 31 && C == MOLORA_MAX_ADAPTERS) offs_s[MOLORA_MAX_ADAPTERS] = run;
-        }
-        __syncthreads();
-        // stable scatter into the CTA's copy of perm
-#pragma unroll
-        for (int j = 0; j < STEPS; ++j) {
-            if (begin + j * 32 < end) {
-                const int v = vreg[j];
-                const bool routed = v >= 0 && v < C;
-                const unsigned peers = peers_of(v, routed, C);
-                if (routed) perm_s[offs_s[v] + hist[warp][v] + __popc(peers & lt_mask)] = begin + j * 32 + lane;
-                __syncwarp();
-                if (routed && lane == __ffs(peers) - 1) hist[warp][v] += __popc(peers);
-                __syncwarp();
-            }
-        }
-        if (blockIdx.x == 0) {
-            for (int c = tid; c <= C; c += kFsThreads) prm.offsets_out[c] = offs_s[c];
-            if (prm.dev_status != nullptr && __any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(prm.dev_status, MOLORA_DEV_BAD_ROUTE);
-        }
-        __syncthreads();
-      }
-        {   // my slice of perm
-            const int C = prm.C;
-            const int total = offs_s[C];
-            const int per = (total + (int)gridDim.x - 1) / (int)gridDim.x;
-            const int lo = (int)blockIdx.x * per, hi = min(lo + per, total);
-            for (int i = lo + tid; i < hi; i += kFsThreads) prm.perm_out[i] = perm_s[i];
-        }
+        // the grouping itself, on this CTA, while the ring is idle (its memory is the scratch)
+        group_in_cta<kFsThreads, kFsPermCache>(prm.r, prm.N, prm.C, offs_s, tstart_s, perm_s, dsm, true, prm.counts_out,
+                                               prm.offsets_out, prm.perm_out, prm.dev_status);
     } else {
         // segment table and (small calls) the permutation on chip in one memory round trip
         for (int i = tid; i <= prm.C; i += kFsThreads) offs_s[i] = __ldg(prm.offsets + i);

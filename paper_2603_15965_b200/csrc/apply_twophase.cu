@@ -31,6 +31,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "group_inline.cuh"
 #include "pipeline.cuh"
 #include "sm100_ptx.cuh"
 
@@ -54,6 +55,11 @@ struct TwoPhaseParams {
     const int32_t* perm;
     uint32_t* dev_status;
     int32_t N, P, C, max_rows;                // segments with at least max_rows rows belong to the tcgen05 kernel
+    // grouping variant only: the routing decisions and where counts / offsets / perm are written (as by molora_group)
+    const int32_t* r;
+    int32_t* counts_out;
+    int32_t* offsets_out;
+    int32_t* perm_out;
 #ifdef MOLORA_TRACE
     long long* trace;                         // development builds only: globaltimer stamps per CTA
 #endif
@@ -125,12 +131,23 @@ struct TpCfg {
 
 // Segment table and (for small calls) the permutation on chip in one memory round trip.  Returns the number of
 // tiles of the segments that belong to this path (1 <= rows < max_rows): work items are (tile, unit) pairs.
-__device__ __forceinline__ int tp_load_tables(const TwoPhaseParams& prm, int32_t* offs_s, int32_t* tstart_s, int32_t* perm_s)
+// GROUP: the call starts from the routing decisions r (at most kTpPermCache tokens): every CTA of both kernels runs
+// the grouping itself (group_in_cta) in the staging area, which is idle at this point; the shrink kernel's CTAs also
+// write counts, offsets and perm out.  The expand kernel recomputes rather than reads them, so that it can still
+// request its first item before the shrink kernel has finished.
+template <bool GROUP>
+__device__ __forceinline__ int tp_load_tables(const TwoPhaseParams& prm, int32_t* offs_s, int32_t* tstart_s, int32_t* perm_s,
+                                              unsigned char* scratch, bool write_out)
 {
     const int tid = threadIdx.x;
-    for (int i = tid; i <= prm.C; i += kTpThreads) offs_s[i] = __ldg(prm.offsets + i);
-    if (prm.N <= kTpPermCache)
-        for (int i = tid; i < prm.N; i += kTpThreads) perm_s[i] = __ldg(prm.perm + i);
+    if constexpr (GROUP) {
+        group_in_cta<kTpThreads, kTpPermCache>(prm.r, prm.N, prm.C, offs_s, tstart_s, perm_s, scratch, write_out, prm.counts_out,
+                                               prm.offsets_out, prm.perm_out, prm.dev_status);
+    } else {
+        for (int i = tid; i <= prm.C; i += kTpThreads) offs_s[i] = __ldg(prm.offsets + i);
+        if (prm.N <= kTpPermCache)
+            for (int i = tid; i < prm.N; i += kTpThreads) perm_s[i] = __ldg(prm.perm + i);
+    }
     __syncthreads();
     if (tid < 32) tile_starts(offs_s, prm.C, kTpRows, 1, prm.max_rows, tstart_s);
     __syncthreads();
@@ -153,7 +170,7 @@ __device__ __forceinline__ void tp_drain(uint32_t bar, uint32_t parity)
 }
 
 // ------------------------------------------------------------------------------------------------ shrink
-template <int R>
+template <int R, bool GROUP>
 __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_constant__ TwoPhaseParams prm,
                                                                const __grid_constant__ TpUnits units)
 {
@@ -177,7 +194,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
     TP_GT(0, 0);
     grid_dependency_sync();                        // offsets and perm come from the grouping kernel
     TP_GT(0, 1);
-    const int T = tp_load_tables(prm, offs_s, tstart_s, perm_s);
+    const int T = tp_load_tables<GROUP>(prm, offs_s, tstart_s, perm_s, dsm, true);
     const int nitems = T * units.start[prm.P];
     TP_GT(0, 2);
 
@@ -283,7 +300,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
 }
 
 // ------------------------------------------------------------------------------------------------ expand
-template <int R>
+template <int R, bool GROUP>
 __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_constant__ TwoPhaseParams prm,
                                                                const __grid_constant__ TpUnits units)
 {
@@ -306,7 +323,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
     }
     // Nothing read before the dependency wait below is written by the shrink kernel (see the file header).
     TP_GT(1, 0);
-    const int T = tp_load_tables(prm, offs_s, tstart_s, perm_s);
+    const int T = tp_load_tables<GROUP>(prm, offs_s, tstart_s, perm_s, dsm, false);
     const int nitems = T * units.start[prm.P];
 
     const uint32_t ys = smem_u32(dsm), bs = ys + Cfg::YBYTES;
@@ -480,22 +497,25 @@ size_t decode_workspace_bytes(int64_t N, int32_t d_in, int32_t rank)
     return align256((size_t)shrink_slices(d_in, rank) * (size_t)N * (size_t)rank * sizeof(float));
 }
 
-template <int R>
+template <int R, bool GROUP>
 static cudaError_t twophase_launch(const TwoPhaseParams& prm, int64_t N, cudaStream_t s)
 {
+    static_assert(kGroupInCtaTableMaxC * kTpThreads * 4 + 4 * kGroupInCtaTableMaxC <= TpCfg<R>::SHRINK_SMEM &&
+                      kGroupInCtaTableMaxC * kTpThreads * 4 + 4 * kGroupInCtaTableMaxC <= TpCfg<R>::EXPAND_SMEM,
+                  "the grouping scratch fits the staging areas");
     using Cfg = TpCfg<R>;
     // resident CTAs of each kernel on this device: the size of a wave
     static int wave[2] = {0, 0};
     if (wave[0] == 0) {
-        cudaError_t e = cudaFuncSetAttribute(shrink_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SHRINK_SMEM);
+        cudaError_t e = cudaFuncSetAttribute(shrink_kernel<R, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SHRINK_SMEM);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(expand_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::EXPAND_SMEM);
+            e = cudaFuncSetAttribute(expand_kernel<R, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::EXPAND_SMEM);
         if (e != cudaSuccess) return e;
         int dev = 0, sms = 0, occ_s = 0, occ_e = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, shrink_kernel<R>, kTpThreads, Cfg::SHRINK_SMEM);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_e, expand_kernel<R>, kTpThreads, Cfg::EXPAND_SMEM);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, shrink_kernel<R, GROUP>, kTpThreads, Cfg::SHRINK_SMEM);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_e, expand_kernel<R, GROUP>, kTpThreads, Cfg::EXPAND_SMEM);
         wave[1] = std::max(1, sms * occ_e);
         wave[0] = std::max(1, sms * occ_s);
     }
@@ -511,17 +531,14 @@ static cudaError_t twophase_launch(const TwoPhaseParams& prm, int64_t N, cudaStr
     }
     const unsigned grid_s = (unsigned)std::min<int64_t>(tiles * su.start[prm.P], wave[0]);
     const unsigned grid_e = (unsigned)std::min<int64_t>(tiles * eu.start[prm.P], wave[1]);
-    cudaError_t e = launch_kernel(shrink_kernel<R>, dim3(grid_s), dim3(kTpThreads), Cfg::SHRINK_SMEM, s, 1, false, prm, su);
+    cudaError_t e = launch_kernel(shrink_kernel<R, GROUP>, dim3(grid_s), dim3(kTpThreads), Cfg::SHRINK_SMEM, s, 1, false, prm, su);
     if (e != cudaSuccess) return e;
-    return launch_kernel(expand_kernel<R>, dim3(grid_e), dim3(kTpThreads), Cfg::EXPAND_SMEM, s, 1, true, prm, eu);
+    return launch_kernel(expand_kernel<R, GROUP>, dim3(grid_e), dim3(kTpThreads), Cfg::EXPAND_SMEM, s, 1, true, prm, eu);
 }
 
-molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
-                                    const int32_t* offsets, const int32_t* perm, int32_t max_rows, void* ws,
-                                    size_t ws_bytes, uint32_t* dev_status, cudaStream_t s)
+static molora_status_t decode_enqueue(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C, TwoPhaseParams& prm,
+                                      void* ws, size_t ws_bytes, bool group, cudaStream_t s)
 {
-    if (N == 0 || P == 0) return MOLORA_OK;
-    TwoPhaseParams prm;
     bool has[3] = {false, false, false};
     size_t need = 0;
     for (int i = 0; i < P; ++i) {
@@ -538,21 +555,56 @@ molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, 
     }
     if (ws == nullptr || ws_bytes < need || !aligned16(ws)) return MOLORA_ERR_WORKSPACE;
     prm.tws = static_cast<float*>(ws);
-    prm.offsets = offsets;
-    prm.perm = perm;
-    prm.dev_status = dev_status;
     prm.P = P;
     prm.C = C;
-    prm.max_rows = max_rows;
     prm.N = (int32_t)N;
 #ifdef MOLORA_TRACE
     prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
 #endif
     cudaError_t e = cudaSuccess;
-    if (has[0] && e == cudaSuccess) e = twophase_launch<16>(prm, N, s);
-    if (has[1] && e == cudaSuccess) e = twophase_launch<32>(prm, N, s);
-    if (has[2] && e == cudaSuccess) e = twophase_launch<64>(prm, N, s);
+    if (group) {                                   // one rank only (checked by the caller)
+        if (has[0]) e = twophase_launch<16, true>(prm, N, s);
+        else if (has[1]) e = twophase_launch<32, true>(prm, N, s);
+        else e = twophase_launch<64, true>(prm, N, s);
+        return cuda_ok(e);
+    }
+    if (has[0] && e == cudaSuccess) e = twophase_launch<16, false>(prm, N, s);
+    if (has[1] && e == cudaSuccess) e = twophase_launch<32, false>(prm, N, s);
+    if (has[2] && e == cudaSuccess) e = twophase_launch<64, false>(prm, N, s);
     return cuda_ok(e);
+}
+
+molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
+                                    const int32_t* offsets, const int32_t* perm, int32_t max_rows, void* ws,
+                                    size_t ws_bytes, uint32_t* dev_status, cudaStream_t s)
+{
+    if (N == 0 || P == 0) return MOLORA_OK;
+    TwoPhaseParams prm;
+    prm.offsets = offsets;
+    prm.perm = perm;
+    prm.dev_status = dev_status;
+    prm.max_rows = max_rows;
+    prm.r = nullptr;
+    prm.counts_out = prm.offsets_out = prm.perm_out = nullptr;
+    return decode_enqueue(projs, P, N, C, prm, ws, ws_bytes, false, s);
+}
+
+bool group_apply_decode_eligible(int64_t N) { return N >= 1 && N <= kTpPermCache; }
+
+molora_status_t launch_group_apply_decode(const int32_t* r, const molora_proj_desc_t* projs, int32_t P, int64_t N,
+                                          int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm, void* ws,
+                                          size_t ws_bytes, uint32_t* dev_status, cudaStream_t s)
+{
+    TwoPhaseParams prm;
+    prm.offsets = nullptr;
+    prm.perm = nullptr;
+    prm.dev_status = dev_status;
+    prm.max_rows = INT32_MAX;
+    prm.r = r;
+    prm.counts_out = counts;
+    prm.offsets_out = offsets;
+    prm.perm_out = perm;
+    return decode_enqueue(projs, P, N, C, prm, ws, ws_bytes, true, s);
 }
 
 }  // namespace molora

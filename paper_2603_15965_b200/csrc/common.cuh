@@ -273,6 +273,12 @@ bool group_apply_stream_eligible(int64_t N);
 molora_status_t launch_group_apply_stream(const int32_t* r, const molora_proj_desc_t* projs, int32_t P, int64_t N,
                                           int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
                                           uint32_t* dev_status, cudaStream_t s);
+// The two-launch kernels started from r: both kernels group on chip, the first also writes counts / offsets / perm;
+// one rank, at most 1024 tokens.  Saves the grouping launch.
+bool group_apply_decode_eligible(int64_t N);
+molora_status_t launch_group_apply_decode(const int32_t* r, const molora_proj_desc_t* projs, int32_t P, int64_t N,
+                                          int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm, void* ws,
+                                          size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
 size_t decode_workspace_bytes(int64_t N, int32_t d_in, int32_t rank);
 molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                     const int32_t* offsets, const int32_t* perm, int32_t max_rows, void* ws,

@@ -122,6 +122,9 @@ def test_group_apply_one_call_launch_count_and_refusals(monkeypatch):
     assert one_launch([(2048, 2048, 16)], 4097) == 0                    # more tokens than a CTA groups on its own
     assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 1   # rank 32 streams too
     assert one_launch([(2048, 2048, 64)], 512) == 0                     # rank 64, one projection: two-launch kernels
+    arr64 = (_ProjDescC * 1)(_desc(2048, 2048, 64))
+    assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 512)) == 1    # ... which group on chip
+    assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 1100)) == 0   # more than 1024 tokens: they do not
     assert one_launch([(2048, 2048, 64)] * 3, 512) == 1                 # rank 64, a layer's projections: streaming kernel
     assert one_launch([(2048, 2048, 64)] * 3, 2048) == 0                # rank 64 from 1280 tokens: tcgen05
     assert one_launch([(2048, 2048, 16), (2048, 2048, 32)], 2048) == 0  # two ranks: two apply launches

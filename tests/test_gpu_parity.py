@@ -628,7 +628,10 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode, monk
     (4097, 4, [(256, 256, 16)], "default"),                                     # one token too many: two launches
     (600, 3, [(256, 256, 16), (256, 128, 64)], "default"),                      # mixed ranks: two launches
     (300, 4, [(128, 192, 8)], "default"),                                       # CUDA-core apply: two launches
-    (900, 6, [(512, 512, 16)], "twophase"),                                     # two-launch apply forced: group + 2
+    (900, 6, [(512, 512, 16)], "twophase"),                                     # two-launch kernels forced: they group on chip
+    (1024, 40, [(256, 192, 32)], "twophase"),                                   # ... their largest size, match_any grouping
+    (1025, 4, [(256, 192, 32)], "twophase"),                                    # one token too many: grouping launch + 2
+    (300, 7, [(4096, 512, 64)], "default"), (77, 3, [(512, 4096, 64), (512, 512, 64)], "default"),   # rank 64: two-launch, on chip
 ])
 def test_group_apply_one_call_matches_oracle_and_group(N, C, shapes, mode, monkeypatch):
     force_kernel(monkeypatch, mode)
