@@ -6,19 +6,24 @@
 // and stores it back.  Nothing is exchanged between CTAs, there is no workspace and no second launch; a projection
 // wider than one item re-computes the (cheap, L2-served) shrink per output slice.
 //
-//   warp 8 (copy warp)   walks the list of chunk jobs of the CTA's items in order -- shrink chunks (512 columns of
+//   warps 8-11 (copy)    walk the list of chunk jobs of the CTA's items in order -- shrink chunks (512 columns of
 //                        the x rows + the matching rows of A_c), then expand chunks (512 columns of the y rows +
-//                        B_c) -- and keeps the ring full with bulk asynchronous copies, one request per row,
-//                        completion counted in bytes on the stage's "full" mbarrier.  Before it refills a stage it
-//                        waits for the stage's "done" mbarrier and, if the job in it was an expand chunk, issues the
-//                        bulk stores of the updated y rows and waits until they have been read out.  Because the job
-//                        list runs across items, the x rows of the next item are in flight while this one expands.
+//                        B_c) -- and keep the ring full with bulk asynchronous copies, one request per row (each warp
+//                        a quarter of the rows and of the weight rows; the SM accepts a request every ~25 cycles and
+//                        a warp's lanes issue theirs one after the other), completion counted in bytes on the
+//                        stage's "full" mbarrier.  Before a warp refills a stage it waits for the stage's "done"
+//                        mbarrier and, if the job in it was an expand chunk, issues the bulk stores of its updated
+//                        y rows and waits until they have been read out.  Because the job list runs across items,
+//                        the x rows of the next item are in flight while this one expands.
 //   warps 0-7 (compute)  shrink chunk: interleaved 32-wide k blocks, ldmatrix + mma.sync.m16n8k16, fp32 partial
 //                        t per warp in registers.  After the last shrink chunk the partials are summed in warp order
 //                        through that stage's memory (it has been consumed), scaled (and multiplied by the
 //                        token's routing weight, if given) and split into bf16 hi + lo A-fragments.
 //                        expand chunk: interleaved 32-column groups, y += t B_c in shared memory (fp32 add, one
 //                        rounding), then the warp arrives on "done".
+//
+// Variants: GROUP starts from the routing decisions r and groups on chip (group_inline.cuh) instead of loading offsets
+// and perm; SHORT (rank 16) uses 16-row tiles and 1024-column chunks for small calls.
 //
 // mma.sync is the legacy tensor path on sm_100a; a 32-row tile is far below the 128-row tcgen05 tile, and this path
 // is bound by the bytes it moves, not by its flops.  Every wait is bounded; after a time-out the CTA stops issuing
