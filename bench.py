@@ -241,7 +241,8 @@ def run_ours(args):
     # the two-launch kernels) the apply kernels group on chip, otherwise the grouping launch precedes the apply launches
     arr0, n0, c0, dt0 = sets[0]["packed"]
     fused = bool(lib.molora_group_apply_skips_group_launch(arr0, len(arr0), dt0, n0))   # grouping inside the apply kernels
-    launches_per_step = gate_launches + (apply_launches if fused else 1 + apply_launches)
+    one_launch = bool(lib.molora_group_apply_is_one_launch(arr0, len(arr0), dt0, n0))
+    launches_per_step = gate_launches + (1 if one_launch else apply_launches if fused else 1 + apply_launches)
     for s in sets:
         s["calls"] = marshal_step(lib, w, s, shared, stream.cuda_stream)
 
