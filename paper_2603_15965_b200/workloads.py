@@ -12,7 +12,7 @@ Conventions
   bf16-representable numbers; :func:`bf16_bits` gives the 16-bit patterns to upload.
 * ``N(0, v)`` in the workload descriptions is read with ``v`` the **variance**:
   sigma_A = d_in**-0.5, sigma_W = sigma_G = d**-0.5, sigma_B = 0.1.
-* Generator: configuration ``cfg`` owns ``SeedSequence(260315965).spawn(5)[cfg]``; its child stream 0 draws
+* Generator: configuration ``cfg`` owns ``SeedSequence(260315965).spawn(9)[cfg]``; its child stream 0 draws
   the routing source and the weights (ids / r, A, B per projection, G, in that order) and child stream
   ``1 + b`` draws activation batch ``b`` (x*, then y* / W), so weights do not depend on the token count.
 """
