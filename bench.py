@@ -1,11 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the routed-LoRA hot path (route -> group -> apply) on B200.
 
-One "step" is one pass of the whole path over one batch of synthetic input.  The default workload is
-the Qwen3-1.7B-shaped prefill configuration (N = 4096 tokens, q_proj 2048 -> 2048, bf16, C = 4 adapters
-of rank 16, fp32 linear gate with top-1 argmax).  Prints ONE JSON line (rank 0).
+One "step" is one pass of the whole path over one batch of synthetic input.  With no --workload the headline is the
+largest single-GPU configuration, the Qwen3-8B-shaped prefill layer c4 (N = 8192 tokens, seven projections, bf16,
+C = 16 adapters of rank 64, fp32 linear gate with top-1 argmax), and the same JSON line carries, under "configs",
+the step time, dominant-kernel time, algorithmic bytes and roofline fraction of the other configurations
+(c2, c3, c5, c5-iid; the two c5 records also time the K = 4-pass per-sequence baseline).  Prints ONE JSON line (rank 0).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5|c5-iid] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5|c5-iid|f9-*|t9-*|t6-*] [--impl ours|reference]
+
+Timing does not depend on K: the K steps are captured into CUDA graphs over a rotation of buffer sets larger than
+L2, and that K-step pass is replayed until the timed leg has lasted at least --min-leg-s seconds (0.3 by default);
+every pass has its own CUDA-event pair and the reported step time is the median pass time / K.
 
 N > 1 is launched with torch.distributed.run, one rank per GPU; every rank processes its own batches
 (tokens are independent, Eq. 2: no collective on the data path; weak scaling) and the step time is
@@ -29,8 +35,16 @@ if ROOT not in sys.path:
 METRIC = "routed_lora_tokens_per_s"
 UNIT = "tokens/s"
 L2_BYTES = 126e6
-# dram__bytes_read.sum + dram__bytes_write.sum per apply launch from the committed ncu capture (profiles/), by workload
-NCU_TRAFFIC_BYTES = {"c2": 34.17e6, "c3": 26.81e6, "c5": 615.3e6}
+HBM_SPEC_GBS = 8000.0          # the nominal figure the targets are stated against; the measured copy rate is the peak
+HEADLINE = "c4"
+SUB_CONFIGS = ("c2", "c3", "c5", "c5-iid")
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
+# under profiles/ (file named per entry); None where no capture of that workload is committed
+NCU_TRAFFIC = {
+    "c2": (34.17e6, "profiles/apply_stream_c2_full.md"),
+    "c3": (26.81e6, "profiles/apply_stream_c3_full.md"),
+    "c5": (615.3e6, "profiles/apply_umma_c5_full.md"),
+}
 
 
 def measured_peaks():
@@ -44,6 +58,16 @@ def measured_peaks():
 
 
 # ----------------------------------------------------------------------------- workload description
+FULL_TOKENS = {"c2": 4096, "c3": 256, "c4": 8192, "c5": 16384, "c5-iid": 16384}
+
+
+def workload_label(name, w):
+    """The same description of a workload for both arms (the reference arm runs a bounded sample of it)."""
+    n = FULL_TOKENS.get(name, w.N)
+    return f"{name}: N={n} tokens/GPU, C={w.C}, " + ", ".join(
+        f"{p.name} {p.d_in}->{p.d_out} r{p.rank}" for p in w.projections) + f", router={w.router}"
+
+
 def workload_info(w):
     """Algorithmic bytes / flops of one step's apply launch(es): x once + y read and written + the A_c, B_c
     of every adapter + perm/offsets; 2*N*rank*(d_in + d_out) flop (N token-adapter products, Theorem 3.6)."""
@@ -57,7 +81,7 @@ def workload_info(w):
 
 
 class Clocks(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
     def __init__(self, index: int, period_s: float = 0.01):
         super().__init__(daemon=True)
@@ -147,7 +171,7 @@ def build_sets(W, torch, name, n_sets, rank):
 
 
 def marshal_step(lib, w, s, shared, stream_handle):
-    """The step's three C-ABI calls as closures over already converted ctypes arguments (marshalling only)."""
+    """The step's C-ABI calls as closures over already converted ctypes arguments (marshalling only)."""
     import ctypes
     from functools import partial
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
@@ -183,36 +207,37 @@ def marshal_step(lib, w, s, shared, stream_handle):
     return route, group, apply, group_apply
 
 
-def run_ours(args):
-    import torch
-    import paper_2603_15965_b200 as M
-    import paper_2603_15965_b200.binding  # noqa: F401
-    from paper_2603_15965_b200 import shard
-    from paper_2603_15965_b200 import workloads as W
-    from paper_2603_15965_b200.binding import pack_proj_descs
-    from paper_2603_15965_b200.build import build_library
+def timed_passes(torch, stream, run_pass, min_leg_s, max_passes=100000):
+    """Replay `run_pass(i)` (which enqueues one K-step pass on `stream`) until the leg has lasted min_leg_s seconds of
+    device time; one event pair per pass.  Returns the per-pass times in ms."""
+    def batch(first, n):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for j, (a, b) in enumerate(evs):
+            a.record(stream)
+            run_pass(first + j)
+            b.record(stream)
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs]
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the routed-LoRA path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    if rank == 0:
-        build_library()
-    if dist is not None:
-        dist.barrier()
-    lib = M.load_library()
+    times = batch(0, 2)
+    while sum(times) < min_leg_s * 1e3 and len(times) < max_passes:
+        per = max(1e-4, float(np.median(times)))
+        todo = int(min(max_passes - len(times), max(1, np.ceil((min_leg_s * 1e3 - sum(times)) / per * 1.05)), 4096))
+        times += batch(len(times), todo)
+    return times
 
-    name = args.workload
+
+def measure(name, args, env, headline):
+    """Builds the buffer sets of workload `name`, runs warm-up, the timed step leg, the dominant-kernel leg and (c5) the
+    K-pass baseline leg; returns the record of the workload."""
+    torch, M, lib, W, shard, dist = env["torch"], env["M"], env["lib"], env["W"], env["shard"], env["dist"]
+    rank, world, local = env["rank"], env["world"], env["local"]
+    from paper_2603_15965_b200.binding import molora_apply_batched_workspace_bytes, pack_proj_descs
+
     probe = W.get(name) if name != "c2" else W.get("c2", batch=0)
     step_bytes, step_flops = workload_info(probe)
-    per_set = sum(v.nbytes // (2 if probe.dtype == "bf16" else 1) for v in probe.inputs.values()) + \
-        sum(p.y.nbytes // (2 if probe.dtype == "bf16" else 1) for p in probe.projections)
+    esz = 2 if probe.dtype == "bf16" else 1
+    per_set = sum(v.nbytes // esz for v in probe.inputs.values()) + sum(p.y.nbytes // esz for p in probe.projections)
     n_sets = max(2, int(np.ceil(2.5 * L2_BYTES / per_set)))          # rotation working set >= 2.5 x L2
     n_sets = min(n_sets, args.max_sets)
     del probe
@@ -221,122 +246,119 @@ def run_ours(args):
     stream = torch.cuda.Stream()      # every call of the timed region is enqueued (or captured) on this stream
 
     # per-set routing/grouping outputs (fixed addresses, as a serving stack would keep them)
-    for s in sets:
+    for i, s in enumerate(sets):
+        s["idx"] = i
         s["r"] = torch.empty(N, dtype=torch.int32, device="cuda")
         s["counts"] = torch.empty(C, dtype=torch.int32, device="cuda")
         s["offsets"] = torch.empty(C + 1, dtype=torch.int32, device="cuda")
         s["perm"] = torch.empty(N, dtype=torch.int32, device="cuda")
         s["packed"] = pack_proj_descs([M.ProjDesc(s["x"][p.x_key], y, A, B, 1.0) for p, y, A, B in
-                                                 zip(w.projections, s["y"], s["A"], s["B"])])
-    gate_launches = 0 if w.router == "given" else (2 if (w.router == "gate" and shared["gate_ws"] is not None) else 1)
-    # scratch of the apply (partial shrink results of the two-launch small-tile path); one buffer serves every set
-    from paper_2603_15965_b200.binding import molora_apply_batched_workspace_bytes
+                                       zip(w.projections, s["y"], s["A"], s["B"])])
+    # scratch of the apply; one buffer serves every set (zero-filled: the kernels that keep counters there expect that
+    # on first use and leave it so)
     need = molora_apply_batched_workspace_bytes(sets[0]["packed"][0], N, C)
-    shared["apply_ws"] = torch.empty(need, dtype=torch.uint8, device="cuda") if need else None
-    # launches of the apply: one per rank on the tensor-core path, shrink + expand on the small-tile path (which is the
-    # one that asks for a workspace)
-    apply_launches = sum(2 if any(M.molora_apply_workspace_bytes(N, C, p.d_in, p.d_out, p.rank) > 0
-                                  for p in w.projections if p.rank == rk) else 1 for rk in {p.rank for p in w.projections})
-    # grouping + apply are one C-ABI call; where the library fuses them (every projection on the streaming kernel or on
-    # the two-launch kernels) the apply kernels group on chip, otherwise the grouping launch precedes the apply launches
+    shared["apply_ws"] = torch.zeros(need, dtype=torch.uint8, device="cuda") if need else None
     arr0, n0, c0, dt0 = sets[0]["packed"]
     fused = bool(lib.molora_group_apply_skips_group_launch(arr0, len(arr0), dt0, n0))   # grouping inside the apply kernels
-    one_launch = bool(lib.molora_group_apply_is_one_launch(arr0, len(arr0), dt0, n0))
-    launches_per_step = gate_launches + (1 if one_launch else apply_launches if fused else 1 + apply_launches)
     for s in sets:
         s["calls"] = marshal_step(lib, w, s, shared, stream.cuda_stream)
 
-    def step(s, ev=None):
+    def step(s):
         """route -> group + apply on buffer set s: two C-ABI calls with pre-marshalled arguments."""
         route, group, apply, group_apply = s["calls"]
         if route is not None and route() != 0:
             raise RuntimeError("molora_route_* refused the call")
-        if fused or ev is None:
-            if ev is not None:
-                ev[0].record(stream)
-            if group_apply() != 0:
-                raise RuntimeError("molora_group_apply_batched refused the call")
-        else:
-            # eager timing of a call the library does not fuse: the same two calls it makes, taken apart so that the
-            # apply kernels can be bracketed by events
-            if group() != 0:
-                raise RuntimeError("molora_group refused the call")
-            if ev is not None:
-                ev[0].record(stream)
-            if apply() != 0:
-                raise RuntimeError("molora_apply_batched refused the call")
-        if ev is not None:
-            ev[1].record(stream)
+        if group_apply() != 0:
+            raise RuntimeError("molora_group_apply_batched refused the call")
 
-    # ------------------------------------------------------------------ warm-up, then the timed region
+    def checked(call):
+        def f(s_):
+            if call(s_) != 0:
+                raise RuntimeError("a molora_* call was refused")
+        return f
+
     K = args.steps
     W0 = max(3, args.warmup)
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rec = {}
+    kcall = 3 if fused else 2          # the dominant kernel: grouping + apply in one call, or the apply
     with torch.cuda.stream(stream):
+        # launches of a step and of the dominant kernel's call, counted by the library while the warm-up steps run
+        n0 = M.molora_launch_count()
+        step(sets[0])
+        launches_per_step = M.molora_launch_count() - n0
+        n0 = M.molora_launch_count()
+        if sets[0]["calls"][kcall]() != 0:
+            raise RuntimeError("the dominant kernel's call was refused")
+        kernel_launches = M.molora_launch_count() - n0
         for i in range(W0):
             step(sets[i % n_sets])
         torch.cuda.synchronize()
-        if args.launch == "graph":
-            # The paper replays this path from a CUDA graph (fixed addresses, no host work between kernels); so does
-            # the bench: K steps are captured in chunks and replayed, which removes the Python/driver launch cost
-            # from a step that lasts tens of microseconds.  A second set of graphs holds only the apply calls over
-            # the same buffer rotation; its replay time / K is the kernel time used for the roofline.
-            CH = min(K, 512)
+        CH = min(K, 512)
 
-            def capture(fn, first, n):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=stream):
-                    for k in range(first, first + n):
-                        fn(sets[k % n_sets])
-                return g
+        def capture(fn, first, n):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for k in range(first, first + n):
+                    fn(sets[k % n_sets])
+            return g
 
+        def capture_pass(fn, first):
+            """Graphs that together hold K consecutive steps of the rotation starting at step `first`."""
             reps, rem = divmod(K, CH)
-            g_full, g_rem = capture(step, W0, CH), (capture(step, W0 + reps * CH, rem) if rem else None)
-            kcall = 3 if fused else 2          # the dominant kernel: grouping + apply in one launch, or the apply
-            a_full = capture(lambda s_: s_["calls"][kcall](), W0, CH)
-            a_rem = capture(lambda s_: s_["calls"][kcall](), W0 + reps * CH, rem) if rem else None
-            g_full.replay()
+            gs = [capture(fn, first, CH)] * reps          # the chunk graph is replayed `reps` times
+            if rem:
+                gs.append(capture(fn, first + reps * CH, rem))
+            return gs
+
+        # variants of the pass that start at different points of the rotation, so that a pass shorter than the
+        # rotation still sees every buffer set cold
+        n_var = 1 if args.launch == "eager" else max(1, min(8, int(np.ceil(n_sets / K))))
+        if args.launch == "graph":
+            step_graphs = [capture_pass(step, W0 + v * K) for v in range(n_var)]
+            kern_graphs = [capture_pass(checked(lambda s_: s_["calls"][kcall]()), W0 + v * K) for v in range(n_var)]
+            for gs in step_graphs:
+                for g in gs:
+                    g.replay()
             torch.cuda.synchronize()
+
+            def step_pass(i):
+                for g in step_graphs[i % n_var]:
+                    g.replay()
+
+            def kern_pass(i):
+                for g in kern_graphs[i % n_var]:
+                    g.replay()
+            kernel_timing = ("graphs of the dominant kernel's call alone over the same buffer rotation; CUDA events around "
+                             "each K-launch pass, median pass / K")
+        else:
+            def step_pass(i):
+                for k in range(K):
+                    step(sets[(W0 + i * K + k) % n_sets])
+
+            def kern_pass(i):
+                for k in range(K):
+                    sets[(W0 + i * K + k) % n_sets]["calls"][kcall]()
+            kernel_timing = "eager launches of the dominant kernel's call; CUDA events around each K-launch pass (includes host launch gaps)"
+
         clocks = Clocks(local)
         clocks.start()
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
-        if args.launch == "graph":
-            t0.record(stream)
-            for _ in range(reps):
-                g_full.replay()
-            if g_rem is not None:
-                g_rem.replay()
-            t1.record(stream)
-            torch.cuda.synchronize()
-            total_ms = t0.elapsed_time(t1)
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a0.record(stream)
-            for _ in range(reps):
-                a_full.replay()
-            if a_rem is not None:
-                a_rem.replay()
-            a1.record(stream)
-            torch.cuda.synchronize()
-            apply_ms = a0.elapsed_time(a1) / K
-            kernel_timing = "graphs of the dominant kernel's call alone over the same buffer rotation, CUDA events around K launches"
-        else:
-            ev_every = max(1, K // 2000)                               # bound the number of event pairs
-            pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                     if k % ev_every == 0 else None for k in range(K)]
-            t0.record(stream)
-            for k in range(K):
-                step(sets[(W0 + k) % n_sets], pairs[k])
-            t1.record(stream)
-            torch.cuda.synchronize()
-            total_ms = t0.elapsed_time(t1)
-            apply_ms = float(np.mean([a.elapsed_time(b) for p in pairs if p is not None for a, b in [p]]))
-            kernel_timing = "CUDA event pair around every apply call (includes host launch gaps)"
+        step_times = timed_passes(torch, stream, step_pass, args.min_leg_s)
+        if dist is not None:
+            dist.barrier()
+        kern_times = timed_passes(torch, stream, kern_pass, args.min_leg_s)
+        clk = clocks.stop()
+        ms_per_step = shard.max_over_ranks(float(np.median(step_times)) / K, dist, device="cuda")   # slowest rank
+        apply_ms = float(np.median(kern_times)) / K
+        rec["passes"] = {"step": len(step_times), "kernel": len(kern_times),
+                         "timed_region_s": (sum(step_times) + sum(kern_times)) * 1e-3, "pass_variants": n_var}
+
         # latency of a single step replayed on its own (one graph per buffer set, one event pair per replay): the
         # distribution the paper reports for graph replay (median, P99, coefficient of variation)
         latency = None
-        if args.launch == "graph" and not args.profile:
+        if args.launch == "graph" and not args.profile and headline:
             singles = [capture(step, i, 1) for i in range(min(n_sets, 8))]
             n_lat = 400
             evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
@@ -352,50 +374,99 @@ def run_ours(args):
             latency = {"p50_us": float(lat[len(lat) // 2]), "p99_us": float(lat[int(len(lat) * 0.99) - 1]),
                        "cv": float(lat.std() / lat.mean()), "samples": n_lat,
                        "note": "one step per CUDA-graph replay, event pair around each replay (includes the graph launch)"}
-        if dist is not None:
-            dist.barrier()
-        # keep the GPU busy a little longer (untimed) if the region was too short for the clock sampler
-        t_end = time.time() + (0.25 if total_ms < 250 else 0.0)
-        while time.time() < t_end:
-            step(sets[0])
+
+        kpass = None
+        if name.startswith("c5") and not args.profile and args.launch == "graph":
+            kpass = run_kpass(args, env, w, sets, shared, stream, capture_pass, apply_ms, K, n_var)
         torch.cuda.synchronize()
-    clk = clocks.stop()
 
-    total_ms = shard.max_over_ranks(total_ms, dist, device="cuda")     # the slowest rank defines the step
-    ms_per_step = total_ms / K
-    value = shard.aggregate_tokens_per_s(N, world, ms_per_step)
+    peaks = measured_peaks()
+    achieved = step_bytes / (apply_ms * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC.get(name)
+    rec.update({
+        "workload": workload_label(name, w),
+        "tokens_per_step_per_gpu": N, "buffer_sets": n_sets,
+        "l2": f"rotation over {n_sets} buffer sets ({n_sets * per_set / 1e6:.0f} MB > 126 MB L2)",
+        "value": shard.aggregate_tokens_per_s(N, world, ms_per_step), "ms_per_step": ms_per_step,
+        "launches_per_step": launches_per_step, "latency": latency, "clocks": clk, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+        "roofline": {"bound": "hbm",
+                     "kernel": ("molora_group_apply_batched (grouping + grouped shrink+expand, no grouping launch)" if fused
+                                else "molora_apply_batched (grouped shrink+expand)"),
+                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                     "peak_source": peaks["source"], "frac_of_spec": achieved / HBM_SPEC_GBS, "spec_gbs": HBM_SPEC_GBS,
+                     "traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None,
+                     "algorithmic_bytes": step_bytes, "kernel_ms": apply_ms, "kernel_launches": kernel_launches,
+                     "kernel_timing": kernel_timing, "algorithmic_tflops": step_flops / (apply_ms * 1e-3) / 1e12},
+    })
+    if kpass is not None:
+        rec["kpass_baseline"] = kpass
+    rec["e2e"] = None
+    if headline and not args.profile:
+        rec["e2e"] = run_e2e(args, torch, M, w, sets, shared, world, dist)
+    del sets, shared
+    torch.cuda.empty_cache()
+    return rec
 
-    # ------------------------------------------------------------------ end to end with host buffers
-    e2e = None if args.profile else run_e2e(args, torch, M, w, sets, shared, world, dist)
 
-    out = None
-    if rank == 0:
-        peaks = measured_peaks()
-        achieved = step_bytes / (apply_ms * 1e-3) / 1e9
-        out = {
-            "metric": METRIC, "value": value, "unit": UNIT, "latency": latency, "n_gpus": world, "steps": K, "warmup": args.warmup,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": f"{name}: N={N} tokens/GPU, C={C}, " + ", ".join(
-                f"{p.name} {p.d_in}->{p.d_out} r{p.rank}" for p in w.projections) + f", router={w.router}",
-                "tokens_per_step_per_gpu": N, "buffer_sets": n_sets,
-                "l2": f"rotation over {n_sets} buffer sets ({n_sets * per_set / 1e6:.0f} MB > 126 MB L2)",
-                "launch": ("CUDA graph replay of the C-ABI calls (route, then group + apply)" if args.launch == "graph"
-                           else "eager, one C-ABI call per stage")},
-            "gpu_launches": launches_per_step * K,
-            "clocks": clk,
-            "e2e": e2e,
-            "roofline": {"bound": "hbm", "kernel": ("molora_group_apply_batched (grouping + grouped shrink+expand, no grouping launch)" if fused
-                                                    else "molora_apply (grouped shrink+expand)"), "achieved": achieved,
-                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                         "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES.get(name),
-                         "algorithmic_bytes": step_bytes, "kernel_ms": apply_ms, "kernel_timing": kernel_timing,
-                         "algorithmic_tflops": step_flops / (apply_ms * 1e-3) / 1e12},
-            "cpu_baseline": None if args.profile else cpu_baseline(name),
-        }
-    if dist is not None:
-        dist.destroy_process_group()
-    return out
+def run_kpass(args, env, w, sets, shared, stream, capture_pass, single_ms, K, n_var):
+    """The per-sequence baseline on the same kernels (Theorem 3.6): K_ad = C passes, pass k applies adapter k to ALL N
+    tokens into its own copy of y (constant routing: offsets / perm are prepared once, no grouping inside the timed
+    region), then one row select keeps, for every token, the row of the pass of its own adapter.  Timed like the step."""
+    torch, lib = env["torch"], env["lib"]
+    import ctypes
+    from functools import partial
+    import paper_2603_15965_b200 as M
+    from paper_2603_15965_b200.binding import pack_proj_descs
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    N, C = w.N, w.C
+    ident = torch.arange(N, dtype=torch.int32, device="cuda")
+    offs = []
+    for k in range(C):
+        o = torch.zeros(C + 1, dtype=torch.int32, device="cuda")
+        o[k + 1:] = N
+        offs.append(o)
+    aws = shared.get("apply_ws")
+    st = vp(stream.cuda_stream)
+    # two scratch sets (> 2.5 x L2 together): [C, N, d_out] per projection, pre-filled with y = xW
+    kp_sets = []
+    for s in sets[:2]:
+        stacks = [y.unsqueeze(0).repeat(C, 1, 1).contiguous() for y in s["y"]]
+        outs = [torch.empty_like(y) for y in s["y"]]
+        calls = []
+        for k in range(C):
+            packed = pack_proj_descs([M.ProjDesc(s["x"][p.x_key], stk[k], A, B, 1.0) for p, stk, A, B in
+                                      zip(w.projections, stacks, s["A"], s["B"])])
+            arr, n, c, dt = packed
+            calls.append((packed, partial(lib.molora_apply_batched, arr, i32(len(arr)), dt, i64(n), i32(c),
+                                          vp(offs[k].data_ptr()), vp(ident.data_ptr()),
+                                          vp(aws.data_ptr()) if aws is not None else None,
+                                          ctypes.c_size_t(aws.numel() if aws is not None else 0),
+                                          vp(shared["status"].data_ptr()), st)))
+        rsel = s["r" if w.router != "given" else "r_given"].to(torch.int64).clamp_(min=0) * N + torch.arange(N, device="cuda")
+        kp_sets.append({"stacks": stacks, "outs": outs, "calls": calls, "rsel": rsel})
+
+    def kpass_step(s):
+        ks = kp_sets[s["idx"] % len(kp_sets)]
+        rsel = ks["rsel"]
+        for _, call in ks["calls"]:
+            if call() != 0:
+                raise RuntimeError("molora_apply_batched refused a pass of the K-pass baseline")
+        for stk, out in zip(ks["stacks"], ks["outs"]):
+            torch.index_select(stk.view(C * N, -1), 0, rsel, out=out)
+
+    graphs = [capture_pass(kpass_step, v * K) for v in range(n_var)]
+
+    def kp_pass(i):
+        for g in graphs[i % n_var]:
+            g.replay()
+    kp_pass(0)
+    torch.cuda.synchronize()
+    times = timed_passes(torch, stream, kp_pass, args.min_leg_s)
+    kp_ms = float(np.median(times)) / K
+    return {"K": C, "kpass_ms": kp_ms, "single_pass_ms": single_ms, "ratio": kp_ms / single_ms,
+            "token_adapter_products": {"single_pass": N, "kpass": C * N},
+            "note": "K applies with constant routing over all N tokens into K copies of y + one row select, against the "
+                    "single grouped pass (the dominant-kernel leg); same kernels, same buffer rotation, CUDA-graph replay"}
 
 
 def run_e2e(args, torch, M, w, sets, shared, world, dist):
@@ -416,7 +487,7 @@ def run_e2e(args, torch, M, w, sets, shared, world, dist):
         hy = [p.clone().pin_memory() for p in pristine]
         projs = [M.HostProj(hx[p.x_key], y, A, B, 1.0) for p, y, A, B in zip(w.projections, hy, s0["A"], s0["B"])]
         packed = M.binding.pack_host_projs(projs)
-        arena = torch.empty(M.molora_forward_host_arena_bytes(None, router, gate_proj, packed=packed), dtype=torch.uint8,
+        arena = torch.zeros(M.molora_forward_host_arena_bytes(None, router, gate_proj, packed=packed), dtype=torch.uint8,
                             device="cuda")
         src = None
         if w.router == "vocab":
@@ -474,6 +545,73 @@ def build_pristine_y(w, torch):
     return out
 
 
+def run_ours(args):
+    import torch
+    import paper_2603_15965_b200 as M
+    import paper_2603_15965_b200.binding  # noqa: F401
+    from paper_2603_15965_b200 import shard
+    from paper_2603_15965_b200 import workloads as W
+    from paper_2603_15965_b200.build import build_library
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the routed-LoRA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build_library()
+    if dist is not None:
+        dist.barrier()
+    env = {"torch": torch, "M": M, "lib": M.load_library(), "W": W, "shard": shard, "dist": dist, "rank": rank,
+           "world": world, "local": local}
+
+    name = args.workload or HEADLINE
+    head = measure(name, args, env, headline=True)
+    subs = {}
+    if args.workload is None and not args.profile:
+        for sub in SUB_CONFIGS:
+            subs[sub] = measure(sub, args, env, headline=False)
+
+    out = None
+    if rank == 0:
+        K = args.steps
+        passes = head["passes"]["step"]
+        out = {
+            "metric": METRIC, "value": head["value"], "unit": UNIT, "latency": head["latency"], "n_gpus": world, "steps": K,
+            "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": head["dtype"], "data": "synthetic",
+            "config": {"workload": head["workload"], "tokens_per_step_per_gpu": head["tokens_per_step_per_gpu"],
+                       "buffer_sets": head["buffer_sets"], "l2": head["l2"],
+                       "launch": ("CUDA graph replay of the C-ABI calls (route, then group + apply)" if args.launch == "graph"
+                                  else "eager, one C-ABI call per stage"),
+                       "timing": f"the K-step pass is replayed until the leg lasts >= {args.min_leg_s} s; one CUDA-event pair "
+                                 f"per pass; ms_per_step = median pass / K ({passes} passes here)"},
+            "gpu_launches": head["launches_per_step"] * K * passes, "gpu_launches_per_step": head["launches_per_step"],
+            "passes": head["passes"], "clocks": head["clocks"], "e2e": head["e2e"], "roofline": head["roofline"],
+            "cpu_baseline": None if args.profile else cpu_baseline(name),
+        }
+        if head.get("kpass_baseline") is not None:
+            out["kpass_baseline"] = head["kpass_baseline"]
+        if subs:
+            out["configs"] = {k: {"workload": v["workload"], "tokens_per_s": v["value"], "ms_per_step": v["ms_per_step"],
+                                  "kernel_ms": v["roofline"]["kernel_ms"], "kernel": v["roofline"]["kernel"],
+                                  "algorithmic_bytes": v["roofline"]["algorithmic_bytes"],
+                                  "achieved_gbs": v["roofline"]["achieved"], "frac": v["roofline"]["frac"],
+                                  "frac_of_spec": v["roofline"]["frac_of_spec"], "traffic": v["roofline"]["traffic"],
+                                  "launches_per_step": v["launches_per_step"], "buffer_sets": v["buffer_sets"],
+                                  "passes": v["passes"], "clocks": v["clocks"],
+                                  **({"kpass_baseline": v["kpass_baseline"]} if v.get("kpass_baseline") else {})}
+                              for k, v in subs.items()}
+    if dist is not None:
+        dist.destroy_process_group()
+    return out
+
+
 # ----------------------------------------------------------------------------- oracle legs (CPU)
 def oracle_sample(name):
     """The bounded sample of the workload the oracle is timed on: (workload, description)."""
@@ -484,7 +622,7 @@ def oracle_sample(name):
         return W.get("c3"), "the whole step: 256 tokens, group + 7 applies"
     if name == "c4":
         return W.get("c4", n_tokens=512), "512 of 8192 tokens, gate + group + 7 applies"
-    if name.startswith("f9-") or name.startswith("t9-"):
+    if name.startswith(("f9-", "t9-", "t6-")):
         w = W.get(name)
         return w, f"the whole step: {w.N} tokens, group + apply"
     w = W.c5_multimodal(n_seqs=1, seq_len=2048, iid=name == "c5-iid")
@@ -525,7 +663,8 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return None
-    w, sample = oracle_sample(args.workload)
+    name = args.workload or HEADLINE
+    w, sample = oracle_sample(name)
     for _ in range(min(args.warmup, 2)):
         oracle_step(w)
     K = max(1, min(args.steps, 20))
@@ -537,7 +676,7 @@ def run_reference(args):
     return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
             "warmup": min(args.warmup, 2), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{args.workload}: CPU oracle on a bounded sample ({sample})"},
+            "config": {"workload": workload_label(name, w), "sample": f"CPU oracle on a bounded sample: {sample}"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -547,18 +686,20 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     from paper_2603_15965_b200.workloads import SWEEP_NAMES
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c5-iid", *SWEEP_NAMES],
-                    help="c2 (default, the headline configuration) .. c5; f9-<N> / t9-<skew>: batch and skew sweeps")
+    ap.add_argument("--workload", default=None, choices=["c2", "c3", "c4", "c5", "c5-iid", *SWEEP_NAMES],
+                    help="default: c4 as the headline plus sub-records of c2, c3, c5, c5-iid; "
+                         "f9-<N> / t9-<skew> / t6-<distribution>: batch, skew and modality-distribution sweeps")
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
                     help="replay the timed steps from CUDA graphs (default) or launch them one by one")
+    ap.add_argument("--min-leg-s", type=float, default=0.3, help="every timed leg lasts at least this long")
     ap.add_argument("--max-sets", type=int, default=32)
-    ap.add_argument("--e2e-steps", type=int, default=50)
+    ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--profile", action="store_true",
-                    help="timed steps only: skip the host-buffer e2e leg and the oracle leg (for ncu captures)")
+                    help="timed steps of one workload only: no sub-records, no host-buffer e2e leg, no oracle leg (for ncu captures)")
     args = ap.parse_args()
     out = run_reference(args) if args.impl == "reference" else run_ours(args)
     if out is not None:

@@ -16,9 +16,10 @@
  * Conventions (all entry points unless stated otherwise)
  *   - Every tensor pointer is a DEVICE pointer owned by the caller, valid on the current device, and
  *     must stay valid until the work enqueued on `stream` has completed.  The library allocates no
- *     memory, keeps no global state, never synchronises the host and never reads device memory
- *     from the host: each call only validates its scalar arguments and enqueues kernels on `stream`,
- *     so calls may be captured into a CUDA graph.
+ *     memory, never synchronises the host and never reads device memory from the host: each call only
+ *     validates its scalar arguments and enqueues kernels on `stream`, so calls may be captured into a
+ *     CUDA graph.  The only process-wide state is per-device launch attributes cached on first use, a
+ *     counter of enqueued launches (molora_launch_count) and the debug overrides of molora_debug_set.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Matrices are row-major; `ld*` is the row pitch in ELEMENTS.
  *   - Return value: MOLORA_OK, or an error code detected on the host BEFORE anything is enqueued
@@ -64,6 +65,18 @@ const char *molora_version(void);
 
 /* Human-readable name of a status code.  Static storage. */
 const char *molora_status_string(molora_status_t status);
+
+/* Diagnostics (the paper has no counterpart).
+ * molora_launch_count: kernels this library has enqueued in this process so far (all threads, all devices); callers
+ *   that report launch counts take the difference around a call.
+ * molora_debug_set: overrides one of the library's own choices, for measurements and for tests that target one
+ *   kernel; value 0 restores the default.  Names: "umma_min_tokens" (tcgen05 apply from that many tokens),
+ *   "small_path" (kernel below it: 1 streaming, 2 two-launch, 3 job-list decode kernel), "stream_tile" (16 | 32),
+ *   "umma_split", "umma_tile_rows", "group_split" (cluster sizes / tile height), "chained_launch_off" (1: plain stream
+ *   order).  The start values are read once from the environment variables MOLORA_<NAME>.  Unknown name:
+ *   MOLORA_ERR_INVALID_ARG.  Not meant to be changed while calls are in flight on other threads. */
+uint64_t molora_launch_count(void);
+molora_status_t molora_debug_set(const char *name, int64_t value);
 
 /* ---------------------------------------------------------------------------------------------
  * Router 1: vocabulary routing (Definition 3.1 / Eq. 3; Algorithm 1 "FindModality"), 0-based:

@@ -68,6 +68,10 @@ def load_library():
     lib.molora_version.argtypes = []
     lib.molora_status_string.restype = ctypes.c_char_p
     lib.molora_status_string.argtypes = [ctypes.c_int]
+    lib.molora_launch_count.restype = ctypes.c_uint64
+    lib.molora_launch_count.argtypes = []
+    lib.molora_debug_set.restype = ctypes.c_int
+    lib.molora_debug_set.argtypes = [ctypes.c_char_p, i64]
     lib.molora_route_vocab.argtypes = [vp, i64, vp, i32, vp, vp, vp]
     lib.molora_route_composite.argtypes = [vp, vp, i64, vp, i32, i32, vp, vp, vp]
     lib.molora_topk_softmax.argtypes = [vp, i64, i32, i32, vp, vp, vp]
@@ -152,6 +156,20 @@ def _i32_dev(t: torch.Tensor, name: str) -> torch.Tensor:
 # ----------------------------------------------------------------------------- entry points
 def molora_version() -> str:
     return load_library().molora_version().decode()
+
+
+def molora_launch_count() -> int:
+    """Kernels the library has enqueued in this process so far."""
+    return int(load_library().molora_launch_count())
+
+
+TUNING_NAMES = ("umma_min_tokens", "small_path", "stream_tile", "umma_split", "umma_tile_rows", "group_split",
+                "chained_launch_off")
+
+
+def molora_debug_set(name: str, value: int) -> None:
+    """Override one of the library's kernel choices (0 = default); see include/molora.h."""
+    _check("molora_debug_set", load_library().molora_debug_set(name.encode(), int(value)))
 
 
 def molora_status_string(status: int) -> str:

@@ -3,20 +3,44 @@
 #include "common.cuh"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 using namespace molora;
 
 namespace molora {
-bool chained_launch_enabled()
+namespace {
+std::atomic<int64_t> g_tune[kTuneCount];
+std::atomic<uint64_t> g_launches{0};
+std::once_flag g_tune_once;
+const char* const kTuneNames[kTuneCount] = {"umma_min_tokens", "small_path", "stream_tile", "umma_split",
+                                            "umma_tile_rows", "group_split", "chained_launch_off"};
+void tune_from_environment()
 {
-    static const bool on = [] {
-        const char* v = std::getenv("MOLORA_CHAINED_LAUNCH");
-        return v == nullptr || std::strcmp(v, "0") != 0;
-    }();
-    return on;
+    auto num = [](const char* name) {
+        const char* e = std::getenv(name);
+        return e != nullptr && e[0] != '\0' ? (int64_t)std::atoll(e) : (int64_t)0;
+    };
+    g_tune[kTuneUmmaMinTokens] = std::max<int64_t>(0, num("MOLORA_UMMA_MIN_TOKENS"));
+    const char* sp = std::getenv("MOLORA_SMALL_PATH");
+    g_tune[kTuneSmallPath] = sp == nullptr ? 0 : sp[0] == 's' ? 1 : sp[0] == 't' ? 2 : sp[0] == 'j' ? 3 : 0;
+    g_tune[kTuneStreamTile] = num("MOLORA_STREAM_TILE");
+    g_tune[kTuneUmmaSplit] = num("MOLORA_UMMA_SPLIT");
+    g_tune[kTuneUmmaTileRows] = num("MOLORA_UMMA_TILE_ROWS");
+    g_tune[kTuneGroupSplit] = num("MOLORA_GROUP_SPLIT");
+    const char* ch = std::getenv("MOLORA_CHAINED_LAUNCH");
+    g_tune[kTuneChainedLaunchOff] = ch != nullptr && std::strcmp(ch, "0") == 0 ? 1 : 0;
 }
+}  // namespace
+int64_t tune(TuneKey key)
+{
+    std::call_once(g_tune_once, tune_from_environment);
+    return g_tune[key].load(std::memory_order_relaxed);
+}
+bool chained_launch_enabled() { return tune(kTuneChainedLaunchOff) == 0; }
+void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 }  // namespace molora
 
 namespace {
@@ -30,13 +54,9 @@ namespace {
 //            and loses by a third for a layer's worth of them);
 //   rank 64  below 1280 tokens the two-launch pair for one or two projections and the streaming kernel for more,
 //            tcgen05 above (the streaming kernel has only two stages at this rank).
-// MOLORA_UMMA_MIN_TOKENS=n forces "tcgen05 from n tokens" and MOLORA_SMALL_PATH=stream|twophase forces the kernel used
-// below it, for measurements and for tests that target one kernel.
-int64_t forced_umma_min_tokens()
-{
-    const char* e = std::getenv("MOLORA_UMMA_MIN_TOKENS");   // read per call: tests switch it
-    return e != nullptr && e[0] != '\0' ? std::max<int64_t>(1, std::atoll(e)) : (int64_t)0;
-}
+// The overrides "umma_min_tokens" (tcgen05 from n tokens) and "small_path" (the kernel used below it) of
+// molora_debug_set force a choice, for measurements and for tests that target one kernel.
+int64_t forced_umma_min_tokens() { return std::max<int64_t>(0, tune(kTuneUmmaMinTokens)); }
 constexpr double kUmmaMinBytesR16 = 150e6, kUmmaMinBytesR32 = 60e6;
 constexpr int64_t kUmmaMinTokensR64 = 1280;
 
@@ -54,9 +74,9 @@ bool use_umma(int32_t rank, int64_t N, double group_bytes)
 // the kernel for what the tcgen05 kernel does not take; same_rank: projections of this rank in the call (0: unknown)
 bool small_path_is_stream(int32_t rank, int64_t N, int same_rank)
 {
-    if (const char* e = std::getenv("MOLORA_SMALL_PATH")) {
-        if (e[0] == 's') return true;
-        if (e[0] == 't') return false;
+    if (const int64_t forced = tune(kTuneSmallPath)) {
+        if (forced == 1) return true;
+        if (forced == 2) return false;
     }
     (void)N;
     // rank 64: the two-launch pair for one or two projections (its split of the reduction over CTAs pays there);
@@ -82,7 +102,21 @@ molora_status_t check_proj(const molora_proj_desc_t& p, molora_dtype_t dt)
 
 extern "C" {
 
-const char* molora_version(void) { return "molora-b200 0.1 (sm_100a)"; }
+const char* molora_version(void) { return "molora-b200 0.2 (sm_100a)"; }
+
+molora_status_t molora_debug_set(const char* name, int64_t value)
+{
+    if (name == nullptr) return MOLORA_ERR_INVALID_ARG;
+    (void)tune(kTuneUmmaMinTokens);                 // the environment is read before the first override
+    for (int k = 0; k < kTuneCount; ++k)
+        if (std::strcmp(name, kTuneNames[k]) == 0) {
+            g_tune[k].store(value, std::memory_order_relaxed);
+            return MOLORA_OK;
+        }
+    return MOLORA_ERR_INVALID_ARG;
+}
+
+uint64_t molora_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* molora_status_string(molora_status_t status)
 {
@@ -185,23 +219,33 @@ size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t 
     return decode_workspace_bytes(N, d_in, rank);
 }
 
-molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
-                                     int32_t C, const int32_t* offsets, const int32_t* perm, void* ws, size_t ws_bytes,
-                                     uint32_t* dev_status, void* stream)
+namespace {
+// The projections of a batched apply split by kernel.  With more than kUmmaAllSegmentsMaxC adapters the projections of
+// the tcgen05 kernel are also handed to a small-tile kernel and each segment is taken by exactly one of the two,
+// chosen on the device from its row count.
+struct ApplyPlan {
+    molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], sc[MOLORA_MAX_PROJECTIONS], dc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
+    molora_proj_desc_t small_sc[MOLORA_MAX_PROJECTIONS], small_dc[MOLORA_MAX_PROJECTIONS], small_cc[MOLORA_MAX_PROJECTIONS];
+    int n_tc = 0, n_sc = 0, n_dc = 0, n_cc = 0, n_small_sc = 0, n_small_dc = 0, n_small_cc = 0;
+    int32_t min_rows = 1;          // segments with at least this many rows go to the tcgen05 kernel
+    size_t ws_need = 0;            // scratch of the two-launch kernels (the larger of their two uses in this call)
+};
+
+// Argument checks, kernel split and workspace check of molora_apply_batched: everything that can refuse the call,
+// before anything is enqueued.
+molora_status_t plan_apply(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C,
+                           const int32_t* offsets, const int32_t* perm, bool tables_given, void* ws, size_t ws_bytes,
+                           ApplyPlan& pl)
 {
     if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS) return MOLORA_ERR_INVALID_ARG;
     if (N < 0 || N >= INT32_MAX || C < 1) return MOLORA_ERR_INVALID_ARG;
     if (C > MOLORA_MAX_ADAPTERS) return MOLORA_ERR_UNSUPPORTED;
     if (dt != MOLORA_F32 && dt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
-    if (offsets == nullptr || (N > 0 && perm == nullptr)) return MOLORA_ERR_INVALID_ARG;
+    if (tables_given && (offsets == nullptr || (N > 0 && perm == nullptr))) return MOLORA_ERR_INVALID_ARG;
     for (int i = 0; i < P; ++i) {
         const molora_status_t st = check_proj(projs[i], dt);
         if (st != MOLORA_OK) return st;
     }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // Split the projections by kernel.  For projections of the tcgen05 kernel with many adapters both it and a
-    // small-tile kernel are enqueued and each segment is taken by exactly one of them, chosen on the device from
-    // its row count.
     double group_bytes[3] = {0.0, 0.0, 0.0};       // ranks 16, 32, 64
     auto group_of = [](int32_t rank) { return rank == 16 ? 0 : rank == 32 ? 1 : 2; };
     for (int i = 0; i < P; ++i)
@@ -209,40 +253,57 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
     int same_rank[3] = {0, 0, 0};                  // projections per rank that a small-tile kernel can take
     for (int i = 0; i < P; ++i)
         if (decode_eligible(projs[i], dt)) ++same_rank[group_of(projs[i].rank)];
-    molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], sc[MOLORA_MAX_PROJECTIONS], dc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
-    int n_tc = 0, n_sc = 0, n_dc = 0, n_cc = 0;
     for (int i = 0; i < P; ++i) {
         const int32_t rank = projs[i].rank;
-        if (umma_eligible(projs[i], dt) && use_umma(rank, N, group_bytes[group_of(rank)])) tc[n_tc++] = projs[i];
+        if (umma_eligible(projs[i], dt) && use_umma(rank, N, group_bytes[group_of(rank)])) pl.tc[pl.n_tc++] = projs[i];
         else if (decode_eligible(projs[i], dt)) {
-            if (small_path_is_stream(rank, N, same_rank[group_of(rank)])) sc[n_sc++] = projs[i];
-            else dc[n_dc++] = projs[i];
-        } else cc[n_cc++] = projs[i];
+            if (small_path_is_stream(rank, N, same_rank[group_of(rank)])) pl.sc[pl.n_sc++] = projs[i];
+            else pl.dc[pl.n_dc++] = projs[i];
+        } else pl.cc[pl.n_cc++] = projs[i];
     }
-    molora_status_t st = MOLORA_OK;
-    if (n_tc > 0) {
-        // With few adapters an under-filled 128-row tile is cheap, so the tensor-core kernel takes every segment
-        // and the second launch is saved; with many adapters (up to 256 composite targets) tiny segments are
-        // the norm and go to a small-tile kernel instead.
-        const int32_t min_rows = C <= kUmmaAllSegmentsMaxC ? 1 : kUmmaMinRows;
-        st = launch_apply_umma(tc, n_tc, N, C, offsets, perm, dev_status, min_rows, s);
-        if (st == MOLORA_OK && min_rows > 1) {
-            molora_proj_desc_t small_sc[MOLORA_MAX_PROJECTIONS], small_dc[MOLORA_MAX_PROJECTIONS], small_cc[MOLORA_MAX_PROJECTIONS];
-            int a = 0, b = 0, c = 0;
-            for (int i = 0; i < n_tc; ++i) {
-                if (!decode_eligible(tc[i], dt)) small_cc[c++] = tc[i];
-                else if (small_path_is_stream(tc[i].rank, N, same_rank[group_of(tc[i].rank)])) small_sc[a++] = tc[i];
-                else small_dc[b++] = tc[i];
-            }
-            if (a > 0) st = launch_apply_stream(small_sc, a, N, C, offsets, perm, min_rows, dev_status, s);
-            if (st == MOLORA_OK && b > 0) st = launch_apply_decode(small_dc, b, N, C, offsets, perm, min_rows, ws, ws_bytes, dev_status, s);
-            if (st == MOLORA_OK && c > 0) st = launch_apply_rowtile(small_cc, c, dt, N, C, offsets, perm, min_rows, s);
+    // With few adapters an under-filled 128-row tile is cheap, so the tensor-core kernel takes every segment and the
+    // second launch is saved; with many adapters (up to 256 composite targets) tiny segments are the norm and go to a
+    // small-tile kernel instead.
+    pl.min_rows = C <= kUmmaAllSegmentsMaxC ? 1 : kUmmaMinRows;
+    if (pl.n_tc > 0 && pl.min_rows > 1)
+        for (int i = 0; i < pl.n_tc; ++i) {
+            if (!decode_eligible(pl.tc[i], dt)) pl.small_cc[pl.n_small_cc++] = pl.tc[i];
+            else if (small_path_is_stream(pl.tc[i].rank, N, same_rank[group_of(pl.tc[i].rank)])) pl.small_sc[pl.n_small_sc++] = pl.tc[i];
+            else pl.small_dc[pl.n_small_dc++] = pl.tc[i];
         }
+    size_t need_dc = 0, need_small = 0;
+    for (int i = 0; i < pl.n_dc; ++i) need_dc += decode_workspace_bytes(N, pl.dc[i].d_in, pl.dc[i].rank);
+    for (int i = 0; i < pl.n_small_dc; ++i) need_small += decode_workspace_bytes(N, pl.small_dc[i].d_in, pl.small_dc[i].rank);
+    pl.ws_need = N > 0 ? std::max(need_dc, need_small) : 0;
+    if (pl.ws_need > 0 && (ws == nullptr || ws_bytes < pl.ws_need || !aligned16(ws))) return MOLORA_ERR_WORKSPACE;
+    return MOLORA_OK;
+}
+
+molora_status_t enqueue_apply(const ApplyPlan& pl, molora_dtype_t dt, int64_t N, int32_t C, const int32_t* offsets,
+                              const int32_t* perm, void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s)
+{
+    molora_status_t st = MOLORA_OK;
+    if (pl.n_tc > 0) {
+        st = launch_apply_umma(pl.tc, pl.n_tc, N, C, offsets, perm, dev_status, pl.min_rows, s);
+        if (st == MOLORA_OK && pl.n_small_sc > 0) st = launch_apply_stream(pl.small_sc, pl.n_small_sc, N, C, offsets, perm, pl.min_rows, dev_status, s);
+        if (st == MOLORA_OK && pl.n_small_dc > 0) st = launch_apply_decode(pl.small_dc, pl.n_small_dc, N, C, offsets, perm, pl.min_rows, ws, ws_bytes, dev_status, s);
+        if (st == MOLORA_OK && pl.n_small_cc > 0) st = launch_apply_rowtile(pl.small_cc, pl.n_small_cc, dt, N, C, offsets, perm, pl.min_rows, s);
     }
-    if (st == MOLORA_OK && n_sc > 0) st = launch_apply_stream(sc, n_sc, N, C, offsets, perm, INT32_MAX, dev_status, s);
-    if (st == MOLORA_OK && n_dc > 0) st = launch_apply_decode(dc, n_dc, N, C, offsets, perm, INT32_MAX, ws, ws_bytes, dev_status, s);
-    if (st == MOLORA_OK && n_cc > 0) st = launch_apply_rowtile(cc, n_cc, dt, N, C, offsets, perm, INT32_MAX, s);
+    if (st == MOLORA_OK && pl.n_sc > 0) st = launch_apply_stream(pl.sc, pl.n_sc, N, C, offsets, perm, INT32_MAX, dev_status, s);
+    if (st == MOLORA_OK && pl.n_dc > 0) st = launch_apply_decode(pl.dc, pl.n_dc, N, C, offsets, perm, INT32_MAX, ws, ws_bytes, dev_status, s);
+    if (st == MOLORA_OK && pl.n_cc > 0) st = launch_apply_rowtile(pl.cc, pl.n_cc, dt, N, C, offsets, perm, INT32_MAX, s);
     return st;
+}
+}  // namespace
+
+molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N,
+                                     int32_t C, const int32_t* offsets, const int32_t* perm, void* ws, size_t ws_bytes,
+                                     uint32_t* dev_status, void* stream)
+{
+    ApplyPlan pl;
+    const molora_status_t st = plan_apply(projs, P, dt, N, C, offsets, perm, true, ws, ws_bytes, pl);
+    if (st != MOLORA_OK) return st;
+    return enqueue_apply(pl, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 // How molora_group_apply_batched runs: 1 = one launch (every projection on the streaming kernel, one rank, at most 4096
@@ -295,16 +356,24 @@ molora_status_t molora_group_apply_batched(const int32_t* r, int64_t N, int32_t 
         if (st != MOLORA_OK) return st;
     }
     // When every projection of the call runs on the streaming kernel (or on the two-launch kernels) with one rank, the
-    // CTAs of those kernels do the grouping themselves.  Otherwise the two calls, in stream order.
+    // CTAs of those kernels do the grouping themselves.  Otherwise the two calls, in stream order.  Whatever could
+    // refuse the call (the workspace of the two-launch kernels included) is checked before the first launch.
     const int mode = group_apply_mode(projs, P, dt, N);
     if (mode == 1)
         return launch_group_apply_stream(r, projs, P, N, C, counts, offsets, perm, dev_status, static_cast<cudaStream_t>(stream));
-    if (mode == 2)
+    if (mode == 2) {
+        size_t need = 0;
+        for (int i = 0; i < P; ++i) need += decode_workspace_bytes(N, projs[i].d_in, projs[i].rank);
+        if (need > 0 && (ws == nullptr || ws_bytes < need || !aligned16(ws))) return MOLORA_ERR_WORKSPACE;
         return launch_group_apply_decode(r, projs, P, N, C, counts, offsets, perm, ws, ws_bytes, dev_status,
                                          static_cast<cudaStream_t>(stream));
-    const molora_status_t st = molora_group(r, N, C, counts, offsets, perm, nullptr, 0, dev_status, stream);
+    }
+    ApplyPlan pl;
+    molora_status_t st = plan_apply(projs, P, dt, N, C, offsets, perm, false, ws, ws_bytes, pl);
     if (st != MOLORA_OK) return st;
-    return molora_apply_batched(projs, P, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, stream);
+    st = molora_group(r, N, C, counts, offsets, perm, nullptr, 0, dev_status, stream);
+    if (st != MOLORA_OK) return st;
+    return enqueue_apply(pl, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 molora_status_t molora_apply(const void* x, int64_t ldx, void* y, int64_t ldy, molora_dtype_t dt, int64_t N,

@@ -60,22 +60,7 @@ struct StreamParams {
     int32_t* counts_out;
     int32_t* offsets_out;
     int32_t* perm_out;
-#ifdef MOLORA_TRACE
-    long long* trace;                         // development builds only: globaltimer stamps per CTA
-#endif
 };
-#ifdef MOLORA_TRACE
-#define FS_GT(slot)                                                                                    \
-    do {                                                                                               \
-        if (prm.trace != nullptr && (threadIdx.x & 31) == 0 && blockIdx.x < 160 && (slot) < 64) {      \
-            long long t_;                                                                              \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                     \
-            prm.trace[blockIdx.x * 64 + (slot)] = t_;                                                  \
-        }                                                                                              \
-    } while (0)
-#else
-#define FS_GT(slot) do { } while (0)
-#endif
 // (projection, slice of d_out) pairs of the projections of the launch's rank; projection p owns [start[p], start[p + 1]).
 struct FsUnits {
     int32_t start[MOLORA_MAX_PROJECTIONS + 1];
@@ -184,7 +169,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
     extern __shared__ __align__(128) unsigned char dsm[];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (warp == 0) FS_GT(0);
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&full_s[s]), kFsCopyWarps);
@@ -210,7 +194,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
     __syncthreads();
     const int T = tstart_s[prm.C];
     const int nitems = T * units.start[prm.P];
-    if (warp == 0) FS_GT(1);
     const uint32_t stage0 = smem_u32(dsm);
     float* tfin = reinterpret_cast<float*>(dsm + NS * Cfg::STAGE);
 
@@ -234,7 +217,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                 bulk_wait_group_read<0>();     // the stage may be overwritten
             }
             __syncwarp();                      // every lane has read the stage's record before lane 0 rewrites it
-            if (cw == 0) FS_GT(4 + (int)k * 4 + 1);
         };
         uint32_t g = 0;                        // jobs issued so far; job k lives in stage k % NS
         for (int item = blockIdx.x; item < nitems && !abort_s; item += (int)gridDim.x) {
@@ -252,7 +234,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                 if (g >= (uint32_t)NS) retire(g - NS);
                 if (abort_s) break;
                 const uint32_t sb = stage0 + s * Cfg::STAGE, bar = smem_u32(&full_s[s]);
-                if (cw == 0) FS_GT(4 + (int)g * 4);
                 fence_proxy_async_smem();      // earlier accesses to the stage are ordered before the copies
                 if (j < it.nks) {
                     const int k0 = j * Cfg::CH, kc = min(Cfg::CH, pd.d_in - k0);
@@ -297,7 +278,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             }
         }
         bulk_wait_group<0>();                  // my stores have completed
-        if (cw == 0) FS_GT(2);
         return;
     }
 
@@ -324,7 +304,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             const uint32_t s = g % NS;
             const uint32_t xs = stage0 + s * Cfg::STAGE, as = xs + Cfg::ROWBYTES;
             wait_bar(smem_u32(&full_s[s]), (g / NS) & 1u, &abort_s, prm.dev_status);
-            if (warp == 0) FS_GT(4 + (int)g * 4 + 2);
             const int nb = min(Cfg::CH, pd.d_in - j * Cfg::CH) / 32;
             for (int b = warp; b < nb; b += kFsWarps) {
 #pragma unroll
@@ -350,7 +329,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             }
             if (j + 1 < it.nks) {
                 __syncwarp();
-                if (warp == 0) FS_GT(4 + (int)g * 4 + 3);
                 if (lane == 0) mbar_arrive(smem_u32(&done_s[s]));
             } else {
                 // last chunk: sum the per-warp partials in warp order through this stage, then release it
@@ -385,7 +363,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                 }
                 fence_proxy_async_smem();          // my writes to the stage are ordered before the copies that refill it
                 fs_compute_sync();                 // t is complete; the stage is free
-                if (warp == 0) FS_GT(4 + (int)g * 4 + 3);
                 if (lane == 0) mbar_arrive(smem_u32(&done_s[s]));
             }
         }
@@ -412,7 +389,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             const uint32_t ys = stage0 + s * Cfg::STAGE, bs = ys + Cfg::ROWBYTES;
             unsigned char* ysp = dsm + s * Cfg::STAGE;
             wait_bar(smem_u32(&full_s[s]), (g / NS) & 1u, &abort_s, prm.dev_status);
-            if (warp == 0) FS_GT(4 + (int)g * 4 + 2);
             const int ncols = min(Cfg::CH, pd.d_out - it.col0 - e * Cfg::CH);
             // my 32-column groups, GI at a time: y words first, then the MMAs, then add, round once and write back.
             // Rows past the tile hold stale shared memory; they are updated like the others and never stored.
@@ -490,7 +466,6 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             }
             fence_proxy_async_smem();              // my updates of y are visible to the bulk stores
             __syncwarp();
-            if (warp == 0) FS_GT(4 + (int)g * 4 + 3);
             if (lane == 0) mbar_arrive(smem_u32(&done_s[s]));
         }
     }
@@ -506,7 +481,8 @@ template <int R, bool GROUP, bool SHORT>
 static cudaError_t stream_launch(StreamParams prm, int64_t N, cudaStream_t s)
 {
     using Cfg = FsCfg<R, SHORT>;
-    static int slots = 0;                          // resident CTAs on this device: the size of a wave
+    static int slots_dev[kMaxDevices] = {};        // resident CTAs per device: the size of a wave
+    int& slots = slots_dev[device_slot()];
     if (slots == 0) {
         cudaError_t e = cudaFuncSetAttribute(apply_stream_kernel<R, GROUP, SHORT>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
         if (e != cudaSuccess) return e;
@@ -565,9 +541,6 @@ static molora_status_t stream_enqueue(const molora_proj_desc_t* projs, int32_t P
     prm.P = P;
     prm.C = C;
     prm.N = (int32_t)N;
-#ifdef MOLORA_TRACE
-    prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
-#endif
     // rank 16: the short tile while its tiles of all projections (nearly) fit one wave of CTAs
     int p16 = 0;
     for (int i = 0; i < P; ++i) p16 += projs[i].rank == 16;
@@ -578,7 +551,7 @@ static molora_status_t stream_enqueue(const molora_proj_desc_t* projs, int32_t P
     }
     const int64_t cap_rows = prm.max_rows == INT32_MAX ? N : std::min<int64_t>(N, (int64_t)C * prm.max_rows);
     bool short16 = (ceil_div64(cap_rows, 16) + C) * p16 <= (int64_t)(sms * kFsShortFill);
-    if (const char* e = getenv("MOLORA_STREAM_TILE")) short16 = atoi(e) == 16;
+    if (const int64_t forced = tune(kTuneStreamTile)) short16 = forced == 16;
     cudaError_t e = cudaSuccess;
     if (group) {                                   // one rank only (checked by the caller): one launch does it all
         if (has[0]) e = short16 ? stream_launch<16, true, true>(prm, N, s) : stream_launch<16, true, false>(prm, N, s);

@@ -60,23 +60,7 @@ struct TwoPhaseParams {
     int32_t* counts_out;
     int32_t* offsets_out;
     int32_t* perm_out;
-#ifdef MOLORA_TRACE
-    long long* trace;                         // development builds only: globaltimer stamps per CTA
-#endif
 };
-#ifdef MOLORA_TRACE
-#define TP_GT(kernel, slot)                                                                            \
-    do {                                                                                               \
-        if (prm.trace != nullptr && threadIdx.x == 0) {                                                \
-            const int cta = blockIdx.x;                                                                \
-            long long t_;                                                                              \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                     \
-            if (cta < 1024) prm.trace[((kernel) * 1024 + cta) * 8 + (slot)] = t_;                      \
-        }                                                                                              \
-    } while (0)
-#else
-#define TP_GT(kernel, slot) do { } while (0)
-#endif
 // Work-item units: (projection, slice) pairs of the projections of the launch's rank; projection p owns the unit
 // indices [start[p], start[p + 1]).
 struct TpUnits {
@@ -191,12 +175,9 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
         abort_s = 0;
         fence_mbar_init();
     }
-    TP_GT(0, 0);
     grid_dependency_sync();                        // offsets and perm come from the grouping kernel
-    TP_GT(0, 1);
     const int T = tp_load_tables<GROUP>(prm, offs_s, tstart_s, perm_s, dsm, true);
     const int nitems = T * units.start[prm.P];
-    TP_GT(0, 2);
 
     const uint32_t xs = smem_u32(dsm), as = xs + Cfg::XBYTES;
     float* tparts = reinterpret_cast<float*>(dsm);                       // reuses the staging area after the MMAs
@@ -242,7 +223,6 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
             dead = __syncthreads_or(abort_s);
             if (dead) break;
             parity ^= 1u;
-            TP_GT(0, 3);
             for (int b = warp; b < nb; b += kTpWarps) {
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {                           // two k16 steps per block
@@ -269,7 +249,6 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
             __syncthreads();                       // the staging area is free again
         }
         if (dead) break;
-        TP_GT(0, 4);
         // per-warp partials -> CTA partial (warp order) -> workspace
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
@@ -296,7 +275,6 @@ __global__ void __launch_bounds__(kTpThreads, 2) shrink_kernel(const __grid_cons
         __syncthreads();                           // the partials may be overwritten by the next item's copies
     }
     if (dead && tid == 0) tp_drain(bar, parity);
-    TP_GT(0, 5);
 }
 
 // ------------------------------------------------------------------------------------------------ expand
@@ -322,7 +300,6 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
         fence_mbar_init();
     }
     // Nothing read before the dependency wait below is written by the shrink kernel (see the file header).
-    TP_GT(1, 0);
     const int T = tp_load_tables<GROUP>(prm, offs_s, tstart_s, perm_s, dsm, false);
     const int nitems = T * units.start[prm.P];
 
@@ -358,9 +335,7 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
 
     int item = blockIdx.x;
     if (item < nitems) request(item);
-    TP_GT(1, 1);
     grid_dependency_sync();                        // the partial t of the shrink kernel are complete and visible
-    TP_GT(1, 2);
 
     uint32_t parity = 0;
     int dead = 0;
@@ -399,7 +374,6 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
         dead = __syncthreads_or(abort_s);          // also publishes t
         if (dead) break;
         parity ^= 1u;
-        TP_GT(1, 3);
         // A fragments of t: bf16 hi and lo parts
         uint32_t thi[2][KB][4], tlo[2][KB][4];
 #pragma unroll
@@ -463,7 +437,6 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
         }
         fence_proxy_async_smem();                  // my updates of y are visible to the bulk stores
         __syncthreads();
-        TP_GT(1, 4);
         if (warp == 0) {
             if (lane < t.rows) bulk_store(yrow, ys + lane * Cfg::YP, (uint32_t)ncols * 2u);
             bulk_commit_group();
@@ -475,7 +448,6 @@ __global__ void __launch_bounds__(kTpThreads, 2) expand_kernel(const __grid_cons
     }
     if (warp == 0) bulk_wait_group<0>();           // my stores have completed
     if (dead && tid == 0) tp_drain(bar, parity);
-    TP_GT(1, 5);
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -505,7 +477,8 @@ static cudaError_t twophase_launch(const TwoPhaseParams& prm, int64_t N, cudaStr
                   "the grouping scratch fits the staging areas");
     using Cfg = TpCfg<R>;
     // resident CTAs of each kernel on this device: the size of a wave
-    static int wave[2] = {0, 0};
+    static int wave_dev[kMaxDevices][2] = {};
+    int (&wave)[2] = wave_dev[device_slot()];
     if (wave[0] == 0) {
         cudaError_t e = cudaFuncSetAttribute(shrink_kernel<R, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SHRINK_SMEM);
         if (e == cudaSuccess)
@@ -558,9 +531,6 @@ static molora_status_t decode_enqueue(const molora_proj_desc_t* projs, int32_t P
     prm.P = P;
     prm.C = C;
     prm.N = (int32_t)N;
-#ifdef MOLORA_TRACE
-    prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
-#endif
     cudaError_t e = cudaSuccess;
     if (group) {                                   // one rank only (checked by the caller)
         if (has[0]) e = twophase_launch<16, true>(prm, N, s);

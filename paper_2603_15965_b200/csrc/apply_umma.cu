@@ -77,32 +77,8 @@ struct UmmaParams {
     uint32_t* dev_status;
     int32_t P, C, min_rows;
     int32_t tile_rows;    // positions per tile: 128, or fewer (the MMA tile stays 128 lanes) to spread a small call over more SMs
-#ifdef MOLORA_TRACE
-    long long* trace;     // development builds only: clock64 stamps of CTA 0, [role][iteration][slot]
-#endif
 };
 
-#ifdef MOLORA_TRACE
-#define MOLORA_TR(role, it, slot)                                                        \
-    do {                                                                                 \
-        if (blockIdx.x == 0 && blockIdx.y == 0 && prm.trace != nullptr && (it) < 256)    \
-            prm.trace[((role) * 256 + (it)) * 8 + (slot)] = clock64();                   \
-    } while (0)
-__device__ __forceinline__ long long molora_gtime()
-{
-    long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define MOLORA_TR_CTA(slot)                                                                              \
-    do {                                                                                                 \
-        if (prm.trace != nullptr && threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.x < 2048)            \
-            prm.trace[4 * 256 * 8 + blockIdx.x * 2 + (slot)] = molora_gtime();                           \
-    } while (0)
-#else
-#define MOLORA_TR(role, it, slot) do { } while (0)
-#define MOLORA_TR_CTA(slot) do { } while (0)
-#endif
 
 template <int R>
 struct UmmaCfg {
@@ -137,7 +113,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 {
     using Cfg = UmmaCfg<R>;
     extern __shared__ uint8_t smem_raw[];
-    MOLORA_TR_CTA(0);
     const UmmaProj& pj = prm.p[blockIdx.y];
     if (pj.rank != R) return;
     const uint32_t S = cluster_nctarank(), crank = cluster_ctarank();   // CTAs sharing this tile, and my slice
@@ -155,7 +130,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 
     // ---------------------------------------------------------------- set-up
     // The segment table is requested first; barriers and TMEM are set up while it is on its way.
-    if (tid == 0) MOLORA_TR(3, 0, 0);
     grid_dependency_sync();            // offsets and perm come from the grouping kernel; y from the base projection
     __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
     int32_t offs_v[(MOLORA_MAX_ADAPTERS + kUmmaThreads) / kUmmaThreads];
@@ -207,11 +181,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     const int total = KX + NY;
     if (tid < kTileM) ctrl->rows[tid] = tid < rows ? __ldg(prm.perm + row0 + tid) : -1;
     __syncthreads();
-    if (tid == 0) MOLORA_TR(3, 0, 1);
     // "I am running and my barriers are initialised": the matching wait comes right before the first access to
     // a peer's shared memory (the T exchange), so the cluster barrier costs nothing here
     if (S > 1) cluster_arrive_relaxed();      // (the barrier initialisation was released by fence_mbar_init)
-    if (tid == 0) MOLORA_TR(3, 0, 2);
     const uint32_t tmem = ctrl->tmem_base;
     const uint32_t tmem_T = tmem;                               // columns [0, R)
     auto tmem_D = [&](int b) { return tmem + 64u + 64u * (uint32_t)b; };
@@ -240,9 +212,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         int s = 0;
         uint32_t ph = 1;                                        // parity of the "empty" phase to wait for
         for (int it = 0; it < total; ++it) {
-            if (tid == 0) MOLORA_TR(0, it, 0);
             if (it >= Cfg::kStages) wait_bar(bar(&ctrl->empty[s]), ph, abort_flag, prm.dev_status);   // first round: all free
-            if (tid == 0) MOLORA_TR(0, it, 1);
             const uint32_t dst = stage(s);
             if (!*abort_flag) {
                 if (it < KX) {
@@ -260,7 +230,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 }
             }
             cp_async_arrive_noinc(bar(&ctrl->full[s]));
-            if (tid == 0) MOLORA_TR(0, it, 2);
             if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
         }
     } else if (warp == kWeightWarp) {
@@ -288,9 +257,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             for (int it = 0; it < KX; ++it) {
                 const int s = it % Cfg::kStages;
                 const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
-                MOLORA_TR(1, it, 0);
                 wait_bar(bar(&ctrl->full[s]), ph, abort_flag, prm.dev_status);
-                MOLORA_TR(1, it, 1);
                 fence_proxy_async_smem();     // the gathered rows were written through the generic proxy
                 tc_fence_after();
                 if (!*abort_flag) {
@@ -305,20 +272,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 }
             }
             if (!*abort_flag) umma_commit(bar(&ctrl->t_full));
-            MOLORA_TR(3, 1, 0);
             wait_bar(bar(&ctrl->t_ready), 0, abort_flag, prm.dev_status);
-            MOLORA_TR(3, 1, 1);
             tc_fence_after();
             for (int nc = 0; nc < NY; ++nc) {
                 const int it = KX + nc;
                 const int s = it % Cfg::kStages;
                 const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
                 const int b = nc % kDBufs;
-                MOLORA_TR(1, it, 0);
                 wait_bar(bar(&ctrl->full[s]), ph, abort_flag, prm.dev_status);
-                MOLORA_TR(1, it, 1);
                 wait_bar(bar(&ctrl->d_empty[b]), ((uint32_t)(nc / kDBufs) & 1u) ^ 1u, abort_flag, prm.dev_status);
-                MOLORA_TR(1, it, 2);
                 tc_fence_after();
                 if (!*abort_flag) {
                     const uint32_t w0 = stage(s) + kTileBytes;
@@ -347,9 +309,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 
         if (group == 0) {
             // T -> scaled bf16 hi/lo pair in shared memory, K-major, swizzled like a TMA tile of R*2-byte rows
-            if (et == 0) MOLORA_TR(3, 2, 0);
             wait_bar(bar(&ctrl->t_full), 0, abort_flag, prm.dev_status);
-            if (et == 0) MOLORA_TR(3, 2, 1);
             tc_fence_after();
             uint32_t tv[R];
 #pragma unroll
@@ -376,9 +336,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 }
                 __syncwarp();                                   // the warp's rows are sent; lane q2 tells CTA q2
                 if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
-                if (et == 0) MOLORA_TR(3, 2, 2);
                 wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
-                if (et == 0) MOLORA_TR(3, 2, 3);
 #pragma unroll
                 for (int c4 = 0; c4 < R / 4; ++c4) {            // rank order, in place
                     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -404,8 +362,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                     tv[4 * c4 + 2] = __float_as_uint(a.z);
                     tv[4 * c4 + 3] = __float_as_uint(a.w);
                 }
-                if (et == 0) MOLORA_TR(3, 2, 4);
-                if (et == 0) MOLORA_TR(3, 2, 5);
                 // tv now holds the full T row: the local conversion below finishes it
             } else if (S > 1) {
                 // Exchange of the partial T tiles in two pushes through distributed shared memory.  CTA o owns the
@@ -431,9 +387,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 }
                 __syncwarp();                                   // the warp's rows are sent; lane q2 tells CTA q2
                 if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
-                if (et == 0) MOLORA_TR(3, 2, 2);
                 wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
-                if (et == 0) MOLORA_TR(3, 2, 3);
                 if ((uint32_t)owner == crank) {
                     // sum in rank order, in place: lower ranks' partials, mine (registers), higher ranks'
 #pragma unroll
@@ -480,9 +434,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 }
                 __syncwarp();                                   // the warp's rows are published everywhere
                 if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_free), (uint32_t)lane));
-                if (et == 0) MOLORA_TR(3, 2, 4);
                 wait_bar_cluster(bar(&ctrl->part_free), 0, abort_flag, prm.dev_status);   // all 128 rows of T are here
-                if (et == 0) MOLORA_TR(3, 2, 5);
                 t_published = true;
             }
             if (!t_published) {
@@ -504,7 +456,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(bar(&ctrl->t_ready));
-            if (et == 0) MOLORA_TR(3, 2, 6);
         }
 
         // copy-out mapping: piece (et & 7) of rows (et >> 3) + 16 i
@@ -520,9 +471,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             const int s = it % Cfg::kStages;
             const uint32_t ph = (uint32_t)(it / Cfg::kStages) & 1u;
             const int b = nc % kDBufs;
-            if (et == 0) MOLORA_TR(2, it, 0);
             wait_bar(bar(&ctrl->d_full[b]), (uint32_t)(nc / kDBufs) & 1u, abort_flag, prm.dev_status);
-            if (et == 0) MOLORA_TR(2, it, 1);
             tc_fence_after();
             uint32_t dv[64];
 #pragma unroll
@@ -530,9 +479,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive(bar(&ctrl->d_empty[b]));
-            if (et == 0) MOLORA_TR(2, it, 2);
             wait_bar(bar(&ctrl->full[s]), ph, abort_flag, prm.dev_status);   // the Y chunk of this stage has landed
-            if (et == 0) MOLORA_TR(2, it, 3);
             uint8_t* ytile = smem_raw + (stage(s) - raw);
             {
                 uint4 yp[8];
@@ -549,9 +496,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                         pack<__nv_bfloat16>(yv);
                 }
             }
-            if (et == 0) MOLORA_TR(2, it, 4);
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
-            if (et == 0) MOLORA_TR(2, it, 5);
             if (!*abort_flag) {
                 if (pj.wide_store) {
                     // 32 bytes per lane: four lanes cover a 128-byte row segment, a warp instruction eight rows
@@ -564,7 +509,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                         lo4[i] = *reinterpret_cast<const uint4*>(ytile + swizzle_offset(r * 128u + p32 * 32, 3));
                         hi4[i] = *reinterpret_cast<const uint4*>(ytile + swizzle_offset(r * 128u + p32 * 32 + 16, 3));
                     }
-                    if (et == 0) MOLORA_TR(2, it, 7);
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
                         if (wtok[i] >= 0) stg256(dstc + (int64_t)wtok[i] * pj.ldy, lo4[i], hi4[i]);
@@ -575,30 +519,23 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                     for (int i = 0; i < 8; ++i)
                         op[i] = *reinterpret_cast<const uint4*>(
                             ytile + swizzle_offset((uint32_t)((et >> 3) + 16 * i) * 128u + piece * 16, 3));
-                    if (et == 0) MOLORA_TR(2, it, 7);
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         if (otok[i] >= 0) stg128(dstc + (int64_t)otok[i] * pj.ldy, op[i]);
                 }
             }
-            if (et == 0) MOLORA_TR(2, it, 4);
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
             if (et == 0) mbar_arrive(bar(&ctrl->empty[s]));   // the stage may be refilled
-            if (et == 0) MOLORA_TR(2, it, 6);
         }
     }
 
     // ---------------------------------------------------------------- teardown
-    if (tid == 0) MOLORA_TR(3, 0, 3);
     tc_fence_before();
     __syncthreads();
-    if (tid == 0) MOLORA_TR(3, 0, 4);
     if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
     // threads that took no part in the exchange complete the start-up cluster barrier here (it has long been
     // passed); no closing barrier is needed, see the exchange
     if (S > 1 && !(warp >= kEpiWarp0 && warp < kEpiWarp0 + 4)) cluster_wait();
-    if (tid == 0) MOLORA_TR(3, 0, 5);
-    MOLORA_TR_CTA(1);
 }
 
 // Self-test of the bounded wait: one warp waits on an mbarrier that nothing ever arrives on, with a limit of
@@ -627,6 +564,7 @@ __global__ void bounded_wait_selftest_kernel(uint32_t* dev_status, long long lim
 
 molora_status_t launch_bounded_wait_selftest(uint32_t* dev_status, int64_t limit_cycles, int32_t* result, cudaStream_t s)
 {
+    note_launch();
     bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(dev_status, limit_cycles, result);
     return cuda_ok(cudaGetLastError());
 }
@@ -665,7 +603,8 @@ static cudaError_t umma_launch(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStr
     const int split = plan.split;
     prm.tile_rows = plan.tile_rows;
     using Cfg = UmmaCfg<R>;
-    static bool configured = false;
+    static bool configured_dev[kMaxDevices] = {};
+    bool& configured = configured_dev[device_slot()];
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(apply_umma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              Cfg::kSmemBytes);
@@ -676,6 +615,7 @@ static cudaError_t umma_launch(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStr
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     fill_launch_config<R>(cfg, attr, tiles, prm.P, split, s);
+    note_launch();
     return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R>, prm);
 }
 
@@ -683,7 +623,8 @@ static cudaError_t umma_launch(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStr
 template <int R>
 static int max_active_clusters(int split)
 {
-    static int cache[kMaxSplit + 1] = {};
+    static int cache_dev[kMaxDevices][kMaxSplit + 1] = {};
+    int (&cache)[kMaxSplit + 1] = cache_dev[device_slot()];
     if (cache[split] == 0) {
         cudaFuncSetAttribute(apply_umma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<R>::kSmemBytes);
         cudaLaunchConfig_t cfg = {};
@@ -716,11 +657,10 @@ static UmmaPlan choose_split_for_rank(const UmmaParams& prm, int64_t N)
         return waves * ((rows / 128.0) / split + 0.15 + (split > 1 ? 0.10 : 0.0));
     };
     UmmaPlan best = {1, kTileM};
-    const char* env = getenv("MOLORA_UMMA_SPLIT");          // tuning overrides
-    const char* envr = getenv("MOLORA_UMMA_TILE_ROWS");
-    if (env != nullptr || envr != nullptr) {
-        if (env != nullptr) best.split = std::max(1, std::min(atoi(env), UmmaCfg<R>::kMaxSplitR));
-        if (envr != nullptr) best.tile_rows = std::max(32, std::min(atoi(envr), kTileM));
+    const int64_t fsplit = tune(kTuneUmmaSplit), frows = tune(kTuneUmmaTileRows);          // tuning overrides
+    if (fsplit > 0 || frows > 0) {
+        if (fsplit > 0) best.split = (int)std::max<int64_t>(1, std::min<int64_t>(fsplit, UmmaCfg<R>::kMaxSplitR));
+        if (frows > 0) best.tile_rows = (int)std::max<int64_t>(32, std::min<int64_t>(frows, kTileM));
     } else {
         double best_cost = 1e30, best_waves = 0;
         for (int split = 1; split <= UmmaCfg<R>::kMaxSplitR; ++split) {    // cluster sizes need not be powers of two
@@ -786,9 +726,6 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
     prm.C = C;
     prm.min_rows = min_rows;
     prm.tile_rows = kTileM;
-#ifdef MOLORA_TRACE
-    prm.trace = getenv("MOLORA_TRACE_PTR") ? (long long*)strtoull(getenv("MOLORA_TRACE_PTR"), nullptr, 0) : nullptr;
-#endif
     cudaError_t e = cudaSuccess;
     if (has[0] && e == cudaSuccess) e = umma_launch<16>(prm, N, choose_split_for_rank<16>(prm, N), s);
     if (has[1] && e == cudaSuccess) e = umma_launch<32>(prm, N, choose_split_for_rank<32>(prm, N), s);

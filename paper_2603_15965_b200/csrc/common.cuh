@@ -297,7 +297,23 @@ constexpr int32_t kUmmaAllSegmentsMaxC = 64;   // up to this many adapters the t
 // calls ptx::grid_dependency_wait() before it touches what that kernel writes.  Used only between the two
 // launches of one call (weight split -> tcgen05 gate, decode shrink -> expand), where the predecessor is known;
 // across calls the kernels run in plain stream order (chaining them was measured: no gain on any workload).
-bool chained_launch_enabled();   // false when MOLORA_CHAINED_LAUNCH=0 (plain stream order everywhere, for comparisons)
+bool chained_launch_enabled();   // false when the "chained_launch_off" override is set (plain stream order everywhere)
+// Tuning overrides, for measurements and for tests that target one kernel: process-wide integers, 0 = the library's own
+// choice.  Their start values come from the environment (MOLORA_UMMA_MIN_TOKENS, MOLORA_SMALL_PATH=stream|twophase|jobs,
+// MOLORA_STREAM_TILE, MOLORA_UMMA_SPLIT, MOLORA_UMMA_TILE_ROWS, MOLORA_GROUP_SPLIT, MOLORA_CHAINED_LAUNCH=0), read ONCE
+// when the library is first used; afterwards only molora_debug_set changes them.
+enum TuneKey {
+    kTuneUmmaMinTokens = 0,   // tcgen05 apply from this many tokens
+    kTuneSmallPath,           // kernel below the tcgen05 crossover: 1 streaming, 2 two-launch, 3 job-list decode kernel
+    kTuneStreamTile,          // rank-16 streaming tile: 16 or 32 rows
+    kTuneUmmaSplit,           // cluster size of the tcgen05 apply
+    kTuneUmmaTileRows,        // rows per tile of the tcgen05 apply
+    kTuneGroupSplit,          // cluster size of the grouping kernel
+    kTuneChainedLaunchOff,    // 1: no programmatic dependent launches
+    kTuneCount
+};
+int64_t tune(TuneKey key);
+void note_launch();               // one more kernel enqueued by this library (molora_launch_count)
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
                                  unsigned cluster_x, bool under_predecessor, Args&&... args)
@@ -323,7 +339,18 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
     }
     cfg.attrs = attr;
     cfg.numAttrs = n;
+    note_launch();
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// Launch attributes (opt-in shared memory sizes, occupancy-derived wave sizes) belong to a device: the launchers cache
+// them in small arrays indexed by the ordinal of the current device.
+constexpr int kMaxDevices = 64;
+inline int device_slot()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
+    return dev % kMaxDevices;
 }
 
 inline molora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? MOLORA_OK : MOLORA_ERR_CUDA; }

@@ -181,7 +181,7 @@ molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* co
     // one CTA per ~1024 tokens (one 32-token step per warp), at most 8 CTAs
     int split = 1;
     while (split < kGroupMaxCluster && (int64_t)split * 1024 < N) split *= 2;
-    if (const char* e = getenv("MOLORA_GROUP_SPLIT")) split = std::max(1, std::min(atoi(e), kGroupMaxCluster));
+    if (const int64_t forced = tune(kTuneGroupSplit)) split = (int)std::max<int64_t>(1, std::min<int64_t>(forced, kGroupMaxCluster));
     return cuda_ok(launch_kernel(group_cluster_kernel, dim3((unsigned)split), dim3(kGroupThreads), 0, s, (unsigned)split, false,
                                   r, N, C, counts, offsets, perm, dev_status));
 }

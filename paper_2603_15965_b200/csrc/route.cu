@@ -410,7 +410,8 @@ static molora_status_t gate_resident_launch(const void* x, int64_t N, int d, int
     const size_t smem = (size_t)chunks * 32 * (VEC * CP + 4) * sizeof(float);
     handled = smem <= 96 * 1024;
     if (!handled) return MOLORA_OK;
-    static bool configured = false;
+    static bool configured_dev[kMaxDevices] = {};
+    bool& configured = configured_dev[device_slot()];
     if (!configured) {
         if (cudaFuncSetAttribute(route_gate_resident_kernel<T, CP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  96 * 1024) != cudaSuccess)
@@ -422,7 +423,8 @@ static molora_status_t gate_resident_launch(const void* x, int64_t N, int d, int
     while (tpw > 2 && ceil_div64(N, 4 * tpw) < 148) tpw /= 2;
     const int64_t blocks = ceil_div64(N, 4 * tpw);
     if (tpw <= 4 && chunks <= 8) {   // small call: the burst variant (every load of a warp in flight at once)
-        static bool configured_burst = false;
+        static bool configured_burst_dev[kMaxDevices] = {};
+        bool& configured_burst = configured_burst_dev[device_slot()];
         if (!configured_burst) {
             if (cudaFuncSetAttribute(route_gate_resident_burst_kernel<T, CP, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      96 * 1024) != cudaSuccess ||

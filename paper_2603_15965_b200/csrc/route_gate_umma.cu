@@ -192,7 +192,8 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
     while (split < (CP == 16 ? kGuMaxSplit : 2) && tiles * split * 2 <= 148 && (d / 64) / (split * 2) >= 8) split *= 2;
     const int SMEM = 1024 + STAGES * (kGuTileBytes + NP * 128) + 256 + (kGuMaxSplit - 1) * NP * 128 * 4 * (CP == 16 ? 1 : 0) +
                      (CP == 16 ? 0 : NP * 128 * 4);
-    static bool configured = false;
+    static bool configured_dev[kMaxDevices] = {};
+    bool& configured = configured_dev[device_slot()];
     if (!configured) {
         if (cudaFuncSetAttribute(route_gate_umma_kernel<CP>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
             return MOLORA_ERR_CUDA;
@@ -228,6 +229,7 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = chained_launch_enabled() ? 2 : 1;
+    note_launch();
     return cuda_ok(cudaLaunchKernelEx(&cfg, route_gate_umma_kernel<CP>, prm));
 }
 

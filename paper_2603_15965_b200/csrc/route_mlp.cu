@@ -268,7 +268,8 @@ static molora_status_t mlp_umma_launch(const void* x, int64_t N, int d, int64_t 
     constexpr int NP = 3 * HP;
     constexpr int STAGES = HP == 64 ? 5 : 3;
     constexpr int SMEM = 1024 + STAGES * (kMlpTileBytes + NP * 128) + 256 + (HP * kMlpMaxC + HP) * 4;
-    static bool configured = false;
+    static bool configured_dev[kMaxDevices] = {};
+    bool& configured = configured_dev[device_slot()];
     if (!configured) {
         if (cudaFuncSetAttribute(route_mlp_umma_kernel<HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
             return MOLORA_ERR_CUDA;

@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the Blackwell (sm_100a) features the tensor-core apply kernel uses:
-// mbarrier, TMA (tiled, row-gather and row-scatter forms), tcgen05 MMA / TMEM, proxy fences and
+// mbarrier, TMA (tiled loads, linear bulk copies), tcgen05 MMA / TMEM, proxy fences and
 // the shared-memory / instruction descriptors of tcgen05.mma.
 #pragma once
 #include <cuda_runtime.h>
@@ -102,15 +102,6 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t cluster_addr)
-{
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "r"(cluster_addr)
-                 : "memory");
-    return v;
-}
 
 // ---------------------------------------------------------------- proxy / tcgen05 fences
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -128,25 +119,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int 
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-// Row gather: four rows (r0..r3) of a 2-D tensor, box-width columns starting at column c0, land as four
-// consecutive rows in shared memory.  The tensor map's box is {width, 1}.
-__device__ __forceinline__ void tma_gather4(uint32_t dst, const void* tmap, int c0, int r0, int r1, int r2, int r3,
-                                            uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
-        : "memory");
-}
-// Row scatter: four consecutive shared-memory rows go to rows r0..r3 of the tensor (bulk async group).
-__device__ __forceinline__ void tma_scatter4(const void* tmap, uint32_t src, int c0, int r0, int r1, int r2, int r3)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.global.shared::cta.tile::scatter4.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
-        ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(src), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
         : "memory");
 }
 // Linear bulk copies (no tensor map): `bytes` is a multiple of 16, both addresses are 16-byte aligned.
@@ -178,10 +150,6 @@ __device__ __forceinline__ void bulk_wait_group()
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src)
-{
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 // Arrive on an mbarrier once every cp.async this thread has issued so far has landed (the arrival is counted
 // in the barrier's initial count, hence "noinc").

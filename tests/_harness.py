@@ -102,19 +102,3 @@ def run_and_check(w: W.Workload, rows=None, batched=False, scale=1.0, check_grou
             assert_close(got, ref, ATOL32, RTOL32, what=f"{w.name}/{p.name} (fp32 bound)")
     stats["worst_ratio"] = worst
     return stats
-
-
-def sample_rows(w: W.Workload, r: np.ndarray, n_random: int = 512, seed: int = 0) -> np.ndarray:
-    """Rows for sampled full-size parity: first/last rows of every segment and of every 128-row tile edge,
-    plus seeded random rows."""
-    _, offsets, perm = oracle.group(r, w.C)
-    picks = set()
-    for c in range(w.C):
-        lo, hi = int(offsets[c]), int(offsets[c + 1])
-        for j in list(range(lo, min(hi, lo + 2))) + list(range(max(lo, hi - 2), hi)):
-            picks.add(int(perm[j]))
-        for j in range(lo + 127, hi, 128):
-            picks.update(int(perm[q]) for q in (j, min(j + 1, hi - 1)))
-    rng = np.random.default_rng(seed)
-    picks.update(int(i) for i in rng.integers(0, w.N, size=n_random))
-    return np.array(sorted(picks), dtype=np.int64)

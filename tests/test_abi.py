@@ -2,6 +2,8 @@
 argument validation returns error codes before anything is enqueued.  No GPU needed (no compute calls)."""
 import ctypes
 
+import pytest
+
 import paper_2603_15965_b200 as M
 from paper_2603_15965_b200.build import build_library
 
@@ -13,7 +15,7 @@ def test_library_builds_loads_and_exports_header_symbols():
     assert {"molora_route_vocab", "molora_route_composite", "molora_route_mlp", "molora_route_mlp_workspace_bytes", "molora_topk_softmax", "molora_apply_topk",
             "molora_apply_topk_workspace_bytes", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched", "molora_group_apply_batched",
             "molora_group_workspace_bytes", "molora_apply_workspace_bytes", "molora_route_gate_workspace_bytes",
-            "molora_version",
+            "molora_version", "molora_launch_count", "molora_debug_set",
             "molora_status_string"} <= set(names)
     for name in names:
         assert hasattr(lib, name), f"header declares {name} but the library does not export it"
@@ -69,9 +71,17 @@ def test_invalid_arguments_are_refused_before_any_launch():
     assert apply(N=-3) == 1
 
 
-def test_apply_workspace_sizes_and_refusal_without_it(monkeypatch):
-    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH", "MOLORA_STREAM_TILE"):
-        monkeypatch.delenv(k, raising=False)
+@pytest.fixture
+def default_kernels():
+    """The library's own kernel choices before and after the test (overrides are process-wide)."""
+    for k in M.TUNING_NAMES:
+        M.molora_debug_set(k, 0)
+    yield
+    for k in M.TUNING_NAMES:
+        M.molora_debug_set(k, 0)
+
+
+def test_apply_workspace_sizes_and_refusal_without_it(default_kernels):
     lib = M.load_library()
     fake = ctypes.c_void_p(0x1000)
     # only the two-launch small-tile kernels need scratch: fp32 partial shrink results [slice][N][rank].  They serve
@@ -93,9 +103,9 @@ def test_apply_workspace_sizes_and_refusal_without_it(monkeypatch):
     assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 64) > 0
     assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 16) == 0
     # the two-launch kernels can be forced for every rank, and then ask for their scratch
-    monkeypatch.setenv("MOLORA_SMALL_PATH", "twophase")
+    M.molora_debug_set("small_path", 2)
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 2 * 256 * 16 * 4
-    monkeypatch.delenv("MOLORA_SMALL_PATH")
+    M.molora_debug_set("small_path", 0)
     # a call for the two-launch kernels without its workspace is refused before anything is enqueued
     st = lib.molora_apply(fake, 64, fake, 64, M.BF16, 4, 64, 64, 64, fake, fake, 2, fake, fake, 1.0, None, 0, None, None)
     assert st == 3
@@ -106,11 +116,9 @@ def _desc(d_in, d_out, rank):
     return _ProjDescC(0x1000, d_in, 0x2000, d_out, 0x3000, 0x4000, d_in, d_out, rank, 1.0, None)
 
 
-def test_group_apply_one_call_launch_count_and_refusals(monkeypatch):
+def test_group_apply_one_call_launch_count_and_refusals(default_kernels):
     """Host arithmetic only: when molora_group_apply_batched is one launch, and that it validates both halves."""
     from paper_2603_15965_b200.binding import _ProjDescC
-    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH", "MOLORA_STREAM_TILE"):
-        monkeypatch.delenv(k, raising=False)
     lib = M.load_library()
 
     def one_launch(shapes, N, dt=M.BF16):
@@ -131,9 +139,9 @@ def test_group_apply_one_call_launch_count_and_refusals(monkeypatch):
     assert one_launch([(2048, 2048, 16)] * 8, 4096) == 0                # 400 MB: above the tcgen05 crossover
     assert one_launch([(2048, 2048, 16)], 4096, M.F32) == 0             # fp32 storage: CUDA-core kernel
     assert one_launch([(2048, 2040, 16)], 256) == 0                     # width not a multiple of 32: CUDA-core kernel
-    monkeypatch.setenv("MOLORA_SMALL_PATH", "twophase")
+    M.molora_debug_set("small_path", 2)
     assert one_launch([(2048, 2048, 16)], 4096) == 0
-    monkeypatch.delenv("MOLORA_SMALL_PATH")
+    M.molora_debug_set("small_path", 0)
     # refusals before any launch: null outputs, too many adapters, no projections, unsupported rank
     fake = ctypes.c_void_p(0x1000)
     arr = (_ProjDescC * 1)(_desc(64, 64, 16))

@@ -11,7 +11,7 @@ import oracle
 import paper_2603_15965_b200 as M
 from paper_2603_15965_b200 import workloads as W
 
-from _harness import (assert_close, dev_tensor, gpu_route, oracle_route, run_and_check, sample_rows, to_f64)
+from _harness import (assert_close, dev_tensor, gpu_route, oracle_route, run_and_check, to_f64)
 
 pytestmark = pytest.mark.gpu
 
@@ -20,20 +20,27 @@ pytestmark = pytest.mark.gpu
 # on every shape class, whatever the default choice is.
 KERNEL_MODES = {
     "default": {},
-    "tcgen05": {"MOLORA_UMMA_MIN_TOKENS": "1024"},                                  # tcgen05 from 1024 tokens
-    "stream": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "stream"},
+    "tcgen05": {"umma_min_tokens": 1024},                                          # tcgen05 from 1024 tokens
+    "stream": {"umma_min_tokens": 1000000, "small_path": 1},
     # rank 16 has two tile shapes in the streaming kernel (16 rows x 1024 columns, 32 rows x 512 columns)
-    "stream-short": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "stream", "MOLORA_STREAM_TILE": "16"},
-    "stream-tall": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "stream", "MOLORA_STREAM_TILE": "32"},
-    "twophase": {"MOLORA_UMMA_MIN_TOKENS": "1000000", "MOLORA_SMALL_PATH": "twophase"},
+    "stream-short": {"umma_min_tokens": 1000000, "small_path": 1, "stream_tile": 16},
+    "stream-tall": {"umma_min_tokens": 1000000, "small_path": 1, "stream_tile": 32},
+    "twophase": {"umma_min_tokens": 1000000, "small_path": 2},
 }
 
 
-def force_kernel(monkeypatch, mode):
-    for k in ("MOLORA_UMMA_MIN_TOKENS", "MOLORA_SMALL_PATH", "MOLORA_STREAM_TILE"):
-        monkeypatch.delenv(k, raising=False)
+def force_kernel(mode):
+    for k in M.TUNING_NAMES:
+        M.molora_debug_set(k, 0)
     for k, v in KERNEL_MODES[mode].items():
-        monkeypatch.setenv(k, v)
+        M.molora_debug_set(k, v)
+
+
+@pytest.fixture(autouse=True)
+def _default_kernels_afterwards():
+    yield
+    for k in M.TUNING_NAMES:
+        M.molora_debug_set(k, 0)
 
 
 # ------------------------------------------------------------------ the five configurations
@@ -63,12 +70,18 @@ def test_c5_multimodal_reduced_and_iid():
 
 
 @pytest.mark.parametrize("name", ["c4", "c5", "c5-iid"])
-def test_full_size_sampled_rows(name):
+def test_full_size_every_row(name):
+    # the full-size configurations in the launch configuration the benchmark times (one batched call): EVERY row of every
+    # projection against the oracle (a few seconds of oracle time on the machine's host cores)
     w = W.get(name)
-    r_ref, _ = oracle_route(w)
-    rows = sample_rows(w, r_ref, n_random=384)
-    stats = run_and_check(w, rows=rows, batched=(name == "c4"))
-    print(name, stats, "rows checked:", rows.size)
+    stats = run_and_check(w, batched=True)
+    print(name, stats)
+
+
+@pytest.mark.parametrize("name", ["f9-512", "f9-2048", "t9-95", "t9-80"])
+def test_sweep_workloads_full(name):
+    # the batch and skew sweeps of the benchmark (Figure 9 / Table 9 conditions: 4096 -> 4096, rank 64): every row
+    run_and_check(W.get(name), batched=True)
 
 
 # ------------------------------------------------------------------ routers
@@ -320,8 +333,8 @@ def test_kpass_per_sequence_baseline_matches_single_pass():
 
 # ------------------------------------------------------------------ tensor-core path (forced from 1024 tokens)
 @pytest.mark.parametrize("rank", [16, 32, 64])
-def test_tensor_path_segment_size_sweep(rank, monkeypatch):
-    force_kernel(monkeypatch, "tcgen05")
+def test_tensor_path_segment_size_sweep(rank):
+    force_kernel("tcgen05")
     # segment sizes straddle the 32-row path threshold, the 4-row gather groups and the 128-row tile
     sizes = [0, 1, 31, 32, 33, 63, 64, 65, 127, 128, 129, 130, 131, 255, 256, 257, 300, 385, 700]
     r = W.segment_sizes_routing(sizes)
@@ -333,14 +346,14 @@ def test_tensor_path_segment_size_sweep(rank, monkeypatch):
 @pytest.mark.parametrize("N,C,d_in,d_out,rank", [(3072, 1, 64, 64, 16), (3300, 3, 2048, 1024, 16),
                                                  (1800, 2, 6144, 2048, 32), (2048, 4, 128, 6144, 64),
                                                  (1280, 5, 4096, 256, 64)])
-def test_tensor_path_shapes(N, C, d_in, d_out, rank, monkeypatch):
-    force_kernel(monkeypatch, "tcgen05")
+def test_tensor_path_shapes(N, C, d_in, d_out, rank):
+    force_kernel("tcgen05")
     w = W.random_problem(N + rank, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.05)
     run_and_check(w, scale=0.75)
 
 
-def test_tensor_path_selector_exact_and_status_clean(monkeypatch):
-    force_kernel(monkeypatch, "tcgen05")
+def test_tensor_path_selector_exact_and_status_clean():
+    force_kernel("tcgen05")
     N, C, d_in, d_out, rank = 3200, 2, 128, 192, 16
     rng = np.random.default_rng(6)
     x = rng.integers(-8, 9, size=(N, d_in)).astype(np.float32)
@@ -403,8 +416,8 @@ def test_forward_host_matches_oracle(name):
 # ------------------------------------------------------------------ small-tile kernels: single-launch streaming and two-launch
 @pytest.mark.parametrize("mode", ["stream-short", "stream-tall", "twophase"])
 @pytest.mark.parametrize("rank", [16, 32, 64])
-def test_decode_path_segment_size_sweep(rank, mode, monkeypatch):
-    force_kernel(monkeypatch, mode)
+def test_decode_path_segment_size_sweep(rank, mode):
+    force_kernel(mode)
     sizes = [0, 1, 7, 15, 16, 17, 31, 32, 33, 47, 64, 65, 97]
     r = W.segment_sizes_routing(sizes)
     assert r.size < 1024
@@ -420,8 +433,8 @@ def test_decode_path_segment_size_sweep(rank, mode, monkeypatch):
                                                  (1500, 3, 1056, 2592, 16),   # more tiles than CTAs x items, ragged chunks
                                                  (5000, 4, 512, 512, 32)])    # several items per persistent CTA
 @pytest.mark.parametrize("mode", ["stream-short", "stream-tall", "twophase"])
-def test_decode_path_shapes(N, C, d_in, d_out, rank, mode, monkeypatch):
-    force_kernel(monkeypatch, mode)
+def test_decode_path_shapes(N, C, d_in, d_out, rank, mode):
+    force_kernel(mode)
     w = W.random_problem(N + rank + 7, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.1 if N > 10 else 0.0)
     run_and_check(w)
 
@@ -460,11 +473,11 @@ def test_route_gate_tensor_core_paths(N, d, C):
 # ------------------------------------------------------------------ seeded random shapes across every kernel path
 @pytest.mark.parametrize("mode", ["default", "tcgen05", "stream-short", "stream-tall", "twophase"])
 @pytest.mark.parametrize("seed", range(24))
-def test_random_shapes_all_paths(seed, mode, monkeypatch):
+def test_random_shapes_all_paths(seed, mode):
     # token counts on both sides of the path switches (1024 / 1280 tokens), adapter counts on both sides of the
     # 64-adapter switch, ranks of every kernel, widths that are multiples of 8 / 32 / 64, skewed routing, unrouted
     # tokens; every shape with the default kernel choice and with each bf16 kernel forced
-    force_kernel(monkeypatch, mode)
+    force_kernel(mode)
     rng = np.random.default_rng(1000 + seed)
     N = int(rng.choice([1, 17, 130, 700, 1023, 1024, 1279, 1280, 1792, 2600, 3072, 3500]))
     C = int(rng.choice([1, 2, 5, 8, 33, 70]))
@@ -505,10 +518,10 @@ def test_route_gate_random_shapes_all_kernels(seed):
 
 @pytest.mark.parametrize("mode", ["default", "tcgen05"])
 @pytest.mark.parametrize("N", [300, 1400])
-def test_batched_apply_mixed_ranks_and_paths(N, mode, monkeypatch):
+def test_batched_apply_mixed_ranks_and_paths(N, mode):
     # one batched call whose projections need different kernels: ranks 16 / 32 / 64 (tcgen05, streaming or two-launch
     # kernels), rank 8 and a width that is only a multiple of 8 (CUDA-core kernel); shared routing
-    force_kernel(monkeypatch, mode)
+    force_kernel(mode)
     rng = np.random.default_rng(N)
     C = 6
     r = rng.integers(0, C, size=N).astype(np.int32)
@@ -580,8 +593,8 @@ def test_route_mlp_feeds_group_and_apply():
                                                         (3300, 4, 2, 512, 256, 16, "tcgen05"),
                                                         (200, 6, 3, 128, 96, 8, "default"),      # CUDA-core kernel (rank 8)
                                                         (500, 5, 1, 64, 64, 32, "default")])     # k = 1: weight exactly 1
-def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode, monkeypatch):
-    force_kernel(monkeypatch, mode)
+def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode):
+    force_kernel(mode)
     rng = np.random.default_rng(N + C + k)
     w_ = W.random_problem(500 + N, N, C, d_in, d_out, rank, "bf16")
     p = w_.projections[0]
@@ -633,8 +646,8 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode, monk
     (1025, 4, [(256, 192, 32)], "twophase"),                                    # one token too many: grouping launch + 2
     (300, 7, [(4096, 512, 64)], "default"), (77, 3, [(512, 4096, 64), (512, 512, 64)], "default"),   # rank 64: two-launch, on chip
 ])
-def test_group_apply_one_call_matches_oracle_and_group(N, C, shapes, mode, monkeypatch):
-    force_kernel(monkeypatch, mode)
+def test_group_apply_one_call_matches_oracle_and_group(N, C, shapes, mode):
+    force_kernel(mode)
     rng = np.random.default_rng(N * 31 + C)
     p = rng.dirichlet(np.full(C, 0.6))
     r = rng.choice(C, size=N, p=p).astype(np.int32)

@@ -357,11 +357,30 @@ def test_apply_rows_subset_is_exact():
 
 
 def test_thread_count_does_not_change_results():
-    w = _small(17, N=50)
-    p = w.projections[0]
-    h1, _ = oracle.apply(w.inputs["x"], p.y, p.A, p.B, w.r)
-    h2, _ = oracle.apply(w.inputs["x"][::-1][::-1], p.y, p.A, p.B, w.r)
-    assert np.array_equal(h1, h2) and oracle.num_threads() >= 1
+    # the oracle is parallel over tokens only, so the number of OpenMP threads must not change a single bit: run the
+    # same seeded problem in two fresh processes with 1 and with 4 threads and compare digests of every output
+    import subprocess
+    import sys
+    code = (
+        "import hashlib, sys, numpy as np, oracle\n"
+        "from paper_2603_15965_b200 import workloads as W\n"
+        "w = W.random_problem(17, 203, 5, 96, 72, 8, 'bf16', unrouted_frac=0.1)\n"
+        "p = w.projections[0]\n"
+        "G = np.random.default_rng(3).standard_normal((96, 5)).astype(np.float32)\n"
+        "h, n = oracle.apply(w.inputs['x'], p.y, p.A, p.B, w.r)\n"
+        "hk, nk = oracle.apply_perseq_kpass(w.inputs['x'], p.y, p.A, p.B, w.r)\n"
+        "r, z, m = oracle.route_gate(w.inputs['x'], G)\n"
+        "d = hashlib.sha256()\n"
+        "for a in (h, hk, r, z, m): d.update(np.ascontiguousarray(a).tobytes())\n"
+        "print(oracle.num_threads(), n, nk, d.hexdigest())\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    outs = []
+    for threads in ("1", "4"):
+        env = dict(os.environ, OMP_NUM_THREADS=threads, PYTHONPATH=root)
+        res = subprocess.run([sys.executable, "-c", code], env=env, cwd=root, capture_output=True, text=True, check=True)
+        outs.append(res.stdout.split())
+    assert outs[0][0] == "1" and outs[1][0] == "4"              # the two runs really used different thread counts
+    assert outs[0][1:] == outs[1][1:]
 
 
 # ------------------------------------------------------------------ workload generator sanity (inputs only)
