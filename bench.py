@@ -259,7 +259,7 @@ def measure(name, args, env, headline):
     need = molora_apply_batched_workspace_bytes(sets[0]["packed"][0], N, C)
     shared["apply_ws"] = torch.zeros(need, dtype=torch.uint8, device="cuda") if need else None
     arr0, n0, c0, dt0 = sets[0]["packed"]
-    fused = bool(lib.molora_group_apply_skips_group_launch(arr0, len(arr0), dt0, n0))   # grouping inside the apply kernels
+    fused = bool(lib.molora_group_apply_skips_group_launch(arr0, len(arr0), dt0, n0, c0))   # grouping inside the apply kernels
     for s in sets:
         s["calls"] = marshal_step(lib, w, s, shared, stream.cuda_stream)
 

@@ -188,14 +188,20 @@ molora_status_t molora_group(const int32_t *r, int64_t N, int32_t C, int32_t *co
  * A   device [C, d_in, rank] of type dt, dense;  B  device [C, rank, d_out] of type dt, dense
  * offsets, perm   device outputs of molora_group for the same N, C (read on the device only)
  * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes, 16-byte aligned (NULL if
- *                 that is 0).  Only the two-launch small-tile kernels write it (fp32 partial shrink results
- *                 [slice][N][rank]): bf16 calls of rank 64 below 1280 tokens (with one or two rank-64 projections in
- *                 the call) and, with more than 64 adapters, the short segments of larger rank-64 calls.
- *                 MOLORA_ERR_WORKSPACE if those kernels are needed and ws is NULL, misaligned or too small.
+ *                 that is 0).  Two kernels use it.  The job-list kernel (bf16, at most 1024 tokens, few tiles per SM:
+ *                 decode-sized calls) keeps counters and fp32 partial shrink results there: ws must be ZERO-FILLED
+ *                 before its first use; every call leaves its control words zero again, so the same ws can be passed
+ *                 to any number of later calls (of any shape) without clearing.  Calls that share one ws must not
+ *                 overlap on the GPU.  If a call reports MOLORA_DEV_TIMEOUT, clear ws before using it again.  The
+ *                 two-launch small-tile kernels (bf16 rank 64 below 1280 tokens with one or two rank-64 projections in
+ *                 the call; with more than 64 adapters also the short segments of larger rank-64 calls) keep partial
+ *                 shrink results [slice][N][rank] behind that.
+ *                 MOLORA_ERR_WORKSPACE if ws is needed and NULL, misaligned or too small.
  * dev_status      device uint32 or NULL; MOLORA_DEV_TIMEOUT is OR-ed in if a bounded wait inside a kernel gave
  *                 up (the kernel then returns without hanging; y is incomplete)
  * The kernel variant is chosen per call on the host from rank, token count and bytes (tcgen05 tiles of 128 rows
- * for large calls, a single-launch streaming kernel with 32-row tiles below that, CUDA cores for fp32 storage,
+ * for large calls, a single-launch streaming kernel with 32-row tiles below that, a job-list kernel with 16-row
+ * tiles whose CTAs share chunk-sized shrink and expand jobs for decode-sized calls, CUDA cores for fp32 storage,
  * rank 8 and odd widths) and per segment on the device from the segment sizes; the paper picks its tile shape
  * from the histogram too (Eq. 12-13). */
 size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t d_out, int32_t rank);
@@ -228,20 +234,22 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t *projs, int32_t P,
  * molora_group(r, ...) followed by molora_apply_batched(projs, ...) on its outputs, with the arguments, results
  * (counts, offsets and perm are written, bit-equal to molora_group's), status bits and error behaviour of those two
  * calls; ws / ws_bytes as for molora_apply_batched.  When every projection of the call runs on the single-launch
- * streaming kernel with one rank (bf16, at most 4096 tokens, below the tcgen05 crossover) the whole call is ONE
- * launch: every CTA builds the grouping in its shared memory before its first copy request, which saves the
- * grouping launch; the two-launch small-tile kernels do the same for at most 1024 tokens; otherwise the grouping
- * launch and the apply launches are enqueued in stream order. */
+ * streaming kernel or on the job-list kernel with one rank (bf16, at most 4096 / 1024 tokens, below the tcgen05
+ * crossover) the whole call is ONE launch: every CTA builds the grouping in its shared memory before its first copy
+ * request, which saves the grouping launch; the two-launch small-tile kernels do the same for at most 1024 tokens;
+ * otherwise the grouping launch and the apply launches are enqueued in stream order. */
 molora_status_t molora_group_apply_batched(const int32_t *r, int64_t N, int32_t C, int32_t *counts, int32_t *offsets,
                                            int32_t *perm, const molora_proj_desc_t *projs, int32_t P,
                                            molora_dtype_t dt, void *ws, size_t ws_bytes, uint32_t *dev_status,
                                            void *stream);
-/* 1 if that call is a single launch for these projections (host array, as above) and this token count, else 0;
- * pure host arithmetic, for callers that count launches. */
-int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N);
+/* 1 if that call is a single launch for these projections (host array, as above), this token count and this number
+ * of adapters, else 0; pure host arithmetic, for callers that count launches. */
+int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N,
+                                         int32_t C);
 /* 1 if that call needs no separate grouping launch: the single launch above, or the two-launch small-tile kernels
  * grouping on chip (bf16, one rank, at most 1024 tokens; their launches are then the two of molora_apply_batched). */
-int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N);
+int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N,
+                                              int32_t C);
 
 /* ---------------------------------------------------------------------------------------------
  * Top-k weighted routing (Eq. 8): w_i = softmax(TopK(z_i, k)), delta h_i = sum_j w_ij x_i A^(j) B^(j).
@@ -254,7 +262,8 @@ int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t *projs, i
  * a pass every row of y is touched by one adapter only, so there are no conflicting updates and the result is
  * deterministic; y is rounded to its storage type once per pass.
  *   projs    HOST array of P descriptors as for molora_apply_batched (their row_scale is ignored)
- *   ws       device scratch of at least molora_apply_topk_workspace_bytes(projs, P, N, C) bytes, 256-byte aligned */
+ *   ws       device scratch of at least molora_apply_topk_workspace_bytes(projs, P, N, C) bytes, 256-byte aligned,
+ *            zero-filled before its first use (see molora_apply) */
 molora_status_t molora_topk_softmax(const float *logits, int64_t N, int32_t C, int32_t k, int32_t *idx_out, float *w_out,
                                     void *stream);
 size_t molora_apply_topk_workspace_bytes(const molora_proj_desc_t *projs, int32_t P, int64_t N, int32_t C);
@@ -287,7 +296,8 @@ molora_status_t molora_selftest_bounded_wait(uint32_t *dev_status, int64_t limit
  *              MOLORA_ROUTE_GIVEN: route_src_host = r int32[N]
  * projs        HOST array of P descriptors (1 <= P <= MOLORA_MAX_PROJECTIONS); projections whose x_host
  *              pointers are equal share one staged copy
- * arena        device scratch of at least molora_forward_host_arena_bytes(...) bytes, 256-byte aligned
+ * arena        device scratch of at least molora_forward_host_arena_bytes(...) bytes, 256-byte aligned, zero-filled
+ *              before its first use (it holds the apply workspace, see molora_apply)
  * dev_status   device uint32 or NULL (as for the individual calls)
  * Errors are detected before anything is enqueued, as for the individual calls. */
 typedef enum { MOLORA_ROUTE_VOCAB = 0, MOLORA_ROUTE_GATE = 1, MOLORA_ROUTE_GIVEN = 2 } molora_router_t;

@@ -100,9 +100,9 @@ def load_library():
     lib.molora_group_apply_batched.argtypes = [vp, i64, i32, vp, vp, vp, ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, vp,
                                                sz, vp, vp]
     lib.molora_group_apply_batched.restype = ctypes.c_int
-    lib.molora_group_apply_is_one_launch.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64]
+    lib.molora_group_apply_is_one_launch.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64, i32]
     lib.molora_group_apply_is_one_launch.restype = i32
-    lib.molora_group_apply_skips_group_launch.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64]
+    lib.molora_group_apply_skips_group_launch.argtypes = [ctypes.POINTER(_ProjDescC), i32, ctypes.c_int, i64, i32]
     lib.molora_group_apply_skips_group_launch.restype = i32
     lib.molora_forward_host_arena_bytes.restype = sz
     lib.molora_forward_host_arena_bytes.argtypes = [ctypes.POINTER(_HostProjC), i32, ctypes.c_int, i64, i32, ctypes.c_int,
@@ -226,7 +226,7 @@ def molora_route_mlp(x: torch.Tensor, W1: torch.Tensor, b1: Optional[torch.Tenso
         r_out = torch.empty(N, dtype=torch.int32, device=x.device)
     need = molora_route_mlp_workspace_bytes(_dtype_code(x), d, H, C)
     if ws is None and need > 0:
-        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+        ws = torch.zeros(need, dtype=torch.uint8, device=x.device)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_route_mlp", lib.molora_route_mlp(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(W1), _ptr(b1), H, _ptr(W2),
                                                     _ptr(b2), C, _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
@@ -256,7 +256,7 @@ def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Ten
         raise ValueError("logits_out: expected contiguous fp32 [N, C]")
     need = molora_route_gate_workspace_bytes(_dtype_code(x), d, C)
     if ws is None and need > 0:
-        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+        ws = torch.zeros(need, dtype=torch.uint8, device=x.device)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_route_gate", lib.molora_route_gate(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(G), _ptr(bias), C,
                                                       _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out), _ptr(ws),
@@ -312,7 +312,7 @@ def molora_group(r: torch.Tensor, C: int, counts: Optional[torch.Tensor] = None,
     perm = torch.empty(max(N, 1), dtype=torch.int32, device=dev) if perm is None else _i32_dev(perm, "perm")
     need = molora_group_workspace_bytes(N, C)
     if ws is None and need > 0:
-        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        ws = torch.zeros(need, dtype=torch.uint8, device=dev)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_group", lib.molora_group(_ptr(r), N, C, _ptr(counts), _ptr(offsets), _ptr(perm), _ptr(ws), ws_bytes,
                                             _ptr(dev_status), _stream(stream)))
@@ -342,7 +342,7 @@ def molora_apply(x: torch.Tensor, y: torch.Tensor, A: torch.Tensor, B: torch.Ten
         raise ValueError("offsets must have C + 1 entries")
     need = molora_apply_workspace_bytes(N, C, d_in, d_out, rank)
     if ws is None and need > 0:
-        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+        ws = torch.zeros(need, dtype=torch.uint8, device=x.device)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_apply", lib.molora_apply(_ptr(x), ldx, _ptr(y), ldy, dt, N, d_in, d_out, rank, _ptr(A), _ptr(B), C,
                                             _ptr(_i32_dev(offsets, "offsets")), _ptr(_i32_dev(perm, "perm")),
@@ -399,7 +399,7 @@ def molora_apply_batched(projs, offsets: torch.Tensor, perm: torch.Tensor, ws: O
     if ws is None:
         need = molora_apply_batched_workspace_bytes(arr, N, C)
         if need > 0:
-            ws = torch.empty(need, dtype=torch.uint8, device=offsets.device)
+            ws = torch.zeros(need, dtype=torch.uint8, device=offsets.device)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_apply_batched", lib.molora_apply_batched(arr, len(arr), dt, N, C, _ptr(offsets), _ptr(perm),
                                                             _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
@@ -424,7 +424,7 @@ def molora_group_apply_batched(r: torch.Tensor, projs, C: Optional[int] = None, 
     if ws is None:
         need = molora_apply_batched_workspace_bytes(arr, N, C)
         if need > 0:
-            ws = torch.empty(need, dtype=torch.uint8, device=dev)
+            ws = torch.zeros(need, dtype=torch.uint8, device=dev)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_group_apply_batched",
            lib.molora_group_apply_batched(_ptr(r), N, C, _ptr(counts), _ptr(offsets), _ptr(perm), arr, len(arr), dt, _ptr(ws),
@@ -455,7 +455,7 @@ def molora_apply_topk(projs, idx: torch.Tensor, w: torch.Tensor, C: int, ws: Opt
     k = idx.shape[0]
     need = int(lib.molora_apply_topk_workspace_bytes(arr, len(arr), N, C))
     if ws is None:
-        ws = torch.empty(need + 256, dtype=torch.uint8, device=idx.device)
+        ws = torch.zeros(need + 256, dtype=torch.uint8, device=idx.device)
     off = (-ws.data_ptr()) % 256
     _check("molora_apply_topk", lib.molora_apply_topk(arr, len(arr), dt, N, C, k, _ptr(idx.contiguous()), _ptr(w.contiguous()),
                                                       ctypes.c_void_p(ws.data_ptr() + off), ws.numel() - off,

@@ -84,6 +84,17 @@ bool small_path_is_stream(int32_t rank, int64_t N, int same_rank)
     return rank == 16 || rank == 32 || same_rank > 2;
 }
 
+// The job-list kernel takes decode-sized calls: at most 1024 tokens, and few enough 16-row tiles over the projections of
+// the rank that one CTA per (tile, projection) would leave the launch waiting for its longest items -- the same bound
+// under which the streaming kernel would switch to its short tile.
+constexpr double kJobsFill = 1.25;
+bool use_jobs(const molora_proj_desc_t& p, molora_dtype_t dt, int64_t N, int32_t C, int same_rank)
+{
+    if (!jobs_eligible(p, dt, N)) return false;
+    if (const int64_t forced = tune(kTuneSmallPath)) return forced == 3;
+    return (double)(ceil_div64(N, 16) + C) * same_rank <= kJobsFill * sm_count();
+}
+
 bool rank_supported(int r) { return r == 8 || r == 16 || r == 32 || r == 64; }
 
 molora_status_t check_proj(const molora_proj_desc_t& p, molora_dtype_t dt)
@@ -206,17 +217,27 @@ molora_status_t molora_group(const int32_t* r, int64_t N, int32_t C, int32_t* co
 
 size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t d_out, int32_t rank)
 {
-    // Only the two-launch small-tile kernels need scratch (their partial shrink results); see the path selection at
-    // the top of this file.  The element type is not known here, so the figure assumes bf16 (fp32 calls need none).
-    if (N <= 0 || d_in <= 0 || d_out <= 0 || (rank != 16 && rank != 32 && rank != 64)) return 0;
+    // Two kernels need scratch: the job-list kernel (control words + partial shrink results; decode-sized bf16 calls) and
+    // the two-launch small-tile kernels (partial shrink results).  Which one runs depends on the other projections of
+    // the call, which are not known here, so the figure covers both where both are possible; the element type is not
+    // known either, so it assumes bf16 (fp32 calls need none).
+    if (N <= 0 || C < 1 || d_in <= 0 || d_out <= 0 || (rank != 16 && rank != 32 && rank != 64)) return 0;
     if ((d_in % 32) != 0 || (d_out % 32) != 0) return 0;
-    if (small_path_is_stream(rank, N, 0)) return 0;
+    size_t need = 0;
+    molora_proj_desc_t probe{};
+    probe.d_in = d_in;
+    probe.d_out = d_out;
+    probe.rank = rank;
+    const int64_t small = tune(kTuneSmallPath);
+    if (jobs_eligible(probe, MOLORA_BF16, N) && (small == 0 || small == 3)) need += jobs_control_bytes() + jobs_partial_bytes(N, C, d_in, rank);
+    if (small == 3 && need > 0) return need;
+    if (small_path_is_stream(rank, N, 0)) return need;
     // two-launch kernels: needed unless the tcgen05 kernel is certain to take every segment (for ranks 16 and 32 that
     // depends on the other projections of the call, which are not known here)
     const int64_t forced = forced_umma_min_tokens();
     const bool umma_certain = forced > 0 ? N >= forced : (rank == 64 && N >= kUmmaMinTokensR64);
-    if (umma_certain && C <= kUmmaAllSegmentsMaxC && (d_in % 64) == 0 && (d_out % 64) == 0) return 0;
-    return decode_workspace_bytes(N, d_in, rank);
+    if (umma_certain && C <= kUmmaAllSegmentsMaxC && (d_in % 64) == 0 && (d_out % 64) == 0) return need;
+    return need + decode_workspace_bytes(N, d_in, rank);
 }
 
 namespace {
@@ -226,9 +247,12 @@ namespace {
 struct ApplyPlan {
     molora_proj_desc_t tc[MOLORA_MAX_PROJECTIONS], sc[MOLORA_MAX_PROJECTIONS], dc[MOLORA_MAX_PROJECTIONS], cc[MOLORA_MAX_PROJECTIONS];
     molora_proj_desc_t small_sc[MOLORA_MAX_PROJECTIONS], small_dc[MOLORA_MAX_PROJECTIONS], small_cc[MOLORA_MAX_PROJECTIONS];
-    int n_tc = 0, n_sc = 0, n_dc = 0, n_cc = 0, n_small_sc = 0, n_small_dc = 0, n_small_cc = 0;
+    molora_proj_desc_t jc[3][MOLORA_MAX_PROJECTIONS];     // job-list kernel, by rank (16, 32, 64)
+    int n_tc = 0, n_sc = 0, n_dc = 0, n_cc = 0, n_small_sc = 0, n_small_dc = 0, n_small_cc = 0, n_jc[3] = {0, 0, 0};
     int32_t min_rows = 1;          // segments with at least this many rows go to the tcgen05 kernel
-    size_t ws_need = 0;            // scratch of the two-launch kernels (the larger of their two uses in this call)
+    // workspace layout: [control part of the job-list kernel | its partials, by rank | scratch of the two-launch kernels]
+    size_t jobs_ctl = 0, jobs_part_off[3] = {0, 0, 0}, jobs_part[3] = {0, 0, 0}, decode_off = 0;
+    size_t ws_need = 0;
 };
 
 // Argument checks, kernel split and workspace check of molora_apply_batched: everything that can refuse the call,
@@ -256,6 +280,7 @@ molora_status_t plan_apply(const molora_proj_desc_t* projs, int32_t P, molora_dt
     for (int i = 0; i < P; ++i) {
         const int32_t rank = projs[i].rank;
         if (umma_eligible(projs[i], dt) && use_umma(rank, N, group_bytes[group_of(rank)])) pl.tc[pl.n_tc++] = projs[i];
+        else if (use_jobs(projs[i], dt, N, C, same_rank[group_of(rank)])) pl.jc[group_of(rank)][pl.n_jc[group_of(rank)]++] = projs[i];
         else if (decode_eligible(projs[i], dt)) {
             if (small_path_is_stream(rank, N, same_rank[group_of(rank)])) pl.sc[pl.n_sc++] = projs[i];
             else pl.dc[pl.n_dc++] = projs[i];
@@ -274,7 +299,18 @@ molora_status_t plan_apply(const molora_proj_desc_t* projs, int32_t P, molora_dt
     size_t need_dc = 0, need_small = 0;
     for (int i = 0; i < pl.n_dc; ++i) need_dc += decode_workspace_bytes(N, pl.dc[i].d_in, pl.dc[i].rank);
     for (int i = 0; i < pl.n_small_dc; ++i) need_small += decode_workspace_bytes(N, pl.small_dc[i].d_in, pl.small_dc[i].rank);
-    pl.ws_need = N > 0 ? std::max(need_dc, need_small) : 0;
+    size_t off = 0;
+    if (N > 0 && pl.n_jc[0] + pl.n_jc[1] + pl.n_jc[2] > 0) {
+        pl.jobs_ctl = jobs_control_bytes();
+        off = pl.jobs_ctl;
+        for (int k = 0; k < 3; ++k) {
+            pl.jobs_part_off[k] = off;
+            for (int i = 0; i < pl.n_jc[k]; ++i) pl.jobs_part[k] += jobs_partial_bytes(N, C, pl.jc[k][i].d_in, pl.jc[k][i].rank);
+            off += pl.jobs_part[k];
+        }
+    }
+    pl.decode_off = off;
+    pl.ws_need = N > 0 ? off + std::max(need_dc, need_small) : 0;
     if (pl.ws_need > 0 && (ws == nullptr || ws_bytes < pl.ws_need || !aligned16(ws))) return MOLORA_ERR_WORKSPACE;
     return MOLORA_OK;
 }
@@ -283,14 +319,21 @@ molora_status_t enqueue_apply(const ApplyPlan& pl, molora_dtype_t dt, int64_t N,
                               const int32_t* perm, void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s)
 {
     molora_status_t st = MOLORA_OK;
-    if (pl.n_tc > 0) {
+    char* base = static_cast<char*>(ws);
+    void* dws = ws != nullptr ? base + pl.decode_off : nullptr;              // scratch of the two-launch kernels
+    const size_t dws_bytes = ws != nullptr && ws_bytes > pl.decode_off ? ws_bytes - pl.decode_off : 0;
+    for (int k = 0; k < 3 && st == MOLORA_OK; ++k)
+        if (pl.n_jc[k] > 0)
+            st = launch_apply_jobs(pl.jc[k], pl.n_jc[k], N, C, offsets, perm, base, base + pl.jobs_part_off[k], pl.jobs_part[k],
+                                   dev_status, s);
+    if (st == MOLORA_OK && pl.n_tc > 0) {
         st = launch_apply_umma(pl.tc, pl.n_tc, N, C, offsets, perm, dev_status, pl.min_rows, s);
         if (st == MOLORA_OK && pl.n_small_sc > 0) st = launch_apply_stream(pl.small_sc, pl.n_small_sc, N, C, offsets, perm, pl.min_rows, dev_status, s);
-        if (st == MOLORA_OK && pl.n_small_dc > 0) st = launch_apply_decode(pl.small_dc, pl.n_small_dc, N, C, offsets, perm, pl.min_rows, ws, ws_bytes, dev_status, s);
+        if (st == MOLORA_OK && pl.n_small_dc > 0) st = launch_apply_decode(pl.small_dc, pl.n_small_dc, N, C, offsets, perm, pl.min_rows, dws, dws_bytes, dev_status, s);
         if (st == MOLORA_OK && pl.n_small_cc > 0) st = launch_apply_rowtile(pl.small_cc, pl.n_small_cc, dt, N, C, offsets, perm, pl.min_rows, s);
     }
     if (st == MOLORA_OK && pl.n_sc > 0) st = launch_apply_stream(pl.sc, pl.n_sc, N, C, offsets, perm, INT32_MAX, dev_status, s);
-    if (st == MOLORA_OK && pl.n_dc > 0) st = launch_apply_decode(pl.dc, pl.n_dc, N, C, offsets, perm, INT32_MAX, ws, ws_bytes, dev_status, s);
+    if (st == MOLORA_OK && pl.n_dc > 0) st = launch_apply_decode(pl.dc, pl.n_dc, N, C, offsets, perm, INT32_MAX, dws, dws_bytes, dev_status, s);
     if (st == MOLORA_OK && pl.n_cc > 0) st = launch_apply_rowtile(pl.cc, pl.n_cc, dt, N, C, offsets, perm, INT32_MAX, s);
     return st;
 }
@@ -306,38 +349,42 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
     return enqueue_apply(pl, dt, N, C, offsets, perm, ws, ws_bytes, dev_status, static_cast<cudaStream_t>(stream));
 }
 
-// How molora_group_apply_batched runs: 1 = one launch (every projection on the streaming kernel, one rank, at most 4096
-// tokens), 2 = the two-launch kernels with the grouping inside (one rank, at most 1024 tokens), 0 = the grouping launch
-// followed by the apply launches.
-static int group_apply_mode(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
+// How molora_group_apply_batched runs: 1 = one launch of the streaming kernel (every projection on it, one rank, at
+// most 4096 tokens), 3 = one launch of the job-list kernel (every projection on it, one rank), 2 = the two-launch kernels
+// with the grouping inside (one rank, at most 1024 tokens), 0 = the grouping launch followed by the apply launches.
+static int group_apply_mode(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C)
 {
     if (dt != MOLORA_BF16 || N < 1) return 0;
     double bytes = 0.0;
-    bool same = true, stream = true, twophase = true;
+    bool same = true, stream = true, twophase = true, jobs = true;
     for (int i = 0; i < P; ++i) {
         same = same && projs[i].rank == projs[0].rank && decode_eligible(projs[i], dt);
         if (!same) return 0;
+        const bool jb = use_jobs(projs[i], dt, N, C, P);
         const bool st = small_path_is_stream(projs[i].rank, N, P);
-        stream = stream && st;
-        twophase = twophase && !st;
+        jobs = jobs && jb;
+        stream = stream && !jb && st;
+        twophase = twophase && !jb && !st;
         if (umma_eligible(projs[i], dt)) bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
     }
     if (use_umma(projs[0].rank, N, bytes)) return 0;
+    if (jobs) return 3;
     if (stream && group_apply_stream_eligible(N)) return 1;
     if (twophase && group_apply_decode_eligible(N)) return 2;
     return 0;
 }
 
-int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
+int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C)
 {
-    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 1) return 0;
-    return group_apply_mode(projs, P, dt, N) == 1 ? 1 : 0;
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 1 || C < 1) return 0;
+    const int mode = group_apply_mode(projs, P, dt, N, C);
+    return mode == 1 || mode == 3 ? 1 : 0;
 }
 
-int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N)
+int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C)
 {
-    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 1) return 0;
-    return group_apply_mode(projs, P, dt, N) != 0 ? 1 : 0;
+    if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 1 || C < 1) return 0;
+    return group_apply_mode(projs, P, dt, N, C) != 0 ? 1 : 0;
 }
 
 molora_status_t molora_group_apply_batched(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets,
@@ -358,9 +405,17 @@ molora_status_t molora_group_apply_batched(const int32_t* r, int64_t N, int32_t 
     // When every projection of the call runs on the streaming kernel (or on the two-launch kernels) with one rank, the
     // CTAs of those kernels do the grouping themselves.  Otherwise the two calls, in stream order.  Whatever could
     // refuse the call (the workspace of the two-launch kernels included) is checked before the first launch.
-    const int mode = group_apply_mode(projs, P, dt, N);
+    const int mode = group_apply_mode(projs, P, dt, N, C);
     if (mode == 1)
         return launch_group_apply_stream(r, projs, P, N, C, counts, offsets, perm, dev_status, static_cast<cudaStream_t>(stream));
+    if (mode == 3) {
+        size_t part = 0;
+        for (int i = 0; i < P; ++i) part += jobs_partial_bytes(N, C, projs[i].d_in, projs[i].rank);
+        const size_t ctl = jobs_control_bytes();
+        if (ws == nullptr || ws_bytes < ctl + part || !aligned16(ws)) return MOLORA_ERR_WORKSPACE;
+        return launch_group_apply_jobs(r, projs, P, N, C, counts, offsets, perm, ws, static_cast<char*>(ws) + ctl, part, dev_status,
+                                       static_cast<cudaStream_t>(stream));
+    }
     if (mode == 2) {
         size_t need = 0;
         for (int i = 0; i < P; ++i) need += decode_workspace_bytes(N, projs[i].d_in, projs[i].rank);
@@ -413,15 +468,16 @@ TopkPlan plan_topk(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_
 {
     auto a256 = [](size_t v) { return (v + 255) & ~(size_t)255; };
     TopkPlan pl;
-    size_t off = 0;
-    pl.counts = off;   off = a256(off + sizeof(int32_t) * (size_t)C);
-    pl.offsets = off;  off = a256(off + sizeof(int32_t) * (size_t)(C + 1));
-    pl.perm = off;     off = a256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
-    pl.apply_ws = off;
+    // the apply workspace comes first: its control words stay at the same place (and zero) whatever N and C are
+    pl.apply_ws = 0;
     pl.apply_ws_bytes = 0;
     for (int i = 0; i < P; ++i)
         pl.apply_ws_bytes += molora_apply_workspace_bytes(N, C, projs[i].d_in, projs[i].d_out, projs[i].rank);
-    pl.total = a256(off + pl.apply_ws_bytes);
+    size_t off = a256(pl.apply_ws_bytes);
+    pl.counts = off;   off = a256(off + sizeof(int32_t) * (size_t)C);
+    pl.offsets = off;  off = a256(off + sizeof(int32_t) * (size_t)(C + 1));
+    pl.perm = off;     off = a256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
+    pl.total = off;
     return pl;
 }
 }  // namespace
@@ -481,7 +537,12 @@ bool plan_host(const molora_host_proj_t* projs, int32_t P, molora_dtype_t dt, in
     if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 0 || C < 1 || C > MOLORA_MAX_ADAPTERS) return false;
     if (dt != MOLORA_F32 && dt != MOLORA_BF16) return false;
     const size_t e = dt == MOLORA_BF16 ? 2 : 4;
-    size_t off = 0;
+    // the apply workspace comes first: its control words stay at the same place (and zero) whatever the shapes are
+    pl.apply_ws = 0;
+    pl.apply_ws_bytes = 0;
+    for (int i = 0; i < P; ++i)
+        pl.apply_ws_bytes += molora_apply_workspace_bytes(N, C, projs[i].d_in, projs[i].d_out, projs[i].rank);
+    size_t off = align256(pl.apply_ws_bytes);
     pl.ids = off;      off = align256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
     pl.r = off;        off = align256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
     pl.counts = off;   off = align256(off + sizeof(int32_t) * (size_t)C);
@@ -492,11 +553,6 @@ bool plan_host(const molora_host_proj_t* projs, int32_t P, molora_dtype_t dt, in
         if (gate_proj < 0 || gate_proj >= P) return false;
         off = align256(off + route_gate_workspace_bytes(dt, projs[gate_proj].d_in, C));
     }
-    pl.apply_ws = off;
-    pl.apply_ws_bytes = 0;
-    for (int i = 0; i < P; ++i)
-        pl.apply_ws_bytes += molora_apply_workspace_bytes(N, C, projs[i].d_in, projs[i].d_out, projs[i].rank);
-    off = align256(off + pl.apply_ws_bytes);
     for (int i = 0; i < P; ++i) {
         pl.x_owner[i] = i;
         for (int j = 0; j < i; ++j)

@@ -284,6 +284,20 @@ molora_status_t launch_apply_decode(const molora_proj_desc_t* projs, int32_t P, 
                                     const int32_t* offsets, const int32_t* perm, int32_t max_rows, void* ws,
                                     size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
 
+// Job-list kernel for decode-sized calls (bf16, one rank per launch, at most 1024 tokens): one cooperative launch whose
+// CTAs share chunk-sized shrink and expand jobs; partial shrink results and per-tile counters live in the workspace.
+// ctl: jobs_control_bytes() bytes, zero before the first call and left zero by every call; part: the sum of
+// jobs_partial_bytes over the projections of the launch.
+bool jobs_eligible(const molora_proj_desc_t& p, molora_dtype_t dt, int64_t N);
+size_t jobs_control_bytes();
+size_t jobs_partial_bytes(int64_t N, int32_t C, int32_t d_in, int32_t rank);
+molora_status_t launch_apply_jobs(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C, const int32_t* offsets,
+                                  const int32_t* perm, void* ctl, void* part, size_t part_bytes, uint32_t* dev_status,
+                                  cudaStream_t s);
+molora_status_t launch_group_apply_jobs(const int32_t* r, const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
+                                        int32_t* counts, int32_t* offsets, int32_t* perm, void* ctl, void* part,
+                                        size_t part_bytes, uint32_t* dev_status, cudaStream_t s);
+
 molora_status_t launch_bounded_wait_selftest(uint32_t* dev_status, int64_t limit_cycles, int32_t* result, cudaStream_t s);
 
 // Path selection: a segment goes to the tensor-core kernel when it has at least kUmmaMinRows rows and the call
@@ -351,6 +365,19 @@ inline int device_slot()
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
     return dev % kMaxDevices;
+}
+
+inline int sm_count()
+{
+    static int sms_dev[kMaxDevices] = {};
+    int& sms = sms_dev[device_slot()];
+    if (sms == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            return 148;                           // no device visible (host-only callers of the size queries): B200's count
+        sms = n;
+    }
+    return sms;
 }
 
 inline molora_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? MOLORA_OK : MOLORA_ERR_CUDA; }

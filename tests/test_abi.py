@@ -84,16 +84,28 @@ def default_kernels():
 def test_apply_workspace_sizes_and_refusal_without_it(default_kernels):
     lib = M.load_library()
     fake = ctypes.c_void_p(0x1000)
-    # only the two-launch small-tile kernels need scratch: fp32 partial shrink results [slice][N][rank].  They serve
-    # rank 64 below 1280 tokens:
+    # Two kernels need scratch.  (1) The two-launch small-tile kernels: fp32 partial shrink results [slice][N][rank];
+    # forced here so that their figure stands alone:
+    M.molora_debug_set("small_path", 2)
     # 256 tokens, d_in 2048, rank 64 -> 4 slices of 512 columns -> 4 * 256 * 64 * 4 bytes
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 64) == 4 * 256 * 64 * 4
     assert M.molora_apply_workspace_bytes(256, 8, 6144, 2048, 64) == 12 * 256 * 64 * 4
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 2 * 256 * 16 * 4
+    M.molora_debug_set("small_path", 0)
+    # (2) The job-list kernel (decode-sized calls: at most 1024 tokens, ranks 16 / 32 / 64): control words + partials.
+    M.molora_debug_set("small_path", 3)
+    ctl = 3 * (256 + 8 * (1024 // 16 + 256) * 4)                       # three ranks x (done counter + 8 x 320 tile counters)
+    ctl += 256 - ctl % 256
+    # rank 16, d_in 2048: a full x-group (4 members) gets 384-column chunks -> 6 chunks; 256 / 16 + 8 = 24 tiles at most
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == ctl + 24 * 6 * 16 * 16 * 4
+    assert M.molora_apply_workspace_bytes(1025, 8, 2048, 2048, 16) == 0                 # more tokens than the kernel takes
+    M.molora_debug_set("small_path", 0)
+    # by default a decode-sized call may run on either, so the figure covers both
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 64) == ctl + 24 * 6 * 16 * 64 * 4 + 4 * 256 * 64 * 4
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == ctl + 24 * 6 * 16 * 16 * 4
     assert M.molora_apply_workspace_bytes(1024, 8, 2048, 2048, 64) > 0
-    # ranks 16 and 32 (streaming or tcgen05 kernel), rank 64 from 1280 tokens with few adapters, rank 8 and fp32-only
-    # shapes need none
-    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 0
-    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 32) == 0
+    # larger calls of ranks 16 and 32 (streaming or tcgen05 kernel), rank 64 from 1280 tokens with few adapters, rank 8
+    # and fp32-only shapes need none
     assert M.molora_apply_workspace_bytes(4096, 4, 2048, 2048, 16) == 0
     assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 32) == 0
     assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 64) == 0
@@ -102,13 +114,10 @@ def test_apply_workspace_sizes_and_refusal_without_it(default_kernels):
     # with more than 64 adapters the short segments of a large rank-64 call take the two-launch kernels
     assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 64) > 0
     assert M.molora_apply_workspace_bytes(4096, 128, 2048, 2048, 16) == 0
-    # the two-launch kernels can be forced for every rank, and then ask for their scratch
-    M.molora_debug_set("small_path", 2)
-    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 2 * 256 * 16 * 4
-    M.molora_debug_set("small_path", 0)
-    # a call for the two-launch kernels without its workspace is refused before anything is enqueued
+    # a call that needs scratch is refused without it before anything is enqueued
+    before = M.molora_launch_count()
     st = lib.molora_apply(fake, 64, fake, 64, M.BF16, 4, 64, 64, 64, fake, fake, 2, fake, fake, 1.0, None, 0, None, None)
-    assert st == 3
+    assert st == 3 and M.molora_launch_count() == before
 
 
 def _desc(d_in, d_out, rank):
@@ -121,27 +130,27 @@ def test_group_apply_one_call_launch_count_and_refusals(default_kernels):
     from paper_2603_15965_b200.binding import _ProjDescC
     lib = M.load_library()
 
-    def one_launch(shapes, N, dt=M.BF16):
+    def one_launch(shapes, N, dt=M.BF16, C=8):
         arr = (_ProjDescC * len(shapes))(*[_desc(*s) for s in shapes])
-        return int(lib.molora_group_apply_is_one_launch(arr, len(shapes), dt, N))
+        return int(lib.molora_group_apply_is_one_launch(arr, len(shapes), dt, N, C))
 
-    assert one_launch([(2048, 2048, 16)], 4096) == 1                    # c2's apply
-    assert one_launch([(2048, 2048, 16)] * 4 + [(2048, 6144, 16)] * 2 + [(6144, 2048, 16)], 256) == 1   # a decode layer
+    assert one_launch([(2048, 2048, 16)], 4096) == 1                    # c2's apply: streaming kernel
+    assert one_launch([(2048, 2048, 16)] * 4 + [(2048, 6144, 16)] * 2 + [(6144, 2048, 16)], 256) == 1   # a decode layer: job list
     assert one_launch([(2048, 2048, 16)], 4097) == 0                    # more tokens than a CTA groups on its own
-    assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 1   # rank 32 streams too
-    assert one_launch([(2048, 2048, 64)], 512) == 0                     # rank 64, one projection: two-launch kernels
+    assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 1   # rank 32: streaming / job list
+    assert one_launch([(2048, 2048, 64)], 512) == 1                     # rank 64, decode-sized: job list
+    assert one_launch([(2048, 2048, 64)] * 7, 1024) == 1                # rank 64, a layer's projections: streaming kernel
     arr64 = (_ProjDescC * 1)(_desc(2048, 2048, 64))
-    assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 512)) == 1    # ... which group on chip
-    assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 1100)) == 0   # more than 1024 tokens: they do not
-    assert one_launch([(2048, 2048, 64)] * 3, 512) == 1                 # rank 64, a layer's projections: streaming kernel
+    M.molora_debug_set("small_path", 2)
+    assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 512, 8)) == 1    # two-launch kernels group on chip
+    assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 1100, 8)) == 0   # more than 1024 tokens: they do not
+    assert one_launch([(2048, 2048, 16)], 4096) == 0
+    M.molora_debug_set("small_path", 0)
     assert one_launch([(2048, 2048, 64)] * 3, 2048) == 0                # rank 64 from 1280 tokens: tcgen05
     assert one_launch([(2048, 2048, 16), (2048, 2048, 32)], 2048) == 0  # two ranks: two apply launches
     assert one_launch([(2048, 2048, 16)] * 8, 4096) == 0                # 400 MB: above the tcgen05 crossover
     assert one_launch([(2048, 2048, 16)], 4096, M.F32) == 0             # fp32 storage: CUDA-core kernel
     assert one_launch([(2048, 2040, 16)], 256) == 0                     # width not a multiple of 32: CUDA-core kernel
-    M.molora_debug_set("small_path", 2)
-    assert one_launch([(2048, 2048, 16)], 4096) == 0
-    M.molora_debug_set("small_path", 0)
     # refusals before any launch: null outputs, too many adapters, no projections, unsupported rank
     fake = ctypes.c_void_p(0x1000)
     arr = (_ProjDescC * 1)(_desc(64, 64, 16))
@@ -150,3 +159,24 @@ def test_group_apply_one_call_launch_count_and_refusals(default_kernels):
     assert lib.molora_group_apply_batched(fake, 8, 4, fake, fake, fake, arr, 0, M.BF16, None, 0, None, None) == 1
     bad = (_ProjDescC * 1)(_desc(64, 64, 12))
     assert lib.molora_group_apply_batched(fake, 8, 4, fake, fake, fake, bad, 1, M.BF16, None, 0, None, None) != 0
+
+
+def test_mixed_call_without_workspace_is_refused_before_any_launch(default_kernels):
+    """A batched call whose projections need different kernels, one of them the two-launch kernels' scratch: with
+    ws = NULL (or too small, or misaligned) the call must be refused as a whole, with nothing enqueued for the others."""
+    from paper_2603_15965_b200.binding import _ProjDescC
+    lib = M.load_library()
+    fake = ctypes.c_void_p(0x1000)
+    shapes = [(256, 512, 16), (512, 128, 64), (128, 192, 8), (200, 264, 32)]      # job-list kernel per rank, CUDA cores
+    arr = (_ProjDescC * len(shapes))(*[_desc(*s) for s in shapes])
+    need = sum(M.molora_apply_workspace_bytes(300, 6, *s) for s in shapes)
+    assert need > 0
+    before = M.molora_launch_count()
+    assert lib.molora_apply_batched(arr, len(shapes), M.BF16, 300, 6, fake, fake, None, 0, None, None) == 3
+    assert lib.molora_apply_batched(arr, len(shapes), M.BF16, 300, 6, fake, fake, fake, 4096, None, None) == 3    # too small
+    assert lib.molora_apply_batched(arr, len(shapes), M.BF16, 300, 6, fake, fake, ctypes.c_void_p(0x1008), need, None, None) == 3
+    assert lib.molora_group_apply_batched(fake, 300, 6, fake, fake, fake, arr, len(shapes), M.BF16, None, 0, None, None) == 3
+    # the one-rank call that groups inside the two-launch kernels checks its scratch first as well
+    arr64 = (_ProjDescC * 1)(_desc(512, 128, 64))
+    assert lib.molora_group_apply_batched(fake, 300, 6, fake, fake, fake, arr64, 1, M.BF16, None, 0, None, None) == 3
+    assert M.molora_launch_count() == before

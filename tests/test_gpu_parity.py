@@ -26,6 +26,8 @@ KERNEL_MODES = {
     "stream-short": {"umma_min_tokens": 1000000, "small_path": 1, "stream_tile": 16},
     "stream-tall": {"umma_min_tokens": 1000000, "small_path": 1, "stream_tile": 32},
     "twophase": {"umma_min_tokens": 1000000, "small_path": 2},
+    # the job-list kernel (decode-sized calls, at most 1024 tokens; larger calls fall back to the default small kernel)
+    "jobs": {"umma_min_tokens": 1000000, "small_path": 3},
 }
 
 
@@ -394,7 +396,7 @@ def test_forward_host_matches_oracle(name):
     projs = [M.HostProj(hx[p.x_key], y, dev_tensor(p.A, w.dtype), dev_tensor(p.B, w.dtype)) for p, y in
              zip(w.projections, hy)]
     gate_proj = [p.x_key for p in w.projections].index(w.gate_x_key) if w.router == "gate" else 0
-    arena = torch.empty(M.molora_forward_host_arena_bytes(projs, router, gate_proj), dtype=torch.uint8, device="cuda")
+    arena = torch.zeros(M.molora_forward_host_arena_bytes(projs, router, gate_proj), dtype=torch.uint8, device="cuda")
     src = None
     if w.router == "vocab":
         src = torch.from_numpy(w.ids).pin_memory()
@@ -414,7 +416,7 @@ def test_forward_host_matches_oracle(name):
 
 
 # ------------------------------------------------------------------ small-tile kernels: single-launch streaming and two-launch
-@pytest.mark.parametrize("mode", ["stream-short", "stream-tall", "twophase"])
+@pytest.mark.parametrize("mode", ["stream-short", "stream-tall", "twophase", "jobs"])
 @pytest.mark.parametrize("rank", [16, 32, 64])
 def test_decode_path_segment_size_sweep(rank, mode):
     force_kernel(mode)
@@ -432,7 +434,7 @@ def test_decode_path_segment_size_sweep(rank, mode):
                                                  (90, 3, 2080, 1056, 16),     # ragged last slices (multiples of 32 only)
                                                  (1500, 3, 1056, 2592, 16),   # more tiles than CTAs x items, ragged chunks
                                                  (5000, 4, 512, 512, 32)])    # several items per persistent CTA
-@pytest.mark.parametrize("mode", ["stream-short", "stream-tall", "twophase"])
+@pytest.mark.parametrize("mode", ["stream-short", "stream-tall", "twophase", "jobs"])
 def test_decode_path_shapes(N, C, d_in, d_out, rank, mode):
     force_kernel(mode)
     w = W.random_problem(N + rank + 7, N, C, d_in, d_out, rank, "bf16", unrouted_frac=0.1 if N > 10 else 0.0)
@@ -471,7 +473,7 @@ def test_route_gate_tensor_core_paths(N, d, C):
 
 
 # ------------------------------------------------------------------ seeded random shapes across every kernel path
-@pytest.mark.parametrize("mode", ["default", "tcgen05", "stream-short", "stream-tall", "twophase"])
+@pytest.mark.parametrize("mode", ["default", "tcgen05", "stream-short", "stream-tall", "twophase", "jobs"])
 @pytest.mark.parametrize("seed", range(24))
 def test_random_shapes_all_paths(seed, mode):
     # token counts on both sides of the path switches (1024 / 1280 tokens), adapter counts on both sides of the
@@ -589,6 +591,7 @@ def test_route_mlp_feeds_group_and_apply():
 
 # ------------------------------------------------------------------ top-k weighted routing (Eq. 8, the paper's k = 2)
 @pytest.mark.parametrize("N,C,k,d_in,d_out,rank,mode", [(300, 4, 2, 256, 192, 16, "stream"),
+                                                        (300, 4, 2, 256, 192, 16, "jobs"),
                                                         (300, 4, 2, 256, 192, 16, "twophase"),
                                                         (3300, 4, 2, 512, 256, 16, "tcgen05"),
                                                         (200, 6, 3, 128, 96, 8, "default"),      # CUDA-core kernel (rank 8)
@@ -641,6 +644,9 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode):
     (4097, 4, [(256, 256, 16)], "default"),                                     # one token too many: two launches
     (600, 3, [(256, 256, 16), (256, 128, 64)], "default"),                      # mixed ranks: two launches
     (300, 4, [(128, 192, 8)], "default"),                                       # CUDA-core apply: two launches
+    (256, 8, [(2048, 2048, 16), (2048, 1024, 16), (2048, 1024, 16), (512, 2048, 16), (2048, 6144, 16), (6144, 2048, 16)], "jobs"),
+    (1024, 200, [(256, 192, 32), (256, 320, 32), (512, 64, 32)], "jobs"),       # job list: its largest size, many adapters
+    (77, 3, [(512, 4096, 64), (512, 512, 64)], "jobs"), (1, 1, [(32, 32, 16)], "jobs"),
     (900, 6, [(512, 512, 16)], "twophase"),                                     # two-launch kernels forced: they group on chip
     (1024, 40, [(256, 192, 32)], "twophase"),                                   # ... their largest size, match_any grouping
     (1025, 4, [(256, 192, 32)], "twophase"),                                    # one token too many: grouping launch + 2
@@ -691,3 +697,35 @@ def test_group_apply_one_call_flags_bad_routes():
     ref, _ = oracle.apply(w.inputs["x"], pr.y, pr.A, pr.B, w.r)
     assert_close(to_f64(y), ref, what="bad routes are unrouted")
     assert int(offsets.cpu().numpy()[-1]) == N - 2
+
+
+def test_mixed_call_refused_for_its_workspace_leaves_y_untouched():
+    # mixed ranks, the rank-64 projection needs the two-launch kernels' scratch: without it the whole call is refused and
+    # no projection's y may have been updated (a caller that retries with a workspace must not add a delta twice)
+    N, C = 300, 6
+    rng = np.random.default_rng(5)
+    r = rng.integers(0, C, size=N).astype(np.int32)
+    shapes = [(256, 512, 16), (512, 128, 64), (128, 192, 8), (200, 264, 32)]
+    ws = [W.random_problem(7100 + i, N, C, di, do, rk, "bf16", r=r) for i, (di, do, rk) in enumerate(shapes)]
+    xs = [dev_tensor(w.inputs["x"], "bf16") for w in ws]
+    ys = [dev_tensor(w.projections[0].y, "bf16") for w in ws]
+    y0 = [y.clone() for y in ys]
+    projs = [M.ProjDesc(x, y, dev_tensor(w.projections[0].A, "bf16"), dev_tensor(w.projections[0].B, "bf16"), 1.0)
+             for w, x, y in zip(ws, xs, ys)]
+    counts, offsets, perm = M.molora_group(dev_tensor(r, "i"), C)
+    from paper_2603_15965_b200.binding import pack_proj_descs
+    arr, n, c, dt = pack_proj_descs(projs)
+    lib = M.load_library()
+    import ctypes
+    st = lib.molora_apply_batched(arr, len(arr), dt, n, c, ctypes.c_void_p(offsets.data_ptr()), ctypes.c_void_p(perm.data_ptr()),
+                                  None, 0, None, ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+    torch.cuda.synchronize()
+    assert st == 3
+    for y, y_before in zip(ys, y0):
+        assert torch.equal(y, y_before)
+    # with the workspace the same call goes through and matches the oracle
+    M.molora_apply_batched(projs, offsets, perm)
+    for w, y in zip(ws, ys):
+        p = w.projections[0]
+        ref, _ = oracle.apply(w.inputs["x"], p.y, p.A, p.B, r)
+        assert_close(to_f64(y), ref, what=f"mixed batch after retry {p.d_in}->{p.d_out} r{p.rank}")
