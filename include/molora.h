@@ -189,10 +189,11 @@ molora_status_t molora_group(const int32_t *r, int64_t N, int32_t C, int32_t *co
  * offsets, perm   device outputs of molora_group for the same N, C (read on the device only)
  * ws, ws_bytes    device scratch of at least molora_apply_workspace_bytes(...) bytes, 16-byte aligned (NULL if
  *                 that is 0).  Two kernels use it.  The job-list kernel (bf16, at most 1024 tokens, few tiles per SM:
- *                 decode-sized calls) keeps counters and fp32 partial shrink results there: ws must be ZERO-FILLED
- *                 before its first use; every call leaves its control words zero again, so the same ws can be passed
- *                 to any number of later calls (of any shape) without clearing.  Calls that share one ws must not
- *                 overlap on the GPU.  If a call reports MOLORA_DEV_TIMEOUT, clear ws before using it again.  The
+ *                 decode-sized calls) keeps two control words and the fp32 partial shrink results there, the latter as
+ *                 64-bit records {value, tag of the launch}: ALL of ws must be ZERO-FILLED before its first use (never
+ *                 clear only a part of it later); after that the same ws can be passed to any number of calls, of any
+ *                 shape, without clearing -- every launch counts itself in the control words and old records never
+ *                 carry the current tag.  Calls that share one ws must not overlap on the GPU.  The
  *                 two-launch small-tile kernels (bf16 rank 64 below 1280 tokens with one or two rank-64 projections in
  *                 the call; with more than 64 adapters also the short segments of larger rank-64 calls) keep partial
  *                 shrink results [slice][N][rank] behind that.

@@ -16,7 +16,7 @@ std::atomic<int64_t> g_tune[kTuneCount];
 std::atomic<uint64_t> g_launches{0};
 std::once_flag g_tune_once;
 const char* const kTuneNames[kTuneCount] = {"umma_min_tokens", "small_path", "stream_tile", "umma_split",
-                                            "umma_tile_rows", "group_split", "chained_launch_off"};
+                                            "umma_tile_rows", "group_split", "chained_launch_off", "jobs_launch"};
 void tune_from_environment()
 {
     auto num = [](const char* name) {
@@ -32,6 +32,7 @@ void tune_from_environment()
     g_tune[kTuneGroupSplit] = num("MOLORA_GROUP_SPLIT");
     const char* ch = std::getenv("MOLORA_CHAINED_LAUNCH");
     g_tune[kTuneChainedLaunchOff] = ch != nullptr && std::strcmp(ch, "0") == 0 ? 1 : 0;
+    g_tune[kTuneJobsLaunch] = num("MOLORA_JOBS_LAUNCH");
 }
 }  // namespace
 int64_t tune(TuneKey key)
@@ -84,15 +85,18 @@ bool small_path_is_stream(int32_t rank, int64_t N, int same_rank)
     return rank == 16 || rank == 32 || same_rank > 2;
 }
 
-// The job-list kernel takes decode-sized calls: at most 1024 tokens, and few enough 16-row tiles over the projections of
-// the rank that one CTA per (tile, projection) would leave the launch waiting for its longest items -- the same bound
-// under which the streaming kernel would switch to its short tile.
-constexpr double kJobsFill = 1.25;
+// The job-list kernel shares chunk-sized jobs between all CTAs instead of giving every (tile, projection) pair to one CTA.
+// Its jobs cost more than the streaming kernel's chunks (a partial exchange through L2 per shrink chunk), so it only pays
+// where the streaming kernel's longest items dominate: measured on B200 (seven 2048 / 6144-wide rank-16 projections,
+// 8 adapters, graph replay, us, streaming / job list): 32 tokens 10.4 / 11.7, 128: 12.0 / 13.9, 256: 14.9 / 16.6,
+// 512: 26.4 / 21.7, 1024: 36.3 / 34.1; one projection, ranks 32 and 64: the streaming or the two-launch kernels win at
+// every size.  Hence: rank 16, at least four projections of that rank in the call, more than 256 and at most 1024 tokens.
 bool use_jobs(const molora_proj_desc_t& p, molora_dtype_t dt, int64_t N, int32_t C, int same_rank)
 {
+    (void)C;
     if (!jobs_eligible(p, dt, N)) return false;
     if (const int64_t forced = tune(kTuneSmallPath)) return forced == 3;
-    return (double)(ceil_div64(N, 16) + C) * same_rank <= kJobsFill * sm_count();
+    return p.rank == 16 && same_rank >= 4 && N > 256;
 }
 
 bool rank_supported(int r) { return r == 8 || r == 16 || r == 32 || r == 64; }
@@ -229,7 +233,9 @@ size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t 
     probe.d_out = d_out;
     probe.rank = rank;
     const int64_t small = tune(kTuneSmallPath);
-    if (jobs_eligible(probe, MOLORA_BF16, N) && (small == 0 || small == 3)) need += jobs_control_bytes() + jobs_partial_bytes(N, C, d_in, rank);
+    // (by default the job-list kernel only takes rank 16 above 256 tokens, see use_jobs)
+    if (jobs_eligible(probe, MOLORA_BF16, N) && (small == 3 || (small == 0 && rank == 16 && N > 256)))
+        need += jobs_control_bytes() + jobs_partial_bytes(N, C, d_in, rank);
     if (small == 3 && need > 0) return need;
     if (small_path_is_stream(rank, N, 0)) return need;
     // two-launch kernels: needed unless the tcgen05 kernel is certain to take every segment (for ranks 16 and 32 that

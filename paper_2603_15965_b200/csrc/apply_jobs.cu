@@ -7,12 +7,14 @@
 //
 //   shrink job (x-group, tile, chunk of d_in)   x-group = up to 64 / R projections that read the same x (q / k / v,
 //       gate / up): the tile's x rows are loaded ONCE and multiplied against the chunk's rows of every member's A_c.
-//       The fp32 partial t[16, R] of every member goes to the workspace, then the job adds 1 (release) to the
-//       counter of its (x-group, tile).
+//       The fp32 partial t[16, R] of every member goes to the workspace as 64-bit records {value, tag of this launch}:
+//       a 64-bit store is indivisible, so a reader that finds the tag has the value -- no flag, no fence, no second
+//       round trip.
 //   expand job (projection, tile, chunk of d_out)   its y rows and B_c chunk are requested at once (they depend on
-//       nothing); the CTA's t warp waits (bounded) until the counter of (x-group, tile) shows every shrink chunk, sums
-//       the partials in chunk order (deterministic), scales, splits into bf16 hi + lo and stages them beside the chunk;
-//       the compute warps then update y in shared memory (fp32 add, one rounding) and the copy warps store the rows.
+//       nothing); the CTA's t warp polls (bounded) the records of every shrink chunk of its (x-group, tile) until all
+//       carry the tag, sums them in chunk order (deterministic), scales, splits into bf16 hi + lo and stages them beside
+//       the chunk; the compute warps then update y in shared memory (fp32 add, one rounding) and the copy warps store
+//       the rows.
 //
 // Jobs are numbered shrink jobs first and CTA b takes jobs b, b + gridDim.x, ... in that order, streaming them through
 // a ring of three shared-memory stages exactly as the single-launch streaming kernel does (four copy warps issue one
@@ -20,9 +22,10 @@
 // and every CTA runs its jobs in increasing order, so every wait on a counter ends as long as all CTAs are resident:
 // the launch is cooperative (grid <= resident CTAs), and every wait is bounded in any case.
 //
-// Workspace (caller-owned): [control: per rank a done counter and the counters per (x-group, tile) | partials].  The
-// control part (the first kJbCtlTotal bytes, the same for every call shape) must be zero before the first call; the last
-// CTA to finish clears it again, so every call leaves the workspace as the next one needs it.
+// Workspace (caller-owned, zero-filled before its first use): [control: CTAs finished, launches so far | records].  The
+// tag of a launch is 1 + the number of launches that have used the workspace, which the last CTA to finish counts up
+// (and it clears the CTA counter), so records left by earlier launches -- of any shape -- never carry the current tag and
+// nothing has to be cleared between calls.
 #include <algorithm>
 
 #include "common.cuh"
@@ -35,19 +38,19 @@ namespace molora {
 using namespace ptx;
 
 constexpr int kJbRows = 16;                // positions per tile (one 16-row MMA tile)
-constexpr int kJbWarps = 8;                // compute warps
+constexpr int kJbWarps = 8;                // compute warps: two teams of four that take alternate jobs of the CTA
+constexpr int kJbTeams = 2;
+constexpr int kJbTeamWarps = kJbWarps / kJbTeams;
 constexpr int kJbCopyWarps = 4;            // each moves 4 rows of the tile and a quarter of the weight rows
 constexpr int kJbThreads = (kJbWarps + kJbCopyWarps + 1) * 32;    // + the t warp
 constexpr int kJbMaxTokens = 1024;         // perm stays in shared memory
 constexpr int kJbStages = 3;
 constexpr int kJbStageData = 66048;        // rows + weights of one job
 constexpr int kJbMaxChunk = 1024;          // columns of a chunk at most
-constexpr int kJbCtlBytes = 256;           // done counter (and padding) at the start of a control region
+constexpr int kJbMaxUnits = 256;           // (x-group, chunk) and (projection, chunk) pairs of a launch at most
+constexpr int kJbMaxUnitsPerProj = kJbMaxUnits / MOLORA_MAX_PROJECTIONS;
+constexpr int kJbCtlBytes = 256;           // control words at the start of the workspace: [0] CTAs finished, [1] launches
 constexpr int kJbMaxTiles = kJbMaxTokens / kJbRows + MOLORA_MAX_ADAPTERS;   // every segment adds at most one partial tile
-// control region of one rank: done counter + one counter per (x-group, tile), at a fixed stride so that the region has
-// the same extent for every call shape
-constexpr int kJbCtlRegion = kJbCtlBytes + MOLORA_MAX_PROJECTIONS * kJbMaxTiles * 4;
-constexpr int kJbCtlTotal = 3 * kJbCtlRegion + 256 - (3 * kJbCtlRegion) % 256;   // ranks 16, 32, 64
 
 template <int R>
 struct JbCfg {
@@ -56,7 +59,7 @@ struct JbCfg {
     static constexpr int TBYTES = 2 * kJbRows * TP;        // hi and lo
     static constexpr int STAGE = kJbStageData + (TBYTES + 127) / 128 * 128;
     static constexpr int SMEM = kJbStages * STAGE;
-    static_assert(kJbWarps * MAXM * kJbRows * R * 4 <= kJbStageData, "the per-warp partials are summed through one stage");
+    static_assert(kJbTeamWarps * MAXM * kJbRows * R * 4 <= kJbStageData, "the per-warp partials are summed through one stage");
 };
 
 struct JobParams {
@@ -69,10 +72,9 @@ struct JobParams {
     int32_t pgroup[MOLORA_MAX_PROJECTIONS], pslot[MOLORA_MAX_PROJECTIONS];
     int32_t ech[MOLORA_MAX_PROJECTIONS];                   // columns per expand chunk
     int32_t estart[MOLORA_MAX_PROJECTIONS + 1];            // expand chunks of the projections before p
-    int64_t part_off[MOLORA_MAX_PROJECTIONS];              // first float of the group's partials
-    int32_t* ctl;                                          // [0]: CTAs that have finished
-    int32_t* flags;                                        // [group][kJbMaxTiles]: finished shrink chunks of (group, tile)
-    float* partials;                                       // per group: [tile][chunk][member][16][R]
+    int64_t part_off[MOLORA_MAX_PROJECTIONS];              // first record of the group's partials
+    uint32_t* ctl;                                         // [0]: CTAs that have finished, [1]: launches that have used the workspace
+    unsigned long long* partials;                          // per group: [tile][chunk][member][16][R] records {value, tag}
     const int32_t* offsets;
     const int32_t* perm;
     uint32_t* dev_status;
@@ -88,7 +90,7 @@ namespace {
 
 __device__ __forceinline__ void jb_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
-    asm volatile(
+    asm(   // a pure function of its registers: the compiler may schedule it freely
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -105,21 +107,25 @@ __device__ __forceinline__ void jb_ldsm_t(uint32_t (&r)[4], uint32_t addr)
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
 }
-// barrier of the compute warps only
-__device__ __forceinline__ void jb_compute_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kJbWarps * 32) : "memory"); }
+// barrier of the compute warps of one team
+__device__ __forceinline__ void jb_team_sync(int team) { asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "n"(kJbTeamWarps * 32) : "memory"); }
 
-__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p)
+// A record is one 64-bit word {value: low half, tag: high half}; 64-bit accesses are indivisible, so value and tag
+// always travel together.  Two records at a 16-byte aligned address, straight from L2 (another SM may have just
+// written them):
+__device__ __forceinline__ void ld_records(const unsigned long long* p, unsigned long long& r0, unsigned long long& r1)
 {
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];" : "=l"(r0), "=l"(r1) : "l"(p) : "memory");
 }
-__device__ __forceinline__ void red_release_gpu_add(int32_t* p, int v)
+__device__ __forceinline__ void st_record(unsigned long long* p, float value, uint32_t tag)
 {
-    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+    const unsigned long long rec = (unsigned long long)__float_as_uint(value) | ((unsigned long long)tag << 32);
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(rec) : "memory");
 }
 
-// One job, decoded the same way by every role.
+// Decoding a job costs a division, two prefix searches and a bisection; every role of the CTA needs every job of the
+// CTA, so the two lookups are tabulated once per CTA after the grouping: tile -> (segment, first position, rows) and
+// unit -> (shrink / expand, x-group or projection, chunk, first column, columns).
 struct JbJob {
     int expand;     // 0: shrink job of x-group `unit`, 1: expand job of projection `unit`
     int unit;       // x-group or projection
@@ -127,34 +133,37 @@ struct JbJob {
     int tile, seg, row0, rows;
     int c0, nc;     // first column and columns of the chunk (of d_in or of d_out)
 };
-__device__ __forceinline__ JbJob jb_job(const JobParams& prm, const int32_t* offs_s, const int32_t* tstart_s, int T, int job)
-{
-    JbJob jb;
-    const int n_shrink = T * prm.sstart[prm.ng];
-    jb.expand = job >= n_shrink;
-    const int j = jb.expand ? job - n_shrink : job;
-    const int u = j / T;
-    jb.tile = j - u * T;
-    jb.unit = 0;
-    if (jb.expand) {
-#pragma unroll
-        for (int p = 1; p < MOLORA_MAX_PROJECTIONS; ++p)
-            if (p < prm.P && u >= prm.estart[p]) jb.unit = p;
-        jb.chunk = u - prm.estart[jb.unit];
-        jb.c0 = jb.chunk * prm.ech[jb.unit];
-        jb.nc = min(prm.ech[jb.unit], prm.p[jb.unit].d_out - jb.c0);
-    } else {
-#pragma unroll
-        for (int g = 1; g < MOLORA_MAX_PROJECTIONS; ++g)
-            if (g < prm.ng && u >= prm.sstart[g]) jb.unit = g;
-        jb.chunk = u - prm.sstart[jb.unit];
-        jb.c0 = jb.chunk * prm.gch[jb.unit];
-        jb.nc = min(prm.gch[jb.unit], prm.p[prm.gmem[jb.unit][0]].d_in - jb.c0);
+// Position of a CTA in its job list: job = unit * T + tile, advanced by gridDim.x without dividing.
+struct JbCursor {
+    int unit, tile;
+    __device__ __forceinline__ void start(int job, int T)
+    {
+        unit = T > 0 ? job / T : 0;
+        tile = job - unit * T;
     }
-    jb.seg = 0;
-    jb.row0 = 0;
-    jb.rows = 1;
-    find_tile_bisect(offs_s, tstart_s, prm.C, kJbRows, jb.tile, jb.seg, jb.row0, jb.rows);
+    __device__ __forceinline__ void next(int gq, int gm, int T)
+    {
+        unit += gq;
+        tile += gm;
+        if (tile >= T) {
+            tile -= T;
+            ++unit;
+        }
+    }
+};
+__device__ __forceinline__ JbJob jb_decode(const int4* unit_tab, const int4* tile_tab, const JbCursor& c)
+{
+    const int4 u = unit_tab[c.unit], t = tile_tab[c.tile];
+    JbJob jb;
+    jb.expand = u.x & 1;
+    jb.unit = u.x >> 1;
+    jb.chunk = u.y;
+    jb.c0 = u.z;
+    jb.nc = u.w;
+    jb.tile = c.tile;
+    jb.seg = t.x;
+    jb.row0 = t.y;
+    jb.rows = t.z;
     return jb;
 }
 
@@ -169,12 +178,14 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
     __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
     __shared__ int32_t tstart_s[MOLORA_MAX_ADAPTERS + 1];
     __shared__ int32_t perm_s[kJbMaxTokens];
+    __shared__ int4 tile_tab[kJbMaxTiles];
+    __shared__ int4 unit_tab[kJbMaxUnits];
     __shared__ __align__(8) uint64_t full_s[NS], done_s[NS], free_s[NS];
     __shared__ unsigned long long st_dst[NS][kJbRows];      // expand job in the stage: where its y rows go back to
     __shared__ uint32_t st_bytes[kJbCopyWarps][NS];         // bytes per row to store (0: a shrink job, nothing to store)
     __shared__ uint32_t st_pitch[kJbCopyWarps][NS];
     __shared__ int st_rows[kJbCopyWarps][NS];
-    __shared__ int abort_s, last_s;
+    __shared__ int abort_s;
     extern __shared__ __align__(128) unsigned char dsm[];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -182,13 +193,44 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&full_s[s]), kJbCopyWarps + 1);      // four copy warps (with their bytes) + the t warp
-            mbar_init(smem_u32(&done_s[s]), kJbWarps);
+            mbar_init(smem_u32(&done_s[s]), kJbTeamWarps);
             mbar_init(smem_u32(&free_s[s]), kJbCopyWarps);
         }
         abort_s = 0;
-        last_s = 0;
         fence_mbar_init();
     }
+    grid_dependency_wait();                                  // (a no-op unless the launch is programmatic)
+    // the launch's tag and the routing decisions are requested first (L2 / DRAM round trips) ...
+    const uint32_t tag = __ldcg(prm.ctl + 1) + 1u;          // the launches before this one, + 1: never the tag of an old record
+    int warm = 0;
+    if (GROUP && prm.N > 0) warm = __ldg(prm.r + min(tid, prm.N - 1));
+    // ... and while they travel, the unit table (independent of the routing)
+    const int n_sunits = prm.sstart[prm.ng], n_units = n_sunits + prm.estart[prm.P];
+    for (int u = tid; u < n_units; u += kJbThreads) {
+        int4 e;
+        if (u < n_sunits) {
+            int g = 0;
+#pragma unroll
+            for (int k = 1; k < MOLORA_MAX_PROJECTIONS; ++k)
+                if (k < prm.ng && u >= prm.sstart[k]) g = k;
+            e.x = g << 1;
+            e.y = u - prm.sstart[g];
+            e.z = e.y * prm.gch[g];
+            e.w = min(prm.gch[g], prm.p[prm.gmem[g][0]].d_in - e.z);
+        } else {
+            const int v = u - n_sunits;
+            int p = 0;
+#pragma unroll
+            for (int k = 1; k < MOLORA_MAX_PROJECTIONS; ++k)
+                if (k < prm.P && v >= prm.estart[k]) p = k;
+            e.x = (p << 1) | 1;
+            e.y = v - prm.estart[p];
+            e.z = e.y * prm.ech[p];
+            e.w = min(prm.ech[p], prm.p[p].d_out - e.z);
+        }
+        unit_tab[u] = e;
+    }
+    asm volatile("" ::"r"(warm));
     if constexpr (GROUP) {
         group_in_cta<kJbThreads, kJbMaxTokens>(prm.r, prm.N, prm.C, offs_s, tstart_s, perm_s, dsm, true, prm.counts_out,
                                                prm.offsets_out, prm.perm_out, prm.dev_status);
@@ -197,17 +239,29 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
         for (int i = tid; i < prm.N; i += kJbThreads) perm_s[i] = __ldg(prm.perm + i);
         __syncthreads();
     }
-    if (warp == 0) tile_starts(offs_s, prm.C, kJbRows, 1, INT32_MAX, tstart_s);
+    if (warp == 0) {                                        // tiles per segment, then every tile's (segment, first position, rows)
+        tile_starts(offs_s, prm.C, kJbRows, 1, INT32_MAX, tstart_s);
+        __syncwarp();
+        const int T0 = tstart_s[prm.C];
+        for (int t = lane; t < T0; t += 32) {
+            int seg = 0, row0 = 0, rows = 1;
+            find_tile_bisect(offs_s, tstart_s, prm.C, kJbRows, t, seg, row0, rows);
+            tile_tab[t] = make_int4(seg, row0, rows, 0);
+        }
+    }
     __syncthreads();
     const int T = tstart_s[prm.C];
-    const int njobs = T * (prm.sstart[prm.ng] + prm.estart[prm.P]);
     const uint32_t stage0 = smem_u32(dsm);
     const int G = (int)gridDim.x;
+    const int gq = T > 0 ? G / T : 0, gm = G - gq * T;      // a step of gridDim.x jobs in (unit, tile) coordinates
+    JbCursor cur;
+    cur.start((int)blockIdx.x, T);
+    if (T == 0) cur.unit = n_units;                         // nothing routed: no jobs
 
     if (warp >= kJbWarps && warp < kJbWarps + kJbCopyWarps) {
         // ------------------------------------------------------------------------------------------ copy warps
         // Copy warp w owns 4 consecutive rows of the tile (its first 4 lanes, one bulk request each) and a quarter of the
-        // weight rows (the lanes after them); the four warps run the same job list without talking to one another.
+        // weight rows (the lanes after them); the four warps run the same job list.
         const int cw = warp - kJbWarps;
         constexpr int RPW = kJbRows / kJbCopyWarps;
         const int myrow = cw * RPW + (lane % RPW);
@@ -215,7 +269,7 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
             const uint32_t s = k % NS;
             wait_bar(smem_u32(&done_s[s]), (k / NS) & 1u, &abort_s, prm.dev_status);
             const uint32_t nb = st_bytes[cw][s];
-            if (nb != 0 && !abort_s) {
+            if (nb != 0 && !*aborted) {
                 if (lane < RPW && myrow < st_rows[cw][s])
                     bulk_store(reinterpret_cast<void*>(st_dst[s][myrow]), stage0 + s * Cfg::STAGE + myrow * st_pitch[cw][s], nb);
                 bulk_commit_group();
@@ -228,8 +282,8 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
             wait_bar(smem_u32(&free_s[s]), (k / NS) & 1u, &abort_s, prm.dev_status);
         };
         uint32_t g = 0;
-        for (int job = blockIdx.x; job < njobs && !*aborted; job += G, ++g) {
-            const JbJob jb = jb_job(prm, offs_s, tstart_s, T, job);
+        for (; cur.unit < n_units && !*aborted; cur.next(gq, gm, T), ++g) {
+            const JbJob jb = jb_decode(unit_tab, tile_tab, cur);
             const uint32_t s = g % NS;
             if (g >= (uint32_t)NS) retire(g - NS);
             if (*aborted) break;
@@ -279,9 +333,9 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
             }
         }
         const uint32_t first = g > (uint32_t)NS ? g - NS : 0;      // the jobs still in the ring
-        if (!abort_s)
+        if (!*aborted)
             for (uint32_t k = first; k < g; ++k) retire(k);
-        if (abort_s) {
+        if (*aborted) {
             // stopped early: give the copies in flight into this CTA's shared memory a bounded chance to land
             for (uint32_t k = first; k < g; ++k) {
                 const long long t0 = clock64();
@@ -298,8 +352,8 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
         constexpr int CPL = R / 2;
         const int trow = lane >> 1, tcol = (lane & 1) * CPL;
         uint32_t g = 0;
-        for (int job = blockIdx.x; job < njobs && !*aborted; job += G, ++g) {
-            const JbJob jb = jb_job(prm, offs_s, tstart_s, T, job);
+        for (; cur.unit < n_units && !*aborted; cur.next(gq, gm, T), ++g) {
+            const JbJob jb = jb_decode(unit_tab, tile_tab, cur);
             const uint32_t s = g % NS;
             if (g >= (uint32_t)NS) wait_bar(smem_u32(&done_s[s]), ((g - NS) / NS) & 1u, &abort_s, prm.dev_status);
             if (*aborted) break;
@@ -307,33 +361,46 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
                 const molora_proj_desc_t& pd = prm.p[jb.unit];
                 const int grp = prm.pgroup[jb.unit], slot = prm.pslot[jb.unit], m = prm.gm[grp];
                 const int nk = prm.sstart[grp + 1] - prm.sstart[grp];
-                const int32_t* flag = prm.flags + grp * kJbMaxTiles + jb.tile;
-                if (ld_acquire_gpu(flag) < nk) {
-                    const long long t0 = clock64();
-                    while (ld_acquire_gpu(flag) < nk && !*aborted) {
-                        if (clock64() - t0 > kTimeoutCycles) {
-                            *aborted = 1;
-                            if (prm.dev_status != nullptr) atomicOr(prm.dev_status, MOLORA_DEV_TIMEOUT);
-                        }
-                    }
-                }
+                // my CPL records of chunk c: [tile][chunk][member][16][R]
+                const unsigned long long* rec = prm.partials + prm.part_off[grp] + ((int64_t)jb.tile * nk * m + slot) * (kJbRows * R) + trow * R + tcol;
+                const int64_t cstride = (int64_t)m * (kJbRows * R);
                 float v[CPL];
 #pragma unroll
                 for (int i = 0; i < CPL; ++i) v[i] = 0.f;
-                const float* part = prm.partials + prm.part_off[grp] + ((int64_t)jb.tile * nk * m + slot) * (kJbRows * R) + trow * R + tcol;
-                for (int c = 0; c < nk; ++c) {
+                // Blocks of CB chunks: request every record of the block, then look at the tags; a block is summed (in
+                // chunk order) only once all of its records carry this launch's tag, otherwise it is requested again.
+                constexpr int CB = 32 / CPL >= 1 ? 32 / CPL : 1;      // 32 records (64 registers) in flight per lane
+                const long long t0 = clock64();
+                for (int c0 = 0; c0 < nk && !*aborted;) {
+                    unsigned long long rr[CB][CPL];
+                    bool ready = true;
 #pragma unroll
-                    for (int i = 0; i < CPL; i += 4) {
-                        const float4 u = __ldcg(reinterpret_cast<const float4*>(part + (int64_t)c * m * (kJbRows * R) + i));
-                        v[i] += u.x;
-                        v[i + 1] += u.y;
-                        v[i + 2] += u.z;
-                        v[i + 3] += u.w;
+                    for (int cb = 0; cb < CB; ++cb)
+                        if (c0 + cb < nk) {
+#pragma unroll
+                            for (int i = 0; i < CPL; i += 2) ld_records(rec + (c0 + cb) * cstride + i, rr[cb][i], rr[cb][i + 1]);
+                        }
+#pragma unroll
+                    for (int cb = 0; cb < CB; ++cb)
+                        if (c0 + cb < nk) {
+#pragma unroll
+                            for (int i = 0; i < CPL; ++i) ready = ready && (uint32_t)(rr[cb][i] >> 32) == tag;
+                        }
+                    if (__all_sync(0xFFFFFFFFu, ready)) {
+#pragma unroll
+                        for (int cb = 0; cb < CB; ++cb)
+                            if (c0 + cb < nk) {
+#pragma unroll
+                                for (int i = 0; i < CPL; ++i) v[i] += __uint_as_float((uint32_t)rr[cb][i]);
+                            }
+                        c0 += CB;
+                    } else if (clock64() - t0 > kTimeoutCycles) {
+                        *aborted = 1;
+                        if (prm.dev_status != nullptr && lane == 0) atomicOr(prm.dev_status, MOLORA_DEV_TIMEOUT);
                     }
                 }
                 float sc = pd.scale;           // times the token's routing weight, if the caller passes per-token factors
-                if (trow >= jb.rows) sc = 0.f;
-                else if (pd.row_scale != nullptr) sc *= __ldg(pd.row_scale + perm_s[jb.row0 + trow]);
+                if (trow < jb.rows && pd.row_scale != nullptr) sc *= __ldg(pd.row_scale + perm_s[jb.row0 + trow]);
                 unsigned char* tb = dsm + s * Cfg::STAGE + kJbStageData;
 #pragma unroll
                 for (int i = 0; i < CPL; i += 8) {
@@ -358,17 +425,24 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
         constexpr int NT = R / 8;                  // n8 tiles of t
         constexpr int KB = R / 16;                 // k16 blocks of the expand
         const int g4 = lane >> 2, q = lane & 3;
+        const int mi = lane >> 3;                  // matrix of an x4 ldmatrix this lane addresses
+        // Two teams of four warps take alternate jobs: a job's load, MMA and store phases use different pipes, and the
+        // two teams are in different phases most of the time.
+        const int team = warp / kJbTeamWarps, tw = warp % kJbTeamWarps, ttid = tid - team * (kJbTeamWarps * 32);
         uint32_t g = 0;
-        for (int job = blockIdx.x; job < njobs; job += G, ++g) {
-            const JbJob jb = jb_job(prm, offs_s, tstart_s, T, job);
+        for (; cur.unit < n_units; cur.next(gq, gm, T), ++g) {
+            if ((int)(g % kJbTeams) != team) continue;
+            const JbJob jb = jb_decode(unit_tab, tile_tab, cur);
             const uint32_t s = g % NS;
             const uint32_t sb = stage0 + s * Cfg::STAGE;
             unsigned char* sp = dsm + s * Cfg::STAGE;
             const uint32_t pitch = (uint32_t)jb.nc * 2u + 16u;
             wait_bar(smem_u32(&full_s[s]), (g / NS) & 1u, &abort_s, prm.dev_status);
-            if (*aborted) break;               // uniform across the compute warps soon enough: every later wait falls through
+            // (after a time-out every wait falls through and the team runs its remaining jobs on whatever the stages hold:
+            // nothing of it is stored, and no warp is left alone at a team barrier)
             if (!jb.expand) {
-                // ---- shrink chunk: partial t of every member, interleaved 32-wide k blocks per warp
+                // ---- shrink chunk: partial t of every member, interleaved 32-wide k blocks per warp.  All fragment loads
+                // of a block are issued before its MMAs, so the warp pays the shared-memory latency once per block.
                 const int m = prm.gm[jb.unit];
                 const uint32_t wo = (kJbRows * pitch + 127u) & ~127u;
                 const uint32_t ablock = (uint32_t)jb.nc * R * 2u;
@@ -380,129 +454,134 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
 #pragma unroll
                         for (int i = 0; i < 4; ++i) acc[j][n][i] = 0.f;
                 const int nb = jb.nc / 32;
-                for (int b = warp; b < nb; b += kJbWarps) {
+                const uint32_t xa = sb + (lane & 15) * pitch + (lane >> 4) * 16;
+                const uint32_t wa = sb + wo + ((mi & 1) * 8 + (lane & 7)) * (R * 2) + (mi >> 1) * 16;
+                for (int b = tw; b < nb; b += kJbTeamWarps) {
+                    uint32_t a[2][4];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {                           // two k16 steps per block
-                        uint32_t a[4];
-                        jb_ldsm(a, sb + (lane & 15) * pitch + (b * 32 + h * 16 + (lane >> 4) * 8) * 2);
-                        const int mi = lane >> 3;                           // matrix of the x4 load this lane addresses
+                    for (int h = 0; h < 2; ++h) jb_ldsm(a[h], xa + (b * 32 + h * 16) * 2);
 #pragma unroll
-                        for (int j = 0; j < MAXM; ++j) {
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t bf[MAXM][NT / 2][4];
+#pragma unroll
+                        for (int j = 0; j < MAXM; ++j)
+                            if (j < m) {
+#pragma unroll
+                                for (int n16 = 0; n16 < NT / 2; ++n16)
+                                    jb_ldsm_t(bf[j][n16], wa + j * ablock + (b * 32 + h * 16) * (R * 2) + n16 * 32);
+                            }
+#pragma unroll
+                        for (int j = 0; j < MAXM; ++j)
                             if (j < m) {
 #pragma unroll
                                 for (int n16 = 0; n16 < NT / 2; ++n16) {
-                                    uint32_t bf[4];
-                                    jb_ldsm_t(bf, sb + wo + j * ablock + (b * 32 + h * 16 + (mi & 1) * 8 + (lane & 7)) * (R * 2) +
-                                                      (n16 * 16 + (mi >> 1) * 8) * 2);
-                                    jb_mma(acc[j][2 * n16], a, bf[0], bf[1]);
-                                    jb_mma(acc[j][2 * n16 + 1], a, bf[2], bf[3]);
+                                    jb_mma(acc[j][2 * n16], a[h], bf[j][n16][0], bf[j][n16][1]);
+                                    jb_mma(acc[j][2 * n16 + 1], a[h], bf[j][n16][2], bf[j][n16][3]);
                                 }
                             }
-                        }
                     }
                 }
-                // sum the per-warp partials in warp order through the stage (it has been consumed), then publish
+                // sum the per-warp partials in warp order through the stage (it has been consumed) and send the result to the
+                // workspace as tagged records
                 float* tparts = reinterpret_cast<float*>(sp);
                 const int tfl = m * kJbRows * R;                            // floats of one warp's partial
-                jb_compute_sync();                 // every warp has finished reading the stage
+                jb_team_sync(team);                // every warp of the team has finished reading the stage
 #pragma unroll
                 for (int j = 0; j < MAXM; ++j) {
                     if (j < m) {
 #pragma unroll
                         for (int n = 0; n < NT; ++n) {
-                            float* tp = tparts + warp * tfl + j * (kJbRows * R) + n * 8 + 2 * q;
+                            float* tp = tparts + tw * tfl + j * (kJbRows * R) + n * 8 + 2 * q;
                             *reinterpret_cast<float2*>(tp + g4 * R) = make_float2(acc[j][n][0], acc[j][n][1]);
                             *reinterpret_cast<float2*>(tp + (g4 + 8) * R) = make_float2(acc[j][n][2], acc[j][n][3]);
                         }
                     }
                 }
-                jb_compute_sync();
+                jb_team_sync(team);
                 const int grp = jb.unit;
                 const int nk = prm.sstart[grp + 1] - prm.sstart[grp];
-                float* out = prm.partials + prm.part_off[grp] + ((int64_t)jb.tile * nk + jb.chunk) * tfl;
-                for (int e4 = tid; e4 < tfl / 4; e4 += kJbWarps * 32) {
-                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                unsigned long long* out = prm.partials + prm.part_off[grp] + ((int64_t)jb.tile * nk + jb.chunk) * tfl;
+                for (int e = ttid; e < tfl; e += kJbTeamWarps * 32) {
+                    float v = 0.f;
 #pragma unroll
-                    for (int w = 0; w < kJbWarps; ++w) {
-                        const float4 u = *reinterpret_cast<const float4*>(&tparts[w * tfl + e4 * 4]);
-                        v.x += u.x;
-                        v.y += u.y;
-                        v.z += u.z;
-                        v.w += u.w;
-                    }
-                    __stcg(reinterpret_cast<float4*>(out + e4 * 4), v);
+                    for (int w = 0; w < kJbTeamWarps; ++w) v += tparts[w * tfl + e];
+                    st_record(out + e, v, tag);
                 }
                 fence_proxy_async_smem();          // my accesses to the stage are ordered before the copies that refill it
-                jb_compute_sync();                 // the partial is written (and the stage is free)
-                if (tid == 0 && !*aborted) {
-                    __threadfence();
-                    red_release_gpu_add(prm.flags + grp * kJbMaxTiles + jb.tile, 1);
-                }
+                __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&done_s[s]));
             } else {
                 // ---- expand chunk: y += t B_c in shared memory, t from the stage's hi / lo tiles
                 const uint32_t tb = sb + kJbStageData;
-                const uint32_t bs = sb + kJbRows * pitch;
                 uint32_t thi[KB][4], tlo[KB][4];
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb) {
                     jb_ldsm(thi[kb], tb + (lane & 15) * Cfg::TP + (kb * 16 + (lane >> 4) * 8) * 2);
                     jb_ldsm(tlo[kb], tb + (kJbRows + (lane & 15)) * Cfg::TP + (kb * 16 + (lane >> 4) * 8) * 2);
                 }
-                constexpr int GI = R == 64 ? 1 : 2;
+                constexpr int GI = 1;     // one 32-column group per step: measured faster than two (the MMA and the
+                                          // shared-memory pipe do not overlap, a longer step only adds registers)
                 const int ngroups = jb.nc / 32;
-                for (int grp0 = warp; grp0 < ngroups; grp0 += GI * kJbWarps) {
+                // my element of y in a 32-column group: rows g4, g4 + 8; my rows of B_c for the transposed fragment loads
+                unsigned char* yp = sp + g4 * pitch + q * 4;
+                const uint32_t ba = sb + (kJbRows + (mi & 1) * 8 + (lane & 7)) * pitch + (mi >> 1) * 16;
+                for (int grp0 = tw; grp0 < ngroups; grp0 += GI * kJbTeamWarps) {
                     uint32_t yv[GI][2][4];
+                    uint32_t bf[GI][KB][2][4];
                     float d[GI][4][4];
+                    // every load of the iteration first ...
 #pragma unroll
                     for (int gi = 0; gi < GI; ++gi) {
-                        const int grp = grp0 + gi * kJbWarps;
+                        const int grp = grp0 + gi * kJbTeamWarps;
                         if (grp < ngroups) {
+#pragma unroll
+                            for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                                for (int p2 = 0; p2 < 2; ++p2)
+                                    jb_ldsm_t(bf[gi][kb][p2], ba + kb * 16 * pitch + (grp * 32 + p2 * 16) * 2);
 #pragma unroll
                             for (int h = 0; h < 2; ++h)
 #pragma unroll
                                 for (int nt = 0; nt < 4; ++nt)
-                                    yv[gi][h][nt] = *reinterpret_cast<const uint32_t*>(sp + (g4 + 8 * h) * pitch + (grp * 32 + nt * 8 + 2 * q) * 2);
+                                    yv[gi][h][nt] = *reinterpret_cast<const uint32_t*>(yp + h * 8 * pitch + (grp * 32 + nt * 8) * 2);
                         }
+                    }
+                    // ... then the MMAs: every hi product before the lo products, so that no MMA waits for its predecessor
+#pragma unroll
+                    for (int gi = 0; gi < GI; ++gi) {
 #pragma unroll
                         for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
                             for (int i = 0; i < 4; ++i) d[gi][nt][i] = 0.f;
-                    }
-#pragma unroll
-                    for (int gi = 0; gi < GI; ++gi) {
-                        const int grp = grp0 + gi * kJbWarps;
+                        const int grp = grp0 + gi * kJbTeamWarps;
                         if (grp < ngroups) {
 #pragma unroll
-                            for (int kb = 0; kb < KB; ++kb) {
-                                uint32_t bf[2][4];
-                                const int mi = lane >> 3;
-#pragma unroll
-                                for (int p2 = 0; p2 < 2; ++p2)
-                                    jb_ldsm_t(bf[p2], bs + (kb * 16 + (mi & 1) * 8 + (lane & 7)) * pitch + (grp * 32 + p2 * 16 + (mi >> 1) * 8) * 2);
+                            for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
                                 for (int p2 = 0; p2 < 2; ++p2) {
-                                    jb_mma(d[gi][2 * p2], thi[kb], bf[p2][0], bf[p2][1]);
-                                    jb_mma(d[gi][2 * p2 + 1], thi[kb], bf[p2][2], bf[p2][3]);
+                                    jb_mma(d[gi][2 * p2], thi[kb], bf[gi][kb][p2][0], bf[gi][kb][p2][1]);
+                                    jb_mma(d[gi][2 * p2 + 1], thi[kb], bf[gi][kb][p2][2], bf[gi][kb][p2][3]);
                                 }
 #pragma unroll
+                            for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
                                 for (int p2 = 0; p2 < 2; ++p2) {
-                                    jb_mma(d[gi][2 * p2], tlo[kb], bf[p2][0], bf[p2][1]);
-                                    jb_mma(d[gi][2 * p2 + 1], tlo[kb], bf[p2][2], bf[p2][3]);
+                                    jb_mma(d[gi][2 * p2], tlo[kb], bf[gi][kb][p2][0], bf[gi][kb][p2][1]);
+                                    jb_mma(d[gi][2 * p2 + 1], tlo[kb], bf[gi][kb][p2][2], bf[gi][kb][p2][3]);
                                 }
-                            }
                         }
                     }
+                    // accumulator element (row g4 + 8h, columns 2q, 2q+1 of n8 tile nt): add, round once, write back
 #pragma unroll
                     for (int gi = 0; gi < GI; ++gi) {
-                        const int grp = grp0 + gi * kJbWarps;
+                        const int grp = grp0 + gi * kJbTeamWarps;
                         if (grp < ngroups) {
 #pragma unroll
                             for (int h = 0; h < 2; ++h)
 #pragma unroll
                                 for (int nt = 0; nt < 4; ++nt) {
                                     const uint32_t v = yv[gi][h][nt];
-                                    *reinterpret_cast<uint32_t*>(sp + (g4 + 8 * h) * pitch + (grp * 32 + nt * 8 + 2 * q) * 2) =
+                                    *reinterpret_cast<uint32_t*>(yp + h * 8 * pitch + (grp * 32 + nt * 8) * 2) =
                                         f32x2_to_bf16x2(bf16lo_to_f32(v) + d[gi][nt][2 * h], bf16hi_to_f32(v) + d[gi][nt][2 * h + 1]);
                                 }
                         }
@@ -515,17 +594,15 @@ __global__ void __launch_bounds__(kJbThreads, 1) apply_jobs_kernel(const __grid_
         }
     }
 
-    // ---- the CTA is done: the last one to get here clears the counters for the next call
+    // ---- the CTA is done: the last one to get here counts the launch (the next launch's tag) and clears the CTA counter
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        last_s = atomicAdd(prm.ctl, 1) == G - 1;
-    }
-    __syncthreads();
-    if (last_s) {
-        __threadfence();
-        for (int i = tid; i < prm.ng * kJbMaxTiles; i += kJbThreads) prm.flags[i] = 0;
-        if (tid == 0) prm.ctl[0] = 0;
+        if (atomicAdd(prm.ctl, 1u) == (uint32_t)G - 1u) {
+            __threadfence();
+            prm.ctl[1] = tag;
+            prm.ctl[0] = 0u;
+        }
     }
 }
 
@@ -560,8 +637,15 @@ size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 bool jobs_eligible(const molora_proj_desc_t& p, molora_dtype_t dt, int64_t N)
 {
-    return dt == MOLORA_BF16 && (p.rank == 16 || p.rank == 32 || p.rank == 64) && (p.d_in % 32) == 0 && (p.d_out % 32) == 0 &&
-           N >= 1 && N <= kJbMaxTokens;
+    if (dt != MOLORA_BF16 || (p.rank != 16 && p.rank != 32 && p.rank != 64) || (p.d_in % 32) != 0 || (p.d_out % 32) != 0 ||
+        N < 1 || N > kJbMaxTokens)
+        return false;
+    // the chunks of the projection at the smallest chunk a full x-group gets: the unit table of a launch holds
+    // kJbMaxUnits entries for at most MOLORA_MAX_PROJECTIONS projections
+    int chunk = 0, ns = 0, ne = 0;
+    jb_balanced(p.d_in, jb_max_shrink_chunk(p.rank, 64 / p.rank), chunk, ns);
+    jb_balanced(p.d_out, jb_max_expand_chunk(p.rank), chunk, ne);
+    return ns + ne <= kJbMaxUnitsPerProj;
 }
 
 // Upper bound of the partials one projection adds to a job-list launch, whatever projections it is grouped with (the
@@ -571,9 +655,9 @@ size_t jobs_partial_bytes(int64_t N, int32_t C, int32_t d_in, int32_t rank)
     if (N < 1 || N > kJbMaxTokens) return 0;
     int chunk = 0, count = 0;
     jb_balanced(d_in, jb_max_shrink_chunk(rank, 64 / rank), chunk, count);
-    return align256((size_t)jb_max_tiles(N, C) * (size_t)count * kJbRows * rank * sizeof(float));
+    return align256((size_t)jb_max_tiles(N, C) * (size_t)count * kJbRows * rank * sizeof(unsigned long long));
 }
-size_t jobs_control_bytes() { return kJbCtlTotal; }
+size_t jobs_control_bytes() { return kJbCtlBytes; }
 
 template <int R, bool GROUP>
 static cudaError_t jobs_launch(const JobParams& prm, int64_t njobs_max, cudaStream_t s)
@@ -596,10 +680,16 @@ static cudaError_t jobs_launch(const JobParams& prm, int64_t njobs_max, cudaStre
     cfg.dynamicSmemBytes = Cfg::SMEM;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;   // all CTAs resident at once: a CTA may wait for another's shrink job
-    attr[0].val.cooperative = 1;
+    const int64_t how = tune(kTuneJobsLaunch);     // 0: cooperative (default); 1: plain; 2: programmatic (measurements only)
+    if (how == 2) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+    } else {
+        attr[0].id = cudaLaunchAttributeCooperative;   // all CTAs resident at once: a CTA may wait for another's shrink job
+        attr[0].val.cooperative = 1;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = how == 1 ? 0 : 1;
     note_launch();
     return cudaLaunchKernelEx(&cfg, apply_jobs_kernel<R, GROUP>, prm);
 }
@@ -641,8 +731,8 @@ static molora_status_t jobs_enqueue(const molora_proj_desc_t* projs, int32_t P, 
         if (g < prm.ng) {
             jb_balanced(projs[prm.gmem[g][0]].d_in, jb_max_shrink_chunk(R, prm.gm[g]), chunk, count);
             prm.gch[g] = chunk;
-            prm.part_off[g] = (int64_t)(off / sizeof(float));
-            off += align256((size_t)prm.Tmax * count * prm.gm[g] * kJbRows * R * sizeof(float));
+            prm.part_off[g] = (int64_t)(off / sizeof(unsigned long long));
+            off += align256((size_t)prm.Tmax * count * prm.gm[g] * kJbRows * R * sizeof(unsigned long long));
         }
         prm.sstart[g + 1] = prm.sstart[g] + count;
     }
@@ -656,10 +746,8 @@ static molora_status_t jobs_enqueue(const molora_proj_desc_t* projs, int32_t P, 
         prm.estart[i + 1] = prm.estart[i] + count;
     }
     if (ctl == nullptr || part == nullptr || part_bytes < off || !aligned16(ctl) || !aligned16(part)) return MOLORA_ERR_WORKSPACE;
-    char* region = static_cast<char*>(ctl) + (R == 16 ? 0 : R == 32 ? 1 : 2) * kJbCtlRegion;
-    prm.ctl = reinterpret_cast<int32_t*>(region);
-    prm.flags = reinterpret_cast<int32_t*>(region + kJbCtlBytes);
-    prm.partials = static_cast<float*>(part);
+    prm.ctl = static_cast<uint32_t*>(ctl);
+    prm.partials = static_cast<unsigned long long*>(part);
     const int64_t njobs_max = (int64_t)prm.Tmax * (prm.sstart[prm.ng] + prm.estart[P]);
     cudaError_t e;
     if (group) e = R == 16 ? jobs_launch<16, true>(prm, njobs_max, s) : R == 32 ? jobs_launch<32, true>(prm, njobs_max, s) : jobs_launch<64, true>(prm, njobs_max, s);

@@ -392,7 +392,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             const int ncols = min(Cfg::CH, pd.d_out - it.col0 - e * Cfg::CH);
             // my 32-column groups, GI at a time: y words first, then the MMAs, then add, round once and write back.
             // Rows past the tile hold stale shared memory; they are updated like the others and never stored.
-            constexpr int GI = R == 64 ? 1 : 2;
+            constexpr int GI = 1;
             const int ngroups = ncols / 32;
             for (int grp0 = warp; grp0 < ngroups; grp0 += GI * kFsWarps) {
                 uint32_t yv[GI][MT][2][4];

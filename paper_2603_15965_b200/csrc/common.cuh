@@ -324,6 +324,7 @@ enum TuneKey {
     kTuneUmmaTileRows,        // rows per tile of the tcgen05 apply
     kTuneGroupSplit,          // cluster size of the grouping kernel
     kTuneChainedLaunchOff,    // 1: no programmatic dependent launches
+    kTuneJobsLaunch,          // job-list kernel: 0 cooperative launch, 1 plain, 2 programmatic (measurements only)
     kTuneCount
 };
 int64_t tune(TuneKey key);

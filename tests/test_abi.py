@@ -94,15 +94,18 @@ def test_apply_workspace_sizes_and_refusal_without_it(default_kernels):
     M.molora_debug_set("small_path", 0)
     # (2) The job-list kernel (decode-sized calls: at most 1024 tokens, ranks 16 / 32 / 64): control words + partials.
     M.molora_debug_set("small_path", 3)
-    ctl = 3 * (256 + 8 * (1024 // 16 + 256) * 4)                       # three ranks x (done counter + 8 x 320 tile counters)
-    ctl += 256 - ctl % 256
-    # rank 16, d_in 2048: a full x-group (4 members) gets 384-column chunks -> 6 chunks; 256 / 16 + 8 = 24 tiles at most
-    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == ctl + 24 * 6 * 16 * 16 * 4
+    ctl = 256                                                           # control words (CTAs finished, launches so far)
+    # rank 16, d_in 2048: a full x-group (4 members) gets 384-column chunks -> 6 chunks; 256 / 16 + 8 = 24 tiles at most;
+    # 16 x 16 records of 8 bytes {value, tag} per (tile, chunk)
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == ctl + 24 * 6 * 16 * 16 * 8
     assert M.molora_apply_workspace_bytes(1025, 8, 2048, 2048, 16) == 0                 # more tokens than the kernel takes
     M.molora_debug_set("small_path", 0)
-    # by default a decode-sized call may run on either, so the figure covers both
-    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 64) == ctl + 24 * 6 * 16 * 64 * 4 + 4 * 256 * 64 * 4
-    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == ctl + 24 * 6 * 16 * 16 * 4
+    # by default the job-list kernel takes rank 16 between 257 and 1024 tokens (with at least four projections, which is
+    # not known here), rank 64 below 1280 tokens may run on the two-launch kernels
+    assert M.molora_apply_workspace_bytes(512, 8, 2048, 2048, 16) == ctl + (512 // 16 + 8) * 6 * 16 * 16 * 8
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 0
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 32) == 0
+    assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 64) == 4 * 256 * 64 * 4
     assert M.molora_apply_workspace_bytes(1024, 8, 2048, 2048, 64) > 0
     # larger calls of ranks 16 and 32 (streaming or tcgen05 kernel), rank 64 from 1280 tokens with few adapters, rank 8
     # and fp32-only shapes need none
@@ -135,14 +138,16 @@ def test_group_apply_one_call_launch_count_and_refusals(default_kernels):
         return int(lib.molora_group_apply_is_one_launch(arr, len(shapes), dt, N, C))
 
     assert one_launch([(2048, 2048, 16)], 4096) == 1                    # c2's apply: streaming kernel
-    assert one_launch([(2048, 2048, 16)] * 4 + [(2048, 6144, 16)] * 2 + [(6144, 2048, 16)], 256) == 1   # a decode layer: job list
+    layer = [(2048, 2048, 16)] * 4 + [(2048, 6144, 16)] * 2 + [(6144, 2048, 16)]
+    assert one_launch(layer, 256) == 1                                  # a decode layer: streaming kernel
+    assert one_launch(layer, 512) == 1 and one_launch(layer, 1024) == 1 # ... job-list kernel (also one launch)
     assert one_launch([(2048, 2048, 16)], 4097) == 0                    # more tokens than a CTA groups on its own
-    assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 1   # rank 32: streaming / job list
-    assert one_launch([(2048, 2048, 64)], 512) == 1                     # rank 64, decode-sized: job list
-    assert one_launch([(2048, 2048, 64)] * 7, 1024) == 1                # rank 64, a layer's projections: streaming kernel
+    assert one_launch([(2048, 2048, 32)], 2048) == 1 and one_launch([(2048, 2048, 32)], 512) == 1   # rank 32 streams too
+    assert one_launch([(2048, 2048, 64)], 512) == 0                     # rank 64, one projection: two-launch kernels
+    assert one_launch([(2048, 2048, 64)] * 3, 512) == 1                 # rank 64, a layer's projections: streaming kernel
     arr64 = (_ProjDescC * 1)(_desc(2048, 2048, 64))
-    M.molora_debug_set("small_path", 2)
     assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 512, 8)) == 1    # two-launch kernels group on chip
+    M.molora_debug_set("small_path", 2)
     assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 1100, 8)) == 0   # more than 1024 tokens: they do not
     assert one_launch([(2048, 2048, 16)], 4096) == 0
     M.molora_debug_set("small_path", 0)
