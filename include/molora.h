@@ -47,7 +47,9 @@ typedef enum {
     MOLORA_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned pointer, pitch too small      */
     MOLORA_ERR_UNSUPPORTED = 2, /* rank / dtype / C / dimension outside the supported set                */
     MOLORA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than molora_*_workspace_bytes reports     */
-    MOLORA_ERR_CUDA = 4         /* the CUDA runtime refused a launch or a copy (cudaGetLastError for why)  */
+    MOLORA_ERR_CUDA = 4,        /* the CUDA runtime refused a launch or a copy (cudaGetLastError for why)  */
+    MOLORA_ERR_BUSY = 5,        /* hot-set: every slot is pinned or being filled; try again later          */
+    MOLORA_ERR_NOT_RESIDENT = 6 /* hot-set: the adapter is not (yet) in a slot                             */
 } molora_status_t;
 
 typedef enum { MOLORA_F32 = 0, MOLORA_BF16 = 1 } molora_dtype_t;
@@ -271,6 +273,57 @@ size_t molora_apply_topk_workspace_bytes(const molora_proj_desc_t *projs, int32_
 molora_status_t molora_apply_topk(const molora_proj_desc_t *projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C,
                                   int32_t k, const int32_t *idx, const float *w, void *ws, size_t ws_bytes,
                                   uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Hot-set slot table (Definition 5.1, Eq. 10-11): S adapter slots of caller-owned, fixed-address stacks
+ * A_hot[S, M, d, r] and B_hot[S, M, r, d] per projection, a slot table sigma : [S] -> adapter ids of a catalog of
+ * n_catalog adapters, kept on the host, and its inverse on the device (table_dev: int32[n_catalog], adapter id -> slot,
+ * -1 = not resident) that molora_route_hotset reads.  The table is maintained asynchronously: loads run on a
+ * maintenance stream of the caller's, the compute streams never wait for them, and because every address is fixed the
+ * forward pass can be replayed from a CUDA graph while slots are refilled.
+ *
+ * Life of a load:   molora_hotset_begin_load(adapter)  -> slot (a free one, else the least recently pinned slot that
+ *                       nothing is using; the evicted adapter's table entry is cleared on the maintenance stream first);
+ *                       if the adapter already has a slot, that slot with fresh = 0 and nothing else to do
+ *                   molora_hotset_upload(slot, stack, weights) once per stack (A and B of every projection): copies
+ *                       `bytes_per_slot` bytes from host memory to stack + slot * bytes_per_slot
+ *                   molora_hotset_commit(slot): writes the table entry after the weights (stream order) and records an
+ *                       event; the adapter counts as resident once that event has completed (polled, never waited for)
+ * Life of a step:   molora_hotset_pin(adapter) for every adapter the step routes to (MOLORA_ERR_NOT_RESIDENT if it is not
+ *                   there yet), enqueue the step, molora_hotset_unpin(slot) when the step has completed.  A pinned slot
+ *                   is never chosen for eviction; MOLORA_ERR_BUSY if no slot can be had.
+ * table_dev must hold -1 in every entry before the first load (the caller fills it).  S * M <= 256.  All functions are
+ * thread-safe.  backend: NULL for the CUDA runtime (cudaMemcpyAsync from preferably pinned memory, cudaEvent*), or
+ * replacements for the four calls (a fake stream for tests, another copy engine); `user` is passed through.
+ * The manager allocates host memory for its own bookkeeping only, never device memory. */
+typedef struct molora_hotset molora_hotset_t;
+typedef struct {
+    molora_status_t (*copy_h2d)(void *dst_dev, const void *src_host, size_t bytes, void *stream, void *user);
+    molora_status_t (*event_record)(void **event /* in/out: created on first use */, void *stream, void *user);
+    int32_t (*event_done)(void *event, void *user); /* 1 if everything before the record has completed (no waiting) */
+    void (*event_destroy)(void *event, void *user);
+    void *user;
+} molora_hotset_backend_t;
+molora_status_t molora_hotset_create(int32_t S, int32_t M, int32_t n_catalog, int32_t *table_dev,
+                                     const molora_hotset_backend_t *backend, molora_hotset_t **out);
+void molora_hotset_destroy(molora_hotset_t *h);
+int32_t molora_hotset_slot_of(molora_hotset_t *h, int32_t adapter);  /* slot of a resident adapter, else -1 */
+int32_t molora_hotset_adapter_in(molora_hotset_t *h, int32_t slot);  /* sigma(slot): adapter id, -1 if the slot is free */
+molora_status_t molora_hotset_pin(molora_hotset_t *h, int32_t adapter, int32_t *slot_out);
+molora_status_t molora_hotset_unpin(molora_hotset_t *h, int32_t slot);
+molora_status_t molora_hotset_begin_load(molora_hotset_t *h, int32_t adapter, void *maintenance_stream, int32_t *slot_out,
+                                         int32_t *fresh_out /* 1: upload + commit this slot; 0: already resident or on its way */,
+                                         int32_t *evicted_out /* adapter that lost its slot, -1 if none; may be NULL */);
+molora_status_t molora_hotset_upload(molora_hotset_t *h, int32_t slot, void *stack_dev, const void *weights_host,
+                                     size_t bytes_per_slot, void *maintenance_stream);
+molora_status_t molora_hotset_commit(molora_hotset_t *h, int32_t slot, void *maintenance_stream);
+/* Compositional routing through the slot table (Definition 3.2 with the adapter axis indexed by slot):
+ *     r_out[i] = slot_table_dev[adapter_id[i]] * M + m(ids[i]);  -1 if the id lies in no range, the adapter id is outside
+ *     [0, n_catalog) or the adapter is not resident (MOLORA_DEV_ID_OUT_OF_RANGE is then OR-ed into dev_status).
+ * The result indexes stacks of S * M targets: C = S * M in molora_group / molora_apply. */
+molora_status_t molora_route_hotset(const int32_t *ids, const int32_t *adapter_id, int64_t N, const int32_t *breaks,
+                                    int32_t M, const int32_t *slot_table_dev, int32_t n_catalog, int32_t S,
+                                    int32_t *r_out, uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Failure-detection self-test.  Every device-side wait of the tensor-core apply kernel (on an mbarrier that a

@@ -10,6 +10,6 @@ from .binding import (  # noqa: F401
     molora_route_vocab, molora_route_composite, molora_route_mlp, molora_route_mlp_workspace_bytes, molora_route_gate, molora_route_gate_workspace_bytes, molora_route_gate_noalloc, molora_selftest_bounded_wait,
     molora_group_workspace_bytes, molora_group,
     molora_apply_workspace_bytes, molora_apply, molora_apply_batched, molora_group_apply_batched, molora_topk_softmax, molora_apply_topk,
-    ProjDesc, F32, BF16,
+    ProjDesc, F32, BF16, HotSet, molora_route_hotset,
     HostProj, molora_forward_host, molora_forward_host_arena_bytes, ROUTE_VOCAB, ROUTE_GATE, ROUTE_GIVEN,
 )

@@ -43,6 +43,17 @@ class _ProjDescC(ctypes.Structure):
                 ("rank", ctypes.c_int32), ("scale", ctypes.c_float), ("row_scale", ctypes.c_void_p)]
 
 
+COPY_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p)
+EVENT_RECORD_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.POINTER(ctypes.c_void_p), ctypes.c_void_p, ctypes.c_void_p)
+EVENT_DONE_FN = ctypes.CFUNCTYPE(ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p)
+EVENT_DESTROY_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_void_p)
+
+
+class _HotsetBackendC(ctypes.Structure):
+    _fields_ = [("copy_h2d", COPY_FN), ("event_record", EVENT_RECORD_FN), ("event_done", EVENT_DONE_FN),
+                ("event_destroy", EVENT_DESTROY_FN), ("user", ctypes.c_void_p)]
+
+
 def lib_path() -> str:
     return LIB_PATH
 
@@ -51,7 +62,8 @@ def exported_symbols() -> List[str]:
     """Names of the functions include/molora.h declares (parsed from the header)."""
     with open(os.path.join(ROOT, "include", "molora.h")) as f:
         text = f.read()
-    return sorted(set(re.findall(r"\b(molora_[a-z_]+)\s*\(", text)))
+    names = set(re.findall(r"\b(molora_[a-z_]+)\s*\(", text))
+    return sorted(n for n in names if not n.endswith("_t"))          # type names before function-pointer members
 
 
 def load_library():
@@ -109,6 +121,22 @@ def load_library():
                                                     i32]
     lib.molora_forward_host.argtypes = [ctypes.c_int, vp, vp, i32, vp, vp, i32, ctypes.POINTER(_HostProjC), i32,
                                         ctypes.c_int, i64, i32, vp, sz, vp, vp]
+    lib.molora_hotset_create.argtypes = [i32, i32, i32, vp, ctypes.POINTER(_HotsetBackendC), ctypes.POINTER(vp)]
+    lib.molora_hotset_destroy.argtypes = [vp]
+    lib.molora_hotset_destroy.restype = None
+    lib.molora_hotset_slot_of.argtypes = [vp, i32]
+    lib.molora_hotset_slot_of.restype = i32
+    lib.molora_hotset_adapter_in.argtypes = [vp, i32]
+    lib.molora_hotset_adapter_in.restype = i32
+    lib.molora_hotset_pin.argtypes = [vp, i32, ctypes.POINTER(i32)]
+    lib.molora_hotset_unpin.argtypes = [vp, i32]
+    lib.molora_hotset_begin_load.argtypes = [vp, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.molora_hotset_upload.argtypes = [vp, i32, vp, vp, sz, vp]
+    lib.molora_hotset_commit.argtypes = [vp, i32, vp]
+    lib.molora_route_hotset.argtypes = [vp, vp, i64, vp, i32, vp, i32, i32, vp, vp, vp]
+    for name in ("molora_hotset_create", "molora_hotset_pin", "molora_hotset_unpin", "molora_hotset_begin_load",
+                 "molora_hotset_upload", "molora_hotset_commit", "molora_route_hotset"):
+        getattr(lib, name).restype = ctypes.c_int
     for name in ("molora_route_vocab", "molora_route_gate", "molora_group", "molora_apply", "molora_apply_batched",
                  "molora_forward_host"):
         getattr(lib, name).restype = ctypes.c_int
@@ -514,3 +542,84 @@ def molora_forward_host(router: int, projs, arena: torch.Tensor, route_src: Opti
     _check("molora_forward_host", lib.molora_forward_host(
         router, _ptr(route_src), _ptr(breaks), M, _ptr(G), _ptr(bias), gate_proj, arr, len(arr), dt, N, C,
         _ptr(arena), arena.numel() * arena.element_size(), _ptr(dev_status), _stream(stream)))
+
+
+# ----------------------------------------------------------------------------- hot-set slot table (Definition 5.1)
+ERR_BUSY, ERR_NOT_RESIDENT = 5, 6
+
+
+class HotSet:
+    """Handle of a molora_hotset_t: S slots x M modalities over a catalog of n_catalog adapters.  ``table`` is the device
+    int32[n_catalog] inverse slot table (filled with -1 by the caller); with ``backend`` (a _HotsetBackendC of callbacks)
+    the copies and events go there instead of the CUDA runtime.  Marshalling only: every decision is the library's."""
+
+    def __init__(self, S: int, M: int, n_catalog: int, table, backend=None):
+        self.lib = load_library()
+        self.S, self.M, self.n_catalog, self.table, self._backend = S, M, n_catalog, table, backend
+        h = ctypes.c_void_p()
+        tptr = table.data_ptr() if hasattr(table, "data_ptr") else int(table)
+        _check("molora_hotset_create", self.lib.molora_hotset_create(S, M, n_catalog, ctypes.c_void_p(tptr),
+                                                                      ctypes.byref(backend) if backend is not None else None,
+                                                                      ctypes.byref(h)))
+        self.h = h
+
+    def close(self):
+        if self.h:
+            self.lib.molora_hotset_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        self.close()
+
+    def slot_of(self, adapter: int) -> int:
+        return int(self.lib.molora_hotset_slot_of(self.h, adapter))
+
+    def adapter_in(self, slot: int) -> int:
+        return int(self.lib.molora_hotset_adapter_in(self.h, slot))
+
+    def pin(self, adapter: int) -> int:
+        slot = ctypes.c_int32(-1)
+        _check("molora_hotset_pin", self.lib.molora_hotset_pin(self.h, adapter, ctypes.byref(slot)))
+        return slot.value
+
+    def unpin(self, slot: int) -> None:
+        _check("molora_hotset_unpin", self.lib.molora_hotset_unpin(self.h, slot))
+
+    def begin_load(self, adapter: int, stream=None) -> Tuple[int, bool, int]:
+        """Returns (slot, fresh, evicted adapter or -1): upload and commit only when fresh; raises MoloraError with status
+        ERR_BUSY if no slot can be had."""
+        slot, fresh, ev = ctypes.c_int32(-1), ctypes.c_int32(0), ctypes.c_int32(-1)
+        _check("molora_hotset_begin_load", self.lib.molora_hotset_begin_load(self.h, adapter, ctypes.c_void_p(_stream_or_raw(stream)),
+                                                                              ctypes.byref(slot), ctypes.byref(fresh), ctypes.byref(ev)))
+        return slot.value, bool(fresh.value), ev.value
+
+    def upload(self, slot: int, stack, weights_host, stream=None) -> None:
+        """Copy one adapter's weights (host tensor shaped like stack[slot]) into stack[slot] on the maintenance stream."""
+        nbytes = weights_host.numel() * weights_host.element_size()
+        if hasattr(stack, "shape") and nbytes != stack[0].numel() * stack.element_size():
+            raise ValueError("weights do not have the size of one slot of the stack")
+        _check("molora_hotset_upload", self.lib.molora_hotset_upload(self.h, slot, ctypes.c_void_p(stack.data_ptr()),
+                                                                      ctypes.c_void_p(weights_host.data_ptr()), nbytes,
+                                                                      ctypes.c_void_p(_stream_or_raw(stream))))
+
+    def commit(self, slot: int, stream=None) -> None:
+        _check("molora_hotset_commit", self.lib.molora_hotset_commit(self.h, slot, ctypes.c_void_p(_stream_or_raw(stream))))
+
+
+def _stream_or_raw(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else 0
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def molora_route_hotset(ids: torch.Tensor, adapter_id: torch.Tensor, breaks: torch.Tensor, slot_table: torch.Tensor, S: int,
+                        r_out: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """r[i] = slot_table[adapter_id[i]] * M + modality(ids[i]); -1 where the adapter is not resident."""
+    lib = load_library()
+    N, M = ids.numel(), breaks.numel() - 1
+    if r_out is None:
+        r_out = torch.empty(N, dtype=torch.int32, device=ids.device)
+    _check("molora_route_hotset", lib.molora_route_hotset(_ptr(_i32_dev(ids, "ids")), _ptr(_i32_dev(adapter_id, "adapter_id")), N,
+                                                          _ptr(_i32_dev(breaks, "breaks")), M, _ptr(_i32_dev(slot_table, "slot_table")),
+                                                          slot_table.numel(), S, _ptr(r_out), _ptr(dev_status), _stream(stream)))
+    return r_out

@@ -141,6 +141,8 @@ const char* molora_status_string(molora_status_t status)
         case MOLORA_ERR_UNSUPPORTED: return "unsupported shape, rank or dtype";
         case MOLORA_ERR_WORKSPACE: return "workspace missing or too small";
         case MOLORA_ERR_CUDA: return "CUDA runtime error";
+        case MOLORA_ERR_BUSY: return "every hot-set slot is in use";
+        case MOLORA_ERR_NOT_RESIDENT: return "adapter not resident in the hot set";
     }
     return "unknown status";
 }

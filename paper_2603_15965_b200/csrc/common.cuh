@@ -220,7 +220,7 @@ __device__ __forceinline__ void find_tile_bisect(const int32_t* offs, const int3
 // adapter == nullptr: vocabulary routing; otherwise the compositional gate (r = adapter[i] * M + m)
 molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M,
                                    const int32_t* adapter, int32_t n_adapters, int32_t* r_out, uint32_t* dev_status,
-                                   cudaStream_t s);
+                                   cudaStream_t s, const int32_t* slot_of = nullptr, int32_t n_catalog = 0);
 // tcgen05 gate (bf16 activations, C > 4, d a multiple of 64, at least 1024 tokens).
 bool gate_umma_eligible(int64_t N, int32_t d, int32_t C);
 size_t route_gate_umma_workspace_bytes(int32_t d, int32_t C);

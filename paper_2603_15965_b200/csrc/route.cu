@@ -13,11 +13,14 @@ namespace molora {
 // (an empty range b_m == b_{m+1} can hold no id and is skipped by the count).  M-1 integer compares
 // per token, as the paper notes for Theorem 3.4; boundaries live in shared memory.
 // ------------------------------------------------------------------------------------------------
+// With `slot_of` non-null as well, adapter[i] is an adapter id of a catalog and slot_of[id] the hot-set slot that holds
+// it (Definition 5.1), -1 if it is not resident: the target is slot * M + m.
 // With `adapter` non-null the kernel is the compositional gate of Algorithm 1 (Definition 3.2): the modality m found
 // from the id is combined with the token's adapter index a (request metadata) into the composite target a * M + m.
 __global__ void __launch_bounds__(256) route_vocab_kernel(const int32_t* __restrict__ ids, int64_t N,
                                                           const int32_t* __restrict__ breaks, int M,
                                                           const int32_t* __restrict__ adapter, int n_adapters,
+                                                          const int32_t* slot_of, int n_catalog,
                                                           int32_t* __restrict__ r_out, uint32_t* dev_status)
 {
     __shared__ int32_t b[MOLORA_MAX_ADAPTERS + 1];
@@ -43,7 +46,9 @@ __global__ void __launch_bounds__(256) route_vocab_kernel(const int32_t* __restr
         }
         bool inside = (v >= b[0]) && (v < b[M]);
         if (adapter != nullptr) {
-            const int32_t a = __ldg(adapter + i);
+            int32_t a = __ldg(adapter + i);
+            if (slot_of != nullptr)                // hot-set: adapter id -> slot through the slot table's inverse (may be
+                a = (a >= 0 && a < n_catalog) ? __ldcg(slot_of + a) : -1;      // rewritten by the maintenance stream)
             inside = inside && a >= 0 && a < n_adapters;
             m += a * M;
         }
@@ -56,14 +61,14 @@ __global__ void __launch_bounds__(256) route_vocab_kernel(const int32_t* __restr
 
 molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t* breaks, int32_t M,
                                    const int32_t* adapter, int32_t n_adapters, int32_t* r_out, uint32_t* dev_status,
-                                   cudaStream_t s)
+                                   cudaStream_t s, const int32_t* slot_of, int32_t n_catalog)
 {
     if (N == 0) return MOLORA_OK;
     const int threads = 256;
     const int64_t want = ceil_div64(N, threads);
     const int blocks = (int)(want < 148 * 8 ? want : 148 * 8);
     return cuda_ok(launch_kernel(route_vocab_kernel, dim3(blocks), dim3(threads), 0, s, 1, false, ids, N, breaks, M, adapter,
-                                  n_adapters, r_out, dev_status));
+                                  n_adapters, slot_of, n_catalog, r_out, dev_status));
 }
 
 // ------------------------------------------------------------------------------------------------
