@@ -376,7 +376,7 @@ def measure(name, args, env, headline):
                        "note": "one step per CUDA-graph replay, event pair around each replay (includes the graph launch)"}
 
         kpass = None
-        if name.startswith("c5") and not args.profile and args.launch == "graph":
+        if name.startswith(("c5", "t6-")) and not args.profile and args.launch == "graph":
             kpass = run_kpass(args, env, w, sets, shared, stream, capture_pass, apply_ms, K, n_var)
         torch.cuda.synchronize()
 

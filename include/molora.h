@@ -261,9 +261,12 @@ int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t *projs, i
  *   logits   device fp32 [N, C], 1 <= k <= C <= 32
  *   idx_out  device int32 [k, N] slot-major: idx_out[j*N + i] = the j-th choice of token i (j = 0: largest logit;
  *            equal logits: lowest index first);  w_out  device fp32 [k, N], softmax over the k kept logits
- * molora_apply_topk applies the k choices as k passes of (group, apply) with the weights as per-token factors: within
- * a pass every row of y is touched by one adapter only, so there are no conflicting updates and the result is
- * deterministic; y is rounded to its storage type once per pass.
+ * molora_apply_topk applies the k choices.  Where the streaming kernel can take the call (bf16, k in {2, 4}, rank x k in
+ * {16, 32, 64}, C^k <= 256, below the tcgen05 crossover) it does so in ONE pass over x and y: tokens are grouped by their
+ * SET of kept adapters, a segment shrinks against the stacked A of its k adapters, the k slices of t are weighted per
+ * token and one expand against the stacked B adds all k deltas before the single rounding.  Otherwise: k passes of
+ * (group, apply) with the weights as per-token factors; within a pass every row of y is touched by one adapter only, so
+ * there are no conflicting updates and the result is deterministic, but y is rounded to its storage type once per pass.
  *   projs    HOST array of P descriptors as for molora_apply_batched (their row_scale is ignored)
  *   ws       device scratch of at least molora_apply_topk_workspace_bytes(projs, P, N, C) bytes, 256-byte aligned,
  *            zero-filled before its first use (see molora_apply) */

@@ -470,8 +470,9 @@ molora_status_t molora_topk_softmax(const float* logits, int64_t N, int32_t C, i
 
 namespace {
 struct TopkPlan {
-    size_t counts, offsets, perm, apply_ws, apply_ws_bytes, total;
+    size_t counts, offsets, perm, sets, wsorted, apply_ws, apply_ws_bytes, total;
 };
+constexpr int kTopkMaxParts = 4;
 TopkPlan plan_topk(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C)
 {
     auto a256 = [](size_t v) { return (v + 255) & ~(size_t)255; };
@@ -482,11 +483,38 @@ TopkPlan plan_topk(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_
     for (int i = 0; i < P; ++i)
         pl.apply_ws_bytes += molora_apply_workspace_bytes(N, C, projs[i].d_in, projs[i].d_out, projs[i].rank);
     size_t off = a256(pl.apply_ws_bytes);
-    pl.counts = off;   off = a256(off + sizeof(int32_t) * (size_t)C);
-    pl.offsets = off;  off = a256(off + sizeof(int32_t) * (size_t)(C + 1));
-    pl.perm = off;     off = a256(off + sizeof(int32_t) * (size_t)(N > 0 ? N : 1));
+    // grouping outputs sized for adapter SETS as well (the single-pass path groups by set: up to 256 of them)
+    const size_t n1 = (size_t)(N > 0 ? N : 1);
+    pl.counts = off;   off = a256(off + sizeof(int32_t) * (size_t)MOLORA_MAX_ADAPTERS);
+    pl.offsets = off;  off = a256(off + sizeof(int32_t) * (size_t)(MOLORA_MAX_ADAPTERS + 1));
+    pl.perm = off;     off = a256(off + sizeof(int32_t) * n1);
+    pl.sets = off;     off = a256(off + sizeof(int32_t) * n1);
+    pl.wsorted = off;  off = a256(off + sizeof(float) * n1 * kTopkMaxParts);
     pl.total = off;
     return pl;
+}
+
+// Eq. 8 in ONE pass over x and y: tokens are grouped by their SET of kept adapters, a segment's shrink runs against the
+// stacked A of its k adapters (rank k x r), the k slices of t are weighted per token, and one expand against the stacked
+// B adds all k deltas before the single rounding.  Taken when every projection can run on the streaming kernel with the
+// stacked rank (bf16, r x k in {16, 32, 64}, k in {2, 4}, C^k <= 256 sets) and the call is not one the tcgen05 kernel
+// would take pass by pass.
+bool topk_single_pass(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C, int32_t k)
+{
+    if (dt != MOLORA_BF16 || (k != 2 && k != 4) || N < 1) return false;
+    int64_t sets = 1;
+    for (int j = 0; j < k; ++j) sets *= C;
+    if (sets > MOLORA_MAX_ADAPTERS) return false;
+    const int64_t small = tune(kTuneSmallPath);
+    if (small != 0 && small != 1) return false;                     // a test or a measurement asks for another kernel
+    double bytes = 0.0;
+    for (int i = 0; i < P; ++i) {
+        const int stacked = projs[i].rank * k;
+        if (!stream_eligible(projs[i], dt) || (stacked != 16 && stacked != 32 && stacked != 64)) return false;
+        if (projs[i].rank != projs[0].rank) return false;
+        bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
+    }
+    return !use_umma(projs[0].rank, N, bytes);
 }
 }  // namespace
 
@@ -509,6 +537,29 @@ molora_status_t molora_apply_topk(const molora_proj_desc_t* projs, int32_t P, mo
     int32_t* offsets = reinterpret_cast<int32_t*>(base + pl.offsets);
     int32_t* perm = reinterpret_cast<int32_t*>(base + pl.perm);
     molora_proj_desc_t pass[MOLORA_MAX_PROJECTIONS];
+    if (topk_single_pass(projs, P, dt, N, C, k)) {
+        for (int i = 0; i < P; ++i) {
+            const molora_status_t st = check_proj(projs[i], dt);
+            if (st != MOLORA_OK) return st;
+        }
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        int32_t* sets = reinterpret_cast<int32_t*>(base + pl.sets);
+        float* wsorted = reinterpret_cast<float*>(base + pl.wsorted);
+        int32_t n_sets = 1;
+        for (int j = 0; j < k; ++j) n_sets *= C;
+        for (int i = 0; i < P; ++i) {
+            pass[i] = projs[i];
+            pass[i].rank = projs[i].rank * k;       // the stacked rank of a set
+            pass[i].row_scale = wsorted;            // [k][N], in the order of the set's adapters
+        }
+        molora_status_t st = launch_topk_sets(idx, w, N, C, k, sets, wsorted, s);
+        if (st != MOLORA_OK) return st;
+        if (group_apply_stream_eligible(N))         // the CTAs of the apply group the sets themselves
+            return launch_group_apply_stream_sets(sets, pass, P, N, C, k, counts, offsets, perm, dev_status, s);
+        st = molora_group(sets, N, n_sets, counts, offsets, perm, nullptr, 0, dev_status, stream);
+        if (st != MOLORA_OK) return st;
+        return launch_apply_stream_sets(pass, P, N, C, k, offsets, perm, dev_status, s);
+    }
     for (int32_t j = 0; j < k; ++j) {               // one (group, apply) pass per kept adapter slot
         for (int i = 0; i < P; ++i) {
             pass[i] = projs[i];

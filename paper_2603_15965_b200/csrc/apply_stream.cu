@@ -55,12 +55,23 @@ struct StreamParams {
     const int32_t* perm;
     uint32_t* dev_status;
     int32_t N, P, C, max_rows;                // segments with at least max_rows rows belong to the tcgen05 kernel
+    // Top-k routing in one pass (Eq. 8): a segment is a SET of `parts` adapters (its index spells them in base `cbase`,
+    // most significant first), the launch's rank R is parts x the adapters' rank, A_c and B_c are gathered from the
+    // parts' adapters, and row_scale holds the routing weights [parts][N].  parts == 1: plain top-1 routing.
+    int32_t parts, cbase;
     // grouping variant only: the routing decisions and where counts / offsets / perm are written (as by molora_group)
     const int32_t* r;
     int32_t* counts_out;
     int32_t* offsets_out;
     int32_t* perm_out;
 };
+// adapter of part j of segment `seg`
+__device__ __forceinline__ int fs_part_adapter(const StreamParams& prm, int seg, int j)
+{
+    int div = 1;
+    for (int k = prm.parts - 1; k > j; --k) div *= prm.cbase;
+    return (seg / div) % prm.cbase;
+}
 // (projection, slice of d_out) pairs of the projections of the launch's rank; projection p owns [start[p], start[p + 1]).
 struct FsUnits {
     int32_t start[MOLORA_MAX_PROJECTIONS + 1];
@@ -226,8 +237,14 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             const int64_t tok = rowlane ? fs_token(prm, perm_s, it.row0 + myrow) : 0;
             const char* xrow = static_cast<const char*>(pd.x) + tok * pd.ldx * 2;
             char* yrow = static_cast<char*>(pd.y) + tok * pd.ldy * 2 + (int64_t)it.col0 * 2;
-            const char* Ac = static_cast<const char*>(pd.A) + (int64_t)it.seg * pd.d_in * R * 2;
-            const char* Bc = static_cast<const char*>(pd.B) + ((int64_t)it.seg * R * pd.d_out + it.col0) * 2;
+            const int parts = prm.parts, pr = R / parts;            // adapters per segment, rank of each
+            // my weight source: lane RPW + j loads part j's rows of A; the lanes after RPW load one row of B each
+            const int apart = min(max(lane - RPW, 0), parts - 1);
+            const char* Ac = static_cast<const char*>(pd.A) + (int64_t)fs_part_adapter(prm, it.seg, apart) * pd.d_in * pr * 2;
+            const int brow = cw * (R / kFsCopyWarps) + max(lane - RPW, 0);          // my row of the stacked B (lanes RPW ..)
+            const int bpart = min(brow / pr, parts - 1);
+            const char* Bc = static_cast<const char*>(pd.B) +
+                             (((int64_t)fs_part_adapter(prm, it.seg, bpart) * pr + (brow - bpart * pr)) * pd.d_out + it.col0) * 2;
             const int myrows = max(0, min(RPW, it.rows - cw * RPW));
             for (int j = 0; j < it.nks + it.ne; ++j, ++g) {
                 const uint32_t s = g % NS;
@@ -239,14 +256,16 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                     const int k0 = j * Cfg::CH, kc = min(Cfg::CH, pd.d_in - k0);
                     const uint32_t xbytes = (uint32_t)kc * 2u;
                     // my quarter of the chunk's rows of A_c (kc is a multiple of 32: a quarter is a multiple of 16 bytes)
-                    const uint32_t aq = (uint32_t)kc * R * 2u / kFsCopyWarps;
+                    const uint32_t ablock = (uint32_t)kc * pr * 2u;                // one part's rows of A for this chunk
+                    const uint32_t aq = ablock / kFsCopyWarps;
                     if (lane == 0) {
                         st_bytes[cw][s] = 0;
-                        mbar_arrive_expect_tx(bar, (uint32_t)myrows * xbytes + aq);
+                        mbar_arrive_expect_tx(bar, (uint32_t)myrows * xbytes + (uint32_t)parts * aq);
                     }
                     __syncwarp();
                     if (rowlane) bulk_load(sb + myrow * Cfg::RP, xrow + (int64_t)k0 * 2, xbytes, bar);
-                    if (lane == RPW) bulk_load(sb + Cfg::ROWBYTES + cw * aq, Ac + (int64_t)k0 * R * 2 + cw * aq, aq, bar);
+                    if (lane >= RPW && lane < RPW + parts)
+                        bulk_load(sb + Cfg::ROWBYTES + apart * ablock + cw * aq, Ac + (int64_t)k0 * pr * 2 + cw * aq, aq, bar);
                 } else {
                     const int c0 = (j - it.nks) * Cfg::CH, nc = min(Cfg::CH, pd.d_out - it.col0 - c0);
                     const uint32_t rowbytes = (uint32_t)nc * 2u;
@@ -260,7 +279,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                     if (rowlane) bulk_load(sb + myrow * Cfg::RP, yrow + (int64_t)c0 * 2, rowbytes, bar);
                     if (lane >= RPW && lane < RPW + R / kFsCopyWarps) {
                         const int k = cw * (R / kFsCopyWarps) + lane - RPW;
-                        bulk_load(sb + Cfg::ROWBYTES + k * Cfg::RP, Bc + ((int64_t)k * pd.d_out + c0) * 2, rowbytes, bar);
+                        bulk_load(sb + Cfg::ROWBYTES + k * Cfg::RP, Bc + (int64_t)c0 * 2, rowbytes, bar);
                     }
                 }
             }
@@ -304,7 +323,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             const uint32_t s = g % NS;
             const uint32_t xs = stage0 + s * Cfg::STAGE, as = xs + Cfg::ROWBYTES;
             wait_bar(smem_u32(&full_s[s]), (g / NS) & 1u, &abort_s, prm.dev_status);
-            const int nb = min(Cfg::CH, pd.d_in - j * Cfg::CH) / 32;
+            const int kcols = min(Cfg::CH, pd.d_in - j * Cfg::CH), nb = kcols / 32;
+            const int pr = R / prm.parts;
             for (int b = warp; b < nb; b += kFsWarps) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {                           // two k16 steps per block
@@ -312,7 +332,12 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                     const int m = lane >> 3;                            // matrix of the x4 load this lane addresses
 #pragma unroll
                     for (int n16 = 0; n16 < NT / 2; ++n16)
-                        fs_ldsm_t(bf[n16], as + (b * 32 + h * 16 + (m & 1) * 8 + (lane & 7)) * (R * 2) + (n16 * 16 + (m >> 1) * 8) * 2);
+                        {
+                            // the chunk's rows of A: one dense [k][pr] block per part (pr >= 16: an n16 tile lies in one part)
+                            const int part = (n16 * 16) / pr, pc = n16 * 16 - part * pr;
+                            fs_ldsm_t(bf[n16], as + part * (kcols * pr * 2) + (b * 32 + h * 16 + (m & 1) * 8 + (lane & 7)) * (pr * 2) +
+                                                   (pc + (m >> 1) * 8) * 2);
+                        }
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
                         if (mt == 0 || two) {
@@ -358,7 +383,8 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
                     const int row = e4 * 4 / R;
                     float sc = pd.scale;           // times the token's routing weight, if the caller passes per-token factors
                     if (row >= it.rows) v = make_float4(0.f, 0.f, 0.f, 0.f);   // rows past the tile hold stale shared memory
-                    else if (rscale != nullptr) sc *= __ldg(rscale + fs_token(prm, perm_s, it.row0 + row));
+                    else if (rscale != nullptr)    // (top-k in one pass: the weight of the part this column belongs to)
+                        sc *= __ldg(rscale + (int64_t)((e4 * 4 % R) / (R / prm.parts)) * prm.N + fs_token(prm, perm_s, it.row0 + row));
                     *reinterpret_cast<float4*>(&tfin[e4 * 4]) = make_float4(v.x * sc, v.y * sc, v.z * sc, v.w * sc);
                 }
                 fence_proxy_async_smem();          // my writes to the stage are ordered before the copies that refill it
@@ -541,6 +567,7 @@ static molora_status_t stream_enqueue(const molora_proj_desc_t* projs, int32_t P
     prm.P = P;
     prm.C = C;
     prm.N = (int32_t)N;
+    if (prm.parts < 1) prm.parts = 1;
     // rank 16: the short tile while its tiles of all projections (nearly) fit one wave of CTAs
     int p16 = 0;
     for (int i = 0; i < P; ++i) p16 += projs[i].rank == 16;
@@ -578,7 +605,52 @@ molora_status_t launch_apply_stream(const molora_proj_desc_t* projs, int32_t P, 
     prm.max_rows = max_rows;
     prm.r = nullptr;
     prm.counts_out = prm.offsets_out = prm.perm_out = nullptr;
+    prm.parts = 1;
+    prm.cbase = C;
     return stream_enqueue(projs, P, N, C, prm, false, s);
+}
+
+// Top-k routing in one pass: `projs` carry the STACKED rank (parts x the adapters' rank) and row_scale = weights
+// [parts][N]; offsets / perm group the tokens by adapter set, C_sets = cbase^parts segments.
+molora_status_t launch_apply_stream_sets(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t cbase, int32_t parts,
+                                         const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, cudaStream_t s)
+{
+    if (N == 0 || P == 0) return MOLORA_OK;
+    StreamParams prm;
+    prm.offsets = offsets;
+    prm.perm = perm;
+    prm.dev_status = dev_status;
+    prm.max_rows = INT32_MAX;
+    prm.r = nullptr;
+    prm.counts_out = prm.offsets_out = prm.perm_out = nullptr;
+    prm.parts = parts;
+    prm.cbase = cbase;
+    int32_t sets = 1;
+    for (int j = 0; j < parts; ++j) sets *= cbase;
+    return stream_enqueue(projs, P, N, sets, prm, false, s);
+}
+
+// ... and started from the set indices (at most 4096 tokens): grouping by set and apply in one launch.  (Forming the sets
+// inside this kernel as well was measured and lost: every CTA repeats the sort, 23.2 against 21.5 us at 4096 tokens.)
+molora_status_t launch_group_apply_stream_sets(const int32_t* sets, const molora_proj_desc_t* projs, int32_t P, int64_t N,
+                                               int32_t cbase, int32_t parts, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                               uint32_t* dev_status, cudaStream_t s)
+{
+    if (N == 0 || P == 0) return MOLORA_OK;
+    StreamParams prm;
+    prm.offsets = nullptr;
+    prm.perm = nullptr;
+    prm.dev_status = dev_status;
+    prm.max_rows = INT32_MAX;
+    prm.r = sets;
+    prm.counts_out = counts;
+    prm.offsets_out = offsets;
+    prm.perm_out = perm;
+    prm.parts = parts;
+    prm.cbase = cbase;
+    int32_t n_sets = 1;
+    for (int j = 0; j < parts; ++j) n_sets *= cbase;
+    return stream_enqueue(projs, P, N, n_sets, prm, true, s);
 }
 
 bool group_apply_stream_eligible(int64_t N) { return N >= 1 && N <= kFsPermCache; }
@@ -596,6 +668,8 @@ molora_status_t launch_group_apply_stream(const int32_t* r, const molora_proj_de
     prm.counts_out = counts;
     prm.offsets_out = offsets;
     prm.perm_out = perm;
+    prm.parts = 1;
+    prm.cbase = C;
     return stream_enqueue(projs, P, N, C, prm, true, s);
 }
 

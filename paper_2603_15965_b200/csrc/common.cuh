@@ -246,6 +246,9 @@ molora_status_t launch_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, i
 // Top-k selection and softmax over router logits (Eq. 8); idx / w slot-major [k][N].
 molora_status_t launch_topk_softmax(const float* logits, int64_t N, int32_t C, int32_t k, int32_t* idx_out, float* w_out,
                                     cudaStream_t s);
+// Adapter sets of top-k routing (sorted adapters of a token spelled in base C) and the weights in the same order.
+molora_status_t launch_topk_sets(const int32_t* idx, const float* w, int64_t N, int32_t C, int32_t k, int32_t* set_out,
+                                 float* w_out, cudaStream_t s);
 size_t group_workspace_bytes(int64_t N, int32_t C);
 molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
                              void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
@@ -267,6 +270,14 @@ bool decode_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
 molora_status_t launch_apply_stream(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                     const int32_t* offsets, const int32_t* perm, int32_t max_rows, uint32_t* dev_status,
                                     cudaStream_t s);
+// The same kernel for top-k routing in one pass: segments are adapter sets (cbase^parts of them), the projections carry
+// the stacked rank parts x r and row_scale = weights [parts][N].
+bool stream_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
+molora_status_t launch_apply_stream_sets(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t cbase, int32_t parts,
+                                         const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, cudaStream_t s);
+molora_status_t launch_group_apply_stream_sets(const int32_t* sets, const molora_proj_desc_t* projs, int32_t P, int64_t N,
+                                               int32_t cbase, int32_t parts, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                               uint32_t* dev_status, cudaStream_t s);
 // The same kernel started from the routing decisions r: grouping (counts, offsets, perm as molora_group writes them)
 // and apply in one launch; all projections of one rank, at most 4096 tokens.
 bool group_apply_stream_eligible(int64_t N);

@@ -525,6 +525,50 @@ molora_status_t launch_topk_softmax(const float* logits, int64_t N, int32_t C, i
                                  (int)C, (int)k, idx_out, w_out));
 }
 
+// Top-k routing in one pass: the k adapters of a token, sorted by index, name a SET; its index spells them in base C
+// (most significant first), and the weights are stored in the same order.  Tokens with an adapter outside [0, C) are
+// left unrouted.  k <= 4.
+__global__ void __launch_bounds__(256) topk_sets_kernel(const int32_t* __restrict__ idx, const float* __restrict__ w, int64_t N,
+                                                        int C, int k, int32_t* __restrict__ set_out, float* __restrict__ w_out)
+{
+    ptx::grid_dependency_sync();
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    int a[4];
+    float f[4];
+    bool ok = true;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        a[j] = j < k ? __ldg(idx + (int64_t)j * N + i) : 0x7FFFFFFF;
+        f[j] = j < k ? __ldg(w + (int64_t)j * N + i) : 0.f;
+        ok = ok && (j >= k || (a[j] >= 0 && a[j] < C));
+    }
+#pragma unroll
+    for (int p = 0; p < 3; ++p)                     // three rounds of a bubble sort over four entries
+#pragma unroll
+        for (int j = 0; j < 3 - p; ++j)
+            if (a[j] > a[j + 1]) {
+                const int ta = a[j]; a[j] = a[j + 1]; a[j + 1] = ta;
+                const float tf = f[j]; f[j] = f[j + 1]; f[j + 1] = tf;
+            }
+    int set = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (j < k) {
+            set = set * C + a[j];
+            w_out[(int64_t)j * N + i] = f[j];
+        }
+    set_out[i] = ok ? set : -1;
+}
+
+molora_status_t launch_topk_sets(const int32_t* idx, const float* w, int64_t N, int32_t C, int32_t k, int32_t* set_out,
+                                 float* w_out, cudaStream_t s)
+{
+    if (N == 0) return MOLORA_OK;
+    return cuda_ok(launch_kernel(topk_sets_kernel, dim3((unsigned)ceil_div64(N, 256)), dim3(256), 0, s, 1, false, idx, w, N, (int)C,
+                                 (int)k, set_out, w_out));
+}
+
 size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
 {
     if (xdt != MOLORA_BF16) return 0;

@@ -86,7 +86,7 @@ class Workload:
 
 def _rng(cfg_index: int, stream: int) -> np.random.Generator:
     """Child stream ``stream`` of configuration ``cfg_index`` (0 = routing source + weights, 1+b = batch b)."""
-    ss = np.random.SeedSequence(ROOT_SEED).spawn(9)[cfg_index]      # children 0..4: c1..c5; 7, 8: the sweeps
+    ss = np.random.SeedSequence(ROOT_SEED).spawn(9)[cfg_index]      # children 0..4: c1..c5; 6, 7, 8: the sweeps
     return np.random.default_rng(ss.spawn(stream + 1)[stream])
 
 
@@ -290,7 +290,40 @@ def t9_skew(kind: str, n_tokens: int = 2048) -> Workload:
                     seq_id=np.arange(N, dtype=np.int32))
 
 
-SWEEP_NAMES = tuple(f"f9-{n}" for n in F9_BATCHES) + tuple(f"t9-{k}" for k in T9_SKEWS)
+# Table 6 conditions: how the modalities are arranged inside the sequences.  The paper names three arrangements and gives
+# neither their proportions nor the batch; these are this build's choices: 8 sequences of 256 tokens (its batch-256 point
+# has the same per-token latency), d = 4096, r = 64, 4 modalities over the 160k vocabulary of the multimodal workload.
+T6_KINDS = {"text-heavy": (0.70, 0.10, 0.10, 0.10), "balanced": (0.25, 0.25, 0.25, 0.25), "separated": None}
+
+
+def t6_distribution(kind: str, n_seqs: int = 8, seq_len: int = 256) -> Workload:
+    """Modality arrangement of Table 6: "text-heavy" and "balanced" interleave runs (geometric length, mean 16) whose
+    modality is drawn with the given shares; "separated" gives every sequence one modality (sequence s: s mod 4).
+    Vocabulary-routed, one projection 4096->4096, rank 64, bf16."""
+    wrng, rng = _rng(6, 0), _rng(6, 1 + list(T6_KINDS).index(kind))
+    N, C, d, rank = n_seqs * seq_len, 4, 4096, 64
+    share = T6_KINDS[kind]
+    mod = np.empty(N, dtype=np.int32)
+    for s in range(n_seqs):
+        if share is None:
+            mod[s * seq_len:(s + 1) * seq_len] = s % C
+            continue
+        pos = 0
+        while pos < seq_len:
+            run = int(rng.geometric(1.0 / 16))
+            mod[s * seq_len + pos: s * seq_len + min(seq_len, pos + run)] = int(rng.choice(C, p=share))
+            pos += run
+    lo = C5_BREAKS[:-1][mod].astype(np.int64)
+    hi = C5_BREAKS[1:][mod].astype(np.int64)
+    ids = (lo + (rng.random(N) * (hi - lo)).astype(np.int64)).astype(np.int32)
+    A, B = _adapters(wrng, C, d, d, rank, True)
+    return Workload(name=f"t6-{kind}", N=N, C=C, dtype="bf16", router="vocab", inputs={"x": _normal(rng, (N, d), 1.0, True)},
+                    projections=[Projection("proj", "x", d, d, rank, A, B, _normal(rng, (N, d), 1.0, True))], ids=ids,
+                    breaks=C5_BREAKS.copy(), seq_id=np.repeat(np.arange(n_seqs, dtype=np.int32), seq_len),
+                    notes={"modality": mod})
+
+
+SWEEP_NAMES = tuple(f"f9-{n}" for n in F9_BATCHES) + tuple(f"t9-{k}" for k in T9_SKEWS) + tuple(f"t6-{k}" for k in T6_KINDS)
 
 
 def get(name: str, **kw) -> Workload:
@@ -302,4 +335,6 @@ def get(name: str, **kw) -> Workload:
         return f9_batch(int(name[3:]))
     if name.startswith("t9-"):
         return t9_skew(name[3:], **kw)
+    if name.startswith("t6-"):
+        return t6_distribution(name[3:], **kw)
     return table[name](**kw)

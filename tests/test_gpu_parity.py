@@ -80,9 +80,10 @@ def test_full_size_every_row(name):
     print(name, stats)
 
 
-@pytest.mark.parametrize("name", ["f9-512", "f9-2048", "t9-95", "t9-80"])
+@pytest.mark.parametrize("name", ["f9-512", "f9-2048", "t9-95", "t9-80", "t6-text-heavy", "t6-balanced", "t6-separated"])
 def test_sweep_workloads_full(name):
-    # the batch and skew sweeps of the benchmark (Figure 9 / Table 9 conditions: 4096 -> 4096, rank 64): every row
+    # the batch, skew and modality-arrangement sweeps of the benchmark (Figure 9 / Table 9 / Table 6 conditions:
+    # 4096 -> 4096, rank 64): every row
     run_and_check(W.get(name), batched=True)
 
 
@@ -590,8 +591,13 @@ def test_route_mlp_feeds_group_and_apply():
 
 
 # ------------------------------------------------------------------ top-k weighted routing (Eq. 8, the paper's k = 2)
-@pytest.mark.parametrize("N,C,k,d_in,d_out,rank,mode", [(300, 4, 2, 256, 192, 16, "stream"),
-                                                        (300, 4, 2, 256, 192, 16, "jobs"),
+@pytest.mark.parametrize("N,C,k,d_in,d_out,rank,mode", [(300, 4, 2, 256, 192, 16, "stream"),      # one pass (adapter sets)
+                                                        (4096, 4, 2, 2048, 2048, 16, "default"),   # ... at the prefill shape
+                                                        (700, 4, 4, 256, 320, 16, "default"),      # ... k = 4: stacked rank 64
+                                                        (500, 8, 2, 512, 256, 32, "default"),      # ... rank 32, 64 sets
+                                                        (900, 16, 2, 256, 256, 16, "default"),     # ... 256 sets
+                                                        (6000, 5, 2, 192, 224, 16, "stream"),      # ... perm read from global memory
+                                                        (300, 4, 2, 256, 192, 16, "jobs"),         # k passes from here on
                                                         (300, 4, 2, 256, 192, 16, "twophase"),
                                                         (3300, 4, 2, 512, 256, 16, "tcgen05"),
                                                         (200, 6, 3, 128, 96, 8, "default"),      # CUDA-core kernel (rank 8)
@@ -621,14 +627,16 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode):
     y = dev_tensor(p.y, "bf16")
     M.molora_apply_topk([M.ProjDesc(x, y, dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), 1.0)], idx, wt, C)
     ref = oracle.apply_topk(x_np, p.y, p.A, p.B, idx_ref, w_ref)
-    # y is rounded to bf16 after every pass: besides the usual bound, half a bf16 ulp (2^-9 relative) of each
-    # intermediate result h after passes 1 .. k-1 (which can be much larger than the final value when slots cancel)
-    got, err = to_f64(y), None
-    slack = np.zeros_like(ref)
-    for j in range(1, k):
-        slack += 2.0 ** -9 * np.abs(oracle.apply_topk(x_np, p.y, p.A, p.B, idx_ref[:j], w_ref[:j]))
+    got = to_f64(y)
     err = np.abs(got - ref)
-    bound = 1e-3 + 2e-2 * np.abs(ref) + slack
+    bound = 1e-3 + 2e-2 * np.abs(ref)
+    one_pass = mode in ("stream", "default") and k in (2, 4) and rank * k in (16, 32, 64) and C ** k <= 256
+    if not one_pass:
+        # k passes round y to bf16 after every pass: besides the usual bound, half a bf16 ulp (2^-9 relative) of each
+        # intermediate result h after passes 1 .. k-1 (which can be much larger than the final value when slots cancel).
+        # The single pass over adapter sets rounds once and must meet the stated bound as it is.
+        for j in range(1, k):
+            bound = bound + 2.0 ** -9 * np.abs(oracle.apply_topk(x_np, p.y, p.A, p.B, idx_ref[:j], w_ref[:j]))
     assert np.all(err[keep] <= bound[keep]), f"top-{k} weighted apply: worst ratio {(err / bound)[keep].max():.3f}"
 
 
