@@ -125,7 +125,7 @@ class Clocks(threading.Thread):
 
 
 # ----------------------------------------------------------------------------- our arm
-def build_sets(W, torch, name, n_sets, rank):
+def build_sets(W, torch, name, n_sets, rank, kw=None):
     """Device-resident buffer sets of the workload: shared weights, n_sets activation batches."""
     def dev(a, dtype):
         if a.dtype == np.int32:
@@ -139,11 +139,11 @@ def build_sets(W, torch, name, n_sets, rank):
     sets, w0 = [], None
     for b in range(n_sets):
         if name == "c2":
-            w = W.get("c2", batch=batches[b])
+            w = W.get("c2", batch=batches[b], **(kw or {}))
         elif name == "c3":
-            w = W.get("c3", layer=batches[b])
+            w = W.get("c3", layer=batches[b], **(kw or {}))
         else:
-            w = W.get(name) if b == 0 else None
+            w = W.get(name, **(kw or {})) if b == 0 else None
         if w is None:   # large configs: clone batch 0 into distinct buffers (same values, distinct addresses)
             s0 = sets[0]
             sets.append({"x": {k: v.clone() for k, v in s0["x"].items()}, "y": [t.clone() for t in s0["y"]],
@@ -234,14 +234,16 @@ def measure(name, args, env, headline):
     rank, world, local = env["rank"], env["world"], env["local"]
     from paper_2603_15965_b200.binding import molora_apply_batched_workspace_bytes, pack_proj_descs
 
-    probe = W.get(name) if name != "c2" else W.get("c2", batch=0)
+    # --tokens shrinks c2 / c3 / c4 (for profiler captures, which must stay small); never used for a reported number
+    kw = {"n_tokens": args.tokens} if args.tokens and name in ("c2", "c3", "c4") else {}
+    probe = W.get(name, **kw) if name != "c2" else W.get("c2", batch=0, **kw)
     step_bytes, step_flops = workload_info(probe)
     esz = 2 if probe.dtype == "bf16" else 1
     per_set = sum(v.nbytes // esz for v in probe.inputs.values()) + sum(p.y.nbytes // esz for p in probe.projections)
     n_sets = max(2, int(np.ceil(2.5 * L2_BYTES / per_set)))          # rotation working set >= 2.5 x L2
     n_sets = min(n_sets, args.max_sets)
     del probe
-    w, sets, shared = build_sets(W, torch, name, n_sets, rank)
+    w, sets, shared = build_sets(W, torch, name, n_sets, rank, kw)
     N, C = w.N, w.C
     stream = torch.cuda.Stream()      # every call of the timed region is enqueued (or captured) on this stream
 
@@ -384,7 +386,7 @@ def measure(name, args, env, headline):
     achieved = step_bytes / (apply_ms * 1e-3) / 1e9
     traffic = NCU_TRAFFIC.get(name)
     rec.update({
-        "workload": workload_label(name, w),
+        "workload": workload_label(name, w) + (f" [REDUCED to {w.N} tokens for a profiler capture]" if kw else ""),
         "tokens_per_step_per_gpu": N, "buffer_sets": n_sets,
         "l2": f"rotation over {n_sets} buffer sets ({n_sets * per_set / 1e6:.0f} MB > 126 MB L2)",
         "value": shard.aggregate_tokens_per_s(N, world, ms_per_step), "ms_per_step": ms_per_step,
@@ -698,6 +700,8 @@ def main():
     ap.add_argument("--min-leg-s", type=float, default=0.3, help="every timed leg lasts at least this long")
     ap.add_argument("--max-sets", type=int, default=32)
     ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="profiler captures only: run c2 / c3 / c4 with this many tokens instead of the configuration's")
     ap.add_argument("--profile", action="store_true",
                     help="timed steps of one workload only: no sub-records, no host-buffer e2e leg, no oracle leg (for ncu captures)")
     args = ap.parse_args()

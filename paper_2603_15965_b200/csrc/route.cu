@@ -1,6 +1,8 @@
 // Routers: vocabulary-range routing (Definition 3.1) and the linear gate with top-1 argmax (Eq. 8, k = 1).
 #include <stdlib.h>
 
+#include <algorithm>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 #include "warp_reduce.cuh"
