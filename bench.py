@@ -186,7 +186,7 @@ def marshal_step(lib, w, s, shared, stream_handle):
         route = partial(lib.molora_route_gate, vp(x.data_ptr()), 1 if w.dtype == "bf16" else 0, i64(N), i32(x.shape[1]),
                         i64(x.stride(0)), vp(shared["G"].data_ptr()), None, i32(C), vp(s["r"].data_ptr()), None,
                         vp(gws.data_ptr()) if gws is not None else None,
-                        ctypes.c_size_t(gws.numel() if gws is not None else 0), st)
+                        ctypes.c_size_t(gws.numel() if gws is not None else 0), None, st)
         r = s["r"]
     elif w.router == "vocab":
         route = partial(lib.molora_route_vocab, vp(s["ids"].data_ptr()), i64(N), vp(shared["breaks"].data_ptr()),

@@ -75,7 +75,7 @@ const char *molora_status_string(molora_status_t status);
  *   kernel; value 0 restores the default.  Names: "umma_min_tokens" (tcgen05 apply from that many tokens),
  *   "small_path" (kernel below it: 1 streaming, 2 two-launch, 3 job-list decode kernel), "stream_tile" (16 | 32),
  *   "umma_split", "umma_tile_rows", "group_split" (cluster sizes / tile height), "chained_launch_off" (1: plain stream
- *   order).  The start values are read once from the environment variables MOLORA_<NAME>.  Unknown name:
+ *   order), "jobs_launch" (job-list kernel: 0 cooperative, 1 plain, 2 programmatic launch).  The start values are read once from the environment variables MOLORA_<NAME>.  Unknown name:
  *   MOLORA_ERR_INVALID_ARG.  Not meant to be changed while calls are in flight on other threads. */
 uint64_t molora_launch_count(void);
 molora_status_t molora_debug_set(const char *name, int64_t value);
@@ -114,11 +114,13 @@ molora_status_t molora_route_composite(const int32_t *ids, const int32_t *adapte
  *               (NULL when that is 0).  For bf16 x and C > 4 the kernel runs on the tensor cores (tcgen05 when N >= 1024
  *               and d is a multiple of 64, mma.sync otherwise) and keeps there a three-term bf16 split of G
  *               (hi + mid + lo = 24 mantissa bits), rebuilt on every call.
+ * dev_status  device status word or NULL.  Only the tcgen05 kernel waits on the device (bounded): if a wait runs out,
+ *             MOLORA_DEV_TIMEOUT is OR-ed in and the tokens of that 128-token tile get r_out = -1 (unrouted).
  * Products are exact in fp32 for bf16 x; accumulation is fp32 in a fixed, token-independent order. */
 size_t molora_route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
 molora_status_t molora_route_gate(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float *G,
                                   const float *bias, int32_t C, int32_t *r_out, float *logits_out, void *ws,
-                                  size_t ws_bytes, void *stream);
+                                  size_t ws_bytes, uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Router 3: the paper's learned router (Eq. 9), a 2-layer MLP with GELU, followed by top-1 selection:
@@ -132,11 +134,13 @@ molora_status_t molora_route_gate(const void *x, molora_dtype_t xdt, int64_t N, 
  *               when that is 0): for bf16 x and d a multiple of 64 the first layer runs on the tensor cores with a
  *               three-term bf16 split of W1 kept there (rebuilt on every call); MOLORA_ERR_WORKSPACE if it is
  *               needed (at least 128 tokens) and missing.
+ * dev_status  device status word or NULL; as for molora_route_gate (the tensor-core kernel's waits are bounded:
+ *             MOLORA_DEV_TIMEOUT, and r_out = -1 for the tokens of the tile whose wait ran out).
  * Products of the first layer are exact in fp32 for bf16 x; accumulation, GELU and the second layer are fp32. */
 size_t molora_route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H, int32_t C);
 molora_status_t molora_route_mlp(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float *W1,
                                  const float *b1, int32_t H, const float *W2, const float *b2, int32_t C, int32_t *r_out,
-                                 float *logits_out, void *ws, size_t ws_bytes, void *stream);
+                                 float *logits_out, void *ws, size_t ws_bytes, uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * The same gate for callers that cannot provide a workspace.  (The paper has no counterpart: this entry point
@@ -145,7 +149,8 @@ molora_status_t molora_route_mlp(const void *x, molora_dtype_t xdt, int64_t N, i
  * graph, plug-ins that are handed tensors but no allocator, allocation-free real-time loops -- and so cannot
  * supply molora_route_gate's `ws`.  This variant keeps the scratch inside the library instead: a fixed 2 MiB
  * device array that every GPU loading the library holds until the process exits.
- *   - Same arguments, results and errors as molora_route_gate, without ws / ws_bytes.
+ *   - Same arguments, results and errors as molora_route_gate, without ws / ws_bytes / dev_status (a wait that runs
+ *     out still leaves r_out = -1 for its tile).
  *   - Limit: molora_route_gate_workspace_bytes(xdt, d, C) must not exceed 2 MiB (2 097 152 bytes); e.g.
  *     bf16 x with C <= 16 up to d = 19 328, with C <= 32 up to d = 8 704.  Larger gates are refused with
  *     MOLORA_ERR_WORKSPACE and nothing is enqueued.  Calls that need no scratch (fp32 x, or C <= 4) always fit.

@@ -92,10 +92,10 @@ def load_library():
     lib.molora_apply_topk.argtypes = [vp, i32, ctypes.c_int, i64, i32, i32, vp, vp, vp, sz, vp, vp]
     lib.molora_route_mlp_workspace_bytes.restype = sz
     lib.molora_route_mlp_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i32]
-    lib.molora_route_mlp.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp]
+    lib.molora_route_mlp.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp, vp]
     lib.molora_route_gate_workspace_bytes.restype = sz
     lib.molora_route_gate_workspace_bytes.argtypes = [ctypes.c_int, i32, i32]
-    lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp]
+    lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp, vp]
     lib.molora_route_gate_noalloc.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp]
     lib.molora_route_gate_noalloc.restype = ctypes.c_int
     lib.molora_selftest_bounded_wait.argtypes = [vp, i64, vp, vp]
@@ -192,7 +192,7 @@ def molora_launch_count() -> int:
 
 
 TUNING_NAMES = ("umma_min_tokens", "small_path", "stream_tile", "umma_split", "umma_tile_rows", "group_split",
-                "chained_launch_off")
+                "chained_launch_off", "jobs_launch")
 
 
 def molora_debug_set(name: str, value: int) -> None:
@@ -241,7 +241,7 @@ def molora_route_mlp_workspace_bytes(xdt: int, d: int, H: int, C: int) -> int:
 def molora_route_mlp(x: torch.Tensor, W1: torch.Tensor, b1: Optional[torch.Tensor], W2: torch.Tensor,
                      b2: Optional[torch.Tensor], r_out: Optional[torch.Tensor] = None,
                      logits_out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
-                     stream=None) -> torch.Tensor:
+                     dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """r_out[i] = argmax_c (W2 GELU(W1 x_i + b1) + b2)[c] (Eq. 9, top-1); W1 [d, H], W2 [H, C] fp32."""
     lib = load_library()
     N, d, ldx = _matrix(x, "x")
@@ -258,7 +258,7 @@ def molora_route_mlp(x: torch.Tensor, W1: torch.Tensor, b1: Optional[torch.Tenso
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_route_mlp", lib.molora_route_mlp(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(W1), _ptr(b1), H, _ptr(W2),
                                                     _ptr(b2), C, _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
-                                                    _ptr(ws), ws_bytes, _stream(stream)))
+                                                    _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
     return r_out
 
 
@@ -268,7 +268,8 @@ def molora_route_gate_workspace_bytes(xdt: int, d: int, C: int) -> int:
 
 def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Tensor] = None,
                       r_out: Optional[torch.Tensor] = None, logits_out: Optional[torch.Tensor] = None,
-                      ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+                      ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
     """r_out[i] = argmax_c sum_k x[i,k] G[k,c] (+ bias[c]) (Eq. 8, k = 1); lowest index on ties."""
     lib = load_library()
     N, d, ldx = _matrix(x, "x")
@@ -288,7 +289,7 @@ def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Ten
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check("molora_route_gate", lib.molora_route_gate(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(G), _ptr(bias), C,
                                                       _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out), _ptr(ws),
-                                                      ws_bytes, _stream(stream)))
+                                                      ws_bytes, _ptr(dev_status), _stream(stream)))
     return r_out
 
 

@@ -175,7 +175,7 @@ size_t molora_route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t 
 
 molora_status_t molora_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
                                   const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                  size_t ws_bytes, void* stream)
+                                  size_t ws_bytes, uint32_t* dev_status, void* stream)
 {
     if (N < 0 || N >= INT32_MAX || d <= 0 || C < 1) return MOLORA_ERR_INVALID_ARG;
     if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
@@ -184,7 +184,7 @@ molora_status_t molora_route_gate(const void* x, molora_dtype_t xdt, int64_t N, 
     if (N > 0 && (x == nullptr || r_out == nullptr || !aligned16(x))) return MOLORA_ERR_INVALID_ARG;
     const size_t need = route_gate_workspace_bytes(xdt, d, C);
     if (need > 0 && (ws == nullptr || ws_bytes < need || !aligned16(ws))) return MOLORA_ERR_WORKSPACE;
-    return launch_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, ws, static_cast<cudaStream_t>(stream));
+    return launch_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 size_t molora_route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H, int32_t C)
@@ -195,7 +195,7 @@ size_t molora_route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H
 
 molora_status_t molora_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
                                  const float* b1, int32_t H, const float* W2, const float* b2, int32_t C, int32_t* r_out,
-                                 float* logits_out, void* ws, size_t ws_bytes, void* stream)
+                                 float* logits_out, void* ws, size_t ws_bytes, uint32_t* dev_status, void* stream)
 {
     if (N < 0 || N >= INT32_MAX || d <= 0 || H < 1 || C < 1) return MOLORA_ERR_INVALID_ARG;
     if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
@@ -203,7 +203,7 @@ molora_status_t molora_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, i
     if (ldx < d) return MOLORA_ERR_INVALID_ARG;
     if (W1 == nullptr || W2 == nullptr || (N > 0 && (x == nullptr || r_out == nullptr))) return MOLORA_ERR_INVALID_ARG;
     if (N > 0 && !aligned16(x)) return MOLORA_ERR_INVALID_ARG;
-    return launch_route_mlp(x, xdt, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, ws_bytes,
+    return launch_route_mlp(x, xdt, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, ws_bytes, dev_status,
                             static_cast<cudaStream_t>(stream));
 }
 
@@ -693,7 +693,7 @@ molora_status_t molora_forward_host(molora_router_t router, const int32_t* route
     } else if (router == MOLORA_ROUTE_GATE) {
         const molora_proj_desc_t& gp = dev[gate_proj];
         if ((gp.d_in % 8) != 0) return MOLORA_ERR_UNSUPPORTED;
-        st = launch_route_gate(gp.x, dt, N, gp.d_in, gp.ldx, G_dev, bias_dev, C, r, nullptr, base + pl.gate_ws, s);
+        st = launch_route_gate(gp.x, dt, N, gp.d_in, gp.ldx, G_dev, bias_dev, C, r, nullptr, base + pl.gate_ws, dev_status, s);
     }
     if (st != MOLORA_OK) return st;
     // 3. group, 4. apply

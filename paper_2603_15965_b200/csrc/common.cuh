@@ -226,11 +226,11 @@ bool gate_umma_eligible(int64_t N, int32_t d, int32_t C);
 size_t route_gate_umma_workspace_bytes(int32_t d, int32_t C);
 molora_status_t launch_route_gate_umma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
                                        const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                       cudaStream_t s);
+                                       uint32_t* dev_status, cudaStream_t s);
 size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
 molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
                                   const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                  cudaStream_t s);
+                                  uint32_t* dev_status, cudaStream_t s);
 // Tensor-core (mma.sync) gate for bf16 activations; the CUDA-core kernel above serves fp32 activations.
 // Needs route_gate_mma_workspace_bytes(d, C) bytes of scratch for the split gate weights.
 size_t route_gate_mma_workspace_bytes(int32_t d, int32_t C);
@@ -242,7 +242,7 @@ molora_status_t launch_route_gate_mma(const void* x, int64_t N, int32_t d, int64
 size_t route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H);
 molora_status_t launch_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
                                  const float* b1, int32_t H, const float* W2, const float* b2, int32_t C, int32_t* r_out,
-                                 float* logits_out, void* ws, size_t ws_bytes, cudaStream_t s);
+                                 float* logits_out, void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
 // Top-k selection and softmax over router logits (Eq. 8); idx / w slot-major [k][N].
 molora_status_t launch_topk_softmax(const float* logits, int64_t N, int32_t C, int32_t k, int32_t* idx_out, float* w_out,
                                     cudaStream_t s);

@@ -580,11 +580,11 @@ size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
 
 molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
                                   const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                  cudaStream_t s)
+                                  uint32_t* dev_status, cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
-    if (xdt == MOLORA_BF16 && gate_umma_eligible(N, d, C))
-        return launch_route_gate_umma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
+    if (xdt == MOLORA_BF16 && gate_umma_eligible(N, d, C))       // the only gate kernel with device-side waits
+        return launch_route_gate_umma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s);
     if (xdt == MOLORA_BF16 && C > 4) return launch_route_gate_mma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
     if (xdt == MOLORA_BF16) return gate_dispatch<__nv_bfloat16>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
     return gate_dispatch<float>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);

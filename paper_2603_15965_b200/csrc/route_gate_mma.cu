@@ -303,5 +303,5 @@ extern "C" molora_status_t molora_route_gate_noalloc(const void* x, molora_dtype
         if (st != MOLORA_OK) return st;
     }
     return molora_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, scratch, need > 0 ? kNoAllocScratchBytes : 0,
-                             stream);
+                             nullptr, stream);
 }

@@ -156,6 +156,7 @@ __global__ void __launch_bounds__(kGuThreads, 1) route_gate_umma_kernel(const __
     if (S > 1) cluster_sync_all();
     if (epi && crank == 0) {
         const int64_t i = tok0 + row;
+        if (i < prm.N && *abort_flag) prm.r_out[i] = -1;                // a wait ran out: the tile's tokens stay unrouted
         if (i < prm.N && !*abort_flag) {
             for (uint32_t p2 = 1; p2 < S; ++p2)                         // rank order
 #pragma unroll
@@ -182,7 +183,8 @@ __global__ void __launch_bounds__(kGuThreads, 1) route_gate_umma_kernel(const __
 
 template <int CP>
 static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t ldx, const float* G, const float* bias,
-                                        int C, int32_t* r_out, float* logits_out, void* ws, cudaStream_t s)
+                                        int C, int32_t* r_out, float* logits_out, void* ws, uint32_t* dev_status,
+                                        cudaStream_t s)
 {
     constexpr int NP = 3 * CP;
     constexpr int STAGES = CP == 16 ? kGuStages : kGuStages - 1;
@@ -207,7 +209,7 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
     prm.bias = bias;
     prm.r_out = r_out;
     prm.logits_out = logits_out;
-    prm.dev_status = nullptr;
+    prm.dev_status = dev_status;
     prm.N = N;
     prm.d = d;
     prm.C = C;
@@ -245,11 +247,11 @@ size_t route_gate_umma_workspace_bytes(int32_t d, int32_t C)
 
 molora_status_t launch_route_gate_umma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
                                        const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                       cudaStream_t s)
+                                       uint32_t* dev_status, cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
-    if (C <= 16) return gate_umma_launch<16>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
-    return gate_umma_launch<32>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
+    if (C <= 16) return gate_umma_launch<16>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s);
+    return gate_umma_launch<32>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s);
 }
 
 }  // namespace molora

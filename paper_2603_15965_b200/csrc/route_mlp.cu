@@ -177,6 +177,7 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
             }
         }
         const int64_t i = tok0 + row;
+        if (i < prm.N && *abort_flag) prm.r_out[i] = -1;                // a wait ran out: the tile's tokens stay unrouted
         if (i < prm.N && !*abort_flag) {
             float best = 0.f;
             int arg = 0;
@@ -263,7 +264,7 @@ size_t route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H)
 template <int HP>
 static molora_status_t mlp_umma_launch(const void* x, int64_t N, int d, int64_t ldx, const float* W1, const float* b1, int H,
                                        const float* W2, const float* b2, int C, int32_t* r_out, float* logits_out, void* ws,
-                                       cudaStream_t s)
+                                       uint32_t* dev_status, cudaStream_t s)
 {
     constexpr int NP = 3 * HP;
     constexpr int STAGES = HP == 64 ? 5 : 3;
@@ -285,7 +286,7 @@ static molora_status_t mlp_umma_launch(const void* x, int64_t N, int d, int64_t 
     prm.b2 = b2;
     prm.r_out = r_out;
     prm.logits_out = logits_out;
-    prm.dev_status = nullptr;
+    prm.dev_status = dev_status;
     prm.N = N;
     prm.d = d;
     prm.H = H;
@@ -314,13 +315,13 @@ static molora_status_t mlp_simple_launch(const void* x, int64_t N, int d, int64_
 
 molora_status_t launch_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
                                  const float* b1, int32_t H, const float* W2, const float* b2, int32_t C, int32_t* r_out,
-                                 float* logits_out, void* ws, size_t ws_bytes, cudaStream_t s)
+                                 float* logits_out, void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
     if (mlp_umma_eligible(xdt, N, d, H)) {
         if (ws == nullptr || ws_bytes < route_mlp_workspace_bytes(xdt, d, H) || !aligned16(ws)) return MOLORA_ERR_WORKSPACE;
-        return H <= 64 ? mlp_umma_launch<64>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, s)
-                       : mlp_umma_launch<128>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, s);
+        return H <= 64 ? mlp_umma_launch<64>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, dev_status, s)
+                       : mlp_umma_launch<128>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, dev_status, s);
     }
     return xdt == MOLORA_BF16 ? mlp_simple_launch<__nv_bfloat16>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, s)
                               : mlp_simple_launch<float>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, s);

@@ -36,19 +36,19 @@ def test_invalid_arguments_are_refused_before_any_launch():
     assert lib.molora_route_composite(fake, fake, 4, fake, 4, 65, fake, None, None) == 2
     assert lib.molora_route_composite(fake, None, 4, fake, 4, 64, fake, None, None) == 1
     # MLP router: hidden width and adapter count limits, tensor-core path without its workspace
-    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, fake, None, 129, fake, None, 4, fake, None, None, 0, None) == 2
-    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, fake, None, 64, fake, None, 33, fake, None, None, 0, None) == 2
-    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, None, None, 64, fake, None, 4, fake, None, None, 0, None) == 1
+    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, fake, None, 129, fake, None, 4, fake, None, None, 0, None, None) == 2
+    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, fake, None, 64, fake, None, 33, fake, None, None, 0, None, None) == 2
+    assert lib.molora_route_mlp(fake, M.BF16, 4, 64, 64, None, None, 64, fake, None, 4, fake, None, None, 0, None, None) == 1
     assert M.molora_route_mlp_workspace_bytes(M.BF16, 2560, 128, 4) == 2560 * 3 * 128 * 2
     assert M.molora_route_mlp_workspace_bytes(M.F32, 2560, 128, 4) == 0
-    assert lib.molora_route_mlp(fake, M.BF16, 128, 64, 64, fake, None, 64, fake, None, 4, fake, None, None, 0, None) == 3
+    assert lib.molora_route_mlp(fake, M.BF16, 128, 64, 64, fake, None, 64, fake, None, 4, fake, None, None, 0, None, None) == 3
     # gate: d not a multiple of 8, C too large, pitch too small
-    assert lib.molora_route_gate(fake, M.BF16, 4, 12, 16, fake, None, 4, fake, None, None, 0, None) == 2
-    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 33, fake, None, None, 0, None) == 2
-    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 8, fake, None, 4, fake, None, None, 0, None) == 1
+    assert lib.molora_route_gate(fake, M.BF16, 4, 12, 16, fake, None, 4, fake, None, None, 0, None, None) == 2
+    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 33, fake, None, None, 0, None, None) == 2
+    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 8, fake, None, 4, fake, None, None, 0, None, None) == 1
     # tensor-core gate (bf16, C > 4) without its workspace
     assert M.molora_route_gate_workspace_bytes(M.BF16, 4096, 16) > 0 and M.molora_route_gate_workspace_bytes(M.BF16, 2048, 4) == 0
-    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 16, fake, None, None, 0, None) == 3
+    assert lib.molora_route_gate(fake, M.BF16, 4, 16, 16, fake, None, 16, fake, None, None, 0, None, None) == 3
     # group: C out of range, null outputs
     assert lib.molora_group(fake, 4, 0, fake, fake, fake, None, 0, None, None) == 1
     assert lib.molora_group(fake, 4, 300, fake, fake, fake, None, 0, None, None) == 2

@@ -151,7 +151,10 @@ def test_route_gate_logits_and_argmax(dtype, N, d, C):
     bias = rng.standard_normal(C).astype(np.float32) * 0.1
     r_ref, z_ref, margin = oracle.route_gate(x, G, bias)
     logits = torch.empty(N, C, dtype=torch.float32, device="cuda")
-    r = M.molora_route_gate(dev_tensor(x, dtype), dev_tensor(G, "f32"), dev_tensor(bias, "f32"), logits_out=logits)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    r = M.molora_route_gate(dev_tensor(x, dtype), dev_tensor(G, "f32"), dev_tensor(bias, "f32"), logits_out=logits,
+                            dev_status=status)
+    assert int(status.item()) == 0                            # no device-side wait ran out
     assert_close(to_f64(logits), z_ref, 1e-4, 1e-4, what="gate logits")
     keep = margin >= 1e-3
     assert np.array_equal(r.cpu().numpy()[keep], r_ref[keep])
@@ -461,7 +464,10 @@ def test_route_gate_tensor_core_paths(N, d, C):
     bias = (rng.standard_normal(C) * 0.1).astype(np.float32)
     r_ref, z_ref, margin = oracle.route_gate(x, G, bias)
     logits = torch.empty(N, C, dtype=torch.float32, device="cuda")
-    r = M.molora_route_gate(dev_tensor(x, "bf16"), dev_tensor(G, "f32"), dev_tensor(bias, "f32"), logits_out=logits)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    r = M.molora_route_gate(dev_tensor(x, "bf16"), dev_tensor(G, "f32"), dev_tensor(bias, "f32"), logits_out=logits,
+                            dev_status=status)
+    assert int(status.item()) == 0
     assert_close(to_f64(logits), z_ref, 1e-4, 1e-4, what="gate logits")
     keep = margin >= 1e-3
     assert np.array_equal(r.cpu().numpy()[keep], r_ref[keep])
@@ -562,8 +568,10 @@ def test_route_mlp_logits_and_argmax(dtype, N, d, H, C):
     b2 = (rng.standard_normal(C) * 0.1).astype(np.float32)
     r_ref, z_ref, margin = oracle.route_mlp(x, W1, b1, W2, b2)
     logits = torch.empty(N, C, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
     r = M.molora_route_mlp(dev_tensor(x, dtype), dev_tensor(W1, "f32"), dev_tensor(b1, "f32"), dev_tensor(W2, "f32"),
-                           dev_tensor(b2, "f32"), logits_out=logits)
+                           dev_tensor(b2, "f32"), logits_out=logits, dev_status=status)
+    assert int(status.item()) == 0                            # no device-side wait ran out
     assert_close(to_f64(logits), z_ref, 1e-4, 1e-4, what="MLP router logits")
     keep = margin >= 1e-3
     assert (~keep).sum() <= max(4, N // 100)
