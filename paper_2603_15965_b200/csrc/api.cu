@@ -359,12 +359,14 @@ molora_status_t molora_apply_batched(const molora_proj_desc_t* projs, int32_t P,
 
 // How molora_group_apply_batched runs: 1 = one launch of the streaming kernel (every projection on it, one rank, at
 // most 4096 tokens), 3 = one launch of the job-list kernel (every projection on it, one rank), 2 = the two-launch kernels
-// with the grouping inside (one rank, at most 1024 tokens), 0 = the grouping launch followed by the apply launches.
+// with the grouping inside (one rank, at most 1024 tokens), 4 = one launch of the tcgen05 kernel with the grouping inside
+// (every projection on it, one rank, at most 4096 tokens, few enough adapters that it takes every segment), 0 = the
+// grouping launch followed by the apply launches.
 static int group_apply_mode(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C)
 {
     if (dt != MOLORA_BF16 || N < 1) return 0;
     double bytes = 0.0;
-    bool same = true, stream = true, twophase = true, jobs = true;
+    bool same = true, stream = true, twophase = true, jobs = true, umma = true;
     for (int i = 0; i < P; ++i) {
         same = same && projs[i].rank == projs[0].rank && decode_eligible(projs[i], dt);
         if (!same) return 0;
@@ -373,9 +375,10 @@ static int group_apply_mode(const molora_proj_desc_t* projs, int32_t P, molora_d
         jobs = jobs && jb;
         stream = stream && !jb && st;
         twophase = twophase && !jb && !st;
+        umma = umma && umma_eligible(projs[i], dt);
         if (umma_eligible(projs[i], dt)) bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
     }
-    if (use_umma(projs[0].rank, N, bytes)) return 0;
+    if (use_umma(projs[0].rank, N, bytes)) return umma && group_apply_umma_eligible(N, C) ? 4 : 0;
     if (jobs) return 3;
     if (stream && group_apply_stream_eligible(N)) return 1;
     if (twophase && group_apply_decode_eligible(N)) return 2;
@@ -386,7 +389,7 @@ int32_t molora_group_apply_is_one_launch(const molora_proj_desc_t* projs, int32_
 {
     if (projs == nullptr || P < 1 || P > MOLORA_MAX_PROJECTIONS || N < 1 || C < 1) return 0;
     const int mode = group_apply_mode(projs, P, dt, N, C);
-    return mode == 1 || mode == 3 ? 1 : 0;
+    return mode == 1 || mode == 3 || mode == 4 ? 1 : 0;
 }
 
 int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C)
@@ -416,6 +419,8 @@ molora_status_t molora_group_apply_batched(const int32_t* r, int64_t N, int32_t 
     const int mode = group_apply_mode(projs, P, dt, N, C);
     if (mode == 1)
         return launch_group_apply_stream(r, projs, P, N, C, counts, offsets, perm, dev_status, static_cast<cudaStream_t>(stream));
+    if (mode == 4)
+        return launch_apply_umma(projs, P, N, C, offsets, perm, dev_status, 1, static_cast<cudaStream_t>(stream), r, counts);
     if (mode == 3) {
         size_t part = 0;
         for (int i = 0; i < P; ++i) part += jobs_partial_bytes(N, C, projs[i].d_in, projs[i].rank);

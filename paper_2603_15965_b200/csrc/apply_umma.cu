@@ -38,6 +38,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "group_inline.cuh"
 #include "pipeline.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
@@ -59,6 +60,7 @@ constexpr int kTileBytes = kTileM * 128;    // 16 KB: X or Y chunk
 constexpr int kDBufs = 4;                   // expand accumulators in flight (64 TMEM columns each)
 constexpr int kTmemCols = 512;
 constexpr int kMaxSplit = 4;                // largest cluster a tile is split over
+constexpr int kMaxWideSplit = 8;            // ... by the rank-64 variant for calls with few tiles (portable cluster limit)
 
 struct UmmaProj {
     CUtensorMap tm_a, tm_b;
@@ -77,41 +79,102 @@ struct UmmaParams {
     uint32_t* dev_status;
     int32_t P, C, min_rows;
     int32_t tile_rows;    // positions per tile: 128, or fewer (the MMA tile stays 128 lanes) to spread a small call over more SMs
+    // Grouping inside the kernel (r != NULL; at most kUmmaGroupMaxN tokens): every CTA runs Section 3.3 steps 1-3 on the
+    // routing decisions in its idle ring stages instead of loading offsets / perm, and the CTAs of projection 0 write
+    // counts, offsets and perm out -- the grouping launch in front of a mid-sized call costs as much as a third of it.
+    const int32_t* r;
+    int32_t N;
+    int32_t* counts_out;
+    int32_t* offsets_out;
+    int32_t* perm_out;
 };
+constexpr int kUmmaGroupMaxN = 4096;
 
 
-template <int R>
+// WIDE (rank 64 only): one ring stage fewer, which makes room for the partial rows of up to seven peers, so that a tile
+// can be split over a cluster of up to 8 CTAs -- for calls with so few tiles that the chain of chunks per CTA, not the
+// bytes, sets the time.
+template <int R, bool WIDE = false>
 struct UmmaCfg {
+    static_assert(!WIDE || R == 64, "the wide split exists for rank 64");
     static constexpr int kWBytes = 64 * R * 2;                       // A chunk [64, R] or B chunk [R, 64]
     static constexpr int kStageBytes = kTileBytes + kWBytes;
-    static constexpr int kStages = R == 64 ? 7 : 8;
+    static constexpr int kStages = R == 64 ? (WIDE ? 6 : 7) : 8;
     static constexpr int kTRowBytes = R * 2;                          // one row of T_hi / T_lo
     static constexpr int kTBytes = kTileM * kTRowBytes;
     static constexpr int kSwzBits = R == 64 ? 3 : R == 32 ? 2 : 1;    // swizzle width of R*2-byte rows
     static constexpr uint32_t kWLayout = swizzle_layout_type(static_cast<Swizzle>(kSwzBits));
     // partial T rows received from the cluster peers: (S - 1) * ceil(128 / S) rows of R fp32: 64, 86, 96 rows for
-    // S = 2, 3, 4.  Rank 64 stops at S = 3 (shared memory).
+    // S = 2, 3, 4 and at most 114 (S = 7) up to S = 8.  Rank 64 stops at S = 3 (shared memory) unless WIDE.
     // Ranks 16 and 32 have room for the whole partial of every peer ((S - 1) * 128 rows): one push, every CTA sums
     // for itself.
-    static constexpr int kMaxSplitR = R == 64 ? 3 : kMaxSplit;
+    static constexpr int kMaxSplitR = R == 64 ? (WIDE ? kMaxWideSplit : 3) : kMaxSplit;
     static constexpr bool kOnePush = R != 64;
-    static constexpr int kRecvBytes = kOnePush ? (kMaxSplit - 1) * kTileM * R * 4 : 86 * R * 4;
+    static constexpr int kRecvBytes = kOnePush ? (kMaxSplit - 1) * kTileM * R * 4 : (WIDE ? 114 : 86) * R * 4;
     static constexpr int kCtrlBytes = 768;
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + 2 * kTBytes + kRecvBytes + kCtrlBytes;
 };
 
 struct Ctrl {                         // lives in shared memory after the tiles
-    uint64_t full[8], empty[8], t_full, t_ready, d_full[kDBufs], d_empty[kDBufs], part_full, part_free;
+    uint64_t full[8], empty[8], t_full, t_ready, d_full[kDBufs], d_empty[kDBufs], part_full, part_free, peers_done;
     uint32_t tmem_base;
     int abort_flag;
     alignas(16) int32_t rows[kTileM];
 };
 static_assert(sizeof(Ctrl) <= 768, "control block must fit its slot");
 
-template <int R>
+// Sum of the partial rows of T over the CTAs of a cluster, in rank order (the same bits whoever computes them), in place
+// in tv (this CTA's partial, NWORDS fp32 words of one row).  The peers' partials lie in shared memory as [slot][R / 4][rows]
+// float4 pieces (slot = sender's rank, skipping this CTA); `mine` points at this row's piece 0 of slot 0.  Four
+// independent 16-byte loads per sender keep the loop from running at one shared-memory latency per piece.
+template <int NWORDS>
+__device__ __forceinline__ void sum_partials(uint32_t (&tv)[NWORDS], const float4* mine, int piece_stride, int slot_stride, uint32_t S,
+                                             uint32_t crank)
+{
+    constexpr int R = NWORDS;
+    constexpr int kBatch = R / 4 < 4 ? R / 4 : 4;
+#pragma unroll
+    for (int h = 0; h < R / 4 / kBatch; ++h) {
+        float4 acc[kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint32_t q2 = 0; q2 < S; ++q2) {
+            float4 v[kBatch];
+            if (q2 == crank) {
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const int c4 = h * kBatch + j;
+                    v[j] = make_float4(__uint_as_float(tv[4 * c4]), __uint_as_float(tv[4 * c4 + 1]), __uint_as_float(tv[4 * c4 + 2]),
+                                       __uint_as_float(tv[4 * c4 + 3]));
+                }
+            } else {
+                const float4* src = mine + (size_t)(q2 < crank ? q2 : q2 - 1) * slot_stride + (size_t)(h * kBatch) * piece_stride;
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) v[j] = src[(size_t)j * piece_stride];
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                acc[j].x += v[j].x;
+                acc[j].y += v[j].y;
+                acc[j].z += v[j].z;
+                acc[j].w += v[j].w;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const int c4 = h * kBatch + j;
+            tv[4 * c4] = __float_as_uint(acc[j].x);
+            tv[4 * c4 + 1] = __float_as_uint(acc[j].y);
+            tv[4 * c4 + 2] = __float_as_uint(acc[j].z);
+            tv[4 * c4 + 3] = __float_as_uint(acc[j].w);
+        }
+    }
+}
+
+template <int R, bool WIDE>
 __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __grid_constant__ UmmaParams prm)
 {
-    using Cfg = UmmaCfg<R>;
+    using Cfg = UmmaCfg<R, WIDE>;
     extern __shared__ uint8_t smem_raw[];
     const UmmaProj& pj = prm.p[blockIdx.y];
     if (pj.rank != R) return;
@@ -132,11 +195,19 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     // The segment table is requested first; barriers and TMEM are set up while it is on its way.
     grid_dependency_sync();            // offsets and perm come from the grouping kernel; y from the base projection
     __shared__ int32_t offs_s[MOLORA_MAX_ADAPTERS + 1];
+    const bool grouping = prm.r != nullptr;
+    // grouping: perm, a scratch table and 256 temporary words live in the ring stages, which are idle until the tile is known
+    int32_t* perm_s = reinterpret_cast<int32_t*>(smem_raw + (base - raw));
+    int32_t* gtmp_s = perm_s + kUmmaGroupMaxN;
+    unsigned char* gscratch = reinterpret_cast<unsigned char*>(gtmp_s + MOLORA_MAX_ADAPTERS);
+    static_assert(kUmmaGroupMaxN * 4 + MOLORA_MAX_ADAPTERS * 4 + kGroupInCtaTableMaxC * kUmmaThreads * 4 + 4 * kGroupInCtaTableMaxC <=
+                      Cfg::kStages * Cfg::kStageBytes, "the grouping scratch must fit the ring");
+    static_assert(kUmmaThreads / 32 * MOLORA_MAX_ADAPTERS * 4 <= kGroupInCtaTableMaxC * kUmmaThreads * 4, "ballot-path scratch");
     int32_t offs_v[(MOLORA_MAX_ADAPTERS + kUmmaThreads) / kUmmaThreads];
 #pragma unroll
     for (int j = 0; j < (MOLORA_MAX_ADAPTERS + kUmmaThreads) / kUmmaThreads; ++j) {
         const int i = tid + j * kUmmaThreads;
-        offs_v[j] = i <= prm.C ? __ldg(prm.offsets + i) : 0;
+        offs_v[j] = (!grouping && i <= prm.C) ? __ldg(prm.offsets + i) : 0;
     }
     if (tid == 0) {
         prefetch_tensormap(&pj.tm_a);
@@ -146,13 +217,16 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             mbar_init(bar(&ctrl->empty[s]), 1);
         }
         mbar_init(bar(&ctrl->t_full), 1);
-        mbar_init(bar(&ctrl->t_ready), kTileM);
+        mbar_init(bar(&ctrl->t_ready), 2 * kTileM);      // both epilogue groups
         for (int b = 0; b < kDBufs; ++b) {
             mbar_init(bar(&ctrl->d_full[b]), 1);
             mbar_init(bar(&ctrl->d_empty[b]), kTileM);
         }
-        mbar_init(bar(&ctrl->part_full), 4 * S);     // one arrival per epilogue warp of group 0 of every CTA
-        mbar_init(bar(&ctrl->part_free), 4 * S);
+        mbar_init(bar(&ctrl->part_full), 8 * S);     // one arrival per epilogue warp of every CTA
+        // one push (ranks 16, 32): unused.  Two pushes (rank 64): the finished rows of T arrive by bulk copies that
+        // count their bytes here; the one arrival is this CTA's own, which states the byte count
+        mbar_init(bar(&ctrl->part_free), 1);
+        mbar_init(bar(&ctrl->peers_done), S > 1 ? S - 1 : 1);   // every peer has received the rows this CTA sent it
         ctrl->abort_flag = 0;
         fence_mbar_init();
     }
@@ -160,11 +234,16 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         tmem_alloc(smem_u32(&ctrl->tmem_base), kTmemCols);
         tmem_relinquish();
     }
-    // which tile is mine: the segment table goes on chip, then the tile is looked up there
+    // which tile is mine: the segment table goes on chip (or is built there), then the tile is looked up there
+    if (grouping) {
+        group_in_cta<kUmmaThreads, kUmmaGroupMaxN>(prm.r, prm.N, prm.C, offs_s, gtmp_s, perm_s, gscratch, blockIdx.y == 0,
+                                                   prm.counts_out, prm.offsets_out, prm.perm_out, prm.dev_status);
+    } else {
 #pragma unroll
-    for (int j = 0; j < (MOLORA_MAX_ADAPTERS + kUmmaThreads) / kUmmaThreads; ++j) {
-        const int i = tid + j * kUmmaThreads;
-        if (i <= prm.C) offs_s[i] = offs_v[j];
+        for (int j = 0; j < (MOLORA_MAX_ADAPTERS + kUmmaThreads) / kUmmaThreads; ++j) {
+            const int i = tid + j * kUmmaThreads;
+            if (i <= prm.C) offs_s[i] = offs_v[j];
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -179,8 +258,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     const int kx0 = (int)(crank * KXall / S), KX = (int)((crank + 1) * KXall / S) - kx0;   // my slice of d_in
     const int ny0 = (int)(crank * NYall / S), NY = (int)((crank + 1) * NYall / S) - ny0;   // my slice of d_out
     const int total = KX + NY;
-    if (tid < kTileM) ctrl->rows[tid] = tid < rows ? __ldg(prm.perm + row0 + tid) : -1;
-    __syncthreads();
+    if (tid < kTileM) ctrl->rows[tid] = tid < rows ? (grouping ? perm_s[row0 + tid] : __ldg(prm.perm + row0 + tid)) : -1;
+    __syncthreads();                    // (the ring may be filled from here on: nobody reads perm_s any more)
     // "I am running and my barriers are initialised": the matching wait comes right before the first access to
     // a peer's shared memory (the T exchange), so the cluster barrier costs nothing here
     if (S > 1) cluster_arrive_relaxed();      // (the barrier initialisation was released by fence_mbar_init)
@@ -307,18 +386,44 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         const int row = q * 32 + lane;                // tile row = TMEM lane this thread reads
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
 
-        if (group == 0) {
-            // T -> scaled bf16 hi/lo pair in shared memory, K-major, swizzled like a TMA tile of R*2-byte rows
+        {
+            // T -> scaled bf16 hi/lo pair in shared memory, K-major, swizzled like a TMA tile of R*2-byte rows.  Both
+            // epilogue groups take part, group g with the columns [g R/2, (g+1) R/2) of every row: a lone warp runs the
+            // few hundred dependent instructions of a row at one every four cycles, and its stores into a peer's shared
+            // memory at one every ~0.14 us, so the work per thread is what this step costs.
+            constexpr int RH = R / 2;
+            const int col0 = group * RH;
             wait_bar(bar(&ctrl->t_full), 0, abort_flag, prm.dev_status);
             tc_fence_after();
-            uint32_t tv[R];
+            uint32_t tv[RH];
+            if constexpr (RH == 8) {
+                tmem_ld_x8(tmem_T + lane_addr + col0, tv);
+            } else {
 #pragma unroll
-            for (int c = 0; c < R / 16; ++c) tmem_ld_x16(tmem_T + lane_addr + c * 16, tv + c * 16);
+                for (int c = 0; c < RH / 16; ++c) tmem_ld_x16(tmem_T + lane_addr + col0 + c * 16, tv + c * 16);
+            }
             tmem_wait_ld();
             // LoRA scale times the token's routing weight (1 unless the caller passes per-token factors)
             const int my_tok = ctrl->rows[row];
             const float tscale = pj.scale * ((pj.row_scale != nullptr && my_tok >= 0) ? __ldg(pj.row_scale + my_tok) : 1.f);
-            bool t_published = false;
+            // my half row -> T_hi / T_lo of this CTA
+            auto publish_local = [&]() {
+#pragma unroll
+                for (int c8 = 0; c8 < RH / 8; ++c8) {
+                    float hi[8], lo[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float t = __uint_as_float(tv[c8 * 8 + e]) * tscale;
+                        hi[e] = __bfloat162float(__float2bfloat16_rn(t));
+                        lo[e] = t - hi[e];
+                    }
+                    const uint32_t off = swizzle_offset((uint32_t)row * Cfg::kTRowBytes + (uint32_t)(col0 / 8 + c8) * 16, Cfg::kSwzBits);
+                    const uint4 h = pack<__nv_bfloat16>(hi), l = pack<__nv_bfloat16>(lo);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(thi + off), "r"(h.x), "r"(h.y), "r"(h.z), "r"(h.w) : "memory");
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(tlo + off), "r"(l.x), "r"(l.y), "r"(l.z), "r"(l.w) : "memory");
+                }
+            };
+            const float4* recv_p = reinterpret_cast<const float4*>(smem_raw + (recv - raw));
             if (Cfg::kOnePush && S > 1) {
                 // Exchange of the partial T tiles in one push through distributed shared memory: every CTA writes its
                 // partial into its slot at every peer, one barrier round, and every CTA sums all partials itself in
@@ -330,50 +435,26 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                     const uint32_t slot = crank < q2 ? crank : crank - 1;                   // my slot at CTA q2
                     const uint32_t dst = map_to_cta(recv, q2) + slot * (uint32_t)(kTileM * R * 4);
 #pragma unroll
-                    for (int c4 = 0; c4 < R / 4; ++c4)
-                        st_cluster_u32x4(dst + (uint32_t)(c4 * kTileM + row) * 16u, tv[4 * c4], tv[4 * c4 + 1], tv[4 * c4 + 2],
-                                         tv[4 * c4 + 3]);
+                    for (int c4 = 0; c4 < RH / 4; ++c4)
+                        st_cluster_u32x4(dst + (uint32_t)((col0 / 4 + c4) * kTileM + row) * 16u, tv[4 * c4], tv[4 * c4 + 1],
+                                         tv[4 * c4 + 2], tv[4 * c4 + 3]);
                 }
                 __syncwarp();                                   // the warp's rows are sent; lane q2 tells CTA q2
                 if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
                 wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
-#pragma unroll
-                for (int c4 = 0; c4 < R / 4; ++c4) {            // rank order, in place
-                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (uint32_t q2 = 0; q2 < S; ++q2) {
-                        float4 v;
-                        if (q2 == crank) {
-                            v = make_float4(__uint_as_float(tv[4 * c4]), __uint_as_float(tv[4 * c4 + 1]),
-                                            __uint_as_float(tv[4 * c4 + 2]), __uint_as_float(tv[4 * c4 + 3]));
-                        } else {
-                            const uint32_t src = recv + (q2 < crank ? q2 : q2 - 1) * (uint32_t)(kTileM * R * 4);
-                            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                                         : "r"(src + (uint32_t)(c4 * kTileM + row) * 16u)
-                                         : "memory");
-                        }
-                        a.x += v.x;
-                        a.y += v.y;
-                        a.z += v.z;
-                        a.w += v.w;
-                    }
-                    tv[4 * c4] = __float_as_uint(a.x);
-                    tv[4 * c4 + 1] = __float_as_uint(a.y);
-                    tv[4 * c4 + 2] = __float_as_uint(a.z);
-                    tv[4 * c4 + 3] = __float_as_uint(a.w);
-                }
-                // tv now holds the full T row: the local conversion below finishes it
+                sum_partials<RH>(tv, recv_p + (col0 / 4) * kTileM + row, kTileM, kTileM * R / 4, S, crank);
+                publish_local();                                // tv holds the full half row
             } else if (S > 1) {
                 // Exchange of the partial T tiles in two pushes through distributed shared memory.  CTA o owns the
                 // tile rows [o*128/S, (o+1)*128/S): (1) every CTA sends its partial of a row to the row's owner;
                 // (2) the owner sums the partials in rank order (the same bits whoever computes them), scales,
-                // splits into bf16 hi + lo and writes the finished row into the T_hi / T_lo tiles of every CTA.
-                // Nothing is ever read from a peer, and after step 2 nobody touches this CTA's memory again, so
-                // the CTAs of a cluster retire independently.
+                // splits into bf16 hi + lo and writes the finished rows into its own T_hi / T_lo tiles; (3) bulk copies
+                // carry them into the tiles of every peer.  Nothing is ever read from a peer by a thread; a CTA retires
+                // once every peer has confirmed the arrival of its rows (peers_done, waited for at the very end).
                 const int rows_max = (kTileM + (int)S - 1) / (int)S;
                 int owner = 0;
 #pragma unroll
-                for (int o = 1; o < kMaxSplit; ++o)
+                for (int o = 1; o < Cfg::kMaxSplitR; ++o)
                     if ((uint32_t)o < S && row >= o * kTileM / (int)S) owner = o;
                 const int own_lo = owner * kTileM / (int)S;
                 cluster_wait();                                 // every peer is running, its barriers initialised
@@ -381,77 +462,38 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                     const uint32_t slot = crank < (uint32_t)owner ? crank : crank - 1;      // my slot at the owner
                     const uint32_t dst = map_to_cta(recv, (uint32_t)owner) + slot * (uint32_t)(rows_max * R * 4);
 #pragma unroll
-                    for (int c4 = 0; c4 < R / 4; ++c4)
-                        st_cluster_u32x4(dst + (uint32_t)(c4 * rows_max + (row - own_lo)) * 16u, tv[4 * c4], tv[4 * c4 + 1],
-                                         tv[4 * c4 + 2], tv[4 * c4 + 3]);
+                    for (int c4 = 0; c4 < RH / 4; ++c4)
+                        st_cluster_u32x4(dst + (uint32_t)((col0 / 4 + c4) * rows_max + (row - own_lo)) * 16u, tv[4 * c4],
+                                         tv[4 * c4 + 1], tv[4 * c4 + 2], tv[4 * c4 + 3]);
                 }
                 __syncwarp();                                   // the warp's rows are sent; lane q2 tells CTA q2
                 if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
                 wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
                 if ((uint32_t)owner == crank) {
-                    // sum in rank order, in place: lower ranks' partials, mine (registers), higher ranks'
-#pragma unroll
-                    for (int c4 = 0; c4 < R / 4; ++c4) {
-                        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (uint32_t q2 = 0; q2 < S; ++q2) {
-                            float4 v;
-                            if (q2 == crank) {
-                                v = make_float4(__uint_as_float(tv[4 * c4]), __uint_as_float(tv[4 * c4 + 1]),
-                                                __uint_as_float(tv[4 * c4 + 2]), __uint_as_float(tv[4 * c4 + 3]));
-                            } else {
-                                const uint32_t src = recv + (q2 < crank ? q2 : q2 - 1) * (uint32_t)(rows_max * R * 4);
-                                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                                             : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                                             : "r"(src + (uint32_t)(c4 * rows_max + (row - own_lo)) * 16u)
-                                             : "memory");
-                            }
-                            a.x += v.x;
-                            a.y += v.y;
-                            a.z += v.z;
-                            a.w += v.w;
-                        }
-                        tv[4 * c4] = __float_as_uint(a.x);
-                        tv[4 * c4 + 1] = __float_as_uint(a.y);
-                        tv[4 * c4 + 2] = __float_as_uint(a.z);
-                        tv[4 * c4 + 3] = __float_as_uint(a.w);
-                    }
-#pragma unroll
-                    for (int c8 = 0; c8 < R / 8; ++c8) {
-                        float hi[8], lo[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const float t = __uint_as_float(tv[c8 * 8 + e]) * tscale;
-                            hi[e] = __bfloat162float(__float2bfloat16_rn(t));
-                            lo[e] = t - hi[e];
-                        }
-                        const uint32_t off = swizzle_offset((uint32_t)row * Cfg::kTRowBytes + c8 * 16, Cfg::kSwzBits);
-                        const uint4 h = pack<__nv_bfloat16>(hi), l = pack<__nv_bfloat16>(lo);
-                        for (uint32_t q2 = 0; q2 < S; ++q2) {
-                            st_cluster_u32x4(map_to_cta(thi + off, q2), h.x, h.y, h.z, h.w);
-                            st_cluster_u32x4(map_to_cta(tlo + off, q2), l.x, l.y, l.z, l.w);
-                        }
-                    }
+                    sum_partials<RH>(tv, recv_p + (col0 / 4) * rows_max + (row - own_lo), rows_max, rows_max * R / 4, S, crank);
+                    publish_local();
                 }
-                __syncwarp();                                   // the warp's rows are published everywhere
-                if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_free), (uint32_t)lane));
-                wait_bar_cluster(bar(&ctrl->part_free), 0, abort_flag, prm.dev_status);   // all 128 rows of T are here
-                t_published = true;
-            }
-            if (!t_published) {
-#pragma unroll
-                for (int c8 = 0; c8 < R / 8; ++c8) {
-                    float hi[8], lo[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float t = __uint_as_float(tv[c8 * 8 + e]) * tscale;
-                        hi[e] = __bfloat162float(__float2bfloat16_rn(t));
-                        lo[e] = t - hi[e];
+                // (3) my rows are a contiguous piece of each T tile (the swizzle permutes inside a row): two bulk copies
+                // per peer carry them over and count their bytes on the peer's barrier
+                fence_proxy_async_smem();                       // my rows, written above, are read by the copy engine
+                asm volatile("bar.sync 3, 256;" ::: "memory");  // the eight epilogue warps
+                if (group == 0) {
+                    const int mine_lo = (int)crank * kTileM / (int)S, mine_hi = (int)(crank + 1) * kTileM / (int)S;
+                    const uint32_t out_off = (uint32_t)mine_lo * Cfg::kTRowBytes;
+                    const uint32_t out_bytes = (uint32_t)(mine_hi - mine_lo) * Cfg::kTRowBytes;
+                    if (et == 0) mbar_arrive_expect_tx(bar(&ctrl->part_free), 2u * ((uint32_t)kTileM * Cfg::kTRowBytes - out_bytes));
+                    if (warp == kEpiWarp0 && (uint32_t)lane < S && (uint32_t)lane != crank && !*abort_flag) {   // lane q2 serves CTA q2
+                        const uint32_t pb = map_to_cta(bar(&ctrl->part_free), (uint32_t)lane);
+                        bulk_copy_to_peer(map_to_cta(thi + out_off, (uint32_t)lane), thi + out_off, out_bytes, pb);
+                        bulk_copy_to_peer(map_to_cta(tlo + out_off, (uint32_t)lane), tlo + out_off, out_bytes, pb);
                     }
-                    const uint32_t off = swizzle_offset((uint32_t)row * Cfg::kTRowBytes + c8 * 16, Cfg::kSwzBits);
-                    const uint4 h = pack<__nv_bfloat16>(hi), l = pack<__nv_bfloat16>(lo);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(thi + off), "r"(h.x), "r"(h.y), "r"(h.z), "r"(h.w) : "memory");
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(tlo + off), "r"(l.x), "r"(l.y), "r"(l.z), "r"(l.w) : "memory");
+                    wait_bar_cluster(bar(&ctrl->part_free), 0, abort_flag, prm.dev_status);   // all 128 rows of T are here
+                    // tell every peer that its rows have arrived: it must not retire while the copy engine still reads them
+                    if (warp == kEpiWarp0 && (uint32_t)lane < S && (uint32_t)lane != crank)
+                        mbar_arrive_remote(map_to_cta(bar(&ctrl->peers_done), (uint32_t)lane));
                 }
+            } else {
+                publish_local();
             }
             fence_proxy_async_smem();
             tc_fence_before();
@@ -535,7 +577,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
     // threads that took no part in the exchange complete the start-up cluster barrier here (it has long been
     // passed); no closing barrier is needed, see the exchange
-    if (S > 1 && !(warp >= kEpiWarp0 && warp < kEpiWarp0 + 4)) cluster_wait();
+    if (S > 1 && warp < kEpiWarp0) cluster_wait();
+    // two-push exchange: my rows of T were copied out of my shared memory by the copy engine; every peer has confirmed
+    // their arrival long ago, this wait only makes it certain before the memory is given up
+    if (!Cfg::kOnePush && S > 1 && tid == 0) wait_bar_cluster(bar(&ctrl->peers_done), 0, abort_flag, prm.dev_status);
 }
 
 // Self-test of the bounded wait: one warp waits on an mbarrier that nothing ever arrives on, with a limit of
@@ -581,13 +626,13 @@ struct UmmaPlan {
     int tile_rows;   // positions per tile
 };
 
-template <int R>
+template <int R, bool WIDE>
 static void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int64_t tiles, int P, int split,
                                cudaStream_t s)
 {
     cfg.gridDim = dim3((unsigned)(tiles * split), (unsigned)P, 1);
     cfg.blockDim = dim3(kUmmaThreads, 1, 1);
-    cfg.dynamicSmemBytes = UmmaCfg<R>::kSmemBytes;
+    cfg.dynamicSmemBytes = UmmaCfg<R, WIDE>::kSmemBytes;
     cfg.stream = s;
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)split;
@@ -597,16 +642,16 @@ static void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* att
     cfg.numAttrs = 1;
 }
 
-template <int R>
-static cudaError_t umma_launch(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStream_t s)
+template <int R, bool WIDE>
+static cudaError_t umma_launch_variant(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStream_t s)
 {
     const int split = plan.split;
     prm.tile_rows = plan.tile_rows;
-    using Cfg = UmmaCfg<R>;
+    using Cfg = UmmaCfg<R, WIDE>;
     static bool configured_dev[kMaxDevices] = {};
     bool& configured = configured_dev[device_slot()];
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(apply_umma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(apply_umma_kernel<R, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              Cfg::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
@@ -614,28 +659,51 @@ static cudaError_t umma_launch(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStr
     const int64_t tiles = ceil_div64(N, prm.tile_rows) + prm.C;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
-    fill_launch_config<R>(cfg, attr, tiles, prm.P, split, s);
+    fill_launch_config<R, WIDE>(cfg, attr, tiles, prm.P, split, s);
     note_launch();
-    return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R>, prm);
+    return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R, WIDE>, prm);
+}
+
+template <int R>
+static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, UmmaPlan plan, cudaStream_t s)
+{
+    if constexpr (R == 64) {
+        if (plan.split > UmmaCfg<64, false>::kMaxSplitR) return umma_launch_variant<64, true>(prm, N, plan, s);
+    }
+    return umma_launch_variant<R, false>(prm, N, plan, s);
 }
 
 // Clusters of `split` CTAs of this kernel that can be resident at once (cached per rank and split).
-template <int R>
-static int max_active_clusters(int split)
+template <int R, bool WIDE>
+static int max_active_clusters_variant(int split)
 {
-    static int cache_dev[kMaxDevices][kMaxSplit + 1] = {};
-    int (&cache)[kMaxSplit + 1] = cache_dev[device_slot()];
+    static int cache_dev[kMaxDevices][kMaxWideSplit + 1] = {};
+    int (&cache)[kMaxWideSplit + 1] = cache_dev[device_slot()];
     if (cache[split] == 0) {
-        cudaFuncSetAttribute(apply_umma_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, UmmaCfg<R>::kSmemBytes);
+        cudaFuncSetAttribute(apply_umma_kernel<R, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             UmmaCfg<R, WIDE>::kSmemBytes);
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute attr[1];
-        fill_launch_config<R>(cfg, attr, 148, 1, split, nullptr);
+        fill_launch_config<R, WIDE>(cfg, attr, 148, 1, split, nullptr);
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, apply_umma_kernel<R>, &cfg) != cudaSuccess || n <= 0) n = 148 / split;
+        if (cudaOccupancyMaxActiveClusters(&n, apply_umma_kernel<R, WIDE>, &cfg) != cudaSuccess || n <= 0) n = 148 / split;
         cache[split] = n;
     }
     return cache[split];
 }
+
+template <int R>
+static int max_active_clusters(int split)
+{
+    if constexpr (R == 64) {
+        if (split > UmmaCfg<64, false>::kMaxSplitR) return max_active_clusters_variant<64, true>(split);
+    }
+    return max_active_clusters_variant<R, false>(split);
+}
+
+// Largest cluster a tile of rank R may be split over (rank 64: through the variant with the larger exchange buffer).
+template <int R>
+constexpr int max_split_for_rank() { return R == 64 ? kMaxWideSplit : UmmaCfg<R>::kMaxSplitR; }
 
 // CTAs per tile.  Tiles are 128 rows, so small calls have too few of them for 148 SMs; a tile can be split over
 // a cluster of 2 or 4 CTAs.  Pick the split with the smallest estimated time: waves of resident clusters times
@@ -659,7 +727,7 @@ static UmmaPlan choose_split_for_rank(const UmmaParams& prm, int64_t N)
     UmmaPlan best = {1, kTileM};
     const int64_t fsplit = tune(kTuneUmmaSplit), frows = tune(kTuneUmmaTileRows);          // tuning overrides
     if (fsplit > 0 || frows > 0) {
-        if (fsplit > 0) best.split = (int)std::max<int64_t>(1, std::min<int64_t>(fsplit, UmmaCfg<R>::kMaxSplitR));
+        if (fsplit > 0) best.split = (int)std::max<int64_t>(1, std::min<int64_t>(fsplit, max_split_for_rank<R>()));
         if (frows > 0) best.tile_rows = (int)std::max<int64_t>(32, std::min<int64_t>(frows, kTileM));
     } else {
         double best_cost = 1e30, best_waves = 0;
@@ -683,12 +751,26 @@ static UmmaPlan choose_split_for_rank(const UmmaParams& prm, int64_t N)
     return best;
 }
 
+bool group_apply_umma_eligible(int64_t N, int32_t C) { return N >= 1 && N <= kUmmaGroupMaxN && C <= kUmmaAllSegmentsMaxC; }
+
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                   const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
-                                  cudaStream_t s)
+                                  cudaStream_t s, const int32_t* r, int32_t* counts_out)
 {
     if (N == 0 || P == 0) return MOLORA_OK;
     UmmaParams prm;
+    // r given: the kernel groups on chip and writes counts / offsets / perm (the pointers are then outputs); one launch
+    // only, so every projection must have the same rank
+    prm.r = r;
+    prm.N = (int32_t)N;
+    prm.counts_out = counts_out;
+    prm.offsets_out = const_cast<int32_t*>(offsets);
+    prm.perm_out = const_cast<int32_t*>(perm);
+    if (r != nullptr) {
+        if (!group_apply_umma_eligible(N, C) || min_rows > 1) return MOLORA_ERR_UNSUPPORTED;
+        for (int i = 1; i < P; ++i)
+            if (projs[i].rank != projs[0].rank) return MOLORA_ERR_UNSUPPORTED;
+    }
     bool has[3] = {false, false, false};
     // CTAs are dispatched projection by projection (blockIdx.y): put the projections that move the most bytes
     // per tile first, so that the last, partly filled wave consists of the cheap tiles.

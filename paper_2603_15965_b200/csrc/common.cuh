@@ -258,9 +258,12 @@ molora_status_t launch_apply_rowtile(const molora_proj_desc_t* projs, int32_t P,
                                      cudaStream_t s);
 // tcgen05 path for the segments with at least min_rows rows (bf16, rank 16/32/64, d_in and d_out multiples of 64).
 bool umma_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
+// With r (routing decisions, at most 4096 tokens, one rank, min_rows 1) the kernel groups on chip: offsets / perm /
+// counts_out are then OUTPUTS, bit-equal to launch_group's.
+bool group_apply_umma_eligible(int64_t N, int32_t C);
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                   const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
-                                  cudaStream_t s);
+                                  cudaStream_t s, const int32_t* r = nullptr, int32_t* counts_out = nullptr);
 
 // mma.sync path for decode-sized calls (bf16, rank 16/32/64, d_in and d_out multiples of 32): a shrink launch and
 // an expand launch; takes the segments with fewer than max_rows rows.  The workspace holds the fp32 partial
