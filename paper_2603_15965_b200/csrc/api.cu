@@ -53,24 +53,34 @@ namespace {
 //   rank 16  streaming wins until the projections of the call move ~150 MB (x once, y twice), tcgen05 above;
 //   rank 32  streaming until ~60 MB, tcgen05 above (below 1024 tokens the two-launch pair ties for one projection
 //            and loses by a third for a layer's worth of them);
-//   rank 64  below 1280 tokens the two-launch pair for one or two projections and the streaming kernel for more,
-//            tcgen05 above (the streaming kernel has only two stages at this rank).
+//   rank 64  tcgen05 (tiles split over clusters of up to 8 CTAs) once the projections of the call move ~12 MB with at
+//            least 256 tokens and segments of 32 rows on average (one 4096-wide projection: from 512 tokens, 21.0 us
+//            against 24.3; two: 23.2 against 38.9 at 512 tokens; a layer of seven: 89.7 against 134.9), and from 1280
+//            tokens in any case; below, the two-launch pair for one or two projections and the streaming kernel for
+//            more (the streaming kernel has only two stages at this rank).
 // The overrides "umma_min_tokens" (tcgen05 from n tokens) and "small_path" (the kernel used below it) of
 // molora_debug_set force a choice, for measurements and for tests that target one kernel.
 int64_t forced_umma_min_tokens() { return std::max<int64_t>(0, tune(kTuneUmmaMinTokens)); }
 constexpr double kUmmaMinBytesR16 = 150e6, kUmmaMinBytesR32 = 60e6;
-constexpr int64_t kUmmaMinTokensR64 = 1280;
+constexpr int64_t kUmmaMinTokensR64 = 1280, kUmmaMinTokensR64Wide = 256;
+constexpr double kUmmaMinBytesR64 = 12e6;
 
 double proj_bytes(int64_t N, int32_t d_in, int32_t d_out) { return (double)N * ((double)d_in + 2.0 * d_out) * 2.0; }
 
 // group_bytes: bytes moved by all projections of this rank in the call
-bool use_umma(int32_t rank, int64_t N, double group_bytes)
+// rank 64: group_bytes may be a lower bound (one projection's own bytes when the others are not known)
+bool use_umma_r64(int64_t N, int32_t C, double group_bytes)
+{
+    if (N >= kUmmaMinTokensR64) return true;
+    return N >= kUmmaMinTokensR64Wide && N >= (int64_t)C * kUmmaMinRows && group_bytes >= kUmmaMinBytesR64;
+}
+bool use_umma(int32_t rank, int64_t N, int32_t C, double group_bytes)
 {
     if (const int64_t forced = forced_umma_min_tokens()) return N >= forced;
+    if (rank == 64) return use_umma_r64(N, C, group_bytes);
     if (N < kUmmaMinTokens) return false;
     if (rank == 16) return group_bytes >= kUmmaMinBytesR16;
-    if (rank == 32) return group_bytes >= kUmmaMinBytesR32;
-    return N >= kUmmaMinTokensR64;
+    return group_bytes >= kUmmaMinBytesR32;
 }
 // the kernel for what the tcgen05 kernel does not take; same_rank: projections of this rank in the call (0: unknown)
 bool small_path_is_stream(int32_t rank, int64_t N, int same_rank)
@@ -243,7 +253,7 @@ size_t molora_apply_workspace_bytes(int64_t N, int32_t C, int32_t d_in, int32_t 
     // two-launch kernels: needed unless the tcgen05 kernel is certain to take every segment (for ranks 16 and 32 that
     // depends on the other projections of the call, which are not known here)
     const int64_t forced = forced_umma_min_tokens();
-    const bool umma_certain = forced > 0 ? N >= forced : (rank == 64 && N >= kUmmaMinTokensR64);
+    const bool umma_certain = forced > 0 ? N >= forced : (rank == 64 && use_umma_r64(N, C, proj_bytes(N, d_in, d_out)));
     if (umma_certain && C <= kUmmaAllSegmentsMaxC && (d_in % 64) == 0 && (d_out % 64) == 0) return need;
     return need + decode_workspace_bytes(N, d_in, rank);
 }
@@ -287,7 +297,7 @@ molora_status_t plan_apply(const molora_proj_desc_t* projs, int32_t P, molora_dt
         if (decode_eligible(projs[i], dt)) ++same_rank[group_of(projs[i].rank)];
     for (int i = 0; i < P; ++i) {
         const int32_t rank = projs[i].rank;
-        if (umma_eligible(projs[i], dt) && use_umma(rank, N, group_bytes[group_of(rank)])) pl.tc[pl.n_tc++] = projs[i];
+        if (umma_eligible(projs[i], dt) && use_umma(rank, N, C, group_bytes[group_of(rank)])) pl.tc[pl.n_tc++] = projs[i];
         else if (use_jobs(projs[i], dt, N, C, same_rank[group_of(rank)])) pl.jc[group_of(rank)][pl.n_jc[group_of(rank)]++] = projs[i];
         else if (decode_eligible(projs[i], dt)) {
             if (small_path_is_stream(rank, N, same_rank[group_of(rank)])) pl.sc[pl.n_sc++] = projs[i];
@@ -378,7 +388,7 @@ static int group_apply_mode(const molora_proj_desc_t* projs, int32_t P, molora_d
         umma = umma && umma_eligible(projs[i], dt);
         if (umma_eligible(projs[i], dt)) bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
     }
-    if (use_umma(projs[0].rank, N, bytes)) return umma && group_apply_umma_eligible(N, C) ? 4 : 0;
+    if (use_umma(projs[0].rank, N, C, bytes)) return umma && group_apply_umma_eligible(N, C) ? 4 : 0;
     if (jobs) return 3;
     if (stream && group_apply_stream_eligible(N)) return 1;
     if (twophase && group_apply_decode_eligible(N)) return 2;
@@ -519,7 +529,7 @@ bool topk_single_pass(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t
         if (projs[i].rank != projs[0].rank) return false;
         bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
     }
-    return !use_umma(projs[0].rank, N, bytes);
+    return !use_umma(projs[0].rank, N, C, bytes);
 }
 }  // namespace
 

@@ -705,45 +705,67 @@ static int max_active_clusters(int split)
 template <int R>
 constexpr int max_split_for_rank() { return R == 64 ? kMaxWideSplit : UmmaCfg<R>::kMaxSplitR; }
 
-// CTAs per tile.  Tiles are 128 rows, so small calls have too few of them for 148 SMs; a tile can be split over
-// a cluster of 2 or 4 CTAs.  Pick the split with the smallest estimated time: waves of resident clusters times
-// (work per CTA, which shrinks with the split, plus a fixed per-CTA cost and the cost of the exchange).
+// CTAs per tile.  Tiles are 128 rows, so small calls have too few of them for 148 SMs; a tile can be split over a
+// cluster (up to 4 CTAs; up to 8 at rank 64).  Pick the split with the smallest estimated time, in microseconds, from a
+// model fitted to one-projection 4096 -> 4096 calls at rank 64 (64 ... 4096 tokens, every split, graph replay): a wave of
+// resident clusters costs a fixed 9 us (launch, tile look-up, first arrival, last stores), 3 us more for the exchange
+// of the partial T tiles, and 0.40 us per 64-column chunk a CTA walks (shrink chunks + expand chunks divided by the
+// split); shorter tiles make a chunk only a little cheaper (the gathers are bound by requests in flight, not bytes).
 template <int R>
 static UmmaPlan choose_split_for_rank(const UmmaParams& prm, int64_t N)
 {
     int min_kx = INT32_MAX, nproj = 0;
+    double chunks[MOLORA_MAX_PROJECTIONS];         // 64-column chunks a tile of each projection of this rank walks
     for (int i = 0; i < prm.P; ++i) {
         if (prm.p[i].rank != R) continue;
         min_kx = std::min(min_kx, prm.p[i].d_in / kChunkCols);
-        ++nproj;
+        chunks[nproj++] = (double)((prm.p[i].d_in + prm.p[i].d_out) / kChunkCols);
     }
-    // expected tiles: every segment ends in a partial tile
-    auto tiles_for = [&](int rows) { return (ceil_div64(N, rows) + prm.C / 2) * nproj; };
-    auto cost_for = [&](int rows, int split, double& waves) {
+    // expected tiles per projection: every segment has at least one and ends in a partial one
+    auto tiles_for = [&](int rows) { return std::max<int64_t>(prm.C, ceil_div64(N, rows) + prm.C / 2); };
+    // Estimated time of the launch: the CTAs are dispatched heaviest projection first onto the resident clusters, so the
+    // launch lasts as long as its heaviest tile or as the whole work spread over the cluster slots (plus a quarter of a
+    // light tile of imbalance), whichever is longer; with equal tiles it is whole waves.
+    auto cost_for = [&](int rows, int split, bool& one_wave) {
         const int resident = max_active_clusters<R>(split);
-        waves = (double)((tiles_for(rows) + resident - 1) / resident);
-        return waves * ((rows / 128.0) / split + 0.15 + (split > 1 ? 0.10 : 0.0));
+        const int64_t tiles = tiles_for(rows);
+        // (a chunk costs up to 1.4 times as much once every SM streams: 35 GB/s per SM instead of ~50)
+        const double load = std::min(1.0, (double)(tiles * nproj * split) / 148.0);
+        const double fixed = 9.0 + (split > 1 ? 3.0 : 0.0);
+        const double per_chunk = 0.40 * (1.0 + 0.4 * load * load) * (0.7 + 0.3 * rows / 128.0) / split;
+        double cmax = 0.0, cmin = 1e30, total = 0.0;
+        for (int i = 0; i < nproj; ++i) {
+            const double c = fixed + per_chunk * chunks[i];
+            cmax = std::max(cmax, c);
+            cmin = std::min(cmin, c);
+            total += c * (double)tiles;
+        }
+        one_wave = tiles * nproj * 1.1 <= resident;         // (margin: the tile count is an estimate)
+        if (one_wave) return cmax;
+        if (cmax - cmin < 1e-9) return cmax * (double)((tiles * nproj + resident - 1) / resident);
+        return std::max(cmax, total / resident + 0.25 * cmin);
     };
     UmmaPlan best = {1, kTileM};
     const int64_t fsplit = tune(kTuneUmmaSplit), frows = tune(kTuneUmmaTileRows);          // tuning overrides
     if (fsplit > 0 || frows > 0) {
         if (fsplit > 0) best.split = (int)std::max<int64_t>(1, std::min<int64_t>(fsplit, max_split_for_rank<R>()));
         if (frows > 0) best.tile_rows = (int)std::max<int64_t>(32, std::min<int64_t>(frows, kTileM));
-    } else {
-        double best_cost = 1e30, best_waves = 0;
-        for (int split = 1; split <= UmmaCfg<R>::kMaxSplitR; ++split) {    // cluster sizes need not be powers of two
-            double waves;
-            const double cost = cost_for(kTileM, split, waves);
-            if (cost < best_cost - 1e-9) { best_cost = cost; best_waves = waves; best = {split, kTileM}; }
+    } else if (nproj > 0) {
+        double best_cost = 1e30;
+        bool best_one_wave = false;
+        for (int split = 1; split <= max_split_for_rank<R>(); ++split) {    // cluster sizes need not be powers of two
+            bool one_wave;
+            const double cost = cost_for(kTileM, split, one_wave);
+            if (cost < best_cost - 1e-9) { best_cost = cost; best_one_wave = one_wave; best = {split, kTileM}; }
         }
         // A call that does not even fill one wave can use shorter tiles (the MMA tile keeps 128 lanes, the extra
         // lanes idle) to put more SMs to work, as long as everything still fits in one wave.
-        if (best_waves <= 1.0 && tiles_for(kTileM) * best.split < 0.85 * 148) {
+        if (best_one_wave && tiles_for(kTileM) * nproj * best.split < 0.85 * 148) {
             for (int rows = 96; rows >= 64; rows -= 32)
-                for (int split = 1; split <= UmmaCfg<R>::kMaxSplitR; ++split) {
-                    double waves;
-                    const double cost = cost_for(rows, split, waves);
-                    if (waves <= 1.0 && cost < best_cost - 1e-9) { best_cost = cost; best = {split, rows}; }
+                for (int split = 1; split <= max_split_for_rank<R>(); ++split) {
+                    bool one_wave;
+                    const double cost = cost_for(rows, split, one_wave);
+                    if (one_wave && cost < best_cost - 1e-9) { best_cost = cost; best = {split, rows}; }
                 }
         }
     }

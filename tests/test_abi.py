@@ -101,13 +101,16 @@ def test_apply_workspace_sizes_and_refusal_without_it(default_kernels):
     assert M.molora_apply_workspace_bytes(1025, 8, 2048, 2048, 16) == 0                 # more tokens than the kernel takes
     M.molora_debug_set("small_path", 0)
     # by default the job-list kernel takes rank 16 between 257 and 1024 tokens (with at least four projections, which is
-    # not known here), rank 64 below 1280 tokens may run on the two-launch kernels
+    # not known here); rank 64 runs on the two-launch kernels while the projection moves less than ~12 MB (x once, y
+    # twice) or has fewer than 256 tokens, on the tcgen05 kernel (no scratch) above
     assert M.molora_apply_workspace_bytes(512, 8, 2048, 2048, 16) == ctl + (512 // 16 + 8) * 6 * 16 * 16 * 8
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 16) == 0
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 32) == 0
     assert M.molora_apply_workspace_bytes(256, 8, 2048, 2048, 64) == 4 * 256 * 64 * 4
-    assert M.molora_apply_workspace_bytes(1024, 8, 2048, 2048, 64) > 0
-    # larger calls of ranks 16 and 32 (streaming or tcgen05 kernel), rank 64 from 1280 tokens with few adapters, rank 8
+    assert M.molora_apply_workspace_bytes(512, 8, 2048, 2048, 64) > 0          # 6.3 MB
+    assert M.molora_apply_workspace_bytes(1024, 8, 2048, 2048, 64) == 0        # 12.6 MB
+    assert M.molora_apply_workspace_bytes(1024, 64, 2048, 2048, 64) > 0        # 16-row segments on average: small tiles
+    # larger calls of ranks 16 and 32 (streaming or tcgen05 kernel), rank 64 from 1280 tokens in any case, rank 8
     # and fp32-only shapes need none
     assert M.molora_apply_workspace_bytes(4096, 4, 2048, 2048, 16) == 0
     assert M.molora_apply_workspace_bytes(2048, 4, 2048, 2048, 32) == 0
@@ -148,12 +151,19 @@ def test_group_apply_one_call_launch_count_and_refusals(default_kernels):
     arr64 = (_ProjDescC * 1)(_desc(2048, 2048, 64))
     assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 512, 8)) == 1    # two-launch kernels group on chip
     M.molora_debug_set("small_path", 2)
+    M.molora_debug_set("umma_min_tokens", 1000000)
     assert int(lib.molora_group_apply_skips_group_launch(arr64, 1, M.BF16, 1100, 8)) == 0   # more than 1024 tokens: they do not
     assert one_launch([(2048, 2048, 16)], 4096) == 0
     M.molora_debug_set("small_path", 0)
-    assert one_launch([(2048, 2048, 64)] * 3, 2048) == 0                # rank 64 from 1280 tokens: tcgen05
+    M.molora_debug_set("umma_min_tokens", 0)
+    # rank 64 on the tcgen05 kernel (from ~12 MB with 256 tokens, from 1280 tokens in any case): it groups on chip, one
+    # launch, up to 4096 tokens and 64 adapters
+    assert one_launch([(2048, 2048, 64)] * 3, 2048) == 1
+    assert one_launch([(4096, 4096, 64)], 1024) == 1 and one_launch([(4096, 4096, 64)], 4096) == 1
+    assert one_launch([(4096, 4096, 64)], 4097) == 0 and one_launch([(4096, 4096, 64)], 2048, C=128) == 0
     assert one_launch([(2048, 2048, 16), (2048, 2048, 32)], 2048) == 0  # two ranks: two apply launches
-    assert one_launch([(2048, 2048, 16)] * 8, 4096) == 0                # 400 MB: above the tcgen05 crossover
+    assert one_launch([(2048, 2048, 16)] * 8, 4096) == 1                # 400 MB: tcgen05 kernel, grouping inside
+    assert one_launch([(2048, 2048, 16)] * 8, 8192) == 0                # ... beyond 4096 tokens: grouping launch + apply
     assert one_launch([(2048, 2048, 16)], 4096, M.F32) == 0             # fp32 storage: CUDA-core kernel
     assert one_launch([(2048, 2040, 16)], 256) == 0                     # width not a multiple of 32: CUDA-core kernel
     # refusals before any launch: null outputs, too many adapters, no projections, unsupported rank
