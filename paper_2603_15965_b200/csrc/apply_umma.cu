@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             mbar_init(bar(&ctrl->d_full[b]), 1);
             mbar_init(bar(&ctrl->d_empty[b]), kTileM);
         }
-        mbar_init(bar(&ctrl->part_full), 8 * S);     // one arrival per epilogue warp of every CTA
+        mbar_init(bar(&ctrl->part_full), 1);         // the partials arrive as asynchronous stores that count their bytes here
         // one push (ranks 16, 32): unused.  Two pushes (rank 64): the finished rows of T arrive by bulk copies that
         // count their bytes here; the one arrival is this CTA's own, which states the byte count
         mbar_init(bar(&ctrl->part_free), 1);
@@ -430,17 +430,17 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 // rank order (the same bits in every CTA).  Nothing is read from a peer and nobody touches this CTA's
                 // memory afterwards, so the CTAs of a cluster retire independently.
                 cluster_wait();                                 // every peer is running, its barriers initialised
+                if (group == 0 && et == 0) mbar_arrive_expect_tx(bar(&ctrl->part_full), (S - 1) * (uint32_t)(kTileM * R * 4));
                 for (uint32_t q2 = 0; q2 < S; ++q2) {
                     if (q2 == crank) continue;
                     const uint32_t slot = crank < q2 ? crank : crank - 1;                   // my slot at CTA q2
                     const uint32_t dst = map_to_cta(recv, q2) + slot * (uint32_t)(kTileM * R * 4);
+                    const uint32_t pb = map_to_cta(bar(&ctrl->part_full), q2);              // counts the bytes it receives
 #pragma unroll
                     for (int c4 = 0; c4 < RH / 4; ++c4)
-                        st_cluster_u32x4(dst + (uint32_t)((col0 / 4 + c4) * kTileM + row) * 16u, tv[4 * c4], tv[4 * c4 + 1],
-                                         tv[4 * c4 + 2], tv[4 * c4 + 3]);
+                        st_async_cluster_u32x4(dst + (uint32_t)((col0 / 4 + c4) * kTileM + row) * 16u, tv[4 * c4], tv[4 * c4 + 1],
+                                               tv[4 * c4 + 2], tv[4 * c4 + 3], pb);
                 }
-                __syncwarp();                                   // the warp's rows are sent; lane q2 tells CTA q2
-                if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
                 wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
                 sum_partials<RH>(tv, recv_p + (col0 / 4) * kTileM + row, kTileM, kTileM * R / 4, S, crank);
                 publish_local();                                // tv holds the full half row
@@ -458,16 +458,19 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                     if ((uint32_t)o < S && row >= o * kTileM / (int)S) owner = o;
                 const int own_lo = owner * kTileM / (int)S;
                 cluster_wait();                                 // every peer is running, its barriers initialised
+                if (group == 0 && et == 0) {                    // what the peers will send me: their partials of my rows
+                    const int mine = (int)(crank + 1) * kTileM / (int)S - (int)crank * kTileM / (int)S;
+                    mbar_arrive_expect_tx(bar(&ctrl->part_full), (S - 1) * (uint32_t)(mine * R * 4));
+                }
                 if ((uint32_t)owner != crank) {
                     const uint32_t slot = crank < (uint32_t)owner ? crank : crank - 1;      // my slot at the owner
                     const uint32_t dst = map_to_cta(recv, (uint32_t)owner) + slot * (uint32_t)(rows_max * R * 4);
+                    const uint32_t pb = map_to_cta(bar(&ctrl->part_full), (uint32_t)owner); // counts the bytes it receives
 #pragma unroll
                     for (int c4 = 0; c4 < RH / 4; ++c4)
-                        st_cluster_u32x4(dst + (uint32_t)((col0 / 4 + c4) * rows_max + (row - own_lo)) * 16u, tv[4 * c4],
-                                         tv[4 * c4 + 1], tv[4 * c4 + 2], tv[4 * c4 + 3]);
+                        st_async_cluster_u32x4(dst + (uint32_t)((col0 / 4 + c4) * rows_max + (row - own_lo)) * 16u, tv[4 * c4],
+                                               tv[4 * c4 + 1], tv[4 * c4 + 2], tv[4 * c4 + 3], pb);
                 }
-                __syncwarp();                                   // the warp's rows are sent; lane q2 tells CTA q2
-                if ((uint32_t)lane < S) mbar_arrive_remote(map_to_cta(bar(&ctrl->part_full), (uint32_t)lane));
                 wait_bar_cluster(bar(&ctrl->part_full), 0, abort_flag, prm.dev_status);
                 if ((uint32_t)owner == crank) {
                     sum_partials<RH>(tv, recv_p + (col0 / 4) * rows_max + (row - own_lo), rows_max, rows_max * R / 4, S, crank);

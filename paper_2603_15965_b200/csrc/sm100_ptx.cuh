@@ -79,6 +79,15 @@ __device__ __forceinline__ void st_cluster_u32x4(uint32_t cluster_addr, uint32_t
 {
     asm volatile("st.shared::cluster.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(cluster_addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
+// Asynchronous 16-byte store into a cluster peer's shared memory; its bytes are counted on the PEER's mbarrier `bar_cluster`
+// (the issuing warp does not wait for the store, unlike st.shared::cluster).
+__device__ __forceinline__ void st_async_cluster_u32x4(uint32_t cluster_addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d,
+                                                       uint32_t bar_cluster)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1,%2,%3,%4}, [%5];" ::"r"(cluster_addr),
+                 "r"(a), "r"(b), "r"(c), "r"(d), "r"(bar_cluster)
+                 : "memory");
+}
 // Address of the same shared-memory location in the CTA of rank `rank` of this cluster.
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
 {
