@@ -28,6 +28,16 @@ KERNEL_MODES = {
     "twophase": {"umma_min_tokens": 1000000, "small_path": 2},
     # the job-list kernel (decode-sized calls, at most 1024 tokens; larger calls fall back to the default small kernel)
     "jobs": {"umma_min_tokens": 1000000, "small_path": 3},
+    # the tcgen05 kernel for every call, with the split its model picks or a forced cluster size / tile height (rank 64
+    # splits a tile over up to 8 CTAs; the launcher lowers a split that would leave a CTA fewer than four chunks of d_in)
+    "tcgen05-all": {"umma_min_tokens": 1},
+    "tcgen05-s2": {"umma_min_tokens": 1, "umma_split": 2},
+    "tcgen05-s3": {"umma_min_tokens": 1, "umma_split": 3},
+    "tcgen05-s4": {"umma_min_tokens": 1, "umma_split": 4},
+    "tcgen05-s5": {"umma_min_tokens": 1, "umma_split": 5},
+    "tcgen05-s6r64": {"umma_min_tokens": 1, "umma_split": 6, "umma_tile_rows": 64},
+    "tcgen05-s7r96": {"umma_min_tokens": 1, "umma_split": 7, "umma_tile_rows": 96},
+    "tcgen05-s8": {"umma_min_tokens": 1, "umma_split": 8},
 }
 
 
@@ -648,6 +658,24 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode):
     assert np.all(err[keep] <= bound[keep]), f"top-{k} weighted apply: worst ratio {(err / bound)[keep].max():.3f}"
 
 
+@pytest.mark.parametrize("mode", ["tcgen05-s2", "tcgen05-s3", "tcgen05-s4", "tcgen05-s5", "tcgen05-s6r64", "tcgen05-s7r96", "tcgen05-s8"])
+@pytest.mark.parametrize("N,C,d_in,d_out,rank", [(900, 6, 2048, 1024, 64), (130, 2, 4096, 256, 64), (2100, 11, 2048, 320, 32),
+                                                 (1000, 5, 1024, 512, 16)])
+def test_tcgen05_tile_split_over_a_cluster(mode, N, C, d_in, d_out, rank):
+    # split-K shrink, exchange of the partial T tiles through distributed shared memory, split-N expand: every cluster
+    # size the kernel supports (ranks 16 and 32 stop at 4 CTAs; the launcher clamps), full and partial tiles, a LoRA scale
+    force_kernel(mode)
+    w = W.random_problem(9300 + N + rank, N, C, d_in, d_out, rank, "bf16")
+    pr = w.projections[0]
+    x, y = dev_tensor(w.inputs["x"], "bf16"), dev_tensor(pr.y, "bf16")
+    counts, offsets, perm = M.molora_group(dev_tensor(w.r, "i"), C)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    M.molora_apply(x, y, dev_tensor(pr.A, "bf16"), dev_tensor(pr.B, "bf16"), offsets, perm, scale=0.5, dev_status=status)
+    assert int(status.item()) == 0
+    ref, _ = oracle.apply(w.inputs["x"], pr.y, pr.A, pr.B, w.r, scale=0.5)
+    assert_close(to_f64(y), ref, what=f"tcgen05 {mode} {d_in}->{d_out} r{rank}")
+
+
 # ------------------------------------------------------------------ grouping + apply in one call (one launch where fused)
 @pytest.mark.parametrize("N,C,shapes,mode", [
     (4096, 4, [(2048, 2048, 16)], "default"),                                   # c2's apply: fused, the largest fused size
@@ -667,6 +695,11 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode):
     (1024, 40, [(256, 192, 32)], "twophase"),                                   # ... their largest size, match_any grouping
     (1025, 4, [(256, 192, 32)], "twophase"),                                    # one token too many: grouping launch + 2
     (300, 7, [(4096, 512, 64)], "default"), (77, 3, [(512, 4096, 64), (512, 512, 64)], "default"),   # rank 64: two-launch, on chip
+    # the tcgen05 kernel with the grouping inside (at most 4096 tokens and 64 adapters): one launch
+    (1024, 8, [(2048, 512, 64)], "tcgen05-s8"), (700, 5, [(2048, 768, 64), (2048, 256, 64)], "tcgen05-s5"),
+    (4096, 9, [(2048, 256, 64)], "tcgen05-s7r96"), (1300, 4, [(4096, 4096, 64)], "default"),
+    (2000, 33, [(256, 256, 16), (256, 512, 16)], "tcgen05-all"), (1500, 3, [(1024, 256, 32)], "tcgen05-s4"),
+    (33, 70, [(256, 256, 64)], "tcgen05-all"), (4097, 4, [(256, 256, 64)], "tcgen05-all"),          # not eligible: two launches
 ])
 def test_group_apply_one_call_matches_oracle_and_group(N, C, shapes, mode):
     force_kernel(mode)
