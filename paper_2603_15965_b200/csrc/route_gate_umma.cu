@@ -45,7 +45,7 @@ struct GateUmmaParams {
 };
 
 struct GateCtrl {
-    uint64_t full[kGuStages], empty[kGuStages], done;
+    uint64_t full[kGuStages], empty[kGuStages], done, parts;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(kGuThreads, 1) route_gate_umma_kernel(const __
             mbar_init(bar(&ctrl->empty[s]), 1);
         }
         mbar_init(bar(&ctrl->done), 1);
+        mbar_init(bar(&ctrl->parts), 1);       // rank 0: the peers' partial logits arrive as asynchronous stores counted in bytes
         ctrl->abort_flag = 0;
         fence_mbar_init();
     }
@@ -90,7 +91,8 @@ __global__ void __launch_bounds__(kGuThreads, 1) route_gate_umma_kernel(const __
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (S > 1) cluster_sync_all();                        // every CTA of the cluster is running before anyone writes to a peer
+    // "I am running and my barriers are initialised": the matching wait comes right before the first store into a peer
+    if (S > 1) cluster_arrive_relaxed();
     const uint32_t tmem = ctrl->tmem_base;
 
     if (warp == 0) {
@@ -147,21 +149,38 @@ __global__ void __launch_bounds__(kGuThreads, 1) route_gate_umma_kernel(const __
 #pragma unroll
         for (int c16 = 0; c16 < NP / 16; ++c16) tmem_ld_x16(tmem + ((uint32_t)(q * 32) << 16) + c16 * 16, v + c16 * 16);
         tmem_wait_ld();
-        if (crank != 0) {            // push my partial logits into rank 0's shared memory, slot crank - 1
-            const uint32_t dst = map_to_cta(smem_u32(partials + (size_t)(crank - 1) * NP * 128 + row), 0);
+        if (S > 1) {
+            cluster_wait();          // every CTA of the cluster is running
+            if (crank != 0) {
+                // push my partial logits into rank 0's shared memory, slot crank - 1, as [NP / 4][128] 16-byte pieces; the
+                // stores are asynchronous and count their bytes on rank 0's barrier (a warp's plain stores into a peer's
+                // memory complete one after the other, ~0.14 us each)
+                const uint32_t dst = map_to_cta(smem_u32(partials + (size_t)(crank - 1) * NP * 128) + (uint32_t)row * 16u, 0);
+                const uint32_t pb = map_to_cta(bar(&ctrl->parts), 0);
 #pragma unroll
-            for (int c = 0; c < NP; ++c) st_cluster_f32(dst + (uint32_t)c * 128u * 4u, __uint_as_float(v[c]));
+                for (int c4 = 0; c4 < NP / 4; ++c4)
+                    st_async_cluster_u32x4(dst + (uint32_t)c4 * 128u * 16u, v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3], pb);
+            } else {
+                if (warp == 2 && lane == 0) mbar_arrive_expect_tx(bar(&ctrl->parts), (S - 1) * (uint32_t)(NP * 128 * 4));
+                wait_bar_cluster(bar(&ctrl->parts), 0, abort_flag, prm.dev_status);
+            }
         }
     }
-    if (S > 1) cluster_sync_all();
     if (epi && crank == 0) {
         const int64_t i = tok0 + row;
         if (i < prm.N && *abort_flag) prm.r_out[i] = -1;                // a wait ran out: the tile's tokens stay unrouted
         if (i < prm.N && !*abort_flag) {
-            for (uint32_t p2 = 1; p2 < S; ++p2)                         // rank order
+            for (uint32_t p2 = 1; p2 < S; ++p2) {                       // rank order
+                const float4* src = reinterpret_cast<const float4*>(partials + (size_t)(p2 - 1) * NP * 128) + row;
 #pragma unroll
-                for (int c = 0; c < NP; ++c)
-                    v[c] = __float_as_uint(__uint_as_float(v[c]) + partials[((size_t)(p2 - 1) * NP + c) * 128 + row]);
+                for (int c4 = 0; c4 < NP / 4; ++c4) {
+                    const float4 pv = src[c4 * 128];
+                    v[4 * c4] = __float_as_uint(__uint_as_float(v[4 * c4]) + pv.x);
+                    v[4 * c4 + 1] = __float_as_uint(__uint_as_float(v[4 * c4 + 1]) + pv.y);
+                    v[4 * c4 + 2] = __float_as_uint(__uint_as_float(v[4 * c4 + 2]) + pv.z);
+                    v[4 * c4 + 3] = __float_as_uint(__uint_as_float(v[4 * c4 + 3]) + pv.w);
+                }
+            }
             float best = 0.f;
             int arg = 0;
 #pragma unroll
@@ -179,6 +198,12 @@ __global__ void __launch_bounds__(kGuThreads, 1) route_gate_umma_kernel(const __
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, 128);
+    if (S > 1) {
+        // the warps that took no part in the exchange complete the start-up barrier; then one closing barrier keeps rank 0
+        // alive until every peer's stores have been issued and the peers until rank 0 has taken them
+        if (!epi) cluster_wait();
+        cluster_sync_all();
+    }
 }
 
 template <int CP>
