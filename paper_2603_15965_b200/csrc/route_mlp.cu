@@ -9,7 +9,9 @@
 // products are exact in fp32 and the epilogue adds (lo + mid) + hi, so the pre-activations have the accuracy of an
 // fp32 FMA chain.  The epilogue (one thread per token) walks the hidden units in slices of 16 TMEM columns: bias,
 // exact GELU 0.5 t (1 + erf(t / sqrt 2)), and the second layer as FMAs against W2 held in shared memory; then the
-// output bias and the argmax.  The hidden activations never leave the SM.
+// output bias and the argmax.  The hidden activations never leave the SM.  Calls with few tiles split the input
+// dimension of a tile over a cluster of 2 or 4 CTAs (see SPLIT below): measured on B200, graph replay, both launches,
+// 4096 tokens 2048 -> 64 -> 4: 25.8 -> 17.8 us; 2560 -> 128 -> 4: 47.6 -> 29.8 us; 256 tokens: 23.5 -> 16.0 us.
 //
 // Other inputs (fp32 activations, d not a multiple of 64, H not a multiple of 16) take a CUDA-core kernel: one warp
 // per token, lanes split d, HP partial pre-activations per lane, butterfly sums, GELU and the second layer in lanes.
@@ -46,21 +48,36 @@ struct MlpParams {
 };
 
 struct MlpCtrl {
-    uint64_t full[6], empty[6], done;
+    uint64_t full[6], empty[6], done, parts;
     uint32_t tmem_base;
     int abort_flag;
 };
 
 __device__ __forceinline__ float gelu_exact(float t) { return 0.5f * t * (1.f + erff(t * 0.70710678118654752f)); }
 
-// HP: padded hidden width, 64 or 128
-template <int HP>
+// HP: padded hidden width, 64 or 128.
+// SPLIT: the input dimension of a 128-token tile is split over a cluster of S = 2 or 4 CTAs (calls with so few tiles that
+// the chunks a CTA walks, ~0.7 us each, set the time).  Every CTA accumulates its slice of d, turns the three terms into
+// partial pre-activations (lo + mid) + hi, and sends the rows [128 o / S, 128 (o + 1) / S) to CTA o (asynchronous stores
+// that count their bytes on o's barrier; its own rows go into its own slot); CTA o sums the S partials in rank order and
+// finishes its 128 / S tokens -- bias, GELU, second layer, argmax -- with all four epilogue warps, each a slice of the
+// hidden units.
+template <int HP, bool SPLIT>
+struct MlpCfg {
+    static constexpr int NP = 3 * HP;
+    static constexpr int STAGE = kMlpTileBytes + NP * 128;
+    static constexpr int STAGES = SPLIT ? (HP == 64 ? 4 : 2) : (HP == 64 ? 5 : 3);
+    static constexpr int RECV = SPLIT ? 128 * HP * 4 : 0;            // [S slots][HP / 4][128 / S tokens] float4
+    static constexpr int SMEM = 1024 + STAGES * STAGE + 256 + (HP * kMlpMaxC + HP) * 4 + RECV;
+};
+
+template <int HP, bool SPLIT>
 __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __grid_constant__ MlpParams prm)
 {
+    using Cfg = MlpCfg<HP, SPLIT>;
     constexpr int NP = 3 * HP;                      // accumulator columns: three term blocks of HP hidden units
-    constexpr int WBYTES = NP * 128;                // W1 image of one chunk
-    constexpr int STAGE = kMlpTileBytes + WBYTES;
-    constexpr int STAGES = HP == 64 ? 5 : 3;
+    constexpr int STAGE = Cfg::STAGE;
+    constexpr int STAGES = Cfg::STAGES;
     constexpr int NMMA = NP / 192;                  // MMAs of N = 192 per k step
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -68,13 +85,16 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
     MlpCtrl* ctrl = reinterpret_cast<MlpCtrl*>(smem_raw + (base + STAGES * STAGE - raw));
     float* w2s = reinterpret_cast<float*>(smem_raw + (base + STAGES * STAGE + 256 - raw));   // [HP][C], then b1[HP]
     float* b1s = w2s + HP * kMlpMaxC;
+    float4* recv = reinterpret_cast<float4*>(b1s + HP);                                       // SPLIT only
+    const uint32_t S = SPLIT ? cluster_nctarank() : 1u, crank = SPLIT ? cluster_ctarank() : 0u;
     volatile int* abort_flag = &ctrl->abort_flag;
     auto stage = [&](int s) { return base + (uint32_t)s * STAGE; };
     auto bar = [&](const uint64_t* b) { return smem_u32(b); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int chunks = prm.d / 64;
-    const int64_t tok0 = (int64_t)blockIdx.x * 128;
+    const int all_chunks = prm.d / 64;
+    const int kc0 = (int)(crank * all_chunks / S), kc1 = (int)((crank + 1) * all_chunks / S);   // my slice of d
+    const int64_t tok0 = (int64_t)(blockIdx.x / S) * 128;
 
     if (tid == 0) {
         prefetch_tensormap(&prm.tm_x);
@@ -84,6 +104,7 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
             mbar_init(bar(&ctrl->empty[s]), 1);
         }
         mbar_init(bar(&ctrl->done), 1);
+        mbar_init(bar(&ctrl->parts), 1);        // SPLIT: the peers' partial rows arrive as asynchronous stores counted in bytes
         ctrl->abort_flag = 0;
         fence_mbar_init();
     }
@@ -100,6 +121,8 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // "I am running and my barriers are initialised": the matching wait comes right before the first store into a peer
+    if (SPLIT) cluster_arrive_relaxed();
     const uint32_t tmem = ctrl->tmem_base;
 
     if (warp == 0) {
@@ -107,7 +130,7 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
             int s = 0;
             uint32_t ph = 1;
             bool images_ready = false;
-            for (int kc = 0; kc < chunks; ++kc) {
+            for (int kc = kc0; kc < kc1; ++kc) {
                 wait_bar(bar(&ctrl->empty[s]), ph, abort_flag, prm.dev_status);
                 if (*abort_flag) break;
                 const uint32_t fb = bar(&ctrl->full[s]);
@@ -130,7 +153,7 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
             constexpr uint32_t kL128 = swizzle_layout_type(Swizzle::B128);
             int s = 0;
             uint32_t ph = 0;
-            for (int kc = 0; kc < chunks; ++kc) {
+            for (int kc = kc0; kc < kc1; ++kc) {
                 wait_bar(bar(&ctrl->full[s]), ph, abort_flag, prm.dev_status);
                 tc_fence_after();
                 if (!*abort_flag) {
@@ -140,7 +163,7 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
 #pragma unroll
                         for (int h2 = 0; h2 < NMMA; ++h2)
                             umma_bf16(tmem + 192u * h2, smem_desc(a0 + j * 32, 16, 1024, kL128),
-                                      smem_desc(b0 + h2 * 192 * 128 + j * 32, 16, 1024, kL128), idesc, kc > 0 || j > 0);
+                                      smem_desc(b0 + h2 * 192 * 128 + j * 32, 16, 1024, kL128), idesc, kc > kc0 || j > 0);
                     umma_commit(bar(&ctrl->empty[s]));
                 }
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -158,6 +181,88 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
         float z[kMlpMaxC];
 #pragma unroll
         for (int c = 0; c < kMlpMaxC; ++c) z[c] = 0.f;
+        if constexpr (SPLIT) {
+            const int et = tid - 64;                               // 0..127 among the epilogue threads
+            const int RO = 128 / (int)S;                           // tokens a CTA finishes
+            const int owner = row / RO, tl = row - owner * RO;
+            const int nj16 = (prm.H + 15) / 16;
+            cluster_wait();                                        // every CTA of the cluster is running
+            if (et == 0) mbar_arrive_expect_tx(bar(&ctrl->parts), (S - 1) * (uint32_t)(RO * nj16 * 16 * 4));
+            {
+                // my partial pre-activations, 16 hidden units at a time, to the slot `crank` of the row's owner
+                const uint32_t slot = smem_u32(recv) + crank * (uint32_t)(RO * HP * 4);
+                const uint32_t dst0 = (uint32_t)owner == crank ? slot : map_to_cta(slot, (uint32_t)owner);
+                const uint32_t pb = map_to_cta(bar(&ctrl->parts), (uint32_t)owner);
+                for (int j16 = 0; j16 < nj16; ++j16) {
+                    uint32_t hi[16], mid[16], lo[16];
+                    tmem_ld_x16(tmem + lane_addr + j16 * 16, hi);
+                    tmem_ld_x16(tmem + lane_addr + HP + j16 * 16, mid);
+                    tmem_ld_x16(tmem + lane_addr + 2 * HP + j16 * 16, lo);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e4 = 0; e4 < 4; ++e4) {
+                        uint32_t pv[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            pv[e] = __float_as_uint((__uint_as_float(lo[4 * e4 + e]) + __uint_as_float(mid[4 * e4 + e])) +
+                                                    __uint_as_float(hi[4 * e4 + e]));
+                        const uint32_t a = dst0 + (uint32_t)((j16 * 4 + e4) * RO + tl) * 16u;
+                        if ((uint32_t)owner == crank)
+                            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(pv[0]), "r"(pv[1]), "r"(pv[2]), "r"(pv[3]) : "memory");
+                        else
+                            st_async_cluster_u32x4(a, pv[0], pv[1], pv[2], pv[3], pb);
+                    }
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");         // my CTA's own rows are in its slot
+            wait_bar_cluster(bar(&ctrl->parts), 0, abort_flag, prm.dev_status);   // ... and the peers' partials of them
+            // finish my RO tokens: thread (token tl2, part) takes a slice of the hidden units
+            const int parts = 128 / RO, tl2 = et % RO, part = et / RO;
+            const int hp = HP / parts;                             // hidden units per thread: 16 ... 64
+            for (int j4 = part * hp / 4; j4 < (part + 1) * hp / 4; ++j4) {
+                if (j4 * 4 >= nj16 * 16) break;
+                float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (uint32_t r2 = 0; r2 < S; ++r2) {                                   // rank order
+                    const float4 v = recv[(size_t)r2 * (RO * HP / 4) + (size_t)j4 * RO + tl2];
+                    t.x += v.x;
+                    t.y += v.y;
+                    t.z += v.z;
+                    t.w += v.w;
+                }
+                const float tt[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int j = j4 * 4 + e;
+                    const float h = gelu_exact(tt[e] + b1s[j]);
+                    const float* w2 = w2s + j * kMlpMaxC;
+#pragma unroll
+                    for (int c = 0; c < kMlpMaxC; ++c)
+                        if (c < prm.C) z[c] = fmaf(h, w2[c], z[c]);
+                }
+            }
+            // the parts of a token meet in the (now idle) ring: [part][token][adapter]
+            float* zbuf = reinterpret_cast<float*>(smem_raw + (base - raw));
+#pragma unroll
+            for (int c = 0; c < kMlpMaxC; ++c)
+                if (c < prm.C) zbuf[(part * RO + tl2) * kMlpMaxC + c] = z[c];
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (part == 0) {
+                const int64_t i = tok0 + (int64_t)crank * RO + tl2;
+                if (i < prm.N && *abort_flag) prm.r_out[i] = -1;        // a wait ran out: the tile's tokens stay unrouted
+                if (i < prm.N && !*abort_flag) {
+                    float best = 0.f;
+                    int arg = 0;
+                    for (int c = 0; c < prm.C; ++c) {
+                        float v = 0.f;
+                        for (int p2 = 0; p2 < parts; ++p2) v += zbuf[(p2 * RO + tl2) * kMlpMaxC + c];
+                        if (prm.b2 != nullptr) v += __ldg(prm.b2 + c);
+                        if (prm.logits_out != nullptr) prm.logits_out[i * prm.C + c] = v;
+                        if (c == 0 || v > best) { best = v; arg = c; }   // strict '>' keeps the lowest index on ties
+                    }
+                    prm.r_out[i] = arg;
+                }
+            }
+        } else {
         for (int j16 = 0; j16 < HP / 16; ++j16) {
             if (j16 * 16 >= prm.H) break;
             uint32_t hi[16], mid[16], lo[16];
@@ -192,10 +297,17 @@ __global__ void __launch_bounds__(kMlpThreads, 1) route_mlp_umma_kernel(const __
             }
             prm.r_out[i] = arg;
         }
+        }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, 512);
+    if constexpr (SPLIT) {
+        // the warps that took no part in the exchange complete the start-up barrier; one closing barrier keeps every CTA
+        // alive until the stores addressed to it have been issued and taken
+        if (warp < 2) cluster_wait();
+        cluster_sync_all();
+    }
 }
 
 // ------------------------------------------------------------------------------------------------ CUDA-core kernel
@@ -267,15 +379,21 @@ static molora_status_t mlp_umma_launch(const void* x, int64_t N, int d, int64_t 
                                        uint32_t* dev_status, cudaStream_t s)
 {
     constexpr int NP = 3 * HP;
-    constexpr int STAGES = HP == 64 ? 5 : 3;
-    constexpr int SMEM = 1024 + STAGES * (kMlpTileBytes + NP * 128) + 256 + (HP * kMlpMaxC + HP) * 4;
     static bool configured_dev[kMaxDevices] = {};
     bool& configured = configured_dev[device_slot()];
     if (!configured) {
-        if (cudaFuncSetAttribute(route_mlp_umma_kernel<HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess)
+        if (cudaFuncSetAttribute(route_mlp_umma_kernel<HP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 MlpCfg<HP, false>::SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(route_mlp_umma_kernel<HP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 MlpCfg<HP, true>::SMEM) != cudaSuccess)
             return MOLORA_ERR_CUDA;
         configured = true;
     }
+    // CTAs per 128-token tile (split along d) while the tiles alone leave most SMs idle; at least four chunks each
+    const int64_t tiles = ceil_div64(N, 128);
+    unsigned split = 1;
+    if (tiles * 4 <= 148 && d / 64 / 4 >= 4) split = 4;
+    else if (tiles * 2 <= 148 && d / 64 / 2 >= 4) split = 2;
     __nv_bfloat16* img = static_cast<__nv_bfloat16*>(ws);
     MlpParams prm;
     if (!make_tensor_map_bf16_2d(&prm.tm_x, x, (uint64_t)d, (uint64_t)N, (uint64_t)ldx, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -295,8 +413,11 @@ static molora_status_t mlp_umma_launch(const void* x, int64_t N, int d, int64_t 
     if (launch_kernel(gate_umma_split_kernel<HP>, dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)), dim3(256),
                       0, s, 1, false, W1, d, H, img) != cudaSuccess)
         return MOLORA_ERR_CUDA;
-    return cuda_ok(launch_kernel(route_mlp_umma_kernel<HP>, dim3((unsigned)ceil_div64(N, 128)), dim3(kMlpThreads), SMEM, s, 1,
-                                 true, prm));
+    if (split > 1)
+        return cuda_ok(launch_kernel(route_mlp_umma_kernel<HP, true>, dim3((unsigned)tiles * split), dim3(kMlpThreads),
+                                     MlpCfg<HP, true>::SMEM, s, split, true, prm));
+    return cuda_ok(launch_kernel(route_mlp_umma_kernel<HP, false>, dim3((unsigned)tiles), dim3(kMlpThreads),
+                                 MlpCfg<HP, false>::SMEM, s, 1, true, prm));
 }
 
 template <typename T>

@@ -560,10 +560,12 @@ def test_batched_apply_mixed_ranks_and_paths(N, mode):
 
 
 # ------------------------------------------------------------------ the paper's MLP router (Eq. 9)
-@pytest.mark.parametrize("dtype,N,d,H,C", [("bf16", 4096, 2048, 64, 4),      # c2-sized, Eq. 9's hidden width
-                                           ("bf16", 1000, 2560, 128, 4),     # the 2560 -> 128 -> 4 variant, ragged tile
-                                           ("bf16", 300, 512, 48, 9),        # hidden width below the padded 64
+@pytest.mark.parametrize("dtype,N,d,H,C", [("bf16", 4096, 2048, 64, 4),      # c2-sized, Eq. 9's hidden width; d split over clusters of 4
+                                           ("bf16", 1000, 2560, 128, 4),     # the 2560 -> 128 -> 4 variant, ragged tile, clusters of 4
+                                           ("bf16", 300, 512, 48, 9),        # hidden width below the padded 64, clusters of 2
                                            ("bf16", 128, 64, 100, 32),       # one chunk, hidden width below 128
+                                           ("bf16", 5000, 1024, 64, 7),      # 40 tiles: d split over clusters of 2
+                                           ("bf16", 20000, 512, 64, 4),      # more tiles than SMs: no split
                                            ("bf16", 50, 2048, 64, 4),        # small call: CUDA-core kernel
                                            ("bf16", 700, 72, 16, 3),         # d not a multiple of 64
                                            ("f32", 200, 264, 64, 5)])
