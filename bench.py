@@ -43,7 +43,7 @@ SUB_CONFIGS = ("c2", "c3", "c5", "c5-iid")
 NCU_TRAFFIC = {
     "c2": (34.17e6, "profiles/apply_stream_c2_full.md"),
     "c3": (26.81e6, "profiles/apply_stream_c3_full.md"),
-    "c4": (1777e6, "profiles/apply_umma_c4_full.md (a 2048-token capture scaled to 8192 tokens: the per-token part x 4, the weights once)"),
+    "c4": (1875e6, "profiles/apply_umma_c4_full.md (dram__bytes_read + write of one launch at full size, a one-pass capture)"),
     "c5": (615.4e6, "profiles/apply_umma_c5_full.md"),
     "c5-iid": (615.4e6, "profiles/apply_umma_c5_full.md (the c5 capture: same bytes, another routing)"),
 }
