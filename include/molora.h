@@ -143,6 +143,30 @@ molora_status_t molora_route_mlp(const void *x, molora_dtype_t xdt, int64_t N, i
                                  float *logits_out, void *ws, size_t ws_bytes, uint32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * The same two routers with the weight images built ONCE.  Router weights are static while a model is served; the
+ * tensor-core routers (bf16 x; the gate with C > 4, the MLP with d a multiple of 64) spend a preparation launch per call on
+ * the three-term split of G / W1.  molora_route_*_prepare runs that launch alone and leaves the images in `ws`;
+ * molora_route_*_prepared routes with them: same arguments, results and errors as molora_route_gate / molora_route_mlp,
+ * bit-identical decisions and logits, one launch fewer.  The caller keeps `ws` unchanged between the two and calls
+ * prepare again (on the same stream, or otherwise ordered) whenever G / W1 change; the library cannot tell.
+ *   gate: ws of at least molora_route_gate_prepared_workspace_bytes(xdt, d, C) bytes, 256-byte aligned (it holds the
+ *         images of both tensor-core gates, since the token count decides which one runs; 0: nothing to prepare)
+ *   MLP:  ws as for molora_route_mlp (molora_route_mlp_workspace_bytes), 16-byte aligned */
+size_t molora_route_gate_prepared_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
+molora_status_t molora_route_gate_prepare(molora_dtype_t xdt, int32_t d, int32_t C, const float *G, void *ws,
+                                          size_t ws_bytes, void *stream);
+molora_status_t molora_route_gate_prepared(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx,
+                                           const float *G, const float *bias, int32_t C, int32_t *r_out,
+                                           float *logits_out, const void *ws, size_t ws_bytes, uint32_t *dev_status,
+                                           void *stream);
+molora_status_t molora_route_mlp_prepare(molora_dtype_t xdt, int32_t d, int32_t H, int32_t C, const float *W1, void *ws,
+                                         size_t ws_bytes, void *stream);
+molora_status_t molora_route_mlp_prepared(const void *x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx,
+                                          const float *W1, const float *b1, int32_t H, const float *W2, const float *b2,
+                                          int32_t C, int32_t *r_out, float *logits_out, const void *ws, size_t ws_bytes,
+                                          uint32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * The same gate for callers that cannot provide a workspace.  (The paper has no counterpart: this entry point
  * exists for integration reasons only.)  Some hosts of this library may not allocate device memory at the
  * point where they route tokens -- code running between the capture and replay of a fixed-address serving

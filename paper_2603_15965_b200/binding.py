@@ -96,6 +96,12 @@ def load_library():
     lib.molora_route_gate_workspace_bytes.restype = sz
     lib.molora_route_gate_workspace_bytes.argtypes = [ctypes.c_int, i32, i32]
     lib.molora_route_gate.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp, vp]
+    lib.molora_route_gate_prepared_workspace_bytes.restype = sz
+    lib.molora_route_gate_prepared_workspace_bytes.argtypes = [ctypes.c_int, i32, i32]
+    lib.molora_route_gate_prepare.argtypes = [ctypes.c_int, i32, i32, vp, vp, sz, vp]
+    lib.molora_route_gate_prepared.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp, sz, vp, vp]
+    lib.molora_route_mlp_prepare.argtypes = [ctypes.c_int, i32, i32, i32, vp, vp, sz, vp]
+    lib.molora_route_mlp_prepared.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, i32, vp, vp, vp, sz, vp, vp]
     lib.molora_route_gate_noalloc.argtypes = [vp, ctypes.c_int, i64, i32, i64, vp, vp, i32, vp, vp, vp]
     lib.molora_route_gate_noalloc.restype = ctypes.c_int
     lib.molora_selftest_bounded_wait.argtypes = [vp, i64, vp, vp]
@@ -241,8 +247,9 @@ def molora_route_mlp_workspace_bytes(xdt: int, d: int, H: int, C: int) -> int:
 def molora_route_mlp(x: torch.Tensor, W1: torch.Tensor, b1: Optional[torch.Tensor], W2: torch.Tensor,
                      b2: Optional[torch.Tensor], r_out: Optional[torch.Tensor] = None,
                      logits_out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
-                     dev_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """r_out[i] = argmax_c (W2 GELU(W1 x_i + b1) + b2)[c] (Eq. 9, top-1); W1 [d, H], W2 [H, C] fp32."""
+                     dev_status: Optional[torch.Tensor] = None, stream=None, prepared: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """r_out[i] = argmax_c (W2 GELU(W1 x_i + b1) + b2)[c] (Eq. 9, top-1); W1 [d, H], W2 [H, C] fp32.
+    ``prepared``: the workspace molora_route_mlp_prepare returned for this W1 (saves the preparation launch)."""
     lib = load_library()
     N, d, ldx = _matrix(x, "x")
     if W1.dtype != torch.float32 or W2.dtype != torch.float32 or not W1.is_contiguous() or not W2.is_contiguous():
@@ -256,6 +263,11 @@ def molora_route_mlp(x: torch.Tensor, W1: torch.Tensor, b1: Optional[torch.Tenso
     if ws is None and need > 0:
         ws = torch.zeros(need, dtype=torch.uint8, device=x.device)
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    if prepared is not None:
+        _check("molora_route_mlp_prepared", lib.molora_route_mlp_prepared(
+            _ptr(x), _dtype_code(x), N, d, ldx, _ptr(W1), _ptr(b1), H, _ptr(W2), _ptr(b2), C, _ptr(_i32_dev(r_out, "r_out")),
+            _ptr(logits_out), _ptr(prepared), prepared.numel(), _ptr(dev_status), _stream(stream)))
+        return r_out
     _check("molora_route_mlp", lib.molora_route_mlp(_ptr(x), _dtype_code(x), N, d, ldx, _ptr(W1), _ptr(b1), H, _ptr(W2),
                                                     _ptr(b2), C, _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
                                                     _ptr(ws), ws_bytes, _ptr(dev_status), _stream(stream)))
@@ -269,8 +281,9 @@ def molora_route_gate_workspace_bytes(xdt: int, d: int, C: int) -> int:
 def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Tensor] = None,
                       r_out: Optional[torch.Tensor] = None, logits_out: Optional[torch.Tensor] = None,
                       ws: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
-                      stream=None) -> torch.Tensor:
-    """r_out[i] = argmax_c sum_k x[i,k] G[k,c] (+ bias[c]) (Eq. 8, k = 1); lowest index on ties."""
+                      stream=None, prepared: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """r_out[i] = argmax_c sum_k x[i,k] G[k,c] (+ bias[c]) (Eq. 8, k = 1); lowest index on ties.
+    ``prepared``: the workspace molora_route_gate_prepare returned for this G (saves the preparation launch)."""
     lib = load_library()
     N, d, ldx = _matrix(x, "x")
     if G.dtype != torch.float32 or not G.is_cuda or not G.is_contiguous() or G.dim() != 2 or G.shape[0] != d:
@@ -283,6 +296,11 @@ def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Ten
     if logits_out is not None and (logits_out.dtype != torch.float32 or logits_out.shape != (N, C)
                                    or not logits_out.is_contiguous()):
         raise ValueError("logits_out: expected contiguous fp32 [N, C]")
+    if prepared is not None:
+        _check("molora_route_gate_prepared", lib.molora_route_gate_prepared(
+            _ptr(x), _dtype_code(x), N, d, ldx, _ptr(G), _ptr(bias), C, _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out),
+            _ptr(prepared), prepared.numel(), _ptr(dev_status), _stream(stream)))
+        return r_out
     need = molora_route_gate_workspace_bytes(_dtype_code(x), d, C)
     if ws is None and need > 0:
         ws = torch.zeros(need, dtype=torch.uint8, device=x.device)
@@ -291,6 +309,39 @@ def molora_route_gate(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Ten
                                                       _ptr(_i32_dev(r_out, "r_out")), _ptr(logits_out), _ptr(ws),
                                                       ws_bytes, _ptr(dev_status), _stream(stream)))
     return r_out
+
+
+def molora_route_gate_prepare(x_dtype: torch.dtype, G: torch.Tensor, ws: Optional[torch.Tensor] = None, stream=None):
+    """Build the gate's weight images once (static router weights); returns the workspace to pass to
+    molora_route_gate(..., prepared=ws).  None when this gate needs no image (fp32 activations or at most 4 adapters)."""
+    lib = load_library()
+    if G.dtype != torch.float32 or not G.is_cuda or not G.is_contiguous() or G.dim() != 2:
+        raise ValueError("G: expected a contiguous fp32 CUDA tensor of shape [d, C]")
+    d, C = G.shape
+    xdt = BF16 if x_dtype == torch.bfloat16 else F32
+    need = int(lib.molora_route_gate_prepared_workspace_bytes(xdt, d, C))
+    if need == 0:
+        return None
+    if ws is None:
+        ws = torch.empty(need, dtype=torch.uint8, device=G.device)
+    _check("molora_route_gate_prepare", lib.molora_route_gate_prepare(xdt, d, C, _ptr(G), _ptr(ws), ws.numel(), _stream(stream)))
+    return ws
+
+
+def molora_route_mlp_prepare(x_dtype: torch.dtype, W1: torch.Tensor, C: int, ws: Optional[torch.Tensor] = None, stream=None):
+    """Build the MLP router's first-layer images once; returns the workspace for molora_route_mlp(..., prepared=ws)."""
+    lib = load_library()
+    if W1.dtype != torch.float32 or not W1.is_cuda or not W1.is_contiguous() or W1.dim() != 2:
+        raise ValueError("W1: expected a contiguous fp32 CUDA tensor of shape [d, H]")
+    d, H = W1.shape
+    xdt = BF16 if x_dtype == torch.bfloat16 else F32
+    need = molora_route_mlp_workspace_bytes(xdt, d, H, C)
+    if need == 0:
+        return None
+    if ws is None:
+        ws = torch.empty(need, dtype=torch.uint8, device=W1.device)
+    _check("molora_route_mlp_prepare", lib.molora_route_mlp_prepare(xdt, d, H, C, _ptr(W1), _ptr(ws), ws.numel(), _stream(stream)))
+    return ws
 
 
 def molora_route_gate_noalloc(x: torch.Tensor, G: torch.Tensor, bias: Optional[torch.Tensor] = None,

@@ -197,6 +197,65 @@ molora_status_t molora_route_gate(const void* x, molora_dtype_t xdt, int64_t N, 
     return launch_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+// ---- the same routers with the weight images built once (static router weights)
+size_t molora_route_gate_prepared_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
+{
+    if (d <= 0 || C < 1 || C > 32) return 0;
+    return route_gate_prepared_workspace_bytes(xdt, d, C);
+}
+
+molora_status_t molora_route_gate_prepare(molora_dtype_t xdt, int32_t d, int32_t C, const float* G, void* ws, size_t ws_bytes,
+                                          void* stream)
+{
+    if (d <= 0 || C < 1 || G == nullptr) return MOLORA_ERR_INVALID_ARG;
+    if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
+    if (C > 32 || (d % 8) != 0) return MOLORA_ERR_UNSUPPORTED;
+    const size_t need = route_gate_prepared_workspace_bytes(xdt, d, C);
+    if (need > 0 && (ws == nullptr || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) % 256) != 0)) return MOLORA_ERR_WORKSPACE;
+    return launch_route_gate(nullptr, xdt, 0, d, 0, G, nullptr, C, nullptr, nullptr, ws, nullptr, static_cast<cudaStream_t>(stream),
+                             kImageBuildOnly);
+}
+
+molora_status_t molora_route_gate_prepared(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
+                                           const float* bias, int32_t C, int32_t* r_out, float* logits_out, const void* ws,
+                                           size_t ws_bytes, uint32_t* dev_status, void* stream)
+{
+    if (N < 0 || N >= INT32_MAX || d <= 0 || C < 1) return MOLORA_ERR_INVALID_ARG;
+    if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
+    if (C > 32 || (d % 8) != 0 || (ldx % 8) != 0) return MOLORA_ERR_UNSUPPORTED;
+    if (ldx < d || G == nullptr) return MOLORA_ERR_INVALID_ARG;
+    if (N > 0 && (x == nullptr || r_out == nullptr || !aligned16(x))) return MOLORA_ERR_INVALID_ARG;
+    const size_t need = route_gate_prepared_workspace_bytes(xdt, d, C);
+    if (need > 0 && (ws == nullptr || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) % 256) != 0)) return MOLORA_ERR_WORKSPACE;
+    return launch_route_gate(x, xdt, N, d, ldx, G, bias, C, r_out, logits_out, const_cast<void*>(ws), dev_status,
+                             static_cast<cudaStream_t>(stream), kImageUseOnly);
+}
+
+molora_status_t molora_route_mlp_prepare(molora_dtype_t xdt, int32_t d, int32_t H, int32_t C, const float* W1, void* ws,
+                                         size_t ws_bytes, void* stream)
+{
+    if (d <= 0 || H < 1 || C < 1 || W1 == nullptr) return MOLORA_ERR_INVALID_ARG;
+    if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
+    if ((d % 8) != 0 || H > 128 || C > 32) return MOLORA_ERR_UNSUPPORTED;
+    return launch_route_mlp(nullptr, xdt, 0, d, 0, W1, nullptr, H, nullptr, nullptr, C, nullptr, nullptr, ws, ws_bytes, nullptr,
+                            static_cast<cudaStream_t>(stream), kImageBuildOnly);
+}
+
+molora_status_t molora_route_mlp_prepared(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
+                                          const float* b1, int32_t H, const float* W2, const float* b2, int32_t C,
+                                          int32_t* r_out, float* logits_out, const void* ws, size_t ws_bytes,
+                                          uint32_t* dev_status, void* stream)
+{
+    if (N < 0 || N >= INT32_MAX || d <= 0 || H < 1 || C < 1) return MOLORA_ERR_INVALID_ARG;
+    if (xdt != MOLORA_F32 && xdt != MOLORA_BF16) return MOLORA_ERR_UNSUPPORTED;
+    if ((d % 8) != 0 || (ldx % 8) != 0 || H > 128 || C > 32) return MOLORA_ERR_UNSUPPORTED;
+    if (ldx < d) return MOLORA_ERR_INVALID_ARG;
+    if (W1 == nullptr || W2 == nullptr || (N > 0 && (x == nullptr || r_out == nullptr))) return MOLORA_ERR_INVALID_ARG;
+    if (N > 0 && !aligned16(x)) return MOLORA_ERR_INVALID_ARG;
+    return launch_route_mlp(x, xdt, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, const_cast<void*>(ws), ws_bytes, dev_status,
+                            static_cast<cudaStream_t>(stream), kImageUseOnly);
+}
+
 size_t molora_route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H, int32_t C)
 {
     if (d <= 0 || H < 1 || H > 128 || C < 1 || C > 32) return 0;

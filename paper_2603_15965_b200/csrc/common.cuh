@@ -224,25 +224,32 @@ molora_status_t launch_route_vocab(const int32_t* ids, int64_t N, const int32_t*
 // tcgen05 gate (bf16 activations, C > 4, d a multiple of 64, at least 1024 tokens).
 bool gate_umma_eligible(int64_t N, int32_t d, int32_t C);
 size_t route_gate_umma_workspace_bytes(int32_t d, int32_t C);
+// The routers that run on tensor cores first write a three-term bf16 split of their fp32 weights into the workspace.
+// image: 0 = build it, then route (the launches are chained); 1 = build only (molora_route_*_prepare); 2 = route with an
+// image built earlier (molora_route_*_prepared: the weights are static in serving, so the preparation launch is saved).
+enum ImageMode : int { kImageBuildAndUse = 0, kImageBuildOnly = 1, kImageUseOnly = 2 };
 molora_status_t launch_route_gate_umma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
                                        const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                       uint32_t* dev_status, cudaStream_t s);
+                                       uint32_t* dev_status, cudaStream_t s, int image = kImageBuildAndUse);
 size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
 molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
                                   const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                  uint32_t* dev_status, cudaStream_t s);
+                                  uint32_t* dev_status, cudaStream_t s, int image = kImageBuildAndUse);
+// workspace of the prepared form: both tensor-core gates' images side by side (which one runs depends on N)
+size_t route_gate_prepared_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C);
 // Tensor-core (mma.sync) gate for bf16 activations; the CUDA-core kernel above serves fp32 activations.
 // Needs route_gate_mma_workspace_bytes(d, C) bytes of scratch for the split gate weights.
 size_t route_gate_mma_workspace_bytes(int32_t d, int32_t C);
 molora_status_t launch_route_gate_mma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
                                       const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                      cudaStream_t s);
+                                      cudaStream_t s, int image = kImageBuildAndUse);
 // The paper's MLP router (Eq. 9).  The tensor-core path (bf16 x, d a multiple of 64, at least 128 tokens) needs
 // route_mlp_workspace_bytes(...) bytes for the split first-layer weights.
 size_t route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H);
 molora_status_t launch_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
                                  const float* b1, int32_t H, const float* W2, const float* b2, int32_t C, int32_t* r_out,
-                                 float* logits_out, void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
+                                 float* logits_out, void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s,
+                                 int image = kImageBuildAndUse);
 // Top-k selection and softmax over router logits (Eq. 8); idx / w slot-major [k][N].
 molora_status_t launch_topk_softmax(const float* logits, int64_t N, int32_t C, int32_t k, int32_t* idx_out, float* w_out,
                                     cudaStream_t s);

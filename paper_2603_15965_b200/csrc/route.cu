@@ -578,14 +578,33 @@ size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
     return a > b ? a : b;      // which kernel runs depends on N, which this query does not know
 }
 
+size_t route_gate_prepared_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)
+{
+    if (xdt != MOLORA_BF16 || C <= 4) return 0;
+    return (route_gate_umma_workspace_bytes(d, C) + 255) / 256 * 256 + route_gate_mma_workspace_bytes(d, C);
+}
+
 molora_status_t launch_route_gate(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* G,
                                   const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                  uint32_t* dev_status, cudaStream_t s)
+                                  uint32_t* dev_status, cudaStream_t s, int image)
 {
+    // prepared form: the workspace holds the tcgen05 gate's image (if that kernel can take this d and C) and behind it
+    // the mma.sync gate's; otherwise one image at the start of the workspace, whichever kernel runs
+    const bool two = image != kImageBuildAndUse;
+    char* ws_mma = static_cast<char*>(ws) + (two ? (route_gate_umma_workspace_bytes(d, C) + 255) / 256 * 256 : 0);
+    if (image == kImageBuildOnly) {
+        if (xdt != MOLORA_BF16 || C <= 4) return MOLORA_OK;       // the CUDA-core gates read G as it is
+        if (gate_umma_eligible(1 << 20, d, C)) {
+            const molora_status_t st = launch_route_gate_umma(nullptr, 0, d, 0, G, nullptr, C, nullptr, nullptr, ws, nullptr, s, image);
+            if (st != MOLORA_OK) return st;
+        }
+        return launch_route_gate_mma(nullptr, 0, d, 0, G, nullptr, C, nullptr, nullptr, ws_mma, s, image);
+    }
     if (N == 0) return MOLORA_OK;
     if (xdt == MOLORA_BF16 && gate_umma_eligible(N, d, C))       // the only gate kernel with device-side waits
-        return launch_route_gate_umma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s);
-    if (xdt == MOLORA_BF16 && C > 4) return launch_route_gate_mma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
+        return launch_route_gate_umma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s, image);
+    if (xdt == MOLORA_BF16 && C > 4)
+        return launch_route_gate_mma(x, N, d, ldx, G, bias, C, r_out, logits_out, ws_mma, s, image);
     if (xdt == MOLORA_BF16) return gate_dispatch<__nv_bfloat16>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
     return gate_dispatch<float>(x, N, d, ldx, G, bias, C, r_out, logits_out, s);
 }

@@ -220,18 +220,22 @@ __global__ void __launch_bounds__(WARPS * 32) route_gate_mma_kernel(const __nv_b
 
 template <int NT, int WARPS, int KC>
 static molora_status_t gate_mma_launch(const void* x, int64_t N, int d, int64_t ldx, const float* G, const float* bias,
-                                       int C, int32_t* r_out, float* logits_out, void* ws, cudaStream_t s)
+                                       int C, int32_t* r_out, float* logits_out, void* ws, cudaStream_t s, int image)
 {
     __nv_bfloat16* img = static_cast<__nv_bfloat16*>(ws);
     const int chunks = (d + KC - 1) / KC;
     const int64_t elems = (int64_t)chunks * KC * NT * 8;
-    if (cudaError_t e = launch_kernel(gate_split_kernel<NT, KC>,
-                                       dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)), dim3(256), 0, s,
-                                      1, false, G, d, C, img);
-        e != cudaSuccess)
-        return MOLORA_ERR_CUDA;
+    if (image != kImageUseOnly) {
+        if (cudaError_t e = launch_kernel(gate_split_kernel<NT, KC>,
+                                          dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)), dim3(256), 0, s,
+                                          1, false, G, d, C, img);
+            e != cudaSuccess)
+            return MOLORA_ERR_CUDA;
+    }
+    if (image == kImageBuildOnly) return MOLORA_OK;
     const int64_t blocks = ceil_div64(N, 16 * WARPS);
-    return cuda_ok(launch_kernel(route_gate_mma_kernel<NT, WARPS, KC>, dim3((unsigned)blocks), dim3(WARPS * 32), 0, s, 1, true,
+    return cuda_ok(launch_kernel(route_gate_mma_kernel<NT, WARPS, KC>, dim3((unsigned)blocks), dim3(WARPS * 32), 0, s, 1,
+                                 image == kImageBuildAndUse,
                                   static_cast<const __nv_bfloat16*>(x), N, d, ldx, img, bias, C, r_out, logits_out));
 }
 
@@ -245,12 +249,12 @@ size_t route_gate_mma_workspace_bytes(int32_t d, int32_t C)
 
 molora_status_t launch_route_gate_mma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
                                       const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                      cudaStream_t s)
+                                      cudaStream_t s, int image)
 {
-    if (N == 0) return MOLORA_OK;
-    if (C <= 8) return gate_mma_launch<1, 4, 128>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
-    if (C <= 16) return gate_mma_launch<2, 4, 128>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
-    return gate_mma_launch<4, 4, 64>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s);
+    if (N == 0 && image != kImageBuildOnly) return MOLORA_OK;
+    if (C <= 8) return gate_mma_launch<1, 4, 128>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s, image);
+    if (C <= 16) return gate_mma_launch<2, 4, 128>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s, image);
+    return gate_mma_launch<4, 4, 64>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, s, image);
 }
 
 }  // namespace molora

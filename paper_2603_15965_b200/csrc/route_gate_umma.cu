@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kGuThreads, 1) route_gate_umma_kernel(const __
 template <int CP>
 static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t ldx, const float* G, const float* bias,
                                         int C, int32_t* r_out, float* logits_out, void* ws, uint32_t* dev_status,
-                                        cudaStream_t s)
+                                        cudaStream_t s, int image)
 {
     constexpr int NP = 3 * CP;
     constexpr int STAGES = CP == 16 ? kGuStages : kGuStages - 1;
@@ -227,6 +227,12 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
         configured = true;
     }
     __nv_bfloat16* img = static_cast<__nv_bfloat16*>(ws);
+    const int64_t elems = (int64_t)d * CP;
+    if (image != kImageUseOnly &&
+        launch_kernel(gate_umma_split_kernel<CP>, dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)),
+                      dim3(256), 0, s, 1, false, G, d, C, img) != cudaSuccess)
+        return MOLORA_ERR_CUDA;
+    if (image == kImageBuildOnly) return MOLORA_OK;
     GateUmmaParams prm;
     if (!make_tensor_map_bf16_2d(&prm.tm_x, x, (uint64_t)d, (uint64_t)N, (uint64_t)ldx, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_tensor_map_bf16_2d(&prm.tm_g, img, 64, (uint64_t)(d / 64) * NP, 64, 64, NP, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -238,10 +244,6 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
     prm.N = N;
     prm.d = d;
     prm.C = C;
-    const int64_t elems = (int64_t)d * CP;
-    if (launch_kernel(gate_umma_split_kernel<CP>, dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)),
-                       dim3(256), 0, s, 1, false, G, d, C, img) != cudaSuccess)
-        return MOLORA_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(tiles * split), 1, 1);
     cfg.blockDim = dim3(kGuThreads, 1, 1);
@@ -255,7 +257,7 @@ static molora_status_t gate_umma_launch(const void* x, int64_t N, int d, int64_t
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // overlap with the tail of the preparation kernel
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = chained_launch_enabled() ? 2 : 1;
+    cfg.numAttrs = (chained_launch_enabled() && image == kImageBuildAndUse) ? 2 : 1;   // chained to the preparation kernel only
     note_launch();
     return cuda_ok(cudaLaunchKernelEx(&cfg, route_gate_umma_kernel<CP>, prm));
 }
@@ -272,11 +274,11 @@ size_t route_gate_umma_workspace_bytes(int32_t d, int32_t C)
 
 molora_status_t launch_route_gate_umma(const void* x, int64_t N, int32_t d, int64_t ldx, const float* G,
                                        const float* bias, int32_t C, int32_t* r_out, float* logits_out, void* ws,
-                                       uint32_t* dev_status, cudaStream_t s)
+                                       uint32_t* dev_status, cudaStream_t s, int image)
 {
-    if (N == 0) return MOLORA_OK;
-    if (C <= 16) return gate_umma_launch<16>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s);
-    return gate_umma_launch<32>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s);
+    if (N == 0 && image != kImageBuildOnly) return MOLORA_OK;
+    if (C <= 16) return gate_umma_launch<16>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s, image);
+    return gate_umma_launch<32>(x, N, d, ldx, G, bias, C, r_out, logits_out, ws, dev_status, s, image);
 }
 
 }  // namespace molora

@@ -376,7 +376,7 @@ size_t route_mlp_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t H)
 template <int HP>
 static molora_status_t mlp_umma_launch(const void* x, int64_t N, int d, int64_t ldx, const float* W1, const float* b1, int H,
                                        const float* W2, const float* b2, int C, int32_t* r_out, float* logits_out, void* ws,
-                                       uint32_t* dev_status, cudaStream_t s)
+                                       uint32_t* dev_status, cudaStream_t s, int image)
 {
     constexpr int NP = 3 * HP;
     static bool configured_dev[kMaxDevices] = {};
@@ -395,6 +395,15 @@ static molora_status_t mlp_umma_launch(const void* x, int64_t N, int d, int64_t 
     if (tiles * 4 <= 148 && d / 64 / 4 >= 4) split = 4;
     else if (tiles * 2 <= 148 && d / 64 / 2 >= 4) split = 2;
     __nv_bfloat16* img = static_cast<__nv_bfloat16*>(ws);
+    {
+        const int64_t elems = (int64_t)d * HP;
+        if (image != kImageUseOnly &&
+            launch_kernel(gate_umma_split_kernel<HP>, dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)), dim3(256),
+                          0, s, 1, false, W1, d, H, img) != cudaSuccess)
+            return MOLORA_ERR_CUDA;
+        if (image == kImageBuildOnly) return MOLORA_OK;
+    }
+    const bool chained = image == kImageBuildAndUse;       // overlap with the tail of the preparation kernel
     MlpParams prm;
     if (!make_tensor_map_bf16_2d(&prm.tm_x, x, (uint64_t)d, (uint64_t)N, (uint64_t)ldx, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_tensor_map_bf16_2d(&prm.tm_w, img, 64, (uint64_t)(d / 64) * NP, 64, 64, 192, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -409,15 +418,11 @@ static molora_status_t mlp_umma_launch(const void* x, int64_t N, int d, int64_t 
     prm.d = d;
     prm.H = H;
     prm.C = C;
-    const int64_t elems = (int64_t)d * HP;
-    if (launch_kernel(gate_umma_split_kernel<HP>, dim3((unsigned)std::min<int64_t>(ceil_div64(elems, 256), 148 * 4)), dim3(256),
-                      0, s, 1, false, W1, d, H, img) != cudaSuccess)
-        return MOLORA_ERR_CUDA;
     if (split > 1)
         return cuda_ok(launch_kernel(route_mlp_umma_kernel<HP, true>, dim3((unsigned)tiles * split), dim3(kMlpThreads),
-                                     MlpCfg<HP, true>::SMEM, s, split, true, prm));
+                                     MlpCfg<HP, true>::SMEM, s, split, chained, prm));
     return cuda_ok(launch_kernel(route_mlp_umma_kernel<HP, false>, dim3((unsigned)tiles), dim3(kMlpThreads),
-                                 MlpCfg<HP, false>::SMEM, s, 1, true, prm));
+                                 MlpCfg<HP, false>::SMEM, s, 1, chained, prm));
 }
 
 template <typename T>
@@ -436,14 +441,15 @@ static molora_status_t mlp_simple_launch(const void* x, int64_t N, int d, int64_
 
 molora_status_t launch_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, int32_t d, int64_t ldx, const float* W1,
                                  const float* b1, int32_t H, const float* W2, const float* b2, int32_t C, int32_t* r_out,
-                                 float* logits_out, void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s)
+                                 float* logits_out, void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s, int image)
 {
-    if (N == 0) return MOLORA_OK;
-    if (mlp_umma_eligible(xdt, N, d, H)) {
+    if (N == 0 && image != kImageBuildOnly) return MOLORA_OK;
+    if (mlp_umma_eligible(xdt, image == kImageBuildOnly ? 128 : N, d, H)) {
         if (ws == nullptr || ws_bytes < route_mlp_workspace_bytes(xdt, d, H) || !aligned16(ws)) return MOLORA_ERR_WORKSPACE;
-        return H <= 64 ? mlp_umma_launch<64>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, dev_status, s)
-                       : mlp_umma_launch<128>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, dev_status, s);
+        return H <= 64 ? mlp_umma_launch<64>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, dev_status, s, image)
+                       : mlp_umma_launch<128>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, ws, dev_status, s, image);
     }
+    if (image == kImageBuildOnly) return MOLORA_OK;          // the CUDA-core router reads W1 as it is
     return xdt == MOLORA_BF16 ? mlp_simple_launch<__nv_bfloat16>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, s)
                               : mlp_simple_launch<float>(x, N, d, ldx, W1, b1, H, W2, b2, C, r_out, logits_out, s);
 }

@@ -185,6 +185,43 @@ def test_route_gate_ties_pick_lowest_index_and_unit_vectors():
     assert np.array_equal(r.cpu().numpy(), np.argmax(G, axis=1))
 
 
+@pytest.mark.parametrize("N,d,C", [(1500, 4096, 16), (300, 520, 9), (2049, 2048, 32), (700, 264, 4), (64, 2048, 8)])
+def test_route_gate_prepared_images_give_identical_results(N, d, C):
+    # static router weights: the three-term images are built once, every later call skips the preparation launch
+    rng = np.random.default_rng(N + d + C)
+    G = dev_tensor((rng.standard_normal((d, C)) * d ** -0.5).astype(np.float32), "f32")
+    bias = dev_tensor((rng.standard_normal(C) * 0.1).astype(np.float32), "f32")
+    prepared = M.molora_route_gate_prepare(torch.bfloat16, G)
+    assert (prepared is None) == (C <= 4)
+    for k in range(2):                                            # the images survive a call
+        x = dev_tensor(W.round_to_bf16(rng.standard_normal((N, d), dtype=np.float32)), "bf16")
+        l0 = torch.empty(N, C, dtype=torch.float32, device="cuda")
+        l1 = torch.empty(N, C, dtype=torch.float32, device="cuda")
+        r0 = M.molora_route_gate(x, G, bias, logits_out=l0)
+        before = M.molora_launch_count()
+        if prepared is not None:
+            r1 = M.molora_route_gate(x, G, bias, logits_out=l1, prepared=prepared)
+            assert M.molora_launch_count() - before == 1
+            assert torch.equal(r0, r1) and torch.equal(l0, l1)
+
+
+@pytest.mark.parametrize("N,d,H,C", [(4096, 2048, 64, 4), (1000, 2560, 128, 4), (20000, 512, 64, 4)])
+def test_route_mlp_prepared_images_give_identical_results(N, d, H, C):
+    rng = np.random.default_rng(N + d + H)
+    W1 = dev_tensor((rng.standard_normal((d, H)) * d ** -0.5).astype(np.float32), "f32")
+    W2 = dev_tensor((rng.standard_normal((H, C)) * H ** -0.5).astype(np.float32), "f32")
+    b1 = dev_tensor((rng.standard_normal(H) * 0.2).astype(np.float32), "f32")
+    prepared = M.molora_route_mlp_prepare(torch.bfloat16, W1, C)
+    x = dev_tensor(W.round_to_bf16(rng.standard_normal((N, d), dtype=np.float32)), "bf16")
+    l0 = torch.empty(N, C, dtype=torch.float32, device="cuda")
+    l1 = torch.empty(N, C, dtype=torch.float32, device="cuda")
+    r0 = M.molora_route_mlp(x, W1, b1, W2, None, logits_out=l0)
+    before = M.molora_launch_count()
+    r1 = M.molora_route_mlp(x, W1, b1, W2, None, logits_out=l1, prepared=prepared)
+    assert M.molora_launch_count() - before == 1
+    assert torch.equal(r0, r1) and torch.equal(l0, l1)
+
+
 # ------------------------------------------------------------------ grouping
 @pytest.mark.parametrize("N,C", [(0, 4), (1, 1), (6, 3), (31, 2), (32, 5), (33, 256), (1000, 16), (16384, 4),
                                  (40000, 64), (100003, 7)])
