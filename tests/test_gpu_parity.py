@@ -770,6 +770,35 @@ def test_group_apply_one_call_matches_oracle_and_group(N, C, shapes, mode):
         assert_close(to_f64(y), ref, what=f"group+apply {pr.d_in}->{pr.d_out} r{pr.rank}")
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_group_apply_random_calls_default_kernels(seed):
+    # whatever kernel, cluster size and tile height the library picks by itself (mid-sized rank-64 calls: the tcgen05 kernel
+    # with the grouping inside and a split chosen by its cost model): grouping outputs and every row against the oracle
+    rng = np.random.default_rng(4200 + seed)
+    rank = int(rng.choice([16, 32, 64]))
+    N = int(rng.integers(200, 5000))
+    C = int(rng.choice([2, 5, 8, 16, 40, 64]))
+    P = int(rng.integers(1, 4))
+    shapes = [(int(rng.choice([512, 1024, 2048, 4096])), int(rng.choice([256, 1024, 2048, 3072])), rank) for _ in range(P)]
+    p = rng.dirichlet(np.full(C, 0.8))
+    r = rng.choice(C, size=N, p=p).astype(np.int32)
+    r[rng.random(N) < 0.03] = -1
+    ws = [W.random_problem(4300 + 10 * seed + i, N, C, di, do, rk, "bf16", r=r) for i, (di, do, rk) in enumerate(shapes)]
+    ys = [dev_tensor(w.projections[0].y, "bf16") for w in ws]
+    projs = [M.ProjDesc(dev_tensor(w.inputs["x"], "bf16"), y, dev_tensor(w.projections[0].A, "bf16"),
+                        dev_tensor(w.projections[0].B, "bf16"), 1.0) for w, y in zip(ws, ys)]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    counts, offsets, perm = M.molora_group_apply_batched(dev_tensor(r, "i"), projs, dev_status=status)
+    assert int(status.item()) == 0
+    c_ref, o_ref, p_ref = oracle.group(r, C)
+    assert np.array_equal(counts.cpu().numpy(), c_ref) and np.array_equal(offsets.cpu().numpy(), o_ref)
+    assert np.array_equal(perm.cpu().numpy()[: o_ref[-1]], p_ref)
+    for w, y in zip(ws, ys):
+        pr = w.projections[0]
+        ref, _ = oracle.apply(w.inputs["x"], pr.y, pr.A, pr.B, r)
+        assert_close(to_f64(y), ref, what=f"random call {seed}: {pr.d_in}->{pr.d_out} r{pr.rank} N={N} C={C}")
+
+
 def test_group_apply_one_call_flags_bad_routes():
     N, C = 500, 4
     rng = np.random.default_rng(77)
