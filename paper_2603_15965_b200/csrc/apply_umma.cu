@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         prefetch_tensormap(&pj.tm_b);
         for (int s = 0; s < Cfg::kStages; ++s) {
             mbar_init(bar(&ctrl->full[s]), kProducerThreads + 1);   // every gathering thread + the weight-chunk arrival
-            mbar_init(bar(&ctrl->empty[s]), 1);
+            mbar_init(bar(&ctrl->empty[s]), 4);      // the four warps of an epilogue group; the MMA thread arrives for all four
         }
         mbar_init(bar(&ctrl->t_full), 1);
         mbar_init(bar(&ctrl->t_ready), 2 * kTileM);      // both epilogue groups
@@ -362,7 +362,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                         const uint64_t bd = smem_desc(w0 + j * (16 * Cfg::kTRowBytes), 0, 8 * Cfg::kTRowBytes, Cfg::kWLayout);
                         umma_bf16(tmem_T, ad, bd, idesc_shrink, it > 0 || j > 0);
                     }
-                    umma_commit(bar(&ctrl->empty[s]));
+                    umma_commit(bar(&ctrl->empty[s]));          // arrives when the MMAs have read the stage ...
+#pragma unroll
+                    for (int k = 0; k < 3; ++k) mbar_arrive(bar(&ctrl->empty[s]));   // ... and completes the count of four
                 }
             }
             if (!*abort_flag) umma_commit(bar(&ctrl->t_full));
@@ -518,14 +520,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             mbar_arrive(bar(&ctrl->t_ready));
         }
 
-        // copy-out mapping: piece (et & 7) of rows (et >> 3) + 16 i
-        const int piece = et & 7;
+        // Copy-out mapping: a warp finishes and stores its OWN 32 rows (the TMEM lanes it reads), so the four warps of a
+        // group never wait for one another inside a chunk: piece (lane & 7) of rows q*32 + (lane >> 3) + 4 i.
+        const int piece = lane & 7;
         int otok[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) otok[i] = ctrl->rows[(et >> 3) + 16 * i];
-        int wtok[4];                                    // 256-bit variant: rows (et >> 2) + 32 i
+        for (int i = 0; i < 8; ++i) otok[i] = ctrl->rows[q * 32 + (lane >> 3) + 4 * i];
+        int wtok[4];                                    // 256-bit variant: rows q*32 + (lane >> 2) + 8 i
 #pragma unroll
-        for (int i = 0; i < 4; ++i) wtok[i] = ctrl->rows[(et >> 2) + 32 * i];
+        for (int i = 0; i < 4; ++i) wtok[i] = ctrl->rows[q * 32 + (lane >> 2) + 8 * i];
         for (int nc = group; nc < NY; nc += kEpiGroups) {
             const int it = KX + nc;
             const int s = it % Cfg::kStages;
@@ -556,16 +559,16 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                         pack<__nv_bfloat16>(yv);
                 }
             }
-            asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
+            __syncwarp();                              // my warp's 32 rows are finished in the stage
             if (!*abort_flag) {
                 if (pj.wide_store) {
                     // 32 bytes per lane: four lanes cover a 128-byte row segment, a warp instruction eight rows
-                    const int p32 = et & 3;
+                    const int p32 = lane & 3;
                     __nv_bfloat16* dstc = pj.y + (ny0 + nc) * kChunkCols + p32 * 16;
                     uint4 lo4[4], hi4[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const uint32_t r = (uint32_t)((et >> 2) + 32 * i);
+                        const uint32_t r = (uint32_t)(q * 32 + (lane >> 2) + 8 * i);
                         lo4[i] = *reinterpret_cast<const uint4*>(ytile + swizzle_offset(r * 128u + p32 * 32, 3));
                         hi4[i] = *reinterpret_cast<const uint4*>(ytile + swizzle_offset(r * 128u + p32 * 32 + 16, 3));
                     }
@@ -578,14 +581,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         op[i] = *reinterpret_cast<const uint4*>(
-                            ytile + swizzle_offset((uint32_t)((et >> 3) + 16 * i) * 128u + piece * 16, 3));
+                            ytile + swizzle_offset((uint32_t)(q * 32 + (lane >> 3) + 4 * i) * 128u + piece * 16, 3));
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         if (otok[i] >= 0) stg128(dstc + (int64_t)otok[i] * pj.ldy, op[i]);
                 }
             }
-            asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");
-            if (et == 0) mbar_arrive(bar(&ctrl->empty[s]));   // the stage may be refilled
+            __syncwarp();                              // every lane has read its pieces
+            if (lane == 0) mbar_arrive(bar(&ctrl->empty[s]));   // one of four: the stage may be refilled when all warps are done
         }
     }
 
