@@ -364,7 +364,7 @@ def measure(name, args, env, headline):
         # latency of a single step replayed on its own (one graph per buffer set, one event pair per replay): the
         # distribution the paper reports for graph replay (median, P99, coefficient of variation)
         latency = None
-        if args.launch == "graph" and not args.profile and headline:
+        if args.launch == "graph" and not args.profile:
             singles = [capture(step, i, 1) for i in range(min(n_sets, 8))]
             n_lat = 400
             evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
@@ -610,7 +610,7 @@ def run_ours(args):
                                   "achieved_gbs": v["roofline"]["achieved"], "frac": v["roofline"]["frac"],
                                   "frac_of_spec": v["roofline"]["frac_of_spec"], "traffic": v["roofline"]["traffic"],
                                   "launches_per_step": v["launches_per_step"], "buffer_sets": v["buffer_sets"],
-                                  "passes": v["passes"], "clocks": v["clocks"],
+                                  "passes": v["passes"], "clocks": v["clocks"], "latency": v["latency"],
                                   **({"kpass_baseline": v["kpass_baseline"]} if v.get("kpass_baseline") else {})}
                               for k, v in subs.items()}
     if dist is not None:
