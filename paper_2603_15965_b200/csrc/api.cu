@@ -573,22 +573,28 @@ TopkPlan plan_topk(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_
 // B adds all k deltas before the single rounding.  Taken when every projection can run on the streaming kernel with the
 // stacked rank (bf16, r x k in {16, 32, 64}, k in {2, 4}, C^k <= 256 sets) and the call is not one the tcgen05 kernel
 // would take pass by pass.
-bool topk_single_pass(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C, int32_t k)
+// Returns 0: k passes; 1: one pass on the streaming kernel; 2: one pass on the tcgen05 kernel (adapters of rank >= 16, at
+// most 64 adapter sets, widths that are multiples of 64, and a call large enough for that kernel at the stacked rank).
+int topk_single_pass(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C, int32_t k)
 {
-    if (dt != MOLORA_BF16 || (k != 2 && k != 4) || N < 1) return false;
+    if (dt != MOLORA_BF16 || (k != 2 && k != 4) || N < 1) return 0;
     int64_t sets = 1;
     for (int j = 0; j < k; ++j) sets *= C;
-    if (sets > MOLORA_MAX_ADAPTERS) return false;
-    const int64_t small = tune(kTuneSmallPath);
-    if (small != 0 && small != 1) return false;                     // a test or a measurement asks for another kernel
+    if (sets > MOLORA_MAX_ADAPTERS) return 0;
     double bytes = 0.0;
+    bool umma_ok = sets <= kUmmaAllSegmentsMaxC && projs[0].rank >= 16;
     for (int i = 0; i < P; ++i) {
         const int stacked = projs[i].rank * k;
-        if (!stream_eligible(projs[i], dt) || (stacked != 16 && stacked != 32 && stacked != 64)) return false;
-        if (projs[i].rank != projs[0].rank) return false;
+        if (!stream_eligible(projs[i], dt) || (stacked != 16 && stacked != 32 && stacked != 64)) return 0;
+        if (projs[i].rank != projs[0].rank) return 0;
+        umma_ok = umma_ok && umma_eligible(projs[i], dt);
         bytes += proj_bytes(N, projs[i].d_in, projs[i].d_out);
     }
-    return !use_umma(projs[0].rank, N, C, bytes);
+    // (with many sets every 128-row tile is a partial one: 64 sets at 8192 tokens lost to two passes, 113 against 106 us)
+    if (umma_ok && (sets <= 16 || N >= sets * 256) && use_umma(projs[0].rank * k, N, (int32_t)sets, bytes)) return 2;
+    const int64_t small = tune(kTuneSmallPath);
+    if (small != 0 && small != 1) return 0;                         // a test or a measurement asks for another kernel
+    return use_umma(projs[0].rank, N, C, bytes) ? 0 : 1;
 }
 }  // namespace
 
@@ -611,7 +617,7 @@ molora_status_t molora_apply_topk(const molora_proj_desc_t* projs, int32_t P, mo
     int32_t* offsets = reinterpret_cast<int32_t*>(base + pl.offsets);
     int32_t* perm = reinterpret_cast<int32_t*>(base + pl.perm);
     molora_proj_desc_t pass[MOLORA_MAX_PROJECTIONS];
-    if (topk_single_pass(projs, P, dt, N, C, k)) {
+    if (const int one_pass = topk_single_pass(projs, P, dt, N, C, k)) {
         for (int i = 0; i < P; ++i) {
             const molora_status_t st = check_proj(projs[i], dt);
             if (st != MOLORA_OK) return st;
@@ -628,6 +634,13 @@ molora_status_t molora_apply_topk(const molora_proj_desc_t* projs, int32_t P, mo
         }
         molora_status_t st = launch_topk_sets(idx, w, N, C, k, sets, wsorted, s);
         if (st != MOLORA_OK) return st;
+        if (one_pass == 2) {                         // tcgen05 kernel: one MMA per part in the shrink, stacked B in the expand
+            if (group_apply_umma_eligible(N, n_sets))
+                return launch_apply_umma(pass, P, N, n_sets, offsets, perm, dev_status, 1, s, sets, counts, k, C);
+            st = molora_group(sets, N, n_sets, counts, offsets, perm, nullptr, 0, dev_status, stream);
+            if (st != MOLORA_OK) return st;
+            return launch_apply_umma(pass, P, N, n_sets, offsets, perm, dev_status, 1, s, nullptr, nullptr, k, C);
+        }
         if (group_apply_stream_eligible(N))         // the CTAs of the apply group the sets themselves
             return launch_group_apply_stream_sets(sets, pass, P, N, C, k, counts, offsets, perm, dev_status, s);
         st = molora_group(sets, N, n_sets, counts, offsets, perm, nullptr, 0, dev_status, stream);

@@ -91,8 +91,15 @@ struct UmmaParams {
     int32_t* counts_out;
     int32_t* offsets_out;
     int32_t* perm_out;
+    // Top-k routing in one pass (Eq. 8): a segment is a SET of `parts` adapters (its index spells them in base `cbase`, most
+    // significant first) and the launch's rank R is parts x the adapters' rank r.  The shrink runs one MMA per part into
+    // its own r columns of T (the part's A chunk is its own shared-memory tile), every part of a row of T is scaled by the
+    // token's weight for that part (row_scale[part * N + token]), and the expand contracts all R columns against the
+    // parts' B chunks stacked by rows -- one read of x and y, one rounding.  parts == 1: plain top-1 routing.
+    int32_t parts, cbase;
 };
 constexpr int kUmmaGroupMaxN = 4096;
+constexpr int kUmmaMaxParts = 4;
 
 
 // WIDE (rank 64 only): one ring stage fewer, which makes room for the partial rows of up to seven peers, so that a tile
@@ -269,6 +276,17 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         if (warp == kMmaWarp) tmem_dealloc(ctrl->tmem_base, kTmemCols);
         return;
     }
+    // adapters of the segment's set (one adapter when parts == 1) and the rank of each
+    const int parts = prm.parts, rp = R / parts;
+    int adapter[kUmmaMaxParts];
+    {
+        int rest = seg;
+        for (int j = parts - 1; j >= 0; --j) {
+            adapter[j] = parts == 1 ? seg : rest % prm.cbase;
+            rest /= prm.cbase;
+        }
+        for (int j = parts; j < kUmmaMaxParts; ++j) adapter[j] = 0;
+    }
     const int KXall = pj.d_in / kChunkCols, NYall = pj.d_out / kChunkCols;
     const int kx0 = (int)(crank * KXall / S), KX = (int)((crank + 1) * KXall / S) - kx0;   // my slice of d_in
     const int ny0 = (int)(crank * NYall / S), NY = (int)((crank + 1) * NYall / S) - ny0;   // my slice of d_out
@@ -336,8 +354,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 if (*abort_flag) break;
                 const uint32_t fb = bar(&ctrl->full[s]);
                 mbar_arrive_expect_tx(fb, (uint32_t)Cfg::kWBytes);
-                if (it < KX) tma_load_2d(stage(s) + kTileBytes, &pj.tm_a, 0, seg * pj.d_in + (kx0 + it) * kChunkCols, fb);
-                else tma_load_2d(stage(s) + kTileBytes, &pj.tm_b, (ny0 + it - KX) * kChunkCols, seg * R, fb);
+                // one box per part: A chunks [64, r] side by side as tiles of their own, B chunks [r, 64] stacked by rows
+                for (int j = 0; j < parts; ++j) {
+                    if (it < KX)
+                        tma_load_2d(stage(s) + kTileBytes + (uint32_t)(j * kChunkCols * rp * 2), &pj.tm_a, 0,
+                                    adapter[j] * pj.d_in + (kx0 + it) * kChunkCols, fb);
+                    else
+                        tma_load_2d(stage(s) + kTileBytes + (uint32_t)(j * rp * 128), &pj.tm_b, (ny0 + it - KX) * kChunkCols,
+                                    adapter[j] * rp, fb);
+                }
                 if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
             }
         }
@@ -345,7 +370,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     } else if (warp == kMmaWarp) {
         // ============================================================ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc_shrink = idesc_bf16_f32(kTileM, R, 0, 1);
+            const uint32_t idesc_shrink = idesc_bf16_f32(kTileM, rp, 0, 1);
+            // rows of an A chunk are r x 2 bytes: 128-, 64- or 32-byte swizzle
+            const uint32_t wlayout = swizzle_layout_type(rp == 64 ? Swizzle::B128 : rp == 32 ? Swizzle::B64 : Swizzle::B32);
+            const uint32_t wrow = (uint32_t)rp * 2u;
             constexpr uint32_t idesc_expand = idesc_bf16_f32(kTileM, kChunkCols, 0, 1);
             constexpr uint32_t kL128 = swizzle_layout_type(Swizzle::B128);
             for (int it = 0; it < KX; ++it) {
@@ -359,8 +387,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {   // four K = 16 steps per 64-column chunk
                         const uint64_t ad = smem_desc(a0 + j * 32, 16, 1024, kL128);
-                        const uint64_t bd = smem_desc(w0 + j * (16 * Cfg::kTRowBytes), 0, 8 * Cfg::kTRowBytes, Cfg::kWLayout);
-                        umma_bf16(tmem_T, ad, bd, idesc_shrink, it > 0 || j > 0);
+                        for (int pt = 0; pt < parts; ++pt) {          // part pt -> columns [pt r, (pt + 1) r) of T
+                            const uint64_t bd = smem_desc(w0 + (uint32_t)pt * kChunkCols * wrow + j * (16 * wrow), 0, 8 * wrow, wlayout);
+                            umma_bf16(tmem_T + (uint32_t)(pt * rp), ad, bd, idesc_shrink, it > 0 || j > 0);
+                        }
                     }
                     umma_commit(bar(&ctrl->empty[s]));          // arrives when the MMAs have read the stage ...
 #pragma unroll
@@ -422,15 +452,21 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
             tmem_wait_ld();
             // LoRA scale times the token's routing weight (1 unless the caller passes per-token factors)
             const int my_tok = ctrl->rows[row];
-            const float tscale = pj.scale * ((pj.row_scale != nullptr && my_tok >= 0) ? __ldg(pj.row_scale + my_tok) : 1.f);
+            float tscale[kUmmaMaxParts];
+#pragma unroll
+            for (int j = 0; j < kUmmaMaxParts; ++j)
+                tscale[j] = pj.scale * ((pj.row_scale != nullptr && my_tok >= 0 && j < parts)
+                                            ? __ldg(pj.row_scale + (int64_t)j * prm.N + my_tok) : 1.f);
             // my half row -> T_hi / T_lo of this CTA
             auto publish_local = [&]() {
 #pragma unroll
                 for (int c8 = 0; c8 < RH / 8; ++c8) {
                     float hi[8], lo[8];
+                    const int tpart = (col0 + c8 * 8) / rp;       // (r is a multiple of 16: a block of 8 columns has one part)
+                    const float ts = tpart == 0 ? tscale[0] : tpart == 1 ? tscale[1] : tpart == 2 ? tscale[2] : tscale[3];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        const float t = __uint_as_float(tv[c8 * 8 + e]) * tscale;
+                        const float t = __uint_as_float(tv[c8 * 8 + e]) * ts;
                         hi[e] = __bfloat162float(__float2bfloat16_rn(t));
                         lo[e] = t - hi[e];
                     }
@@ -798,10 +834,14 @@ bool group_apply_umma_eligible(int64_t N, int32_t C) { return N >= 1 && N <= kUm
 
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                   const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
-                                  cudaStream_t s, const int32_t* r, int32_t* counts_out)
+                                  cudaStream_t s, const int32_t* r, int32_t* counts_out, int32_t parts, int32_t cbase)
 {
     if (N == 0 || P == 0) return MOLORA_OK;
+    if (parts < 1 || parts > kUmmaMaxParts) return MOLORA_ERR_INVALID_ARG;
     UmmaParams prm;
+    prm.parts = parts;
+    prm.cbase = parts > 1 ? cbase : C;
+    const int32_t n_adapters = parts > 1 ? cbase : C;          // C counts adapter SETS when parts > 1
     // r given: the kernel groups on chip and writes counts / offsets / perm (the pointers are then outputs); one launch
     // only, so every projection must have the same rank
     prm.r = r;
@@ -849,10 +889,12 @@ molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, in
     for (int i = 0; i < P; ++i) {
         const molora_proj_desc_t& d = projs[order[i]];
         UmmaProj& u = prm.p[i];
-        const CUtensorMapSwizzle wswz = d.rank == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
-                                        : d.rank == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
-        bool ok = make_tensor_map_bf16_2d(&u.tm_a, d.A, d.rank, (uint64_t)C * d.d_in, d.rank, d.rank, kChunkCols, wswz);
-        ok = ok && make_tensor_map_bf16_2d(&u.tm_b, d.B, d.d_out, (uint64_t)C * d.rank, d.d_out, kChunkCols, d.rank,
+        const int32_t rr = d.rank / parts;                    // the adapters' own rank (d.rank is the stacked rank of a set)
+        if (rr * parts != d.rank || (rr != 16 && rr != 32 && rr != 64)) return MOLORA_ERR_UNSUPPORTED;
+        const CUtensorMapSwizzle wswz = rr == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                        : rr == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+        bool ok = make_tensor_map_bf16_2d(&u.tm_a, d.A, rr, (uint64_t)n_adapters * d.d_in, rr, rr, kChunkCols, wswz);
+        ok = ok && make_tensor_map_bf16_2d(&u.tm_b, d.B, d.d_out, (uint64_t)n_adapters * rr, d.d_out, kChunkCols, rr,
                             CU_TENSOR_MAP_SWIZZLE_128B);
         if (!ok) return MOLORA_ERR_CUDA;
         u.x = static_cast<const __nv_bfloat16*>(d.x);

@@ -270,7 +270,10 @@ bool umma_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
 bool group_apply_umma_eligible(int64_t N, int32_t C);
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                   const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
-                                  cudaStream_t s, const int32_t* r = nullptr, int32_t* counts_out = nullptr);
+                                  cudaStream_t s, const int32_t* r = nullptr, int32_t* counts_out = nullptr,
+                                  int32_t parts = 1, int32_t cbase = 0);
+// (parts > 1: top-k routing in one pass -- C counts adapter SETS of `parts` adapters out of `cbase`, the projections carry
+// the stacked rank parts x r and row_scale = the weights [parts][N]; adapters' rank 16, 32 or 64)
 
 // mma.sync path for decode-sized calls (bf16, rank 16/32/64, d_in and d_out multiples of 32): a shrink launch and
 // an expand launch; takes the segments with fewer than max_rows rows.  The workspace holds the fp32 partial
