@@ -40,6 +40,7 @@ HEADLINE = "c4"
 SUB_CONFIGS = ("c2", "c3", "c5", "c5-iid")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
 # under profiles/ (file named per entry); None where no capture of that workload is committed
+GATHER_RW_GBS = 5277.0        # microbench/gather_rw.cu on this machine's B200: gathered 128-byte pieces, 2 reads : 1 write
 NCU_TRAFFIC = {
     "c2": (34.17e6, "profiles/apply_stream_c2_full.md"),
     "c3": (26.81e6, "profiles/apply_stream_c3_full.md"),
@@ -404,6 +405,13 @@ def measure(name, args, env, headline):
                      "algorithmic_bytes": step_bytes, "kernel_ms": apply_ms, "kernel_launches": kernel_launches,
                      "kernel_timing": kernel_timing, "algorithmic_tflops": step_flops / (apply_ms * 1e-3) / 1e12},
     })
+    if traffic and name in ("c4", "c5", "c5-iid") and not kw:
+        # the measured DRAM traffic of the launch against what a do-nothing kernel with the same access pattern (gathered
+        # 128-byte row pieces, 2 reads : 1 write) gets out of DRAM; context for `frac`, whose denominator is a sequential copy
+        rate = traffic[0] / (apply_ms * 1e-3) / 1e9
+        rec["roofline"]["traffic_rate_gbs"] = rate
+        rec["roofline"]["pattern_ceiling"] = {"gbs": GATHER_RW_GBS, "frac": rate / GATHER_RW_GBS,
+                                              "source": "profiles/gather_pattern_microbench.md"}
     if kpass is not None:
         rec["kpass_baseline"] = kpass
     rec["e2e"] = None
