@@ -182,7 +182,9 @@ __device__ __forceinline__ void sum_partials(uint32_t (&tv)[NWORDS], const float
     }
 }
 
-template <int R, bool WIDE>
+// PARTS: adapters per segment (1: top-1 routing; 2 or 4: adapter sets of top-k routing, see UmmaParams) -- a compile-time
+// constant so that the top-1 kernel is exactly the code it was before sets existed (a run-time `parts` cost it 13 %).
+template <int R, bool WIDE, int PARTS>
 __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __grid_constant__ UmmaParams prm)
 {
     using Cfg = UmmaCfg<R, WIDE>;
@@ -277,12 +279,13 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
         return;
     }
     // adapters of the segment's set (one adapter when parts == 1) and the rank of each
-    const int parts = prm.parts, rp = R / parts;
+    constexpr int parts = PARTS, rp = R / PARTS;
+    static_assert(rp >= 16 && rp * PARTS == R, "adapters of rank 16, 32 or 64");
     int adapter[kUmmaMaxParts];
     {
         int rest = seg;
         for (int j = parts - 1; j >= 0; --j) {
-            adapter[j] = parts == 1 ? seg : rest % prm.cbase;
+            adapter[j] = PARTS == 1 ? seg : rest % prm.cbase;
             rest /= prm.cbase;
         }
         for (int j = parts; j < kUmmaMaxParts; ++j) adapter[j] = 0;
@@ -355,7 +358,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 const uint32_t fb = bar(&ctrl->full[s]);
                 mbar_arrive_expect_tx(fb, (uint32_t)Cfg::kWBytes);
                 // one box per part: A chunks [64, r] side by side as tiles of their own, B chunks [r, 64] stacked by rows
-                for (int j = 0; j < parts; ++j) {
+#pragma unroll
+                for (int j = 0; j < PARTS; ++j) {
                     if (it < KX)
                         tma_load_2d(stage(s) + kTileBytes + (uint32_t)(j * kChunkCols * rp * 2), &pj.tm_a, 0,
                                     adapter[j] * pj.d_in + (kx0 + it) * kChunkCols, fb);
@@ -370,10 +374,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     } else if (warp == kMmaWarp) {
         // ============================================================ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc_shrink = idesc_bf16_f32(kTileM, rp, 0, 1);
+            constexpr uint32_t idesc_shrink = idesc_bf16_f32(kTileM, rp, 0, 1);
             // rows of an A chunk are r x 2 bytes: 128-, 64- or 32-byte swizzle
-            const uint32_t wlayout = swizzle_layout_type(rp == 64 ? Swizzle::B128 : rp == 32 ? Swizzle::B64 : Swizzle::B32);
-            const uint32_t wrow = (uint32_t)rp * 2u;
+            constexpr uint32_t wlayout = swizzle_layout_type(rp == 64 ? Swizzle::B128 : rp == 32 ? Swizzle::B64 : Swizzle::B32);
+            constexpr uint32_t wrow = (uint32_t)rp * 2u;
             constexpr uint32_t idesc_expand = idesc_bf16_f32(kTileM, kChunkCols, 0, 1);
             constexpr uint32_t kL128 = swizzle_layout_type(Swizzle::B128);
             for (int it = 0; it < KX; ++it) {
@@ -387,7 +391,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {   // four K = 16 steps per 64-column chunk
                         const uint64_t ad = smem_desc(a0 + j * 32, 16, 1024, kL128);
-                        for (int pt = 0; pt < parts; ++pt) {          // part pt -> columns [pt r, (pt + 1) r) of T
+#pragma unroll
+                        for (int pt = 0; pt < PARTS; ++pt) {          // part pt -> columns [pt r, (pt + 1) r) of T
                             const uint64_t bd = smem_desc(w0 + (uint32_t)pt * kChunkCols * wrow + j * (16 * wrow), 0, 8 * wrow, wlayout);
                             umma_bf16(tmem_T + (uint32_t)(pt * rp), ad, bd, idesc_shrink, it > 0 || j > 0);
                         }
@@ -463,7 +468,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
                 for (int c8 = 0; c8 < RH / 8; ++c8) {
                     float hi[8], lo[8];
                     const int tpart = (col0 + c8 * 8) / rp;       // (r is a multiple of 16: a block of 8 columns has one part)
-                    const float ts = tpart == 0 ? tscale[0] : tpart == 1 ? tscale[1] : tpart == 2 ? tscale[2] : tscale[3];
+                    const float ts = PARTS == 1 ? tscale[0] : tpart == 0 ? tscale[0] : tpart == 1 ? tscale[1] : tpart == 2 ? tscale[2] : tscale[3];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const float t = __uint_as_float(tv[c8 * 8 + e]) * ts;
@@ -683,7 +688,7 @@ struct UmmaPlan {
     int tile_rows;   // positions per tile
 };
 
-template <int R, bool WIDE>
+template <int R, bool WIDE, int PARTS = 1>
 static void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, int64_t tiles, int P, int split,
                                cudaStream_t s)
 {
@@ -699,7 +704,7 @@ static void fill_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* att
     cfg.numAttrs = 1;
 }
 
-template <int R, bool WIDE>
+template <int R, bool WIDE, int PARTS>
 static cudaError_t umma_launch_variant(UmmaParams prm, int64_t N, UmmaPlan plan, cudaStream_t s)
 {
     const int split = plan.split;
@@ -708,7 +713,7 @@ static cudaError_t umma_launch_variant(UmmaParams prm, int64_t N, UmmaPlan plan,
     static bool configured_dev[kMaxDevices] = {};
     bool& configured = configured_dev[device_slot()];
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(apply_umma_kernel<R, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(apply_umma_kernel<R, WIDE, PARTS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              Cfg::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
@@ -718,16 +723,30 @@ static cudaError_t umma_launch_variant(UmmaParams prm, int64_t N, UmmaPlan plan,
     cudaLaunchAttribute attr[1];
     fill_launch_config<R, WIDE>(cfg, attr, tiles, prm.P, split, s);
     note_launch();
-    return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R, WIDE>, prm);
+    return cudaLaunchKernelEx(&cfg, apply_umma_kernel<R, WIDE, PARTS>, prm);
+}
+
+// adapters per segment -> the instantiation (stacked rank R = parts x 16 | 32 | 64)
+template <int R, bool WIDE>
+static cudaError_t umma_launch_parts(const UmmaParams& prm, int64_t N, UmmaPlan plan, cudaStream_t s)
+{
+    if constexpr (R >= 32) {
+        if (prm.parts == 2) return umma_launch_variant<R, WIDE, 2>(prm, N, plan, s);
+    }
+    if constexpr (R == 64) {
+        if (prm.parts == 4) return umma_launch_variant<R, WIDE, 4>(prm, N, plan, s);
+    }
+    if (prm.parts != 1) return cudaErrorInvalidValue;
+    return umma_launch_variant<R, WIDE, 1>(prm, N, plan, s);
 }
 
 template <int R>
 static cudaError_t umma_launch(const UmmaParams& prm, int64_t N, UmmaPlan plan, cudaStream_t s)
 {
     if constexpr (R == 64) {
-        if (plan.split > UmmaCfg<64, false>::kMaxSplitR) return umma_launch_variant<64, true>(prm, N, plan, s);
+        if (plan.split > UmmaCfg<64, false>::kMaxSplitR) return umma_launch_parts<64, true>(prm, N, plan, s);
     }
-    return umma_launch_variant<R, false>(prm, N, plan, s);
+    return umma_launch_parts<R, false>(prm, N, plan, s);
 }
 
 // Clusters of `split` CTAs of this kernel that can be resident at once (cached per rank and split).
@@ -737,13 +756,13 @@ static int max_active_clusters_variant(int split)
     static int cache_dev[kMaxDevices][kMaxWideSplit + 1] = {};
     int (&cache)[kMaxWideSplit + 1] = cache_dev[device_slot()];
     if (cache[split] == 0) {
-        cudaFuncSetAttribute(apply_umma_kernel<R, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(apply_umma_kernel<R, WIDE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              UmmaCfg<R, WIDE>::kSmemBytes);
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute attr[1];
         fill_launch_config<R, WIDE>(cfg, attr, 148, 1, split, nullptr);
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, apply_umma_kernel<R, WIDE>, &cfg) != cudaSuccess || n <= 0) n = 148 / split;
+        if (cudaOccupancyMaxActiveClusters(&n, apply_umma_kernel<R, WIDE, 1>, &cfg) != cudaSuccess || n <= 0) n = 148 / split;
         cache[split] = n;
     }
     return cache[split];
