@@ -291,7 +291,7 @@ int32_t molora_group_apply_skips_group_launch(const molora_proj_desc_t *projs, i
  *   idx_out  device int32 [k, N] slot-major: idx_out[j*N + i] = the j-th choice of token i (j = 0: largest logit;
  *            equal logits: lowest index first);  w_out  device fp32 [k, N], softmax over the k kept logits
  * molora_apply_topk applies the k choices.  Where the streaming kernel can take the call (bf16, k in {2, 4}, rank x k in
- * {16, 32, 64}, C^k <= 256, below the tcgen05 crossover) or the tcgen05 kernel can (adapters of rank 16 or 32, rank x k in
+ * {16, 32, 64}, at most 256 adapter sets = binom(C + k - 1, k), below the tcgen05 crossover) or the tcgen05 kernel can (adapters of rank 16 or 32, rank x k in
  * {32, 64}, at most 64 adapter sets, widths multiples of 64) it does so in ONE pass over x and y: tokens are grouped by their
  * SET of kept adapters, a segment shrinks against the stacked A of its k adapters, the k slices of t are weighted per
  * token and one expand against the stacked B adds all k deltas before the single rounding.  Otherwise: k passes of

@@ -544,7 +544,7 @@ molora_status_t molora_topk_softmax(const float* logits, int64_t N, int32_t C, i
 
 namespace {
 struct TopkPlan {
-    size_t counts, offsets, perm, sets, wsorted, apply_ws, apply_ws_bytes, total;
+    size_t counts, offsets, perm, sets, wsorted, table, apply_ws, apply_ws_bytes, total;
 };
 constexpr int kTopkMaxParts = 4;
 TopkPlan plan_topk(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C)
@@ -564,6 +564,7 @@ TopkPlan plan_topk(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_
     pl.perm = off;     off = a256(off + sizeof(int32_t) * n1);
     pl.sets = off;     off = a256(off + sizeof(int32_t) * n1);
     pl.wsorted = off;  off = a256(off + sizeof(float) * n1 * kTopkMaxParts);
+    pl.table = off;    off = a256(off + kTopkSetTableBytes);         // adapter set -> its adapters
     pl.total = off;
     return pl;
 }
@@ -571,15 +572,14 @@ TopkPlan plan_topk(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_
 // Eq. 8 in ONE pass over x and y: tokens are grouped by their SET of kept adapters, a segment's shrink runs against the
 // stacked A of its k adapters (rank k x r), the k slices of t are weighted per token, and one expand against the stacked
 // B adds all k deltas before the single rounding.  Taken when every projection can run on the streaming kernel with the
-// stacked rank (bf16, r x k in {16, 32, 64}, k in {2, 4}, C^k <= 256 sets) and the call is not one the tcgen05 kernel
-// would take pass by pass.
+// stacked rank (bf16, r x k in {16, 32, 64}, k in {2, 4}, at most 256 adapter sets = multisets of k out of C adapters:
+// binom(C + k - 1, k)) and the call is not one the tcgen05 kernel would take pass by pass.
 // Returns 0: k passes; 1: one pass on the streaming kernel; 2: one pass on the tcgen05 kernel (adapters of rank >= 16, at
 // most 64 adapter sets, widths that are multiples of 64, and a call large enough for that kernel at the stacked rank).
 int topk_single_pass(const molora_proj_desc_t* projs, int32_t P, molora_dtype_t dt, int64_t N, int32_t C, int32_t k)
 {
     if (dt != MOLORA_BF16 || (k != 2 && k != 4) || N < 1) return 0;
-    int64_t sets = 1;
-    for (int j = 0; j < k; ++j) sets *= C;
+    const int64_t sets = topk_set_count(C, k);
     if (sets > MOLORA_MAX_ADAPTERS) return 0;
     double bytes = 0.0;
     bool umma_ok = sets <= kUmmaAllSegmentsMaxC && projs[0].rank >= 16;
@@ -625,27 +625,27 @@ molora_status_t molora_apply_topk(const molora_proj_desc_t* projs, int32_t P, mo
         cudaStream_t s = static_cast<cudaStream_t>(stream);
         int32_t* sets = reinterpret_cast<int32_t*>(base + pl.sets);
         float* wsorted = reinterpret_cast<float*>(base + pl.wsorted);
-        int32_t n_sets = 1;
-        for (int j = 0; j < k; ++j) n_sets *= C;
+        const int32_t n_sets = (int32_t)topk_set_count(C, k);
+        uint8_t* table = reinterpret_cast<uint8_t*>(base + pl.table);
         for (int i = 0; i < P; ++i) {
             pass[i] = projs[i];
             pass[i].rank = projs[i].rank * k;       // the stacked rank of a set
             pass[i].row_scale = wsorted;            // [k][N], in the order of the set's adapters
         }
-        molora_status_t st = launch_topk_sets(idx, w, N, C, k, sets, wsorted, s);
+        molora_status_t st = launch_topk_sets(idx, w, N, C, k, sets, wsorted, table, s);
         if (st != MOLORA_OK) return st;
         if (one_pass == 2) {                         // tcgen05 kernel: one MMA per part in the shrink, stacked B in the expand
             if (group_apply_umma_eligible(N, n_sets))
-                return launch_apply_umma(pass, P, N, n_sets, offsets, perm, dev_status, 1, s, sets, counts, k, C);
+                return launch_apply_umma(pass, P, N, n_sets, offsets, perm, dev_status, 1, s, sets, counts, k, C, table);
             st = molora_group(sets, N, n_sets, counts, offsets, perm, nullptr, 0, dev_status, stream);
             if (st != MOLORA_OK) return st;
-            return launch_apply_umma(pass, P, N, n_sets, offsets, perm, dev_status, 1, s, nullptr, nullptr, k, C);
+            return launch_apply_umma(pass, P, N, n_sets, offsets, perm, dev_status, 1, s, nullptr, nullptr, k, C, table);
         }
         if (group_apply_stream_eligible(N))         // the CTAs of the apply group the sets themselves
-            return launch_group_apply_stream_sets(sets, pass, P, N, C, k, counts, offsets, perm, dev_status, s);
+            return launch_group_apply_stream_sets(sets, pass, P, N, n_sets, k, table, counts, offsets, perm, dev_status, s);
         st = molora_group(sets, N, n_sets, counts, offsets, perm, nullptr, 0, dev_status, stream);
         if (st != MOLORA_OK) return st;
-        return launch_apply_stream_sets(pass, P, N, C, k, offsets, perm, dev_status, s);
+        return launch_apply_stream_sets(pass, P, N, n_sets, k, table, offsets, perm, dev_status, s);
     }
     for (int32_t j = 0; j < k; ++j) {               // one (group, apply) pass per kept adapter slot
         for (int i = 0; i < P; ++i) {

@@ -55,10 +55,11 @@ struct StreamParams {
     const int32_t* perm;
     uint32_t* dev_status;
     int32_t N, P, C, max_rows;                // segments with at least max_rows rows belong to the tcgen05 kernel
-    // Top-k routing in one pass (Eq. 8): a segment is a SET of `parts` adapters (its index spells them in base `cbase`,
-    // most significant first), the launch's rank R is parts x the adapters' rank, A_c and B_c are gathered from the
+    // Top-k routing in one pass (Eq. 8): a segment is a SET of `parts` adapters (set_table[4 * segment + j] names them, in
+    // ascending order), the launch's rank R is parts x the adapters' rank, A_c and B_c are gathered from the
     // parts' adapters, and row_scale holds the routing weights [parts][N].  parts == 1: plain top-1 routing.
     int32_t parts, cbase;
+    const uint8_t* set_table;
     // grouping variant only: the routing decisions and where counts / offsets / perm are written (as by molora_group)
     const int32_t* r;
     int32_t* counts_out;
@@ -66,11 +67,10 @@ struct StreamParams {
     int32_t* perm_out;
 };
 // adapter of part j of segment `seg`
-__device__ __forceinline__ int fs_part_adapter(const StreamParams& prm, int seg, int j)
+// (set_tab: the kernel's shared-memory copy of prm.set_table)
+__device__ __forceinline__ int fs_part_adapter(const StreamParams& prm, const uint8_t* set_tab, int seg, int j)
 {
-    int div = 1;
-    for (int k = prm.parts - 1; k > j; --k) div *= prm.cbase;
-    return (seg / div) % prm.cbase;
+    return prm.parts == 1 ? seg : (int)set_tab[seg * 4 + j];
 }
 // (projection, slice of d_out) pairs of the projections of the launch's rank; projection p owns [start[p], start[p + 1]).
 struct FsUnits {
@@ -177,6 +177,7 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
     __shared__ uint32_t st_bytes[kFsCopyWarps][NS];      // bytes per row to store (0: a shrink job, nothing to store)
     __shared__ int st_rows[kFsCopyWarps][NS];
     __shared__ int abort_s;
+    __shared__ __align__(16) uint8_t set_tab_s[MOLORA_MAX_ADAPTERS * 4];   // adapter sets of top-k routing: set -> adapters
     extern __shared__ __align__(128) unsigned char dsm[];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -188,6 +189,9 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
         abort_s = 0;
         fence_mbar_init();
     }
+    if (prm.parts > 1)                         // (visible after the block-wide barriers of the prologue below)
+        for (int i = tid; i < prm.C; i += kFsThreads)
+            reinterpret_cast<uint32_t*>(set_tab_s)[i] = __ldg(reinterpret_cast<const uint32_t*>(prm.set_table) + i);
     if constexpr (GROUP) {
         // the grouping itself, on this CTA, while the ring is idle (its memory is the scratch)
         group_in_cta<kFsThreads, kFsPermCache>(prm.r, prm.N, prm.C, offs_s, tstart_s, perm_s, dsm, true, prm.counts_out,
@@ -240,11 +244,11 @@ __global__ void __launch_bounds__(kFsThreads, 1) apply_stream_kernel(const __gri
             const int parts = prm.parts, pr = R / parts;            // adapters per segment, rank of each
             // my weight source: lane RPW + j loads part j's rows of A; the lanes after RPW load one row of B each
             const int apart = min(max(lane - RPW, 0), parts - 1);
-            const char* Ac = static_cast<const char*>(pd.A) + (int64_t)fs_part_adapter(prm, it.seg, apart) * pd.d_in * pr * 2;
+            const char* Ac = static_cast<const char*>(pd.A) + (int64_t)fs_part_adapter(prm, set_tab_s, it.seg, apart) * pd.d_in * pr * 2;
             const int brow = cw * (R / kFsCopyWarps) + max(lane - RPW, 0);          // my row of the stacked B (lanes RPW ..)
             const int bpart = min(brow / pr, parts - 1);
             const char* Bc = static_cast<const char*>(pd.B) +
-                             (((int64_t)fs_part_adapter(prm, it.seg, bpart) * pr + (brow - bpart * pr)) * pd.d_out + it.col0) * 2;
+                             (((int64_t)fs_part_adapter(prm, set_tab_s, it.seg, bpart) * pr + (brow - bpart * pr)) * pd.d_out + it.col0) * 2;
             const int myrows = max(0, min(RPW, it.rows - cw * RPW));
             for (int j = 0; j < it.nks + it.ne; ++j, ++g) {
                 const uint32_t s = g % NS;
@@ -607,13 +611,15 @@ molora_status_t launch_apply_stream(const molora_proj_desc_t* projs, int32_t P, 
     prm.counts_out = prm.offsets_out = prm.perm_out = nullptr;
     prm.parts = 1;
     prm.cbase = C;
+    prm.set_table = nullptr;
     return stream_enqueue(projs, P, N, C, prm, false, s);
 }
 
 // Top-k routing in one pass: `projs` carry the STACKED rank (parts x the adapters' rank) and row_scale = weights
 // [parts][N]; offsets / perm group the tokens by adapter set, C_sets = cbase^parts segments.
-molora_status_t launch_apply_stream_sets(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t cbase, int32_t parts,
-                                         const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, cudaStream_t s)
+molora_status_t launch_apply_stream_sets(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t n_sets, int32_t parts,
+                                         const uint8_t* set_table, const int32_t* offsets, const int32_t* perm,
+                                         uint32_t* dev_status, cudaStream_t s)
 {
     if (N == 0 || P == 0) return MOLORA_OK;
     StreamParams prm;
@@ -624,17 +630,16 @@ molora_status_t launch_apply_stream_sets(const molora_proj_desc_t* projs, int32_
     prm.r = nullptr;
     prm.counts_out = prm.offsets_out = prm.perm_out = nullptr;
     prm.parts = parts;
-    prm.cbase = cbase;
-    int32_t sets = 1;
-    for (int j = 0; j < parts; ++j) sets *= cbase;
-    return stream_enqueue(projs, P, N, sets, prm, false, s);
+    prm.cbase = 0;
+    prm.set_table = set_table;
+    return stream_enqueue(projs, P, N, n_sets, prm, false, s);
 }
 
 // ... and started from the set indices (at most 4096 tokens): grouping by set and apply in one launch.  (Forming the sets
 // inside this kernel as well was measured and lost: every CTA repeats the sort, 23.2 against 21.5 us at 4096 tokens.)
 molora_status_t launch_group_apply_stream_sets(const int32_t* sets, const molora_proj_desc_t* projs, int32_t P, int64_t N,
-                                               int32_t cbase, int32_t parts, int32_t* counts, int32_t* offsets, int32_t* perm,
-                                               uint32_t* dev_status, cudaStream_t s)
+                                               int32_t n_sets, int32_t parts, const uint8_t* set_table, int32_t* counts,
+                                               int32_t* offsets, int32_t* perm, uint32_t* dev_status, cudaStream_t s)
 {
     if (N == 0 || P == 0) return MOLORA_OK;
     StreamParams prm;
@@ -647,9 +652,8 @@ molora_status_t launch_group_apply_stream_sets(const int32_t* sets, const molora
     prm.offsets_out = offsets;
     prm.perm_out = perm;
     prm.parts = parts;
-    prm.cbase = cbase;
-    int32_t n_sets = 1;
-    for (int j = 0; j < parts; ++j) n_sets *= cbase;
+    prm.cbase = 0;
+    prm.set_table = set_table;
     return stream_enqueue(projs, P, N, n_sets, prm, true, s);
 }
 
@@ -670,6 +674,7 @@ molora_status_t launch_group_apply_stream(const int32_t* r, const molora_proj_de
     prm.perm_out = perm;
     prm.parts = 1;
     prm.cbase = C;
+    prm.set_table = nullptr;
     return stream_enqueue(projs, P, N, C, prm, true, s);
 }
 

@@ -91,12 +91,13 @@ struct UmmaParams {
     int32_t* counts_out;
     int32_t* offsets_out;
     int32_t* perm_out;
-    // Top-k routing in one pass (Eq. 8): a segment is a SET of `parts` adapters (its index spells them in base `cbase`, most
-    // significant first) and the launch's rank R is parts x the adapters' rank r.  The shrink runs one MMA per part into
+    // Top-k routing in one pass (Eq. 8): a segment is a SET of `parts` adapters (named by set_table, `cbase` adapters
+    // in all) and the launch's rank R is parts x the adapters' rank r.  The shrink runs one MMA per part into
     // its own r columns of T (the part's A chunk is its own shared-memory tile), every part of a row of T is scaled by the
     // token's weight for that part (row_scale[part * N + token]), and the expand contracts all R columns against the
     // parts' B chunks stacked by rows -- one read of x and y, one rounding.  parts == 1: plain top-1 routing.
     int32_t parts, cbase;
+    const uint8_t* set_table;         // parts > 1: set_table[4 * segment + j] = the j-th adapter of the set
 };
 constexpr int kUmmaGroupMaxN = 4096;
 constexpr int kUmmaMaxParts = 4;
@@ -282,14 +283,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) apply_umma_kernel(const __gri
     constexpr int parts = PARTS, rp = R / PARTS;
     static_assert(rp >= 16 && rp * PARTS == R, "adapters of rank 16, 32 or 64");
     int adapter[kUmmaMaxParts];
-    {
-        int rest = seg;
-        for (int j = parts - 1; j >= 0; --j) {
-            adapter[j] = PARTS == 1 ? seg : rest % prm.cbase;
-            rest /= prm.cbase;
-        }
-        for (int j = parts; j < kUmmaMaxParts; ++j) adapter[j] = 0;
-    }
+#pragma unroll
+    for (int j = 0; j < kUmmaMaxParts; ++j)
+        adapter[j] = PARTS == 1 ? seg : (j < PARTS ? (int)__ldg(prm.set_table + seg * 4 + j) : 0);
     const int KXall = pj.d_in / kChunkCols, NYall = pj.d_out / kChunkCols;
     const int kx0 = (int)(crank * KXall / S), KX = (int)((crank + 1) * KXall / S) - kx0;   // my slice of d_in
     const int ny0 = (int)(crank * NYall / S), NY = (int)((crank + 1) * NYall / S) - ny0;   // my slice of d_out
@@ -853,13 +849,16 @@ bool group_apply_umma_eligible(int64_t N, int32_t C) { return N >= 1 && N <= kUm
 
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                   const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
-                                  cudaStream_t s, const int32_t* r, int32_t* counts_out, int32_t parts, int32_t cbase)
+                                  cudaStream_t s, const int32_t* r, int32_t* counts_out, int32_t parts, int32_t cbase,
+                                  const uint8_t* set_table)
 {
     if (N == 0 || P == 0) return MOLORA_OK;
     if (parts < 1 || parts > kUmmaMaxParts) return MOLORA_ERR_INVALID_ARG;
     UmmaParams prm;
     prm.parts = parts;
     prm.cbase = parts > 1 ? cbase : C;
+    prm.set_table = set_table;
+    if (parts > 1 && set_table == nullptr) return MOLORA_ERR_INVALID_ARG;
     const int32_t n_adapters = parts > 1 ? cbase : C;          // C counts adapter SETS when parts > 1
     // r given: the kernel groups on chip and writes counts / offsets / perm (the pointers are then outputs); one launch
     // only, so every projection must have the same rank

@@ -254,8 +254,24 @@ molora_status_t launch_route_mlp(const void* x, molora_dtype_t xdt, int64_t N, i
 molora_status_t launch_topk_softmax(const float* logits, int64_t N, int32_t C, int32_t k, int32_t* idx_out, float* w_out,
                                     cudaStream_t s);
 // Adapter sets of top-k routing (sorted adapters of a token spelled in base C) and the weights in the same order.
+// Adapter sets of top-k routing are numbered densely: the k adapters of a token, sorted (repeats allowed), are the
+// topk_set_count(C, k) = binom(C + k - 1, k) multisets in colexicographic order, rank = sum_j binom(a_j + j, j + 1).
+__host__ __device__ inline int64_t binom_small(int64_t n64, int r)         // r <= 4, n < 1000: closed forms in 32 bits
+{
+    const int n = (int)n64;
+    if (n < r) return 0;
+    switch (r) {
+        case 0: return 1;
+        case 1: return n;
+        case 2: return n * (n - 1) / 2;
+        case 3: return n * (n - 1) / 2 * (n - 2) / 3;
+        default: return n * (n - 1) / 2 * (n - 2) / 3 * (n - 3) / 4;
+    }
+}
+__host__ __device__ inline int64_t topk_set_count(int C, int k) { return binom_small((int64_t)C + k - 1, k); }
+constexpr int kTopkSetTableBytes = MOLORA_MAX_ADAPTERS * 4;               // set -> its (up to four) adapters, one byte each
 molora_status_t launch_topk_sets(const int32_t* idx, const float* w, int64_t N, int32_t C, int32_t k, int32_t* set_out,
-                                 float* w_out, cudaStream_t s);
+                                 float* w_out, uint8_t* table_out, cudaStream_t s);
 size_t group_workspace_bytes(int64_t N, int32_t C);
 molora_status_t launch_group(const int32_t* r, int64_t N, int32_t C, int32_t* counts, int32_t* offsets, int32_t* perm,
                              void* ws, size_t ws_bytes, uint32_t* dev_status, cudaStream_t s);
@@ -271,9 +287,10 @@ bool group_apply_umma_eligible(int64_t N, int32_t C);
 molora_status_t launch_apply_umma(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                   const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, int32_t min_rows,
                                   cudaStream_t s, const int32_t* r = nullptr, int32_t* counts_out = nullptr,
-                                  int32_t parts = 1, int32_t cbase = 0);
-// (parts > 1: top-k routing in one pass -- C counts adapter SETS of `parts` adapters out of `cbase`, the projections carry
-// the stacked rank parts x r and row_scale = the weights [parts][N]; adapters' rank 16, 32 or 64)
+                                  int32_t parts = 1, int32_t n_adapters = 0, const uint8_t* set_table = nullptr);
+// (parts > 1: top-k routing in one pass -- C counts adapter SETS of `parts` adapters out of `n_adapters`, set_table[4 * set +
+// j] names them, the projections carry the stacked rank parts x r and row_scale = the weights [parts][N]; adapters' rank
+// 16, 32 or 64)
 
 // mma.sync path for decode-sized calls (bf16, rank 16/32/64, d_in and d_out multiples of 32): a shrink launch and
 // an expand launch; takes the segments with fewer than max_rows rows.  The workspace holds the fp32 partial
@@ -283,14 +300,15 @@ bool decode_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
 molora_status_t launch_apply_stream(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t C,
                                     const int32_t* offsets, const int32_t* perm, int32_t max_rows, uint32_t* dev_status,
                                     cudaStream_t s);
-// The same kernel for top-k routing in one pass: segments are adapter sets (cbase^parts of them), the projections carry
-// the stacked rank parts x r and row_scale = weights [parts][N].
+// The same kernel for top-k routing in one pass: segments are adapter sets (n_sets of them, set_table[4 * set + j] = the
+// j-th adapter of the set), the projections carry the stacked rank parts x r and row_scale = weights [parts][N].
 bool stream_eligible(const molora_proj_desc_t& p, molora_dtype_t dt);
-molora_status_t launch_apply_stream_sets(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t cbase, int32_t parts,
-                                         const int32_t* offsets, const int32_t* perm, uint32_t* dev_status, cudaStream_t s);
+molora_status_t launch_apply_stream_sets(const molora_proj_desc_t* projs, int32_t P, int64_t N, int32_t n_sets, int32_t parts,
+                                         const uint8_t* set_table, const int32_t* offsets, const int32_t* perm,
+                                         uint32_t* dev_status, cudaStream_t s);
 molora_status_t launch_group_apply_stream_sets(const int32_t* sets, const molora_proj_desc_t* projs, int32_t P, int64_t N,
-                                               int32_t cbase, int32_t parts, int32_t* counts, int32_t* offsets, int32_t* perm,
-                                               uint32_t* dev_status, cudaStream_t s);
+                                               int32_t n_sets, int32_t parts, const uint8_t* set_table, int32_t* counts,
+                                               int32_t* offsets, int32_t* perm, uint32_t* dev_status, cudaStream_t s);
 // The same kernel started from the routing decisions r: grouping (counts, offsets, perm as molora_group writes them)
 // and apply in one launch; all projections of one rank, at most 4096 tokens.
 bool group_apply_stream_eligible(int64_t N);

@@ -527,13 +527,29 @@ molora_status_t launch_topk_softmax(const float* logits, int64_t N, int32_t C, i
                                  (int)C, (int)k, idx_out, w_out));
 }
 
-// Top-k routing in one pass: the k adapters of a token, sorted by index, name a SET; its index spells them in base C
-// (most significant first), and the weights are stored in the same order.  Tokens with an adapter outside [0, C) are
-// left unrouted.  k <= 4.
+// Top-k routing in one pass: the k adapters of a token, sorted by index, name a SET (a multiset: a caller may repeat an
+// adapter); sets are numbered densely, rank = sum_j binom(a_j + j, j + 1) over the sorted adapters, and the weights are
+// stored in the same order.  Tokens with an adapter outside [0, C) are left unrouted.  k <= 4.  The first block also
+// writes the table set -> adapters (4 bytes per set) that the apply kernels read.
 __global__ void __launch_bounds__(256) topk_sets_kernel(const int32_t* __restrict__ idx, const float* __restrict__ w, int64_t N,
-                                                        int C, int k, int32_t* __restrict__ set_out, float* __restrict__ w_out)
+                                                        int C, int k, int32_t* __restrict__ set_out, float* __restrict__ w_out,
+                                                        uint8_t* __restrict__ table_out)
 {
     ptx::grid_dependency_sync();
+    if (blockIdx.x == 0) {
+        const int n_sets = (int)topk_set_count(C, k);
+        for (int t = threadIdx.x; t < n_sets; t += blockDim.x) {
+            int rest = t;
+            uint8_t a[4] = {0, 0, 0, 0};
+            for (int j = k - 1; j >= 0; --j) {                      // largest b with binom(b, j + 1) <= rest; a_j = b - j
+                int b = j;
+                while (binom_small(b + 1, j + 1) <= rest) ++b;
+                rest -= (int)binom_small(b, j + 1);
+                a[j] = (uint8_t)(b - j);
+            }
+            for (int j = 0; j < 4; ++j) table_out[t * 4 + j] = a[j];
+        }
+    }
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N) return;
     int a[4];
@@ -557,18 +573,18 @@ __global__ void __launch_bounds__(256) topk_sets_kernel(const int32_t* __restric
 #pragma unroll
     for (int j = 0; j < 4; ++j)
         if (j < k) {
-            set = set * C + a[j];
+            if (ok) set += (int)binom_small(a[j] + j, j + 1);
             w_out[(int64_t)j * N + i] = f[j];
         }
     set_out[i] = ok ? set : -1;
 }
 
 molora_status_t launch_topk_sets(const int32_t* idx, const float* w, int64_t N, int32_t C, int32_t k, int32_t* set_out,
-                                 float* w_out, cudaStream_t s)
+                                 float* w_out, uint8_t* table_out, cudaStream_t s)
 {
     if (N == 0) return MOLORA_OK;
     return cuda_ok(launch_kernel(topk_sets_kernel, dim3((unsigned)ceil_div64(N, 256)), dim3(256), 0, s, 1, false, idx, w, N, (int)C,
-                                 (int)k, set_out, w_out));
+                                 (int)k, set_out, w_out, table_out));
 }
 
 size_t route_gate_workspace_bytes(molora_dtype_t xdt, int32_t d, int32_t C)

@@ -652,17 +652,21 @@ def test_route_mlp_feeds_group_and_apply():
                                                         (4096, 4, 2, 2048, 2048, 16, "default"),   # ... at the prefill shape
                                                         (700, 4, 4, 256, 320, 16, "default"),      # ... k = 4: stacked rank 64
                                                         (500, 8, 2, 512, 256, 32, "default"),      # ... rank 32, 64 sets
-                                                        (900, 16, 2, 256, 256, 16, "default"),     # ... 256 sets
+                                                        (900, 16, 2, 256, 256, 16, "default"),     # ... 136 sets
+                                                        (800, 22, 2, 256, 256, 16, "default"),     # ... 253 sets
+                                                        (800, 23, 2, 256, 256, 16, "default"),     # 276 sets: k passes
                                                         (6000, 5, 2, 192, 224, 16, "stream"),      # ... perm read from global memory
                                                         (300, 4, 2, 256, 192, 16, "jobs"),         # k passes from here on
                                                         (300, 4, 2, 256, 192, 16, "twophase"),
                                                         (3300, 4, 2, 512, 256, 16, "tcgen05"),     # one pass on the tcgen05 kernel
                                                         (5000, 4, 2, 2048, 1024, 32, "tcgen05-all"),  # ... stacked rank 64, grouping launch
-                                                        (2000, 4, 4, 1024, 512, 16, "tcgen05-all"),   # k = 4: 256 sets, k passes
+                                                        (2000, 4, 4, 1024, 512, 16, "tcgen05-all"),   # ... k = 4: 35 sets, too few tokens per set: k passes
+                                                        (9000, 4, 4, 1024, 256, 16, "tcgen05-all"),   # ... k = 4 in one pass (stacked rank 64)
                                                         (2000, 3, 2, 1024, 512, 16, "tcgen05-all"),   # ... 9 sets, grouping inside
                                                         (1500, 4, 2, 512, 320, 16, "tcgen05-s3"),     # ... tiles split over 3 CTAs
                                                         (1200, 3, 2, 2048, 256, 32, "tcgen05-s5"),    # ... over 5 CTAs (rank-64 exchange)
-                                                        (900, 9, 2, 512, 256, 16, "tcgen05-all"),     # 81 sets: k passes
+                                                        (900, 9, 2, 512, 256, 16, "tcgen05-all"),     # 45 sets, too few tokens per set: k passes
+                                                        (700, 12, 2, 512, 256, 16, "tcgen05-all"),    # 78 sets: k passes
                                                         (200, 6, 3, 128, 96, 8, "default"),      # CUDA-core kernel (rank 8)
                                                         (500, 5, 1, 64, 64, 32, "default")])     # k = 1: weight exactly 1
 def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode):
@@ -693,9 +697,11 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode):
     got = to_f64(y)
     err = np.abs(got - ref)
     bound = 1e-3 + 2e-2 * np.abs(ref)
-    one_pass = mode in ("stream", "default") and k in (2, 4) and rank * k in (16, 32, 64) and C ** k <= 256
+    import math
+    n_sets = math.comb(C + k - 1, k)                          # adapter sets are multisets of k out of C adapters
+    one_pass = mode in ("stream", "default") and k in (2, 4) and rank * k in (16, 32, 64) and n_sets <= 256
     if mode.startswith("tcgen05"):
-        one_pass = (k in (2, 4) and rank >= 16 and rank * k in (32, 64) and (C ** k <= 16 or (C ** k <= 64 and N >= 256 * C ** k))
+        one_pass = (k in (2, 4) and rank >= 16 and rank * k in (32, 64) and (n_sets <= 16 or (n_sets <= 64 and N >= 256 * n_sets))
                     and d_in % 64 == 0 and d_out % 64 == 0)
     if not one_pass:
         # k passes round y to bf16 after every pass: besides the usual bound, half a bf16 ulp (2^-9 relative) of each
@@ -704,6 +710,24 @@ def test_topk_weighted_routing_end_to_end(N, C, k, d_in, d_out, rank, mode):
         for j in range(1, k):
             bound = bound + 2.0 ** -9 * np.abs(oracle.apply_topk(x_np, p.y, p.A, p.B, idx_ref[:j], w_ref[:j]))
     assert np.all(err[keep] <= bound[keep]), f"top-{k} weighted apply: worst ratio {(err / bound)[keep].max():.3f}"
+
+
+def test_topk_apply_accepts_repeated_adapters():
+    # the kept adapters of a token need not be distinct for the apply (a caller's own routing may repeat one): adapter
+    # sets are multisets
+    N, C, k, d_in, d_out, rank = 600, 4, 2, 256, 320, 16
+    rng = np.random.default_rng(99)
+    w_ = W.random_problem(990, N, C, d_in, d_out, rank, "bf16")
+    p = w_.projections[0]
+    idx = rng.integers(0, C, size=(k, N)).astype(np.int32)
+    idx[1, ::3] = idx[0, ::3]                                 # every third token names one adapter twice
+    wt = rng.random((k, N)).astype(np.float32)
+    wt /= wt.sum(axis=0, keepdims=True)
+    y = dev_tensor(p.y, "bf16")
+    M.molora_apply_topk([M.ProjDesc(dev_tensor(w_.inputs["x"], "bf16"), y, dev_tensor(p.A, "bf16"), dev_tensor(p.B, "bf16"), 1.0)],
+                        dev_tensor(idx, "i"), dev_tensor(wt, "f32"), C)
+    ref = oracle.apply_topk(w_.inputs["x"], p.y, p.A, p.B, idx, wt)
+    assert_close(to_f64(y), ref, what="top-2 with repeated adapters")
 
 
 @pytest.mark.parametrize("mode", ["tcgen05-s2", "tcgen05-s3", "tcgen05-s4", "tcgen05-s5", "tcgen05-s6r64", "tcgen05-s7r96", "tcgen05-s8"])
