@@ -386,6 +386,11 @@ def measure(name, args, env, headline):
         if name.startswith(("c5", "t6-")) and not args.profile and args.launch == "graph":
             kpass = run_kpass(args, env, w, sets, shared, stream, capture_pass, apply_ms, K, n_var)
         torch.cuda.synchronize()
+        # every kernel of the timed region ORs what it detects into one status word: a bounded wait that gave up (or a
+        # routing value out of range) would make the timing meaningless
+        dev_status = int(shared["status"].item())
+        if dev_status != 0:
+            raise RuntimeError(f"device status word after the timed region: {dev_status:#x}")
 
     peaks = measured_peaks()
     achieved = step_bytes / (apply_ms * 1e-3) / 1e9
